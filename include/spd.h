@@ -1,0 +1,146 @@
+/*
+ * spd.h - C ABI of the B200 (sm_100a) Sync-Point Drop block library.
+ *
+ * The library runs the forward pass of a stack of tensor-parallel (TP) LLaMA-style
+ * decoder blocks whose T devices ("shards") are emulated on ONE GPU.  Each block is
+ * either a fully synchronous TP block (Sec. 3, Fig. 1(a)) or an SPD block (Sec. 4.1.1,
+ * Fig. 1(b), Fig. 3(a)), chosen per block by a mask - the block list that Algorithm 1
+ * produces.  Both kinds use the same parameters (Sec. 4.2.3).
+ *
+ * Conventions common to every call
+ *   - All tensor pointers are DEVICE pointers unless marked "host".  Nothing passed in is
+ *     ever freed or retained beyond what is stated; the library allocates no device memory.
+ *   - dtype 0: float32 storage and arithmetic.  dtype 1: bfloat16 storage (weights,
+ *     activations in/out, KV pages), float32 accumulation, float32 residual stream.
+ *   - Linear weights use the torch.nn.Linear layout [out_features, in_features], row-major,
+ *     contiguous.  Shard i of a column-split matrix (wq, wk, wv, w_gate, w_up) is its rows
+ *     [i*n/T, (i+1)*n/T); shard i of a row-split matrix (wo, w_down) is its columns
+ *     [i*k/T, (i+1)*k/T) (Sec. 4.1.2).  Head grouping (Sec. 4.2.4) is a permutation the
+ *     caller applies to the weights beforehand.
+ *   - KV pages of one layer: [n_pages, n_kv_heads, kv_block_size, head_dim] in the storage
+ *     dtype, separately for K and V.  block_table[b, j] (int32) is the page holding tokens
+ *     [j*kv_block_size, (j+1)*kv_block_size) of sequence b.
+ *   - Every call returns SPD_OK (0) or a negative SPD_E* code and never throws, aborts or
+ *     traps.  Work is enqueued on `stream` (a cudaStream_t passed as void*) and is
+ *     asynchronous; a CUDA error of an earlier launch may be reported by a later call.
+ */
+#ifndef SPD_H
+#define SPD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPD_OK 0
+#define SPD_EINVAL (-1)     /* bad dimension, divisibility (nq % T, nkv % T, ffn % T), batch > max ... */
+#define SPD_ENULL (-2)      /* a required pointer is null                                            */
+#define SPD_EWORKSPACE (-3) /* workspace too small or misaligned (256 bytes)                          */
+#define SPD_ECAPACITY (-4)  /* sequence would outgrow max_seq_len or the block table                  */
+#define SPD_ECUDA (-5)      /* a CUDA call failed; see spd_last_cuda_error()                          */
+#define SPD_EDEVICE (-6)    /* a kernel recorded a bounds / bounded-wait failure in its error flag   */
+
+typedef struct spd_ctx spd_ctx; /* opaque; owned by the library, freed by spd_destroy */
+
+typedef struct {
+    int32_t n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn;
+    int32_t T;            /* emulated tensor-parallel devices                                   */
+    int32_t dtype;        /* 0 = float32, 1 = bfloat16                                          */
+    float rms_eps;
+    float rope_base;      /* <= 0 disables the rotary embedding                                 */
+    int32_t kv_block_size;      /* tokens per KV page (16)                                      */
+    int32_t max_batch;          /* largest B of spd_decode_step / spd_prefill                   */
+    int32_t max_seq_len;        /* largest context (cached + new tokens) of one sequence        */
+    int32_t max_prefill_tokens; /* tokens processed per internal prefill chunk (bounds workspace)*/
+} spd_dims;
+
+typedef struct {
+    const void *attn_norm; /* [hidden]                      RMSNorm gain before attention        */
+    const void *wq;        /* [n_q_heads*head_dim, hidden]                                       */
+    const void *wk;        /* [n_kv_heads*head_dim, hidden]                                      */
+    const void *wv;        /* [n_kv_heads*head_dim, hidden]                                      */
+    const void *wo;        /* [hidden, n_q_heads*head_dim]                                       */
+    const void *mlp_norm;  /* [hidden]                      RMSNorm gain before the MLP          */
+    const void *w_gate;    /* [ffn, hidden]                                                      */
+    const void *w_up;      /* [ffn, hidden]                                                      */
+    const void *w_down;    /* [hidden, ffn]                                                      */
+    void *k_pages;         /* [n_pages, n_kv_heads, kv_block_size, head_dim]  written by the lib */
+    void *v_pages;         /* same shape                                                         */
+} spd_layer;               /* device pointers, BORROWED: the caller keeps the tensors alive      */
+
+/* Bytes of device workspace spd_create needs for these dims and mask (host call, no GPU
+ * work).  sync_mask: host array [n_layers], 1 = synchronous TP block, 0 = SPD block.
+ * Errors: SPD_ENULL, SPD_EINVAL. */
+int spd_workspace_bytes(const spd_dims *dims, const uint8_t *sync_mask, size_t *out_bytes);
+
+/* Build a context for a stack of blocks: Algorithm 1's block list, entry l being a TP block
+ * when sync_mask[l] != 0 and an SPD block otherwise (Sec. 4.2; the block designs are those
+ * of Sec. 3 and Sec. 4.1.1).
+ *   layers    : host array [n_layers] of device pointers (copied; the tensors are borrowed)
+ *   n_pages   : pages in every k_pages / v_pages tensor (block-table entries are checked
+ *               against it on the device)
+ *   workspace : device memory, 256-byte aligned, >= spd_workspace_bytes(); borrowed until
+ *               spd_destroy; must not be shared by contexts running concurrently
+ * Requires a CUDA device of compute capability 10.x as the current device.
+ * Errors: SPD_ENULL, SPD_EINVAL, SPD_EWORKSPACE, SPD_ECUDA. */
+int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *layers,
+               int32_t n_pages, void *workspace, size_t workspace_bytes, spd_ctx **out);
+
+/* Prefill: run B prompts of S tokens each through the stack, writing their K/V into the
+ * pages named by block_table (positions 0..S-1) and the last block's output to `out`.
+ *   x, out      : [B, S, hidden] storage dtype; must not alias
+ *   block_table : [B, max_pages] int32, max_pages*kv_block_size >= S
+ * Attention is causal within each prompt (Sec. 3: each shard attends over its own heads).
+ * Errors: SPD_ENULL, SPD_EINVAL (B > max_batch), SPD_ECAPACITY, SPD_ECUDA. */
+int spd_prefill(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int32_t *block_table,
+                int32_t max_pages, void *out, void *stream);
+
+/* One decode step: one new token per sequence.  Appends the token's K/V at position
+ * seq_lens[b] and attends over seq_lens[b] + 1 tokens; the caller advances seq_lens.
+ *   x, out       : [B, hidden] storage dtype; must not alias
+ *   seq_lens     : [B] int32 device, tokens already cached per sequence
+ *   max_context  : host-side upper bound of seq_lens[b] + 1 over the batch (sizes the
+ *                  split of the KV range over thread blocks; <= max_seq_len)
+ * A sequence whose seq_lens[b] + 1 exceeds max_context or its block-table row is skipped and
+ * the device error flag is set (see spd_device_error).
+ * Errors: SPD_ENULL, SPD_EINVAL, SPD_ECAPACITY, SPD_ECUDA. */
+int spd_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_lens,
+                    const int32_t *block_table, int32_t max_pages, int32_t max_context,
+                    void *out, void *stream);
+
+/* Number of shard sums ("sync-points", Sec. 3) one forward pass of this stack executes:
+ * 2 per TP block, 1 per SPD block. */
+int spd_sync_points(const spd_ctx *ctx);
+
+/* Number of kernels one spd_decode_step / one spd_prefill chunk launches (bookkeeping). */
+int spd_launches_per_decode_step(const spd_ctx *ctx);
+
+/* Read and clear the device error flag (synchronises `stream`).  0 = clean; otherwise a bit
+ * set: 1 block-table entry out of range, 2 position beyond capacity, 4 bounded wait gave up.
+ * Kernels that meet such a condition skip the access, set the flag and return normally. */
+int spd_device_error(spd_ctx *ctx, void *stream, int32_t *out_flag);
+
+/* Per-kernel-kind timing for benchmarks.  Between spd_profile_begin and spd_profile_end every
+ * kernel launch of spd_prefill / spd_decode_step is bracketed by CUDA events on the call's
+ * stream (the launches are not fused or reordered, only time-stamped).  spd_profile_end
+ * synchronises `stream` and fills ms_by_kind / launches_by_kind (host arrays of
+ * spd_profile_kinds() entries; a "launch" here is one bracketed call site, which for decode
+ * attention covers its split and merge kernels).  Not to be used under stream capture. */
+int spd_profile_begin(spd_ctx *ctx);
+int spd_profile_end(spd_ctx *ctx, void *stream, float *ms_by_kind, int32_t *launches_by_kind);
+int spd_profile_kinds(void);
+const char *spd_profile_kind_name(int kind);
+
+/* Free the context (host state, descriptors, graphs).  Never touches caller tensors. */
+void spd_destroy(spd_ctx *ctx);
+
+const char *spd_status_string(int status);
+/* cudaError_t value of the most recent failing CUDA call seen by this thread (0 = none). */
+int spd_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPD_H */

@@ -1,0 +1,227 @@
+"""Thin Python binding of the SPD block library (``include/spd.h``).
+
+Argument marshalling only: PyTorch supplies device memory and streams, every step of the
+block runs in the CUDA library.  There is no fallback: if ``libspd_b200.so`` is missing or a
+call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libspd_b200.so")
+
+SPD_OK = 0
+STATUS_NAMES = {0: "SPD_OK", -1: "SPD_EINVAL", -2: "SPD_ENULL", -3: "SPD_EWORKSPACE", -4: "SPD_ECAPACITY",
+                -5: "SPD_ECUDA", -6: "SPD_EDEVICE"}
+WEIGHT_NAMES = ("attn_norm", "wq", "wk", "wv", "wo", "mlp_norm", "w_gate", "w_up", "w_down")
+EXPORTS = ("spd_workspace_bytes", "spd_create", "spd_prefill", "spd_decode_step", "spd_sync_points",
+           "spd_launches_per_decode_step", "spd_device_error", "spd_destroy", "spd_status_string",
+           "spd_last_cuda_error", "spd_profile_begin", "spd_profile_end", "spd_profile_kinds",
+           "spd_profile_kind_name")
+
+
+class SpdError(RuntimeError):
+    def __init__(self, where: str, status: int, detail: str = ""):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} {detail}".strip())
+
+
+class spd_dims(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int32), ("hidden", ctypes.c_int32), ("n_q_heads", ctypes.c_int32),
+                ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("ffn", ctypes.c_int32),
+                ("T", ctypes.c_int32), ("dtype", ctypes.c_int32), ("rms_eps", ctypes.c_float),
+                ("rope_base", ctypes.c_float), ("kv_block_size", ctypes.c_int32), ("max_batch", ctypes.c_int32),
+                ("max_seq_len", ctypes.c_int32), ("max_prefill_tokens", ctypes.c_int32)]
+
+
+class spd_layer(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in WEIGHT_NAMES] + [("k_pages", ctypes.c_void_p), ("v_pages", ctypes.c_void_p)]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load the in-tree CUDA library; raise if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2502_20727_b200.build` "
+                          "(there is no CPU or PyTorch fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+    lib.spd_workspace_bytes.argtypes = [ctypes.POINTER(spd_dims), vp, ctypes.POINTER(sz)]
+    lib.spd_create.argtypes = [ctypes.POINTER(spd_dims), vp, ctypes.POINTER(spd_layer), i32, vp, sz,
+                               ctypes.POINTER(vp)]
+    lib.spd_prefill.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp]
+    lib.spd_decode_step.argtypes = [vp, vp, i32, vp, vp, i32, i32, vp, vp]
+    lib.spd_sync_points.argtypes = [vp]
+    lib.spd_launches_per_decode_step.argtypes = [vp]
+    lib.spd_device_error.argtypes = [vp, vp, ctypes.POINTER(i32)]
+    lib.spd_destroy.argtypes = [vp]
+    lib.spd_destroy.restype = None
+    lib.spd_status_string.argtypes = [ctypes.c_int]
+    lib.spd_status_string.restype = ctypes.c_char_p
+    lib.spd_last_cuda_error.argtypes = []
+    lib.spd_profile_begin.argtypes = [vp]
+    lib.spd_profile_end.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
+    lib.spd_profile_kinds.argtypes = []
+    lib.spd_profile_kind_name.argtypes = [ctypes.c_int]
+    lib.spd_profile_kind_name.restype = ctypes.c_char_p
+    for n in EXPORTS:
+        if n not in ("spd_destroy", "spd_status_string", "spd_profile_kind_name"):
+            getattr(lib, n).restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def _check(where: str, rc: int):
+    if rc != SPD_OK:
+        lib = load_library()
+        detail = lib.spd_status_string(rc).decode()
+        if rc == -5:
+            detail += f" (cudaError {lib.spd_last_cuda_error()})"
+        raise SpdError(where, rc, detail)
+
+
+def _stream_ptr() -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class SpdStack:
+    """A stack of TP / SPD decoder blocks over caller-held weights and paged KV tensors.
+
+    layers: one dict per layer with the tensors of ``WEIGHT_NAMES`` (CUDA, contiguous, dtype
+    float32 or bfloat16, torch.nn.Linear layout).  sync_mask[l] = 1 runs layer l as the
+    synchronous TP block, 0 as the SPD block.
+    """
+
+    def __init__(self, *, hidden: int, n_q_heads: int, n_kv_heads: int, head_dim: int, ffn: int, T: int,
+                 sync_mask: Sequence[int], layers: List[Dict[str, torch.Tensor]], n_pages: int,
+                 max_batch: int, max_seq_len: int, max_prefill_tokens: int, rms_eps: float = 1e-5,
+                 rope_base: float = 10000.0, kv_block_size: int = 16, device: Optional[torch.device] = None):
+        self.lib = load_library()
+        self.device = torch.device(device if device is not None else "cuda:0")
+        dt = layers[0]["wq"].dtype
+        if dt not in (torch.float32, torch.bfloat16):
+            raise ValueError("weights must be float32 or bfloat16")
+        self.dtype = dt
+        self.dims = spd_dims(len(layers), hidden, n_q_heads, n_kv_heads, head_dim, ffn, T,
+                             0 if dt == torch.float32 else 1, rms_eps, rope_base, kv_block_size, max_batch,
+                             max_seq_len, max_prefill_tokens)
+        self.mask = (ctypes.c_uint8 * len(layers))(*[1 if m else 0 for m in sync_mask])
+        if len(sync_mask) != len(layers):
+            raise ValueError("one mask entry per layer")
+        self.layers = layers
+        self.n_pages = n_pages
+        for lw in layers:
+            for n in WEIGHT_NAMES:
+                t = lw[n]
+                if not (t.is_cuda and t.is_contiguous() and t.dtype == dt):
+                    raise ValueError(f"{n}: need a contiguous CUDA tensor of dtype {dt}")
+        with torch.cuda.device(self.device):
+            page_shape = (n_pages, n_kv_heads, kv_block_size, head_dim)
+            self.k_pages = [torch.zeros(page_shape, dtype=dt, device=self.device) for _ in layers]
+            self.v_pages = [torch.zeros(page_shape, dtype=dt, device=self.device) for _ in layers]
+            nbytes = ctypes.c_size_t(0)
+            _check("spd_workspace_bytes", self.lib.spd_workspace_bytes(ctypes.byref(self.dims), self.mask,
+                                                                         ctypes.byref(nbytes)))
+            self.workspace = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=self.device)
+            base = (self.workspace.data_ptr() + 255) // 256 * 256
+            arr = (spd_layer * len(layers))()
+            for i, lw in enumerate(layers):
+                for n in WEIGHT_NAMES:
+                    setattr(arr[i], n, lw[n].data_ptr())
+                arr[i].k_pages = self.k_pages[i].data_ptr()
+                arr[i].v_pages = self.v_pages[i].data_ptr()
+            self._ctx = ctypes.c_void_p()
+            _check("spd_create", self.lib.spd_create(ctypes.byref(self.dims), self.mask, arr, n_pages,
+                                                      ctypes.c_void_p(base), nbytes.value, ctypes.byref(self._ctx)))
+        self.workspace_bytes = nbytes.value
+
+    # -- calls ---------------------------------------------------------------------------
+    def prefill(self, x: torch.Tensor, block_table: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        B, S, H = x.shape
+        self._check_io(x, block_table)
+        out = torch.empty_like(x) if out is None else out
+        with torch.cuda.device(self.device):
+            _check("spd_prefill", self.lib.spd_prefill(self._ctx, x.data_ptr(), B, S, block_table.data_ptr(),
+                                                        block_table.shape[1], out.data_ptr(), _stream_ptr()))
+        return out
+
+    def decode_step(self, x: torch.Tensor, seq_lens: torch.Tensor, block_table: torch.Tensor, max_context: int,
+                    out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        B, H = x.shape
+        self._check_io(x, block_table)
+        if not (seq_lens.is_cuda and seq_lens.dtype == torch.int32 and seq_lens.numel() == B):
+            raise ValueError("seq_lens: int32 CUDA tensor [B]")
+        out = torch.empty_like(x) if out is None else out
+        with torch.cuda.device(self.device):
+            _check("spd_decode_step", self.lib.spd_decode_step(self._ctx, x.data_ptr(), B, seq_lens.data_ptr(),
+                                                                block_table.data_ptr(), block_table.shape[1],
+                                                                int(max_context), out.data_ptr(), _stream_ptr()))
+        return out
+
+    def device_error(self) -> int:
+        flag = ctypes.c_int32(0)
+        with torch.cuda.device(self.device):
+            _check("spd_device_error", self.lib.spd_device_error(self._ctx, _stream_ptr(), ctypes.byref(flag)))
+        return flag.value
+
+    def profile_begin(self):
+        _check("spd_profile_begin", self.lib.spd_profile_begin(self._ctx))
+
+    def profile_end(self) -> Dict[str, Dict[str, float]]:
+        """Returns {kind: {"ms": total, "launches": n}} for the calls since profile_begin."""
+        n = self.lib.spd_profile_kinds()
+        ms = (ctypes.c_float * n)()
+        cnt = (ctypes.c_int32 * n)()
+        with torch.cuda.device(self.device):
+            _check("spd_profile_end", self.lib.spd_profile_end(self._ctx, _stream_ptr(), ms, cnt))
+        return {self.lib.spd_profile_kind_name(i).decode(): {"ms": float(ms[i]), "launches": int(cnt[i])}
+                for i in range(n)}
+
+    def sync_points(self) -> int:
+        return self.lib.spd_sync_points(self._ctx)
+
+    def launches_last_call(self) -> int:
+        return self.lib.spd_launches_per_decode_step(self._ctx)
+
+    def _check_io(self, x, block_table):
+        if not (x.is_cuda and x.is_contiguous() and x.dtype == self.dtype and x.shape[-1] == self.dims.hidden):
+            raise ValueError("x: contiguous CUDA tensor [..., hidden] of the weights' dtype")
+        if not (block_table.is_cuda and block_table.dtype == torch.int32 and block_table.is_contiguous()
+                and block_table.shape[0] == x.shape[0]):
+            raise ValueError("block_table: contiguous int32 CUDA tensor [B, max_pages]")
+
+    def close(self):
+        if getattr(self, "_ctx", None) is not None and self._ctx.value:
+            self.lib.spd_destroy(self._ctx)
+            self._ctx = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def stack_from_workload(w, layers, *, sync_mask=None, max_batch=None, max_seq_len=None, max_prefill_tokens=None,
+                        n_pages=None, device="cuda:0") -> SpdStack:
+    """Build an SpdStack for a ``spd_inputs.Workload``-like object (duck-typed: the binding does
+    not import the input generators)."""
+    max_batch = max_batch or w.batch
+    max_seq_len = max_seq_len or (w.prompt + w.decode_steps)
+    pages_per_seq = (max_seq_len + w.kv_block - 1) // w.kv_block
+    n_pages = n_pages or max_batch * pages_per_seq
+    return SpdStack(hidden=w.hidden, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, head_dim=w.head_dim,
+                    ffn=w.ffn, T=w.T, sync_mask=list(w.mask if sync_mask is None else sync_mask), layers=layers,
+                    n_pages=n_pages, max_batch=max_batch, max_seq_len=max_seq_len,
+                    max_prefill_tokens=max_prefill_tokens or min(w.batch * w.prompt, 8192), rms_eps=w.rms_eps,
+                    rope_base=w.rope_base, kv_block_size=w.kv_block, device=device)

@@ -1,0 +1,134 @@
+// Shared device helpers and host-side launch declarations of the SPD block library.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace spd {
+
+typedef __nv_bfloat16 bf16;
+
+// Bits of the device error flag (read back by spd_device_error / the next call).
+enum : int {
+    ERR_PAGE_RANGE = 1,   // block-table entry outside [0, n_pages)
+    ERR_CAPACITY = 2,     // position beyond the block-table row / max_context
+    ERR_WAIT_TIMEOUT = 4, // a bounded mbarrier wait gave up
+};
+
+template <typename T> __device__ __forceinline__ float to_f(T v);
+template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f<bf16>(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// Where the tokens of a launch sit in their sequences.
+//   prefill chunk: token m = bi * ns + si is position s0 + si of sequence b0 + bi
+//   decode       : token m is position seq_lens[m] of sequence m
+struct TokMap {
+    int decode;
+    int b0, ns, s0;
+    const int32_t *seq_lens;
+    __device__ __forceinline__ void locate(int m, int &b, int &pos) const
+    {
+        if (decode) { b = m; pos = seq_lens[m]; }
+        else { b = b0 + m / ns; pos = s0 + m % ns; }
+    }
+};
+
+struct PageTable {
+    const int32_t *block_table; // [B, max_pages]
+    int max_pages, n_pages, block, n_kv_heads;
+};
+
+// ---- host-side launchers (defined in the .cu files) ----------------------------------
+
+// C[z][m][n] (+)= sum_k A_s[m][k] * W[s*n_per_shard + n][k] over split z's K range.
+struct GemmProblem {
+    const void *A;          // [M, K] row-major, leading dimension lda (elements)
+    long lda;
+    long a_shard_stride;    // elements between the A operands of consecutive shards (0: shared)
+    const void *W;          // [n_shards * n_per_shard, K] row-major, leading dimension ldw
+    long ldw;
+    float *C;               // fp32 [splits][M][ldc]; column = s * n_per_shard + n
+    long ldc;
+    long c_split_stride;    // elements between split planes
+    int M, n_per_shard, n_shards, K;
+    int splits;             // K is cut into `splits` equal ranges of k_per_split
+    int k_per_split;
+};
+template <typename T> cudaError_t launch_gemm_simt(const GemmProblem &p, cudaStream_t st);
+
+struct NormArgs {
+    const void *x_in;     // storage dtype [M,H] (first layer) or null
+    const float *res_in;  // fp32 [M,H] or null
+    const float *part;    // fp32 [n_groups * per_group][M][H] partial sums, or null
+    long part_stride;     // elements between partial planes
+    int n_groups;         // 1: everything is summed; T: SPD, one group per shard
+    int per_group;        // partial planes per group
+    float *res_out;       // fp32 [M,H]: res + all partials (may alias res_in)
+    void *h_out;          // storage [n_groups][M][H] (plane stride h_stride): norm(res + group)*g ; or null
+    long h_stride;
+    const void *gain;     // storage [H] or null (then no norm output)
+    void *final_out;      // storage [M,H] copy of res_out, or null
+    int M, H;
+    float eps;
+};
+template <typename T> cudaError_t launch_residual_norm(const NormArgs &a, cudaStream_t st);
+
+cudaError_t launch_rope_table(float2 *table, TokMap tm, int M, int head_dim, float base, cudaStream_t st);
+
+struct RopeKvArgs {
+    const float *qkv;     // fp32 [splits][M][ldq]: columns [q | k | v]
+    long ldq, split_stride;
+    int splits;
+    const float2 *table;  // [M][d/2] cos,sin
+    void *q_out;          // storage [M, nq*d]
+    void *k_pages, *v_pages;
+    PageTable pt;
+    TokMap tm;
+    int M, n_q_heads, head_dim;
+    int use_rope;
+    int *err;
+};
+template <typename T> cudaError_t launch_rope_kv(const RopeKvArgs &a, cudaStream_t st);
+
+struct SiluMulArgs {
+    const float *gate, *up; // fp32 [splits][M][ld]
+    long ld, split_stride;
+    int splits;
+    void *act;              // storage [M,F]
+    int M, F;
+};
+template <typename T> cudaError_t launch_silu_mul(const SiluMulArgs &a, cudaStream_t st);
+
+struct AttnArgs {
+    const void *q;          // storage [M, nq*d]
+    const void *k_pages, *v_pages;
+    PageTable pt;
+    TokMap tm;
+    void *out;              // storage [M, nq*d]
+    int M, n_q_heads, head_dim;
+    // decode only
+    int B, splits, max_context;
+    float *part_o;          // fp32 [B][nq][splits][d]
+    float *part_ml;         // fp32 [B][nq][splits][2]
+    int *err;
+};
+template <typename T> cudaError_t launch_prefill_attention(const AttnArgs &a, cudaStream_t st);
+template <typename T> cudaError_t launch_decode_attention(const AttnArgs &a, cudaStream_t st);
+
+} // namespace spd

@@ -1,0 +1,192 @@
+// Row-wise kernels between the GEMMs: the residual adds and RMSNorms of the TP and SPD
+// blocks (Sec. 3; Sec. 4.1.1: MLP input X + Y_i per shard, output X + sum_i (Y_i + Z_i)),
+// the rotary embedding + KV-page append, and SwiGLU.
+#include "common.cuh"
+
+namespace spd {
+
+constexpr int MAX_T = 8;
+
+__device__ __forceinline__ float block_sum(float v, float *red)
+{
+    v = warp_sum(v);
+    int w = threadIdx.x >> 5, l = threadIdx.x & 31, nw = blockDim.x >> 5;
+    __syncthreads();
+    if (l == 0) red[w] = v;
+    __syncthreads();
+    float t = (l < nw) ? red[l] : 0.f;
+    return warp_sum(t);
+}
+
+template <typename T> __device__ __forceinline__ float base_value(const NormArgs &a, long idx)
+{
+    return a.x_in ? to_f<T>(((const T *)a.x_in)[idx]) : a.res_in[idx];
+}
+
+__device__ __forceinline__ float group_sum(const NormArgs &a, int g, long idx)
+{
+    float y = 0.f;
+    for (int p = 0; p < a.per_group; ++p) y += a.part[(long)(g * a.per_group + p) * a.part_stride + idx];
+    return y;
+}
+
+// One CTA per token row.
+//   res_out  = base + sum over ALL partial planes   (base = x_in or res_in; res_out != res_in)
+//   h_out[g] = rmsnorm(base + sum of group g's planes) * gain
+// n_groups == 1 is the synchronous block's "all-reduce, residual add, norm"; n_groups == T is
+// the SPD block, where shard g only ever sees its own partial attention output Y_g while the
+// residual carried to the block output still collects every Y_g.
+template <typename T>
+__global__ void __launch_bounds__(256) residual_norm_kernel(NormArgs a)
+{
+    __shared__ float red[32];
+    const int m = blockIdx.x, H = a.H, G = a.n_groups;
+    float ss[MAX_T];
+#pragma unroll
+    for (int g = 0; g < MAX_T; ++g) ss[g] = 0.f;
+
+    for (int j = threadIdx.x; j < H; j += blockDim.x) {
+        const long idx = (long)m * H + j;
+        float base = base_value<T>(a, idx), tot = 0.f;
+#pragma unroll
+        for (int g = 0; g < MAX_T; ++g)
+            if (g < G) {
+                float y = a.part ? group_sum(a, g, idx) : 0.f;
+                tot += y;
+                ss[g] += (base + y) * (base + y);
+            }
+        float r_all = base + tot;
+        if (a.res_out) a.res_out[idx] = r_all;
+        if (a.final_out) ((T *)a.final_out)[idx] = from_f<T>(r_all);
+    }
+    if (!a.h_out) return;
+    float rs[MAX_T];
+#pragma unroll
+    for (int g = 0; g < MAX_T; ++g) rs[g] = (g < G) ? rsqrtf(block_sum(ss[g], red) / (float)H + a.eps) : 0.f;
+    // second pass re-reads the row (L1/L2 resident)
+    const T *gain = (const T *)a.gain;
+    for (int j = threadIdx.x; j < H; j += blockDim.x) {
+        const long idx = (long)m * H + j;
+        float base = base_value<T>(a, idx), gj = to_f<T>(gain[j]);
+#pragma unroll
+        for (int g = 0; g < MAX_T; ++g)
+            if (g < G) {
+                float y = a.part ? group_sum(a, g, idx) : 0.f;
+                ((T *)a.h_out)[(long)g * a.h_stride + idx] = from_f<T>((base + y) * rs[g] * gj);
+            }
+    }
+}
+
+template <typename T> cudaError_t launch_residual_norm(const NormArgs &a, cudaStream_t st)
+{
+    if (a.M <= 0) return cudaSuccess;
+    residual_norm_kernel<T><<<a.M, 256, 0, st>>>(a);
+    return cudaGetLastError();
+}
+template cudaError_t launch_residual_norm<float>(const NormArgs &, cudaStream_t);
+template cudaError_t launch_residual_norm<bf16>(const NormArgs &, cudaStream_t);
+
+// cos/sin of pos * base^(-2j/d), evaluated in double once per call and shared by all layers.
+__global__ void rope_table_kernel(float2 *table, TokMap tm, int M, int half, double log_base, int d)
+{
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= M * half) return;
+    int m = i / half, j = i % half, b, pos;
+    tm.locate(m, b, pos);
+    double theta = exp(-2.0 * (double)j / (double)d * log_base);
+    double s, c;
+    sincos((double)pos * theta, &s, &c);
+    table[i] = make_float2((float)c, (float)s);
+}
+
+cudaError_t launch_rope_table(float2 *table, TokMap tm, int M, int head_dim, float base, cudaStream_t st)
+{
+    int n = M * (head_dim / 2);
+    if (n <= 0) return cudaSuccess;
+    rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(table, tm, M, head_dim / 2, log((double)base), head_dim);
+    return cudaGetLastError();
+}
+
+// grid (M, n_q_heads + n_kv_heads): sums the split-K planes of one head's projection, rotates
+// q and k (pairs (j, j + d/2)), stores q for the attention kernel and k, v into their page.
+template <typename T> __global__ void rope_kv_kernel(RopeKvArgs a)
+{
+    const int m = blockIdx.x, head = blockIdx.y, d = a.head_dim, half = d / 2;
+    const int nq = a.n_q_heads, nkv = a.pt.n_kv_heads;
+    int b, pos;
+    a.tm.locate(m, b, pos);
+    const bool is_q = head < nq;
+    const int kvh = head - nq;
+    long kv_off = 0;
+    if (!is_q) {
+        int pi = pos / a.pt.block;
+        if (pos < 0 || pi >= a.pt.max_pages) { if (threadIdx.x == 0) atomicOr(a.err, ERR_CAPACITY); return; }
+        int page = a.pt.block_table[(long)b * a.pt.max_pages + pi];
+        if (page < 0 || page >= a.pt.n_pages) { if (threadIdx.x == 0) atomicOr(a.err, ERR_PAGE_RANGE); return; }
+        kv_off = (((long)page * nkv + kvh) * a.pt.block + pos % a.pt.block) * d;
+    }
+    const long col_q = (long)head * d;                 // q or k column of this head
+    const long col_v = (long)(nq + nkv + kvh) * d;     // v column (kv heads only)
+    for (int j = threadIdx.x; j < half; j += blockDim.x) {
+        float x0 = 0.f, x1 = 0.f, v0 = 0.f, v1 = 0.f;
+        for (int s = 0; s < a.splits; ++s) {
+            const float *row = a.qkv + (long)s * a.split_stride + (long)m * a.ldq;
+            x0 += row[col_q + j];
+            x1 += row[col_q + j + half];
+            if (!is_q) { v0 += row[col_v + j]; v1 += row[col_v + j + half]; }
+        }
+        float c = 1.f, sn = 0.f;
+        if (a.use_rope) { float2 cs = a.table[(long)m * half + j]; c = cs.x; sn = cs.y; }
+        float r0 = x0 * c - x1 * sn, r1 = x1 * c + x0 * sn;
+        if (is_q) {
+            T *q = (T *)a.q_out + (long)m * nq * d + (long)head * d;
+            q[j] = from_f<T>(r0);
+            q[j + half] = from_f<T>(r1);
+        } else {
+            T *kp = (T *)a.k_pages + kv_off, *vp = (T *)a.v_pages + kv_off;
+            kp[j] = from_f<T>(r0);
+            kp[j + half] = from_f<T>(r1);
+            vp[j] = from_f<T>(v0);
+            vp[j + half] = from_f<T>(v1);
+        }
+    }
+}
+
+template <typename T> cudaError_t launch_rope_kv(const RopeKvArgs &a, cudaStream_t st)
+{
+    if (a.M <= 0) return cudaSuccess;
+    dim3 grid(a.M, a.n_q_heads + a.pt.n_kv_heads);
+    int threads = a.head_dim / 2 >= 64 ? 64 : 32;
+    rope_kv_kernel<T><<<grid, threads, 0, st>>>(a);
+    return cudaGetLastError();
+}
+template cudaError_t launch_rope_kv<float>(const RopeKvArgs &, cudaStream_t);
+template cudaError_t launch_rope_kv<bf16>(const RopeKvArgs &, cudaStream_t);
+
+// act = silu(sum_s gate_s) * (sum_s up_s)
+template <typename T> __global__ void silu_mul_kernel(SiluMulArgs a)
+{
+    long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    long n = (long)a.M * a.F;
+    if (i >= n) return;
+    long m = i / a.F, f = i % a.F;
+    float g = 0.f, u = 0.f;
+    for (int s = 0; s < a.splits; ++s) {
+        g += a.gate[(long)s * a.split_stride + m * a.ld + f];
+        u += a.up[(long)s * a.split_stride + m * a.ld + f];
+    }
+    float act = g / (1.f + __expf(-g)) * u;
+    ((T *)a.act)[i] = from_f<T>(act);
+}
+
+template <typename T> cudaError_t launch_silu_mul(const SiluMulArgs &a, cudaStream_t st)
+{
+    long n = (long)a.M * a.F;
+    if (n <= 0) return cudaSuccess;
+    silu_mul_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, st>>>(a);
+    return cudaGetLastError();
+}
+template cudaError_t launch_silu_mul<float>(const SiluMulArgs &, cudaStream_t);
+template cudaError_t launch_silu_mul<bf16>(const SiluMulArgs &, cudaStream_t);
+
+} // namespace spd

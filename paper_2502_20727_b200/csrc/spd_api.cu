@@ -1,0 +1,487 @@
+// C ABI of the SPD block library: validation, workspace layout and the per-layer launch
+// sequence of the synchronous TP block (Sec. 3) and the SPD block (Sec. 4.1.1).
+#include "../../include/spd.h"
+#include "common.cuh"
+
+#include <math.h>
+#include <new>
+#include <string.h>
+#include <vector>
+
+using namespace spd;
+
+static thread_local int g_last_cuda_error = 0;
+
+#define CU_TRY(expr)                                                   \
+    do {                                                               \
+        cudaError_t e__ = (expr);                                      \
+        if (e__ != cudaSuccess) { g_last_cuda_error = (int)e__; return SPD_ECUDA; } \
+    } while (0)
+
+namespace {
+
+constexpr int N_SM = 148;
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// How one launch sequence cuts its GEMMs.
+struct Plan {
+    int qkv_splits, qkv_kps;
+    int o_per_group, o_groups, o_kps;  // planes = o_groups * o_per_group
+    int gu_splits, gu_kps;
+    int down_splits, down_kps;
+    int attn_splits;
+};
+
+// Largest s <= want such that K splits into s ranges that are multiples of `align`.
+int fit_splits(int K, int want, int align)
+{
+    for (int s = want; s > 1; --s)
+        if (K % s == 0 && (K / s) % align == 0) return s;
+    return 1;
+}
+
+int want_splits(int M, int N)
+{
+    long tiles = (long)((M + 63) / 64) * ((N + 63) / 64);
+    long s = (2 * N_SM + tiles - 1) / tiles;
+    return (int)(s < 1 ? 1 : (s > 16 ? 16 : s));
+}
+
+struct Ctx {
+    spd_dims d;
+    std::vector<uint8_t> mask;
+    std::vector<spd_layer> layers;
+    int n_pages;
+    bool any_spd;
+    char *ws;
+    size_t ws_bytes;
+    // workspace regions
+    float *res[2];
+    void *h, *q, *attn, *act;
+    float *qkv32, *proj32, *gu32, *part_o, *part_ml;
+    float2 *rope;
+    int *err;
+    int launches_last;
+    // optional per-kernel-kind timing (spd_profile_begin / spd_profile_end)
+    bool profiling;
+    std::vector<cudaEvent_t> ev_pool;
+    std::vector<int> ev_kind; // kind of the launch bracketed by events 2i, 2i+1
+    size_t ev_used;
+};
+
+enum Kind { K_NORM = 0, K_QKV, K_ROPE_KV, K_ATTN, K_OPROJ, K_GATE_UP, K_SILU_MUL, K_DOWN, K_ROPE_TABLE, K_COUNT };
+const char *const kind_names[K_COUNT] = {"residual_rmsnorm", "gemm_qkv", "rope_kv_append", "attention", "gemm_o_proj",
+                                         "gemm_gate_up", "silu_mul", "gemm_down", "rope_table"};
+
+cudaError_t prof_mark(Ctx *c, int kind, cudaStream_t st)
+{
+    if (!c->profiling) return cudaSuccess;
+    if (c->ev_used == c->ev_pool.size()) {
+        cudaEvent_t e;
+        cudaError_t rc = cudaEventCreate(&e);
+        if (rc != cudaSuccess) return rc;
+        c->ev_pool.push_back(e);
+    }
+    if (kind >= 0) c->ev_kind.push_back(kind);
+    return cudaEventRecord(c->ev_pool[c->ev_used++], st);
+}
+
+#define LAUNCH(kind, expr)                   \
+    do {                                     \
+        CU_TRY(prof_mark(c, (kind), st));    \
+        CU_TRY(expr);                        \
+        CU_TRY(prof_mark(c, -1, st));        \
+        ++launches;                          \
+    } while (0)
+
+size_t esize(const spd_dims &d) { return d.dtype == 0 ? 4 : 2; }
+
+Plan make_plan(const spd_dims &d, int M, bool decode, bool spd_layer_present, int max_context)
+{
+    (void)spd_layer_present;
+    Plan p;
+    const int H = d.hidden, qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, F = d.ffn, T = d.T;
+    if (!decode) {
+        p.qkv_splits = 1; p.gu_splits = 1; p.down_splits = 1; p.o_per_group = 1;
+    } else {
+        p.qkv_splits = fit_splits(H, want_splits(M, qd + 2 * kd), 16);
+        p.gu_splits = fit_splits(H, want_splits(M, 2 * F), 16);
+        p.down_splits = fit_splits(F, want_splits(M, H), 16);
+        int w = want_splits(M, H);
+        p.o_per_group = fit_splits(qd / T, (w + T - 1) / T, 16);
+    }
+    p.o_groups = T;
+    p.qkv_kps = H / p.qkv_splits;
+    p.gu_kps = H / p.gu_splits;
+    p.down_kps = F / p.down_splits;
+    p.o_kps = qd / (p.o_groups * p.o_per_group);
+    // decode attention: enough CTAs for the machine, at least 2 pages per split
+    if (decode) {
+        long ctas = (long)M * d.n_q_heads;
+        int s = (int)((2 * N_SM + ctas - 1) / ctas);
+        int pages = (max_context + d.kv_block_size - 1) / d.kv_block_size;
+        int smax = pages / 2 < 1 ? 1 : pages / 2;
+        if (s > smax) s = smax;
+        if (s > 32) s = 32;
+        if (s < 1) s = 1;
+        p.attn_splits = s;
+    } else p.attn_splits = 1;
+    return p;
+}
+
+struct Layout {
+    size_t res[2], h, q, attn, act, qkv32, proj32, gu32, part_o, part_ml, rope, err, total;
+};
+
+// Sizes every region for the worse of the two regimes (prefill chunk, decode batch).
+Layout make_layout(const spd_dims &d, bool any_spd)
+{
+    const size_t es = esize(d);
+    const size_t H = d.hidden, qd = (size_t)d.n_q_heads * d.head_dim, kd = (size_t)d.n_kv_heads * d.head_dim;
+    const size_t F = d.ffn, T = d.T, nqkv = qd + 2 * kd;
+    size_t Mp = d.max_prefill_tokens, Md = d.max_batch;
+    size_t Mmax = Mp > Md ? Mp : Md;
+    Plan pp = make_plan(d, (int)Mp, false, any_spd, d.max_seq_len);
+    Plan pd = make_plan(d, (int)Md, true, any_spd, d.max_seq_len);
+    auto mx = [](size_t a, size_t b) { return a > b ? a : b; };
+    Layout L;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    L.err = take(256);
+    L.res[0] = take(Mmax * H * 4);
+    L.res[1] = take(Mmax * H * 4);
+    L.h = take((any_spd ? T : 1) * Mmax * H * es);
+    L.q = take(Mmax * qd * es);
+    L.attn = take(Mmax * qd * es);
+    L.act = take(Mmax * F * es);
+    L.rope = take(Mmax * (d.head_dim / 2) * sizeof(float2));
+    L.qkv32 = take(mx(pp.qkv_splits * Mp, pd.qkv_splits * Md) * nqkv * 4);
+    size_t o_planes_p = (size_t)pp.o_groups * pp.o_per_group, o_planes_d = (size_t)pd.o_groups * pd.o_per_group;
+    L.proj32 = take(mx(mx(o_planes_p, pp.down_splits) * Mp, mx(o_planes_d, pd.down_splits) * Md) * H * 4);
+    L.gu32 = take(mx(pp.gu_splits * Mp, pd.gu_splits * Md) * 2 * F * 4);
+    L.part_o = take(Md * d.n_q_heads * 32 * d.head_dim * 4);
+    L.part_ml = take(Md * d.n_q_heads * 32 * 2 * 4);
+    L.total = off;
+    return L;
+}
+
+int check_dims(const spd_dims *d, const uint8_t *mask)
+{
+    if (!d || !mask) return SPD_ENULL;
+    if (d->n_layers < 1 || d->hidden < 8 || d->n_q_heads < 1 || d->n_kv_heads < 1 || d->ffn < 1) return SPD_EINVAL;
+    if (d->T < 1 || d->T > 8) return SPD_EINVAL;
+    if (d->dtype != 0 && d->dtype != 1) return SPD_EINVAL;
+    if (d->head_dim != 32 && d->head_dim != 64 && d->head_dim != 128) return SPD_EINVAL;
+    if (d->n_q_heads % d->n_kv_heads) return SPD_EINVAL;
+    if (d->n_q_heads % d->T || d->n_kv_heads % d->T || d->ffn % d->T) return SPD_EINVAL;
+    if (d->hidden % 8 || (d->ffn / d->T) % 8) return SPD_EINVAL;
+    if (d->kv_block_size < 1 || d->max_batch < 1 || d->max_seq_len < 1 || d->max_prefill_tokens < 1) return SPD_EINVAL;
+    if (!(d->rms_eps > 0.f)) return SPD_EINVAL;
+    return SPD_OK;
+}
+
+template <typename T>
+int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t *bt, int max_pages,
+               bool decode, int max_context, cudaStream_t st)
+{
+    const spd_dims &d = c->d;
+    const int H = d.hidden, qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, F = d.ffn, Tn = d.T;
+    const int nqkv = qd + 2 * kd;
+    const Plan p = make_plan(d, M, decode, c->any_spd, max_context);
+    PageTable pt{bt, max_pages, c->n_pages, d.kv_block_size, d.n_kv_heads};
+    int launches = 0;
+
+    if (d.rope_base > 0.f) LAUNCH(K_ROPE_TABLE, launch_rope_table(c->rope, tm, M, d.head_dim, d.rope_base, st));
+
+    // block input -> fp32 residual stream and its attention RMSNorm
+    {
+        NormArgs a{};
+        a.x_in = x; a.res_out = c->res[0]; a.h_out = c->h; a.h_stride = (long)M * H;
+        a.gain = c->layers[0].attn_norm; a.n_groups = 1; a.per_group = 0; a.M = M; a.H = H; a.eps = d.rms_eps;
+        LAUNCH(K_NORM, launch_residual_norm<T>(a, st));
+    }
+    for (int l = 0; l < d.n_layers; ++l) {
+        const spd_layer &w = c->layers[l];
+        const bool sync = c->mask[l] != 0;
+        // a2: column-split Q/K/V projections of all shards = the full matrices
+        const void *wm[3] = {w.wq, w.wk, w.wv};
+        const int wn[3] = {qd, kd, kd}, wcol[3] = {0, qd, qd + kd};
+        for (int i = 0; i < 3; ++i) {
+            GemmProblem g{};
+            g.A = c->h; g.lda = H; g.a_shard_stride = 0; g.W = wm[i]; g.ldw = H;
+            g.C = c->qkv32 + wcol[i]; g.ldc = nqkv; g.c_split_stride = (long)M * nqkv;
+            g.M = M; g.n_per_shard = wn[i]; g.n_shards = 1; g.K = H; g.splits = p.qkv_splits; g.k_per_split = p.qkv_kps;
+            LAUNCH(K_QKV, launch_gemm_simt<T>(g, st));
+        }
+        // a3: rotary embedding, KV-page append
+        {
+            RopeKvArgs a{};
+            a.qkv = c->qkv32; a.ldq = nqkv; a.split_stride = (long)M * nqkv; a.splits = p.qkv_splits;
+            a.table = c->rope; a.q_out = c->q; a.k_pages = w.k_pages; a.v_pages = w.v_pages; a.pt = pt; a.tm = tm;
+            a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.use_rope = d.rope_base > 0.f; a.err = c->err;
+            LAUNCH(K_ROPE_KV, launch_rope_kv<T>(a, st));
+        }
+        // a4: attention, each shard over its own heads
+        {
+            AttnArgs a{};
+            a.q = c->q; a.k_pages = w.k_pages; a.v_pages = w.v_pages; a.pt = pt; a.tm = tm; a.out = c->attn;
+            a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.B = M; a.splits = p.attn_splits;
+            a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.err = c->err;
+            if (decode) { LAUNCH(K_ATTN, launch_decode_attention<T>(a, st)); ++launches; }
+            else LAUNCH(K_ATTN, launch_prefill_attention<T>(a, st));
+        }
+        // a5: row-split output projection; plane (i, j) holds the part of Y_i from K sub-range j
+        // (a synchronous block in prefill needs only the sum: one plane over all of K)
+        const bool o_single = sync && !decode;
+        const int o_planes = o_single ? 1 : p.o_groups * p.o_per_group;
+        {
+            GemmProblem g{};
+            g.A = c->attn; g.lda = qd; g.W = w.wo; g.ldw = qd; g.C = c->proj32; g.ldc = H; g.c_split_stride = (long)M * H;
+            g.M = M; g.n_per_shard = H; g.n_shards = 1; g.K = qd; g.splits = o_planes; g.k_per_split = o_single ? qd : p.o_kps;
+            LAUNCH(K_OPROJ, launch_gemm_simt<T>(g, st));
+        }
+        // a6 + a7: sync-point #1 (sync) or its drop (SPD), residual add, MLP RMSNorm
+        {
+            NormArgs a{};
+            a.res_in = c->res[0]; a.part = c->proj32; a.part_stride = (long)M * H;
+            a.n_groups = sync ? 1 : Tn; a.per_group = sync ? o_planes : p.o_per_group;
+            a.res_out = c->res[1]; a.h_out = c->h; a.h_stride = (long)M * H; a.gain = w.mlp_norm;
+            a.M = M; a.H = H; a.eps = d.rms_eps;
+            LAUNCH(K_NORM, launch_residual_norm<T>(a, st));
+        }
+        // a8: column-split gate / up; in an SPD block shard i reads its own MLP input plane
+        const void *gm[2] = {w.w_gate, w.w_up};
+        for (int i = 0; i < 2; ++i) {
+            GemmProblem g{};
+            g.A = c->h; g.lda = H; g.a_shard_stride = sync ? 0 : (long)M * H; g.W = gm[i]; g.ldw = H;
+            g.C = c->gu32 + (long)i * p.gu_splits * M * F; g.ldc = F; g.c_split_stride = (long)M * F;
+            g.M = M; g.n_per_shard = F / Tn; g.n_shards = Tn; g.K = H; g.splits = p.gu_splits; g.k_per_split = p.gu_kps;
+            LAUNCH(K_GATE_UP, launch_gemm_simt<T>(g, st));
+        }
+        {
+            SiluMulArgs a{};
+            a.gate = c->gu32; a.up = c->gu32 + (long)p.gu_splits * M * F; a.ld = F; a.split_stride = (long)M * F;
+            a.splits = p.gu_splits; a.act = c->act; a.M = M; a.F = F;
+            LAUNCH(K_SILU_MUL, launch_silu_mul<T>(a, st));
+        }
+        // a9: row-split down projection; summing over all of K = F IS the kept sync-point
+        {
+            GemmProblem g{};
+            g.A = c->act; g.lda = F; g.W = w.w_down; g.ldw = F; g.C = c->proj32; g.ldc = H; g.c_split_stride = (long)M * H;
+            g.M = M; g.n_per_shard = H; g.n_shards = 1; g.K = F; g.splits = p.down_splits; g.k_per_split = p.down_kps;
+            LAUNCH(K_DOWN, launch_gemm_simt<T>(g, st));
+        }
+        // a10: output residual.  res[1] already holds X + sum_i Y_i in both modes
+        // (sync: R; SPD: Y_i before the sum, X after it), so out = res[1] + sum_i Z_i.
+        {
+            NormArgs a{};
+            a.res_in = c->res[1]; a.part = c->proj32; a.part_stride = (long)M * H; a.n_groups = 1; a.per_group = p.down_splits;
+            a.res_out = c->res[0]; a.M = M; a.H = H; a.eps = d.rms_eps;
+            if (l + 1 < d.n_layers) { a.h_out = c->h; a.h_stride = (long)M * H; a.gain = c->layers[l + 1].attn_norm; }
+            else a.final_out = out;
+            LAUNCH(K_NORM, launch_residual_norm<T>(a, st));
+        }
+    }
+    c->launches_last = launches;
+    return SPD_OK;
+}
+
+int read_err_flag(Ctx *c, cudaStream_t st, int *flag)
+{
+    CU_TRY(cudaMemcpyAsync(flag, c->err, sizeof(int), cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaStreamSynchronize(st));
+    if (*flag) CU_TRY(cudaMemsetAsync(c->err, 0, sizeof(int), st));
+    return SPD_OK;
+}
+
+} // namespace
+
+struct spd_ctx { Ctx c; };
+
+extern "C" {
+
+int spd_workspace_bytes(const spd_dims *dims, const uint8_t *sync_mask, size_t *out_bytes)
+{
+    if (!out_bytes) return SPD_ENULL;
+    int rc = check_dims(dims, sync_mask);
+    if (rc) return rc;
+    bool any_spd = false;
+    for (int l = 0; l < dims->n_layers; ++l) any_spd |= sync_mask[l] == 0;
+    *out_bytes = make_layout(*dims, any_spd).total;
+    return SPD_OK;
+}
+
+int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *layers, int32_t n_pages,
+               void *workspace, size_t workspace_bytes, spd_ctx **out)
+{
+    if (!out || !layers || !workspace) return SPD_ENULL;
+    int rc = check_dims(dims, sync_mask);
+    if (rc) return rc;
+    if (n_pages < 1) return SPD_EINVAL;
+    for (int l = 0; l < dims->n_layers; ++l) {
+        const spd_layer &w = layers[l];
+        if (!w.attn_norm || !w.wq || !w.wk || !w.wv || !w.wo || !w.mlp_norm || !w.w_gate || !w.w_up || !w.w_down ||
+            !w.k_pages || !w.v_pages)
+            return SPD_ENULL;
+    }
+    int dev = 0;
+    cudaDeviceProp prop;
+    CU_TRY(cudaGetDevice(&dev));
+    CU_TRY(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major != 10) return SPD_EINVAL;
+    bool any_spd = false;
+    for (int l = 0; l < dims->n_layers; ++l) any_spd |= sync_mask[l] == 0;
+    Layout L = make_layout(*dims, any_spd);
+    if (workspace_bytes < L.total || ((uintptr_t)workspace & 255)) return SPD_EWORKSPACE;
+    spd_ctx *h = new (std::nothrow) spd_ctx();
+    if (!h) return SPD_EINVAL;
+    Ctx &c = h->c;
+    c.d = *dims;
+    c.mask.assign(sync_mask, sync_mask + dims->n_layers);
+    c.layers.assign(layers, layers + dims->n_layers);
+    c.n_pages = n_pages;
+    c.any_spd = any_spd;
+    c.ws = (char *)workspace;
+    c.ws_bytes = workspace_bytes;
+    c.err = (int *)(c.ws + L.err);
+    c.res[0] = (float *)(c.ws + L.res[0]);
+    c.res[1] = (float *)(c.ws + L.res[1]);
+    c.h = c.ws + L.h; c.q = c.ws + L.q; c.attn = c.ws + L.attn; c.act = c.ws + L.act;
+    c.rope = (float2 *)(c.ws + L.rope);
+    c.qkv32 = (float *)(c.ws + L.qkv32); c.proj32 = (float *)(c.ws + L.proj32); c.gu32 = (float *)(c.ws + L.gu32);
+    c.part_o = (float *)(c.ws + L.part_o); c.part_ml = (float *)(c.ws + L.part_ml);
+    c.launches_last = 0;
+    c.profiling = false;
+    c.ev_used = 0;
+    cudaError_t e = cudaMemset(c.err, 0, 256);
+    if (e != cudaSuccess) { g_last_cuda_error = (int)e; delete h; return SPD_ECUDA; }
+    *out = h;
+    return SPD_OK;
+}
+
+int spd_prefill(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int32_t *block_table, int32_t max_pages,
+                void *out, void *stream)
+{
+    if (!ctx || !x || !block_table || !out) return SPD_ENULL;
+    Ctx &c = ctx->c;
+    const spd_dims &d = c.d;
+    if (B < 1 || S < 1 || B > d.max_batch || x == out) return SPD_EINVAL;
+    if (S > d.max_seq_len || (long)max_pages * d.kv_block_size < S) return SPD_ECAPACITY;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t es = esize(d);
+    const int Mp = d.max_prefill_tokens;
+    int total_launches = 0;
+    auto run = [&](int b0, int nb, int s0, int ns) -> int {
+        TokMap tm{0, b0, ns, s0, nullptr};
+        size_t off = ((size_t)b0 * S + s0) * d.hidden * es;
+        int rc = d.dtype == 0 ? run_tokens<float>(&c, (const char *)x + off, (char *)out + off, nb * ns, tm, block_table, max_pages, false, S, st)
+                              : run_tokens<bf16>(&c, (const char *)x + off, (char *)out + off, nb * ns, tm, block_table, max_pages, false, S, st);
+        total_launches += c.launches_last;
+        return rc;
+    };
+    if (S <= Mp) {
+        int nb = Mp / S;
+        for (int b0 = 0; b0 < B; b0 += nb) {
+            int rc = run(b0, (B - b0 < nb) ? B - b0 : nb, 0, S);
+            if (rc) return rc;
+        }
+    } else {
+        for (int b = 0; b < B; ++b)
+            for (int s0 = 0; s0 < S; s0 += Mp) {
+                int rc = run(b, 1, s0, (S - s0 < Mp) ? S - s0 : Mp);
+                if (rc) return rc;
+            }
+    }
+    c.launches_last = total_launches;
+    return SPD_OK;
+}
+
+int spd_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_lens, const int32_t *block_table,
+                    int32_t max_pages, int32_t max_context, void *out, void *stream)
+{
+    if (!ctx || !x || !seq_lens || !block_table || !out) return SPD_ENULL;
+    Ctx &c = ctx->c;
+    const spd_dims &d = c.d;
+    if (B < 1 || B > d.max_batch || x == out || max_context < 1) return SPD_EINVAL;
+    if (max_context > d.max_seq_len || (long)max_pages * d.kv_block_size < max_context) return SPD_ECAPACITY;
+    cudaStream_t st = (cudaStream_t)stream;
+    TokMap tm{1, 0, 1, 0, seq_lens};
+    return d.dtype == 0 ? run_tokens<float>(&c, x, out, B, tm, block_table, max_pages, true, max_context, st)
+                        : run_tokens<bf16>(&c, x, out, B, tm, block_table, max_pages, true, max_context, st);
+}
+
+int spd_sync_points(const spd_ctx *ctx)
+{
+    if (!ctx) return SPD_ENULL;
+    int n = 0;
+    for (uint8_t m : ctx->c.mask) n += m ? 2 : 1;
+    return n;
+}
+
+int spd_launches_per_decode_step(const spd_ctx *ctx) { return ctx ? ctx->c.launches_last : SPD_ENULL; }
+
+int spd_device_error(spd_ctx *ctx, void *stream, int32_t *out_flag)
+{
+    if (!ctx || !out_flag) return SPD_ENULL;
+    int flag = 0;
+    int rc = read_err_flag(&ctx->c, (cudaStream_t)stream, &flag);
+    *out_flag = flag;
+    return rc;
+}
+
+int spd_profile_begin(spd_ctx *ctx)
+{
+    if (!ctx) return SPD_ENULL;
+    ctx->c.profiling = true;
+    ctx->c.ev_used = 0;
+    ctx->c.ev_kind.clear();
+    return SPD_OK;
+}
+
+int spd_profile_end(spd_ctx *ctx, void *stream, float *ms_by_kind, int32_t *launches_by_kind)
+{
+    if (!ctx || !ms_by_kind || !launches_by_kind) return SPD_ENULL;
+    Ctx &c = ctx->c;
+    c.profiling = false;
+    CU_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    for (int k = 0; k < K_COUNT; ++k) { ms_by_kind[k] = 0.f; launches_by_kind[k] = 0; }
+    for (size_t i = 0; i < c.ev_kind.size(); ++i) {
+        float ms = 0.f;
+        CU_TRY(cudaEventElapsedTime(&ms, c.ev_pool[2 * i], c.ev_pool[2 * i + 1]));
+        ms_by_kind[c.ev_kind[i]] += ms;
+        launches_by_kind[c.ev_kind[i]] += 1;
+    }
+    c.ev_used = 0;
+    c.ev_kind.clear();
+    return SPD_OK;
+}
+
+int spd_profile_kinds(void) { return K_COUNT; }
+
+const char *spd_profile_kind_name(int kind) { return (kind >= 0 && kind < K_COUNT) ? kind_names[kind] : "?"; }
+
+void spd_destroy(spd_ctx *ctx)
+{
+    if (!ctx) return;
+    for (cudaEvent_t e : ctx->c.ev_pool) cudaEventDestroy(e);
+    delete ctx;
+}
+
+const char *spd_status_string(int s)
+{
+    switch (s) {
+    case SPD_OK: return "ok";
+    case SPD_EINVAL: return "invalid argument or dimension";
+    case SPD_ENULL: return "null pointer";
+    case SPD_EWORKSPACE: return "workspace too small or misaligned";
+    case SPD_ECAPACITY: return "sequence exceeds the KV capacity";
+    case SPD_ECUDA: return "CUDA error";
+    case SPD_EDEVICE: return "device-side error flag set";
+    default: return "unknown status";
+    }
+}
+
+int spd_last_cuda_error(void) { return g_last_cuda_error; }
+
+} // extern "C"

@@ -1,0 +1,97 @@
+"""Shared plumbing of the GPU parity tests: run the CUDA library and the CPU oracle on the
+same seeded inputs and compare.  No arithmetic of the method lives here."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+import spd_inputs as si
+
+TOL = {"fp32": 1e-4, "bf16": 2e-2}
+
+
+def rel_err(got, ref) -> float:
+    """max |got - ref| / max |ref| over the tensor: the bound the tolerances are stated on."""
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    return float(np.max(np.abs(got - ref)) / max(float(np.max(np.abs(ref))), 1e-30))
+
+
+def oracle_dims(w: si.Workload) -> oracle.Dims:
+    return oracle.Dims(w.n_layers, w.hidden, w.n_q_heads, w.n_kv_heads, w.head_dim, w.ffn, w.T, w.rms_eps,
+                       w.rope_base)
+
+
+def to_np(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to("cpu", torch.float64).numpy()
+
+
+class Pair:
+    """One workload instantiated on both sides."""
+
+    def __init__(self, w: si.Workload, *, mask=None, B=None, max_len=None, max_prefill_tokens=None, seed=0,
+                 device="cuda:0", n_pages=None, layers=None):
+        import paper_2502_20727_b200 as spd
+        self.w = w
+        self.B = B or w.batch
+        self.max_len = max_len or (w.prompt + w.decode_steps)
+        self.mask = list(w.mask if mask is None else mask)
+        self.device = device
+        self.layers = layers if layers is not None else si.make_stack(w, "cpu", seed)
+        self.layers_gpu = [{n: t.to(device) for n, t in lw.items()} for lw in self.layers]
+        self.layers_np = si.to_oracle_layers(self.layers)
+        self.dims = oracle_dims(w)
+        self.cache = oracle.Cache(self.dims, self.B, self.max_len)
+        pages_per_seq = (self.max_len + w.kv_block - 1) // w.kv_block
+        self.n_pages = n_pages or (self.B * pages_per_seq + 3)
+        self.block_table = si.make_block_table(self.B, pages_per_seq, self.n_pages, seed).to(device)
+        self.stack = spd.stack_from_workload(w, self.layers_gpu, sync_mask=self.mask, max_batch=self.B,
+                                             max_seq_len=self.max_len, n_pages=self.n_pages,
+                                             max_prefill_tokens=max_prefill_tokens or 4096, device=device)
+        self.pos = np.zeros(self.B, dtype=np.int32)
+
+    def prefill(self, S, seed=0):
+        x = si.make_hidden(self.w, (self.B, S, self.w.hidden), "cpu", seed, 0)
+        ref, syncs, _ = oracle.stack_forward(self.dims, self.mask, self.layers_np, to_np(x), self.pos, self.cache)
+        got = self.stack.prefill(x.to(self.device), self.block_table)
+        torch.cuda.synchronize()
+        self.pos = self.pos + S
+        return to_np(got), ref, syncs
+
+    def decode(self, t, seed=0):
+        x = si.make_hidden(self.w, (self.B, self.w.hidden), "cpu", seed, 1 + t)
+        ref, _, _ = oracle.stack_forward(self.dims, self.mask, self.layers_np, to_np(x)[:, None, :], self.pos, self.cache)
+        seq = torch.from_numpy(self.pos.copy()).to(self.device)
+        got = self.stack.decode_step(x.to(self.device), seq, self.block_table, int(self.pos.max()) + 1)
+        torch.cuda.synchronize()
+        self.pos = self.pos + 1
+        return to_np(got), ref[:, 0, :]
+
+    def fill_cache(self, lens, seed=0):
+        """Put the same synthetic K/V (N(0,1), storage dtype) into the GPU pages and the oracle's
+        cache for positions [0, lens[b]) of every sequence and layer."""
+        w = self.w
+        bs, kvw = w.kv_block, w.n_kv_heads * w.head_dim
+        bt = self.block_table.cpu().numpy()
+        for l in range(w.n_layers):
+            for which, pages in (("k", self.stack.k_pages[l]), ("v", self.stack.v_pages[l])):
+                fill = si.make_kv_fill(w, (self.B, self.max_len, w.n_kv_heads, w.head_dim), "cpu", seed,
+                                       2 * l + (which == "v"))
+                host_pages = torch.zeros(pages.shape, dtype=pages.dtype)
+                for b in range(self.B):
+                    n = int(lens[b])
+                    getattr(self.cache, which)[l, b, :n] = to_np(fill[b, :n]).reshape(n, kvw)
+                    for j in range((n + bs - 1) // bs):
+                        cnt = min(bs, n - j * bs)
+                        host_pages[bt[b, j], :, :cnt] = fill[b, j * bs:j * bs + cnt].transpose(0, 1)
+                pages.copy_(host_pages)
+        self.pos = np.asarray(lens, dtype=np.int32).copy()
+
+    def gpu_cache(self, layer, which, b, n):
+        """K or V of sequence b, positions [0, n), gathered from the GPU pages -> [n, nkv*d]."""
+        w = self.w
+        pages = (self.stack.k_pages if which == "k" else self.stack.v_pages)[layer].cpu()
+        bt = self.block_table.cpu().numpy()
+        rows = [pages[bt[b, t // w.kv_block], :, t % w.kv_block, :].reshape(-1) for t in range(n)]
+        return to_np(torch.stack(rows))

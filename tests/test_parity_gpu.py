@@ -1,0 +1,120 @@
+"""GPU parity: the CUDA library through its C ABI against the CPU oracle, element by element,
+on the same seeded inputs.  Bound: max|gpu-ref|/max|ref| <= 1e-4 (float32), 2e-2 (bfloat16)."""
+import numpy as np
+import pytest
+import torch
+
+import spd_inputs as si
+from parity_util import TOL, Pair, rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+def run_case(w, mask, B, S, steps, max_prefill_tokens=None, check_cache=True):
+    p = Pair(w, mask=mask, B=B, max_len=S + steps, max_prefill_tokens=max_prefill_tokens)
+    tol = TOL[w.dtype]
+    got, ref, syncs = p.prefill(S)
+    assert got.shape == ref.shape
+    e = rel_err(got, ref)
+    assert e <= tol, f"prefill rel err {e}"
+    assert p.stack.sync_points() == syncs
+    for t in range(steps):
+        got, ref = p.decode(t)
+        e = rel_err(got, ref)
+        assert e <= tol, f"decode step {t} rel err {e}"
+    if check_cache:
+        n = S + steps
+        for l in (0, w.n_layers - 1):
+            for which in ("k", "v"):
+                ref_c = getattr(p.cache, which)[l, B - 1, :n]
+                e = rel_err(p.gpu_cache(l, which, B - 1, n), ref_c)
+                assert e <= tol, f"{which} cache layer {l} rel err {e}"
+    assert p.stack.device_error() == 0
+    p.stack.close()
+
+
+@pytest.mark.parametrize("mask", [(0,), (1,)])
+def test_c1_tiny_fp32_full(mask):
+    """configs[0]: 1 layer, hidden 256, 4 heads x 64, FFN 688, T=2, batch 1, 16 prompt + 8 decode."""
+    w = si.WORKLOADS["c1"]
+    run_case(w, mask, w.batch, w.prompt, w.decode_steps)
+
+
+@pytest.mark.parametrize("T", [1, 2, 4])
+@pytest.mark.parametrize("mask", [(0, 0), (1, 1), (1, 0)])
+def test_fp32_two_layers_any_T(T, mask):
+    w = si.WORKLOADS["c1"].with_(n_layers=2, T=T, mask=mask)
+    run_case(w, mask, 3, 21, 3)
+
+
+def test_fp32_without_rope_and_head_dim_32():
+    w = si.WORKLOADS["c1"].with_(rope_base=0.0, head_dim=32, n_q_heads=8, n_kv_heads=4, T=4)
+    run_case(w, (0,), 2, 19, 2)
+
+
+@pytest.mark.parametrize("mask", [(0, 1, 0), (1, 1, 1)])
+def test_bf16_small_ragged(mask):
+    """Odd sizes: 5 tokens over a page boundary, FFN/T = 344 (not a tile multiple), GQA 8/4."""
+    w = si.Workload("small", "bf16", 3, 512, 8, 4, 64, 1376, 4, mask, 3, 37, 3)
+    run_case(w, mask, 3, 37, 3)
+
+
+def test_bf16_chunked_prefill_inside_a_sequence():
+    """max_prefill_tokens smaller than the prompt: later chunks attend to cached earlier ones."""
+    w = si.Workload("small", "bf16", 2, 256, 4, 4, 64, 512, 2, (0, 1), 2, 50, 1)
+    run_case(w, (0, 1), 2, 50, 1, max_prefill_tokens=16)
+
+
+def test_bf16_chunked_prefill_by_sequences():
+    w = si.Workload("small", "bf16", 2, 256, 4, 4, 64, 512, 2, (0, 0), 5, 20, 1)
+    run_case(w, (0, 0), 5, 20, 1, max_prefill_tokens=45)
+
+
+@pytest.mark.parametrize("name,layers,B,S", [("c2", 2, 2, 24), ("c3_t4", 1, 2, 20), ("c3_t8", 1, 1, 20),
+                                             ("c4_b32", 1, 2, 18)])
+def test_full_model_dims_reduced_tokens(name, layers, B, S):
+    """Full hidden / head / FFN sizes of configs[1..3] with few tokens and layers."""
+    w0 = si.WORKLOADS[name]
+    mask = tuple(w0.mask[:layers]) if name != "c3_t4" else (0,)
+    w = w0.with_(n_layers=layers, mask=mask)
+    run_case(w, mask, B, S, 2, check_cache=False)
+
+
+def test_mask_is_honoured_on_the_gpu():
+    """An SPD mask on the GPU must NOT match the oracle's synchronous stack."""
+    w = si.Workload("small", "bf16", 2, 256, 4, 4, 64, 512, 4, (0, 0), 2, 12, 0)
+    lay = si.make_stack(w, "cpu", 0)
+    for lw in lay:  # make the attention branch large enough to matter
+        lw["wo"] = (lw["wo"].float() * 20).to(torch.bfloat16)
+    p_spd = Pair(w, mask=(0, 0), B=2, max_len=12, layers=lay)
+    got_spd, ref_spd, _ = p_spd.prefill(12)
+    p_sync = Pair(w, mask=(1, 1), B=2, max_len=12, layers=lay)
+    got_sync, ref_sync, _ = p_sync.prefill(12)
+    assert rel_err(got_spd, ref_spd) <= TOL["bf16"]
+    assert rel_err(got_sync, ref_sync) <= TOL["bf16"]
+    assert rel_err(got_spd, ref_sync) > 5 * TOL["bf16"]
+
+
+def test_decode_at_bench_size_on_synthetic_cache():
+    """configs[1] at its full decode shape (4 layers, batch 8, context 512+) with the KV cache
+    pre-filled with seeded values on both sides, so the oracle only pays for the decode step."""
+    w = si.WORKLOADS["c2"]
+    p = Pair(w, B=8, max_len=w.prompt + 4)
+    lens = np.array([512, 512, 500, 512, 17, 512, 1, 511], dtype=np.int32)
+    p.fill_cache(lens)
+    for t in range(2):
+        got, ref = p.decode(t)
+        e = rel_err(got, ref)
+        assert e <= TOL["bf16"], f"step {t}: {e}"
+    assert p.stack.device_error() == 0
+
+
+def test_run_twice_bitwise_identical():
+    w = si.Workload("small", "bf16", 2, 512, 8, 8, 64, 1024, 4, (0, 1), 4, 33, 2)
+    outs = []
+    for _ in range(2):
+        p = Pair(w, B=4, max_len=40)
+        a, _, _ = p.prefill(33)
+        b, _ = p.decode(0)
+        outs.append((a, b))
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
