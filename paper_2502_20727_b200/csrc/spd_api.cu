@@ -175,7 +175,7 @@ int check_dims(const spd_dims *d, const uint8_t *mask)
     if (d->head_dim != 32 && d->head_dim != 64 && d->head_dim != 128) return SPD_EINVAL;
     if (d->n_q_heads % d->n_kv_heads) return SPD_EINVAL;
     if (d->n_q_heads % d->T || d->n_kv_heads % d->T || d->ffn % d->T) return SPD_EINVAL;
-    if (d->hidden % 8 || (d->ffn / d->T) % 8) return SPD_EINVAL;
+    if (d->dtype == 1 && (d->hidden % 8 || (d->ffn / d->T) % 8)) return SPD_EINVAL; // 16-byte rows for bf16 tiles
     if (d->kv_block_size < 1 || d->max_batch < 1 || d->max_seq_len < 1 || d->max_prefill_tokens < 1) return SPD_EINVAL;
     if (!(d->rms_eps > 0.f)) return SPD_EINVAL;
     return SPD_OK;

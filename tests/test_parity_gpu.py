@@ -84,8 +84,10 @@ def test_mask_is_honoured_on_the_gpu():
     """An SPD mask on the GPU must NOT match the oracle's synchronous stack."""
     w = si.Workload("small", "bf16", 2, 256, 4, 4, 64, 512, 4, (0, 0), 2, 12, 0)
     lay = si.make_stack(w, "cpu", 0)
-    for lw in lay:  # make the attention branch large enough to matter
+    for lw in lay:  # make the attention and MLP branches as large as the residual stream
         lw["wo"] = (lw["wo"].float() * 20).to(torch.bfloat16)
+        for n in ("w_gate", "w_up", "w_down"):
+            lw[n] = (lw[n].float() * 5).to(torch.bfloat16)
     p_spd = Pair(w, mask=(0, 0), B=2, max_len=12, layers=lay)
     got_spd, ref_spd, _ = p_spd.prefill(12)
     p_sync = Pair(w, mask=(1, 1), B=2, max_len=12, layers=lay)
