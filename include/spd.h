@@ -110,6 +110,18 @@ int spd_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_l
                     const int32_t *block_table, int32_t max_pages, int32_t max_context,
                     void *out, void *stream);
 
+/* The projection building block on its own (exposed for kernel-level tests): the bf16
+ * tensor-core GEMM every projection of the block uses, with the batching that expresses the
+ * shard structure of Sec. 4.1.1 - per-shard weight row blocks (column split) and, when
+ * a_batched != 0, a separate input per shard (the SPD block's per-device MLP input).
+ *   a : bf16 [a_batched ? batches : 1][M][K]      w : bf16 [batches][N][K]
+ *   c : fp32 [splits][M][batches*N];  c[s][m][z*N + n] = sum over K-range s of a_z[m][:] . w_z[n][:]
+ *   swap != 0 puts the weight rows on the 128-row MMA side (the decode configuration)
+ *   err_flag : device int32, bit 4 is set if a bounded wait inside the kernel gave up
+ * K must be a multiple of 8; 1 <= splits <= ceil(K/64).  Errors: SPD_ENULL, SPD_EINVAL, SPD_ECUDA. */
+int spd_gemm_bf16(const void *a, const void *w, float *c, int32_t M, int32_t N, int32_t K, int32_t batches,
+                  int32_t a_batched, int32_t splits, int32_t swap, int32_t *err_flag, void *stream);
+
 /* Number of shard sums ("sync-points", Sec. 3) one forward pass of this stack executes:
  * 2 per TP block, 1 per SPD block. */
 int spd_sync_points(const spd_ctx *ctx);

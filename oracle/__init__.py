@@ -170,3 +170,12 @@ def rope(v, pos: int, base: float):
     v = np.array(v, dtype=np.float64).copy()
     lib().oracle_rope(_p(v), v.shape[0], int(pos), ctypes.c_double(base))
     return v
+
+
+def linear(x, w):
+    """y = x @ w.T in float64 (x float64 [M,K], w float32 [N,K])."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    w = _f32(w)
+    out = np.empty((x.shape[0], w.shape[0]), dtype=np.float64)
+    lib().oracle_linear(_p(x), _p(w), x.shape[0], w.shape[0], x.shape[1], _p(out))
+    return out

@@ -400,3 +400,10 @@ int oracle_block_forward(const oracle_dims *D, const oracle_layer *layer, int mo
         if (pos0[b] < 0 || pos0[b] + S > max_len) return -1;
     return block_sharded(D, layer, mode, x, B, S, pos0, kcache, vcache, max_len, out, y_out);
 }
+
+/* A plain linear layer y = x W^T (W in torch.nn.Linear layout), the building block of every
+ * projection above; exported so that the GEMM kernels can be checked in isolation. */
+void oracle_linear(const double *x, const float *w, int M, int N, int K, double *y)
+{
+    linear_slice(x, M, K, K, w, K, 0, N, 0, y, N);
+}

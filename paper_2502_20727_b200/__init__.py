@@ -22,7 +22,7 @@ WEIGHT_NAMES = ("attn_norm", "wq", "wk", "wv", "wo", "mlp_norm", "w_gate", "w_up
 EXPORTS = ("spd_workspace_bytes", "spd_create", "spd_prefill", "spd_decode_step", "spd_sync_points",
            "spd_launches_per_decode_step", "spd_device_error", "spd_destroy", "spd_status_string",
            "spd_last_cuda_error", "spd_profile_begin", "spd_profile_end", "spd_profile_kinds",
-           "spd_profile_kind_name")
+           "spd_profile_kind_name", "spd_gemm_bf16")
 
 
 class SpdError(RuntimeError):
@@ -69,13 +69,14 @@ def load_library() -> ctypes.CDLL:
     lib.spd_status_string.argtypes = [ctypes.c_int]
     lib.spd_status_string.restype = ctypes.c_char_p
     lib.spd_last_cuda_error.argtypes = []
+    lib.spd_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, vp]
     lib.spd_profile_begin.argtypes = [vp]
     lib.spd_profile_end.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     lib.spd_profile_kinds.argtypes = []
     lib.spd_profile_kind_name.argtypes = [ctypes.c_int]
     lib.spd_profile_kind_name.restype = ctypes.c_char_p
     for n in EXPORTS:
-        if n not in ("spd_destroy", "spd_status_string", "spd_profile_kind_name"):
+        if n not in ("spd_destroy", "spd_status_string", "spd_profile_kind_name", "spd_gemm_bf16"):
             getattr(lib, n).restype = ctypes.c_int
     _lib = lib
     return lib
@@ -92,6 +93,30 @@ def _check(where: str, rc: int):
 
 def _stream_ptr() -> ctypes.c_void_p:
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def gemm_bf16(a: torch.Tensor, w: torch.Tensor, *, splits: int = 1, swap: bool = False) -> torch.Tensor:
+    """The projection GEMM on its own.  a: bf16 [M,K] or [batches,M,K]; w: bf16 [N,K] or [batches,N,K].
+    Returns fp32 [splits, M, batches*N]."""
+    lib = load_library()
+    wb = w if w.dim() == 3 else w[None]
+    a_batched = a.dim() == 3
+    batches, N, K = wb.shape
+    M = a.shape[-2]
+    if a_batched and a.shape[0] != batches:
+        raise ValueError("a and w disagree on the batch count")
+    for t in (a, w):
+        if not (t.is_cuda and t.is_contiguous() and t.dtype == torch.bfloat16):
+            raise ValueError("contiguous CUDA bf16 tensors expected")
+    c = torch.empty((splits, M, batches * N), dtype=torch.float32, device=a.device)
+    err = torch.zeros(1, dtype=torch.int32, device=a.device)
+    with torch.cuda.device(a.device):
+        _check("spd_gemm_bf16", lib.spd_gemm_bf16(a.data_ptr(), w.data_ptr(), c.data_ptr(), M, N, K, batches,
+                                                   1 if a_batched else 0, splits, 1 if swap else 0, err.data_ptr(),
+                                                   _stream_ptr()))
+    if int(err.item()) != 0:
+        raise SpdError("spd_gemm_bf16", -6, f"device flag {int(err.item())}")
+    return c
 
 
 class SpdStack:

@@ -1,0 +1,320 @@
+// bf16 projection GEMM on the 5th-generation tensor cores: TMA (cp.async.bulk.tensor, no
+// multicast) -> 128B-swizzled shared-memory ring -> tcgen05.mma (cta_group::1, kind::f16)
+// with the fp32 accumulator in tensor memory -> tcgen05.ld epilogue.
+//
+// One launch computes, for every batch z (an emulated TP shard, or a single batch) and K-split s,
+//     C[z, s][m][col0(z) + n] = sum_{k in split s} A_z[m][k] * W_z[n][k]
+// Both operands are K-major ([rows, K] row-major), so no transposes are needed for
+// activations x torch.nn.Linear weights.  Batching over z is how the shard structure of the
+// SPD block (Sec. 4.1.1) is expressed: per-shard K-slices of the row-split o_proj whose
+// planes Y_z are kept apart, and per-shard MLP inputs for the column-split gate/up.
+//
+// SWAP = true  (decode, few tokens): the 128-row MMA "M" side holds WEIGHT rows and the tokens
+//               sit on the N side (BN = 16..64), so a CTA streams a 128 x K weight slab.
+// SWAP = false (prefill): tokens on the M side, BN weight rows on the N side.
+#include "common.cuh"
+#include "gemm_tc.cuh"
+
+#include <cuda.h>
+
+namespace spd {
+
+namespace {
+
+constexpr int BM = 128;      // MMA M (TMEM lanes)
+constexpr int BK = 64;       // one 128-byte swizzle atom of bf16 per row
+constexpr int UMMA_K = 16;
+constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL; // about one second
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+// Bounded wait: gives up after WAIT_LIMIT_CYCLES, records it, and lets the caller unwind.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int *err, volatile int *abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*abort_flag || clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            *abort_flag = 1;
+            atomicOr(err, ERR_WAIT_TIMEOUT);
+            return false;
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) and
+// 128B-swizzled: 8-row groups 1024 bytes apart, descriptor version 1 (sm_100), layout type 2.
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);   // start address
+    d |= (uint64_t)1 << 16;                        // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;              // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                        // version
+    d |= (uint64_t)2 << 61;                        // SWIZZLE_128B
+    return d;
+}
+
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v)
+{
+    uint32_t r[16];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                 : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+constexpr uint32_t make_idesc(int n)
+{
+    // fp32 accumulator, bf16 A and B, both K-major, M = 128
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+template <int BN> struct Cfg {
+    static constexpr int STAGES = (BN <= 64) ? 5 : 3;
+    static constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+template <int BN, bool SWAP>
+__global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a,
+                                                      const __grid_constant__ CUtensorMap tm_b, TcGemmArgs g)
+{
+    using C = Cfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t bars = base + C::STAGES * C::STAGE_BYTES; // full[S], empty[S], tmem_full
+    uint32_t *tmem_slot = (uint32_t *)(gen_base + C::STAGES * C::STAGE_BYTES + 8 * (2 * C::STAGES + 1));
+    volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (C::STAGES + s); };
+    const uint32_t tmem_full_bar = bars + 8u * (2 * C::STAGES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // tile coordinates: x -> (batch z, weight tile), y -> token tile, z -> split
+    const int z = blockIdx.x / g.w_tiles_per_batch;
+    const int w_row0 = (blockIdx.x % g.w_tiles_per_batch) * (SWAP ? BM : BN);
+    const int t_row0 = blockIdx.y * (SWAP ? BN : BM);
+    const int split = blockIdx.z;
+    const int kb_begin = (int)((long)g.num_kb * split / g.splits);
+    const int kb_end = (int)((long)g.num_kb * (split + 1) / g.splits);
+    const int n_kb = kb_end - kb_begin;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        mbar_init(tmem_full_bar, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_a) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_b) : "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_acc = *tmem_slot;
+
+    // A side = 128-row operand, B side = BN-row operand
+    const int a_row0 = SWAP ? w_row0 : t_row0, b_row0 = SWAP ? t_row0 : w_row0;
+    const int a_z = SWAP ? (g.w_batched ? z : 0) : (g.t_batched ? z : 0);
+    const int b_z = SWAP ? (g.t_batched ? z : 0) : (g.w_batched ? z : 0);
+
+    if (warp == 0 && lane == 0) {
+        // TMA producer
+        for (int i = 0; i < n_kb; ++i) {
+            const int s = i % C::STAGES;
+            if (!mbar_wait(empty_bar(s), ((i / C::STAGES) & 1) ^ 1, g.err, abort_flag)) break;
+            mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
+            const uint32_t sa = base + s * C::STAGE_BYTES, sb = sa + C::A_BYTES;
+            const int kx = (kb_begin + i) * BK;
+            tma_load_3d(sa, &tm_a, kx, a_row0, a_z, full_bar(s));
+            tma_load_3d(sb, &tm_b, kx, b_row0, b_z, full_bar(s));
+        }
+    } else if (warp == 1 && lane == 0) {
+        // MMA issuer
+        constexpr uint32_t idesc = make_idesc(BN);
+        bool ok = true;
+        for (int i = 0; i < n_kb && ok; ++i) {
+            const int s = i % C::STAGES;
+            ok = mbar_wait(full_bar(s), (i / C::STAGES) & 1, g.err, abort_flag);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t sa = base + s * C::STAGE_BYTES, sb = sa + C::A_BYTES;
+            const uint64_t da = make_desc(sa), db = make_desc(sb);
+#pragma unroll
+            for (int k = 0; k < BK / UMMA_K; ++k)
+                umma(tmem_acc, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
+                     (i > 0 || k > 0) ? 1u : 0u);
+            umma_commit(empty_bar(s)); // frees the stage once these MMAs have read it
+        }
+        umma_commit(tmem_full_bar);    // arrives when every MMA above has completed
+    }
+    __syncwarp();
+
+    // epilogue: warp w owns TMEM lanes [32w, 32w+32)
+    const bool acc_ok = (n_kb > 0) && mbar_wait(tmem_full_bar, 0, g.err, abort_flag);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    __syncwarp();
+    float *Cz = g.C + (long)z * g.c_batch_stride + (long)split * g.c_split_stride;
+    const int row = warp * 32 + lane; // accumulator row = TMEM lane
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN; c0 += 16) {
+        float v[16];
+        if (acc_ok) tmem_ld16(tmem_acc + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+        else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] = 0.f;
+        }
+        if (SWAP) {
+            // row = weight row n, columns = tokens m
+            const int n = w_row0 + row;
+            if (n < g.w_rows) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int m = t_row0 + c0 + j;
+                    if (m < g.t_rows) Cz[(long)m * g.ldc + n] = v[j];
+                }
+            }
+        } else {
+            // row = token m, columns = weight rows n
+            const int m = t_row0 + row;
+            if (m < g.t_rows) {
+                float *dst = Cz + (long)m * g.ldc + w_row0 + c0;
+                if (w_row0 + c0 + 16 <= g.w_rows && ((((uintptr_t)dst) & 15) == 0)) {
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4) *(float4 *)(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (w_row0 + c0 + j < g.w_rows) dst[j] = v[j];
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(C::TMEM_COLS) : "memory");
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+template <int BN, bool SWAP> cudaError_t launch_cfg(const CUtensorMap &ta, const CUtensorMap &tb, const TcGemmArgs &g, dim3 grid, cudaStream_t st)
+{
+    using C = Cfg<BN>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, SWAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    gemm_tc_kernel<BN, SWAP><<<grid, 128, C::SMEM_BYTES, st>>>(ta, tb, g);
+    return cudaGetLastError();
+}
+
+} // namespace
+
+// rows x K bf16 matrix (row stride ld elements), optionally `batches` of them, as a 3-D map
+// {K, rows, batches} with a {64, box_rows, 1} box and the 128-byte swizzle.
+int make_operand_map(TcMap *out, const void *ptr, long k_inner, long rows, long batches, long ld_elems,
+                     long batch_stride_elems, int box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return -1;
+    if (((uintptr_t)ptr & 15) || (ld_elems * 2) % 16 || (batches > 1 && (batch_stride_elems * 2) % 16)) return -2;
+    cuuint64_t dims[3] = {(cuuint64_t)k_inner, (cuuint64_t)rows, (cuuint64_t)(batches < 1 ? 1 : batches)};
+    cuuint64_t strides[2] = {(cuuint64_t)ld_elems * 2, (cuuint64_t)(batches > 1 ? batch_stride_elems : ld_elems * rows) * 2};
+    cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn((CUtensorMap *)out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? 0 : -3;
+}
+
+int tc_token_box(bool swap, int tokens)
+{
+    if (!swap) return BM;
+    return tokens <= 16 ? 16 : (tokens <= 32 ? 32 : 64);
+}
+int tc_weight_box(bool swap) { return BM; }
+
+cudaError_t launch_gemm_tc(const TcMap &weights, const TcMap &tokens, const TcGemmArgs &g, bool swap, cudaStream_t st)
+{
+    if (g.t_rows <= 0 || g.w_rows <= 0) return cudaSuccess;
+    if (g.splits < 1 || g.splits > g.num_kb) return cudaErrorInvalidValue;
+    const CUtensorMap &tw = *(const CUtensorMap *)&weights, &tt = *(const CUtensorMap *)&tokens;
+    if (swap) {
+        const int bn = tc_token_box(true, g.t_rows);
+        TcGemmArgs a = g;
+        a.w_tiles_per_batch = (g.w_rows + BM - 1) / BM;
+        dim3 grid(a.w_tiles_per_batch * g.batches, (g.t_rows + bn - 1) / bn, g.splits);
+        switch (bn) {
+        case 16: return launch_cfg<16, true>(tw, tt, a, grid, st);
+        case 32: return launch_cfg<32, true>(tw, tt, a, grid, st);
+        default: return launch_cfg<64, true>(tw, tt, a, grid, st);
+        }
+    }
+    TcGemmArgs a = g;
+    a.w_tiles_per_batch = (g.w_rows + 127) / 128;
+    dim3 grid(a.w_tiles_per_batch * g.batches, (g.t_rows + BM - 1) / BM, g.splits);
+    return launch_cfg<128, false>(tt, tw, a, grid, st);
+}
+
+} // namespace spd

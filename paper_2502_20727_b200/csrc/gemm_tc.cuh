@@ -1,0 +1,38 @@
+// Host interface of the tcgen05 projection GEMM (gemm_tc.cu).
+#pragma once
+#include <cuda_runtime.h>
+
+namespace spd {
+
+// A CUtensorMap kept opaque so that callers need not include the driver header.
+struct alignas(64) TcMap { unsigned long long opaque[16]; };
+
+struct TcGemmArgs {
+    float *C;             // fp32 output
+    long ldc;             // elements between token rows of C
+    long c_batch_stride;  // elements added per batch z (a column offset or a plane offset)
+    long c_split_stride;  // elements between K-split planes
+    int t_rows;           // valid token rows
+    int w_rows;           // valid weight rows per batch
+    int batches;          // z extent
+    int w_batched;        // weight operand has a batch dimension
+    int t_batched;        // token operand has a batch dimension
+    int num_kb;           // 64-wide K blocks per batch (ceil)
+    int splits;           // K splits, <= num_kb
+    int w_tiles_per_batch; // filled by the launcher
+    int *err;             // device error flag
+};
+
+// Encode rows x k_inner bf16 (row stride ld_elems), `batches` of them batch_stride_elems apart.
+// Returns 0, or <0 when the driver entry point is missing / alignment is violated / encode fails.
+int make_operand_map(TcMap *out, const void *ptr, long k_inner, long rows, long batches, long ld_elems,
+                     long batch_stride_elems, int box_rows);
+
+// Box rows of the token-side operand for a given token count (swap: 16/32/64, else 128).
+int tc_token_box(bool swap, int tokens);
+int tc_weight_box(bool swap);
+
+// swap = weights on the 128-row MMA side (decode); otherwise tokens on it (prefill).
+cudaError_t launch_gemm_tc(const TcMap &weights, const TcMap &tokens, const TcGemmArgs &g, bool swap, cudaStream_t st);
+
+} // namespace spd

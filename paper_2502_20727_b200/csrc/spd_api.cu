@@ -2,6 +2,7 @@
 // sequence of the synchronous TP block (Sec. 3) and the SPD block (Sec. 4.1.1).
 #include "../../include/spd.h"
 #include "common.cuh"
+#include "gemm_tc.cuh"
 
 #include <math.h>
 #include <new>
@@ -23,14 +24,13 @@ namespace {
 constexpr int N_SM = 148;
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int cdiv(int a, int b) { return (a + b - 1) / b; }
 
-// How one launch sequence cuts its GEMMs.
+// How one launch sequence cuts its GEMMs along K (per-call-site split counts).
 struct Plan {
-    int qkv_splits, qkv_kps;
-    int o_per_group, o_groups, o_kps;  // planes = o_groups * o_per_group
-    int gu_splits, gu_kps;
-    int down_splits, down_kps;
-    int attn_splits;
+    int qkv_splits, o_per_group, gu_splits, down_splits, attn_splits;
+    // float32 (CUDA-core) path only: elements of K per split
+    int qkv_kps, o_kps, gu_kps, down_kps;
 };
 
 // Largest s <= want such that K splits into s ranges that are multiples of `align`.
@@ -41,38 +41,45 @@ int fit_splits(int K, int want, int align)
     return 1;
 }
 
-int want_splits(int M, int N)
+int want_splits(long tiles, int cap)
 {
-    long tiles = (long)((M + 63) / 64) * ((N + 63) / 64);
     long s = (2 * N_SM + tiles - 1) / tiles;
-    return (int)(s < 1 ? 1 : (s > 16 ? 16 : s));
+    if (s > cap) s = cap;
+    return (int)(s < 1 ? 1 : s);
 }
+
+enum ActBuf { AB_H = 0, AB_ATTN, AB_ATTN_SHARD, AB_ACT, AB_COUNT };
+enum Kind { K_NORM = 0, K_QKV, K_ROPE_KV, K_ATTN, K_OPROJ, K_GATE_UP, K_SILU_MUL, K_DOWN, K_ROPE_TABLE, K_COUNT };
+const char *const kind_names[K_COUNT] = {"residual_rmsnorm", "gemm_qkv", "rope_kv_append", "attention", "gemm_o_proj",
+                                         "gemm_gate_up", "silu_mul", "gemm_down", "rope_table"};
+
+struct LayerMaps { TcMap wq, wk, wv, wo_full, wo_shard, w_gate, w_up, w_down; };
 
 struct Ctx {
     spd_dims d;
     std::vector<uint8_t> mask;
     std::vector<spd_layer> layers;
+    std::vector<LayerMaps> maps; // bf16 only
     int n_pages;
     bool any_spd;
+    long Mcap; // token capacity of every activation buffer (plane stride = Mcap * width)
     char *ws;
     size_t ws_bytes;
-    // workspace regions
     float *res[2];
     void *h, *q, *attn, *act;
     float *qkv32, *proj32, *gu32, *part_o, *part_ml;
     float2 *rope;
     int *err;
     int launches_last;
+    // activation tensor maps, by buffer and token box (16, 32, 64, 128), built on first use
+    TcMap act_maps[AB_COUNT][4];
+    bool act_map_ready[AB_COUNT][4];
     // optional per-kernel-kind timing (spd_profile_begin / spd_profile_end)
     bool profiling;
     std::vector<cudaEvent_t> ev_pool;
     std::vector<int> ev_kind; // kind of the launch bracketed by events 2i, 2i+1
     size_t ev_used;
 };
-
-enum Kind { K_NORM = 0, K_QKV, K_ROPE_KV, K_ATTN, K_OPROJ, K_GATE_UP, K_SILU_MUL, K_DOWN, K_ROPE_TABLE, K_COUNT };
-const char *const kind_names[K_COUNT] = {"residual_rmsnorm", "gemm_qkv", "rope_kv_append", "attention", "gemm_o_proj",
-                                         "gemm_gate_up", "silu_mul", "gemm_down", "rope_table"};
 
 cudaError_t prof_mark(Ctx *c, int kind, cudaStream_t st)
 {
@@ -97,41 +104,49 @@ cudaError_t prof_mark(Ctx *c, int kind, cudaStream_t st)
 
 size_t esize(const spd_dims &d) { return d.dtype == 0 ? 4 : 2; }
 
-Plan make_plan(const spd_dims &d, int M, bool decode, bool spd_layer_present, int max_context)
+// M = tokens of the launch.  decode: few tokens, the weight-streaming GEMMs are cut along K so
+// that about two CTAs per SM are in flight; prefill: no K splits.
+Plan make_plan(const spd_dims &d, int M, bool decode, int max_context)
 {
-    (void)spd_layer_present;
-    Plan p;
+    Plan p{};
     const int H = d.hidden, qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, F = d.ffn, T = d.T;
-    if (!decode) {
-        p.qkv_splits = 1; p.gu_splits = 1; p.down_splits = 1; p.o_per_group = 1;
-    } else {
-        p.qkv_splits = fit_splits(H, want_splits(M, qd + 2 * kd), 16);
-        p.gu_splits = fit_splits(H, want_splits(M, 2 * F), 16);
-        p.down_splits = fit_splits(F, want_splits(M, H), 16);
-        int w = want_splits(M, H);
-        p.o_per_group = fit_splits(qd / T, (w + T - 1) / T, 16);
+    p.qkv_splits = p.gu_splits = p.down_splits = p.o_per_group = 1;
+    if (decode && d.dtype == 1) {
+        // tcgen05 path: 128-row weight tiles, 64-wide K blocks, uneven splits allowed, >= 4 blocks each
+        const int tok_tiles = cdiv(M, 64);
+        auto cap = [](int kb) { int c = kb / 4; return c < 1 ? 1 : (c > 16 ? 16 : c); };
+        p.qkv_splits = want_splits((long)cdiv(kd < qd ? kd : qd, 128) * tok_tiles * 2, cap(cdiv(H, 64)));
+        p.gu_splits = want_splits((long)cdiv(F / T, 128) * T * tok_tiles, cap(cdiv(H, 64)));
+        p.down_splits = want_splits((long)cdiv(H, 128) * tok_tiles, cap(cdiv(F, 64)));
+        p.o_per_group = want_splits((long)cdiv(H, 128) * T * tok_tiles, cap(cdiv(qd / T, 64)));
+    } else if (decode) {
+        const long mt = cdiv(M, 64);
+        p.qkv_splits = fit_splits(H, want_splits(mt * cdiv(qd, 64), 16), 16);
+        p.gu_splits = fit_splits(H, want_splits(mt * cdiv(F, 64), 16), 16);
+        p.down_splits = fit_splits(F, want_splits(mt * cdiv(H, 64), 16), 16);
+        p.o_per_group = fit_splits(qd / T, cdiv(want_splits(mt * cdiv(H, 64), 16), T), 16);
     }
-    p.o_groups = T;
     p.qkv_kps = H / p.qkv_splits;
     p.gu_kps = H / p.gu_splits;
     p.down_kps = F / p.down_splits;
-    p.o_kps = qd / (p.o_groups * p.o_per_group);
-    // decode attention: enough CTAs for the machine, at least 2 pages per split
+    p.o_kps = qd / (T * p.o_per_group);
+    p.attn_splits = 1;
     if (decode) {
+        // decode attention: enough CTAs for the machine, at least 2 pages per split
         long ctas = (long)M * d.n_q_heads;
         int s = (int)((2 * N_SM + ctas - 1) / ctas);
-        int pages = (max_context + d.kv_block_size - 1) / d.kv_block_size;
+        int pages = cdiv(max_context, d.kv_block_size);
         int smax = pages / 2 < 1 ? 1 : pages / 2;
         if (s > smax) s = smax;
         if (s > 32) s = 32;
-        if (s < 1) s = 1;
-        p.attn_splits = s;
-    } else p.attn_splits = 1;
+        p.attn_splits = s < 1 ? 1 : s;
+    }
     return p;
 }
 
 struct Layout {
     size_t res[2], h, q, attn, act, qkv32, proj32, gu32, part_o, part_ml, rope, err, total;
+    size_t Mcap;
 };
 
 // Sizes every region for the worse of the two regimes (prefill chunk, decode batch).
@@ -142,12 +157,13 @@ Layout make_layout(const spd_dims &d, bool any_spd)
     const size_t F = d.ffn, T = d.T, nqkv = qd + 2 * kd;
     size_t Mp = d.max_prefill_tokens, Md = d.max_batch;
     size_t Mmax = Mp > Md ? Mp : Md;
-    Plan pp = make_plan(d, (int)Mp, false, any_spd, d.max_seq_len);
-    Plan pd = make_plan(d, (int)Md, true, any_spd, d.max_seq_len);
+    Plan pp = make_plan(d, (int)Mp, false, d.max_seq_len);
+    Plan pd = make_plan(d, 1, true, d.max_seq_len); // one token gives the largest split counts
     auto mx = [](size_t a, size_t b) { return a > b ? a : b; };
     Layout L;
+    L.Mcap = Mmax;
     size_t off = 0;
-    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
     L.err = take(256);
     L.res[0] = take(Mmax * H * 4);
     L.res[1] = take(Mmax * H * 4);
@@ -157,8 +173,7 @@ Layout make_layout(const spd_dims &d, bool any_spd)
     L.act = take(Mmax * F * es);
     L.rope = take(Mmax * (d.head_dim / 2) * sizeof(float2));
     L.qkv32 = take(mx(pp.qkv_splits * Mp, pd.qkv_splits * Md) * nqkv * 4);
-    size_t o_planes_p = (size_t)pp.o_groups * pp.o_per_group, o_planes_d = (size_t)pd.o_groups * pd.o_per_group;
-    L.proj32 = take(mx(mx(o_planes_p, pp.down_splits) * Mp, mx(o_planes_d, pd.down_splits) * Md) * H * 4);
+    L.proj32 = take(mx(mx(T * pp.o_per_group, (size_t)pp.down_splits) * Mp, mx(T * pd.o_per_group, (size_t)pd.down_splits) * Md) * H * 4);
     L.gu32 = take(mx(pp.gu_splits * Mp, pd.gu_splits * Md) * 2 * F * 4);
     L.part_o = take(Md * d.n_q_heads * 32 * d.head_dim * 4);
     L.part_ml = take(Md * d.n_q_heads * 32 * 2 * 4);
@@ -181,15 +196,45 @@ int check_dims(const spd_dims *d, const uint8_t *mask)
     return SPD_OK;
 }
 
+int box_index(int box) { return box == 16 ? 0 : (box == 32 ? 1 : (box == 64 ? 2 : 3)); }
+
+// Tensor map of an activation buffer for a token box, built once.
+const TcMap *act_map(Ctx *c, ActBuf buf, int box)
+{
+    const int bi = box_index(box);
+    if (c->act_map_ready[buf][bi]) return &c->act_maps[buf][bi];
+    const spd_dims &d = c->d;
+    const long H = d.hidden, qd = (long)d.n_q_heads * d.head_dim, F = d.ffn, T = d.T, Mc = c->Mcap;
+    int rc = -1;
+    switch (buf) {
+    case AB_H: rc = make_operand_map(&c->act_maps[buf][bi], c->h, H, Mc, c->any_spd ? T : 1, H, Mc * H, box); break;
+    case AB_ATTN: rc = make_operand_map(&c->act_maps[buf][bi], c->attn, qd, Mc, 1, qd, 0, box); break;
+    case AB_ATTN_SHARD: rc = make_operand_map(&c->act_maps[buf][bi], c->attn, qd / T, Mc, T, qd, qd / T, box); break;
+    case AB_ACT: rc = make_operand_map(&c->act_maps[buf][bi], c->act, F, Mc, 1, F, 0, box); break;
+    default: break;
+    }
+    if (rc) return nullptr;
+    c->act_map_ready[buf][bi] = true;
+    return &c->act_maps[buf][bi];
+}
+
+#define MAP_OR_FAIL(var, expr)                     \
+    const TcMap *var = (expr);                     \
+    if (!var) { g_last_cuda_error = (int)cudaErrorInvalidValue; return SPD_ECUDA; }
+
 template <typename T>
 int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t *bt, int max_pages,
                bool decode, int max_context, cudaStream_t st)
 {
+    constexpr bool TC = sizeof(T) == 2; // bf16 -> tcgen05 GEMMs; float32 -> CUDA-core GEMMs
     const spd_dims &d = c->d;
     const int H = d.hidden, qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, F = d.ffn, Tn = d.T;
     const int nqkv = qd + 2 * kd;
-    const Plan p = make_plan(d, M, decode, c->any_spd, max_context);
+    const long Mc = c->Mcap;
+    const Plan p = make_plan(d, M, decode, max_context);
     PageTable pt{bt, max_pages, c->n_pages, d.kv_block_size, d.n_kv_heads};
+    const bool swap = decode;
+    const int tbox = TC ? tc_token_box(swap, M) : 0;
     int launches = 0;
 
     if (d.rope_base > 0.f) LAUNCH(K_ROPE_TABLE, launch_rope_table(c->rope, tm, M, d.head_dim, d.rope_base, st));
@@ -197,7 +242,7 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
     // block input -> fp32 residual stream and its attention RMSNorm
     {
         NormArgs a{};
-        a.x_in = x; a.res_out = c->res[0]; a.h_out = c->h; a.h_stride = (long)M * H;
+        a.x_in = x; a.res_out = c->res[0]; a.h_out = c->h; a.h_stride = Mc * H;
         a.gain = c->layers[0].attn_norm; a.n_groups = 1; a.per_group = 0; a.M = M; a.H = H; a.eps = d.rms_eps;
         LAUNCH(K_NORM, launch_residual_norm<T>(a, st));
     }
@@ -205,14 +250,26 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
         const spd_layer &w = c->layers[l];
         const bool sync = c->mask[l] != 0;
         // a2: column-split Q/K/V projections of all shards = the full matrices
-        const void *wm[3] = {w.wq, w.wk, w.wv};
-        const int wn[3] = {qd, kd, kd}, wcol[3] = {0, qd, qd + kd};
-        for (int i = 0; i < 3; ++i) {
-            GemmProblem g{};
-            g.A = c->h; g.lda = H; g.a_shard_stride = 0; g.W = wm[i]; g.ldw = H;
-            g.C = c->qkv32 + wcol[i]; g.ldc = nqkv; g.c_split_stride = (long)M * nqkv;
-            g.M = M; g.n_per_shard = wn[i]; g.n_shards = 1; g.K = H; g.splits = p.qkv_splits; g.k_per_split = p.qkv_kps;
-            LAUNCH(K_QKV, launch_gemm_simt<T>(g, st));
+        {
+            const void *wm[3] = {w.wq, w.wk, w.wv};
+            const int wn[3] = {qd, kd, kd}, wcol[3] = {0, qd, qd + kd};
+            for (int i = 0; i < 3; ++i) {
+                if (TC) {
+                    const TcMap *wmaps[3] = {&c->maps[l].wq, &c->maps[l].wk, &c->maps[l].wv};
+                    MAP_OR_FAIL(am, act_map(c, AB_H, tbox));
+                    TcGemmArgs g{};
+                    g.C = c->qkv32 + wcol[i]; g.ldc = nqkv; g.c_batch_stride = 0; g.c_split_stride = (long)M * nqkv;
+                    g.t_rows = M; g.w_rows = wn[i]; g.batches = 1; g.w_batched = 0; g.t_batched = 0;
+                    g.num_kb = cdiv(H, 64); g.splits = p.qkv_splits; g.err = c->err;
+                    LAUNCH(K_QKV, launch_gemm_tc(*wmaps[i], *am, g, swap, st));
+                } else {
+                    GemmProblem g{};
+                    g.A = c->h; g.lda = H; g.a_shard_stride = 0; g.W = wm[i]; g.ldw = H;
+                    g.C = c->qkv32 + wcol[i]; g.ldc = nqkv; g.c_split_stride = (long)M * nqkv;
+                    g.M = M; g.n_per_shard = wn[i]; g.n_shards = 1; g.K = H; g.splits = p.qkv_splits; g.k_per_split = p.qkv_kps;
+                    LAUNCH(K_QKV, launch_gemm_simt<T>(g, st));
+                }
+            }
         }
         // a3: rotary embedding, KV-page append
         {
@@ -231,11 +288,19 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
             if (decode) { LAUNCH(K_ATTN, launch_decode_attention<T>(a, st)); ++launches; }
             else LAUNCH(K_ATTN, launch_prefill_attention<T>(a, st));
         }
-        // a5: row-split output projection; plane (i, j) holds the part of Y_i from K sub-range j
-        // (a synchronous block in prefill needs only the sum: one plane over all of K)
+        // a5: row-split output projection.  Plane (i, j) holds the part of Y_i that comes from
+        // sub-range j of shard i's K slice.  A synchronous block in prefill needs only the sum:
+        // one plane over all of K.
         const bool o_single = sync && !decode;
-        const int o_planes = o_single ? 1 : p.o_groups * p.o_per_group;
-        {
+        const int o_planes = o_single ? 1 : Tn * p.o_per_group;
+        if (TC) {
+            MAP_OR_FAIL(am, act_map(c, o_single ? AB_ATTN : AB_ATTN_SHARD, tbox));
+            TcGemmArgs g{};
+            g.C = c->proj32; g.ldc = H; g.c_batch_stride = (long)p.o_per_group * M * H; g.c_split_stride = (long)M * H;
+            g.t_rows = M; g.w_rows = H; g.batches = o_single ? 1 : Tn; g.w_batched = !o_single; g.t_batched = !o_single;
+            g.num_kb = cdiv(o_single ? qd : qd / Tn, 64); g.splits = o_single ? 1 : p.o_per_group; g.err = c->err;
+            LAUNCH(K_OPROJ, launch_gemm_tc(o_single ? c->maps[l].wo_full : c->maps[l].wo_shard, *am, g, swap, st));
+        } else {
             GemmProblem g{};
             g.A = c->attn; g.lda = qd; g.W = w.wo; g.ldw = qd; g.C = c->proj32; g.ldc = H; g.c_split_stride = (long)M * H;
             g.M = M; g.n_per_shard = H; g.n_shards = 1; g.K = qd; g.splits = o_planes; g.k_per_split = o_single ? qd : p.o_kps;
@@ -246,18 +311,30 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
             NormArgs a{};
             a.res_in = c->res[0]; a.part = c->proj32; a.part_stride = (long)M * H;
             a.n_groups = sync ? 1 : Tn; a.per_group = sync ? o_planes : p.o_per_group;
-            a.res_out = c->res[1]; a.h_out = c->h; a.h_stride = (long)M * H; a.gain = w.mlp_norm;
+            a.res_out = c->res[1]; a.h_out = c->h; a.h_stride = Mc * H; a.gain = w.mlp_norm;
             a.M = M; a.H = H; a.eps = d.rms_eps;
             LAUNCH(K_NORM, launch_residual_norm<T>(a, st));
         }
         // a8: column-split gate / up; in an SPD block shard i reads its own MLP input plane
-        const void *gm[2] = {w.w_gate, w.w_up};
-        for (int i = 0; i < 2; ++i) {
-            GemmProblem g{};
-            g.A = c->h; g.lda = H; g.a_shard_stride = sync ? 0 : (long)M * H; g.W = gm[i]; g.ldw = H;
-            g.C = c->gu32 + (long)i * p.gu_splits * M * F; g.ldc = F; g.c_split_stride = (long)M * F;
-            g.M = M; g.n_per_shard = F / Tn; g.n_shards = Tn; g.K = H; g.splits = p.gu_splits; g.k_per_split = p.gu_kps;
-            LAUNCH(K_GATE_UP, launch_gemm_simt<T>(g, st));
+        {
+            const void *gm[2] = {w.w_gate, w.w_up};
+            for (int i = 0; i < 2; ++i) {
+                float *Cg = c->gu32 + (long)i * p.gu_splits * M * F;
+                if (TC) {
+                    MAP_OR_FAIL(am, act_map(c, AB_H, tbox));
+                    TcGemmArgs g{};
+                    g.C = Cg; g.ldc = F; g.c_batch_stride = F / Tn; g.c_split_stride = (long)M * F;
+                    g.t_rows = M; g.w_rows = F / Tn; g.batches = Tn; g.w_batched = 1; g.t_batched = sync ? 0 : 1;
+                    g.num_kb = cdiv(H, 64); g.splits = p.gu_splits; g.err = c->err;
+                    LAUNCH(K_GATE_UP, launch_gemm_tc(i == 0 ? c->maps[l].w_gate : c->maps[l].w_up, *am, g, swap, st));
+                } else {
+                    GemmProblem g{};
+                    g.A = c->h; g.lda = H; g.a_shard_stride = sync ? 0 : Mc * H; g.W = gm[i]; g.ldw = H;
+                    g.C = Cg; g.ldc = F; g.c_split_stride = (long)M * F;
+                    g.M = M; g.n_per_shard = F / Tn; g.n_shards = Tn; g.K = H; g.splits = p.gu_splits; g.k_per_split = p.gu_kps;
+                    LAUNCH(K_GATE_UP, launch_gemm_simt<T>(g, st));
+                }
+            }
         }
         {
             SiluMulArgs a{};
@@ -266,7 +343,14 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
             LAUNCH(K_SILU_MUL, launch_silu_mul<T>(a, st));
         }
         // a9: row-split down projection; summing over all of K = F IS the kept sync-point
-        {
+        if (TC) {
+            MAP_OR_FAIL(am, act_map(c, AB_ACT, tbox));
+            TcGemmArgs g{};
+            g.C = c->proj32; g.ldc = H; g.c_batch_stride = 0; g.c_split_stride = (long)M * H;
+            g.t_rows = M; g.w_rows = H; g.batches = 1; g.w_batched = 0; g.t_batched = 0;
+            g.num_kb = cdiv(F, 64); g.splits = p.down_splits; g.err = c->err;
+            LAUNCH(K_DOWN, launch_gemm_tc(c->maps[l].w_down, *am, g, swap, st));
+        } else {
             GemmProblem g{};
             g.A = c->act; g.lda = F; g.W = w.w_down; g.ldw = F; g.C = c->proj32; g.ldc = H; g.c_split_stride = (long)M * H;
             g.M = M; g.n_per_shard = H; g.n_shards = 1; g.K = F; g.splits = p.down_splits; g.k_per_split = p.down_kps;
@@ -278,7 +362,7 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
             NormArgs a{};
             a.res_in = c->res[1]; a.part = c->proj32; a.part_stride = (long)M * H; a.n_groups = 1; a.per_group = p.down_splits;
             a.res_out = c->res[0]; a.M = M; a.H = H; a.eps = d.rms_eps;
-            if (l + 1 < d.n_layers) { a.h_out = c->h; a.h_stride = (long)M * H; a.gain = c->layers[l + 1].attn_norm; }
+            if (l + 1 < d.n_layers) { a.h_out = c->h; a.h_stride = Mc * H; a.gain = c->layers[l + 1].attn_norm; }
             else a.final_out = out;
             LAUNCH(K_NORM, launch_residual_norm<T>(a, st));
         }
@@ -292,6 +376,28 @@ int read_err_flag(Ctx *c, cudaStream_t st, int *flag)
     CU_TRY(cudaMemcpyAsync(flag, c->err, sizeof(int), cudaMemcpyDeviceToHost, st));
     CU_TRY(cudaStreamSynchronize(st));
     if (*flag) CU_TRY(cudaMemsetAsync(c->err, 0, sizeof(int), st));
+    return SPD_OK;
+}
+
+int build_weight_maps(Ctx &c)
+{
+    const spd_dims &d = c.d;
+    const long H = d.hidden, qd = (long)d.n_q_heads * d.head_dim, kd = (long)d.n_kv_heads * d.head_dim, F = d.ffn, T = d.T;
+    c.maps.resize(d.n_layers);
+    for (int l = 0; l < d.n_layers; ++l) {
+        const spd_layer &w = c.layers[l];
+        LayerMaps &m = c.maps[l];
+        int rc = 0;
+        rc |= make_operand_map(&m.wq, w.wq, H, qd, 1, H, 0, 128);
+        rc |= make_operand_map(&m.wk, w.wk, H, kd, 1, H, 0, 128);
+        rc |= make_operand_map(&m.wv, w.wv, H, kd, 1, H, 0, 128);
+        rc |= make_operand_map(&m.wo_full, w.wo, qd, H, 1, qd, 0, 128);
+        rc |= make_operand_map(&m.wo_shard, w.wo, qd / T, H, T, qd, qd / T, 128);
+        rc |= make_operand_map(&m.w_gate, w.w_gate, H, F / T, T, H, (F / T) * H, 128);
+        rc |= make_operand_map(&m.w_up, w.w_up, H, F / T, T, H, (F / T) * H, 128);
+        rc |= make_operand_map(&m.w_down, w.w_down, F, H, 1, F, 0, 128);
+        if (rc) return SPD_EINVAL;
+    }
     return SPD_OK;
 }
 
@@ -342,6 +448,8 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     c.layers.assign(layers, layers + dims->n_layers);
     c.n_pages = n_pages;
     c.any_spd = any_spd;
+    c.Mcap = (long)L.Mcap;
+    // regions are laid out from a 1024-byte aligned base inside the caller's buffer
     c.ws = (char *)workspace;
     c.ws_bytes = workspace_bytes;
     c.err = (int *)(c.ws + L.err);
@@ -354,7 +462,13 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     c.launches_last = 0;
     c.profiling = false;
     c.ev_used = 0;
-    cudaError_t e = cudaMemset(c.err, 0, 256);
+    memset(c.act_map_ready, 0, sizeof(c.act_map_ready));
+    if (dims->dtype == 1) {
+        rc = build_weight_maps(c);
+        if (rc) { delete h; return rc; }
+    }
+    // zero the workspace once: token rows beyond a launch's M are read (never used) by tiled loads
+    cudaError_t e = cudaMemset(workspace, 0, L.total);
     if (e != cudaSuccess) { g_last_cuda_error = (int)e; delete h; return SPD_ECUDA; }
     *out = h;
     return SPD_OK;
@@ -409,6 +523,23 @@ int spd_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_l
     TokMap tm{1, 0, 1, 0, seq_lens};
     return d.dtype == 0 ? run_tokens<float>(&c, x, out, B, tm, block_table, max_pages, true, max_context, st)
                         : run_tokens<bf16>(&c, x, out, B, tm, block_table, max_pages, true, max_context, st);
+}
+
+int spd_gemm_bf16(const void *a, const void *w, float *c, int32_t M, int32_t N, int32_t K, int32_t batches,
+                  int32_t a_batched, int32_t splits, int32_t swap, int32_t *err_flag, void *stream)
+{
+    if (!a || !w || !c || !err_flag) return SPD_ENULL;
+    if (M < 1 || N < 1 || K < 8 || K % 8 || batches < 1 || splits < 1 || splits > (K + 63) / 64) return SPD_EINVAL;
+    TcMap wm, am;
+    const int tbox = tc_token_box(swap != 0, M);
+    if (make_operand_map(&wm, w, K, N, batches, K, (long)N * K, 128)) return SPD_EINVAL;
+    if (make_operand_map(&am, a, K, M, a_batched ? batches : 1, K, (long)M * K, tbox)) return SPD_EINVAL;
+    TcGemmArgs g{};
+    g.C = c; g.ldc = (long)batches * N; g.c_batch_stride = N; g.c_split_stride = (long)M * batches * N;
+    g.t_rows = M; g.w_rows = N; g.batches = batches; g.w_batched = batches > 1; g.t_batched = a_batched && batches > 1;
+    g.num_kb = (K + 63) / 64; g.splits = splits; g.err = err_flag;
+    CU_TRY(launch_gemm_tc(wm, am, g, swap != 0, (cudaStream_t)stream));
+    return SPD_OK;
 }
 
 int spd_sync_points(const spd_ctx *ctx)

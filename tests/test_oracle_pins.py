@@ -51,6 +51,12 @@ def test_rmsnorm_matches_torch_library():
     assert rel_err(oracle.rmsnorm(x, g, 1e-5), ref) < 1e-14
 
 
+def test_linear_matches_numpy_matmul():
+    rng = np.random.default_rng(0)
+    x, w = rng.standard_normal((5, 37)), rng.standard_normal((11, 37)).astype(np.float32)
+    assert rel_err(oracle.linear(x, w), x @ w.astype(np.float64).T) < 1e-14
+
+
 def test_rope_is_a_rotation_by_pos_times_theta():
     d, base = 8, 10000.0
     v = np.arange(1.0, d + 1.0)
