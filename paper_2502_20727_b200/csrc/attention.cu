@@ -105,91 +105,214 @@ template <typename T> cudaError_t launch_prefill_attention(const AttnArgs &a, cu
 template cudaError_t launch_prefill_attention<float>(const AttnArgs &, cudaStream_t);
 template cudaError_t launch_prefill_attention<bf16>(const AttnArgs &, cudaStream_t);
 
-// Decode: grid (n_q_heads, B, splits); the 4 warps of a CTA interleave the tokens of the
-// split's range, then merge through shared memory; splits are merged by the next kernel.
-template <typename T, int VEC>
+// ---------------------------------------------------------------------------------------
+// Paged decode attention: one query token per sequence.
+// grid (n_q_heads / GT, B, splits).  A CTA serves GT query heads that share one KV head
+// (grouped-query attention reads each K/V row once for the whole tile) over one slice of the
+// context.  Every K/V row is fetched with 16-byte loads, LPT = row_bytes / 16 lanes per token,
+// so a warp instruction covers TPW = 32 / LPT whole rows; NG such instructions per operand are
+// issued back to back before any arithmetic.  Scores are reduced with warp shuffles, the
+// softmax is the online form per token slot, slots / warps / splits are merged at the end
+// (the last CTA of a (sequence, head tile) to finish merges the splits, in a fixed order).
+template <typename T> struct Row16;
+template <> struct Row16<float> {
+    static constexpr int E = 4;
+    static __device__ __forceinline__ void cvt(const uint4 &u, float *o)
+    { o[0] = __uint_as_float(u.x); o[1] = __uint_as_float(u.y); o[2] = __uint_as_float(u.z); o[3] = __uint_as_float(u.w); }
+};
+template <> struct Row16<bf16> {
+    static constexpr int E = 8;
+    static __device__ __forceinline__ void cvt(const uint4 &u, float *o)
+    {
+        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { o[2 * i] = __uint_as_float(w[i] << 16); o[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
+    }
+};
+
+template <typename T, int D, int GT>
 __global__ void __launch_bounds__(128) decode_attention_kernel(AttnArgs a)
 {
-    const int d = 32 * VEC, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int hq = blockIdx.x, b = blockIdx.y, sp = blockIdx.z;
-    __shared__ float sm_o[4][32 * VEC];
-    __shared__ float sm_ml[4][2];
+    constexpr int E = Row16<T>::E, LPT = D / E, TPW = 32 / LPT, NG = 8, CHUNK = NG * TPW;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int slot = lane / LPT, li = lane % LPT;
+    const int hq0 = blockIdx.x * GT, b = blockIdx.y, sp = blockIdx.z;
+    const int kvh = hq0 / (a.n_q_heads / a.pt.n_kv_heads);
+    __shared__ float sm_o[4][GT][D];
+    __shared__ float sm_ml[4][GT][2];
+    __shared__ int sm_last;
+
     const int ctx = a.tm.seq_lens[b] + 1;
-    float *po = a.part_o + (((long)b * a.n_q_heads + hq) * a.splits + sp) * d;
-    float *pml = a.part_ml + (((long)b * a.n_q_heads + hq) * a.splits + sp) * 2;
-    const bool bad = ctx > a.max_context || (ctx - 1) / a.pt.block >= a.pt.max_pages || ctx < 1;
-    // tokens per split, rounded to whole pages
+    const bool bad = ctx < 1 || ctx > a.max_context || (ctx - 1) / a.pt.block >= a.pt.max_pages;
     int per = (a.max_context + a.splits - 1) / a.splits;
-    per = (per + a.pt.block - 1) / a.pt.block * a.pt.block;
-    const int t0 = sp * per, t1 = min(ctx, t0 + per);
-    if (bad || t0 >= t1) {
-        if (bad && threadIdx.x == 0) atomicOr(a.err, ERR_CAPACITY);
-        for (int i = threadIdx.x; i < d; i += blockDim.x) po[i] = 0.f;
-        if (threadIdx.x == 0) { pml[0] = -INFINITY; pml[1] = 0.f; }
-        return;
+    per = (per + CHUNK - 1) / CHUNK * CHUNK;
+    const int t0 = sp * per, t1 = bad ? t0 : min(ctx, t0 + per);
+    if (bad && threadIdx.x == 0) atomicOr(a.err, ERR_CAPACITY);
+
+    // query tile, pre-scaled so that the softmax can use exp2
+    float q[GT][E];
+    {
+        const float sc = rsqrtf((float)D) * 1.4426950408889634f;
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+            const T *qp = (const T *)a.q + ((long)b * a.n_q_heads + hq0 + g) * D + li * E;
+            uint4 u = *(const uint4 *)qp;
+            Row16<T>::cvt(u, q[g]);
+#pragma unroll
+            for (int e = 0; e < E; ++e) q[g][e] *= sc;
+        }
     }
-    const int kvh = hq / (a.n_q_heads / a.pt.n_kv_heads);
-    float q[VEC], o[VEC];
-    VecLoad<T, VEC>::ld((const T *)a.q + ((long)b * a.n_q_heads + hq) * d + lane * VEC, q);
+    float mx[GT], den[GT], o[GT][E];
 #pragma unroll
-    for (int i = 0; i < VEC; ++i) o[i] = 0.f;
-    float mx = -INFINITY, den = 0.f;
-    const float scale = rsqrtf((float)d);
-    // warp w takes pages w, w+4, ... of the range
-    for (int p0 = t0 + warp * a.pt.block; p0 < t1; p0 += 4 * a.pt.block)
-        attend_range<T, VEC>(q, (const T *)a.k_pages, (const T *)a.v_pages, a.pt, b, kvh, p0,
-                             min(t1, p0 + a.pt.block), scale, mx, den, o, a.err);
+    for (int g = 0; g < GT; ++g) {
+        mx[g] = -INFINITY; den[g] = 0.f;
 #pragma unroll
-    for (int i = 0; i < VEC; ++i) sm_o[warp][lane * VEC + i] = o[i];
-    if (lane == 0) { sm_ml[warp][0] = mx; sm_ml[warp][1] = den; }
+        for (int e = 0; e < E; ++e) o[g][e] = 0.f;
+    }
+    const T *kp = (const T *)a.k_pages, *vp = (const T *)a.v_pages;
+    for (int c0 = t0 + warp * CHUNK; c0 < t1; c0 += 4 * CHUNK) {
+        uint4 kr[NG], vr[NG];
+        bool valid[NG];
+#pragma unroll
+        for (int i = 0; i < NG; ++i) {
+            const int t = c0 + i * TPW + slot;
+            valid[i] = t < t1;
+            kr[i] = make_uint4(0, 0, 0, 0);
+            vr[i] = make_uint4(0, 0, 0, 0);
+            if (valid[i]) {
+                int page = a.pt.block_table[(long)b * a.pt.max_pages + t / a.pt.block];
+                if (page < 0 || page >= a.pt.n_pages) { atomicOr(a.err, ERR_PAGE_RANGE); page = 0; }
+                const long row = (((long)page * a.pt.n_kv_heads + kvh) * a.pt.block + t % a.pt.block) * D + li * E;
+                kr[i] = *(const uint4 *)(kp + row);
+                vr[i] = *(const uint4 *)(vp + row);
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+            float s[NG], cmax = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < NG; ++i) {
+                float kf[E], acc = 0.f;
+                Row16<T>::cvt(kr[i], kf);
+#pragma unroll
+                for (int e = 0; e < E; ++e) acc = fmaf(q[g][e], kf[e], acc);
+#pragma unroll
+                for (int off = LPT / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+                s[i] = valid[i] ? acc : -INFINITY;
+                cmax = fmaxf(cmax, s[i]);
+            }
+            const float nm = fmaxf(mx[g], cmax);
+            if (nm == -INFINITY) continue; // nothing valid in this slot so far
+            const float corr = exp2f(mx[g] - nm);
+            mx[g] = nm;
+            den[g] *= corr;
+#pragma unroll
+            for (int e = 0; e < E; ++e) o[g][e] *= corr;
+#pragma unroll
+            for (int i = 0; i < NG; ++i) {
+                const float p = exp2f(s[i] - nm); // 0 for masked tokens
+                den[g] += p;
+                float vf[E];
+                Row16<T>::cvt(vr[i], vf);
+#pragma unroll
+                for (int e = 0; e < E; ++e) o[g][e] = fmaf(p, vf[e], o[g][e]);
+            }
+        }
+    }
+    // merge the token slots of the warp
+#pragma unroll
+    for (int off = LPT; off < 32; off <<= 1) {
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+            const float om = __shfl_xor_sync(0xffffffffu, mx[g], off), od = __shfl_xor_sync(0xffffffffu, den[g], off);
+            const float nm = fmaxf(mx[g], om);
+            const float ca = (mx[g] == -INFINITY) ? 0.f : exp2f(mx[g] - nm), cb = (om == -INFINITY) ? 0.f : exp2f(om - nm);
+            den[g] = den[g] * ca + od * cb;
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                const float oo = __shfl_xor_sync(0xffffffffu, o[g][e], off);
+                o[g][e] = o[g][e] * ca + oo * cb;
+            }
+            mx[g] = nm;
+        }
+    }
+    if (slot == 0) {
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+#pragma unroll
+            for (int e = 0; e < E; ++e) sm_o[warp][g][li * E + e] = o[g][e];
+            if (li == 0) { sm_ml[warp][g][0] = mx[g]; sm_ml[warp][g][1] = den[g]; }
+        }
+    }
     __syncthreads();
-    float gm = fmaxf(fmaxf(sm_ml[0][0], sm_ml[1][0]), fmaxf(sm_ml[2][0], sm_ml[3][0]));
-    float gden = 0.f;
+    // merge the 4 warps; thread -> (head of the tile, dim)
+    const long pbase = ((long)b * a.n_q_heads + hq0) * a.splits + sp;
+    for (int idx = threadIdx.x; idx < GT * D; idx += blockDim.x) {
+        const int g = idx / D, dd = idx % D;
+        float gm = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < 4; ++w) gden += sm_ml[w][1] * ((sm_ml[w][0] == -INFINITY) ? 0.f : __expf(sm_ml[w][0] - gm));
-    for (int i = threadIdx.x; i < d; i += blockDim.x) {
-        float acc = 0.f;
+        for (int w = 0; w < 4; ++w) gm = fmaxf(gm, sm_ml[w][g][0]);
+        float acc = 0.f, gden = 0.f;
 #pragma unroll
-        for (int w = 0; w < 4; ++w) acc += sm_o[w][i] * ((sm_ml[w][0] == -INFINITY) ? 0.f : __expf(sm_ml[w][0] - gm));
-        po[i] = acc; // un-normalised
+        for (int w = 0; w < 4; ++w) {
+            const float c = (sm_ml[w][g][0] == -INFINITY) ? 0.f : exp2f(sm_ml[w][g][0] - gm);
+            acc += sm_o[w][g][dd] * c;
+            gden += sm_ml[w][g][1] * c;
+        }
+        if (a.splits == 1) {
+            ((T *)a.out)[((long)b * a.n_q_heads + hq0 + g) * D + dd] = from_f<T>(gden > 0.f ? acc / gden : 0.f);
+        } else {
+            const long pi = pbase + (long)g * a.splits;
+            a.part_o[pi * D + dd] = acc; // un-normalised
+            if (dd == 0) { a.part_ml[pi * 2] = gm; a.part_ml[pi * 2 + 1] = gden; }
+        }
     }
-    if (threadIdx.x == 0) { pml[0] = gm; pml[1] = gden; }
+    if (a.splits == 1) return;
+    // the last CTA of this (sequence, head tile) to arrive merges the splits
+    __threadfence();
+    __syncthreads();
+    int *cnt = a.counters + (long)b * gridDim.x + blockIdx.x;
+    if (threadIdx.x == 0) sm_last = (atomicAdd(cnt, 1) == a.splits - 1);
+    __syncthreads();
+    if (!sm_last) return;
+    __threadfence();
+    for (int idx = threadIdx.x; idx < GT * D; idx += blockDim.x) {
+        const int g = idx / D, dd = idx % D;
+        const long p0 = ((long)b * a.n_q_heads + hq0 + g) * a.splits;
+        float gm = -INFINITY;
+        for (int s2 = 0; s2 < a.splits; ++s2) gm = fmaxf(gm, __ldcg(a.part_ml + (p0 + s2) * 2));
+        float acc = 0.f, gden = 0.f;
+        for (int s2 = 0; s2 < a.splits; ++s2) {
+            const float m2 = __ldcg(a.part_ml + (p0 + s2) * 2);
+            const float c = (m2 == -INFINITY) ? 0.f : exp2f(m2 - gm);
+            acc += __ldcg(a.part_o + (p0 + s2) * D + dd) * c;
+            gden += __ldcg(a.part_ml + (p0 + s2) * 2 + 1) * c;
+        }
+        ((T *)a.out)[((long)b * a.n_q_heads + hq0 + g) * D + dd] = from_f<T>(gden > 0.f ? acc / gden : 0.f);
+    }
+    if (threadIdx.x == 0) *cnt = 0; // ready for the next launch
 }
 
-// grid (n_q_heads, B): combine the splits' (max, denominator, numerator) triples.
-template <typename T> __global__ void decode_merge_kernel(AttnArgs a)
+template <typename T, int D> cudaError_t launch_decode_d(const AttnArgs &a, cudaStream_t st)
 {
-    const int hq = blockIdx.x, b = blockIdx.y, d = a.head_dim;
-    const float *po = a.part_o + (((long)b * a.n_q_heads + hq) * a.splits) * d;
-    const float *pml = a.part_ml + (((long)b * a.n_q_heads + hq) * a.splits) * 2;
-    float gm = -INFINITY;
-    for (int s = 0; s < a.splits; ++s) gm = fmaxf(gm, pml[2 * s]);
-    float den = 0.f;
-    for (int s = 0; s < a.splits; ++s)
-        if (pml[2 * s] != -INFINITY) den += pml[2 * s + 1] * __expf(pml[2 * s] - gm);
-    T *out = (T *)a.out + ((long)b * a.n_q_heads + hq) * d;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) {
-        float acc = 0.f;
-        for (int s = 0; s < a.splits; ++s)
-            if (pml[2 * s] != -INFINITY) acc += po[(long)s * d + i] * __expf(pml[2 * s] - gm);
-        out[i] = from_f<T>(den > 0.f ? acc / den : 0.f);
-    }
+    const int group = a.n_q_heads / a.pt.n_kv_heads;
+    const int gt = (group % 4 == 0) ? 4 : ((group % 2 == 0) ? 2 : 1);
+    dim3 grid(a.n_q_heads / gt, a.B, a.splits);
+    if (gt == 4) decode_attention_kernel<T, D, 4><<<grid, 128, 0, st>>>(a);
+    else if (gt == 2) decode_attention_kernel<T, D, 2><<<grid, 128, 0, st>>>(a);
+    else decode_attention_kernel<T, D, 1><<<grid, 128, 0, st>>>(a);
+    return cudaGetLastError();
 }
 
 template <typename T> cudaError_t launch_decode_attention(const AttnArgs &a, cudaStream_t st)
 {
     if (a.B <= 0) return cudaSuccess;
-    dim3 grid(a.n_q_heads, a.B, a.splits);
     switch (a.head_dim) {
-    case 128: decode_attention_kernel<T, 4><<<grid, 128, 0, st>>>(a); break;
-    case 64: decode_attention_kernel<T, 2><<<grid, 128, 0, st>>>(a); break;
-    case 32: decode_attention_kernel<T, 1><<<grid, 128, 0, st>>>(a); break;
+    case 128: return launch_decode_d<T, 128>(a, st);
+    case 64: return launch_decode_d<T, 64>(a, st);
+    case 32: return launch_decode_d<T, 32>(a, st);
     default: return cudaErrorInvalidValue;
     }
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    decode_merge_kernel<T><<<dim3(a.n_q_heads, a.B), a.head_dim >= 64 ? 64 : 32, 0, st>>>(a);
-    return cudaGetLastError();
 }
 template cudaError_t launch_decode_attention<float>(const AttnArgs &, cudaStream_t);
 template cudaError_t launch_decode_attention<bf16>(const AttnArgs &, cudaStream_t);

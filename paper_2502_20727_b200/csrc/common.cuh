@@ -126,6 +126,7 @@ struct AttnArgs {
     int B, splits, max_context;
     float *part_o;          // fp32 [B][nq][splits][d]
     float *part_ml;         // fp32 [B][nq][splits][2]
+    int *counters;          // [B][nq] zero-initialised arrival counters (split merge)
     int *err;
 };
 template <typename T> cudaError_t launch_prefill_attention(const AttnArgs &a, cudaStream_t st);

@@ -18,69 +18,93 @@ __device__ __forceinline__ float block_sum(float v, float *red)
     return warp_sum(t);
 }
 
-template <typename T> __device__ __forceinline__ float base_value(const NormArgs &a, long idx)
+template <typename T> __device__ __forceinline__ float4 load4(const T *p);
+template <> __device__ __forceinline__ float4 load4<float>(const float *p) { return *(const float4 *)p; }
+template <> __device__ __forceinline__ float4 load4<bf16>(const bf16 *p)
 {
-    return a.x_in ? to_f<T>(((const T *)a.x_in)[idx]) : a.res_in[idx];
+    uint2 v = *(const uint2 *)p;
+    float2 a = __bfloat1622float2(*(const __nv_bfloat162 *)&v.x), b = __bfloat1622float2(*(const __nv_bfloat162 *)&v.y);
+    return make_float4(a.x, a.y, b.x, b.y);
+}
+template <typename T> __device__ __forceinline__ void store4(T *p, float4 v);
+template <> __device__ __forceinline__ void store4<float>(float *p, float4 v) { *(float4 *)p = v; }
+template <> __device__ __forceinline__ void store4<bf16>(bf16 *p, float4 v)
+{
+    __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+    uint2 u;
+    u.x = *(uint32_t *)&a;
+    u.y = *(uint32_t *)&b;
+    *(uint2 *)p = u;
 }
 
-__device__ __forceinline__ float group_sum(const NormArgs &a, int g, long idx)
+__device__ __forceinline__ float4 f4add(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
+
+__device__ __forceinline__ float4 group_sum4(const NormArgs &a, int g, long idx)
 {
-    float y = 0.f;
-    for (int p = 0; p < a.per_group; ++p) y += a.part[(long)(g * a.per_group + p) * a.part_stride + idx];
-    return y;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (a.part)
+        for (int p = 0; p < a.per_group; ++p)
+            acc = f4add(acc, *(const float4 *)(a.part + (long)(g * a.per_group + p) * a.part_stride + idx));
+    return acc;
 }
 
-// One CTA per token row.
+// One CTA per token row; float4 column chunks.
 //   res_out  = base + sum over ALL partial planes   (base = x_in or res_in; res_out != res_in)
 //   h_out[g] = rmsnorm(base + sum of group g's planes) * gain
 // n_groups == 1 is the synchronous block's "all-reduce, residual add, norm"; n_groups == T is
 // the SPD block, where shard g only ever sees its own partial attention output Y_g while the
-// residual carried to the block output still collects every Y_g.
+// residual carried to the block output still collects every Y_g.  The second pass re-reads the
+// planes (cache resident) instead of holding T x hidden values in registers.
 template <typename T>
-__global__ void __launch_bounds__(256) residual_norm_kernel(NormArgs a)
+__global__ void __launch_bounds__(512) residual_norm_kernel(NormArgs a)
 {
     __shared__ float red[32];
-    const int m = blockIdx.x, H = a.H, G = a.n_groups;
+    const int m = blockIdx.x, H = a.H, G = a.n_groups, H4 = H >> 2;
     float ss[MAX_T];
 #pragma unroll
     for (int g = 0; g < MAX_T; ++g) ss[g] = 0.f;
-
-    for (int j = threadIdx.x; j < H; j += blockDim.x) {
-        const long idx = (long)m * H + j;
-        float base = base_value<T>(a, idx), tot = 0.f;
+    for (int c = threadIdx.x; c < H4; c += blockDim.x) {
+        const long idx = (long)m * H + 4 * c;
+        const float4 base = a.x_in ? load4<T>((const T *)a.x_in + idx) : *(const float4 *)(a.res_in + idx);
+        float4 tot = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int g = 0; g < MAX_T; ++g)
-            if (g < G) {
-                float y = a.part ? group_sum(a, g, idx) : 0.f;
-                tot += y;
-                ss[g] += (base + y) * (base + y);
-            }
-        float r_all = base + tot;
-        if (a.res_out) a.res_out[idx] = r_all;
-        if (a.final_out) ((T *)a.final_out)[idx] = from_f<T>(r_all);
+        for (int g = 0; g < MAX_T; ++g) {
+            if (g >= G) continue;
+            const float4 y = group_sum4(a, g, idx);
+            tot = f4add(tot, y);
+            const float4 r = f4add(base, y);
+            ss[g] += r.x * r.x + r.y * r.y + r.z * r.z + r.w * r.w;
+        }
+        const float4 r = f4add(base, tot);
+        if (a.res_out) *(float4 *)(a.res_out + idx) = r;
+        if (a.final_out) store4<T>((T *)a.final_out + idx, r);
     }
     if (!a.h_out) return;
     float rs[MAX_T];
 #pragma unroll
     for (int g = 0; g < MAX_T; ++g) rs[g] = (g < G) ? rsqrtf(block_sum(ss[g], red) / (float)H + a.eps) : 0.f;
-    // second pass re-reads the row (L1/L2 resident)
     const T *gain = (const T *)a.gain;
-    for (int j = threadIdx.x; j < H; j += blockDim.x) {
-        const long idx = (long)m * H + j;
-        float base = base_value<T>(a, idx), gj = to_f<T>(gain[j]);
+    for (int c = threadIdx.x; c < H4; c += blockDim.x) {
+        const long idx = (long)m * H + 4 * c;
+        const float4 base = a.x_in ? load4<T>((const T *)a.x_in + idx) : *(const float4 *)(a.res_in + idx);
+        const float4 gj = load4<T>(gain + 4 * c);
 #pragma unroll
-        for (int g = 0; g < MAX_T; ++g)
-            if (g < G) {
-                float y = a.part ? group_sum(a, g, idx) : 0.f;
-                ((T *)a.h_out)[(long)g * a.h_stride + idx] = from_f<T>((base + y) * rs[g] * gj);
-            }
+        for (int g = 0; g < MAX_T; ++g) {
+            if (g >= G) continue;
+            const float4 r = f4add(base, group_sum4(a, g, idx));
+            store4<T>((T *)a.h_out + (long)g * a.h_stride + idx,
+                      make_float4(r.x * rs[g] * gj.x, r.y * rs[g] * gj.y, r.z * rs[g] * gj.z, r.w * rs[g] * gj.w));
+        }
     }
 }
 
 template <typename T> cudaError_t launch_residual_norm(const NormArgs &a, cudaStream_t st)
 {
     if (a.M <= 0) return cudaSuccess;
-    residual_norm_kernel<T><<<a.M, 256, 0, st>>>(a);
+    if (a.H % 4 || a.n_groups > MAX_T) return cudaErrorInvalidValue;
+    const int h4 = a.H / 4;
+    const int threads = h4 >= 512 ? 512 : (h4 + 31) / 32 * 32;
+    residual_norm_kernel<T><<<a.M, threads, 0, st>>>(a);
     return cudaGetLastError();
 }
 template cudaError_t launch_residual_norm<float>(const NormArgs &, cudaStream_t);

@@ -114,8 +114,9 @@ template <int BN> struct Cfg {
 };
 
 template <int BN, bool SWAP>
-__global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a,
-                                                      const __grid_constant__ CUtensorMap tm_b, TcGemmArgs g)
+__global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_w0, const __grid_constant__ CUtensorMap tm_w1,
+                                                      const __grid_constant__ CUtensorMap tm_w2,
+                                                      const __grid_constant__ CUtensorMap tm_t, TcGemmArgs g)
 {
     using C = Cfg<BN>;
     extern __shared__ uint8_t smem_raw[];
@@ -130,8 +131,13 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // tile coordinates: x -> (batch z, weight tile), y -> token tile, z -> split
+    // (a launch may cover up to three weight matrices that share the token operand: Q|K|V, gate|up)
     const int z = blockIdx.x / g.w_tiles_per_batch;
-    const int w_row0 = (blockIdx.x % g.w_tiles_per_batch) * (SWAP ? BM : BN);
+    const int wt = blockIdx.x % g.w_tiles_per_batch;
+    const int wi = (wt >= g.tile_start[2]) ? 2 : ((wt >= g.tile_start[1]) ? 1 : 0);
+    const CUtensorMap *tm_w = wi == 0 ? &tm_w0 : (wi == 1 ? &tm_w1 : &tm_w2);
+    const int w_rows = g.w_rows[wi];
+    const int w_row0 = (wt - g.tile_start[wi]) * (SWAP ? BM : BN);
     const int t_row0 = blockIdx.y * (SWAP ? BN : BM);
     const int split = blockIdx.z;
     const int kb_begin = (int)((long)g.num_kb * split / g.splits);
@@ -143,8 +149,8 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
         mbar_init(tmem_full_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_a) : "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_b) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(tm_w) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_t) : "memory");
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::TMEM_COLS) : "memory");
@@ -168,8 +174,8 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
             mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
             const uint32_t sa = base + s * C::STAGE_BYTES, sb = sa + C::A_BYTES;
             const int kx = (kb_begin + i) * BK;
-            tma_load_3d(sa, &tm_a, kx, a_row0, a_z, full_bar(s));
-            tma_load_3d(sb, &tm_b, kx, b_row0, b_z, full_bar(s));
+            tma_load_3d(sa, SWAP ? tm_w : &tm_t, kx, a_row0, a_z, full_bar(s));
+            tma_load_3d(sb, SWAP ? &tm_t : tm_w, kx, b_row0, b_z, full_bar(s));
         }
     } else if (warp == 1 && lane == 0) {
         // MMA issuer
@@ -196,7 +202,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
     const bool acc_ok = (n_kb > 0) && mbar_wait(tmem_full_bar, 0, g.err, abort_flag);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     __syncwarp();
-    float *Cz = g.C + (long)z * g.c_batch_stride + (long)split * g.c_split_stride;
+    float *Cz = g.C + g.c_off[wi] + (long)z * g.c_batch_stride + (long)split * g.c_split_stride;
     const int row = warp * 32 + lane; // accumulator row = TMEM lane
 #pragma unroll 1
     for (int c0 = 0; c0 < BN; c0 += 16) {
@@ -209,7 +215,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
         if (SWAP) {
             // row = weight row n, columns = tokens m
             const int n = w_row0 + row;
-            if (n < g.w_rows) {
+            if (n < w_rows) {
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     const int m = t_row0 + c0 + j;
@@ -221,13 +227,13 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
             const int m = t_row0 + row;
             if (m < g.t_rows) {
                 float *dst = Cz + (long)m * g.ldc + w_row0 + c0;
-                if (w_row0 + c0 + 16 <= g.w_rows && ((((uintptr_t)dst) & 15) == 0)) {
+                if (w_row0 + c0 + 16 <= w_rows && ((((uintptr_t)dst) & 15) == 0)) {
 #pragma unroll
                     for (int j = 0; j < 16; j += 4) *(float4 *)(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
                 } else {
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        if (w_row0 + c0 + j < g.w_rows) dst[j] = v[j];
+                        if (w_row0 + c0 + j < w_rows) dst[j] = v[j];
                 }
             }
         }
@@ -255,7 +261,8 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
-template <int BN, bool SWAP> cudaError_t launch_cfg(const CUtensorMap &ta, const CUtensorMap &tb, const TcGemmArgs &g, dim3 grid, cudaStream_t st)
+template <int BN, bool SWAP>
+cudaError_t launch_cfg(const CUtensorMap *const *tw, const CUtensorMap &tt, const TcGemmArgs &g, dim3 grid, cudaStream_t st)
 {
     using C = Cfg<BN>;
     static bool attr_done = false;
@@ -264,7 +271,7 @@ template <int BN, bool SWAP> cudaError_t launch_cfg(const CUtensorMap &ta, const
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    gemm_tc_kernel<BN, SWAP><<<grid, 128, C::SMEM_BYTES, st>>>(ta, tb, g);
+    gemm_tc_kernel<BN, SWAP><<<grid, 128, C::SMEM_BYTES, st>>>(*tw[0], *tw[1], *tw[2], tt, g);
     return cudaGetLastError();
 }
 
@@ -295,26 +302,41 @@ int tc_token_box(bool swap, int tokens)
 }
 int tc_weight_box(bool swap) { return BM; }
 
-cudaError_t launch_gemm_tc(const TcMap &weights, const TcMap &tokens, const TcGemmArgs &g, bool swap, cudaStream_t st)
+cudaError_t launch_gemm_tc(const TcMap *const *weights, int n_weights, const TcMap &tokens, const TcGemmArgs &g,
+                           bool swap, cudaStream_t st)
 {
-    if (g.t_rows <= 0 || g.w_rows <= 0) return cudaSuccess;
+    if (n_weights < 1 || n_weights > 3) return cudaErrorInvalidValue;
+    if (g.t_rows <= 0) return cudaSuccess;
     if (g.splits < 1 || g.splits > g.num_kb) return cudaErrorInvalidValue;
-    const CUtensorMap &tw = *(const CUtensorMap *)&weights, &tt = *(const CUtensorMap *)&tokens;
+    const CUtensorMap *tw[3];
+    for (int i = 0; i < 3; ++i) tw[i] = (const CUtensorMap *)weights[i < n_weights ? i : 0];
+    const CUtensorMap &tt = *(const CUtensorMap *)&tokens;
+    const int w_tile = swap ? BM : 128;
+    TcGemmArgs a = g;
+    int tiles = 0;
+    for (int i = 0; i < 3; ++i) {
+        a.tile_start[i] = tiles;
+        if (i < n_weights) {
+            if (g.w_rows[i] <= 0) return cudaErrorInvalidValue;
+            tiles += (g.w_rows[i] + w_tile - 1) / w_tile;
+        } else {
+            a.tile_start[i] = 1 << 30; // never selected
+            a.w_rows[i] = 0;
+            a.c_off[i] = 0;
+        }
+    }
+    a.w_tiles_per_batch = tiles;
     if (swap) {
         const int bn = tc_token_box(true, g.t_rows);
-        TcGemmArgs a = g;
-        a.w_tiles_per_batch = (g.w_rows + BM - 1) / BM;
-        dim3 grid(a.w_tiles_per_batch * g.batches, (g.t_rows + bn - 1) / bn, g.splits);
+        dim3 grid(tiles * g.batches, (g.t_rows + bn - 1) / bn, g.splits);
         switch (bn) {
         case 16: return launch_cfg<16, true>(tw, tt, a, grid, st);
         case 32: return launch_cfg<32, true>(tw, tt, a, grid, st);
         default: return launch_cfg<64, true>(tw, tt, a, grid, st);
         }
     }
-    TcGemmArgs a = g;
-    a.w_tiles_per_batch = (g.w_rows + 127) / 128;
-    dim3 grid(a.w_tiles_per_batch * g.batches, (g.t_rows + BM - 1) / BM, g.splits);
-    return launch_cfg<128, false>(tt, tw, a, grid, st);
+    dim3 grid(tiles * g.batches, (g.t_rows + BM - 1) / BM, g.splits);
+    return launch_cfg<128, false>(tw, tt, a, grid, st);
 }
 
 } // namespace spd

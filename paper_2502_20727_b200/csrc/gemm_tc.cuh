@@ -7,20 +7,24 @@ namespace spd {
 // A CUtensorMap kept opaque so that callers need not include the driver header.
 struct alignas(64) TcMap { unsigned long long opaque[16]; };
 
+// One launch covers up to three weight matrices that share the token operand (Q|K|V, gate|up).
 struct TcGemmArgs {
     float *C;             // fp32 output
+    long c_off[3];        // element offset of weight i's output inside C (column or plane offset)
     long ldc;             // elements between token rows of C
     long c_batch_stride;  // elements added per batch z (a column offset or a plane offset)
     long c_split_stride;  // elements between K-split planes
     int t_rows;           // valid token rows
-    int w_rows;           // valid weight rows per batch
+    int w_rows[3];        // valid rows per batch of weight i
     int batches;          // z extent
-    int w_batched;        // weight operand has a batch dimension
+    int w_batched;        // weight operands have a batch dimension
     int t_batched;        // token operand has a batch dimension
     int num_kb;           // 64-wide K blocks per batch (ceil)
     int splits;           // K splits, <= num_kb
-    int w_tiles_per_batch; // filled by the launcher
     int *err;             // device error flag
+    // filled by the launcher
+    int w_tiles_per_batch;
+    int tile_start[3];
 };
 
 // Encode rows x k_inner bf16 (row stride ld_elems), `batches` of them batch_stride_elems apart.
@@ -33,6 +37,7 @@ int tc_token_box(bool swap, int tokens);
 int tc_weight_box(bool swap);
 
 // swap = weights on the 128-row MMA side (decode); otherwise tokens on it (prefill).
-cudaError_t launch_gemm_tc(const TcMap &weights, const TcMap &tokens, const TcGemmArgs &g, bool swap, cudaStream_t st);
+cudaError_t launch_gemm_tc(const TcMap *const *weights, int n_weights, const TcMap &tokens, const TcGemmArgs &g,
+                           bool swap, cudaStream_t st);
 
 } // namespace spd

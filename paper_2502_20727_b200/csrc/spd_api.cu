@@ -69,7 +69,7 @@ struct Ctx {
     void *h, *q, *attn, *act;
     float *qkv32, *proj32, *gu32, *part_o, *part_ml;
     float2 *rope;
-    int *err;
+    int *err, *attn_cnt;
     int launches_last;
     // activation tensor maps, by buffer and token box (16, 32, 64, 128), built on first use
     TcMap act_maps[AB_COUNT][4];
@@ -115,8 +115,8 @@ Plan make_plan(const spd_dims &d, int M, bool decode, int max_context)
         // tcgen05 path: 128-row weight tiles, 64-wide K blocks, uneven splits allowed, >= 4 blocks each
         const int tok_tiles = cdiv(M, 64);
         auto cap = [](int kb) { int c = kb / 4; return c < 1 ? 1 : (c > 16 ? 16 : c); };
-        p.qkv_splits = want_splits((long)cdiv(kd < qd ? kd : qd, 128) * tok_tiles * 2, cap(cdiv(H, 64)));
-        p.gu_splits = want_splits((long)cdiv(F / T, 128) * T * tok_tiles, cap(cdiv(H, 64)));
+        p.qkv_splits = want_splits((long)(cdiv(qd, 128) + 2 * cdiv(kd, 128)) * tok_tiles, cap(cdiv(H, 64)));
+        p.gu_splits = want_splits((long)cdiv(F / T, 128) * T * 2 * tok_tiles, cap(cdiv(H, 64)));
         p.down_splits = want_splits((long)cdiv(H, 128) * tok_tiles, cap(cdiv(F, 64)));
         p.o_per_group = want_splits((long)cdiv(H, 128) * T * tok_tiles, cap(cdiv(qd / T, 64)));
     } else if (decode) {
@@ -145,7 +145,7 @@ Plan make_plan(const spd_dims &d, int M, bool decode, int max_context)
 }
 
 struct Layout {
-    size_t res[2], h, q, attn, act, qkv32, proj32, gu32, part_o, part_ml, rope, err, total;
+    size_t res[2], h, q, attn, act, qkv32, proj32, gu32, part_o, part_ml, attn_cnt, rope, err, total;
     size_t Mcap;
 };
 
@@ -177,6 +177,7 @@ Layout make_layout(const spd_dims &d, bool any_spd)
     L.gu32 = take(mx(pp.gu_splits * Mp, pd.gu_splits * Md) * 2 * F * 4);
     L.part_o = take(Md * d.n_q_heads * 32 * d.head_dim * 4);
     L.part_ml = take(Md * d.n_q_heads * 32 * 2 * 4);
+    L.attn_cnt = take(Md * d.n_q_heads * 4);
     L.total = off;
     return L;
 }
@@ -190,6 +191,7 @@ int check_dims(const spd_dims *d, const uint8_t *mask)
     if (d->head_dim != 32 && d->head_dim != 64 && d->head_dim != 128) return SPD_EINVAL;
     if (d->n_q_heads % d->n_kv_heads) return SPD_EINVAL;
     if (d->n_q_heads % d->T || d->n_kv_heads % d->T || d->ffn % d->T) return SPD_EINVAL;
+    if (d->hidden % 4 || d->hidden > 65536) return SPD_EINVAL;
     if (d->dtype == 1 && (d->hidden % 8 || (d->ffn / d->T) % 8)) return SPD_EINVAL; // 16-byte rows for bf16 tiles
     if (d->kv_block_size < 1 || d->max_batch < 1 || d->max_seq_len < 1 || d->max_prefill_tokens < 1) return SPD_EINVAL;
     if (!(d->rms_eps > 0.f)) return SPD_EINVAL;
@@ -253,16 +255,19 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
         {
             const void *wm[3] = {w.wq, w.wk, w.wv};
             const int wn[3] = {qd, kd, kd}, wcol[3] = {0, qd, qd + kd};
-            for (int i = 0; i < 3; ++i) {
-                if (TC) {
-                    const TcMap *wmaps[3] = {&c->maps[l].wq, &c->maps[l].wk, &c->maps[l].wv};
-                    MAP_OR_FAIL(am, act_map(c, AB_H, tbox));
-                    TcGemmArgs g{};
-                    g.C = c->qkv32 + wcol[i]; g.ldc = nqkv; g.c_batch_stride = 0; g.c_split_stride = (long)M * nqkv;
-                    g.t_rows = M; g.w_rows = wn[i]; g.batches = 1; g.w_batched = 0; g.t_batched = 0;
-                    g.num_kb = cdiv(H, 64); g.splits = p.qkv_splits; g.err = c->err;
-                    LAUNCH(K_QKV, launch_gemm_tc(*wmaps[i], *am, g, swap, st));
-                } else {
+            if (TC) {
+                // one launch over the three matrices
+                const TcMap *wmaps[3] = {&c->maps[l].wq, &c->maps[l].wk, &c->maps[l].wv};
+                MAP_OR_FAIL(am, act_map(c, AB_H, tbox));
+                TcGemmArgs g{};
+                g.C = c->qkv32; g.ldc = nqkv; g.c_batch_stride = 0; g.c_split_stride = (long)M * nqkv;
+                for (int i = 0; i < 3; ++i) { g.w_rows[i] = wn[i]; g.c_off[i] = wcol[i]; }
+                g.t_rows = M; g.batches = 1; g.w_batched = 0; g.t_batched = 0;
+                g.num_kb = cdiv(H, 64); g.splits = p.qkv_splits; g.err = c->err;
+                LAUNCH(K_QKV, launch_gemm_tc(wmaps, 3, *am, g, swap, st));
+            }
+            for (int i = 0; i < 3 && !TC; ++i) {
+                {
                     GemmProblem g{};
                     g.A = c->h; g.lda = H; g.a_shard_stride = 0; g.W = wm[i]; g.ldw = H;
                     g.C = c->qkv32 + wcol[i]; g.ldc = nqkv; g.c_split_stride = (long)M * nqkv;
@@ -284,8 +289,8 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
             AttnArgs a{};
             a.q = c->q; a.k_pages = w.k_pages; a.v_pages = w.v_pages; a.pt = pt; a.tm = tm; a.out = c->attn;
             a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.B = M; a.splits = p.attn_splits;
-            a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.err = c->err;
-            if (decode) { LAUNCH(K_ATTN, launch_decode_attention<T>(a, st)); ++launches; }
+            a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.counters = c->attn_cnt; a.err = c->err;
+            if (decode) LAUNCH(K_ATTN, launch_decode_attention<T>(a, st));
             else LAUNCH(K_ATTN, launch_prefill_attention<T>(a, st));
         }
         // a5: row-split output projection.  Plane (i, j) holds the part of Y_i that comes from
@@ -297,9 +302,10 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
             MAP_OR_FAIL(am, act_map(c, o_single ? AB_ATTN : AB_ATTN_SHARD, tbox));
             TcGemmArgs g{};
             g.C = c->proj32; g.ldc = H; g.c_batch_stride = (long)p.o_per_group * M * H; g.c_split_stride = (long)M * H;
-            g.t_rows = M; g.w_rows = H; g.batches = o_single ? 1 : Tn; g.w_batched = !o_single; g.t_batched = !o_single;
+            g.t_rows = M; g.w_rows[0] = H; g.batches = o_single ? 1 : Tn; g.w_batched = !o_single; g.t_batched = !o_single;
             g.num_kb = cdiv(o_single ? qd : qd / Tn, 64); g.splits = o_single ? 1 : p.o_per_group; g.err = c->err;
-            LAUNCH(K_OPROJ, launch_gemm_tc(o_single ? c->maps[l].wo_full : c->maps[l].wo_shard, *am, g, swap, st));
+            const TcMap *wmaps[1] = {o_single ? &c->maps[l].wo_full : &c->maps[l].wo_shard};
+            LAUNCH(K_OPROJ, launch_gemm_tc(wmaps, 1, *am, g, swap, st));
         } else {
             GemmProblem g{};
             g.A = c->attn; g.lda = qd; g.W = w.wo; g.ldw = qd; g.C = c->proj32; g.ldc = H; g.c_split_stride = (long)M * H;
@@ -318,16 +324,20 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
         // a8: column-split gate / up; in an SPD block shard i reads its own MLP input plane
         {
             const void *gm[2] = {w.w_gate, w.w_up};
-            for (int i = 0; i < 2; ++i) {
+            if (TC) {
+                // gate and up in one launch: same token operand, two weight matrices
+                const TcMap *wmaps[2] = {&c->maps[l].w_gate, &c->maps[l].w_up};
+                MAP_OR_FAIL(am, act_map(c, AB_H, tbox));
+                TcGemmArgs g{};
+                g.C = c->gu32; g.ldc = F; g.c_batch_stride = F / Tn; g.c_split_stride = (long)M * F;
+                g.c_off[0] = 0; g.c_off[1] = (long)p.gu_splits * M * F;
+                g.t_rows = M; g.w_rows[0] = g.w_rows[1] = F / Tn; g.batches = Tn; g.w_batched = 1; g.t_batched = sync ? 0 : 1;
+                g.num_kb = cdiv(H, 64); g.splits = p.gu_splits; g.err = c->err;
+                LAUNCH(K_GATE_UP, launch_gemm_tc(wmaps, 2, *am, g, swap, st));
+            }
+            for (int i = 0; i < 2 && !TC; ++i) {
                 float *Cg = c->gu32 + (long)i * p.gu_splits * M * F;
-                if (TC) {
-                    MAP_OR_FAIL(am, act_map(c, AB_H, tbox));
-                    TcGemmArgs g{};
-                    g.C = Cg; g.ldc = F; g.c_batch_stride = F / Tn; g.c_split_stride = (long)M * F;
-                    g.t_rows = M; g.w_rows = F / Tn; g.batches = Tn; g.w_batched = 1; g.t_batched = sync ? 0 : 1;
-                    g.num_kb = cdiv(H, 64); g.splits = p.gu_splits; g.err = c->err;
-                    LAUNCH(K_GATE_UP, launch_gemm_tc(i == 0 ? c->maps[l].w_gate : c->maps[l].w_up, *am, g, swap, st));
-                } else {
+                {
                     GemmProblem g{};
                     g.A = c->h; g.lda = H; g.a_shard_stride = sync ? 0 : Mc * H; g.W = gm[i]; g.ldw = H;
                     g.C = Cg; g.ldc = F; g.c_split_stride = (long)M * F;
@@ -347,9 +357,10 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
             MAP_OR_FAIL(am, act_map(c, AB_ACT, tbox));
             TcGemmArgs g{};
             g.C = c->proj32; g.ldc = H; g.c_batch_stride = 0; g.c_split_stride = (long)M * H;
-            g.t_rows = M; g.w_rows = H; g.batches = 1; g.w_batched = 0; g.t_batched = 0;
+            g.t_rows = M; g.w_rows[0] = H; g.batches = 1; g.w_batched = 0; g.t_batched = 0;
             g.num_kb = cdiv(F, 64); g.splits = p.down_splits; g.err = c->err;
-            LAUNCH(K_DOWN, launch_gemm_tc(c->maps[l].w_down, *am, g, swap, st));
+            const TcMap *wmaps[1] = {&c->maps[l].w_down};
+            LAUNCH(K_DOWN, launch_gemm_tc(wmaps, 1, *am, g, swap, st));
         } else {
             GemmProblem g{};
             g.A = c->act; g.lda = F; g.W = w.w_down; g.ldw = F; g.C = c->proj32; g.ldc = H; g.c_split_stride = (long)M * H;
@@ -459,6 +470,7 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     c.rope = (float2 *)(c.ws + L.rope);
     c.qkv32 = (float *)(c.ws + L.qkv32); c.proj32 = (float *)(c.ws + L.proj32); c.gu32 = (float *)(c.ws + L.gu32);
     c.part_o = (float *)(c.ws + L.part_o); c.part_ml = (float *)(c.ws + L.part_ml);
+    c.attn_cnt = (int *)(c.ws + L.attn_cnt);
     c.launches_last = 0;
     c.profiling = false;
     c.ev_used = 0;
@@ -536,9 +548,10 @@ int spd_gemm_bf16(const void *a, const void *w, float *c, int32_t M, int32_t N, 
     if (make_operand_map(&am, a, K, M, a_batched ? batches : 1, K, (long)M * K, tbox)) return SPD_EINVAL;
     TcGemmArgs g{};
     g.C = c; g.ldc = (long)batches * N; g.c_batch_stride = N; g.c_split_stride = (long)M * batches * N;
-    g.t_rows = M; g.w_rows = N; g.batches = batches; g.w_batched = batches > 1; g.t_batched = a_batched && batches > 1;
+    g.t_rows = M; g.w_rows[0] = N; g.batches = batches; g.w_batched = batches > 1; g.t_batched = a_batched && batches > 1;
     g.num_kb = (K + 63) / 64; g.splits = splits; g.err = err_flag;
-    CU_TRY(launch_gemm_tc(wm, am, g, swap != 0, (cudaStream_t)stream));
+    const TcMap *wmaps[1] = {&wm};
+    CU_TRY(launch_gemm_tc(wmaps, 1, am, g, swap != 0, (cudaStream_t)stream));
     return SPD_OK;
 }
 
