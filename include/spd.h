@@ -110,6 +110,16 @@ int spd_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_l
                     const int32_t *block_table, int32_t max_pages, int32_t max_context,
                     void *out, void *stream);
 
+/* Decode steps are replayed from CUDA graphs (on by default): the first call with a given
+ * (x, seq_lens, block_table, out, B, max_pages, max_context rounded up to 256) captures the
+ * step's kernels on `stream` and later calls with the same values launch the captured graph;
+ * tensor CONTENTS (inputs, seq_lens, block table) may change freely between calls.  Up to 8
+ * graphs are kept per context.  A caller that passes fresh pointers every step should turn
+ * this off (each new pointer set costs a capture).  Calls on the legacy default stream (which
+ * cannot be captured), calls made while `stream` is itself being captured, and calls made
+ * while profiling launch the kernels directly. */
+int spd_set_graphs(spd_ctx *ctx, int32_t enabled);
+
 /* The projection building block on its own (exposed for kernel-level tests): the bf16
  * tensor-core GEMM every projection of the block uses, with the batching that expresses the
  * shard structure of Sec. 4.1.1 - per-shard weight row blocks (column split) and, when

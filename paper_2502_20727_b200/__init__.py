@@ -22,7 +22,7 @@ WEIGHT_NAMES = ("attn_norm", "wq", "wk", "wv", "wo", "mlp_norm", "w_gate", "w_up
 EXPORTS = ("spd_workspace_bytes", "spd_create", "spd_prefill", "spd_decode_step", "spd_sync_points",
            "spd_launches_per_decode_step", "spd_device_error", "spd_destroy", "spd_status_string",
            "spd_last_cuda_error", "spd_profile_begin", "spd_profile_end", "spd_profile_kinds",
-           "spd_profile_kind_name", "spd_gemm_bf16")
+           "spd_profile_kind_name", "spd_gemm_bf16", "spd_set_graphs")
 
 
 class SpdError(RuntimeError):
@@ -70,6 +70,7 @@ def load_library() -> ctypes.CDLL:
     lib.spd_status_string.restype = ctypes.c_char_p
     lib.spd_last_cuda_error.argtypes = []
     lib.spd_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, vp]
+    lib.spd_set_graphs.argtypes = [vp, i32]
     lib.spd_profile_begin.argtypes = [vp]
     lib.spd_profile_end.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     lib.spd_profile_kinds.argtypes = []
@@ -211,6 +212,10 @@ class SpdStack:
             _check("spd_profile_end", self.lib.spd_profile_end(self._ctx, _stream_ptr(), ms, cnt))
         return {self.lib.spd_profile_kind_name(i).decode(): {"ms": float(ms[i]), "launches": int(cnt[i])}
                 for i in range(n)}
+
+    def set_graphs(self, enabled: bool):
+        """Replay decode steps from captured CUDA graphs (default on); see spd_set_graphs."""
+        _check("spd_set_graphs", self.lib.spd_set_graphs(self._ctx, 1 if enabled else 0))
 
     def sync_points(self) -> int:
         return self.lib.spd_sync_points(self._ctx)

@@ -70,6 +70,8 @@ __device__ __forceinline__ void attend_range(const float *q, const T *kp, const 
 template <typename T, int VEC>
 __global__ void __launch_bounds__(128) prefill_attention_kernel(AttnArgs a)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int d = 32 * VEC, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int m = blockIdx.x * 4 + warp, hq = blockIdx.y;
     if (m >= a.M) return;
@@ -95,12 +97,11 @@ template <typename T> cudaError_t launch_prefill_attention(const AttnArgs &a, cu
     if (a.M <= 0) return cudaSuccess;
     dim3 grid((a.M + 3) / 4, a.n_q_heads);
     switch (a.head_dim) {
-    case 128: prefill_attention_kernel<T, 4><<<grid, 128, 0, st>>>(a); break;
-    case 64: prefill_attention_kernel<T, 2><<<grid, 128, 0, st>>>(a); break;
-    case 32: prefill_attention_kernel<T, 1><<<grid, 128, 0, st>>>(a); break;
+    case 128: return launch_kernel(prefill_attention_kernel<T, 4>, grid, dim3(128), 0, st, 0, a);
+    case 64: return launch_kernel(prefill_attention_kernel<T, 2>, grid, dim3(128), 0, st, 0, a);
+    case 32: return launch_kernel(prefill_attention_kernel<T, 1>, grid, dim3(128), 0, st, 0, a);
     default: return cudaErrorInvalidValue;
     }
-    return cudaGetLastError();
 }
 template cudaError_t launch_prefill_attention<float>(const AttnArgs &, cudaStream_t);
 template cudaError_t launch_prefill_attention<bf16>(const AttnArgs &, cudaStream_t);
@@ -133,6 +134,8 @@ template <> struct Row16<bf16> {
 template <typename T, int D, int GT>
 __global__ void __launch_bounds__(128) decode_attention_kernel(AttnArgs a)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     constexpr int E = Row16<T>::E, LPT = D / E, TPW = 32 / LPT, NG = 8, CHUNK = NG * TPW;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int slot = lane / LPT, li = lane % LPT;
@@ -298,10 +301,9 @@ template <typename T, int D> cudaError_t launch_decode_d(const AttnArgs &a, cuda
     const int group = a.n_q_heads / a.pt.n_kv_heads;
     const int gt = (group % 4 == 0) ? 4 : ((group % 2 == 0) ? 2 : 1);
     dim3 grid(a.n_q_heads / gt, a.B, a.splits);
-    if (gt == 4) decode_attention_kernel<T, D, 4><<<grid, 128, 0, st>>>(a);
-    else if (gt == 2) decode_attention_kernel<T, D, 2><<<grid, 128, 0, st>>>(a);
-    else decode_attention_kernel<T, D, 1><<<grid, 128, 0, st>>>(a);
-    return cudaGetLastError();
+    if (gt == 4) return launch_kernel(decode_attention_kernel<T, D, 4>, grid, dim3(128), 0, st, 0, a);
+    if (gt == 2) return launch_kernel(decode_attention_kernel<T, D, 2>, grid, dim3(128), 0, st, 0, a);
+    return launch_kernel(decode_attention_kernel<T, D, 1>, grid, dim3(128), 0, st, 0, a);
 }
 
 template <typename T> cudaError_t launch_decode_attention(const AttnArgs &a, cudaStream_t st)

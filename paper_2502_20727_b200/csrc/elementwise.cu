@@ -3,6 +3,10 @@
 // the rotary embedding + KV-page append, and SwiGLU.
 #include "common.cuh"
 
+#include <cooperative_groups.h>
+
+namespace cg = cooperative_groups;
+
 namespace spd {
 
 constexpr int MAX_T = 8;
@@ -58,6 +62,8 @@ __device__ __forceinline__ float4 group_sum4(const NormArgs &a, int g, long idx)
 template <typename T>
 __global__ void __launch_bounds__(512) residual_norm_kernel(NormArgs a)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     __shared__ float red[32];
     const int m = blockIdx.x, H = a.H, G = a.n_groups, H4 = H >> 2;
     float ss[MAX_T];
@@ -98,14 +104,108 @@ __global__ void __launch_bounds__(512) residual_norm_kernel(NormArgs a)
     }
 }
 
+// The same computation with a thread-block cluster of CS CTAs per token row: each CTA owns
+// hidden/CS columns, keeps its chunks in registers (single pass over the planes) and the
+// row's sums of squares are combined through distributed shared memory.
+template <typename T, int NCH>
+__global__ void __launch_bounds__(256) residual_norm_cluster_kernel(NormArgs a)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    cg::cluster_group cluster = cg::this_cluster();
+    const int CS = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+    const int m = blockIdx.x / CS, H = a.H, G = a.n_groups, P = a.per_group;
+    const int cpc = (H >> 2) / CS; // float4 chunks per CTA
+    __shared__ float warp_ss[8][MAX_T];
+    __shared__ float cta_ss[MAX_T];
+    float4 base[NCH], y[NCH][MAX_T];
+    float ss[MAX_T];
+#pragma unroll
+    for (int g = 0; g < MAX_T; ++g) ss[g] = 0.f;
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+        const int lc = threadIdx.x + i * blockDim.x;
+        if (lc >= cpc) continue;
+        const long idx = (long)m * H + 4 * (rank * cpc + lc);
+        base[i] = a.x_in ? load4<T>((const T *)a.x_in + idx) : *(const float4 *)(a.res_in + idx);
+        float4 tot = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int g = 0; g < MAX_T; ++g) {
+            if (g >= G) continue;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (a.part) {
+#pragma unroll 4
+                for (int p = 0; p < P; ++p)
+                    acc = f4add(acc, *(const float4 *)(a.part + (long)(g * P + p) * a.part_stride + idx));
+            }
+            y[i][g] = acc;
+            tot = f4add(tot, acc);
+            const float4 r = f4add(base[i], acc);
+            ss[g] += r.x * r.x + r.y * r.y + r.z * r.z + r.w * r.w;
+        }
+        const float4 r = f4add(base[i], tot);
+        if (a.res_out) *(float4 *)(a.res_out + idx) = r;
+        if (a.final_out) store4<T>((T *)a.final_out + idx, r);
+    }
+    if (!a.h_out) return; // uniform over the whole grid: no CTA of the cluster waits below
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+#pragma unroll
+    for (int g = 0; g < MAX_T; ++g) {
+        if (g >= G) continue;
+        const float v = warp_sum(ss[g]);
+        if (lane == 0) warp_ss[warp][g] = v;
+    }
+    __syncthreads();
+    if (threadIdx.x < MAX_T) {
+        float v = 0.f;
+        if ((int)threadIdx.x < G)
+            for (int w = 0; w < nw; ++w) v += warp_ss[w][threadIdx.x];
+        cta_ss[threadIdx.x] = v;
+    }
+    cluster.sync();
+    float rs[MAX_T];
+#pragma unroll
+    for (int g = 0; g < MAX_T; ++g) {
+        rs[g] = 0.f;
+        if (g >= G) continue;
+        float tot = 0.f;
+        for (int r = 0; r < CS; ++r) tot += cluster.map_shared_rank(cta_ss, r)[g];
+        rs[g] = rsqrtf(tot / (float)H + a.eps);
+    }
+    cluster.sync(); // no CTA may exit while its shared memory is still being read
+    const T *gain = (const T *)a.gain;
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+        const int lc = threadIdx.x + i * blockDim.x;
+        if (lc >= cpc) continue;
+        const int col = 4 * (rank * cpc + lc);
+        const long idx = (long)m * H + col;
+        const float4 gj = load4<T>(gain + col);
+#pragma unroll
+        for (int g = 0; g < MAX_T; ++g) {
+            if (g >= G) continue;
+            const float4 r = f4add(base[i], y[i][g]);
+            store4<T>((T *)a.h_out + (long)g * a.h_stride + idx,
+                      make_float4(r.x * rs[g] * gj.x, r.y * rs[g] * gj.y, r.z * rs[g] * gj.z, r.w * rs[g] * gj.w));
+        }
+    }
+}
+
 template <typename T> cudaError_t launch_residual_norm(const NormArgs &a, cudaStream_t st)
 {
     if (a.M <= 0) return cudaSuccess;
     if (a.H % 4 || a.n_groups > MAX_T) return cudaErrorInvalidValue;
     const int h4 = a.H / 4;
+    constexpr int CS = 8;
+    if (h4 % CS == 0 && h4 / CS <= 512 && (long)a.M * CS < 2147483647L) {
+        const int cpc = h4 / CS;
+        const int threads = cpc >= 256 ? 256 : (cpc + 31) / 32 * 32;
+        const dim3 grid((unsigned)(a.M * CS));
+        if (cpc <= threads) return launch_kernel(residual_norm_cluster_kernel<T, 1>, grid, dim3(threads), 0, st, CS, a);
+        return launch_kernel(residual_norm_cluster_kernel<T, 2>, grid, dim3(threads), 0, st, CS, a);
+    }
     const int threads = h4 >= 512 ? 512 : (h4 + 31) / 32 * 32;
-    residual_norm_kernel<T><<<a.M, threads, 0, st>>>(a);
-    return cudaGetLastError();
+    return launch_kernel(residual_norm_kernel<T>, dim3(a.M), dim3(threads), 0, st, 0, a);
 }
 template cudaError_t launch_residual_norm<float>(const NormArgs &, cudaStream_t);
 template cudaError_t launch_residual_norm<bf16>(const NormArgs &, cudaStream_t);
@@ -113,6 +213,8 @@ template cudaError_t launch_residual_norm<bf16>(const NormArgs &, cudaStream_t);
 // cos/sin of pos * base^(-2j/d), evaluated in double once per call and shared by all layers.
 __global__ void rope_table_kernel(float2 *table, TokMap tm, int M, int half, double log_base, int d)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= M * half) return;
     int m = i / half, j = i % half, b, pos;
@@ -127,14 +229,16 @@ cudaError_t launch_rope_table(float2 *table, TokMap tm, int M, int head_dim, flo
 {
     int n = M * (head_dim / 2);
     if (n <= 0) return cudaSuccess;
-    rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(table, tm, M, head_dim / 2, log((double)base), head_dim);
-    return cudaGetLastError();
+    return launch_kernel(rope_table_kernel, dim3((n + 255) / 256), dim3(256), 0, st, 0, table, tm, M, head_dim / 2,
+                         log((double)base), head_dim);
 }
 
 // grid (M, n_q_heads + n_kv_heads): sums the split-K planes of one head's projection, rotates
 // q and k (pairs (j, j + d/2)), stores q for the attention kernel and k, v into their page.
 template <typename T> __global__ void rope_kv_kernel(RopeKvArgs a)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int m = blockIdx.x, head = blockIdx.y, d = a.head_dim, half = d / 2;
     const int nq = a.n_q_heads, nkv = a.pt.n_kv_heads;
     int b, pos;
@@ -181,8 +285,7 @@ template <typename T> cudaError_t launch_rope_kv(const RopeKvArgs &a, cudaStream
     if (a.M <= 0) return cudaSuccess;
     dim3 grid(a.M, a.n_q_heads + a.pt.n_kv_heads);
     int threads = a.head_dim / 2 >= 64 ? 64 : 32;
-    rope_kv_kernel<T><<<grid, threads, 0, st>>>(a);
-    return cudaGetLastError();
+    return launch_kernel(rope_kv_kernel<T>, grid, dim3(threads), 0, st, 0, a);
 }
 template cudaError_t launch_rope_kv<float>(const RopeKvArgs &, cudaStream_t);
 template cudaError_t launch_rope_kv<bf16>(const RopeKvArgs &, cudaStream_t);
@@ -190,6 +293,8 @@ template cudaError_t launch_rope_kv<bf16>(const RopeKvArgs &, cudaStream_t);
 // act = silu(sum_s gate_s) * (sum_s up_s)
 template <typename T> __global__ void silu_mul_kernel(SiluMulArgs a)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
     long n = (long)a.M * a.F;
     if (i >= n) return;
@@ -207,8 +312,7 @@ template <typename T> cudaError_t launch_silu_mul(const SiluMulArgs &a, cudaStre
 {
     long n = (long)a.M * a.F;
     if (n <= 0) return cudaSuccess;
-    silu_mul_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, st>>>(a);
-    return cudaGetLastError();
+    return launch_kernel(silu_mul_kernel<T>, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, 0, a);
 }
 template cudaError_t launch_silu_mul<float>(const SiluMulArgs &, cudaStream_t);
 template cudaError_t launch_silu_mul<bf16>(const SiluMulArgs &, cudaStream_t);

@@ -13,6 +13,8 @@ constexpr int BM = 64, BN = 64, BK = 16;
 template <typename T>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmProblem p, int tiles_per_shard)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     __shared__ float As[BK][BM + 4];
     __shared__ float Ws[BK][BN + 4];
     const int shard = blockIdx.x / tiles_per_shard;
@@ -72,8 +74,7 @@ template <typename T> cudaError_t launch_gemm_simt(const GemmProblem &p, cudaStr
     if (p.M <= 0 || p.n_per_shard <= 0) return cudaSuccess;
     int tiles_per_shard = (p.n_per_shard + BN - 1) / BN;
     dim3 grid(tiles_per_shard * p.n_shards, (p.M + BM - 1) / BM, p.splits);
-    gemm_simt_kernel<T><<<grid, 256, 0, st>>>(p, tiles_per_shard);
-    return cudaGetLastError();
+    return launch_kernel(gemm_simt_kernel<T>, grid, dim3(256), 0, st, 0, p, tiles_per_shard);
 }
 template cudaError_t launch_gemm_simt<float>(const GemmProblem &, cudaStream_t);
 template cudaError_t launch_gemm_simt<bf16>(const GemmProblem &, cudaStream_t);

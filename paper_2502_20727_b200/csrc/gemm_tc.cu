@@ -144,6 +144,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
     const int kb_end = (int)((long)g.num_kb * (split + 1) / g.splits);
     const int n_kb = kb_end - kb_begin;
 
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         mbar_init(tmem_full_bar, 1);
@@ -167,15 +168,30 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
     const int b_z = SWAP ? (g.t_batched ? z : 0) : (g.w_batched ? z : 0);
 
     if (warp == 0 && lane == 0) {
-        // TMA producer
+        // TMA producer.  The weight tiles do not depend on the preceding kernel, so the first
+        // ring of them is requested before waiting for it (programmatic dependent launch): the
+        // weight stream of this GEMM overlaps the tail of whatever ran before.
+        const int pre = n_kb < C::STAGES ? n_kb : C::STAGES;
+        for (int i = 0; i < pre; ++i) {
+            mbar_expect_tx(full_bar(i), C::STAGE_BYTES);
+            const uint32_t sa = base + i * C::STAGE_BYTES, sb = sa + C::A_BYTES;
+            const int kx = (kb_begin + i) * BK;
+            if (SWAP) tma_load_3d(sa, tm_w, kx, a_row0, a_z, full_bar(i));
+            else tma_load_3d(sb, tm_w, kx, b_row0, b_z, full_bar(i));
+        }
+        pdl_wait();
         for (int i = 0; i < n_kb; ++i) {
             const int s = i % C::STAGES;
-            if (!mbar_wait(empty_bar(s), ((i / C::STAGES) & 1) ^ 1, g.err, abort_flag)) break;
-            mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
             const uint32_t sa = base + s * C::STAGE_BYTES, sb = sa + C::A_BYTES;
             const int kx = (kb_begin + i) * BK;
-            tma_load_3d(sa, SWAP ? tm_w : &tm_t, kx, a_row0, a_z, full_bar(s));
-            tma_load_3d(sb, SWAP ? &tm_t : tm_w, kx, b_row0, b_z, full_bar(s));
+            if (i >= pre) {
+                if (!mbar_wait(empty_bar(s), ((i / C::STAGES) & 1) ^ 1, g.err, abort_flag)) break;
+                mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
+                if (SWAP) tma_load_3d(sa, tm_w, kx, a_row0, a_z, full_bar(s));
+                else tma_load_3d(sb, tm_w, kx, b_row0, b_z, full_bar(s));
+            }
+            if (SWAP) tma_load_3d(sb, &tm_t, kx, b_row0, b_z, full_bar(s));
+            else tma_load_3d(sa, &tm_t, kx, a_row0, a_z, full_bar(s));
         }
     } else if (warp == 1 && lane == 0) {
         // MMA issuer
@@ -197,6 +213,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const __grid_constant__ CU
         umma_commit(tmem_full_bar);    // arrives when every MMA above has completed
     }
     __syncwarp();
+    pdl_wait(); // the output buffer may still be read by an earlier kernel until this returns
 
     // epilogue: warp w owns TMEM lanes [32w, 32w+32)
     const bool acc_ok = (n_kb > 0) && mbar_wait(tmem_full_bar, 0, g.err, abort_flag);
@@ -271,8 +288,7 @@ cudaError_t launch_cfg(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    gemm_tc_kernel<BN, SWAP><<<grid, 128, C::SMEM_BYTES, st>>>(*tw[0], *tw[1], *tw[2], tt, g);
-    return cudaGetLastError();
+    return launch_kernel(gemm_tc_kernel<BN, SWAP>, grid, dim3(128), C::SMEM_BYTES, st, 0, *tw[0], *tw[1], *tw[2], tt, g);
 }
 
 } // namespace

@@ -55,8 +55,25 @@ const char *const kind_names[K_COUNT] = {"residual_rmsnorm", "gemm_qkv", "rope_k
 
 struct LayerMaps { TcMap wq, wk, wv, wo_full, wo_shard, w_gate, w_up, w_down; };
 
+// A captured decode step is valid for exactly these arguments.
+struct GraphKey {
+    const void *x;
+    const int32_t *seq_lens, *block_table;
+    void *out;
+    int B, max_pages, ctx_bucket;
+    bool operator==(const GraphKey &o) const
+    {
+        return x == o.x && seq_lens == o.seq_lens && block_table == o.block_table && out == o.out && B == o.B &&
+               max_pages == o.max_pages && ctx_bucket == o.ctx_bucket;
+    }
+};
+struct GraphEntry { GraphKey key; cudaGraphExec_t exec; unsigned long long last_use; int launches; };
+
 struct Ctx {
     spd_dims d;
+    bool use_graphs;
+    std::vector<GraphEntry> graphs;
+    unsigned long long graph_clock;
     std::vector<uint8_t> mask;
     std::vector<spd_layer> layers;
     std::vector<LayerMaps> maps; // bf16 only
@@ -132,12 +149,13 @@ Plan make_plan(const spd_dims &d, int M, bool decode, int max_context)
     p.o_kps = qd / (T * p.o_per_group);
     p.attn_splits = 1;
     if (decode) {
-        // decode attention: enough CTAs for the machine, at least 2 pages per split
-        long ctas = (long)M * d.n_q_heads;
-        int s = (int)((2 * N_SM + ctas - 1) / ctas);
-        int pages = cdiv(max_context, d.kv_block_size);
-        int smax = pages / 2 < 1 ? 1 : pages / 2;
-        if (s > smax) s = smax;
+        // decode attention: short dependent chains - about 128 tokens per CTA (one or two
+        // 16-token chunks per warp) - within 16 CTAs per SM and 32 splits
+        const int gt = (d.n_q_heads / d.n_kv_heads) % 4 == 0 ? 4 : ((d.n_q_heads / d.n_kv_heads) % 2 == 0 ? 2 : 1);
+        const long ctas = (long)M * (d.n_q_heads / gt);
+        int s = cdiv(max_context, 128);
+        const long smax = (16L * N_SM + ctas - 1) / ctas;
+        if (s > smax) s = (int)smax;
         if (s > 32) s = 32;
         p.attn_splits = s < 1 ? 1 : s;
     }
@@ -472,6 +490,8 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     c.part_o = (float *)(c.ws + L.part_o); c.part_ml = (float *)(c.ws + L.part_ml);
     c.attn_cnt = (int *)(c.ws + L.attn_cnt);
     c.launches_last = 0;
+    c.use_graphs = true;
+    c.graph_clock = 0;
     c.profiling = false;
     c.ev_used = 0;
     memset(c.act_map_ready, 0, sizeof(c.act_map_ready));
@@ -533,8 +553,57 @@ int spd_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_l
     if (max_context > d.max_seq_len || (long)max_pages * d.kv_block_size < max_context) return SPD_ECAPACITY;
     cudaStream_t st = (cudaStream_t)stream;
     TokMap tm{1, 0, 1, 0, seq_lens};
-    return d.dtype == 0 ? run_tokens<float>(&c, x, out, B, tm, block_table, max_pages, true, max_context, st)
-                        : run_tokens<bf16>(&c, x, out, B, tm, block_table, max_pages, true, max_context, st);
+    // The launch sequence only depends on a coarse bucket of the context bound (it sizes the
+    // KV split), so a step can be replayed from a captured graph until a pointer or the
+    // bucket changes.
+    int ctx_bucket = (max_context + 255) / 256 * 256;
+    if (ctx_bucket > d.max_seq_len) ctx_bucket = d.max_seq_len;
+    if ((long)ctx_bucket > (long)max_pages * d.kv_block_size) ctx_bucket = max_pages * d.kv_block_size;
+    auto run = [&]() {
+        return d.dtype == 0 ? run_tokens<float>(&c, x, out, B, tm, block_table, max_pages, true, ctx_bucket, st)
+                            : run_tokens<bf16>(&c, x, out, B, tm, block_table, max_pages, true, ctx_bucket, st);
+    };
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    CU_TRY(cudaStreamIsCapturing(st, &cap));
+    // (the legacy default stream cannot be captured)
+    if (!c.use_graphs || c.profiling || cap != cudaStreamCaptureStatusNone || st == 0 || st == cudaStreamLegacy) return run();
+
+    const GraphKey key{x, seq_lens, block_table, out, B, max_pages, ctx_bucket};
+    GraphEntry *hit = nullptr;
+    for (GraphEntry &e : c.graphs)
+        if (e.key == key) hit = &e;
+    if (!hit) {
+        CU_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+        const int rc = run();
+        cudaGraph_t graph = nullptr;
+        cudaError_t e = cudaStreamEndCapture(st, &graph);
+        if (rc != SPD_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
+        if (e != cudaSuccess) { g_last_cuda_error = (int)e; return SPD_ECUDA; }
+        cudaGraphExec_t exec = nullptr;
+        e = cudaGraphInstantiate(&exec, graph, 0);
+        cudaGraphDestroy(graph);
+        if (e != cudaSuccess) { g_last_cuda_error = (int)e; return SPD_ECUDA; }
+        if (c.graphs.size() >= 8) { // evict the least recently used
+            size_t lru = 0;
+            for (size_t i = 1; i < c.graphs.size(); ++i)
+                if (c.graphs[i].last_use < c.graphs[lru].last_use) lru = i;
+            cudaGraphExecDestroy(c.graphs[lru].exec);
+            c.graphs.erase(c.graphs.begin() + lru);
+        }
+        c.graphs.push_back(GraphEntry{key, exec, 0, c.launches_last});
+        hit = &c.graphs.back();
+    }
+    hit->last_use = ++c.graph_clock;
+    c.launches_last = hit->launches;
+    CU_TRY(cudaGraphLaunch(hit->exec, st));
+    return SPD_OK;
+}
+
+int spd_set_graphs(spd_ctx *ctx, int32_t enabled)
+{
+    if (!ctx) return SPD_ENULL;
+    ctx->c.use_graphs = enabled != 0;
+    return SPD_OK;
 }
 
 int spd_gemm_bf16(const void *a, const void *w, float *c, int32_t M, int32_t N, int32_t K, int32_t batches,
@@ -609,6 +678,7 @@ void spd_destroy(spd_ctx *ctx)
 {
     if (!ctx) return;
     for (cudaEvent_t e : ctx->c.ev_pool) cudaEventDestroy(e);
+    for (GraphEntry &g : ctx->c.graphs) cudaGraphExecDestroy(g.exec);
     delete ctx;
 }
 

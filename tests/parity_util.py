@@ -9,6 +9,7 @@ import oracle
 import spd_inputs as si
 
 TOL = {"fp32": 1e-4, "bf16": 2e-2}
+_STREAM = None
 
 
 def rel_err(got, ref) -> float:
@@ -33,6 +34,12 @@ class Pair:
     def __init__(self, w: si.Workload, *, mask=None, B=None, max_len=None, max_prefill_tokens=None, seed=0,
                  device="cuda:0", n_pages=None, layers=None):
         import paper_2502_20727_b200 as spd
+        # a non-default stream: the legacy default stream cannot be captured into the graphs
+        # that replay decode steps
+        global _STREAM
+        if _STREAM is None:
+            _STREAM = torch.cuda.Stream(device=device)
+        torch.cuda.set_stream(_STREAM)
         self.w = w
         self.B = B or w.batch
         self.max_len = max_len or (w.prompt + w.decode_steps)
@@ -62,8 +69,15 @@ class Pair:
     def decode(self, t, seed=0):
         x = si.make_hidden(self.w, (self.B, self.w.hidden), "cpu", seed, 1 + t)
         ref, _, _ = oracle.stack_forward(self.dims, self.mask, self.layers_np, to_np(x)[:, None, :], self.pos, self.cache)
-        seq = torch.from_numpy(self.pos.copy()).to(self.device)
-        got = self.stack.decode_step(x.to(self.device), seq, self.block_table, int(self.pos.max()) + 1)
+        # fixed device buffers, as a serving loop has them: after the first step the library
+        # replays its captured graph, so both the capture and the replay path are compared
+        if not hasattr(self, "x_dev"):
+            self.x_dev = torch.empty((self.B, self.w.hidden), dtype=self.w.torch_dtype, device=self.device)
+            self.seq_dev = torch.empty(self.B, dtype=torch.int32, device=self.device)
+            self.out_dev = torch.empty_like(self.x_dev)
+        self.x_dev.copy_(x)
+        self.seq_dev.copy_(torch.from_numpy(self.pos.copy()))
+        got = self.stack.decode_step(self.x_dev, self.seq_dev, self.block_table, int(self.pos.max()) + 1, self.out_dev)
         torch.cuda.synchronize()
         self.pos = self.pos + 1
         return to_np(got), ref[:, 0, :]
