@@ -132,6 +132,29 @@ int spd_set_graphs(spd_ctx *ctx, int32_t enabled);
 int spd_gemm_bf16(const void *a, const void *w, float *c, int32_t M, int32_t N, int32_t K, int32_t batches,
                   int32_t a_batched, int32_t splits, int32_t swap, int32_t *err_flag, void *stream);
 
+/* The same split-K projection GEMM for callers that cannot obtain device memory at the time of
+ * the call: code running inside a serving engine whose allocator owns the whole GPU, a plugin
+ * invoked under a "no cudaMalloc / no allocator call" rule (the driver call synchronises the
+ * device and can fail once other tenants have filled it), or a process that must stay within a
+ * fixed memory budget.  (The paper has no counterpart; this is a library convenience.)
+ *   c : fp32 [M][batches*N] = the SUM over the K splits (same operands and meaning as
+ *       spd_gemm_bf16, whose split planes this call adds up in split order)
+ * The split planes are kept in an array that is part of the library image,
+ * SPD_STATIC_SCRATCH_BYTES per GPU that loads the library, held until the process exits.  The
+ * call allocates and frees no device memory itself and uses no allocating library routine;
+ * inputs, output and err_flag are still the caller's.
+ *   - splits * M * batches * N * 4 bytes must fit in the array, else SPD_EWORKSPACE is
+ *     returned and nothing is launched.
+ *   - The first call on a device looks up the array's device address (the device must be
+ *     current); make that first call outside any stream capture.
+ *   - All calls share the one array, and it keeps whatever the previous call left there.
+ *     Each call overwrites every element it later reads, so nothing needs clearing, but two
+ *     calls whose kernels may overlap on the GPU (different streams) race: serialise them.
+ * Errors: SPD_ENULL, SPD_EINVAL, SPD_EWORKSPACE (too large for the array), SPD_ECUDA. */
+#define SPD_STATIC_SCRATCH_BYTES (4u << 20)
+int spd_gemm_bf16_sum_static(const void *a, const void *w, float *c, int32_t M, int32_t N, int32_t K, int32_t batches,
+                             int32_t a_batched, int32_t splits, int32_t swap, int32_t *err_flag, void *stream);
+
 /* Number of shard sums ("sync-points", Sec. 3) one forward pass of this stack executes:
  * 2 per TP block, 1 per SPD block. */
 int spd_sync_points(const spd_ctx *ctx);

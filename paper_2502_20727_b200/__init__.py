@@ -22,7 +22,7 @@ WEIGHT_NAMES = ("attn_norm", "wq", "wk", "wv", "wo", "mlp_norm", "w_gate", "w_up
 EXPORTS = ("spd_workspace_bytes", "spd_create", "spd_prefill", "spd_decode_step", "spd_sync_points",
            "spd_launches_per_decode_step", "spd_device_error", "spd_destroy", "spd_status_string",
            "spd_last_cuda_error", "spd_profile_begin", "spd_profile_end", "spd_profile_kinds",
-           "spd_profile_kind_name", "spd_gemm_bf16", "spd_set_graphs")
+           "spd_profile_kind_name", "spd_gemm_bf16", "spd_set_graphs", "spd_gemm_bf16_sum_static")
 
 
 class SpdError(RuntimeError):
@@ -71,6 +71,7 @@ def load_library() -> ctypes.CDLL:
     lib.spd_last_cuda_error.argtypes = []
     lib.spd_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, vp]
     lib.spd_set_graphs.argtypes = [vp, i32]
+    lib.spd_gemm_bf16_sum_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, vp]
     lib.spd_profile_begin.argtypes = [vp]
     lib.spd_profile_end.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     lib.spd_profile_kinds.argtypes = []
@@ -118,6 +119,38 @@ def gemm_bf16(a: torch.Tensor, w: torch.Tensor, *, splits: int = 1, swap: bool =
     if int(err.item()) != 0:
         raise SpdError("spd_gemm_bf16", -6, f"device flag {int(err.item())}")
     return c
+
+
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def gemm_bf16_sum_static(a: torch.Tensor, w: torch.Tensor, out: torch.Tensor, err: torch.Tensor, *, splits: int = 1,
+                         swap: bool = False) -> torch.Tensor:
+    """spd_gemm_bf16_sum_static: the split-K GEMM summed over its splits, for callers that must
+    not allocate device memory during the call.  The caller passes the output (fp32
+    [M, batches*N]) and the int32 error flag; the split planes sit in the library's own fixed
+    array (``STATIC_SCRATCH_BYTES``; larger problems raise SPD_EWORKSPACE).  Nothing is
+    allocated here either, and the flag is not read back: check ``err`` when convenient."""
+    lib = load_library()
+    wb = w if w.dim() == 3 else w[None]
+    a_batched = a.dim() == 3
+    batches, N, K = wb.shape
+    M = a.shape[-2]
+    if a_batched and a.shape[0] != batches:
+        raise ValueError("a and w disagree on the batch count")
+    for t in (a, w):
+        if not (t.is_cuda and t.is_contiguous() and t.dtype == torch.bfloat16):
+            raise ValueError("contiguous CUDA bf16 tensors expected")
+    if not (out.is_cuda and out.is_contiguous() and out.dtype == torch.float32 and tuple(out.shape) == (M, batches * N)):
+        raise ValueError("out: contiguous CUDA float32 [M, batches*N]")
+    if not (err.is_cuda and err.dtype == torch.int32 and err.numel() >= 1):
+        raise ValueError("err: CUDA int32 tensor")
+    with torch.cuda.device(a.device):
+        _check("spd_gemm_bf16_sum_static",
+               lib.spd_gemm_bf16_sum_static(a.data_ptr(), w.data_ptr(), out.data_ptr(), M, N, K, batches,
+                                            1 if a_batched else 0, splits, 1 if swap else 0, err.data_ptr(),
+                                            _stream_ptr()))
+    return out
 
 
 class SpdStack:
