@@ -120,6 +120,15 @@ int spd_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_l
  * while profiling launch the kernels directly. */
 int spd_set_graphs(spd_ctx *ctx, int32_t enabled);
 
+/* Tuning knob of the bf16 decode step: how many ranges the K dimension of each weight-streaming
+ * projection is cut into (more ranges = more thread blocks pulling weights at once; the ranges
+ * of one output tile form a thread-block cluster that adds up its partials through shared
+ * memory).  0 = automatic (about three resident thread blocks per SM).  Values are clamped to
+ * at least four 64-wide K blocks per range and to 8 ranges per tile (8 / T for o_proj, whose
+ * T shard slices are ranges already).  Results stay deterministic for a
+ * given setting.  Drops the captured decode graphs.  Errors: SPD_ENULL, SPD_EINVAL. */
+int spd_set_decode_splits(spd_ctx *ctx, int32_t qkv, int32_t o_proj, int32_t gate_up, int32_t down);
+
 /* The projection building block on its own (exposed for kernel-level tests): the bf16
  * tensor-core GEMM every projection of the block uses, with the batching that expresses the
  * shard structure of Sec. 4.1.1 - per-shard weight row blocks (column split) and, when

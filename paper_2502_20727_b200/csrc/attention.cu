@@ -2,6 +2,7 @@
 // ranges, so one launch over all heads IS the T per-shard attentions side by side; nothing
 // crosses a shard boundary here.  K and V are always read from the paged cache.
 #include "common.cuh"
+#include "trace.cuh"
 
 namespace spd {
 
@@ -135,7 +136,9 @@ template <typename T, int D, int GT>
 __global__ void __launch_bounds__(128) decode_attention_kernel(AttnArgs a)
 {
     pdl_launch_dependents();
+    if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_START);
     pdl_wait();
+    if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_DEP_DONE);
     constexpr int E = Row16<T>::E, LPT = D / E, TPW = 32 / LPT, NG = 8, CHUNK = NG * TPW;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int slot = lane / LPT, li = lane % LPT;
@@ -270,6 +273,7 @@ __global__ void __launch_bounds__(128) decode_attention_kernel(AttnArgs a)
             if (dd == 0) { a.part_ml[pi * 2] = gm; a.part_ml[pi * 2 + 1] = gden; }
         }
     }
+    if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_MAIN_DONE);
     if (a.splits == 1) return;
     // the last CTA of this (sequence, head tile) to arrive merges the splits
     __threadfence();
@@ -294,6 +298,7 @@ __global__ void __launch_bounds__(128) decode_attention_kernel(AttnArgs a)
         ((T *)a.out)[((long)b * a.n_q_heads + hq0 + g) * D + dd] = from_f<T>(gden > 0.f ? acc / gden : 0.f);
     }
     if (threadIdx.x == 0) *cnt = 0; // ready for the next launch
+    if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_END);
 }
 
 template <typename T, int D> cudaError_t launch_decode_d(const AttnArgs &a, cudaStream_t st)

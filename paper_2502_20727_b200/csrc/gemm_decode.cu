@@ -1,0 +1,558 @@
+// Fused decode projections.  A decode step is bound by streaming every weight once, so each of
+// the four projections of a block is one weight-streaming tcgen05 GEMM (weights on the 128-row
+// MMA side, the few tokens on the N side), with the step that follows it folded into its tail.
+//
+// K is cut into P ranges so that every SM pulls weights; the P thread blocks of one output tile
+// form a thread-block cluster.  After its main loop each block parks its fp32 partial tile in
+// its own shared memory; after one cluster barrier block c adds up, in range order, the
+// partials of the tokens c, c+P, ... through distributed shared memory and applies the fused
+// step to them.  No partial ever goes through global memory and nobody spins on a flag.
+//
+//   EPI_QKV    : attention-RMSNorm rstd, rotary embedding, q store, K/V page append   (a2, a3)
+//   EPI_OPROJ  : the cluster is the T emulated devices (K slice i gives Y_i).  sync block:
+//                R = X + sum_i Y_i; SPD block (Sec. 4.1.1): R_i = X + Y_i per device, and
+//                X + sum_i Y_i for the output residual; gain-scaled MLP inputs and their
+//                partial sums of squares                                               (a5-a7)
+//   EPI_GATEUP : MLP-RMSNorm rstd (per device in an SPD block), SwiGLU                 (a8)
+//   EPI_DOWN   : the kept sync-point (sum over devices = K accumulation over all of F), output
+//                residual, next block's gain-scaled input / final output               (a9, a10)
+//
+// Warps 0-3 own the accumulator rows (TMEM lanes) and run the epilogue; while the main loop runs
+// they fetch what the epilogue needs (rstd, page addresses).  Warp 4 issues the TMA loads,
+// warp 5 the MMAs.
+#include "gemm_decode.cuh"
+#include "tc_ptx.cuh"
+#include "trace.cuh"
+
+namespace spd {
+
+namespace {
+
+using namespace tc;
+
+constexpr int MAX_GROUPS = 8; // emulated devices
+constexpr int MAX_P = 8;      // portable cluster size
+constexpr int THREADS = 192;
+
+template <int BN> struct DCfg {
+    static constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    // Three thread blocks per SM with a short ring each (measured faster than two blocks with a
+    // deep ring: more blocks pull weights at once, and clusters of up to 8 blocks always find room).
+    static constexpr int RING_BYTES = 56 * 1024;
+    static constexpr int STAGES = RING_BYTES / STAGE_BYTES < 3 ? 3 : RING_BYTES / STAGE_BYTES;
+    static constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static_assert(STAGES * STAGE_BYTES >= 2 * BN * 128 * 4, "ring too small for the staging tiles");
+};
+
+struct DecTile {
+    int z, wt, wi, w_row0, t_row0, split, rank, P;
+};
+
+// Launcher-filled tiling constants travel behind the public arguments.
+struct DecLaunch {
+    DecGemmArgs g;
+    int w_tiles_per_batch;
+    int tile_start[3];
+    int P; // K ranges per output tile = cluster size = gridDim.z
+};
+
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// 16 bytes of block `rank`'s shared memory at the offset that `local_addr` has in ours.
+__device__ __forceinline__ float4 ld_peer4(uint32_t local_addr, uint32_t rank)
+{
+    uint32_t ra;
+    float4 v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(ra) : "memory");
+    return v;
+}
+__device__ __forceinline__ void add4(float4 &a, const float4 &b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
+__device__ __forceinline__ float sq4(float4 v) { return v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w; }
+__device__ __forceinline__ void store_bf16x4(bf16 *p, float4 v, float4 gn)
+{
+    __nv_bfloat162 a = __floats2bfloat162_rn(v.x * gn.x, v.y * gn.y), b = __floats2bfloat162_rn(v.z * gn.z, v.w * gn.w);
+    uint2 u;
+    u.x = *(uint32_t *)&a;
+    u.y = *(uint32_t *)&b;
+    *(uint2 *)p = u;
+}
+
+// The partials of token j, columns 4*lane..4*lane+3, from every block of the cluster (y[s] = range s).
+__device__ __forceinline__ void load_partials(float4 (&y)[MAX_P], const float *S, int j, int lane, int P)
+{
+    const float *src = S + j * 128 + 4 * lane;
+    if (P == 1) { y[0] = *(const float4 *)src; return; }
+    const uint32_t a = smem_u32(src);
+#pragma unroll
+    for (int s = 0; s < MAX_P; ++s)
+        if (s < P) y[s] = ld_peer4(a, (uint32_t)s);
+}
+
+// rstd of the tile's tokens from the partial sums of squares, by the 128 epilogue threads:
+// thread t adds every (128/BN)-th partial of token t % BN, then the parts are added in order.
+template <int BN>
+__device__ __forceinline__ void compute_rstd(const SumSq &ss, int group, int t_row0, int t_rows, float *red, float *sm_rstd)
+{
+    constexpr int PARTS = 128 / BN;
+    const int t = threadIdx.x, j = t % BN, part = t / BN, m = t_row0 + j;
+    float acc = 0.f;
+    if (m < t_rows)
+        for (int tile = part; tile < ss.tiles; tile += PARTS) acc += __ldcg(ss.part + ((long)tile * ss.groups + group) * ss.Mcap + m);
+    red[t] = acc;
+    epi_sync();
+    if (t < BN) {
+        float tot = 0.f;
+#pragma unroll
+        for (int q = 0; q < PARTS; ++q) tot += red[q * BN + t];
+        sm_rstd[t] = rsqrtf(tot / (float)ss.H + ss.eps);
+    }
+}
+
+// ---- epilogues: block `rank` of the cluster finishes tokens rank, rank+P, ... of the tile ----------
+// Gathers run with warp w on the block's w-th, (w+4)-th ... token and lane l on columns 4l..4l+3.
+
+template <int BN>
+__device__ __forceinline__ void gather_my_tokens(const DecGemmArgs &g, const DecTile &t, const float *S, float *Gb)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int q = warp;; q += 4) {
+        const int j = t.rank + t.P * q;
+        if (j >= BN || t.t_row0 + j >= g.t_rows) break;
+        float4 y[MAX_P];
+        load_partials(y, S, j, lane, t.P);
+        float4 v = y[0];
+#pragma unroll
+        for (int s = 1; s < MAX_P; ++s)
+            if (s < t.P) add4(v, y[s]);
+        *(float4 *)(Gb + q * 128 + 4 * lane) = v;
+    }
+}
+
+template <int BN>
+__device__ __forceinline__ void epilogue_qkv(const DecGemmArgs &g, const DecTile &t, const float *S, float *Gb,
+                                             const float *sm_rstd, const long *sm_kvoff)
+{
+    const int r = threadIdx.x, d = g.head_dim, half = d >> 1;
+    const int row = t.w_row0 + r, head = row / d, jd = row % d, nq = g.n_q_heads;
+    const bool row_valid = row < g.w_rows[t.wi];
+    const bool rot = t.wi < 2 && g.rope != nullptr;
+    // the rotary factors do not depend on the gather: request them first
+    float2 cs[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const int m = t.t_row0 + t.rank + t.P * q;
+        cs[q] = make_float2(1.f, 0.f);
+        if (rot && row_valid && t.rank + t.P * q < BN && m < g.t_rows) cs[q] = g.rope[(long)m * half + (jd < half ? jd : jd - half)];
+    }
+    gather_my_tokens<BN>(g, t, S, Gb);
+    epi_sync();
+    if (!row_valid) return;
+    const int partner = jd < half ? r + half : r - half;
+    for (int q = 0;; ++q) {
+        const int j = t.rank + t.P * q, m = t.t_row0 + j;
+        if (j >= BN || m >= g.t_rows) break;
+        float v = Gb[q * 128 + r] * sm_rstd[j];
+        if (rot) {
+            const float2 c = q < 4 ? cs[q < 4 ? q : 0] : g.rope[(long)m * half + (jd < half ? jd : jd - half)];
+            const float o = Gb[q * 128 + partner] * sm_rstd[j];
+            v = jd < half ? v * c.x - o * c.y : v * c.x + o * c.y;
+        }
+        if (t.wi == 0) {
+            ((bf16 *)g.q_out)[((long)m * nq + head) * d + jd] = __float2bfloat16_rn(v);
+        } else {
+            const long off = sm_kvoff[j];
+            if (off >= 0) ((bf16 *)(t.wi == 1 ? g.k_pages : g.v_pages))[off + (long)head * g.pt.block * d + jd] = __float2bfloat16_rn(v);
+        }
+    }
+}
+
+template <int BN>
+__device__ __forceinline__ void epilogue_gateup(const DecGemmArgs &g, const DecTile &t, const float *S, float *Gb, const float *sm_rstd)
+{
+    gather_my_tokens<BN>(g, t, S, Gb);
+    epi_sync();
+    // two FFN columns per thread: 32 threads cover the tile's 64 columns of one token
+    for (int idx = threadIdx.x;; idx += 128) {
+        const int q = idx >> 5, rr = 2 * (idx & 31), j = t.rank + t.P * q, m = t.t_row0 + j, f = t.w_row0 + rr;
+        if (j >= BN || m >= g.t_rows) break;
+        if (f >= g.Fs) continue;
+        const float rs = sm_rstd[j];
+        const float2 gt = *(const float2 *)(Gb + q * 128 + rr), up = *(const float2 *)(Gb + q * 128 + 64 + rr);
+        const float g0 = gt.x * rs, g1 = gt.y * rs;
+        *(__nv_bfloat162 *)((bf16 *)g.act + (long)m * g.F + (long)t.z * g.Fs + f) =
+            __floats2bfloat162_rn(g0 / (1.f + __expf(-g0)) * (up.x * rs), g1 / (1.f + __expf(-g1)) * (up.y * rs));
+    }
+}
+
+// Residual stream out, gain-scaled bf16 copy (the next GEMM's input) and the tile's partial sums
+// of squares.  spd_groups (o_proj of an SPD block): range i of the cluster is emulated device i,
+// which only ever sees its own partial attention output Y_i (R_i = X + Y_i), while the carried
+// residual collects every Y_i.
+template <int BN>
+__device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const DecTile &t, const float *S, bool spd_groups)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n = t.w_row0 + 4 * lane, H = g.H;
+    const bool valid = n < H;
+    const int G = spd_groups ? g.n_groups : 1, per = t.P / G; // ranges per device
+    const float4 one = make_float4(1.f, 1.f, 1.f, 1.f);
+    float4 gn = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (valid && g.gain) {
+        const uint2 u = *(const uint2 *)((const bf16 *)g.gain + n);
+        const float2 a = __bfloat1622float2(*(const __nv_bfloat162 *)&u.x), b = __bfloat1622float2(*(const __nv_bfloat162 *)&u.y);
+        gn = make_float4(a.x, a.y, b.x, b.y);
+    }
+    for (int q = warp;; q += 4) {
+        const int j = t.rank + t.P * q, m = t.t_row0 + j;
+        if (j >= BN || m >= g.t_rows) break;
+        const long idx = (long)m * H + n;
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (valid) x = *(const float4 *)(g.res_in + idx);
+        float4 y[MAX_P];
+        load_partials(y, S, j, lane, t.P);
+        float4 tot = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (spd_groups) {
+            // ranges i*per .. i*per+per-1 are device i
+            float4 yi = make_float4(0.f, 0.f, 0.f, 0.f);
+            int cnt = 0, i = 0;
+#pragma unroll
+            for (int s = 0; s < MAX_P; ++s) {
+                if (s >= t.P) continue;
+                add4(yi, y[s]);
+                if (++cnt < per) continue;
+                add4(tot, yi);
+                float4 ri = x;
+                add4(ri, yi);
+                if (valid && g.hg) store_bf16x4((bf16 *)g.hg + (long)i * g.hg_stride + idx, ri, gn);
+                const float sq = warp_sum(valid ? sq4(ri) : 0.f);
+                if (lane == 0 && g.ss_out) g.ss_out[((long)t.wt * G + i) * g.Mcap + m] = sq;
+                yi = make_float4(0.f, 0.f, 0.f, 0.f);
+                cnt = 0;
+                ++i;
+            }
+            add4(x, tot);
+            if (valid && g.res_out) *(float4 *)(g.res_out + idx) = x;
+        } else {
+#pragma unroll
+            for (int s = 0; s < MAX_P; ++s)
+                if (s < t.P) add4(tot, y[s]);
+            add4(x, tot);
+            if (valid) {
+                if (g.res_out) *(float4 *)(g.res_out + idx) = x;
+                if (g.final_out) store_bf16x4((bf16 *)g.final_out + idx, x, one);
+                if (g.hg) store_bf16x4((bf16 *)g.hg + idx, x, gn);
+            }
+            if (g.ss_out) {
+                const float sq = warp_sum(valid ? sq4(x) : 0.f);
+                if (lane == 0) g.ss_out[(long)t.wt * g.Mcap + m] = sq;
+            }
+        }
+    }
+}
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_w0,
+                                                              const __grid_constant__ CUtensorMap tm_w1,
+                                                              const __grid_constant__ CUtensorMap tm_w2,
+                                                              const __grid_constant__ CUtensorMap tm_t,
+                                                              const __grid_constant__ DecLaunch L)
+{
+    using C = DCfg<BN>;
+    constexpr int SUB = (EPI == EPI_GATEUP) ? 2 : 1; // weight boxes per tile
+    constexpr int ROWS = BM / SUB;                   // weight rows per box
+    const DecGemmArgs &g = L.g;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ float sm_red[128];
+    __shared__ float sm_rstd[64];
+    __shared__ long sm_kvoff[64];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t bars = base + C::STAGES * C::STAGE_BYTES; // full[S], empty[S], tmem_full
+    uint32_t *tmem_slot = (uint32_t *)(gen_base + C::STAGES * C::STAGE_BYTES + 8 * (2 * C::STAGES + 1));
+    volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (C::STAGES + s); };
+    const uint32_t tmem_full_bar = bars + 8u * (2 * C::STAGES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    DecTile t;
+    t.P = L.P;
+    t.rank = t.P > 1 ? (int)cluster_rank() : 0;
+    if (g.z_is_plane) { t.z = t.rank / g.splits; t.split = t.rank % g.splits; t.wt = blockIdx.x; }
+    else { t.z = blockIdx.x / L.w_tiles_per_batch; t.split = t.rank; t.wt = blockIdx.x % L.w_tiles_per_batch; }
+    t.wi = (SUB == 2) ? 0 : ((t.wt >= L.tile_start[2]) ? 2 : ((t.wt >= L.tile_start[1]) ? 1 : 0));
+    t.w_row0 = (t.wt - L.tile_start[t.wi]) * ROWS;
+    t.t_row0 = blockIdx.y * BN;
+    const CUtensorMap *tm_w = t.wi == 0 ? &tm_w0 : (t.wi == 1 ? &tm_w1 : &tm_w2);
+    const int kb_begin = (int)((long)g.num_kb * t.split / g.splits);
+    const int kb_end = (int)((long)g.num_kb * (t.split + 1) / g.splits);
+    const int n_kb = kb_end - kb_begin;
+
+    pdl_launch_dependents();
+    if (threadIdx.x == 0) {
+        SPD_TRACE_EVENT(EPI, TR_START);
+        for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        mbar_init(tmem_full_bar, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_acc = *tmem_slot;
+
+    const int a_z = g.w_batched ? t.z : 0, b_z = g.t_batched ? t.z : 0;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            // TMA producer.  Weights do not depend on the preceding kernel: the first ring of
+            // weight tiles is requested before waiting for it, so this GEMM's weight stream
+            // starts under the tail of whatever ran before.
+            asm volatile("prefetch.tensormap [%0];" ::"l"(tm_w) : "memory");
+            if (SUB == 2) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_w1) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_t) : "memory");
+            auto load_w = [&](int s, int kx) {
+                const uint32_t sa = base + s * C::STAGE_BYTES;
+                if (SUB == 1) tma_load_3d(sa, tm_w, kx, t.w_row0, a_z, full_bar(s));
+                else {
+                    tma_load_3d(sa, &tm_w0, kx, t.w_row0, a_z, full_bar(s));
+                    tma_load_3d(sa + ROWS * BK * 2, &tm_w1, kx, t.w_row0, a_z, full_bar(s));
+                }
+            };
+            const int pre = n_kb < C::STAGES ? n_kb : C::STAGES;
+            for (int i = 0; i < pre; ++i) {
+                mbar_expect_tx(full_bar(i), C::STAGE_BYTES);
+                load_w(i, (kb_begin + i) * BK);
+            }
+            pdl_wait();
+            SPD_TRACE_EVENT(EPI, TR_DEP_DONE);
+            for (int i = 0; i < n_kb; ++i) {
+                const int s = i % C::STAGES;
+                const int kx = (kb_begin + i) * BK;
+                if (i >= pre) {
+                    if (!mbar_wait(empty_bar(s), ((i / C::STAGES) & 1) ^ 1, g.err, abort_flag)) break;
+                    mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
+                    load_w(s, kx);
+                }
+                tma_load_3d(base + s * C::STAGE_BYTES + C::A_BYTES, &tm_t, kx, t.t_row0, b_z, full_bar(s));
+            }
+        }
+        __syncwarp();
+    } else if (warp == 5) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(BN);
+            for (int i = 0; i < n_kb; ++i) {
+                const int s = i % C::STAGES;
+                if (!mbar_wait(full_bar(s), (i / C::STAGES) & 1, g.err, abort_flag)) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t sa = base + s * C::STAGE_BYTES, sb = sa + C::A_BYTES;
+                const uint64_t da = make_desc(sa), db = make_desc(sb);
+#pragma unroll
+                for (int k = 0; k < BK / UMMA_K; ++k)
+                    umma(tmem_acc, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
+                         (i > 0 || k > 0) ? 1u : 0u);
+                umma_commit(empty_bar(s));
+            }
+            umma_commit(tmem_full_bar);
+        }
+        __syncwarp();
+    } else {
+        // epilogue warps: fetch what the tail needs while the weights stream
+        pdl_wait();
+        if (EPI == EPI_QKV || EPI == EPI_GATEUP)
+            compute_rstd<BN>(g.ss_in, (EPI == EPI_GATEUP && g.rstd_per_shard) ? t.z : 0, t.t_row0, g.t_rows, sm_red, sm_rstd);
+        if (EPI == EPI_QKV && t.wi > 0 && threadIdx.x < BN) {
+            // where this token's K / V row of kv head 0 goes; < 0: skip (the error flag says why)
+            const int m = t.t_row0 + threadIdx.x;
+            long off = -1;
+            if (m < g.t_rows) {
+                int b, pos;
+                g.tm.locate(m, b, pos);
+                const int pi = pos / g.pt.block;
+                if (pos < 0 || pi >= g.pt.max_pages) atomicOr(g.err, ERR_CAPACITY);
+                else {
+                    const int page = g.pt.block_table[(long)b * g.pt.max_pages + pi];
+                    if (page < 0 || page >= g.pt.n_pages) atomicOr(g.err, ERR_PAGE_RANGE);
+                    else off = ((long)page * g.pt.n_kv_heads * g.pt.block + pos % g.pt.block) * g.head_dim;
+                }
+            }
+            sm_kvoff[threadIdx.x] = off;
+        }
+        // accumulator -> registers: warp w owns TMEM lanes [32w, 32w+32); thread r = accumulator row r
+        const bool acc_ok = mbar_wait(tmem_full_bar, 0, g.err, abort_flag);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (threadIdx.x == 0) SPD_TRACE_EVENT(EPI, TR_MAIN_DONE);
+        float acc[BN];
+#pragma unroll
+        for (int c0 = 0; c0 < BN; c0 += 16) {
+            if (acc_ok) tmem_ld16(tmem_acc + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, acc + c0);
+            else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) acc[c0 + i] = 0.f;
+            }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        // The ring is free once the accumulator is complete (every TMA write has landed and every
+        // MMA has read its operands): park the partial tile there, token-major.
+        float *S = (float *)gen_base;
+#pragma unroll
+        for (int j = 0; j < BN; ++j) S[j * 128 + threadIdx.x] = acc[j];
+    }
+    // partial tiles of all ranges visible cluster-wide
+    if (t.P > 1) cluster_sync_all();
+    else __syncthreads();
+    if (warp == 5) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(C::TMEM_COLS) : "memory");
+    }
+    if (warp < 4) {
+        if (threadIdx.x == 0) SPD_TRACE_EVENT(EPI, TR_ARRIVED);
+        const float *S = (const float *)gen_base;
+        float *Gb = (float *)gen_base + BN * 128; // this block's gathered tokens
+        if (EPI == EPI_QKV) epilogue_qkv<BN>(g, t, S, Gb, sm_rstd, sm_kvoff);
+        else if (EPI == EPI_GATEUP) epilogue_gateup<BN>(g, t, S, Gb, sm_rstd);
+        else epilogue_residual<BN>(g, t, S, EPI == EPI_OPROJ && g.n_groups > 1);
+        if (threadIdx.x == 0) SPD_TRACE_EVENT(EPI, TR_END);
+    }
+    // no block may exit while a peer still reads its shared memory
+    if (t.P > 1) cluster_sync_all();
+}
+
+template <int BN, int EPI>
+cudaError_t launch_cfg(const CUtensorMap *const *tw, const CUtensorMap &tt, const DecLaunch &L, dim3 grid, cudaStream_t st)
+{
+    using C = DCfg<BN>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_decode_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = C::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    at[1].id = cudaLaunchAttributeClusterDimension;
+    at[1].val.clusterDim.x = 1;
+    at[1].val.clusterDim.y = 1;
+    at[1].val.clusterDim.z = (unsigned)L.P;
+    cfg.attrs = at;
+    cfg.numAttrs = L.P > 1 ? 2 : 1;
+    return cudaLaunchKernelEx(&cfg, gemm_decode_kernel<BN, EPI>, *tw[0], *tw[1], *tw[2], tt, L);
+}
+
+template <int EPI>
+cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, const DecLaunch &L, int tiles, cudaStream_t st)
+{
+    const int bn = tc_token_box(true, L.g.t_rows);
+    dim3 grid(tiles * (L.g.z_is_plane ? 1 : L.g.batches), (L.g.t_rows + bn - 1) / bn, L.P);
+    switch (bn) {
+    case 16: return launch_cfg<16, EPI>(tw, tt, L, grid, st);
+    case 32: return launch_cfg<32, EPI>(tw, tt, L, grid, st);
+    default: return launch_cfg<64, EPI>(tw, tt, L, grid, st);
+    }
+}
+
+// One thread block per 128 columns, all tokens: the same outputs EPI_DOWN leaves for the next block.
+__global__ void __launch_bounds__(128) decode_prologue_kernel(PrologueArgs a)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    __shared__ float sm[4];
+    const int r = threadIdx.x, warp = r >> 5, lane = r & 31, n = blockIdx.x * 128 + r;
+    const bool valid = n < a.H;
+    const float gn = valid ? __bfloat162float(((const bf16 *)a.gain)[n]) : 0.f;
+    for (int m = 0; m < a.M; ++m) {
+        const long idx = (long)m * a.H + n;
+        const float x = valid ? __bfloat162float(((const bf16 *)a.x)[idx]) : 0.f;
+        if (valid) {
+            a.res_out[idx] = x;
+            ((bf16 *)a.hg)[idx] = __float2bfloat16_rn(x * gn);
+        }
+        const float q = warp_sum(x * x);
+        __syncthreads();
+        if (lane == 0) sm[warp] = q;
+        __syncthreads();
+        if (r == 0) a.ss_out[(long)blockIdx.x * a.Mcap + m] = sm[0] + sm[1] + sm[2] + sm[3];
+    }
+}
+
+} // namespace
+
+int decode_tiles_per_batch(DecEpilogue epi, const int *w_rows, int n_weights)
+{
+    if (epi == EPI_GATEUP) return (w_rows[0] + 63) / 64;
+    int tiles = 0;
+    for (int i = 0; i < n_weights; ++i) tiles += (w_rows[i] + BM - 1) / BM;
+    return tiles;
+}
+
+cudaError_t launch_gemm_decode(DecEpilogue epi, const TcMap *const *weights, const TcMap &tokens, const DecGemmArgs &g,
+                               cudaStream_t st)
+{
+    const int nw = g.n_weights;
+    if (nw < 1 || nw > 3 || (epi == EPI_GATEUP && nw != 2)) return cudaErrorInvalidValue;
+    if (g.t_rows <= 0) return cudaSuccess;
+    if (g.splits < 1 || g.splits > g.num_kb || g.n_groups > MAX_GROUPS) return cudaErrorInvalidValue;
+    const int P = g.z_is_plane ? g.batches * g.splits : g.splits;
+    if (P > MAX_P) return cudaErrorInvalidValue;
+    if (epi == EPI_OPROJ && g.n_groups > 1 && (g.n_groups != g.batches || !g.z_is_plane)) return cudaErrorInvalidValue;
+    if (epi == EPI_QKV && (BM % g.head_dim) != 0) return cudaErrorInvalidValue;
+    const CUtensorMap *tw[3];
+    for (int i = 0; i < 3; ++i) tw[i] = (const CUtensorMap *)weights[i < nw ? i : 0];
+    const CUtensorMap &tt = *(const CUtensorMap *)&tokens;
+    DecLaunch L;
+    L.g = g;
+    int tiles = 0;
+    for (int i = 0; i < 3; ++i) {
+        L.tile_start[i] = tiles;
+        if (i < nw && epi != EPI_GATEUP) {
+            if (g.w_rows[i] <= 0) return cudaErrorInvalidValue;
+            tiles += (g.w_rows[i] + BM - 1) / BM;
+        } else if (i >= nw) {
+            L.tile_start[i] = 1 << 30; // never selected
+        }
+    }
+    if (epi == EPI_GATEUP) {
+        tiles = (g.w_rows[0] + 63) / 64;
+        L.tile_start[0] = 0;
+        L.tile_start[1] = L.tile_start[2] = 1 << 30;
+    }
+    L.w_tiles_per_batch = tiles;
+    L.P = P;
+    switch (epi) {
+    case EPI_QKV: return launch_epi<EPI_QKV>(tw, tt, L, tiles, st);
+    case EPI_OPROJ: return launch_epi<EPI_OPROJ>(tw, tt, L, tiles, st);
+    case EPI_GATEUP: return launch_epi<EPI_GATEUP>(tw, tt, L, tiles, st);
+    default: return launch_epi<EPI_DOWN>(tw, tt, L, tiles, st);
+    }
+}
+
+cudaError_t launch_decode_prologue(const PrologueArgs &a, cudaStream_t st)
+{
+    if (a.M <= 0) return cudaSuccess;
+    return launch_kernel(decode_prologue_kernel, dim3((a.H + 127) / 128), dim3(128), 0, st, 0, a);
+}
+
+} // namespace spd

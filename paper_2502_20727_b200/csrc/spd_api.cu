@@ -3,6 +3,7 @@
 #include "../../include/spd.h"
 #include "common.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_decode.cuh"
 
 #include <math.h>
 #include <new>
@@ -50,10 +51,11 @@ int want_splits(long tiles, int cap)
 
 enum ActBuf { AB_H = 0, AB_ATTN, AB_ATTN_SHARD, AB_ACT, AB_COUNT };
 enum Kind { K_NORM = 0, K_QKV, K_ROPE_KV, K_ATTN, K_OPROJ, K_GATE_UP, K_SILU_MUL, K_DOWN, K_ROPE_TABLE, K_COUNT };
+enum Site { SITE_QKV = 0, SITE_O, SITE_GU, SITE_DOWN, SITE_COUNT };
 const char *const kind_names[K_COUNT] = {"residual_rmsnorm", "gemm_qkv", "rope_kv_append", "attention", "gemm_o_proj",
                                          "gemm_gate_up", "silu_mul", "gemm_down", "rope_table"};
 
-struct LayerMaps { TcMap wq, wk, wv, wo_full, wo_shard, w_gate, w_up, w_down; };
+struct LayerMaps { TcMap wq, wk, wv, wo_full, wo_shard, w_gate, w_up, w_down, w_gate64, w_up64; };
 
 // A captured decode step is valid for exactly these arguments.
 struct GraphKey {
@@ -87,6 +89,8 @@ struct Ctx {
     float *qkv32, *proj32, *gu32, *part_o, *part_ml;
     float2 *rope;
     int *err, *attn_cnt;
+    float *ss_attn, *ss_mlp;     // partial row sums of squares (fused decode path)
+    int split_override[SITE_COUNT];
     int launches_last;
     // activation tensor maps, by buffer and token box (16, 32, 64, 128), built on first use
     TcMap act_maps[AB_COUNT][4];
@@ -162,8 +166,34 @@ Plan make_plan(const spd_dims &d, int M, bool decode, int max_context)
     return p;
 }
 
+// K ranges of a fused decode GEMM: as many as keep the launch within three resident thread blocks
+// per SM, each at least four K blocks long, at most `max_ranges` (the ranges of one output tile
+// form a thread-block cluster of at most 8 blocks).
+int decode_splits(long tiles, int num_kb, int override_, int max_ranges)
+{
+    long s = override_ > 0 ? override_ : (3L * N_SM) / (tiles < 1 ? 1 : tiles);
+    const long cap = num_kb / 4 < 1 ? 1 : num_kb / 4;
+    if (s > cap) s = cap;
+    if (s > max_ranges) s = max_ranges;
+    return (int)(s < 1 ? 1 : s);
+}
+
+// Shape of the four fused decode GEMMs: output tiles per token tile, K blocks per range unit and
+// how many ranges the shard structure already contributes (T for the row-split o_proj).
+struct SiteGeom { long tiles; int num_kb; int shard_ranges; };
+SiteGeom site_geom(const spd_dims &d, int site)
+{
+    const int H = d.hidden, qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, F = d.ffn, T = d.T;
+    switch (site) {
+    case SITE_QKV: return {cdiv(qd, 128) + 2L * cdiv(kd, 128), cdiv(H, 64), 1};
+    case SITE_O: return {(long)cdiv(H, 128) * T, cdiv(qd / T, 64), T};
+    case SITE_GU: return {(long)cdiv(F / T, 64) * T, cdiv(H, 64), 1};
+    default: return {cdiv(H, 128), cdiv(F, 64), 1};
+    }
+}
+
 struct Layout {
-    size_t res[2], h, q, attn, act, qkv32, proj32, gu32, part_o, part_ml, attn_cnt, rope, err, total;
+    size_t res[2], h, q, attn, act, qkv32, proj32, gu32, part_o, part_ml, attn_cnt, rope, err, ss_attn, ss_mlp, total;
     size_t Mcap;
 };
 
@@ -196,6 +226,10 @@ Layout make_layout(const spd_dims &d, bool any_spd)
     L.part_o = take(Md * d.n_q_heads * 32 * d.head_dim * 4);
     L.part_ml = take(Md * d.n_q_heads * 32 * 2 * 4);
     L.attn_cnt = take(Md * d.n_q_heads * 4);
+    // fused decode path: partial sums of squares per 128-column tile
+    const size_t h_tiles = (H + 127) / 128;
+    L.ss_attn = take(h_tiles * Mmax * 4);
+    L.ss_mlp = take(h_tiles * T * Mmax * 4);
     L.total = off;
     return L;
 }
@@ -400,11 +434,110 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
     return SPD_OK;
 }
 
+// One decode step of the bf16 stack with the fused projections: per block QKV(+rotary, KV append),
+// paged attention, o_proj(+residuals, MLP norm input), gate/up(+SwiGLU), down(+shard sum, residual).
+int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t *bt, int max_pages,
+                     int max_context, cudaStream_t st)
+{
+    const spd_dims &d = c->d;
+    const int H = d.hidden, qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, F = d.ffn, Tn = d.T;
+    const int Fs = F / Tn;
+    const long Mc = c->Mcap;
+    const Plan p = make_plan(d, M, true, max_context);
+    PageTable pt{bt, max_pages, c->n_pages, d.kv_block_size, d.n_kv_heads};
+    const int tbox = tc_token_box(true, M);
+    const int tok_tiles = cdiv(M, tbox), h_tiles = cdiv(H, 128);
+    int launches = 0;
+    const bool rope = d.rope_base > 0.f;
+    // K ranges of a site: automatic or overridden; a tile's ranges (times the shards for o_proj) fit a cluster of 8
+    auto splits_of = [&](int site) {
+        const SiteGeom sg = site_geom(d, site);
+        return decode_splits(sg.tiles * tok_tiles, sg.num_kb, c->split_override[site], 8 / sg.shard_ranges);
+    };
+    if (rope) LAUNCH(K_ROPE_TABLE, launch_rope_table(c->rope, tm, M, d.head_dim, d.rope_base, st));
+    {
+        PrologueArgs a{};
+        a.x = x; a.res_out = c->res[0]; a.gain = c->layers[0].attn_norm; a.hg = c->h; a.ss_out = c->ss_attn;
+        a.Mcap = Mc; a.M = M; a.H = H;
+        LAUNCH(K_NORM, launch_decode_prologue(a, st));
+    }
+    auto base_args = [&]() {
+        DecGemmArgs g{};
+        g.t_rows = M; g.err = c->err; g.H = H; g.Mcap = Mc; g.batches = 1; g.n_weights = 1; g.n_groups = 1;
+        return g;
+    };
+    for (int l = 0; l < d.n_layers; ++l) {
+        const spd_layer &w = c->layers[l];
+        const bool sync = c->mask[l] != 0;
+        {   // a2 + a3
+            DecGemmArgs g = base_args();
+            const TcMap *wmaps[3] = {&c->maps[l].wq, &c->maps[l].wk, &c->maps[l].wv};
+            MAP_OR_FAIL(am, act_map(c, AB_H, tbox));
+            g.n_weights = 3; g.w_rows[0] = qd; g.w_rows[1] = g.w_rows[2] = kd;
+            g.num_kb = cdiv(H, 64);
+            g.splits = splits_of(SITE_QKV);
+            g.ss_in = SumSq{c->ss_attn, h_tiles, 1, Mc, H, d.rms_eps};
+            g.rope = rope ? c->rope : nullptr; g.q_out = c->q; g.k_pages = w.k_pages; g.v_pages = w.v_pages; g.pt = pt; g.tm = tm;
+            g.n_q_heads = d.n_q_heads; g.head_dim = d.head_dim;
+            LAUNCH(K_QKV, launch_gemm_decode(EPI_QKV, wmaps, *am, g, st));
+        }
+        {   // a4
+            AttnArgs a{};
+            a.q = c->q; a.k_pages = w.k_pages; a.v_pages = w.v_pages; a.pt = pt; a.tm = tm; a.out = c->attn;
+            a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.B = M; a.splits = p.attn_splits;
+            a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.counters = c->attn_cnt; a.err = c->err;
+            LAUNCH(K_ATTN, launch_decode_attention<bf16>(a, st));
+        }
+        {   // a5 - a7: shard i's K slice gives the plane group Y_i
+            DecGemmArgs g = base_args();
+            const TcMap *wmaps[1] = {&c->maps[l].wo_shard};
+            MAP_OR_FAIL(am, act_map(c, AB_ATTN_SHARD, tbox));
+            g.w_rows[0] = H; g.batches = Tn; g.w_batched = 1; g.t_batched = 1; g.z_is_plane = 1;
+            g.num_kb = cdiv(qd / Tn, 64);
+            g.splits = splits_of(SITE_O);
+            g.res_in = c->res[0]; g.res_out = c->res[1]; g.gain = w.mlp_norm; g.hg = c->h; g.hg_stride = Mc * H;
+            g.ss_out = c->ss_mlp;
+            g.n_groups = sync ? 1 : Tn;
+            LAUNCH(K_OPROJ, launch_gemm_decode(EPI_OPROJ, wmaps, *am, g, st));
+        }
+        {   // a8: 64 gate rows and the 64 up rows of the same FFN columns per tile
+            DecGemmArgs g = base_args();
+            const TcMap *wmaps[2] = {&c->maps[l].w_gate64, &c->maps[l].w_up64};
+            MAP_OR_FAIL(am, act_map(c, AB_H, tbox));
+            g.n_weights = 2; g.w_rows[0] = g.w_rows[1] = Fs; g.batches = Tn; g.w_batched = 1; g.t_batched = sync ? 0 : 1;
+            g.num_kb = cdiv(H, 64);
+            g.splits = splits_of(SITE_GU);
+            g.ss_in = SumSq{c->ss_mlp, h_tiles, sync ? 1 : Tn, Mc, H, d.rms_eps};
+            g.rstd_per_shard = sync ? 0 : 1;
+            g.act = c->act; g.F = F; g.Fs = Fs;
+            LAUNCH(K_GATE_UP, launch_gemm_decode(EPI_GATEUP, wmaps, *am, g, st));
+        }
+        {   // a9 + a10: res[1] holds X + sum_i Y_i in both modes, so out = res[1] + sum_i Z_i
+            DecGemmArgs g = base_args();
+            const TcMap *wmaps[1] = {&c->maps[l].w_down};
+            MAP_OR_FAIL(am, act_map(c, AB_ACT, tbox));
+            g.w_rows[0] = H;
+            g.num_kb = cdiv(F, 64);
+            g.splits = splits_of(SITE_DOWN);
+            g.res_in = c->res[1]; g.res_out = c->res[0];
+            if (l + 1 < d.n_layers) { g.gain = c->layers[l + 1].attn_norm; g.hg = c->h; g.hg_stride = Mc * H; g.ss_out = c->ss_attn; }
+            else g.final_out = out;
+            LAUNCH(K_DOWN, launch_gemm_decode(EPI_DOWN, wmaps, *am, g, st));
+        }
+    }
+    c->launches_last = launches;
+    return SPD_OK;
+}
+
 int read_err_flag(Ctx *c, cudaStream_t st, int *flag)
 {
     CU_TRY(cudaMemcpyAsync(flag, c->err, sizeof(int), cudaMemcpyDeviceToHost, st));
     CU_TRY(cudaStreamSynchronize(st));
-    if (*flag) CU_TRY(cudaMemsetAsync(c->err, 0, sizeof(int), st));
+    if (*flag) {
+        // a kernel that gave up may have left arrival counters mid-count
+        CU_TRY(cudaMemsetAsync(c->err, 0, sizeof(int), st));
+        CU_TRY(cudaMemsetAsync(c->attn_cnt, 0, (size_t)c->d.max_batch * c->d.n_q_heads * 4, st));
+    }
     return SPD_OK;
 }
 
@@ -425,6 +558,8 @@ int build_weight_maps(Ctx &c)
         rc |= make_operand_map(&m.w_gate, w.w_gate, H, F / T, T, H, (F / T) * H, 128);
         rc |= make_operand_map(&m.w_up, w.w_up, H, F / T, T, H, (F / T) * H, 128);
         rc |= make_operand_map(&m.w_down, w.w_down, F, H, 1, F, 0, 128);
+        rc |= make_operand_map(&m.w_gate64, w.w_gate, H, F / T, T, H, (F / T) * H, 64);
+        rc |= make_operand_map(&m.w_up64, w.w_up, H, F / T, T, H, (F / T) * H, 64);
         if (rc) return SPD_EINVAL;
     }
     return SPD_OK;
@@ -489,6 +624,8 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     c.qkv32 = (float *)(c.ws + L.qkv32); c.proj32 = (float *)(c.ws + L.proj32); c.gu32 = (float *)(c.ws + L.gu32);
     c.part_o = (float *)(c.ws + L.part_o); c.part_ml = (float *)(c.ws + L.part_ml);
     c.attn_cnt = (int *)(c.ws + L.attn_cnt);
+    c.ss_attn = (float *)(c.ws + L.ss_attn); c.ss_mlp = (float *)(c.ws + L.ss_mlp);
+    for (int i = 0; i < SITE_COUNT; ++i) c.split_override[i] = 0;
     c.launches_last = 0;
     c.use_graphs = true;
     c.graph_clock = 0;
@@ -561,7 +698,7 @@ int spd_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_l
     if ((long)ctx_bucket > (long)max_pages * d.kv_block_size) ctx_bucket = max_pages * d.kv_block_size;
     auto run = [&]() {
         return d.dtype == 0 ? run_tokens<float>(&c, x, out, B, tm, block_table, max_pages, true, ctx_bucket, st)
-                            : run_tokens<bf16>(&c, x, out, B, tm, block_table, max_pages, true, ctx_bucket, st);
+                            : run_decode_fused(&c, x, out, B, tm, block_table, max_pages, ctx_bucket, st);
     };
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     CU_TRY(cudaStreamIsCapturing(st, &cap));
@@ -603,6 +740,18 @@ int spd_set_graphs(spd_ctx *ctx, int32_t enabled)
 {
     if (!ctx) return SPD_ENULL;
     ctx->c.use_graphs = enabled != 0;
+    return SPD_OK;
+}
+
+int spd_set_decode_splits(spd_ctx *ctx, int32_t qkv, int32_t o_proj, int32_t gate_up, int32_t down)
+{
+    if (!ctx) return SPD_ENULL;
+    if (qkv < 0 || o_proj < 0 || gate_up < 0 || down < 0) return SPD_EINVAL;
+    Ctx &c = ctx->c;
+    c.split_override[SITE_QKV] = qkv; c.split_override[SITE_O] = o_proj;
+    c.split_override[SITE_GU] = gate_up; c.split_override[SITE_DOWN] = down;
+    for (GraphEntry &g : c.graphs) cudaGraphExecDestroy(g.exec); // captured steps used the old cuts
+    c.graphs.clear();
     return SPD_OK;
 }
 
