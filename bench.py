@@ -136,8 +136,8 @@ def run_native(args, rank, world):
                                     max_prefill_tokens=min(B * S, args.prefill_chunk), device=dev)
     pages_per_seq = (max_len + w.kv_block - 1) // w.kv_block
     bt = si.make_block_table(B, pages_per_seq, stack.n_pages, rank).to(dev)
-    if args.splits:
-        stack.set_decode_splits(*[int(v) for v in args.splits.split(",")])
+    if args.tune:
+        stack.set_tuning(**{kv.split("=")[0]: int(kv.split("=")[1]) for kv in args.tune.split(",")})
 
     # ---- prefill (reported, not the headline step) -----------------------------------
     xp = si.make_hidden(w, (B, S, w.hidden), dev, rank, 0)
@@ -328,7 +328,7 @@ def main():
     ap.add_argument("--prefill-reps", type=int, default=3)
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--splits", default="", help="K cuts of the decode projections: qkv,o_proj,gate_up,down (0 = automatic)")
+    ap.add_argument("--tune", default="", help="decode tuning knobs, e.g. qkv_splits=4,l2_prefetch_blocks=8 (see spd_set_tuning)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))

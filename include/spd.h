@@ -120,14 +120,22 @@ int spd_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_l
  * while profiling launch the kernels directly. */
 int spd_set_graphs(spd_ctx *ctx, int32_t enabled);
 
-/* Tuning knob of the bf16 decode step: how many ranges the K dimension of each weight-streaming
- * projection is cut into (more ranges = more thread blocks pulling weights at once; the ranges
- * of one output tile form a thread-block cluster that adds up its partials through shared
- * memory).  0 = automatic (about three resident thread blocks per SM).  Values are clamped to
- * at least four 64-wide K blocks per range and to 8 ranges per tile (8 / T for o_proj, whose
- * T shard slices are ranges already).  Results stay deterministic for a
- * given setting.  Drops the captured decode graphs.  Errors: SPD_ENULL, SPD_EINVAL. */
-int spd_set_decode_splits(spd_ctx *ctx, int32_t qkv, int32_t o_proj, int32_t gate_up, int32_t down);
+/* Tuning knobs of the bf16 decode step (results stay deterministic for a given setting; every
+ * change drops the captured decode graphs).  value 0 restores the automatic choice of a split key.
+ *   "qkv_splits", "o_proj_splits", "gate_up_splits", "down_splits"
+ *       how many ranges the K dimension of that weight-streaming projection is cut into (more
+ *       ranges = more thread blocks pulling weights at once; the ranges of one output tile form
+ *       a thread-block cluster that adds up its partials through shared memory).  Automatic:
+ *       about three resident thread blocks per SM.  Clamped to at least four 64-wide K blocks
+ *       per range and to 8 ranges per tile (8 / T for o_proj, whose T shard slices are ranges).
+ *   "attention_splits"
+ *       ranges the cached context of a sequence is cut into for the paged decode attention
+ *       (clamped to 32 and to four pages per range).
+ *   "l2_prefetch_blocks"
+ *       64-wide K blocks of weights each thread block of a projection pulls into L2 before it
+ *       waits for the preceding kernel (default 0 = off, at most 64; measured neutral to harmful).
+ * Errors: SPD_ENULL, SPD_EINVAL (unknown key, negative value). */
+int spd_set_tuning(spd_ctx *ctx, const char *key, int32_t value);
 
 /* The projection building block on its own (exposed for kernel-level tests): the bf16
  * tensor-core GEMM every projection of the block uses, with the batching that expresses the

@@ -23,7 +23,7 @@ EXPORTS = ("spd_workspace_bytes", "spd_create", "spd_prefill", "spd_decode_step"
            "spd_launches_per_decode_step", "spd_device_error", "spd_destroy", "spd_status_string",
            "spd_last_cuda_error", "spd_profile_begin", "spd_profile_end", "spd_profile_kinds",
            "spd_profile_kind_name", "spd_gemm_bf16", "spd_set_graphs", "spd_gemm_bf16_sum_static",
-           "spd_set_decode_splits")
+           "spd_set_tuning")
 
 
 class SpdError(RuntimeError):
@@ -72,7 +72,7 @@ def load_library() -> ctypes.CDLL:
     lib.spd_last_cuda_error.argtypes = []
     lib.spd_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, vp]
     lib.spd_set_graphs.argtypes = [vp, i32]
-    lib.spd_set_decode_splits.argtypes = [vp, i32, i32, i32, i32]
+    lib.spd_set_tuning.argtypes = [vp, ctypes.c_char_p, i32]
     lib.spd_gemm_bf16_sum_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, vp]
     lib.spd_profile_begin.argtypes = [vp]
     lib.spd_profile_end.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
@@ -252,9 +252,11 @@ class SpdStack:
         """Replay decode steps from captured CUDA graphs (default on); see spd_set_graphs."""
         _check("spd_set_graphs", self.lib.spd_set_graphs(self._ctx, 1 if enabled else 0))
 
-    def set_decode_splits(self, qkv: int = 0, o_proj: int = 0, gate_up: int = 0, down: int = 0):
-        """K cuts of the four decode projections (0 = automatic); see spd_set_decode_splits."""
-        _check("spd_set_decode_splits", self.lib.spd_set_decode_splits(self._ctx, qkv, o_proj, gate_up, down))
+    def set_tuning(self, **kw: int):
+        """Tuning knobs of the decode step, e.g. ``set_tuning(qkv_splits=4, l2_prefetch_blocks=8)``;
+        see spd_set_tuning."""
+        for k, v in kw.items():
+            _check("spd_set_tuning", self.lib.spd_set_tuning(self._ctx, k.encode(), int(v)))
 
     def sync_points(self) -> int:
         return self.lib.spd_sync_points(self._ctx)

@@ -163,6 +163,10 @@ struct AttnArgs {
     int *counters;          // [B][nq] zero-initialised arrival counters (split merge)
     int *err;
 };
+// Paged decode attention with 16-token pages: query heads per thread block for a GQA group
+// size, and the most pages one block may be given (the host picks splits accordingly).
+constexpr int DECODE_MAX_PAGES_PER_BLOCK = 512;
+inline int decode_heads_per_block(int group) { return group % 4 == 0 ? 4 : (group % 2 == 0 ? 2 : 1); }
 template <typename T> cudaError_t launch_prefill_attention(const AttnArgs &a, cudaStream_t st);
 template <typename T> cudaError_t launch_decode_attention(const AttnArgs &a, cudaStream_t st);
 

@@ -327,18 +327,27 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
             asm volatile("prefetch.tensormap [%0];" ::"l"(tm_w) : "memory");
             if (SUB == 2) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_w1) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_t) : "memory");
+            const uint64_t stream_once = policy_evict_first();
             auto load_w = [&](int s, int kx) {
                 const uint32_t sa = base + s * C::STAGE_BYTES;
-                if (SUB == 1) tma_load_3d(sa, tm_w, kx, t.w_row0, a_z, full_bar(s));
+                if (SUB == 1) tma_load_3d_hint(sa, tm_w, kx, t.w_row0, a_z, full_bar(s), stream_once);
                 else {
-                    tma_load_3d(sa, &tm_w0, kx, t.w_row0, a_z, full_bar(s));
-                    tma_load_3d(sa + ROWS * BK * 2, &tm_w1, kx, t.w_row0, a_z, full_bar(s));
+                    tma_load_3d_hint(sa, &tm_w0, kx, t.w_row0, a_z, full_bar(s), stream_once);
+                    tma_load_3d_hint(sa + ROWS * BK * 2, &tm_w1, kx, t.w_row0, a_z, full_bar(s), stream_once);
                 }
             };
             const int pre = n_kb < C::STAGES ? n_kb : C::STAGES;
             for (int i = 0; i < pre; ++i) {
                 mbar_expect_tx(full_bar(i), C::STAGE_BYTES);
                 load_w(i, (kb_begin + i) * BK);
+            }
+            // ... and the K blocks after the ring are pulled into L2, so that HBM keeps
+            // streaming this GEMM's weights while the preceding kernel drains.
+            const int pf_end = n_kb < pre + g.l2_prefetch_kb ? n_kb : pre + g.l2_prefetch_kb;
+            for (int i = pre; i < pf_end; ++i) {
+                const int kx = (kb_begin + i) * BK;
+                if (SUB == 1) tma_prefetch_l2_3d(tm_w, kx, t.w_row0, a_z);
+                else { tma_prefetch_l2_3d(&tm_w0, kx, t.w_row0, a_z); tma_prefetch_l2_3d(&tm_w1, kx, t.w_row0, a_z); }
             }
             pdl_wait();
             SPD_TRACE_EVENT(EPI, TR_DEP_DONE);
@@ -442,6 +451,9 @@ cudaError_t launch_cfg(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(gemm_decode_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(gemm_decode_kernel<BN, EPI>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 (int)cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }

@@ -36,6 +36,7 @@ struct DecGemmArgs {
     int w_rows[3];         // valid rows per batch of weight i
     int n_weights;
     int z_is_plane;        // o_proj: batch z is a K range of the same output tile (the K slice of shard z)
+    int l2_prefetch_kb;    // K blocks of weights per thread block pulled into L2 before the dependency wait
     int *err;
     // ---- epilogue operands -----------------------------------------------------------
     SumSq ss_in;           // QKV, GATEUP: sums of squares of the GEMM input's rows

@@ -51,7 +51,7 @@ int want_splits(long tiles, int cap)
 
 enum ActBuf { AB_H = 0, AB_ATTN, AB_ATTN_SHARD, AB_ACT, AB_COUNT };
 enum Kind { K_NORM = 0, K_QKV, K_ROPE_KV, K_ATTN, K_OPROJ, K_GATE_UP, K_SILU_MUL, K_DOWN, K_ROPE_TABLE, K_COUNT };
-enum Site { SITE_QKV = 0, SITE_O, SITE_GU, SITE_DOWN, SITE_COUNT };
+enum Site { SITE_QKV = 0, SITE_O, SITE_GU, SITE_DOWN, SITE_ATTN, SITE_COUNT };
 const char *const kind_names[K_COUNT] = {"residual_rmsnorm", "gemm_qkv", "rope_kv_append", "attention", "gemm_o_proj",
                                          "gemm_gate_up", "silu_mul", "gemm_down", "rope_table"};
 
@@ -91,6 +91,7 @@ struct Ctx {
     int *err, *attn_cnt;
     float *ss_attn, *ss_mlp;     // partial row sums of squares (fused decode path)
     int split_override[SITE_COUNT];
+    int l2_prefetch_kb;          // K blocks per thread block prefetched into L2 by the decode GEMMs
     int launches_last;
     // activation tensor maps, by buffer and token box (16, 32, 64, 128), built on first use
     TcMap act_maps[AB_COUNT][4];
@@ -127,7 +128,7 @@ size_t esize(const spd_dims &d) { return d.dtype == 0 ? 4 : 2; }
 
 // M = tokens of the launch.  decode: few tokens, the weight-streaming GEMMs are cut along K so
 // that about two CTAs per SM are in flight; prefill: no K splits.
-Plan make_plan(const spd_dims &d, int M, bool decode, int max_context)
+Plan make_plan(const spd_dims &d, int M, bool decode, int max_context, int attn_override = 0)
 {
     Plan p{};
     const int H = d.hidden, qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, F = d.ffn, T = d.T;
@@ -153,14 +154,15 @@ Plan make_plan(const spd_dims &d, int M, bool decode, int max_context)
     p.o_kps = qd / (T * p.o_per_group);
     p.attn_splits = 1;
     if (decode) {
-        // decode attention: short dependent chains - about 128 tokens per CTA (one or two
-        // 16-token chunks per warp) - within 16 CTAs per SM and 32 splits
-        const int gt = (d.n_q_heads / d.n_kv_heads) % 4 == 0 ? 4 : ((d.n_q_heads / d.n_kv_heads) % 2 == 0 ? 2 : 1);
+        // decode attention: up to four thread blocks per SM, at least four 16-token pages each
+        const int gt = decode_heads_per_block(d.n_q_heads / d.n_kv_heads);
         const long ctas = (long)M * (d.n_q_heads / gt);
-        int s = cdiv(max_context, 128);
-        const long smax = (16L * N_SM + ctas - 1) / ctas;
-        if (s > smax) s = (int)smax;
+        const int pages = cdiv(max_context, 16);
+        int s = attn_override > 0 ? attn_override : (int)((4L * N_SM) / ctas);
+        if (s < 1) s = 1;
+        if (s > pages / 4) s = pages / 4;
         if (s > 32) s = 32;
+        if (s < cdiv(pages, DECODE_MAX_PAGES_PER_BLOCK)) s = cdiv(pages, DECODE_MAX_PAGES_PER_BLOCK);
         p.attn_splits = s < 1 ? 1 : s;
     }
     return p;
@@ -443,7 +445,7 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
     const int H = d.hidden, qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, F = d.ffn, Tn = d.T;
     const int Fs = F / Tn;
     const long Mc = c->Mcap;
-    const Plan p = make_plan(d, M, true, max_context);
+    const Plan p = make_plan(d, M, true, max_context, c->split_override[SITE_ATTN]);
     PageTable pt{bt, max_pages, c->n_pages, d.kv_block_size, d.n_kv_heads};
     const int tbox = tc_token_box(true, M);
     const int tok_tiles = cdiv(M, tbox), h_tiles = cdiv(H, 128);
@@ -464,6 +466,7 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
     auto base_args = [&]() {
         DecGemmArgs g{};
         g.t_rows = M; g.err = c->err; g.H = H; g.Mcap = Mc; g.batches = 1; g.n_weights = 1; g.n_groups = 1;
+        g.l2_prefetch_kb = c->l2_prefetch_kb;
         return g;
     };
     for (int l = 0; l < d.n_layers; ++l) {
@@ -626,6 +629,7 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     c.attn_cnt = (int *)(c.ws + L.attn_cnt);
     c.ss_attn = (float *)(c.ws + L.ss_attn); c.ss_mlp = (float *)(c.ws + L.ss_mlp);
     for (int i = 0; i < SITE_COUNT; ++i) c.split_override[i] = 0;
+    c.l2_prefetch_kb = 0;
     c.launches_last = 0;
     c.use_graphs = true;
     c.graph_clock = 0;
@@ -743,14 +747,18 @@ int spd_set_graphs(spd_ctx *ctx, int32_t enabled)
     return SPD_OK;
 }
 
-int spd_set_decode_splits(spd_ctx *ctx, int32_t qkv, int32_t o_proj, int32_t gate_up, int32_t down)
+int spd_set_tuning(spd_ctx *ctx, const char *key, int32_t value)
 {
-    if (!ctx) return SPD_ENULL;
-    if (qkv < 0 || o_proj < 0 || gate_up < 0 || down < 0) return SPD_EINVAL;
+    if (!ctx || !key) return SPD_ENULL;
+    if (value < 0) return SPD_EINVAL;
     Ctx &c = ctx->c;
-    c.split_override[SITE_QKV] = qkv; c.split_override[SITE_O] = o_proj;
-    c.split_override[SITE_GU] = gate_up; c.split_override[SITE_DOWN] = down;
-    for (GraphEntry &g : c.graphs) cudaGraphExecDestroy(g.exec); // captured steps used the old cuts
+    static const char *const site_keys[SITE_COUNT] = {"qkv_splits", "o_proj_splits", "gate_up_splits", "down_splits", "attention_splits"};
+    bool found = false;
+    for (int i = 0; i < SITE_COUNT; ++i)
+        if (!strcmp(key, site_keys[i])) { c.split_override[i] = value; found = true; }
+    if (!strcmp(key, "l2_prefetch_blocks")) { c.l2_prefetch_kb = value > 64 ? 64 : value; found = true; }
+    if (!found) return SPD_EINVAL;
+    for (GraphEntry &g : c.graphs) cudaGraphExecDestroy(g.exec); // captured steps used the old setting
     c.graphs.clear();
     return SPD_OK;
 }
