@@ -94,9 +94,242 @@ __global__ void __launch_bounds__(128) prefill_attention_kernel(AttnArgs a)
     for (int i = 0; i < VEC; ++i) out[i] = from_f<T>(o[i] * inv);
 }
 
+// ---------------------------------------------------------------------------------------
+// Causal prefill attention on tensor cores (bf16): one thread block per 64 query rows of one
+// (sequence, query head); K/V tiles of 64 cached tokens are gathered from their pages into
+// double-buffered, XOR-swizzled shared memory with cp.async; each of the 4 warps owns 16 query
+// rows: S = Q K^T and O += P V as m16n8k16 MMAs with fp32 accumulators, online softmax in
+// base 2 on the accumulator fragments, P re-used in registers as the A operand of the second
+// product.  Chunked prefill: queries at positions s0.. attend to every cached position <= their own.
+namespace fa {
+
+constexpr int BQ = 64, BKV = 64;
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid)
+{
+    const int n = valid ? 16 : 0; // 0 source bytes: the 16 destination bytes are zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *(uint32_t *)&v;
+}
+// byte offset of 16-byte chunk `c` of row `r` in a [rows][D] bf16 tile (chunks XOR-swizzled by row)
+template <int D> __device__ __forceinline__ uint32_t tile_off(int r, int c) { return (uint32_t)(r * D * 2 + ((c ^ (r & 7)) << 4)); }
+
+template <int D>
+__global__ void __launch_bounds__(128) prefill_attention_mma_kernel(AttnArgs a)
+{
+    constexpr int CH = D / 8;       // 16-byte chunks per row
+    constexpr int KS = D / 16;      // k-steps of Q K^T
+    constexpr int NT = BKV / 8;     // n-tiles of S
+    constexpr int DT = D / 8;       // n-tiles of O
+    extern __shared__ __align__(128) uint8_t fa_smem[];
+    const uint32_t sQ = tc::smem_u32(fa_smem), sK = sQ + BQ * D * 2, sV = sK + 2 * BKV * D * 2;
+    pdl_launch_dependents();
+    pdl_wait();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
+    const int q0 = blockIdx.x * BQ, hq = blockIdx.y, bi = blockIdx.z;
+    const int ns = a.tm.ns, s0 = a.tm.s0, b = a.tm.b0 + bi;
+    const int kvh = hq / (a.n_q_heads / a.pt.n_kv_heads);
+    const int q_rows = min(BQ, ns - q0);
+    const int kv_len = s0 + q0 + q_rows;                 // keys 0 .. last query position of the tile
+    const int n_tiles = (kv_len + BKV - 1) / BKV;
+    const bf16 *kp = (const bf16 *)a.k_pages, *vp = (const bf16 *)a.v_pages;
+
+    auto load_kv = [&](int tile, int buf) {
+        const uint32_t dK = sK + buf * BKV * D * 2, dV = sV + buf * BKV * D * 2;
+#pragma unroll
+        for (int i = 0; i < BKV * CH / 128; ++i) {
+            const int idx = tid + i * 128, r = idx / CH, c = idx % CH, tkn = tile * BKV + r;
+            const bool valid = tkn < kv_len;
+            long off = 0;
+            if (valid) {
+                int page = a.pt.block_table[(long)b * a.pt.max_pages + tkn / a.pt.block];
+                if (page < 0 || page >= a.pt.n_pages) { atomicOr(a.err, ERR_PAGE_RANGE); page = 0; }
+                off = (((long)page * a.pt.n_kv_heads + kvh) * a.pt.block + tkn % a.pt.block) * D + c * 8;
+            }
+            cp_async16(dK + tile_off<D>(r, c), kp + off, valid);
+            cp_async16(dV + tile_off<D>(r, c), vp + off, valid);
+        }
+    };
+    // Q tile
+#pragma unroll
+    for (int i = 0; i < BQ * CH / 128; ++i) {
+        const int idx = tid + i * 128, r = idx / CH, c = idx % CH;
+        const bool valid = r < q_rows;
+        const bf16 *src = (const bf16 *)a.q + ((long)(bi * ns + q0 + (valid ? r : 0)) * a.n_q_heads + hq) * D + c * 8;
+        cp_async16(sQ + tile_off<D>(r, c), src, valid);
+    }
+    cp_async_commit();
+    load_kv(0, 0);
+    cp_async_commit();
+    cp_async_wait<1>();
+    __syncthreads();
+    // A fragments of this warp's 16 query rows
+    uint32_t qf[KS][4];
+#pragma unroll
+    for (int kk = 0; kk < KS; ++kk) {
+        const int r = warp * 16 + (lane & 15), c = kk * 2 + (lane >> 4);
+        ldsm_x4(qf[kk], sQ + tile_off<D>(r, c));
+    }
+    float o[DT][4];
+#pragma unroll
+    for (int i = 0; i < DT; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    const float sc = rsqrtf((float)D) * 1.4426950408889634f;
+    // positions of this thread's two rows (g and g + 8 of the warp's 16); -1 for rows past the tile
+    int pos_q[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int r = warp * 16 + g + 8 * h;
+        pos_q[h] = r < q_rows ? s0 + q0 + r : -1;
+    }
+    for (int j = 0; j < n_tiles; ++j) {
+        const int buf = j & 1;
+        if (j + 1 < n_tiles) load_kv(j + 1, buf ^ 1);
+        cp_async_commit();
+        cp_async_wait<1>();
+        __syncthreads();
+        const uint32_t bK = sK + buf * BKV * D * 2, bV = sV + buf * BKV * D * 2;
+        float s[NT][4];
+#pragma unroll
+        for (int i = 0; i < NT; ++i) { s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f; }
+#pragma unroll
+        for (int kk = 0; kk < KS; ++kk) {
+#pragma unroll
+            for (int np = 0; np < NT / 2; ++np) {
+                // matrices: (tokens np*16 + 0..7, dims kk*16 + 0..7), (same tokens, dims + 8), (tokens + 8, dims), (tokens + 8, dims + 8)
+                uint32_t kf[4];
+                const int r = np * 16 + (lane & 7) + ((lane >> 4) << 3), c = kk * 2 + ((lane >> 3) & 1);
+                ldsm_x4(kf, bK + tile_off<D>(r, c));
+                mma_bf16(s[2 * np], qf[kk], kf[0], kf[1]);
+                mma_bf16(s[2 * np + 1], qf[kk], kf[2], kf[3]);
+            }
+        }
+        // scale, causal mask, running max
+        float m_new[2] = {m_run[0], m_run[1]};
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int key = j * BKV + nt * 8 + 2 * t4 + (e & 1), h = e >> 1;
+                const float v = key <= pos_q[h] ? s[nt][e] * sc : -INFINITY;
+                s[nt][e] = v;
+                m_new[h] = fmaxf(m_new[h], v);
+            }
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            m_new[h] = fmaxf(m_new[h], __shfl_xor_sync(0xffffffffu, m_new[h], 1));
+            m_new[h] = fmaxf(m_new[h], __shfl_xor_sync(0xffffffffu, m_new[h], 2));
+        }
+        float corr[2], base[2], rs[2] = {0.f, 0.f};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            base[h] = m_new[h] == -INFINITY ? 0.f : m_new[h];
+            corr[h] = m_run[h] == -INFINITY ? 0.f : exp2f(m_run[h] - base[h]);
+            m_run[h] = m_new[h];
+        }
+        uint32_t pf[NT / 2][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            float p[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                p[e] = exp2f(s[nt][e] - base[e >> 1]);
+                rs[e >> 1] += p[e];
+            }
+            // accumulator layout of two adjacent n-tiles = A layout of one 16-wide k-step
+            pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p[0], p[1]);
+            pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p[2], p[3]);
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) l_run[h] = l_run[h] * corr[h] + rs[h];
+#pragma unroll
+        for (int dt = 0; dt < DT; ++dt) { o[dt][0] *= corr[0]; o[dt][1] *= corr[0]; o[dt][2] *= corr[1]; o[dt][3] *= corr[1]; }
+#pragma unroll
+        for (int k2 = 0; k2 < BKV / 16; ++k2) {
+#pragma unroll
+            for (int dp = 0; dp < DT / 2; ++dp) {
+                // transposed loads: (tokens k2*16 + 0..7, dims dp*16 + 0..7), (tokens + 8, dims), (tokens, dims + 8), (tokens + 8, dims + 8)
+                uint32_t vf[4];
+                const int r = k2 * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), c = dp * 2 + (lane >> 4);
+                ldsm_x4_t(vf, bV + tile_off<D>(r, c));
+                mma_bf16(o[2 * dp], pf[k2], vf[0], vf[1]);
+                mma_bf16(o[2 * dp + 1], pf[k2], vf[2], vf[3]);
+            }
+        }
+        __syncthreads(); // this buffer is refilled two iterations from now
+    }
+    // row sums across the quad, normalise, store
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        l_run[h] += __shfl_xor_sync(0xffffffffu, l_run[h], 1);
+        l_run[h] += __shfl_xor_sync(0xffffffffu, l_run[h], 2);
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int r = warp * 16 + g + 8 * h;
+        if (r >= q_rows) continue;
+        const float inv = l_run[h] > 0.f ? 1.f / l_run[h] : 0.f;
+        bf16 *dst = (bf16 *)a.out + ((long)(bi * ns + q0 + r) * a.n_q_heads + hq) * D;
+#pragma unroll
+        for (int dt = 0; dt < DT; ++dt)
+            *(uint32_t *)(dst + dt * 8 + 2 * t4) = pack_bf16(o[dt][2 * h] * inv, o[dt][2 * h + 1] * inv);
+    }
+}
+
+template <int D> cudaError_t launch(const AttnArgs &a, int n_seq, cudaStream_t st)
+{
+    constexpr int SMEM = (BQ + 4 * BKV) * D * 2;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(prefill_attention_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    dim3 grid((a.tm.ns + BQ - 1) / BQ, a.n_q_heads, n_seq);
+    return launch_kernel(prefill_attention_mma_kernel<D>, grid, dim3(128), SMEM, st, 0, a);
+}
+
+} // namespace fa
+
+template <typename T> cudaError_t launch_prefill_attention_tc(const AttnArgs &, cudaStream_t, bool &done) { done = false; return cudaSuccess; }
+template <> cudaError_t launch_prefill_attention_tc<bf16>(const AttnArgs &a, cudaStream_t st, bool &done)
+{
+    done = false;
+    if (a.tm.decode || a.tm.ns <= 0 || a.M % a.tm.ns) return cudaSuccess;
+    done = true;
+    switch (a.head_dim) {
+    case 128: return fa::launch<128>(a, a.M / a.tm.ns, st);
+    case 64: return fa::launch<64>(a, a.M / a.tm.ns, st);
+    default: done = false; return cudaSuccess;
+    }
+}
+
 template <typename T> cudaError_t launch_prefill_attention(const AttnArgs &a, cudaStream_t st)
 {
     if (a.M <= 0) return cudaSuccess;
+    bool done = false;
+    cudaError_t e = launch_prefill_attention_tc<T>(a, st, done);
+    if (done || e != cudaSuccess) return e;
     dim3 grid((a.M + 3) / 4, a.n_q_heads);
     switch (a.head_dim) {
     case 128: return launch_kernel(prefill_attention_kernel<T, 4>, grid, dim3(128), 0, st, 0, a);
