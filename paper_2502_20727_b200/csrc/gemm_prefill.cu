@@ -1,0 +1,528 @@
+// Fused prefill projections.  With thousands of tokens in flight the projections are bound by
+// the tensor cores, so each is one persistent tcgen05 GEMM: one thread block per SM walks the
+// output tiles (128 tokens x 256 weight rows), a TMA warp keeps a shared-memory ring of
+// K blocks full, an MMA warp accumulates into one of two tensor-memory buffers, and the four
+// epilogue warps drain the other buffer meanwhile - applying the step that follows the
+// projection to the fp32 accumulator (thread = token row), so nothing but the next operand
+// (bf16) and the fp32 residual stream goes to memory.
+//
+//   PRE_QKV       : attention-RMSNorm rstd, rotary embedding, q store, K/V page append   (a2, a3)
+//   PRE_RESID     : sync block o_proj (R = X + sum_i Y_i as ONE GEMM over all of K) and down
+//                   (sum_i Z_i likewise): residual add, gain-scaled next operand, sums of squares
+//   PRE_GATEUP    : MLP-RMSNorm rstd (per emulated device in an SPD block), SwiGLU       (a8)
+//   PRE_OPROJ_SPD : SPD block (Sec. 4.1.1): the T K-slices of a 128 x 128 output tile in turn;
+//                   device i's pass gives Y_i, from which R_i = X + Y_i (its own MLP input) is
+//                   stored, while a third tensor-memory buffer adds up sum_i Y_i for the
+//                   residual that is carried to the block output.
+#include "gemm_prefill.cuh"
+#include "tc_ptx.cuh"
+
+namespace spd {
+
+namespace {
+
+using namespace tc;
+
+constexpr int THREADS = 192;
+constexpr int TMEM_ALL = 512;
+constexpr int TOT_COL = 256; // PRE_OPROJ_SPD: running sum of the Y_i
+
+template <int EPI> struct PCfg {
+    static constexpr int BN = (EPI == PRE_OPROJ_SPD) ? 128 : 256;
+    static constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int STAGES = (192 * 1024) / STAGE_BYTES;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+struct PreLaunch {
+    PreGemmArgs g;
+    int m_tiles, n_tiles, passes;
+    int tile_start[3]; // QKV: first n-tile of weight i
+    int f_tiles;       // GATEUP: n-tiles per device
+};
+
+struct PreTile {
+    int m0;     // first token
+    int wi;     // QKV: which weight
+    int row0;   // first weight row (QKV, RESID, OPROJ_SPD: output column; GATEUP: FFN column within the device)
+    int z;      // GATEUP: device
+    int nt;     // n-tile index (for the sums of squares)
+};
+
+__device__ __forceinline__ PreTile decode_tile(const PreLaunch &L, int EPI, int tile)
+{
+    PreTile t;
+    const int mt = tile % L.m_tiles, nt = tile / L.m_tiles;
+    t.m0 = mt * BM;
+    t.nt = nt;
+    t.wi = 0;
+    t.z = 0;
+    if (EPI == PRE_QKV) {
+        t.wi = nt >= L.tile_start[2] ? 2 : (nt >= L.tile_start[1] ? 1 : 0);
+        t.row0 = (nt - L.tile_start[t.wi]) * 256;
+    } else if (EPI == PRE_GATEUP) {
+        t.z = nt / L.f_tiles;
+        t.row0 = (nt % L.f_tiles) * 128;
+    } else if (EPI == PRE_OPROJ_SPD) {
+        t.row0 = nt * 128;
+    } else {
+        t.row0 = nt * 256;
+    }
+    return t;
+}
+
+// two 16-column accumulator chunks of this thread's row, one wait
+__device__ __forceinline__ void tmem_ld16x2(uint32_t ta, uint32_t tb, float *va, float *vb)
+{
+    uint32_t r[32];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%32];\n\t"
+                 "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%33];\n\t"
+                 "tcgen05.wait::ld.sync.aligned;"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(ta), "r"(tb)
+                 : "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { va[i] = __uint_as_float(r[i]); vb[i] = __uint_as_float(r[16 + i]); }
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float *v)
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+                 ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+                   "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+                   "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
+                   "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+                   "r"(__float_as_uint(v[15]))
+                 : "memory");
+}
+
+// 8 consecutive bf16 (16 bytes) from 8 floats
+__device__ __forceinline__ uint4 pack8(const float *v)
+{
+    __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+    __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]), d = __floats2bfloat162_rn(v[6], v[7]);
+    return make_uint4(*(uint32_t *)&a, *(uint32_t *)&b, *(uint32_t *)&c, *(uint32_t *)&d);
+}
+__device__ __forceinline__ void unpack8(uint4 u, float *v)
+{
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { v[2 * i] = __uint_as_float(w[i] << 16); v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
+}
+
+__device__ __forceinline__ float row_rstd(const SumSq &s, int group, int m)
+{
+    float acc = 0.f;
+    for (int t = 0; t < s.tiles; ++t) acc += s.part[((long)t * s.groups + group) * s.Mcap + m];
+    return rsqrtf(acc / (float)s.H + s.eps);
+}
+
+// ---- epilogues: thread = token row m, columns read from tensor memory 16 at a time ----------------
+
+__device__ __forceinline__ void epi_qkv(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, int m, bool valid)
+{
+    const int d = g.head_dim, half = d >> 1, nq = g.n_q_heads;
+    const float rs = valid ? row_rstd(g.ss_in, 0, m) : 0.f;
+    const bool rot = t.wi < 2 && g.rope != nullptr;
+    long kv_off = -1;
+    if (t.wi > 0 && valid) {
+        int b, pos;
+        g.tm.locate(m, b, pos);
+        const int pi = pos / g.pt.block;
+        if (pos < 0 || pi >= g.pt.max_pages) atomicOr(g.err, ERR_CAPACITY);
+        else {
+            const int page = g.pt.block_table[(long)b * g.pt.max_pages + pi];
+            if (page < 0 || page >= g.pt.n_pages) atomicOr(g.err, ERR_PAGE_RANGE);
+            else kv_off = ((long)page * g.pt.n_kv_heads * g.pt.block + pos % g.pt.block) * d;
+        }
+    }
+    const int heads = 256 / d;
+    for (int hh = 0; hh < heads; ++hh) {
+        const int row_h = t.row0 + hh * d;
+        if (row_h >= g.w_rows[t.wi]) break;
+        const int head = row_h / d;
+        bf16 *dst = nullptr;
+        if (valid) {
+            if (t.wi == 0) dst = (bf16 *)g.q_out + ((long)m * nq + head) * d;
+            else if (kv_off >= 0) dst = (bf16 *)(t.wi == 1 ? g.k_pages : g.v_pages) + kv_off + (long)head * g.pt.block * d;
+        }
+        for (int j0 = 0; j0 < half; j0 += 16) {
+            float lo[16], hi[16];
+            tmem_ld16x2(tacc + hh * d + j0, tacc + hh * d + half + j0, lo, hi);
+            if (!dst) continue;
+            float olo[16], ohi[16];
+            if (rot) {
+                const float4 *cs = (const float4 *)(g.rope + (long)m * half + j0);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float4 c2 = cs[i]; // cos, sin of two consecutive dims
+                    const float a0 = lo[2 * i] * rs, b0 = hi[2 * i] * rs, a1 = lo[2 * i + 1] * rs, b1 = hi[2 * i + 1] * rs;
+                    olo[2 * i] = a0 * c2.x - b0 * c2.y;
+                    ohi[2 * i] = b0 * c2.x + a0 * c2.y;
+                    olo[2 * i + 1] = a1 * c2.z - b1 * c2.w;
+                    ohi[2 * i + 1] = b1 * c2.z + a1 * c2.w;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) { olo[i] = lo[i] * rs; ohi[i] = hi[i] * rs; }
+            }
+            *(uint4 *)(dst + j0) = pack8(olo);
+            *(uint4 *)(dst + j0 + 8) = pack8(olo + 8);
+            *(uint4 *)(dst + half + j0) = pack8(ohi);
+            *(uint4 *)(dst + half + j0 + 8) = pack8(ohi + 8);
+        }
+    }
+}
+
+__device__ __forceinline__ void epi_gateup(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, int m, bool valid)
+{
+    const float rs = valid ? row_rstd(g.ss_in, g.rstd_per_shard ? t.z : 0, m) : 0.f;
+    bf16 *dst = (bf16 *)g.act + (long)m * g.F + (long)t.z * g.Fs + t.row0;
+#pragma unroll 1
+    for (int c = 0; c < 8; ++c) {
+        const int f = t.row0 + c * 16;
+        if (f >= g.Fs) break;
+        float gt[16], up[16], o[16];
+        tmem_ld16x2(tacc + c * 16, tacc + 128 + c * 16, gt, up);
+        if (!valid) continue;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const float x = gt[i] * rs;
+            o[i] = x / (1.f + __expf(-x)) * (up[i] * rs);
+        }
+        *(uint4 *)(dst + c * 16) = pack8(o);
+        if (f + 8 < g.Fs) *(uint4 *)(dst + c * 16 + 8) = pack8(o + 8);
+    }
+}
+
+// y: 16 accumulator columns at output column n.  r = x + y; stores what the arguments ask for.
+__device__ __forceinline__ float resid_chunk(const PreGemmArgs &g, long idx, int n, const float *x, const float *y, bf16 *hg,
+                                             bool store_res)
+{
+    float r[16], sq = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { r[i] = x[i] + y[i]; sq = fmaf(r[i], r[i], sq); }
+    if (store_res) {
+        if (g.res_out) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) *(float4 *)(g.res_out + idx + 4 * i) = make_float4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+        }
+        if (g.final_out) {
+            *(uint4 *)((bf16 *)g.final_out + idx) = pack8(r);
+            *(uint4 *)((bf16 *)g.final_out + idx + 8) = pack8(r + 8);
+        }
+    }
+    if (hg) {
+        float gn[16];
+        unpack8(*(const uint4 *)((const bf16 *)g.gain + n), gn);
+        unpack8(*(const uint4 *)((const bf16 *)g.gain + n + 8), gn + 8);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) gn[i] *= r[i];
+        *(uint4 *)(hg + idx) = pack8(gn);
+        *(uint4 *)(hg + idx + 8) = pack8(gn + 8);
+    }
+    return sq;
+}
+
+__device__ __forceinline__ void load_x16(const float *p, float *x)
+{
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float4 v = *(const float4 *)(p + 4 * i);
+        x[4 * i] = v.x; x[4 * i + 1] = v.y; x[4 * i + 2] = v.z; x[4 * i + 3] = v.w;
+    }
+}
+
+__device__ __forceinline__ void epi_resid(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, int m, bool valid)
+{
+    float ssq = 0.f;
+#pragma unroll 1
+    for (int c = 0; c < 16; c += 2) {
+        const int n = t.row0 + c * 16;
+        if (n >= g.H) break;
+        float ya[16], yb[16];
+        tmem_ld16x2(tacc + c * 16, tacc + c * 16 + 16, ya, yb);
+        if (!valid) continue;
+        const long idx = (long)m * g.H + n;
+        float x[16];
+        load_x16(g.res_in + idx, x);
+        ssq += resid_chunk(g, idx, n, x, ya, g.hg ? (bf16 *)g.hg : nullptr, true);
+        if (n + 16 < g.H) {
+            load_x16(g.res_in + idx + 16, x);
+            ssq += resid_chunk(g, idx + 16, n + 16, x, yb, g.hg ? (bf16 *)g.hg : nullptr, true);
+        }
+    }
+    if (valid && g.ss_out) g.ss_out[(long)t.nt * g.Mcap + m] = ssq;
+}
+
+__device__ __forceinline__ void epi_oproj_spd(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, uint32_t ttot, int z, int m, bool valid)
+{
+    const int T = g.batches;
+    float ssq = 0.f;
+#pragma unroll 1
+    for (int c = 0; c < 8; ++c) {
+        const int n = t.row0 + c * 16;
+        if (n >= g.H) break;
+        float y[16], tot[16];
+        if (z == 0) {
+            tmem_ld16(tacc + c * 16, y);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) tot[i] = y[i];
+        } else {
+            tmem_ld16x2(tacc + c * 16, ttot + c * 16, y, tot);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) tot[i] += y[i];
+        }
+        if (z + 1 < T) tmem_st16(ttot + c * 16, tot);
+        if (!valid) continue;
+        const long idx = (long)m * g.H + n;
+        float x[16];
+        load_x16(g.res_in + idx, x);
+        // device z only ever sees its own partial attention output
+        ssq += resid_chunk(g, idx, n, x, y, g.hg ? (bf16 *)g.hg + (long)z * g.hg_stride : nullptr, false);
+        if (z + 1 == T && g.res_out) {
+            // the residual carried to the block output collects every Y_i
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                *(float4 *)(g.res_out + idx + 4 * i) =
+                    make_float4(x[4 * i] + tot[4 * i], x[4 * i + 1] + tot[4 * i + 1], x[4 * i + 2] + tot[4 * i + 2], x[4 * i + 3] + tot[4 * i + 3]);
+        }
+    }
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+    if (valid && g.ss_out) g.ss_out[((long)t.nt * T + z) * g.Mcap + m] = ssq;
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(THREADS, 1) gemm_prefill_kernel(const __grid_constant__ CUtensorMap tm_w0,
+                                                                  const __grid_constant__ CUtensorMap tm_w1,
+                                                                  const __grid_constant__ CUtensorMap tm_w2,
+                                                                  const __grid_constant__ CUtensorMap tm_t,
+                                                                  const __grid_constant__ PreLaunch L)
+{
+    using C = PCfg<EPI>;
+    constexpr int BN = C::BN, S = C::STAGES;
+    const PreGemmArgs &g = L.g;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t bars = base + S * C::STAGE_BYTES; // full[S], empty[S], tmem_full[2], tmem_empty[2]
+    uint32_t *tmem_slot = (uint32_t *)(gen_base + S * C::STAGE_BYTES + 8 * (2 * S + 4));
+    volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (S + s); };
+    auto tfull_bar = [&](int b) { return bars + 8u * (2 * S + b); };
+    auto tempty_bar = [&](int b) { return bars + 8u * (2 * S + 2 + b); };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int total_tiles = L.m_tiles * L.n_tiles;
+
+    pdl_launch_dependents();
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_ALL) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();
+
+    if (warp == 4) {
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_w0) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_t) : "memory");
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const PreTile t = decode_tile(L, EPI, tile);
+                const CUtensorMap *tm_w = t.wi == 0 ? &tm_w0 : (t.wi == 1 ? &tm_w1 : &tm_w2);
+                for (int pass = 0; pass < L.passes && ok; ++pass) {
+                    const int tz = EPI == PRE_OPROJ_SPD ? pass : (EPI == PRE_GATEUP && g.t_batched ? t.z : 0);
+                    const int wz = EPI == PRE_OPROJ_SPD ? pass : t.z;
+                    for (int kb = 0; kb < g.num_kb; ++kb, ++it) {
+                        const int s = it % S;
+                        if (!mbar_wait(empty_bar(s), ((it / S) & 1) ^ 1, g.err, abort_flag)) { ok = false; break; }
+                        mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
+                        const uint32_t sa = base + s * C::STAGE_BYTES, sb = sa + C::A_BYTES;
+                        tma_load_3d(sa, &tm_t, kb * BK, t.m0, tz, full_bar(s));
+                        if (EPI == PRE_GATEUP) {
+                            tma_load_3d(sb, &tm_w0, kb * BK, t.row0, wz, full_bar(s));
+                            tma_load_3d(sb + 128 * BK * 2, &tm_w1, kb * BK, t.row0, wz, full_bar(s));
+                        } else {
+                            tma_load_3d(sb, tm_w, kb * BK, t.row0, wz, full_bar(s));
+                        }
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 5) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(BN);
+            uint32_t it = 0, pc = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                for (int pass = 0; pass < L.passes && ok; ++pass, ++pc) {
+                    const int buf = pc & 1;
+                    if (!mbar_wait(tempty_bar(buf), ((pc >> 1) & 1) ^ 1, g.err, abort_flag)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t tacc = tmem_base + (uint32_t)(buf * BN);
+                    for (int kb = 0; kb < g.num_kb; ++kb, ++it) {
+                        const int s = it % S;
+                        if (!mbar_wait(full_bar(s), (it / S) & 1, g.err, abort_flag)) { ok = false; break; }
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        const uint32_t sa = base + s * C::STAGE_BYTES, sb = sa + C::A_BYTES;
+                        const uint64_t da = make_desc(sa), db = make_desc(sb);
+#pragma unroll
+                        for (int k = 0; k < BK / UMMA_K; ++k)
+                            umma(tacc, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
+                                 (kb > 0 || k > 0) ? 1u : 0u);
+                        umma_commit(empty_bar(s));
+                    }
+                    if (ok) umma_commit(tfull_bar(buf));
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        uint32_t pc = 0;
+        bool ok = true;
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            const PreTile t = decode_tile(L, EPI, tile);
+            const int m = t.m0 + warp * 32 + lane;
+            const bool valid = m < g.t_rows;
+            for (int pass = 0; pass < L.passes; ++pass, ++pc) {
+                const int buf = pc & 1;
+                if (!mbar_wait(tfull_bar(buf), (pc >> 1) & 1, g.err, abort_flag)) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tacc = tmem_base + lane_base + (uint32_t)(buf * BN);
+                if (EPI == PRE_QKV) epi_qkv(g, t, tacc, m, valid);
+                else if (EPI == PRE_GATEUP) epi_gateup(g, t, tacc, m, valid);
+                else if (EPI == PRE_RESID) epi_resid(g, t, tacc, m, valid);
+                else epi_oproj_spd(g, t, tacc, tmem_base + lane_base + TOT_COL, pass, m, valid);
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(tempty_bar(buf)) : "memory");
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 5) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_ALL) : "memory");
+    }
+}
+
+template <int EPI>
+cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, const PreLaunch &L, cudaStream_t st)
+{
+    using C = PCfg<EPI>;
+    static int n_sm = 0;
+    if (!n_sm) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_prefill_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        int dev = 0, n = 0;
+        if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+        if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        n_sm = n;
+    }
+    const int total = L.m_tiles * L.n_tiles;
+    const dim3 grid(total < n_sm ? total : n_sm);
+    return launch_kernel(gemm_prefill_kernel<EPI>, grid, dim3(THREADS), C::SMEM_BYTES, st, 0, *tw[0], *tw[1], *tw[2], tt, L);
+}
+
+// One thread block per token: whole-row sum of squares in one partial.
+__global__ void __launch_bounds__(256) prefill_prologue_kernel(PrologueArgs a)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    __shared__ float red[8];
+    const int m = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float sq = 0.f;
+    for (int n = threadIdx.x * 8; n < a.H; n += blockDim.x * 8) {
+        const long idx = (long)m * a.H + n;
+        float x[8], gn[8];
+        unpack8(*(const uint4 *)((const bf16 *)a.x + idx), x);
+        unpack8(*(const uint4 *)((const bf16 *)a.gain + n), gn);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { sq = fmaf(x[i], x[i], sq); gn[i] *= x[i]; }
+        *(float4 *)(a.res_out + idx) = make_float4(x[0], x[1], x[2], x[3]);
+        *(float4 *)(a.res_out + idx + 4) = make_float4(x[4], x[5], x[6], x[7]);
+        *(uint4 *)((bf16 *)a.hg + idx) = pack8(gn);
+    }
+    sq = warp_sum(sq);
+    if (lane == 0) red[warp] = sq;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float tot = 0.f;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];
+        a.ss_out[m] = tot;
+    }
+}
+
+} // namespace
+
+int pre_ss_tiles(PreEpilogue epi, int H) { return epi == PRE_OPROJ_SPD ? (H + 127) / 128 : (H + 255) / 256; }
+
+cudaError_t launch_gemm_prefill(PreEpilogue epi, const TcMap *const *weights, const TcMap &tokens, const PreGemmArgs &g,
+                                cudaStream_t st)
+{
+    const int nw = g.n_weights;
+    if (nw < 1 || nw > 3 || (epi == PRE_GATEUP && nw != 2)) return cudaErrorInvalidValue;
+    if (g.t_rows <= 0) return cudaSuccess;
+    if (g.num_kb < 1 || g.batches < 1 || g.batches > 8) return cudaErrorInvalidValue;
+    if (epi == PRE_QKV && (256 % g.head_dim || g.head_dim < 32)) return cudaErrorInvalidValue;
+    if ((epi == PRE_RESID || epi == PRE_OPROJ_SPD) && g.H % 16) return cudaErrorInvalidValue;
+    if (epi == PRE_GATEUP && g.Fs % 8) return cudaErrorInvalidValue;
+    const CUtensorMap *tw[3];
+    for (int i = 0; i < 3; ++i) tw[i] = (const CUtensorMap *)weights[i < nw ? i : 0];
+    PreLaunch L;
+    L.g = g;
+    L.m_tiles = (g.t_rows + BM - 1) / BM;
+    L.passes = 1;
+    L.f_tiles = 1;
+    for (int i = 0; i < 3; ++i) L.tile_start[i] = 1 << 30;
+    switch (epi) {
+    case PRE_QKV: {
+        int tiles = 0;
+        for (int i = 0; i < nw; ++i) {
+            if (g.w_rows[i] <= 0) return cudaErrorInvalidValue;
+            L.tile_start[i] = tiles;
+            tiles += (g.w_rows[i] + 255) / 256;
+        }
+        L.n_tiles = tiles;
+        return launch_epi<PRE_QKV>(tw, *(const CUtensorMap *)&tokens, L, st);
+    }
+    case PRE_GATEUP:
+        L.f_tiles = (g.Fs + 127) / 128;
+        L.n_tiles = L.f_tiles * g.batches;
+        return launch_epi<PRE_GATEUP>(tw, *(const CUtensorMap *)&tokens, L, st);
+    case PRE_OPROJ_SPD:
+        L.n_tiles = (g.H + 127) / 128;
+        L.passes = g.batches;
+        return launch_epi<PRE_OPROJ_SPD>(tw, *(const CUtensorMap *)&tokens, L, st);
+    default:
+        L.n_tiles = (g.H + 255) / 256;
+        return launch_epi<PRE_RESID>(tw, *(const CUtensorMap *)&tokens, L, st);
+    }
+}
+
+cudaError_t launch_prefill_prologue(const PrologueArgs &a, cudaStream_t st)
+{
+    if (a.M <= 0) return cudaSuccess;
+    if (a.H % 8) return cudaErrorInvalidValue;
+    return launch_kernel(prefill_prologue_kernel, dim3(a.M), dim3(256), 0, st, 0, a);
+}
+
+} // namespace spd

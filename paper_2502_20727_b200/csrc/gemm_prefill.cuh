@@ -1,0 +1,61 @@
+// Host interface of the fused prefill projections (gemm_prefill.cu): persistent tcgen05 GEMMs
+// with many tokens on the 128-row MMA side and the step that follows each projection applied
+// straight from tensor memory.
+#pragma once
+#include "common.cuh"
+#include "gemm_decode.cuh"
+#include "gemm_tc.cuh"
+
+namespace spd {
+
+enum PreEpilogue {
+    PRE_QKV = 0,       // a2 + a3: rstd, rotary embedding, q store, K/V page append
+    PRE_RESID = 1,     // sync o_proj (a5-a7) and down (a9, a10): residual add, next norm's input and sums of squares
+    PRE_GATEUP = 2,    // a8: rstd (per emulated device in an SPD block), SwiGLU
+    PRE_OPROJ_SPD = 3, // a5-a7 of an SPD block: the T K-slices of one output tile in turn, R_i = X + Y_i kept apart
+};
+
+struct PreGemmArgs {
+    int t_rows;          // tokens of this launch
+    int num_kb;          // 64-wide K blocks (per shard slice where the operands are batched)
+    int batches;         // emulated devices: column blocks for GATEUP, K slices for OPROJ_SPD
+    int t_batched;       // GATEUP in an SPD block: device z reads token-operand plane z
+    int w_rows[3];       // valid rows (per device for GATEUP) of weight i
+    int n_weights;
+    int *err;
+    SumSq ss_in;         // QKV, GATEUP
+    int rstd_per_shard;
+    // QKV
+    const float2 *rope;  // [tokens][d/2] cos,sin or null
+    void *q_out;         // bf16 [tokens][nq*d]
+    void *k_pages, *v_pages;
+    PageTable pt;
+    TokMap tm;
+    int n_q_heads, head_dim;
+    // RESID, OPROJ_SPD
+    const float *res_in; // fp32 [tokens][H]
+    float *res_out;      // fp32 [tokens][H]
+    const void *gain;    // bf16 [H] or null
+    void *hg;            // bf16 [groups][Mcap][H]
+    long hg_stride;
+    float *ss_out;       // [tiles][groups][Mcap]; tiles = pre_ss_tiles(epilogue, H)
+    long Mcap;
+    void *final_out;     // bf16 [tokens][H] or null
+    int H;
+    // GATEUP
+    void *act;           // bf16 [tokens][F]
+    int F, Fs;
+};
+
+// Weight maps: 256-row boxes (QKV, RESID), 128-row boxes (GATEUP: gate and up; OPROJ_SPD: the
+// shard-sliced W_O).  Token map: 128-row box.
+cudaError_t launch_gemm_prefill(PreEpilogue epi, const TcMap *const *weights, const TcMap &tokens, const PreGemmArgs &g,
+                                cudaStream_t st);
+
+// Column tiles (= partial sums of squares per token) the residual epilogues write.
+int pre_ss_tiles(PreEpilogue epi, int H);
+
+// Block input -> fp32 residual stream, x * gain, whole-row sum of squares (one tile).
+cudaError_t launch_prefill_prologue(const PrologueArgs &a, cudaStream_t st);
+
+} // namespace spd

@@ -4,6 +4,7 @@
 #include "common.cuh"
 #include "gemm_tc.cuh"
 #include "gemm_decode.cuh"
+#include "gemm_prefill.cuh"
 
 #include <math.h>
 #include <new>
@@ -55,7 +56,7 @@ enum Site { SITE_QKV = 0, SITE_O, SITE_GU, SITE_DOWN, SITE_ATTN, SITE_COUNT };
 const char *const kind_names[K_COUNT] = {"residual_rmsnorm", "gemm_qkv", "rope_kv_append", "attention", "gemm_o_proj",
                                          "gemm_gate_up", "silu_mul", "gemm_down", "rope_table"};
 
-struct LayerMaps { TcMap wq, wk, wv, wo_full, wo_shard, w_gate, w_up, w_down, w_gate64, w_up64; };
+struct LayerMaps { TcMap wq, wk, wv, wo_full, wo_shard, w_gate, w_up, w_down, w_gate64, w_up64, wq256, wk256, wv256, wo256, wd256; };
 
 // A captured decode step is valid for exactly these arguments.
 struct GraphKey {
@@ -532,6 +533,97 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
     return SPD_OK;
 }
 
+// One prefill chunk of the bf16 stack with the fused projections (same five kernels per block as
+// a decode step, in their many-token form).
+int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t *bt, int max_pages,
+                      int max_context, cudaStream_t st)
+{
+    const spd_dims &d = c->d;
+    const int H = d.hidden, qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, F = d.ffn, Tn = d.T;
+    const int Fs = F / Tn;
+    const long Mc = c->Mcap;
+    PageTable pt{bt, max_pages, c->n_pages, d.kv_block_size, d.n_kv_heads};
+    int launches = 0;
+    const bool rope = d.rope_base > 0.f;
+    if (rope) LAUNCH(K_ROPE_TABLE, launch_rope_table(c->rope, tm, M, d.head_dim, d.rope_base, st));
+    {
+        PrologueArgs a{};
+        a.x = x; a.res_out = c->res[0]; a.gain = c->layers[0].attn_norm; a.hg = c->h; a.ss_out = c->ss_attn;
+        a.Mcap = Mc; a.M = M; a.H = H;
+        LAUNCH(K_NORM, launch_prefill_prologue(a, st));
+    }
+    int attn_tiles = 1; // partial sums of squares per token in ss_attn
+    auto base_args = [&]() {
+        PreGemmArgs g{};
+        g.t_rows = M; g.err = c->err; g.H = H; g.Mcap = Mc; g.batches = 1; g.n_weights = 1;
+        return g;
+    };
+    for (int l = 0; l < d.n_layers; ++l) {
+        const spd_layer &w = c->layers[l];
+        const bool sync = c->mask[l] != 0;
+        {   // a2 + a3
+            PreGemmArgs g = base_args();
+            const TcMap *wmaps[3] = {&c->maps[l].wq256, &c->maps[l].wk256, &c->maps[l].wv256};
+            MAP_OR_FAIL(am, act_map(c, AB_H, 128));
+            g.n_weights = 3; g.w_rows[0] = qd; g.w_rows[1] = g.w_rows[2] = kd;
+            g.num_kb = cdiv(H, 64);
+            g.ss_in = SumSq{c->ss_attn, attn_tiles, 1, Mc, H, d.rms_eps};
+            g.rope = rope ? c->rope : nullptr; g.q_out = c->q; g.k_pages = w.k_pages; g.v_pages = w.v_pages; g.pt = pt; g.tm = tm;
+            g.n_q_heads = d.n_q_heads; g.head_dim = d.head_dim;
+            LAUNCH(K_QKV, launch_gemm_prefill(PRE_QKV, wmaps, *am, g, st));
+        }
+        {   // a4
+            AttnArgs a{};
+            a.q = c->q; a.k_pages = w.k_pages; a.v_pages = w.v_pages; a.pt = pt; a.tm = tm; a.out = c->attn;
+            a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.B = M; a.splits = 1;
+            a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.counters = c->attn_cnt; a.err = c->err;
+            LAUNCH(K_ATTN, launch_prefill_attention<bf16>(a, st));
+        }
+        int mlp_tiles, mlp_groups;
+        if (sync) {   // a5 - a7, sync block: sum_i Y_i is the K accumulation over all heads
+            PreGemmArgs g = base_args();
+            const TcMap *wmaps[1] = {&c->maps[l].wo256};
+            MAP_OR_FAIL(am, act_map(c, AB_ATTN, 128));
+            g.w_rows[0] = H; g.num_kb = cdiv(qd, 64);
+            g.res_in = c->res[0]; g.res_out = c->res[1]; g.gain = w.mlp_norm; g.hg = c->h; g.hg_stride = Mc * H; g.ss_out = c->ss_mlp;
+            LAUNCH(K_OPROJ, launch_gemm_prefill(PRE_RESID, wmaps, *am, g, st));
+            mlp_tiles = pre_ss_tiles(PRE_RESID, H); mlp_groups = 1;
+        } else {      // a5 - a7, SPD block: device i's K slice gives Y_i, kept apart
+            PreGemmArgs g = base_args();
+            const TcMap *wmaps[1] = {&c->maps[l].wo_shard};
+            MAP_OR_FAIL(am, act_map(c, AB_ATTN_SHARD, 128));
+            g.w_rows[0] = H; g.num_kb = cdiv(qd / Tn, 64); g.batches = Tn;
+            g.res_in = c->res[0]; g.res_out = c->res[1]; g.gain = w.mlp_norm; g.hg = c->h; g.hg_stride = Mc * H; g.ss_out = c->ss_mlp;
+            LAUNCH(K_OPROJ, launch_gemm_prefill(PRE_OPROJ_SPD, wmaps, *am, g, st));
+            mlp_tiles = pre_ss_tiles(PRE_OPROJ_SPD, H); mlp_groups = Tn;
+        }
+        {   // a8
+            PreGemmArgs g = base_args();
+            const TcMap *wmaps[2] = {&c->maps[l].w_gate, &c->maps[l].w_up};
+            MAP_OR_FAIL(am, act_map(c, AB_H, 128));
+            g.n_weights = 2; g.w_rows[0] = g.w_rows[1] = Fs; g.batches = Tn; g.t_batched = sync ? 0 : 1;
+            g.num_kb = cdiv(H, 64);
+            g.ss_in = SumSq{c->ss_mlp, mlp_tiles, mlp_groups, Mc, H, d.rms_eps};
+            g.rstd_per_shard = sync ? 0 : 1;
+            g.act = c->act; g.F = F; g.Fs = Fs;
+            LAUNCH(K_GATE_UP, launch_gemm_prefill(PRE_GATEUP, wmaps, *am, g, st));
+        }
+        {   // a9 + a10: res[1] holds X + sum_i Y_i in both modes, so out = res[1] + sum_i Z_i
+            PreGemmArgs g = base_args();
+            const TcMap *wmaps[1] = {&c->maps[l].wd256};
+            MAP_OR_FAIL(am, act_map(c, AB_ACT, 128));
+            g.w_rows[0] = H; g.num_kb = cdiv(F, 64);
+            g.res_in = c->res[1]; g.res_out = c->res[0];
+            if (l + 1 < d.n_layers) { g.gain = c->layers[l + 1].attn_norm; g.hg = c->h; g.hg_stride = Mc * H; g.ss_out = c->ss_attn; }
+            else g.final_out = out;
+            LAUNCH(K_DOWN, launch_gemm_prefill(PRE_RESID, wmaps, *am, g, st));
+            attn_tiles = pre_ss_tiles(PRE_RESID, H);
+        }
+    }
+    c->launches_last = launches;
+    return SPD_OK;
+}
+
 int read_err_flag(Ctx *c, cudaStream_t st, int *flag)
 {
     CU_TRY(cudaMemcpyAsync(flag, c->err, sizeof(int), cudaMemcpyDeviceToHost, st));
@@ -561,6 +653,11 @@ int build_weight_maps(Ctx &c)
         rc |= make_operand_map(&m.w_gate, w.w_gate, H, F / T, T, H, (F / T) * H, 128);
         rc |= make_operand_map(&m.w_up, w.w_up, H, F / T, T, H, (F / T) * H, 128);
         rc |= make_operand_map(&m.w_down, w.w_down, F, H, 1, F, 0, 128);
+        rc |= make_operand_map(&m.wq256, w.wq, H, qd, 1, H, 0, 256);
+        rc |= make_operand_map(&m.wk256, w.wk, H, kd, 1, H, 0, 256);
+        rc |= make_operand_map(&m.wv256, w.wv, H, kd, 1, H, 0, 256);
+        rc |= make_operand_map(&m.wo256, w.wo, qd, H, 1, qd, 0, 256);
+        rc |= make_operand_map(&m.wd256, w.w_down, F, H, 1, F, 0, 256);
         rc |= make_operand_map(&m.w_gate64, w.w_gate, H, F / T, T, H, (F / T) * H, 64);
         rc |= make_operand_map(&m.w_up64, w.w_up, H, F / T, T, H, (F / T) * H, 64);
         if (rc) return SPD_EINVAL;
@@ -662,7 +759,9 @@ int spd_prefill(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int32_t
     auto run = [&](int b0, int nb, int s0, int ns) -> int {
         TokMap tm{0, b0, ns, s0, nullptr};
         size_t off = ((size_t)b0 * S + s0) * d.hidden * es;
+        const bool fused = d.dtype == 1 && d.hidden % 16 == 0;
         int rc = d.dtype == 0 ? run_tokens<float>(&c, (const char *)x + off, (char *)out + off, nb * ns, tm, block_table, max_pages, false, S, st)
+                 : fused      ? run_prefill_fused(&c, (const char *)x + off, (char *)out + off, nb * ns, tm, block_table, max_pages, S, st)
                               : run_tokens<bf16>(&c, (const char *)x + off, (char *)out + off, nb * ns, tm, block_table, max_pages, false, S, st);
         total_launches += c.launches_last;
         return rc;
