@@ -366,6 +366,50 @@ template <> struct Row16<bf16> {
     }
 };
 
+// Merge of the context splits by the last thread block of a (sequence, head tile): the
+// per-split maxima and denominators are turned into weights once (shared memory), then every
+// thread adds up its output elements with the partial loads issued eight at a time.
+// scratch: at least 2 * GT * splits floats of shared memory no longer in use.
+template <typename T, int D, int GT>
+__device__ __forceinline__ void merge_splits(const AttnArgs &a, int b, int hq0, float *scratch)
+{
+    const int S = a.splits;
+    float *wgt = scratch, *inv = scratch + GT * S; // weight of split s2 for head g; 1 / denominator per head
+    for (int i = threadIdx.x; i < GT * S; i += blockDim.x) {
+        const int g = i / S;
+        const long q0 = ((long)b * a.n_q_heads + hq0 + g) * S;
+        wgt[i] = __ldcg(a.part_ml + (q0 + i % S) * 2); // the split's maximum for now
+    }
+    __syncthreads();
+    if (threadIdx.x < GT) {
+        const int g = threadIdx.x;
+        const long q0 = ((long)b * a.n_q_heads + hq0 + g) * S;
+        float gm = -INFINITY, den = 0.f;
+        for (int s2 = 0; s2 < S; ++s2) gm = fmaxf(gm, wgt[g * S + s2]);
+        for (int s2 = 0; s2 < S; ++s2) {
+            const float m2 = wgt[g * S + s2];
+            const float c = (m2 == -INFINITY) ? 0.f : exp2f(m2 - gm);
+            wgt[g * S + s2] = c;
+            den += __ldcg(a.part_ml + (q0 + s2) * 2 + 1) * c;
+        }
+        inv[g] = den > 0.f ? 1.f / den : 0.f;
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < GT * D; idx += blockDim.x) {
+        const int g = idx / D, dd = idx % D;
+        const float *po = a.part_o + ((long)b * a.n_q_heads + hq0 + g) * S * D + dd;
+        float acc = 0.f;
+        for (int s0 = 0; s0 < S; s0 += 8) {
+            float v[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) v[k] = s0 + k < S ? __ldcg(po + (long)(s0 + k) * D) : 0.f;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc += v[k] * (s0 + k < S ? wgt[g * S + s0 + k] : 0.f);
+        }
+        ((T *)a.out)[((long)b * a.n_q_heads + hq0 + g) * D + dd] = from_f<T>(acc * inv[g]);
+    }
+}
+
 // Ring of the bulk-copy decode kernel: K and V page per slot, 32 KB in all (measured better than
 // 64 KB: four thread blocks per SM keep every block of a step resident at once).
 template <typename T, int D> struct DecodeRing {
@@ -752,20 +796,7 @@ __global__ void __launch_bounds__(160) decode_attention_ring_kernel(AttnArgs a)
     __syncthreads();
     if (!*sm_last) return;
     __threadfence();
-    for (int idx = threadIdx.x; idx < GT * D; idx += blockDim.x) {
-        const int g = idx / D, dd = idx % D;
-        const long q0 = ((long)b * a.n_q_heads + hq0 + g) * a.splits;
-        float gm = -INFINITY;
-        for (int s2 = 0; s2 < a.splits; ++s2) gm = fmaxf(gm, __ldcg(a.part_ml + (q0 + s2) * 2));
-        float acc = 0.f, gden = 0.f;
-        for (int s2 = 0; s2 < a.splits; ++s2) {
-            const float m2 = __ldcg(a.part_ml + (q0 + s2) * 2);
-            const float c = (m2 == -INFINITY) ? 0.f : exp2f(m2 - gm);
-            acc += __ldcg(a.part_o + (q0 + s2) * D + dd) * c;
-            gden += __ldcg(a.part_ml + (q0 + s2) * 2 + 1) * c;
-        }
-        ((T *)a.out)[((long)b * a.n_q_heads + hq0 + g) * D + dd] = from_f<T>(gden > 0.f ? acc / gden : 0.f);
-    }
+    merge_splits<T, D, GT>(a, b, hq0, &sm_o[0][0][0]);
     if (threadIdx.x == 0) *cnt = 0; // ready for the next launch
     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_END);
 }
@@ -788,11 +819,233 @@ template <typename T, int D, int GT> cudaError_t launch_ring(const AttnArgs &a, 
     return launch_kernel(decode_attention_ring_kernel<T, D, GT>, grid, dim3(160), SMEM, st, 0, a);
 }
 
+// ---------------------------------------------------------------------------------------
+// Grouped-query decode attention on tensor cores (bf16, head_dim 128, 16-token pages).  With a
+// GQA group of 8 query heads per KV head the CUDA-core kernel above is bound by arithmetic
+// (8 x 2 flops per cached element), not by the KV stream.  Here the group's query heads are the
+// rows of an m16n8k16 MMA: S[heads x 16 tokens] = Q K^T and O[heads x 128] += P V per page.
+// Pages arrive through TMA tensor copies (4 boxes of 64 dims x 16 tokens per page: K and V,
+// low and high half of the head dimension) in the 128-byte swizzle that ldmatrix reads without
+// bank conflicts.  Warp roles, page ring, split merge: as in the bulk-copy kernel.
+template <int GT>
+__global__ void __launch_bounds__(160) decode_attention_mma_kernel(const __grid_constant__ CUtensorMap tm_k,
+                                                                   const __grid_constant__ CUtensorMap tm_v, AttnArgs a)
+{
+    using namespace tc;
+    using fa::ldsm_x4;
+    using fa::ldsm_x4_t;
+    using fa::mma_bf16;
+    using fa::pack_bf16;
+    constexpr int D = 128, BLK = 16, R = 4, SUB = 2048 /* 16 tokens x 64 dims */, SLOT = 4 * SUB;
+    extern __shared__ uint8_t smem_dyn[];
+    const uint32_t ring = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    uint8_t *gen = smem_dyn + (ring - smem_u32(smem_dyn));
+    float(*sm_o)[GT][D] = (float(*)[GT][D])(gen + R * SLOT);
+    float(*sm_ml)[GT][2] = (float(*)[GT][2])(gen + R * SLOT + 4 * GT * D * 4);
+    uint8_t *tail = gen + R * SLOT + 4 * GT * D * 4 + 4 * GT * 2 * 4;
+    const uint32_t bars = smem_u32(tail);             // full[R], empty[R]
+    int *sm_bt = (int *)(tail + 2 * R * 8);
+    volatile int *abort_flag = (volatile int *)(sm_bt + DECODE_MAX_PAGES_PER_BLOCK);
+    int *sm_last = (int *)(sm_bt + DECODE_MAX_PAGES_PER_BLOCK + 1);
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (R + s); };
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t4 = lane & 3;
+    const int hq0 = blockIdx.x * GT, b = blockIdx.y, sp = blockIdx.z;
+    const int kvh = hq0 / (a.n_q_heads / a.pt.n_kv_heads);
+
+    pdl_launch_dependents();
+    if (threadIdx.x == 0) {
+        SPD_TRACE_EVENT(TRK_ATTN, TR_START);
+        for (int s = 0; s < R; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    const int ctx = a.tm.seq_lens[b] + 1;
+    const bool bad = ctx < 1 || ctx > a.max_context || (ctx - 1) / BLK >= a.pt.max_pages;
+    const int pages_bucket = (a.max_context + BLK - 1) / BLK;
+    const int per = (pages_bucket + a.splits - 1) / a.splits;
+    const int p0 = sp * per;
+    const int ctx_pages = bad ? 0 : (ctx + BLK - 1) / BLK;
+    const int n_pages = max(0, min(ctx_pages, p0 + per) - p0);
+    const int new_page = (ctx - 1) / BLK;
+    if (bad && threadIdx.x == 0) atomicOr(a.err, ERR_CAPACITY);
+
+    if (warp == 4) {
+        for (int i = lane; i < n_pages; i += 32) {
+            int page = a.pt.block_table[(long)b * a.pt.max_pages + p0 + i];
+            if (page < 0 || page >= a.pt.n_pages) { atomicOr(a.err, ERR_PAGE_RANGE); page = 0; }
+            sm_bt[i] = page;
+        }
+        __syncwarp();
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_v) : "memory");
+            bool waited = false;
+            for (int i = 0; i < n_pages; ++i) {
+                const int s = i % R;
+                if (!waited && p0 + i >= new_page) { pdl_wait(); waited = true; }
+                if (i >= R && !mbar_wait(empty_bar(s), ((i / R) & 1) ^ 1, a.err, abort_flag)) break;
+                const int row = (sm_bt[i] * a.pt.n_kv_heads + kvh) * BLK; // first of the page's 16 token rows
+                const uint32_t dst = ring + s * SLOT;
+                mbar_expect_tx(full_bar(s), SLOT);
+                tma_load_3d(dst, &tm_k, 0, row, 0, full_bar(s));
+                tma_load_3d(dst + SUB, &tm_k, 64, row, 0, full_bar(s));
+                tma_load_3d(dst + 2 * SUB, &tm_v, 0, row, 0, full_bar(s));
+                tma_load_3d(dst + 3 * SUB, &tm_v, 64, row, 0, full_bar(s));
+            }
+        }
+        __syncwarp();
+    }
+    pdl_wait(); // q comes from the preceding kernel
+    if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_DEP_DONE);
+
+    if (warp < 4) {
+        // A fragments of Q: MMA row g = query head hq0 + g (rows >= GT are padding)
+        uint32_t qf[8][4];
+        {
+            const bf16 *qp = (const bf16 *)a.q + ((long)b * a.n_q_heads + hq0 + g) * D;
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                qf[kk][0] = g < GT ? *(const uint32_t *)(qp + kk * 16 + 2 * t4) : 0u;
+                qf[kk][2] = g < GT ? *(const uint32_t *)(qp + kk * 16 + 8 + 2 * t4) : 0u;
+                qf[kk][1] = 0u;
+                qf[kk][3] = 0u;
+            }
+        }
+        float o[16][4];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+        float m_run = -INFINITY, l_run = 0.f;
+        const float sc = rsqrtf((float)D) * 1.4426950408889634f;
+        for (int pi = warp; pi < n_pages; pi += 4) {
+            const int s = pi % R;
+            if (!mbar_wait(full_bar(s), (pi / R) & 1, a.err, abort_flag)) break;
+            const uint32_t kb = ring + s * SLOT, vb = kb + 2 * SUB;
+            float sv[2][4];
+#pragma unroll
+            for (int i = 0; i < 2; ++i) { sv[i][0] = sv[i][1] = sv[i][2] = sv[i][3] = 0.f; }
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                uint32_t kf[4];
+                const int r = (lane & 7) + ((lane >> 4) << 3), c = (kk & 3) * 2 + ((lane >> 3) & 1);
+                ldsm_x4(kf, kb + (kk >> 2) * SUB + r * 128 + ((c ^ (r & 7)) << 4));
+                mma_bf16(sv[0], qf[kk], kf[0], kf[1]);
+                mma_bf16(sv[1], qf[kk], kf[2], kf[3]);
+            }
+            // this thread's row g: tokens nt*8 + 2*t4 + {0,1}
+            const int tbase = (p0 + pi) * BLK;
+            float pv[2][2], mx = m_run;
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const bool ok = tbase + nt * 8 + 2 * t4 + e < ctx;
+                    pv[nt][e] = ok ? sv[nt][e] * sc : -INFINITY;
+                    mx = fmaxf(mx, pv[nt][e]);
+                }
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            const float base = mx == -INFINITY ? 0.f : mx;
+            const float corr = m_run == -INFINITY ? 0.f : exp2f(m_run - base);
+            m_run = mx;
+            float rs = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) { pv[nt][e] = exp2f(pv[nt][e] - base); rs += pv[nt][e]; }
+            l_run = l_run * corr + rs;
+            uint32_t pf[4];
+            pf[0] = pack_bf16(pv[0][0], pv[0][1]);
+            pf[1] = 0u;
+            pf[2] = pack_bf16(pv[1][0], pv[1][1]);
+            pf[3] = 0u;
+#pragma unroll
+            for (int dt = 0; dt < 16; ++dt) { o[dt][0] *= corr; o[dt][1] *= corr; }
+#pragma unroll
+            for (int dp = 0; dp < 8; ++dp) {
+                uint32_t vf[4];
+                const int r = (lane & 7) + (((lane >> 3) & 1) << 3), c = (dp & 3) * 2 + (lane >> 4);
+                ldsm_x4_t(vf, vb + (dp >> 2) * SUB + r * 128 + ((c ^ (r & 7)) << 4));
+                mma_bf16(o[2 * dp], pf, vf[0], vf[1]);
+                mma_bf16(o[2 * dp + 1], pf, vf[2], vf[3]);
+            }
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(s)) : "memory");
+        }
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+        if (g < GT) {
+#pragma unroll
+            for (int dt = 0; dt < 16; ++dt) {
+                sm_o[warp][g][dt * 8 + 2 * t4] = o[dt][0];
+                sm_o[warp][g][dt * 8 + 2 * t4 + 1] = o[dt][1];
+            }
+            if (t4 == 0) { sm_ml[warp][g][0] = m_run; sm_ml[warp][g][1] = l_run; }
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_MAIN_DONE);
+    // merge the 4 warps; thread -> (head of the tile, dim)
+    const long pbase = ((long)b * a.n_q_heads + hq0) * a.splits + sp;
+    for (int idx = threadIdx.x; idx < GT * D; idx += blockDim.x) {
+        const int gg = idx / D, dd = idx % D;
+        float gm = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) gm = fmaxf(gm, sm_ml[w][gg][0]);
+        float acc = 0.f, gden = 0.f;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const float c = (sm_ml[w][gg][0] == -INFINITY) ? 0.f : exp2f(sm_ml[w][gg][0] - gm);
+            acc += sm_o[w][gg][dd] * c;
+            gden += sm_ml[w][gg][1] * c;
+        }
+        if (a.splits == 1) {
+            ((bf16 *)a.out)[((long)b * a.n_q_heads + hq0 + gg) * D + dd] = __float2bfloat16_rn(gden > 0.f ? acc / gden : 0.f);
+        } else {
+            const long pi = pbase + (long)gg * a.splits;
+            a.part_o[pi * D + dd] = acc; // un-normalised
+            if (dd == 0) { a.part_ml[pi * 2] = gm; a.part_ml[pi * 2 + 1] = gden; }
+        }
+    }
+    if (a.splits == 1) return;
+    // the last block of this (sequence, head tile) to arrive merges the splits
+    __threadfence();
+    __syncthreads();
+    int *cnt = a.counters + (long)b * gridDim.x + blockIdx.x;
+    if (threadIdx.x == 0) *sm_last = (atomicAdd(cnt, 1) == a.splits - 1);
+    __syncthreads();
+    if (!*sm_last) return;
+    __threadfence();
+    merge_splits<bf16, D, GT>(a, b, hq0, &sm_o[0][0][0]);
+    if (threadIdx.x == 0) *cnt = 0; // ready for the next launch
+    if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_END);
+}
+
+template <int GT> cudaError_t launch_decode_mma(const AttnArgs &a, cudaStream_t st)
+{
+    constexpr int SMEM = 1024 + 4 * 8192 + 4 * GT * 128 * 4 + 4 * GT * 2 * 4 + 2 * 4 * 8 + (DECODE_MAX_PAGES_PER_BLOCK + 2) * 4;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(decode_attention_mma_kernel<GT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    dim3 grid(a.n_q_heads / GT, a.B, a.splits);
+    return launch_kernel(decode_attention_mma_kernel<GT>, grid, dim3(160), SMEM, st, 0, *(const CUtensorMap *)a.k_map,
+                         *(const CUtensorMap *)a.v_map, a);
+}
+
 template <typename T, int D> cudaError_t launch_decode_d(const AttnArgs &a, cudaStream_t st)
 {
     const int group = a.n_q_heads / a.pt.n_kv_heads;
     const int pages_bucket = (a.max_context + 15) / 16;
-    if (a.pt.block == 16 && (pages_bucket + a.splits - 1) / a.splits <= DECODE_MAX_PAGES_PER_BLOCK) {
+    const bool fits = (pages_bucket + a.splits - 1) / a.splits <= DECODE_MAX_PAGES_PER_BLOCK;
+    if (fits && a.k_map && a.v_map && decode_uses_mma(group, D, sizeof(T) == 2, a.pt.block))
+        return decode_heads_per_block_mma(group) == 8 ? launch_decode_mma<8>(a, st) : launch_decode_mma<4>(a, st);
+    if (a.pt.block == 16 && fits) {
         switch (decode_heads_per_block(group)) {
         case 4: return launch_ring<T, D, 4>(a, st);
         case 2: return launch_ring<T, D, 2>(a, st);

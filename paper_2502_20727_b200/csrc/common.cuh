@@ -162,11 +162,17 @@ struct AttnArgs {
     float *part_ml;         // fp32 [B][nq][splits][2]
     int *counters;          // [B][nq] zero-initialised arrival counters (split merge)
     int *err;
+    // optional (decode, bf16, head_dim 128, 16-token pages): tensor maps over the K and V pages seen as
+    // [n_pages * n_kv_heads * 16 rows][head_dim], box 64 x 16, 128-byte swizzle (host pointers to CUtensorMap)
+    const void *k_map, *v_map;
 };
 // Paged decode attention with 16-token pages: query heads per thread block for a GQA group
 // size, and the most pages one block may be given (the host picks splits accordingly).
 constexpr int DECODE_MAX_PAGES_PER_BLOCK = 512;
 inline int decode_heads_per_block(int group) { return group % 4 == 0 ? 4 : (group % 2 == 0 ? 2 : 1); }
+// ... and of the tensor-core variant, which serves grouped-query attention with group sizes 4, 8, ...
+inline bool decode_uses_mma(int group, int head_dim, int dtype_bf16, int kv_block) { return dtype_bf16 && head_dim == 128 && kv_block == 16 && group % 4 == 0; }
+inline int decode_heads_per_block_mma(int group) { return group % 8 == 0 ? 8 : 4; }
 template <typename T> cudaError_t launch_prefill_attention(const AttnArgs &a, cudaStream_t st);
 template <typename T> cudaError_t launch_decode_attention(const AttnArgs &a, cudaStream_t st);
 

@@ -56,7 +56,7 @@ enum Site { SITE_QKV = 0, SITE_O, SITE_GU, SITE_DOWN, SITE_ATTN, SITE_COUNT };
 const char *const kind_names[K_COUNT] = {"residual_rmsnorm", "gemm_qkv", "rope_kv_append", "attention", "gemm_o_proj",
                                          "gemm_gate_up", "silu_mul", "gemm_down", "rope_table"};
 
-struct LayerMaps { TcMap wq, wk, wv, wo_full, wo_shard, w_gate, w_up, w_down, w_gate64, w_up64, wq256, wk256, wv256, wo256, wd256; };
+struct LayerMaps { TcMap wq, wk, wv, wo_full, wo_shard, w_gate, w_up, w_down, w_gate64, w_up64, wq256, wk256, wv256, wo256, wd256, kpages, vpages; };
 
 // A captured decode step is valid for exactly these arguments.
 struct GraphKey {
@@ -156,7 +156,9 @@ Plan make_plan(const spd_dims &d, int M, bool decode, int max_context, int attn_
     p.attn_splits = 1;
     if (decode) {
         // decode attention: up to four thread blocks per SM, at least four 16-token pages each
-        const int gt = decode_heads_per_block(d.n_q_heads / d.n_kv_heads);
+        const int group = d.n_q_heads / d.n_kv_heads;
+        const int gt = decode_uses_mma(group, d.head_dim, d.dtype == 1, d.kv_block_size) ? decode_heads_per_block_mma(group)
+                                                                                           : decode_heads_per_block(group);
         const long ctas = (long)M * (d.n_q_heads / gt);
         const int pages = cdiv(max_context, 16);
         int s = attn_override > 0 ? attn_override : (int)((4L * N_SM) / ctas);
@@ -490,6 +492,7 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
             a.q = c->q; a.k_pages = w.k_pages; a.v_pages = w.v_pages; a.pt = pt; a.tm = tm; a.out = c->attn;
             a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.B = M; a.splits = p.attn_splits;
             a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.counters = c->attn_cnt; a.err = c->err;
+            if (d.head_dim == 128 && d.kv_block_size == 16) { a.k_map = &c->maps[l].kpages; a.v_map = &c->maps[l].vpages; }
             LAUNCH(K_ATTN, launch_decode_attention<bf16>(a, st));
         }
         {   // a5 - a7: shard i's K slice gives the plane group Y_i
@@ -658,6 +661,12 @@ int build_weight_maps(Ctx &c)
         rc |= make_operand_map(&m.wv256, w.wv, H, kd, 1, H, 0, 256);
         rc |= make_operand_map(&m.wo256, w.wo, qd, H, 1, qd, 0, 256);
         rc |= make_operand_map(&m.wd256, w.w_down, F, H, 1, F, 0, 256);
+        if (d.head_dim == 128 && d.kv_block_size == 16) {
+            // K / V pages as [n_pages * n_kv_heads * 16 token rows][head_dim]; one box = 64 dims of a page's 16 tokens
+            const long rows = (long)c.n_pages * d.n_kv_heads * 16;
+            rc |= make_operand_map(&m.kpages, w.k_pages, 128, rows, 1, 128, 0, 16);
+            rc |= make_operand_map(&m.vpages, w.v_pages, 128, rows, 1, 128, 0, 16);
+        }
         rc |= make_operand_map(&m.w_gate64, w.w_gate, H, F / T, T, H, (F / T) * H, 64);
         rc |= make_operand_map(&m.w_up64, w.w_up, H, F / T, T, H, (F / T) * H, 64);
         if (rc) return SPD_EINVAL;

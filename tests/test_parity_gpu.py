@@ -111,6 +111,27 @@ def test_decode_at_bench_size_on_synthetic_cache():
     assert p.stack.device_error() == 0
 
 
+@pytest.mark.parametrize("nq,nkv,T", [(8, 2, 2), (16, 2, 2), (8, 1, 1)])
+def test_bf16_grouped_query_head_dim_128(nq, nkv, T):
+    """GQA groups of 4, 8 (tensor-core decode attention) with head_dim 128, ragged prompt over pages."""
+    w = si.Workload("gqa", "bf16", 2, 512, nq, nkv, 128, 1024, T, (0, 1), 3, 45, 4)
+    run_case(w, (0, 1), 3, 45, 4)
+
+
+def test_gqa_decode_long_ragged_context_on_synthetic_cache():
+    """configs[3] dims (64 query / 8 KV heads), one layer, contexts up to 2100 tokens with ragged
+    lengths: several context splits and partially filled last pages."""
+    w = si.WORKLOADS["c4_b32"].with_(n_layers=1, mask=(0,))
+    p = Pair(w, B=4, max_len=2112)
+    lens = np.array([2100, 17, 1, 1030], dtype=np.int32)
+    p.fill_cache(lens)
+    for t in range(2):
+        got, ref = p.decode(t)
+        e = rel_err(got, ref)
+        assert e <= TOL["bf16"], f"step {t}: {e}"
+    assert p.stack.device_error() == 0
+
+
 def test_run_twice_bitwise_identical():
     w = si.Workload("small", "bf16", 2, 512, 8, 8, 64, 1024, 4, (0, 1), 4, 33, 2)
     outs = []
