@@ -29,6 +29,10 @@ import spd_inputs as si  # noqa: E402
 
 METRIC = "decode tokens/s and HBM-roofline fraction (1 B200), sync vs SPD masks"
 GEMM_KINDS = ("gemm_qkv", "gemm_o_proj", "gemm_gate_up", "gemm_down")
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the projection GEMM (average of the four
+# launches of a block), from the ncu capture summarised in profiles/dram_decode_kernels_c2.md.  Valid for
+# that workload with automatic tuning only; set to None when the kernel changes until it is captured again.
+NCU_TRAFFIC_PER_LAUNCH = {"c2": 101.98e6}
 
 
 def measured_peaks():
@@ -251,7 +255,9 @@ def run_native(args, rank, world):
                           "peak_kind": peak_kind},
         "roofline": {"bound": "hbm", "kernel": "weight-streaming projection GEMM (qkv, o_proj, gate/up, down)",
                      "achieved": gemm_gbs, "peak": hbm_peak, "unit": "GB/s",
-                     "frac": (gemm_gbs / hbm_peak) if gemm_gbs else None, "traffic": None, "peak_kind": peak_kind,
+                     "frac": (gemm_gbs / hbm_peak) if gemm_gbs else None,
+                     "traffic": NCU_TRAFFIC_PER_LAUNCH.get(w.name) if not args.tune else None,
+                     "algorithmic_bytes_per_launch": gemm_bytes_step / max(gemm_launches / K, 1), "peak_kind": peak_kind,
                      "launches_per_step": gemm_launches / K, "avg_launch_us": gemm_ms * 1e3 / max(gemm_launches, 1),
                      "bytes_per_step": gemm_bytes_step},
         "kernel_ms_per_step": {k: v["ms"] / K for k, v in prof.items()},
