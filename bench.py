@@ -51,6 +51,22 @@ def pick_mask(w: si.Workload, which: str):
     return tuple(w.mask)
 
 
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def replica_plan(w, rank: int, world: int):
+    """Replicas only: every rank holds a whole emulated stack (its own seed) and its own batch;
+    nothing crosses ranks on the data path.  Returns what rank `rank` runs and what the job counts."""
+    return {"seed": rank, "batch": w.batch, "tokens_per_step_job": w.batch * world, "scaling": "weak"}
+
+
 class ClockSampler:
     """nvidia-smi clocks / throttle reasons while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -135,7 +151,8 @@ def run_native(args, rank, world):
     B, S = w.batch, w.prompt
     K, W = args.steps, args.warmup
     max_len = S + W + K + 1
-    layers = si.make_stack(w, dev, seed=rank)
+    plan = replica_plan(w, rank, world)
+    layers = si.make_stack(w, dev, seed=plan["seed"])
     stack = spd.stack_from_workload(w, layers, sync_mask=mask, max_batch=B, max_seq_len=max_len,
                                     max_prefill_tokens=min(B * S, args.prefill_chunk), device=dev)
     pages_per_seq = (max_len + w.kv_block - 1) // w.kv_block
@@ -221,10 +238,7 @@ def run_native(args, rank, world):
         step(t)
     prof = stack.profile_end()
 
-    if world > 1:
-        tt = torch.tensor([dev_ms, e2e_s], dtype=torch.float64, device=dev)
-        torch.distributed.all_reduce(tt, op=torch.distributed.ReduceOp.MAX)
-        dev_ms, e2e_s = float(tt[0]), float(tt[1])
+    dev_ms, e2e_s = max_over_ranks([dev_ms, e2e_s], dev)
     if rank != 0:
         return None
 

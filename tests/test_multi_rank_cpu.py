@@ -1,0 +1,45 @@
+"""N > 1 on CPU: two gloo ranks run the rank plumbing of bench.py (replicas only: no collective on the
+data path, timing = max over ranks, rank 0 prints the one line)."""
+import json
+import os
+import socket
+import subprocess
+import sys
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def torchrun(script_and_args, n=2):
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(free_port())] + script_and_args
+    env = dict(os.environ, OMP_NUM_THREADS="2")
+    r = subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    return r.stdout
+
+
+def test_two_ranks_replica_plan_and_max_timing():
+    out = torchrun([os.path.join(ROOT, "tests", "rank_worker.py")])
+    lines = [l for l in out.splitlines() if l.startswith("WORKER ")]
+    assert len(lines) == 1
+    res = json.loads(lines[0][7:])
+    assert res["world"] == 2 and res["seeds"] == [0, 1]
+    assert res["t_max"] == 2.0 and res["t_same"] == 5.0        # slowest rank decides
+    assert res["job_tokens"] == 2                               # c1: batch 1 per rank, weak scaling
+    assert res["distinct_weights"] == 2                         # independent replicas
+
+
+def test_reference_arm_prints_one_line_under_torchrun():
+    out = torchrun([os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "c1", "--gpus", "2", "--steps", "2",
+                    "--warmup", "1"])
+    lines = [l for l in out.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    res = json.loads(lines[0])
+    assert res["impl"] == "reference" and res["n_gpus"] == 2 and res["value"] > 0
+    assert res["cpu_baseline"]["kind"] == "oracle" and res["e2e"]["h2d_bytes_per_step"] == 0
