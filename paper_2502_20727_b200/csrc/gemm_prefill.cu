@@ -31,8 +31,11 @@ template <int EPI> struct PCfg {
     static constexpr int BN = (EPI == PRE_OPROJ_SPD) ? 128 : 256;
     static constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (192 * 1024) / STAGE_BYTES;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    // PRE_OPROJ_SPD keeps the X tile (fp32, 64 KB) and one outgoing R_i * g tile (bf16, 32 KB) in shared memory
+    static constexpr int X_BYTES = (EPI == PRE_OPROJ_SPD) ? 128 * 128 * 4 : 0, H_BYTES = (EPI == PRE_OPROJ_SPD) ? 128 * 128 * 2 : 0;
+    static constexpr int STAGES = (192 * 1024 - X_BYTES - H_BYTES) / STAGE_BYTES;
+    static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
+    static constexpr int SMEM_BYTES = RING_BYTES + X_BYTES + H_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
 struct PreLaunch {
@@ -258,9 +261,16 @@ __device__ __forceinline__ void epi_resid(const PreGemmArgs &g, const PreTile &t
     if (valid && g.ss_out) g.ss_out[(long)t.nt * g.Mcap + m] = ssq;
 }
 
-__device__ __forceinline__ void epi_oproj_spd(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, uint32_t ttot, int z, int m, bool valid)
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// One pass (device z) of an SPD o_proj tile.  The X tile sits in shared memory (xs: four 32-column
+// boxes of 128 rows, 128-byte swizzle); R_z * g is staged in hs (two 64-column bf16 boxes) and
+// leaves through a TMA store, as does X + sum_i Y_i after the last pass (written over the X tile).
+// Swizzled layouts: thread = row, eight consecutive rows hit eight different 16-byte columns.
+__device__ __forceinline__ float epi_oproj_spd(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, uint32_t ttot, int z,
+                                               uint8_t *xs, uint8_t *hs)
 {
-    const int T = g.batches;
+    const int T = g.batches, r = threadIdx.x, sw = r & 7;
     float ssq = 0.f;
 #pragma unroll 1
     for (int c = 0; c < 8; ++c) {
@@ -277,22 +287,37 @@ __device__ __forceinline__ void epi_oproj_spd(const PreGemmArgs &g, const PreTil
             for (int i = 0; i < 16; ++i) tot[i] += y[i];
         }
         if (z + 1 < T) tmem_st16(ttot + c * 16, tot);
-        if (!valid) continue;
-        const long idx = (long)m * g.H + n;
+        // X: columns c*16 .. c*16+15 = box c/2, 16-byte chunks (c & 1) * 4 .. + 3 of this row
+        uint8_t *xrow = xs + (c >> 1) * 16384 + r * 128;
         float x[16];
-        load_x16(g.res_in + idx, x);
-        // device z only ever sees its own partial attention output
-        ssq += resid_chunk(g, idx, n, x, y, g.hg ? (bf16 *)g.hg + (long)z * g.hg_stride : nullptr, false);
-        if (z + 1 == T && g.res_out) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float4 v = *(const float4 *)(xrow + ((((c & 1) * 4 + k) ^ sw) << 4));
+            x[4 * k] = v.x; x[4 * k + 1] = v.y; x[4 * k + 2] = v.z; x[4 * k + 3] = v.w;
+        }
+        // device z only ever sees its own partial attention output: R_z = X + Y_z
+        float gn[16];
+        unpack8(*(const uint4 *)((const bf16 *)g.gain + n), gn);
+        unpack8(*(const uint4 *)((const bf16 *)g.gain + n + 8), gn + 8);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const float ri = x[i] + y[i];
+            ssq = fmaf(ri, ri, ssq);
+            gn[i] *= ri;
+        }
+        uint8_t *hrow = hs + (c >> 2) * 16384 + r * 128;
+        *(uint4 *)(hrow + ((((c & 3) * 2) ^ sw) << 4)) = pack8(gn);
+        *(uint4 *)(hrow + ((((c & 3) * 2 + 1) ^ sw) << 4)) = pack8(gn + 8);
+        if (z + 1 == T) {
             // the residual carried to the block output collects every Y_i
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                *(float4 *)(g.res_out + idx + 4 * i) =
-                    make_float4(x[4 * i] + tot[4 * i], x[4 * i + 1] + tot[4 * i + 1], x[4 * i + 2] + tot[4 * i + 2], x[4 * i + 3] + tot[4 * i + 3]);
+            for (int k = 0; k < 4; ++k)
+                *(float4 *)(xrow + ((((c & 1) * 4 + k) ^ sw) << 4)) =
+                    make_float4(x[4 * k] + tot[4 * k], x[4 * k + 1] + tot[4 * k + 1], x[4 * k + 2] + tot[4 * k + 2], x[4 * k + 3] + tot[4 * k + 3]);
         }
     }
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-    if (valid && g.ss_out) g.ss_out[((long)t.nt * T + z) * g.Mcap + m] = ssq;
+    return ssq;
 }
 
 template <int EPI>
@@ -300,6 +325,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_prefill_kernel(const __grid_c
                                                                   const __grid_constant__ CUtensorMap tm_w1,
                                                                   const __grid_constant__ CUtensorMap tm_w2,
                                                                   const __grid_constant__ CUtensorMap tm_t,
+                                                                  const __grid_constant__ CUtensorMap tm_x,
+                                                                  const __grid_constant__ CUtensorMap tm_r,
+                                                                  const __grid_constant__ CUtensorMap tm_h,
                                                                   const __grid_constant__ PreLaunch L)
 {
     using C = PCfg<EPI>;
@@ -308,8 +336,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_prefill_kernel(const __grid_c
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t bars = base + S * C::STAGE_BYTES; // full[S], empty[S], tmem_full[2], tmem_empty[2]
-    uint32_t *tmem_slot = (uint32_t *)(gen_base + S * C::STAGE_BYTES + 8 * (2 * S + 4));
+    uint8_t *xs = gen_base + C::RING_BYTES, *hs = xs + C::X_BYTES; // PRE_OPROJ_SPD staging (1024-byte aligned)
+    const uint32_t bars = base + C::RING_BYTES + C::X_BYTES + C::H_BYTES; // full[S], empty[S], tmem_full[2], tmem_empty[2], x_full
+    uint32_t *tmem_slot = (uint32_t *)(gen_base + C::RING_BYTES + C::X_BYTES + C::H_BYTES + 8 * (2 * S + 5));
+    const uint32_t xfull_bar = bars + 8u * (2 * S + 4);
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (S + s); };
@@ -323,6 +353,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_prefill_kernel(const __grid_c
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+        mbar_init(xfull_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -394,13 +425,22 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_prefill_kernel(const __grid_c
         }
         __syncwarp();
     } else {
-        uint32_t pc = 0;
+        uint32_t pc = 0, tile_cnt = 0;
         bool ok = true;
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_cnt) {
             const PreTile t = decode_tile(L, EPI, tile);
             const int m = t.m0 + warp * 32 + lane;
             const bool valid = m < g.t_rows;
+            if (EPI == PRE_OPROJ_SPD) {
+                // the X tile of this output tile: once the stores of the previous tile have read their source
+                if (threadIdx.x == 0) tma_store_wait_read();
+                epi_sync();
+                if (threadIdx.x == 0) {
+                    mbar_expect_tx(xfull_bar, C::X_BYTES);
+                    for (int bx = 0; bx < 4; ++bx) tma_load_3d(smem_u32(xs) + bx * 16384, &tm_x, t.row0 + 32 * bx, t.m0, 0, xfull_bar);
+                }
+            }
             for (int pass = 0; pass < L.passes; ++pass, ++pc) {
                 const int buf = pc & 1;
                 if (!mbar_wait(tfull_bar(buf), (pc >> 1) & 1, g.err, abort_flag)) { ok = false; break; }
@@ -409,12 +449,31 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_prefill_kernel(const __grid_c
                 if (EPI == PRE_QKV) epi_qkv(g, t, tacc, m, valid);
                 else if (EPI == PRE_GATEUP) epi_gateup(g, t, tacc, m, valid);
                 else if (EPI == PRE_RESID) epi_resid(g, t, tacc, m, valid);
-                else epi_oproj_spd(g, t, tacc, tmem_base + lane_base + TOT_COL, pass, m, valid);
+                else {
+                    if (pass == 0) {
+                        if (!mbar_wait(xfull_bar, tile_cnt & 1, g.err, abort_flag)) { ok = false; break; }
+                    } else {
+                        if (threadIdx.x == 0) tma_store_wait_read(); // the staging tile is free again
+                        epi_sync();
+                    }
+                    const float ssq = epi_oproj_spd(g, t, tacc, tmem_base + lane_base + TOT_COL, pass, xs, hs);
+                    if (valid && g.ss_out) g.ss_out[((long)t.nt * g.batches + pass) * g.Mcap + m] = ssq;
+                    fence_proxy_async();
+                    epi_sync();
+                    if (threadIdx.x == 0) {
+                        tma_store_3d(&tm_h, smem_u32(hs), t.row0, t.m0, pass);
+                        tma_store_3d(&tm_h, smem_u32(hs) + 16384, t.row0 + 64, t.m0, pass);
+                        if (pass + 1 == L.passes)
+                            for (int bx = 0; bx < 4; ++bx) tma_store_3d(&tm_r, smem_u32(xs) + bx * 16384, t.row0 + 32 * bx, t.m0, 0);
+                        tma_store_commit();
+                    }
+                }
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(tempty_bar(buf)) : "memory");
             }
         }
+        if (EPI == PRE_OPROJ_SPD && threadIdx.x == 0) tma_store_wait_all(); // results in memory before the block ends
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -427,6 +486,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_prefill_kernel(const __grid_c
 template <int EPI>
 cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, const PreLaunch &L, cudaStream_t st)
 {
+    const bool spd = EPI == PRE_OPROJ_SPD;
+    const CUtensorMap &tx = *(const CUtensorMap *)(spd ? L.g.x_map : (const void *)&tt);
+    const CUtensorMap &tr = *(const CUtensorMap *)(spd ? L.g.r_map : (const void *)&tt);
+    const CUtensorMap &th = *(const CUtensorMap *)(spd ? L.g.h_map : (const void *)&tt);
     using C = PCfg<EPI>;
     static int n_sm = 0;
     if (!n_sm) {
@@ -439,7 +502,7 @@ cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
     }
     const int total = L.m_tiles * L.n_tiles;
     const dim3 grid(total < n_sm ? total : n_sm);
-    return launch_kernel(gemm_prefill_kernel<EPI>, grid, dim3(THREADS), C::SMEM_BYTES, st, 0, *tw[0], *tw[1], *tw[2], tt, L);
+    return launch_kernel(gemm_prefill_kernel<EPI>, grid, dim3(THREADS), C::SMEM_BYTES, st, 0, *tw[0], *tw[1], *tw[2], tt, tx, tr, th, L);
 }
 
 // One thread block per token: whole-row sum of squares in one partial.
@@ -484,6 +547,7 @@ cudaError_t launch_gemm_prefill(PreEpilogue epi, const TcMap *const *weights, co
     if (g.num_kb < 1 || g.batches < 1 || g.batches > 8) return cudaErrorInvalidValue;
     if (epi == PRE_QKV && (256 % g.head_dim || g.head_dim < 32)) return cudaErrorInvalidValue;
     if ((epi == PRE_RESID || epi == PRE_OPROJ_SPD) && g.H % 16) return cudaErrorInvalidValue;
+    if (epi == PRE_OPROJ_SPD && (!g.x_map || !g.r_map || !g.h_map || !g.gain || !g.hg || !g.res_out)) return cudaErrorInvalidValue;
     if (epi == PRE_GATEUP && g.Fs % 8) return cudaErrorInvalidValue;
     const CUtensorMap *tw[3];
     for (int i = 0; i < 3; ++i) tw[i] = (const CUtensorMap *)weights[i < nw ? i : 0];
