@@ -95,15 +95,15 @@ __global__ void __launch_bounds__(128) prefill_attention_kernel(AttnArgs a)
 }
 
 // ---------------------------------------------------------------------------------------
-// Causal prefill attention on tensor cores (bf16): one thread block per 64 query rows of one
+// Causal prefill attention on tensor cores (bf16): one thread block per 128 query rows of one
 // (sequence, query head); K/V tiles of 64 cached tokens are gathered from their pages into
-// double-buffered, XOR-swizzled shared memory with cp.async; each of the 4 warps owns 16 query
+// double-buffered, XOR-swizzled shared memory with cp.async; each of the 8 warps owns 16 query
 // rows: S = Q K^T and O += P V as m16n8k16 MMAs with fp32 accumulators, online softmax in
 // base 2 on the accumulator fragments, P re-used in registers as the A operand of the second
 // product.  Chunked prefill: queries at positions s0.. attend to every cached position <= their own.
 namespace fa {
 
-constexpr int BQ = 64, BKV = 64;
+constexpr int NW = 8, BQ = 16 * NW, BKV = 64, FA_THREADS = 32 * NW;
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid)
 {
@@ -134,7 +134,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 template <int D> __device__ __forceinline__ uint32_t tile_off(int r, int c) { return (uint32_t)(r * D * 2 + ((c ^ (r & 7)) << 4)); }
 
 template <int D>
-__global__ void __launch_bounds__(128) prefill_attention_mma_kernel(AttnArgs a)
+__global__ void __launch_bounds__(FA_THREADS, 2) prefill_attention_mma_kernel(AttnArgs a)
 {
     constexpr int CH = D / 8;       // 16-byte chunks per row
     constexpr int KS = D / 16;      // k-steps of Q K^T
@@ -145,7 +145,7 @@ __global__ void __launch_bounds__(128) prefill_attention_mma_kernel(AttnArgs a)
     pdl_launch_dependents();
     pdl_wait();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
-    const int q0 = blockIdx.x * BQ, hq = blockIdx.y, bi = blockIdx.z;
+    const int q0 = ((int)gridDim.x - 1 - (int)blockIdx.x) * BQ, hq = blockIdx.y, bi = blockIdx.z; // longest rows first
     const int ns = a.tm.ns, s0 = a.tm.s0, b = a.tm.b0 + bi;
     const int kvh = hq / (a.n_q_heads / a.pt.n_kv_heads);
     const int q_rows = min(BQ, ns - q0);
@@ -156,8 +156,8 @@ __global__ void __launch_bounds__(128) prefill_attention_mma_kernel(AttnArgs a)
     auto load_kv = [&](int tile, int buf) {
         const uint32_t dK = sK + buf * BKV * D * 2, dV = sV + buf * BKV * D * 2;
 #pragma unroll
-        for (int i = 0; i < BKV * CH / 128; ++i) {
-            const int idx = tid + i * 128, r = idx / CH, c = idx % CH, tkn = tile * BKV + r;
+        for (int i = 0; i < BKV * CH / FA_THREADS; ++i) {
+            const int idx = tid + i * FA_THREADS, r = idx / CH, c = idx % CH, tkn = tile * BKV + r;
             const bool valid = tkn < kv_len;
             long off = 0;
             if (valid) {
@@ -171,8 +171,8 @@ __global__ void __launch_bounds__(128) prefill_attention_mma_kernel(AttnArgs a)
     };
     // Q tile
 #pragma unroll
-    for (int i = 0; i < BQ * CH / 128; ++i) {
-        const int idx = tid + i * 128, r = idx / CH, c = idx % CH;
+    for (int i = 0; i < BQ * CH / FA_THREADS; ++i) {
+        const int idx = tid + i * FA_THREADS, r = idx / CH, c = idx % CH;
         const bool valid = r < q_rows;
         const bf16 *src = (const bf16 *)a.q + ((long)(bi * ns + q0 + (valid ? r : 0)) * a.n_q_heads + hq) * D + c * 8;
         cp_async16(sQ + tile_off<D>(r, c), src, valid);
@@ -182,13 +182,9 @@ __global__ void __launch_bounds__(128) prefill_attention_mma_kernel(AttnArgs a)
     cp_async_commit();
     cp_async_wait<1>();
     __syncthreads();
-    // A fragments of this warp's 16 query rows
-    uint32_t qf[KS][4];
-#pragma unroll
-    for (int kk = 0; kk < KS; ++kk) {
-        const int r = warp * 16 + (lane & 15), c = kk * 2 + (lane >> 4);
-        ldsm_x4(qf[kk], sQ + tile_off<D>(r, c));
-    }
+    // the A fragments of this warp's 16 query rows are re-read from the Q tile for every K tile
+    // (keeps the register count at two thread blocks per SM)
+    const uint32_t q_addr_row = warp * 16 + (lane & 15);
     float o[DT][4];
 #pragma unroll
     for (int i = 0; i < DT; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
@@ -213,24 +209,27 @@ __global__ void __launch_bounds__(128) prefill_attention_mma_kernel(AttnArgs a)
         for (int i = 0; i < NT; ++i) { s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f; }
 #pragma unroll
         for (int kk = 0; kk < KS; ++kk) {
+            uint32_t qf[4];
+            ldsm_x4(qf, sQ + tile_off<D>(q_addr_row, kk * 2 + (lane >> 4)));
 #pragma unroll
             for (int np = 0; np < NT / 2; ++np) {
                 // matrices: (tokens np*16 + 0..7, dims kk*16 + 0..7), (same tokens, dims + 8), (tokens + 8, dims), (tokens + 8, dims + 8)
                 uint32_t kf[4];
                 const int r = np * 16 + (lane & 7) + ((lane >> 4) << 3), c = kk * 2 + ((lane >> 3) & 1);
                 ldsm_x4(kf, bK + tile_off<D>(r, c));
-                mma_bf16(s[2 * np], qf[kk], kf[0], kf[1]);
-                mma_bf16(s[2 * np + 1], qf[kk], kf[2], kf[3]);
+                mma_bf16(s[2 * np], qf, kf[0], kf[1]);
+                mma_bf16(s[2 * np + 1], qf, kf[2], kf[3]);
             }
         }
-        // scale, causal mask, running max
+        // scale, causal mask (only tiles that reach past this warp's first query position), running max
         float m_new[2] = {m_run[0], m_run[1]};
+        const bool need_mask = (j + 1) * BKV - 1 > s0 + q0 + warp * 16 || q0 + warp * 16 + 16 > q_rows;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int key = j * BKV + nt * 8 + 2 * t4 + (e & 1), h = e >> 1;
-                const float v = key <= pos_q[h] ? s[nt][e] * sc : -INFINITY;
+                const float v = (!need_mask || key <= pos_q[h]) ? s[nt][e] * sc : -INFINITY;
                 s[nt][e] = v;
                 m_new[h] = fmaxf(m_new[h], v);
             }
@@ -306,7 +305,7 @@ template <int D> cudaError_t launch(const AttnArgs &a, int n_seq, cudaStream_t s
         attr_done = true;
     }
     dim3 grid((a.tm.ns + BQ - 1) / BQ, a.n_q_heads, n_seq);
-    return launch_kernel(prefill_attention_mma_kernel<D>, grid, dim3(128), SMEM, st, 0, a);
+    return launch_kernel(prefill_attention_mma_kernel<D>, grid, dim3(FA_THREADS), SMEM, st, 0, a);
 }
 
 } // namespace fa

@@ -16,6 +16,7 @@
 //                   residual that is carried to the block output.
 #include "gemm_prefill.cuh"
 #include "tc_ptx.cuh"
+#include "trace.cuh"
 
 namespace spd {
 
@@ -25,14 +26,15 @@ using namespace tc;
 
 constexpr int THREADS = 192;
 constexpr int TMEM_ALL = 512;
-constexpr int TOT_COL = 256; // PRE_OPROJ_SPD: running sum of the Y_i
+constexpr int TOT_COL = 256; // PRE_OPROJ_SPD: X + running sum of the Y_i
+constexpr int X_COL = 384;   // PRE_OPROJ_SPD: the X tile
 
 template <int EPI> struct PCfg {
     static constexpr int BN = (EPI == PRE_OPROJ_SPD) ? 128 : 256;
     static constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    // PRE_OPROJ_SPD keeps the X tile (fp32, 64 KB) and one outgoing R_i * g tile (bf16, 32 KB) in shared memory
-    static constexpr int X_BYTES = (EPI == PRE_OPROJ_SPD) ? 128 * 128 * 4 : 0, H_BYTES = (EPI == PRE_OPROJ_SPD) ? 128 * 128 * 2 : 0;
+    // PRE_OPROJ_SPD stages one outgoing R_i * g tile (bf16, 32 KB) in shared memory
+    static constexpr int X_BYTES = 0, H_BYTES = (EPI == PRE_OPROJ_SPD) ? 128 * 128 * 2 : 0;
     static constexpr int STAGES = (192 * 1024 - X_BYTES - H_BYTES) / STAGE_BYTES;
     static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
     static constexpr int SMEM_BYTES = RING_BYTES + X_BYTES + H_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
@@ -102,6 +104,26 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float *v)
                  : "memory");
 }
 
+// three 16-column chunks of this thread's row, one wait
+__device__ __forceinline__ void tmem_ld16x3(uint32_t ta, uint32_t tb, uint32_t tc3, float *va, float *vb, float *vc)
+{
+    uint32_t r[48];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%48];\n\t"
+                 "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%49];\n\t"
+                 "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47}, [%50];\n\t"
+                 "tcgen05.wait::ld.sync.aligned;"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]),
+                   "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]),
+                   "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47])
+                 : "r"(ta), "r"(tb), "r"(tc3)
+                 : "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { va[i] = __uint_as_float(r[i]); vb[i] = __uint_as_float(r[16 + i]); vc[i] = __uint_as_float(r[32 + i]); }
+}
+
 // 8 consecutive bf16 (16 bytes) from 8 floats
 __device__ __forceinline__ uint4 pack8(const float *v)
 {
@@ -114,6 +136,25 @@ __device__ __forceinline__ void unpack8(uint4 u, float *v)
     const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) { v[2 * i] = __uint_as_float(w[i] << 16); v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
+}
+
+// 32-byte global accesses (one row piece per thread: half as many instructions, whole 32-byte sectors)
+__device__ __forceinline__ void ldg8(const float *p, float *v)
+{
+    asm volatile("ld.global.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]) : "l"(p) : "memory");
+}
+__device__ __forceinline__ void stg8(float *p, const float *v)
+{
+    asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"l"(p), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
+}
+// 16 consecutive bf16 (32 bytes, 32-byte aligned) from 16 floats
+__device__ __forceinline__ void stg16_bf16(bf16 *p, const float *v)
+{
+    const uint4 a = pack8(v), b = pack8(v + 8);
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"l"(p), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w) : "memory");
 }
 
 __device__ __forceinline__ float row_rstd(const SumSq &s, int group, int m)
@@ -172,10 +213,8 @@ __device__ __forceinline__ void epi_qkv(const PreGemmArgs &g, const PreTile &t, 
 #pragma unroll
                 for (int i = 0; i < 16; ++i) { olo[i] = lo[i] * rs; ohi[i] = hi[i] * rs; }
             }
-            *(uint4 *)(dst + j0) = pack8(olo);
-            *(uint4 *)(dst + j0 + 8) = pack8(olo + 8);
-            *(uint4 *)(dst + half + j0) = pack8(ohi);
-            *(uint4 *)(dst + half + j0 + 8) = pack8(ohi + 8);
+            stg16_bf16(dst + j0, olo);
+            stg16_bf16(dst + half + j0, ohi);
         }
     }
 }
@@ -209,14 +248,8 @@ __device__ __forceinline__ float resid_chunk(const PreGemmArgs &g, long idx, int
 #pragma unroll
     for (int i = 0; i < 16; ++i) { r[i] = x[i] + y[i]; sq = fmaf(r[i], r[i], sq); }
     if (store_res) {
-        if (g.res_out) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) *(float4 *)(g.res_out + idx + 4 * i) = make_float4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
-        }
-        if (g.final_out) {
-            *(uint4 *)((bf16 *)g.final_out + idx) = pack8(r);
-            *(uint4 *)((bf16 *)g.final_out + idx + 8) = pack8(r + 8);
-        }
+        if (g.res_out) { stg8(g.res_out + idx, r); stg8(g.res_out + idx + 8, r + 8); }
+        if (g.final_out) stg16_bf16((bf16 *)g.final_out + idx, r);
     }
     if (hg) {
         float gn[16];
@@ -224,19 +257,15 @@ __device__ __forceinline__ float resid_chunk(const PreGemmArgs &g, long idx, int
         unpack8(*(const uint4 *)((const bf16 *)g.gain + n + 8), gn + 8);
 #pragma unroll
         for (int i = 0; i < 16; ++i) gn[i] *= r[i];
-        *(uint4 *)(hg + idx) = pack8(gn);
-        *(uint4 *)(hg + idx + 8) = pack8(gn + 8);
+        stg16_bf16(hg + idx, gn);
     }
     return sq;
 }
 
 __device__ __forceinline__ void load_x16(const float *p, float *x)
 {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const float4 v = *(const float4 *)(p + 4 * i);
-        x[4 * i] = v.x; x[4 * i + 1] = v.y; x[4 * i + 2] = v.z; x[4 * i + 3] = v.w;
-    }
+    ldg8(p, x);
+    ldg8(p + 8, x + 8);
 }
 
 __device__ __forceinline__ void epi_resid(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, int m, bool valid)
@@ -263,12 +292,32 @@ __device__ __forceinline__ void epi_resid(const PreGemmArgs &g, const PreTile &t
 
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-// One pass (device z) of an SPD o_proj tile.  The X tile sits in shared memory (xs: four 32-column
-// boxes of 128 rows, 128-byte swizzle); R_z * g is staged in hs (two 64-column bf16 boxes) and
-// leaves through a TMA store, as does X + sum_i Y_i after the last pass (written over the X tile).
-// Swizzled layouts: thread = row, eight consecutive rows hit eight different 16-byte columns.
-__device__ __forceinline__ float epi_oproj_spd(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, uint32_t ttot, int z,
-                                               uint8_t *xs, uint8_t *hs)
+// SPD o_proj: the X tile of an output tile is parked in tensor memory twice - once as is (every
+// device's R_i = X + Y_i needs it) and once as the start of X + sum_i Y_i - by the thread that owns
+// the row, while the MMA warp works on the first K slice.
+__device__ __forceinline__ void spd_park_x(const PreGemmArgs &g, const PreTile &t, uint32_t tx, uint32_t ttot, int m, bool valid)
+{
+#pragma unroll 1
+    for (int c = 0; c < 8; ++c) {
+        const int n = t.row0 + c * 16;
+        if (n >= g.H) break;
+        float x[16];
+        if (valid) load_x16(g.res_in + (long)m * g.H + n, x);
+        else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) x[i] = 0.f;
+        }
+        tmem_st16(tx + c * 16, x);
+        tmem_st16(ttot + c * 16, x);
+    }
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+
+// One pass (device z) of an SPD o_proj tile.  R_z * g is staged in hs (two 64-column bf16 boxes of
+// 128 rows, 128-byte swizzle: thread = row, eight consecutive rows hit eight different 16-byte
+// columns) and leaves through a TMA store; X + sum_i Y_i is written by the last pass.
+__device__ __forceinline__ float epi_oproj_spd(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, uint32_t tx, uint32_t ttot, int z,
+                                               int m, bool valid, uint8_t *hs)
 {
     const int T = g.batches, r = threadIdx.x, sw = r & 7;
     float ssq = 0.f;
@@ -276,25 +325,11 @@ __device__ __forceinline__ float epi_oproj_spd(const PreGemmArgs &g, const PreTi
     for (int c = 0; c < 8; ++c) {
         const int n = t.row0 + c * 16;
         if (n >= g.H) break;
-        float y[16], tot[16];
-        if (z == 0) {
-            tmem_ld16(tacc + c * 16, y);
+        float y[16], x[16], tot[16];
+        tmem_ld16x3(tacc + c * 16, tx + c * 16, ttot + c * 16, y, x, tot);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) tot[i] = y[i];
-        } else {
-            tmem_ld16x2(tacc + c * 16, ttot + c * 16, y, tot);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) tot[i] += y[i];
-        }
+        for (int i = 0; i < 16; ++i) tot[i] += y[i];
         if (z + 1 < T) tmem_st16(ttot + c * 16, tot);
-        // X: columns c*16 .. c*16+15 = box c/2, 16-byte chunks (c & 1) * 4 .. + 3 of this row
-        uint8_t *xrow = xs + (c >> 1) * 16384 + r * 128;
-        float x[16];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const float4 v = *(const float4 *)(xrow + ((((c & 1) * 4 + k) ^ sw) << 4));
-            x[4 * k] = v.x; x[4 * k + 1] = v.y; x[4 * k + 2] = v.z; x[4 * k + 3] = v.w;
-        }
         // device z only ever sees its own partial attention output: R_z = X + Y_z
         float gn[16];
         unpack8(*(const uint4 *)((const bf16 *)g.gain + n), gn);
@@ -308,12 +343,11 @@ __device__ __forceinline__ float epi_oproj_spd(const PreGemmArgs &g, const PreTi
         uint8_t *hrow = hs + (c >> 2) * 16384 + r * 128;
         *(uint4 *)(hrow + ((((c & 3) * 2) ^ sw) << 4)) = pack8(gn);
         *(uint4 *)(hrow + ((((c & 3) * 2 + 1) ^ sw) << 4)) = pack8(gn + 8);
-        if (z + 1 == T) {
-            // the residual carried to the block output collects every Y_i
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                *(float4 *)(xrow + ((((c & 1) * 4 + k) ^ sw) << 4)) =
-                    make_float4(x[4 * k] + tot[4 * k], x[4 * k + 1] + tot[4 * k + 1], x[4 * k + 2] + tot[4 * k + 2], x[4 * k + 3] + tot[4 * k + 3]);
+        if (z + 1 == T && valid) {
+            // the residual carried to the block output has collected every Y_i
+            float *dst = g.res_out + (long)m * g.H + n;
+            stg8(dst, tot);
+            stg8(dst + 8, tot + 8);
         }
     }
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
@@ -336,7 +370,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_prefill_kernel(const __grid_c
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
-    uint8_t *xs = gen_base + C::RING_BYTES, *hs = xs + C::X_BYTES; // PRE_OPROJ_SPD staging (1024-byte aligned)
+    uint8_t *hs = gen_base + C::RING_BYTES; // PRE_OPROJ_SPD staging (1024-byte aligned)
     const uint32_t bars = base + C::RING_BYTES + C::X_BYTES + C::H_BYTES; // full[S], empty[S], tmem_full[2], tmem_empty[2], x_full
     uint32_t *tmem_slot = (uint32_t *)(gen_base + C::RING_BYTES + C::X_BYTES + C::H_BYTES + 8 * (2 * S + 5));
     const uint32_t xfull_bar = bars + 8u * (2 * S + 4);
@@ -432,45 +466,35 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_prefill_kernel(const __grid_c
             const PreTile t = decode_tile(L, EPI, tile);
             const int m = t.m0 + warp * 32 + lane;
             const bool valid = m < g.t_rows;
-            if (EPI == PRE_OPROJ_SPD) {
-                // the X tile of this output tile: once the stores of the previous tile have read their source
-                if (threadIdx.x == 0) tma_store_wait_read();
-                epi_sync();
-                if (threadIdx.x == 0) {
-                    mbar_expect_tx(xfull_bar, C::X_BYTES);
-                    for (int bx = 0; bx < 4; ++bx) tma_load_3d(smem_u32(xs) + bx * 16384, &tm_x, t.row0 + 32 * bx, t.m0, 0, xfull_bar);
-                }
-            }
+            if (EPI == PRE_OPROJ_SPD) spd_park_x(g, t, tmem_base + lane_base + X_COL, tmem_base + lane_base + TOT_COL, m, valid);
             for (int pass = 0; pass < L.passes; ++pass, ++pc) {
                 const int buf = pc & 1;
                 if (!mbar_wait(tfull_bar(buf), (pc >> 1) & 1, g.err, abort_flag)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_PREFILL + EPI, TR_START);
                 const uint32_t tacc = tmem_base + lane_base + (uint32_t)(buf * BN);
                 if (EPI == PRE_QKV) epi_qkv(g, t, tacc, m, valid);
                 else if (EPI == PRE_GATEUP) epi_gateup(g, t, tacc, m, valid);
                 else if (EPI == PRE_RESID) epi_resid(g, t, tacc, m, valid);
                 else {
-                    if (pass == 0) {
-                        if (!mbar_wait(xfull_bar, tile_cnt & 1, g.err, abort_flag)) { ok = false; break; }
-                    } else {
-                        if (threadIdx.x == 0) tma_store_wait_read(); // the staging tile is free again
-                        epi_sync();
-                    }
-                    const float ssq = epi_oproj_spd(g, t, tacc, tmem_base + lane_base + TOT_COL, pass, xs, hs);
+                    if (threadIdx.x == 0) tma_store_wait_read(); // the staging tile is free again
+                    epi_sync();
+                    if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_PREFILL + EPI, TR_DEP_DONE);
+                    const float ssq = epi_oproj_spd(g, t, tacc, tmem_base + lane_base + X_COL, tmem_base + lane_base + TOT_COL, pass, m, valid, hs);
                     if (valid && g.ss_out) g.ss_out[((long)t.nt * g.batches + pass) * g.Mcap + m] = ssq;
                     fence_proxy_async();
+                    if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_PREFILL + EPI, TR_MAIN_DONE);
                     epi_sync();
                     if (threadIdx.x == 0) {
                         tma_store_3d(&tm_h, smem_u32(hs), t.row0, t.m0, pass);
                         tma_store_3d(&tm_h, smem_u32(hs) + 16384, t.row0 + 64, t.m0, pass);
-                        if (pass + 1 == L.passes)
-                            for (int bx = 0; bx < 4; ++bx) tma_store_3d(&tm_r, smem_u32(xs) + bx * 16384, t.row0 + 32 * bx, t.m0, 0);
                         tma_store_commit();
                     }
                 }
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(tempty_bar(buf)) : "memory");
+                if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_PREFILL + EPI, TR_END);
             }
         }
         if (EPI == PRE_OPROJ_SPD && threadIdx.x == 0) tma_store_wait_all(); // results in memory before the block ends
@@ -487,8 +511,7 @@ template <int EPI>
 cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, const PreLaunch &L, cudaStream_t st)
 {
     const bool spd = EPI == PRE_OPROJ_SPD;
-    const CUtensorMap &tx = *(const CUtensorMap *)(spd ? L.g.x_map : (const void *)&tt);
-    const CUtensorMap &tr = *(const CUtensorMap *)(spd ? L.g.r_map : (const void *)&tt);
+    const CUtensorMap &tx = tt, &tr = tt; // spare tensor-map slots
     const CUtensorMap &th = *(const CUtensorMap *)(spd ? L.g.h_map : (const void *)&tt);
     using C = PCfg<EPI>;
     static int n_sm = 0;
@@ -547,7 +570,7 @@ cudaError_t launch_gemm_prefill(PreEpilogue epi, const TcMap *const *weights, co
     if (g.num_kb < 1 || g.batches < 1 || g.batches > 8) return cudaErrorInvalidValue;
     if (epi == PRE_QKV && (256 % g.head_dim || g.head_dim < 32)) return cudaErrorInvalidValue;
     if ((epi == PRE_RESID || epi == PRE_OPROJ_SPD) && g.H % 16) return cudaErrorInvalidValue;
-    if (epi == PRE_OPROJ_SPD && (!g.x_map || !g.r_map || !g.h_map || !g.gain || !g.hg || !g.res_out)) return cudaErrorInvalidValue;
+    if (epi == PRE_OPROJ_SPD && (!g.h_map || !g.gain || !g.hg || !g.res_out)) return cudaErrorInvalidValue;
     if (epi == PRE_GATEUP && g.Fs % 8) return cudaErrorInvalidValue;
     const CUtensorMap *tw[3];
     for (int i = 0; i < 3; ++i) tw[i] = (const CUtensorMap *)weights[i < nw ? i : 0];

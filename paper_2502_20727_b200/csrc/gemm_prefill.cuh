@@ -45,9 +45,9 @@ struct PreGemmArgs {
     // GATEUP
     void *act;           // bf16 [tokens][F]
     int F, Fs;
-    // OPROJ_SPD: tiles go through shared memory with TMA (host pointers to tensor maps): res_in and res_out as
-    // fp32 [Mcap][H] maps with 32 x 128 boxes, hg as the bf16 [groups][Mcap][H] map with a 64 x 128 box
-    const void *x_map, *r_map, *h_map;
+    // OPROJ_SPD: the R_i * g planes leave through shared memory and TMA stores: host pointer to the tensor map of
+    // hg as bf16 [groups][Mcap][H] with a 64 x 128 box
+    const void *h_map;
 };
 
 // Weight maps: 256-row boxes (QKV, RESID), 128-row boxes (GATEUP: gate and up; OPROJ_SPD: the

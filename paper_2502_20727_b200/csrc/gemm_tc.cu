@@ -228,23 +228,6 @@ int make_operand_map(TcMap *out, const void *ptr, long k_inner, long rows, long 
     return r == CUDA_SUCCESS ? 0 : -3;
 }
 
-// rows x cols float32 matrix (row stride ld elements) as a 3-D map {cols, rows, 1} with a
-// {32, box_rows, 1} box (128 bytes wide) and the 128-byte swizzle.
-int make_f32_map(TcMap *out, const void *ptr, long cols, long rows, long ld_elems, int box_rows)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return -1;
-    if (((uintptr_t)ptr & 15) || (ld_elems * 4) % 16) return -2;
-    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, 1};
-    cuuint64_t strides[2] = {(cuuint64_t)ld_elems * 4, (cuuint64_t)ld_elems * rows * 4};
-    cuuint32_t box[3] = {32, (cuuint32_t)box_rows, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = fn((CUtensorMap *)out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void *>(ptr), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? 0 : -3;
-}
-
 int tc_token_box(bool swap, int tokens)
 {
     if (!swap) return BM;

@@ -32,9 +32,6 @@ struct TcGemmArgs {
 int make_operand_map(TcMap *out, const void *ptr, long k_inner, long rows, long batches, long ld_elems,
                      long batch_stride_elems, int box_rows);
 
-// rows x cols float32 matrix as a map with a 32-column (128-byte) x box_rows box, 128-byte swizzle.
-int make_f32_map(TcMap *out, const void *ptr, long cols, long rows, long ld_elems, int box_rows);
-
 // Box rows of the token-side operand for a given token count (swap: 16/32/64, else 128).
 int tc_token_box(bool swap, int tokens);
 int tc_weight_box(bool swap);

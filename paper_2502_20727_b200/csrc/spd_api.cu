@@ -97,8 +97,7 @@ struct Ctx {
     // activation tensor maps, by buffer and token box (16, 32, 64, 128), built on first use
     TcMap act_maps[AB_COUNT][4];
     bool act_map_ready[AB_COUNT][4];
-    TcMap res_maps[2];           // fp32 residual streams, 32 x 128 boxes (prefill SPD o_proj)
-    bool res_maps_ready;
+
     // optional per-kernel-kind timing (spd_profile_begin / spd_profile_end)
     bool profiling;
     std::vector<cudaEvent_t> ev_pool;
@@ -599,15 +598,8 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
             MAP_OR_FAIL(am, act_map(c, AB_ATTN_SHARD, 128));
             g.w_rows[0] = H; g.num_kb = cdiv(qd / Tn, 64); g.batches = Tn;
             g.res_in = c->res[0]; g.res_out = c->res[1]; g.gain = w.mlp_norm; g.hg = c->h; g.hg_stride = Mc * H; g.ss_out = c->ss_mlp;
-            if (!c->res_maps_ready) {
-                if (make_f32_map(&c->res_maps[0], c->res[0], H, Mc, H, 128) || make_f32_map(&c->res_maps[1], c->res[1], H, Mc, H, 128)) {
-                    g_last_cuda_error = (int)cudaErrorInvalidValue;
-                    return SPD_ECUDA;
-                }
-                c->res_maps_ready = true;
-            }
             MAP_OR_FAIL(hm, act_map(c, AB_H, 128));
-            g.x_map = &c->res_maps[0]; g.r_map = &c->res_maps[1]; g.h_map = hm;
+            g.h_map = hm;
             LAUNCH(K_OPROJ, launch_gemm_prefill(PRE_OPROJ_SPD, wmaps, *am, g, st));
             mlp_tiles = pre_ss_tiles(PRE_OPROJ_SPD, H); mlp_groups = Tn;
         }
@@ -753,7 +745,7 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     c.profiling = false;
     c.ev_used = 0;
     memset(c.act_map_ready, 0, sizeof(c.act_map_ready));
-    c.res_maps_ready = false;
+
     if (dims->dtype == 1) {
         rc = build_weight_maps(c);
         if (rc) { delete h; return rc; }

@@ -7,7 +7,7 @@
 namespace spd {
 
 enum TraceEvent : int { TR_START = 0, TR_DEP_DONE = 1, TR_MAIN_DONE = 2, TR_ARRIVED = 3, TR_END = 4 };
-enum TraceKernel : int { TRK_QKV = 0, TRK_OPROJ = 1, TRK_GATEUP = 2, TRK_DOWN = 3, TRK_ATTN = 4, TRK_PROLOGUE = 5 };
+enum TraceKernel : int { TRK_QKV = 0, TRK_OPROJ = 1, TRK_GATEUP = 2, TRK_DOWN = 3, TRK_ATTN = 4, TRK_PROLOGUE = 5, TRK_PREFILL = 8 /* + PreEpilogue */ };
 
 #ifdef SPD_TRACE
 constexpr unsigned TRACE_CAP = 1u << 21;
