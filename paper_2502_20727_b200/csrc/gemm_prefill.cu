@@ -33,8 +33,8 @@ template <int EPI> struct PCfg {
     static constexpr int BN = (EPI == PRE_OPROJ_SPD) ? 128 : 256;
     static constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    // PRE_OPROJ_SPD stages one outgoing R_i * g tile (bf16, 32 KB) in shared memory
-    static constexpr int X_BYTES = 0, H_BYTES = (EPI == PRE_OPROJ_SPD) ? 128 * 128 * 2 : 0;
+    // PRE_OPROJ_SPD stages outgoing R_i * g tiles (bf16, 32 KB each) in shared memory
+    static constexpr int X_BYTES = 0, H_BYTES = (EPI == PRE_OPROJ_SPD) ? 2 * 128 * 128 * 2 : 0; // two staging tiles
     static constexpr int STAGES = (192 * 1024 - X_BYTES - H_BYTES) / STAGE_BYTES;
     static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
     static constexpr int SMEM_BYTES = RING_BYTES + X_BYTES + H_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
@@ -122,6 +122,27 @@ __device__ __forceinline__ void tmem_ld16x3(uint32_t ta, uint32_t tb, uint32_t t
                  : "memory");
 #pragma unroll
     for (int i = 0; i < 16; ++i) { va[i] = __uint_as_float(r[i]); vb[i] = __uint_as_float(r[16 + i]); vc[i] = __uint_as_float(r[32 + i]); }
+}
+
+// three 32-column chunks of this thread's row, one wait
+__device__ __forceinline__ void tmem_ld32x3(uint32_t ta, uint32_t tb, uint32_t tc3, float *va, float *vb, float *vc)
+{
+    uint32_t r[96];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%96];\n\t"
+                 "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%97];\n\t"
+                 "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%64,%65,%66,%67,%68,%69,%70,%71,%72,%73,%74,%75,%76,%77,%78,%79,%80,%81,%82,%83,%84,%85,%86,%87,%88,%89,%90,%91,%92,%93,%94,%95}, [%98];\n\t"
+                 "tcgen05.wait::ld.sync.aligned;"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63]), "=r"(r[64]), "=r"(r[65]), "=r"(r[66]), "=r"(r[67]), "=r"(r[68]), "=r"(r[69]), "=r"(r[70]), "=r"(r[71]), "=r"(r[72]), "=r"(r[73]), "=r"(r[74]), "=r"(r[75]), "=r"(r[76]), "=r"(r[77]), "=r"(r[78]), "=r"(r[79]), "=r"(r[80]), "=r"(r[81]), "=r"(r[82]), "=r"(r[83]), "=r"(r[84]), "=r"(r[85]), "=r"(r[86]), "=r"(r[87]), "=r"(r[88]), "=r"(r[89]), "=r"(r[90]), "=r"(r[91]), "=r"(r[92]), "=r"(r[93]), "=r"(r[94]), "=r"(r[95])
+                 : "r"(ta), "r"(tb), "r"(tc3)
+                 : "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) { va[i] = __uint_as_float(r[i]); vb[i] = __uint_as_float(r[32 + i]); vc[i] = __uint_as_float(r[64 + i]); }
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float *v)
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+                 :: "r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])), "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])), "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+                 : "memory");
 }
 
 // 8 consecutive bf16 (16 bytes) from 8 floats
@@ -322,32 +343,35 @@ __device__ __forceinline__ float epi_oproj_spd(const PreGemmArgs &g, const PreTi
     const int T = g.batches, r = threadIdx.x, sw = r & 7;
     float ssq = 0.f;
 #pragma unroll 1
-    for (int c = 0; c < 8; ++c) {
-        const int n = t.row0 + c * 16;
+    for (int c = 0; c < 4; ++c) { // 32 columns per round: few tensor-memory round trips on the critical path
+        const int n = t.row0 + c * 32;
         if (n >= g.H) break;
-        float y[16], x[16], tot[16];
-        tmem_ld16x3(tacc + c * 16, tx + c * 16, ttot + c * 16, y, x, tot);
+        float y[32], x[32], tot[32];
+        tmem_ld32x3(tacc + c * 32, tx + c * 32, ttot + c * 32, y, x, tot);
 #pragma unroll
-        for (int i = 0; i < 16; ++i) tot[i] += y[i];
-        if (z + 1 < T) tmem_st16(ttot + c * 16, tot);
+        for (int i = 0; i < 32; ++i) tot[i] += y[i];
+        if (z + 1 < T) tmem_st32(ttot + c * 32, tot);
         // device z only ever sees its own partial attention output: R_z = X + Y_z
-        float gn[16];
-        unpack8(*(const uint4 *)((const bf16 *)g.gain + n), gn);
-        unpack8(*(const uint4 *)((const bf16 *)g.gain + n + 8), gn + 8);
+        uint8_t *hrow = hs + (c >> 1) * 16384 + r * 128;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const float ri = x[i] + y[i];
-            ssq = fmaf(ri, ri, ssq);
-            gn[i] *= ri;
+        for (int q = 0; q < 4; ++q) {
+            float gn[8];
+            const bool in_h = n + 8 * q < g.H; // a tile may reach past the last column
+            unpack8(in_h ? *(const uint4 *)((const bf16 *)g.gain + n + 8 * q) : make_uint4(0, 0, 0, 0), gn);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float ri = in_h ? x[8 * q + i] + y[8 * q + i] : 0.f;
+                ssq = fmaf(ri, ri, ssq);
+                gn[i] *= ri;
+            }
+            *(uint4 *)(hrow + ((((c & 1) * 4 + q) ^ sw) << 4)) = pack8(gn);
         }
-        uint8_t *hrow = hs + (c >> 2) * 16384 + r * 128;
-        *(uint4 *)(hrow + ((((c & 3) * 2) ^ sw) << 4)) = pack8(gn);
-        *(uint4 *)(hrow + ((((c & 3) * 2 + 1) ^ sw) << 4)) = pack8(gn + 8);
         if (z + 1 == T && valid) {
             // the residual carried to the block output has collected every Y_i
             float *dst = g.res_out + (long)m * g.H + n;
-            stg8(dst, tot);
-            stg8(dst + 8, tot + 8);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (n + 8 * k < g.H) stg8(dst + 8 * k, tot + 8 * k);
         }
     }
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
@@ -477,17 +501,19 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_prefill_kernel(const __grid_c
                 else if (EPI == PRE_GATEUP) epi_gateup(g, t, tacc, m, valid);
                 else if (EPI == PRE_RESID) epi_resid(g, t, tacc, m, valid);
                 else {
-                    if (threadIdx.x == 0) tma_store_wait_read(); // the staging tile is free again
+                    // two staging tiles in turn: the store issued two passes ago has read its source
+                    uint8_t *hst = hs + (pc & 1) * 32768;
+                    if (threadIdx.x == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                     epi_sync();
                     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_PREFILL + EPI, TR_DEP_DONE);
-                    const float ssq = epi_oproj_spd(g, t, tacc, tmem_base + lane_base + X_COL, tmem_base + lane_base + TOT_COL, pass, m, valid, hs);
+                    const float ssq = epi_oproj_spd(g, t, tacc, tmem_base + lane_base + X_COL, tmem_base + lane_base + TOT_COL, pass, m, valid, hst);
                     if (valid && g.ss_out) g.ss_out[((long)t.nt * g.batches + pass) * g.Mcap + m] = ssq;
                     fence_proxy_async();
                     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_PREFILL + EPI, TR_MAIN_DONE);
                     epi_sync();
                     if (threadIdx.x == 0) {
-                        tma_store_3d(&tm_h, smem_u32(hs), t.row0, t.m0, pass);
-                        tma_store_3d(&tm_h, smem_u32(hs) + 16384, t.row0 + 64, t.m0, pass);
+                        tma_store_3d(&tm_h, smem_u32(hst), t.row0, t.m0, pass);
+                        tma_store_3d(&tm_h, smem_u32(hst) + 16384, t.row0 + 64, t.m0, pass);
                         tma_store_commit();
                     }
                 }
