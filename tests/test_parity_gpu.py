@@ -132,6 +132,48 @@ def test_gqa_decode_long_ragged_context_on_synthetic_cache():
     assert p.stack.device_error() == 0
 
 
+@pytest.mark.parametrize("mask", [(0,), (1,)])
+def test_prefill_over_several_tiles_at_full_width(mask):
+    """configs[1] dims, one layer, one 300-token prompt: three 128-token GEMM tiles with a ragged
+    tail, three 128-row attention tiles, every column tile of the real widths."""
+    w = si.WORKLOADS["c2"].with_(n_layers=1, mask=mask)
+    run_case(w, mask, 1, 300, 1, check_cache=True)
+
+
+def test_single_token_prompt_and_single_sequence():
+    """Degenerate sizes: a one-token prompt (prefill of M = 1), then decode with batch 1."""
+    w = si.Workload("tiny", "bf16", 2, 256, 4, 2, 64, 512, 2, (0, 1), 1, 1, 3)
+    run_case(w, (0, 1), 1, 1, 3)
+
+
+def test_context_up_to_the_last_slot_of_the_last_page():
+    """Decode until the cache is exactly full (max_seq_len = pages * 16): the last step writes the last slot."""
+    w = si.Workload("tiny", "bf16", 1, 256, 4, 4, 64, 512, 2, (0,), 2, 29, 3)
+    run_case(w, (0,), 2, 29, 3)  # 29 + 3 = 32 = two full pages
+
+
+def test_out_of_range_page_is_flagged_not_followed():
+    """A block-table entry outside [0, n_pages) must set the device error flag; the kernels skip or
+    clamp the access instead of touching memory outside the page tensors."""
+    w = si.Workload("tiny", "bf16", 1, 256, 4, 4, 64, 512, 2, (0,), 2, 20, 1)
+    p = Pair(w, B=2, max_len=24)
+    p.prefill(20)
+    assert p.stack.device_error() == 0
+    bad = p.block_table.clone()
+    bad[1, 1] = p.n_pages + 7  # the page the next token of sequence 1 would go to
+    x = si.make_hidden(w, (2, w.hidden), "cpu", 0, 1).to(p.device)
+    seq = torch.full((2,), 20, dtype=torch.int32, device=p.device)
+    p.stack.set_graphs(False)
+    p.stack.decode_step(x, seq, bad, 21)
+    torch.cuda.synchronize()
+    assert p.stack.device_error() & 1
+    assert p.stack.device_error() == 0  # reading clears it
+    # the stack is still usable
+    out = p.stack.decode_step(x, seq, p.block_table, 21)
+    torch.cuda.synchronize()
+    assert torch.isfinite(out.float()).all() and p.stack.device_error() == 0
+
+
 def test_run_twice_bitwise_identical():
     w = si.Workload("small", "bf16", 2, 512, 8, 8, 64, 1024, 4, (0, 1), 4, 33, 2)
     outs = []
