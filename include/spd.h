@@ -172,6 +172,39 @@ int spd_gemm_bf16(const void *a, const void *w, float *c, int32_t M, int32_t N, 
 int spd_gemm_bf16_sum_static(const void *a, const void *w, float *c, int32_t M, int32_t N, int32_t K, int32_t batches,
                              int32_t a_batched, int32_t splits, int32_t swap, int32_t *err_flag, void *stream);
 
+/* Replace the per-block mask of a context (same meaning as in spd_create).  A mask with an SPD
+ * block needs the larger workspace of such a stack: SPD_EWORKSPACE if the context was created
+ * from an all-sync mask.  Drops the captured decode graphs.  Errors: SPD_ENULL, SPD_EWORKSPACE. */
+int spd_set_mask(spd_ctx *ctx, const uint8_t *sync_mask);
+
+/* Block-wise sync-sensitivity identification (Sec. 4.2.1) on this stack, with the mean squared
+ * difference from the all-TP output as the quality metric in place of perplexity (this path
+ * has no LM head).  For i = L-1 .. 0 the prompt batch x is run with blocks i .. L-1 as SPD blocks
+ * and blocks 0 .. i-1 as TP blocks; metric[i] is that output's mean squared difference from the
+ * all-TP output (metric[L] = 0), and sensitivity[i] = metric[i] - metric[i+1]: what turning
+ * block i into an SPD block adds when every later block already is one.
+ *   x, block_table, B, S : as for spd_prefill (the caches of those rows are overwritten by each pass)
+ *   ref_out, tmp_out     : device scratch, [B, S, hidden] storage dtype each (ref_out returns the all-TP output)
+ *   sensitivity          : host [n_layers];  metric : host [n_layers + 1] or null
+ * Runs n_layers + 1 prefills, synchronises `stream`, restores the context's mask.
+ * Errors: those of spd_prefill and spd_set_mask. */
+int spd_sensitivity_scan(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int32_t *block_table, int32_t max_pages,
+                         void *ref_out, void *tmp_out, double *sensitivity, double *metric, void *stream);
+
+/* Algorithm 1: rank the blocks by sensitivity (ascending, ties by index), turn the first n_spd
+ * into SPD blocks and label each by tier: sensitivity <= tau1 in-sensitive (zero-shot dropping,
+ * Sec. 4.2.2), <= tau2 sensitive (wants block-to-block distillation first, Sec. 4.2.3), else
+ * extremely sensitive (wants head grouping and distillation, Sec. 4.2.4).  The library only
+ * runs blocks; distillation and head grouping produce different weights for the same kernels.
+ *   sync_mask : host out [n_blocks], 1 = stays a TP block, 0 = SPD block;  tier : host out [n_blocks]
+ * Pure host function.  Errors: SPD_ENULL, SPD_EINVAL (n_spd outside [0, n_blocks], tau1 > tau2). */
+#define SPD_TIER_TP 0
+#define SPD_TIER_ISB 1
+#define SPD_TIER_SB 2
+#define SPD_TIER_ESB 3
+int spd_alg1_plan(const double *sensitivity, int32_t n_blocks, int32_t n_spd, double tau1, double tau2, uint8_t *sync_mask,
+                  uint8_t *tier);
+
 /* Number of shard sums ("sync-points", Sec. 3) one forward pass of this stack executes:
  * 2 per TP block, 1 per SPD block. */
 int spd_sync_points(const spd_ctx *ctx);

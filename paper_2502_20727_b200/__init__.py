@@ -23,7 +23,7 @@ EXPORTS = ("spd_workspace_bytes", "spd_create", "spd_prefill", "spd_decode_step"
            "spd_launches_per_decode_step", "spd_device_error", "spd_destroy", "spd_status_string",
            "spd_last_cuda_error", "spd_profile_begin", "spd_profile_end", "spd_profile_kinds",
            "spd_profile_kind_name", "spd_gemm_bf16", "spd_set_graphs", "spd_gemm_bf16_sum_static",
-           "spd_set_tuning")
+           "spd_set_tuning", "spd_set_mask", "spd_sensitivity_scan", "spd_alg1_plan")
 
 
 class SpdError(RuntimeError):
@@ -72,6 +72,10 @@ def load_library() -> ctypes.CDLL:
     lib.spd_last_cuda_error.argtypes = []
     lib.spd_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, vp]
     lib.spd_set_graphs.argtypes = [vp, i32]
+    lib.spd_set_mask.argtypes = [vp, vp]
+    lib.spd_sensitivity_scan.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, ctypes.POINTER(ctypes.c_double),
+                                         ctypes.POINTER(ctypes.c_double), vp]
+    lib.spd_alg1_plan.argtypes = [ctypes.POINTER(ctypes.c_double), i32, i32, ctypes.c_double, ctypes.c_double, vp, vp]
     lib.spd_set_tuning.argtypes = [vp, ctypes.c_char_p, i32]
     lib.spd_gemm_bf16_sum_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, vp]
     lib.spd_profile_begin.argtypes = [vp]
@@ -153,6 +157,20 @@ def gemm_bf16_sum_static(a: torch.Tensor, w: torch.Tensor, out: torch.Tensor, er
                                             1 if a_batched else 0, splits, 1 if swap else 0, err.data_ptr(),
                                             _stream_ptr()))
     return out
+
+
+TIER_NAMES = ("TP", "ISB", "SB", "ESB")
+
+
+def alg1_plan(sensitivity: Sequence[float], n_spd: int, tau1: float, tau2: float):
+    """Algorithm 1 on a list of block sensitivities; returns (sync_mask, tiers), see spd_alg1_plan."""
+    lib = load_library()
+    n = len(sensitivity)
+    s = (ctypes.c_double * n)(*[float(v) for v in sensitivity])
+    mask = (ctypes.c_uint8 * n)()
+    tier = (ctypes.c_uint8 * n)()
+    _check("spd_alg1_plan", lib.spd_alg1_plan(s, n, int(n_spd), float(tau1), float(tau2), mask, tier))
+    return [int(v) for v in mask], [int(v) for v in tier]
 
 
 class SpdStack:
@@ -247,6 +265,29 @@ class SpdStack:
             _check("spd_profile_end", self.lib.spd_profile_end(self._ctx, _stream_ptr(), ms, cnt))
         return {self.lib.spd_profile_kind_name(i).decode(): {"ms": float(ms[i]), "launches": int(cnt[i])}
                 for i in range(n)}
+
+    def set_mask(self, sync_mask: Sequence[int]):
+        """Replace the per-block mask (1 = TP block, 0 = SPD block); see spd_set_mask."""
+        if len(sync_mask) != self.dims.n_layers:
+            raise ValueError("one mask entry per layer")
+        m = (ctypes.c_uint8 * len(sync_mask))(*[1 if v else 0 for v in sync_mask])
+        _check("spd_set_mask", self.lib.spd_set_mask(self._ctx, m))
+        self.mask = m
+
+    def sensitivity_scan(self, x: torch.Tensor, block_table: torch.Tensor):
+        """Sec. 4.2.1 scan on prompt batch x [B, S, hidden]; returns (sensitivity[L], metric[L+1]);
+        see spd_sensitivity_scan."""
+        B, S, H = x.shape
+        self._check_io(x, block_table)
+        L = self.dims.n_layers
+        ref, tmp = torch.empty_like(x), torch.empty_like(x)
+        sens = (ctypes.c_double * L)()
+        met = (ctypes.c_double * (L + 1))()
+        with torch.cuda.device(self.device):
+            _check("spd_sensitivity_scan",
+                   self.lib.spd_sensitivity_scan(self._ctx, x.data_ptr(), B, S, block_table.data_ptr(), block_table.shape[1],
+                                                 ref.data_ptr(), tmp.data_ptr(), sens, met, _stream_ptr()))
+        return [float(v) for v in sens], [float(v) for v in met]
 
     def set_graphs(self, enabled: bool):
         """Replay decode steps from captured CUDA graphs (default on); see spd_set_graphs."""

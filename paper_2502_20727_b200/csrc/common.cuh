@@ -176,4 +176,7 @@ inline int decode_heads_per_block_mma(int group) { return group % 8 == 0 ? 8 : 4
 template <typename T> cudaError_t launch_prefill_attention(const AttnArgs &a, cudaStream_t st);
 template <typename T> cudaError_t launch_decode_attention(const AttnArgs &a, cudaStream_t st);
 
+// part[b] = sum over block b's slice of (a - r)^2, fixed order (strategy.cu)
+cudaError_t launch_sq_diff(const void *a, const void *r, long n, int dtype_bf16, float *part, int n_blocks, cudaStream_t st);
+
 } // namespace spd

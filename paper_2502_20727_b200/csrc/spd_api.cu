@@ -852,6 +852,63 @@ int spd_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_l
     return SPD_OK;
 }
 
+static void drop_graphs(Ctx &c)
+{
+    for (GraphEntry &g : c.graphs) cudaGraphExecDestroy(g.exec);
+    c.graphs.clear();
+}
+
+int spd_set_mask(spd_ctx *ctx, const uint8_t *sync_mask)
+{
+    if (!ctx || !sync_mask) return SPD_ENULL;
+    Ctx &c = ctx->c;
+    bool any_spd = false;
+    for (int l = 0; l < c.d.n_layers; ++l) any_spd |= sync_mask[l] == 0;
+    if (any_spd && !c.any_spd) return SPD_EWORKSPACE;
+    c.mask.assign(sync_mask, sync_mask + c.d.n_layers);
+    drop_graphs(c);
+    return SPD_OK;
+}
+
+int spd_sensitivity_scan(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int32_t *block_table, int32_t max_pages,
+                         void *ref_out, void *tmp_out, double *sensitivity, double *metric, void *stream)
+{
+    if (!ctx || !ref_out || !tmp_out || !sensitivity) return SPD_ENULL;
+    Ctx &c = ctx->c;
+    const int L = c.d.n_layers;
+    if (!c.any_spd) return SPD_EWORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const std::vector<uint8_t> saved = c.mask;
+    std::vector<uint8_t> m(L, 1);
+    std::vector<double> met(L + 1, 0.0);
+    constexpr int NB = 1024;
+    std::vector<float> part(NB);
+    float *dpart = c.part_o; // attention split scratch: at least NB floats, idle between the passes
+    const long n = (long)B * S * c.d.hidden;
+    auto restore = [&](int rc) { c.mask = saved; drop_graphs(c); return rc; };
+    if ((size_t)c.d.max_batch * c.d.n_q_heads * 32 * c.d.head_dim < (size_t)NB) return SPD_EWORKSPACE;
+    drop_graphs(c);
+    c.mask = m; // all TP
+    int rc = spd_prefill(ctx, x, B, S, block_table, max_pages, ref_out, stream);
+    if (rc) return restore(rc);
+    for (int i = L - 1; i >= 0; --i) {
+        m[i] = 0; // blocks i .. L-1 are SPD blocks now
+        c.mask = m;
+        rc = spd_prefill(ctx, x, B, S, block_table, max_pages, tmp_out, stream);
+        if (rc) return restore(rc);
+        cudaError_t e = launch_sq_diff(tmp_out, ref_out, n, c.d.dtype == 1, dpart, NB, st);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(part.data(), dpart, NB * sizeof(float), cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+        if (e != cudaSuccess) { g_last_cuda_error = (int)e; return restore(SPD_ECUDA); }
+        double tot = 0.0;
+        for (int b = 0; b < NB; ++b) tot += (double)part[b];
+        met[i] = tot / (double)n;
+    }
+    for (int i = 0; i < L; ++i) sensitivity[i] = met[i] - met[i + 1];
+    if (metric) for (int i = 0; i <= L; ++i) metric[i] = met[i];
+    return restore(SPD_OK);
+}
+
 int spd_set_graphs(spd_ctx *ctx, int32_t enabled)
 {
     if (!ctx) return SPD_ENULL;
