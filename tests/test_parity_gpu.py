@@ -174,6 +174,24 @@ def test_out_of_range_page_is_flagged_not_followed():
     assert torch.isfinite(out.float()).all() and p.stack.device_error() == 0
 
 
+@pytest.mark.parametrize("B", [40, 70])
+def test_bf16_decode_batches_beyond_32(B):
+    """Decode token tiles of 64 (batch 40) and two token tiles (batch 70), SPD and TP blocks."""
+    w = si.Workload("wide", "bf16", 2, 256, 4, 4, 64, 512, 2, (0, 1), B, 18, 2)
+    run_case(w, (0, 1), B, 18, 2, check_cache=False)
+
+
+def test_bf16_head_dim_32_without_rope():
+    """Eight heads per 256-row prefill tile, four per 128-row decode tile, rotary embedding off."""
+    w = si.Workload("d32", "bf16", 2, 256, 8, 4, 32, 512, 4, (0, 1), 3, 21, 2).with_(rope_base=0.0)
+    run_case(w, (0, 1), 3, 21, 2)
+
+
+def test_bf16_hidden_not_a_multiple_of_16_takes_the_unfused_prefill():
+    w = si.Workload("h264", "bf16", 1, 264, 4, 4, 64, 512, 2, (0,), 2, 10, 1)
+    run_case(w, (0,), 2, 10, 1)
+
+
 def test_run_twice_bitwise_identical():
     w = si.Workload("small", "bf16", 2, 512, 8, 8, 64, 1024, 4, (0, 1), 4, 33, 2)
     outs = []
