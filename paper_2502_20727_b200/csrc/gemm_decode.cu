@@ -301,12 +301,41 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
     const int n_kb = kb_end - kb_begin;
 
     pdl_launch_dependents();
-    if (threadIdx.x == 0) {
+    const int a_z = g.w_batched ? t.z : 0, b_z = g.t_batched ? t.z : 0;
+    const uint64_t stream_once = policy_evict_first();
+    auto load_w = [&](int s, int kx) {
+        const uint32_t sa = base + s * C::STAGE_BYTES;
+        if (SUB == 1) tma_load_3d_hint(sa, tm_w, kx, t.w_row0, a_z, full_bar(s), stream_once);
+        else {
+            tma_load_3d_hint(sa, &tm_w0, kx, t.w_row0, a_z, full_bar(s), stream_once);
+            tma_load_3d_hint(sa + ROWS * BK * 2, &tm_w1, kx, t.w_row0, a_z, full_bar(s), stream_once);
+        }
+    };
+    const int pre = n_kb < C::STAGES ? n_kb : C::STAGES;
+    if (warp == 4 && lane == 0) {
+        // The TMA thread sets up the barriers itself and requests the first ring of weight tiles
+        // at once: weights do not depend on the preceding kernel, and they need neither the
+        // accumulator allocation nor the other warps, so this GEMM's weight stream starts the
+        // moment the block is resident - under the tail of whatever ran before.
         SPD_TRACE_EVENT(EPI, TR_START);
         for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         mbar_init(tmem_full_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(tm_w) : "memory");
+        if (SUB == 2) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_w1) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_t) : "memory");
+        for (int i = 0; i < pre; ++i) {
+            mbar_expect_tx(full_bar(i), C::STAGE_BYTES);
+            load_w(i, (kb_begin + i) * BK);
+        }
+        // optionally the K blocks after the ring are pulled into L2
+        const int pf_end = n_kb < pre + g.l2_prefetch_kb ? n_kb : pre + g.l2_prefetch_kb;
+        for (int i = pre; i < pf_end; ++i) {
+            const int kx = (kb_begin + i) * BK;
+            if (SUB == 1) tma_prefetch_l2_3d(tm_w, kx, t.w_row0, a_z);
+            else { tma_prefetch_l2_3d(&tm_w0, kx, t.w_row0, a_z); tma_prefetch_l2_3d(&tm_w1, kx, t.w_row0, a_z); }
+        }
     }
     if (warp == 5) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::TMEM_COLS) : "memory");
@@ -317,38 +346,8 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_acc = *tmem_slot;
 
-    const int a_z = g.w_batched ? t.z : 0, b_z = g.t_batched ? t.z : 0;
-
     if (warp == 4) {
         if (lane == 0) {
-            // TMA producer.  Weights do not depend on the preceding kernel: the first ring of
-            // weight tiles is requested before waiting for it, so this GEMM's weight stream
-            // starts under the tail of whatever ran before.
-            asm volatile("prefetch.tensormap [%0];" ::"l"(tm_w) : "memory");
-            if (SUB == 2) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_w1) : "memory");
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_t) : "memory");
-            const uint64_t stream_once = policy_evict_first();
-            auto load_w = [&](int s, int kx) {
-                const uint32_t sa = base + s * C::STAGE_BYTES;
-                if (SUB == 1) tma_load_3d_hint(sa, tm_w, kx, t.w_row0, a_z, full_bar(s), stream_once);
-                else {
-                    tma_load_3d_hint(sa, &tm_w0, kx, t.w_row0, a_z, full_bar(s), stream_once);
-                    tma_load_3d_hint(sa + ROWS * BK * 2, &tm_w1, kx, t.w_row0, a_z, full_bar(s), stream_once);
-                }
-            };
-            const int pre = n_kb < C::STAGES ? n_kb : C::STAGES;
-            for (int i = 0; i < pre; ++i) {
-                mbar_expect_tx(full_bar(i), C::STAGE_BYTES);
-                load_w(i, (kb_begin + i) * BK);
-            }
-            // ... and the K blocks after the ring are pulled into L2, so that HBM keeps
-            // streaming this GEMM's weights while the preceding kernel drains.
-            const int pf_end = n_kb < pre + g.l2_prefetch_kb ? n_kb : pre + g.l2_prefetch_kb;
-            for (int i = pre; i < pf_end; ++i) {
-                const int kx = (kb_begin + i) * BK;
-                if (SUB == 1) tma_prefetch_l2_3d(tm_w, kx, t.w_row0, a_z);
-                else { tma_prefetch_l2_3d(&tm_w0, kx, t.w_row0, a_z); tma_prefetch_l2_3d(&tm_w1, kx, t.w_row0, a_z); }
-            }
             pdl_wait();
             SPD_TRACE_EVENT(EPI, TR_DEP_DONE);
             for (int i = 0; i < n_kb; ++i) {
