@@ -205,6 +205,33 @@ int spd_sensitivity_scan(spd_ctx *ctx, const void *x, int32_t B, int32_t S, cons
 int spd_alg1_plan(const double *sensitivity, int32_t n_blocks, int32_t n_spd, double tau1, double tau2, uint8_t *sync_mask,
                   uint8_t *tier);
 
+/* SPD-aware attention head grouping (Sec. 4.2.4), measurements.  The prompt batch x runs through
+ * blocks 0 .. layer-1 as TP blocks (Sec. 4.2.3) and through block `layer` as an SPD block with the weights as
+ * they are now (device i = head rows [i*nq/T, (i+1)*nq/T), MLP partition m = FFN rows [m*F/T, (m+1)*F/T)):
+ *   dist  : host out [nq][nq], Euclidean distance between the attention-score vectors of two heads over all
+ *           prompts (softmax probabilities, causal, zeros above the diagonal) - the d(sigma, sigma) of Eq. 2
+ *   norms : host out [T][T], norms[i][m] = Frobenius norm over all tokens of MLP_m(rmsnorm(X + Y_i)), the
+ *           output of MLP partition m (its slice of gate/up/down, before any sum) on device i's input - Eq. 3
+ *   sigma_scratch : device, nq * B * S * S floats;  dist_dev : device, nq * nq floats
+ * bf16 stacks only; B * S <= max_prefill_tokens; overwrites the caches of those rows for blocks 0 .. layer;
+ * synchronises `stream`.  Errors: SPD_ENULL, SPD_EINVAL, SPD_ECAPACITY, SPD_EWORKSPACE (context created from
+ * an all-sync mask), SPD_ECUDA. */
+int spd_head_grouping_stats(spd_ctx *ctx, int32_t layer, const void *x, int32_t B, int32_t S, const int32_t *block_table,
+                            int32_t max_pages, float *sigma_scratch, float *dist_dev, float *dist, double *norms, void *stream);
+
+/* Head scattering, Eq. 2: split the heads into T equal sets so that the sum, over the sets, of the pairwise
+ * distances inside a set is largest (similar heads end up on different devices).  The query heads of one KV head
+ * stay together: a unit is heads_per_unit consecutive heads, the distance of two units the sum over their head
+ * pairs.  Exhaustive for up to 12 units, else a greedy start improved by pairwise swaps until none helps.
+ *   dist : host [n_heads][n_heads];  device_of_unit : host out [n_heads / heads_per_unit]
+ * Pure host function.  Errors: SPD_ENULL, SPD_EINVAL (units not divisible by T, ...). */
+int spd_head_scatter(const float *dist, int32_t n_heads, int32_t heads_per_unit, int32_t T, int32_t *device_of_unit, double *objective);
+
+/* MLP matching, Eq. 3: the assignment of MLP partitions to devices with the largest sum of output norms, over
+ * all T! matchings.  norms : host [T][T] as from spd_head_grouping_stats;  mlp_of_device : host out [T].
+ * Pure host function.  Errors: SPD_ENULL, SPD_EINVAL (T > 8). */
+int spd_mlp_match(const double *norms, int32_t T, int32_t *mlp_of_device, double *objective);
+
 /* Number of shard sums ("sync-points", Sec. 3) one forward pass of this stack executes:
  * 2 per TP block, 1 per SPD block. */
 int spd_sync_points(const spd_ctx *ctx);

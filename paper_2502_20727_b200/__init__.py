@@ -23,7 +23,8 @@ EXPORTS = ("spd_workspace_bytes", "spd_create", "spd_prefill", "spd_decode_step"
            "spd_launches_per_decode_step", "spd_device_error", "spd_destroy", "spd_status_string",
            "spd_last_cuda_error", "spd_profile_begin", "spd_profile_end", "spd_profile_kinds",
            "spd_profile_kind_name", "spd_gemm_bf16", "spd_set_graphs", "spd_gemm_bf16_sum_static",
-           "spd_set_tuning", "spd_set_mask", "spd_sensitivity_scan", "spd_alg1_plan")
+           "spd_set_tuning", "spd_set_mask", "spd_sensitivity_scan", "spd_alg1_plan",
+           "spd_head_grouping_stats", "spd_head_scatter", "spd_mlp_match")
 
 
 class SpdError(RuntimeError):
@@ -75,6 +76,10 @@ def load_library() -> ctypes.CDLL:
     lib.spd_set_mask.argtypes = [vp, vp]
     lib.spd_sensitivity_scan.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, ctypes.POINTER(ctypes.c_double),
                                          ctypes.POINTER(ctypes.c_double), vp]
+    lib.spd_head_grouping_stats.argtypes = [vp, i32, vp, i32, i32, vp, i32, vp, vp, ctypes.POINTER(ctypes.c_float),
+                                            ctypes.POINTER(ctypes.c_double), vp]
+    lib.spd_head_scatter.argtypes = [ctypes.POINTER(ctypes.c_float), i32, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_double)]
+    lib.spd_mlp_match.argtypes = [ctypes.POINTER(ctypes.c_double), i32, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_double)]
     lib.spd_alg1_plan.argtypes = [ctypes.POINTER(ctypes.c_double), i32, i32, ctypes.c_double, ctypes.c_double, vp, vp]
     lib.spd_set_tuning.argtypes = [vp, ctypes.c_char_p, i32]
     lib.spd_gemm_bf16_sum_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, vp]
@@ -171,6 +176,68 @@ def alg1_plan(sensitivity: Sequence[float], n_spd: int, tau1: float, tau2: float
     tier = (ctypes.c_uint8 * n)()
     _check("spd_alg1_plan", lib.spd_alg1_plan(s, n, int(n_spd), float(tau1), float(tau2), mask, tier))
     return [int(v) for v in mask], [int(v) for v in tier]
+
+
+def head_scatter(dist, heads_per_unit: int, T: int):
+    """Eq. 2 on a [n_heads, n_heads] distance matrix; returns (device of every unit, objective); see spd_head_scatter."""
+    import numpy as np
+    lib = load_library()
+    d = np.ascontiguousarray(dist, dtype=np.float32)
+    n = d.shape[0]
+    out = (ctypes.c_int32 * (n // heads_per_unit))()
+    obj = ctypes.c_double(0.0)
+    _check("spd_head_scatter", lib.spd_head_scatter(d.ctypes.data_as(ctypes.POINTER(ctypes.c_float)), n, int(heads_per_unit), int(T), out,
+                                                     ctypes.byref(obj)))
+    return [int(v) for v in out], obj.value
+
+
+def mlp_match(norms):
+    """Eq. 3 on a [T, T] matrix of output norms; returns (MLP partition of every device, objective); see spd_mlp_match."""
+    import numpy as np
+    lib = load_library()
+    nm = np.ascontiguousarray(norms, dtype=np.float64)
+    T = nm.shape[0]
+    out = (ctypes.c_int32 * T)()
+    obj = ctypes.c_double(0.0)
+    _check("spd_mlp_match", lib.spd_mlp_match(nm.ctypes.data_as(ctypes.POINTER(ctypes.c_double)), T, out, ctypes.byref(obj)))
+    return [int(v) for v in out], obj.value
+
+
+def head_order_from_devices(device_of_unit: Sequence[int], heads_per_unit: int, T: int) -> List[int]:
+    """Query-head order that puts the units of device 0 first, then device 1, ... (units keep their order inside a
+    device): position p of the result names the old head that moves to p."""
+    order: List[int] = []
+    for dev in range(T):
+        for u, du in enumerate(device_of_unit):
+            if du == dev:
+                order.extend(range(u * heads_per_unit, (u + 1) * heads_per_unit))
+    return order
+
+
+def permute_layer(lw: Dict[str, torch.Tensor], *, n_q_heads: int, n_kv_heads: int, head_dim: int, T: int,
+                  head_order: Optional[Sequence[int]] = None, mlp_of_device: Optional[Sequence[int]] = None) -> Dict[str, torch.Tensor]:
+    """The weight re-ordering of Sec. 4.2.4 (index moves only): rows of wq / wk / wv and columns of wo by head so that
+    the heads of A_i sit on device i, and the MLP partitions (row blocks of w_gate / w_up, column blocks of w_down) so
+    that device i holds partition mlp_of_device[i].  The function a TP block computes does not change."""
+    out = dict(lw)
+    dev = lw["wq"].device
+    if head_order is not None:
+        group = n_q_heads // n_kv_heads
+        q_idx = torch.tensor([h * head_dim + e for h in head_order for e in range(head_dim)], device=dev)
+        kv_order = [head_order[i] // group for i in range(0, n_q_heads, group)]
+        kv_idx = torch.tensor([h * head_dim + e for h in kv_order for e in range(head_dim)], device=dev)
+        out["wq"] = lw["wq"].index_select(0, q_idx).contiguous()
+        out["wk"] = lw["wk"].index_select(0, kv_idx).contiguous()
+        out["wv"] = lw["wv"].index_select(0, kv_idx).contiguous()
+        out["wo"] = lw["wo"].index_select(1, q_idx).contiguous()
+    if mlp_of_device is not None:
+        F = lw["w_gate"].shape[0]
+        Fs = F // T
+        f_idx = torch.tensor([m * Fs + e for m in mlp_of_device for e in range(Fs)], device=dev)
+        out["w_gate"] = lw["w_gate"].index_select(0, f_idx).contiguous()
+        out["w_up"] = lw["w_up"].index_select(0, f_idx).contiguous()
+        out["w_down"] = lw["w_down"].index_select(1, f_idx).contiguous()
+    return out
 
 
 class SpdStack:
@@ -288,6 +355,25 @@ class SpdStack:
                    self.lib.spd_sensitivity_scan(self._ctx, x.data_ptr(), B, S, block_table.data_ptr(), block_table.shape[1],
                                                  ref.data_ptr(), tmp.data_ptr(), sens, met, _stream_ptr()))
         return [float(v) for v in sens], [float(v) for v in met]
+
+    def head_grouping_stats(self, layer: int, x: torch.Tensor, block_table: torch.Tensor):
+        """Head distances (Eq. 2) and MLP output norms (Eq. 3) of block `layer` on prompt batch x [B, S, hidden];
+        returns (dist [nq, nq], norms [T, T]) as numpy arrays; see spd_head_grouping_stats."""
+        import numpy as np
+        B, S, H = x.shape
+        self._check_io(x, block_table)
+        nq, T = self.dims.n_q_heads, self.dims.T
+        sigma = torch.empty(nq * B * S * S, dtype=torch.float32, device=self.device)
+        dist_dev = torch.empty(nq * nq, dtype=torch.float32, device=self.device)
+        dist = np.zeros((nq, nq), dtype=np.float32)
+        norms = np.zeros((T, T), dtype=np.float64)
+        with torch.cuda.device(self.device):
+            _check("spd_head_grouping_stats",
+                   self.lib.spd_head_grouping_stats(self._ctx, int(layer), x.data_ptr(), B, S, block_table.data_ptr(),
+                                                    block_table.shape[1], sigma.data_ptr(), dist_dev.data_ptr(),
+                                                    dist.ctypes.data_as(ctypes.POINTER(ctypes.c_float)),
+                                                    norms.ctypes.data_as(ctypes.POINTER(ctypes.c_double)), _stream_ptr()))
+        return dist, norms
 
     def set_graphs(self, enabled: bool):
         """Replay decode steps from captured CUDA graphs (default on); see spd_set_graphs."""

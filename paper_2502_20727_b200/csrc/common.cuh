@@ -176,6 +176,12 @@ inline int decode_heads_per_block_mma(int group) { return group % 8 == 0 ? 8 : 4
 template <typename T> cudaError_t launch_prefill_attention(const AttnArgs &a, cudaStream_t st);
 template <typename T> cudaError_t launch_decode_attention(const AttnArgs &a, cudaStream_t st);
 
+// head grouping measurements (head_grouping.cu)
+template <typename T>
+cudaError_t launch_head_scores(const void *q, const void *k_pages, PageTable pt, int b0, int S, int n_seq, int n_q_heads, int d,
+                               float *sigma, int *err, cudaStream_t st);
+cudaError_t launch_head_distance(const float *sigma, long len, int n_heads, float *dist, cudaStream_t st);
+
 // part[b] = sum over block b's slice of (a - r)^2, fixed order (strategy.cu)
 cudaError_t launch_sq_diff(const void *a, const void *r, long n, int dtype_bf16, float *part, int n_blocks, cudaStream_t st);
 

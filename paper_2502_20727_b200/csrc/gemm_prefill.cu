@@ -243,7 +243,7 @@ __device__ __forceinline__ void epi_qkv(const PreGemmArgs &g, const PreTile &t, 
 __device__ __forceinline__ void epi_gateup(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, int m, bool valid)
 {
     const float rs = valid ? row_rstd(g.ss_in, g.rstd_per_shard ? t.z : 0, m) : 0.f;
-    bf16 *dst = (bf16 *)g.act + (long)m * g.F + (long)t.z * g.Fs + t.row0;
+    bf16 *dst = (bf16 *)g.act + (long)m * g.F + (long)((t.z + g.w_rot) % g.batches) * g.Fs + t.row0;
 #pragma unroll 1
     for (int c = 0; c < 8; ++c) {
         const int f = t.row0 + c * 16;
@@ -332,6 +332,25 @@ __device__ __forceinline__ void spd_park_x(const PreGemmArgs &g, const PreTile &
         tmem_st16(ttot + c * 16, x);
     }
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+
+// Sum of squares of this row's 128 accumulator columns (MLP matching: norm of a partition's output).
+__device__ __forceinline__ float epi_row_sumsq(const PreGemmArgs &g, const PreTile &t, uint32_t tacc)
+{
+    float ssq = 0.f;
+#pragma unroll 1
+    for (int c = 0; c < 8; c += 2) {
+        const int n = t.row0 + c * 16;
+        if (n >= g.H) break;
+        float ya[16], yb[16];
+        tmem_ld16x2(tacc + c * 16, tacc + c * 16 + 16, ya, yb);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            ssq = fmaf(ya[i], ya[i], ssq);
+            if (n + 16 < g.H) ssq = fmaf(yb[i], yb[i], ssq);
+        }
+    }
+    return ssq;
 }
 
 // One pass (device z) of an SPD o_proj tile.  R_z * g is staged in hs (two 64-column bf16 boxes of
@@ -436,7 +455,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_prefill_kernel(const __grid_c
                 const CUtensorMap *tm_w = t.wi == 0 ? &tm_w0 : (t.wi == 1 ? &tm_w1 : &tm_w2);
                 for (int pass = 0; pass < L.passes && ok; ++pass) {
                     const int tz = EPI == PRE_OPROJ_SPD ? pass : (EPI == PRE_GATEUP && g.t_batched ? t.z : 0);
-                    const int wz = EPI == PRE_OPROJ_SPD ? pass : t.z;
+                    const int wz = EPI == PRE_OPROJ_SPD ? pass : (EPI == PRE_GATEUP ? (t.z + g.w_rot) % g.batches : t.z);
                     for (int kb = 0; kb < g.num_kb; ++kb, ++it) {
                         const int s = it % S;
                         if (!mbar_wait(empty_bar(s), ((it / S) & 1) ^ 1, g.err, abort_flag)) { ok = false; break; }
@@ -490,7 +509,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_prefill_kernel(const __grid_c
             const PreTile t = decode_tile(L, EPI, tile);
             const int m = t.m0 + warp * 32 + lane;
             const bool valid = m < g.t_rows;
-            if (EPI == PRE_OPROJ_SPD) spd_park_x(g, t, tmem_base + lane_base + X_COL, tmem_base + lane_base + TOT_COL, m, valid);
+            if (EPI == PRE_OPROJ_SPD && !g.norm_only) spd_park_x(g, t, tmem_base + lane_base + X_COL, tmem_base + lane_base + TOT_COL, m, valid);
             for (int pass = 0; pass < L.passes; ++pass, ++pc) {
                 const int buf = pc & 1;
                 if (!mbar_wait(tfull_bar(buf), (pc >> 1) & 1, g.err, abort_flag)) { ok = false; break; }
@@ -500,7 +519,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_prefill_kernel(const __grid_c
                 if (EPI == PRE_QKV) epi_qkv(g, t, tacc, m, valid);
                 else if (EPI == PRE_GATEUP) epi_gateup(g, t, tacc, m, valid);
                 else if (EPI == PRE_RESID) epi_resid(g, t, tacc, m, valid);
-                else {
+                else if (g.norm_only) {
+                    const float ssq = epi_row_sumsq(g, t, tacc);
+                    if (valid) g.ss_out[((long)t.nt * g.batches + pass) * g.Mcap + m] = ssq;
+                } else {
                     // two staging tiles in turn: the store issued two passes ago has read its source
                     uint8_t *hst = hs + (pc & 1) * 32768;
                     if (threadIdx.x == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
@@ -538,7 +560,7 @@ cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
 {
     const bool spd = EPI == PRE_OPROJ_SPD;
     const CUtensorMap &tx = tt, &tr = tt; // spare tensor-map slots
-    const CUtensorMap &th = *(const CUtensorMap *)(spd ? L.g.h_map : (const void *)&tt);
+    const CUtensorMap &th = *(const CUtensorMap *)((spd && !L.g.norm_only) ? L.g.h_map : (const void *)&tt);
     using C = PCfg<EPI>;
     static int n_sm = 0;
     if (!n_sm) {
@@ -596,7 +618,9 @@ cudaError_t launch_gemm_prefill(PreEpilogue epi, const TcMap *const *weights, co
     if (g.num_kb < 1 || g.batches < 1 || g.batches > 8) return cudaErrorInvalidValue;
     if (epi == PRE_QKV && (256 % g.head_dim || g.head_dim < 32)) return cudaErrorInvalidValue;
     if ((epi == PRE_RESID || epi == PRE_OPROJ_SPD) && g.H % 16) return cudaErrorInvalidValue;
-    if (epi == PRE_OPROJ_SPD && (!g.h_map || !g.gain || !g.hg || !g.res_out)) return cudaErrorInvalidValue;
+    if (epi == PRE_OPROJ_SPD && !g.norm_only && (!g.h_map || !g.gain || !g.hg || !g.res_out)) return cudaErrorInvalidValue;
+    if (epi == PRE_OPROJ_SPD && g.norm_only && !g.ss_out) return cudaErrorInvalidValue;
+    if (g.w_rot < 0 || g.w_rot >= g.batches) return cudaErrorInvalidValue;
     if (epi == PRE_GATEUP && g.Fs % 8) return cudaErrorInvalidValue;
     const CUtensorMap *tw[3];
     for (int i = 0; i < 3; ++i) tw[i] = (const CUtensorMap *)weights[i < nw ? i : 0];

@@ -50,13 +50,13 @@ int want_splits(long tiles, int cap)
     return (int)(s < 1 ? 1 : s);
 }
 
-enum ActBuf { AB_H = 0, AB_ATTN, AB_ATTN_SHARD, AB_ACT, AB_COUNT };
+enum ActBuf { AB_H = 0, AB_ATTN, AB_ATTN_SHARD, AB_ACT, AB_ACT_SHARD, AB_COUNT };
 enum Kind { K_NORM = 0, K_QKV, K_ROPE_KV, K_ATTN, K_OPROJ, K_GATE_UP, K_SILU_MUL, K_DOWN, K_ROPE_TABLE, K_COUNT };
 enum Site { SITE_QKV = 0, SITE_O, SITE_GU, SITE_DOWN, SITE_ATTN, SITE_COUNT };
 const char *const kind_names[K_COUNT] = {"residual_rmsnorm", "gemm_qkv", "rope_kv_append", "attention", "gemm_o_proj",
                                          "gemm_gate_up", "silu_mul", "gemm_down", "rope_table"};
 
-struct LayerMaps { TcMap wq, wk, wv, wo_full, wo_shard, w_gate, w_up, w_down, w_gate64, w_up64, wq256, wk256, wv256, wo256, wd256, kpages, vpages; };
+struct LayerMaps { TcMap wq, wk, wv, wo_full, wo_shard, w_gate, w_up, w_down, w_gate64, w_up64, wq256, wk256, wv256, wo256, wd256, wd_shard, kpages, vpages; };
 
 // A captured decode step is valid for exactly these arguments.
 struct GraphKey {
@@ -271,6 +271,7 @@ const TcMap *act_map(Ctx *c, ActBuf buf, int box)
     case AB_ATTN: rc = make_operand_map(&c->act_maps[buf][bi], c->attn, qd, Mc, 1, qd, 0, box); break;
     case AB_ATTN_SHARD: rc = make_operand_map(&c->act_maps[buf][bi], c->attn, qd / T, Mc, T, qd, qd / T, box); break;
     case AB_ACT: rc = make_operand_map(&c->act_maps[buf][bi], c->act, F, Mc, 1, F, 0, box); break;
+    case AB_ACT_SHARD: rc = make_operand_map(&c->act_maps[buf][bi], c->act, F / T, Mc, T, F, F / T, box); break;
     default: break;
     }
     if (rc) return nullptr;
@@ -537,10 +538,20 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
     return SPD_OK;
 }
 
+// Head-grouping measurements (Sec. 4.2.4) taken at one block while a prompt batch runs through the
+// TP blocks before it: attention scores of every head and their pairwise distances (Eq. 2), and the
+// sums of squares of MLP_m(norm(X + Y_i)) for every (device i, MLP partition m) (Eq. 3).
+struct HeadProbe {
+    int layer, n_seq, S;
+    float *sigma;  // device [nq][n_seq][S][S]
+    float *dist;   // device [nq][nq]
+    double *norms; // host [T][T], sums of squares (the caller takes the root)
+};
+
 // One prefill chunk of the bf16 stack with the fused projections (same five kernels per block as
 // a decode step, in their many-token form).
 int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t *bt, int max_pages,
-                      int max_context, cudaStream_t st)
+                      int max_context, cudaStream_t st, const HeadProbe *probe = nullptr)
 {
     const spd_dims &d = c->d;
     const int H = d.hidden, qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, F = d.ffn, Tn = d.T;
@@ -564,7 +575,9 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
     };
     for (int l = 0; l < d.n_layers; ++l) {
         const spd_layer &w = c->layers[l];
-        const bool sync = c->mask[l] != 0;
+        const bool probing = probe && l == probe->layer;
+        // while probing, the blocks before the probed one are TP blocks and the probed one is an SPD block
+        const bool sync = probe ? !probing : c->mask[l] != 0;
         {   // a2 + a3
             PreGemmArgs g = base_args();
             const TcMap *wmaps[3] = {&c->maps[l].wq256, &c->maps[l].wk256, &c->maps[l].wv256};
@@ -575,6 +588,11 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
             g.rope = rope ? c->rope : nullptr; g.q_out = c->q; g.k_pages = w.k_pages; g.v_pages = w.v_pages; g.pt = pt; g.tm = tm;
             g.n_q_heads = d.n_q_heads; g.head_dim = d.head_dim;
             LAUNCH(K_QKV, launch_gemm_prefill(PRE_QKV, wmaps, *am, g, st));
+        }
+        if (probing) {   // Eq. 2: attention score of every head as one long vector, pairwise Euclidean distances
+            CU_TRY(launch_head_scores<bf16>(c->q, w.k_pages, pt, tm.b0, probe->S, probe->n_seq, d.n_q_heads, d.head_dim, probe->sigma,
+                                            c->err, st));
+            CU_TRY(launch_head_distance(probe->sigma, (long)probe->n_seq * probe->S * probe->S, d.n_q_heads, probe->dist, st));
         }
         {   // a4
             AttnArgs a{};
@@ -602,6 +620,46 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
             g.h_map = hm;
             LAUNCH(K_OPROJ, launch_gemm_prefill(PRE_OPROJ_SPD, wmaps, *am, g, st));
             mlp_tiles = pre_ss_tiles(PRE_OPROJ_SPD, H); mlp_groups = Tn;
+        }
+        if (probing) {
+            // Eq. 3: for every rotation r, MLP partition (i + r) % T runs on device i's input X + Y_i; the
+            // per-partition down projections only report the sums of squares of their outputs
+            float *ssq = c->gu32; // [H tiles of 128][T][Mcap], idle in this path
+            const int nt = pre_ss_tiles(PRE_OPROJ_SPD, H);
+            std::vector<float> host((size_t)nt * Tn * M);
+            for (int i = 0; i < Tn * Tn; ++i) probe->norms[i] = 0.0;
+            for (int r = 0; r < Tn; ++r) {
+                {
+                    PreGemmArgs g = base_args();
+                    const TcMap *wmaps[2] = {&c->maps[l].w_gate, &c->maps[l].w_up};
+                    MAP_OR_FAIL(am, act_map(c, AB_H, 128));
+                    g.n_weights = 2; g.w_rows[0] = g.w_rows[1] = Fs; g.batches = Tn; g.t_batched = 1; g.w_rot = r;
+                    g.num_kb = cdiv(H, 64);
+                    g.ss_in = SumSq{c->ss_mlp, mlp_tiles, mlp_groups, Mc, H, d.rms_eps};
+                    g.rstd_per_shard = 1;
+                    g.act = c->act; g.F = F; g.Fs = Fs;
+                    LAUNCH(K_GATE_UP, launch_gemm_prefill(PRE_GATEUP, wmaps, *am, g, st));
+                }
+                {
+                    PreGemmArgs g = base_args();
+                    const TcMap *wmaps[1] = {&c->maps[l].wd_shard};
+                    MAP_OR_FAIL(am, act_map(c, AB_ACT_SHARD, 128));
+                    g.w_rows[0] = H; g.num_kb = cdiv(Fs, 64); g.batches = Tn; g.norm_only = 1; g.ss_out = ssq;
+                    LAUNCH(K_DOWN, launch_gemm_prefill(PRE_OPROJ_SPD, wmaps, *am, g, st));
+                }
+                CU_TRY(cudaMemcpy2DAsync(host.data(), (size_t)M * 4, ssq, (size_t)Mc * 4, (size_t)M * 4, (size_t)nt * Tn,
+                                         cudaMemcpyDeviceToHost, st));
+                CU_TRY(cudaStreamSynchronize(st));
+                for (int t = 0; t < nt; ++t)
+                    for (int wz = 0; wz < Tn; ++wz) {
+                        double acc = 0.0;
+                        const float *row = host.data() + ((size_t)t * Tn + wz) * M;
+                        for (int m = 0; m < M; ++m) acc += (double)row[m];
+                        probe->norms[(size_t)((wz - r + Tn) % Tn) * Tn + wz] += acc; // device (wz - r), partition wz
+                    }
+            }
+            c->launches_last = launches;
+            return SPD_OK;
         }
         {   // a8
             PreGemmArgs g = base_args();
@@ -664,6 +722,7 @@ int build_weight_maps(Ctx &c)
         rc |= make_operand_map(&m.wv256, w.wv, H, kd, 1, H, 0, 256);
         rc |= make_operand_map(&m.wo256, w.wo, qd, H, 1, qd, 0, 256);
         rc |= make_operand_map(&m.wd256, w.w_down, F, H, 1, F, 0, 256);
+        rc |= make_operand_map(&m.wd_shard, w.w_down, F / T, H, T, F, F / T, 128);
         if (d.head_dim == 128 && d.kv_block_size == 16) {
             // K / V pages as [n_pages * n_kv_heads * 16 token rows][head_dim]; one box = 64 dims of a page's 16 tokens
             const long rows = (long)c.n_pages * d.n_kv_heads * 16;
@@ -907,6 +966,27 @@ int spd_sensitivity_scan(spd_ctx *ctx, const void *x, int32_t B, int32_t S, cons
     for (int i = 0; i < L; ++i) sensitivity[i] = met[i] - met[i + 1];
     if (metric) for (int i = 0; i <= L; ++i) metric[i] = met[i];
     return restore(SPD_OK);
+}
+
+int spd_head_grouping_stats(spd_ctx *ctx, int32_t layer, const void *x, int32_t B, int32_t S, const int32_t *block_table,
+                            int32_t max_pages, float *sigma_scratch, float *dist_dev, float *dist, double *norms, void *stream)
+{
+    if (!ctx || !x || !block_table || !sigma_scratch || !dist_dev || !dist || !norms) return SPD_ENULL;
+    Ctx &c = ctx->c;
+    const spd_dims &d = c.d;
+    if (d.dtype != 1 || d.hidden % 16 || layer < 0 || layer >= d.n_layers || B < 1 || S < 1 || B > d.max_batch) return SPD_EINVAL;
+    if ((long)B * S > d.max_prefill_tokens) return SPD_EINVAL; // one chunk
+    if (S > d.max_seq_len || (long)max_pages * d.kv_block_size < S) return SPD_ECAPACITY;
+    if (!c.any_spd) return SPD_EWORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    HeadProbe probe{layer, B, S, sigma_scratch, dist_dev, norms};
+    TokMap tm{0, 0, S, 0, nullptr};
+    int rc = run_prefill_fused(&c, x, nullptr, B * S, tm, block_table, max_pages, S, st, &probe);
+    if (rc) return rc;
+    CU_TRY(cudaMemcpyAsync(dist, dist_dev, (size_t)d.n_q_heads * d.n_q_heads * sizeof(float), cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaStreamSynchronize(st));
+    for (int i = 0; i < d.T * d.T; ++i) norms[i] = sqrt(norms[i]);
+    return SPD_OK;
 }
 
 int spd_set_graphs(spd_ctx *ctx, int32_t enabled)
