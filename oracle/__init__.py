@@ -179,3 +179,85 @@ def linear(x, w):
     out = np.empty((x.shape[0], w.shape[0]), dtype=np.float64)
     lib().oracle_linear(_p(x), _p(w), x.shape[0], w.shape[0], x.shape[1], _p(out))
     return out
+
+
+# ---- the decoder block with bias (OPT-style), Sec. 4.1.2 ------------------------------------------
+BIAS_WEIGHT_NAMES = ("attn_norm", "attn_norm_b", "wq", "bq", "wk", "bk", "wv", "bv", "wo", "bo", "mlp_norm", "mlp_norm_b",
+                     "w_fc1", "b_fc1", "w_fc2", "b_fc2")
+
+
+class _BiasLayer(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in BIAS_WEIGHT_NAMES]
+
+
+def _pack_bias_layers(layers):
+    keep = []
+    arr = (_BiasLayer * len(layers))()
+    for i, lw in enumerate(layers):
+        for n in BIAS_WEIGHT_NAMES:
+            a = _f32(lw[n])
+            keep.append(a)
+            setattr(arr[i], n, a.ctypes.data)
+    return arr, keep
+
+
+def bias_stack_forward(dims: Dims, mask, layers, x, pos0, cache: Cache):
+    """Masked stack of OPT-style blocks (mask[l] = 1 TP, 0 SPD with bias).  dims.rms_eps is the LayerNorm eps;
+    dims.rope_base is ignored.  Returns (out [B,S,H], sync_points)."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    B, S, H = x.shape
+    mask = np.ascontiguousarray(mask, dtype=np.uint8)
+    pos0 = np.ascontiguousarray(pos0, dtype=np.int32)
+    arr, keep = _pack_bias_layers(layers)
+    out = np.empty_like(x)
+    d = dims.c()
+    L = lib()
+    L.oracle_bias_stack_forward.restype = ctypes.c_int
+    rc = L.oracle_bias_stack_forward(ctypes.byref(d), _p(mask), arr, _p(x), B, S, _p(pos0), _p(cache.k), _p(cache.v), cache.max_len, _p(out))
+    if rc < 0:
+        raise ValueError("oracle: bad dims or positions")
+    del keep
+    return out, rc
+
+
+def bias_unsharded_stack_forward(dims: Dims, layers, x, pos0, cache: Cache):
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    B, S, H = x.shape
+    pos0 = np.ascontiguousarray(pos0, dtype=np.int32)
+    arr, keep = _pack_bias_layers(layers)
+    out = np.empty_like(x)
+    d = dims.c()
+    L = lib()
+    L.oracle_bias_unsharded_stack_forward.restype = ctypes.c_int
+    rc = L.oracle_bias_unsharded_stack_forward(ctypes.byref(d), arr, _p(x), B, S, _p(pos0), _p(cache.k), _p(cache.v), cache.max_len, _p(out))
+    if rc < 0:
+        raise ValueError("oracle: bad dims or positions")
+    del keep
+    return out
+
+
+def bias_block_forward(dims: Dims, layer, mode: int, x, pos0, cache: Cache):
+    """One OPT-style block.  mode 1 sync, 0 SPD (Sec. 4.1.2), 2 the rejected design of Table 1(b).
+    Returns (out [B,S,H], p [T, B*S, H], sync_points)."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    B, S, H = x.shape
+    pos0 = np.ascontiguousarray(pos0, dtype=np.int32)
+    arr, keep = _pack_bias_layers([layer])
+    out = np.empty((B, S, H), dtype=np.float64)
+    p = np.empty((dims.T, B * S, H), dtype=np.float64)
+    d = dims.c()
+    L = lib()
+    L.oracle_bias_block_forward.restype = ctypes.c_int
+    rc = L.oracle_bias_block_forward(ctypes.byref(d), arr, mode, _p(x), B, S, _p(pos0), _p(cache.k[0]), _p(cache.v[0]), cache.max_len,
+                                     _p(out), _p(p))
+    if rc < 0:
+        raise ValueError("oracle: bad dims or positions")
+    del keep
+    return out, p, rc
+
+
+def layernorm(x, g, b, eps):
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    out = np.empty_like(x)
+    lib().oracle_layernorm(_p(x), _p(_f32(g)), _p(_f32(b)), x.shape[0], x.shape[1], ctypes.c_double(eps), _p(out))
+    return out

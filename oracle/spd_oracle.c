@@ -26,6 +26,13 @@
  *     of the LLaMA-2 models it evaluates (Sec. 5.1).  In an SPD block the MLP
  *     RMSNorm is applied per device to X + Y_i.
  *
+ *   - decoder block with bias (OPT-style): Y_i = P_i + b; MLP input of device i is
+ *     X + P_i + b; P_i joins before the kept all-reduce, b and X after it, giving
+ *     X + sum_i P_i + b + sum_i Z_i             : Sec. 4.1.2, Fig. 3(b); rejected design
+ *     "b before the all-reduce"                 : Table 1(b).  Pre-LayerNorm OPT block
+ *     (LayerNorm, biased projections, ReLU, no rotary embedding): the OPT models of Sec. 5.1.
+ *     Pins: tests/test_oracle_bias_pins.py (transformers OPT decoder layer, invariants).
+ *
  * Parity pins (tests/test_oracle_pins.py): the unsharded block against the
  * `transformers` LLaMA decoder layer and torch library attention; all-sync
  * stacks of any T against the unsharded block; T = 1 SPD against sync;
@@ -325,6 +332,187 @@ static void block_unsharded(const oracle_dims *D, const oracle_layer *W, const d
 }
 
 /* ------------------------------------------------------------------ */
+/* the decoder block with bias (OPT-style), Sec. 4.1.2, Fig. 3(b)      */
+/* ------------------------------------------------------------------ */
+
+/* Pre-LayerNorm OPT decoder block (the OPT models of Sec. 5.1): LayerNorm with gain and shift,
+ * biased q/k/v/out projections, no rotary embedding (OPT adds learned position embeddings
+ * before the first block, i.e. outside it), fc1 + ReLU + fc2 with biases.
+ * Tensor parallelism as in Sec. 3: q/k/v and fc1 column-split (their biases split with them),
+ * out_proj and fc2 row-split; the bias of a row-split layer cannot be split and is added once,
+ * after the all-reduce (Sec. 4.1.2: "the bias residual ... after the sync operation"). */
+typedef struct {
+    const float *attn_norm, *attn_norm_b; /* [H] gain, shift of the LayerNorm before attention */
+    const float *wq, *bq;                 /* [nq*d, H], [nq*d]   */
+    const float *wk, *bk, *wv, *bv;       /* [nkv*d, H], [nkv*d] */
+    const float *wo, *bo;                 /* [H, nq*d], [H]: Y_i = P_i + b with b = bo */
+    const float *mlp_norm, *mlp_norm_b;   /* [H] */
+    const float *w_fc1, *b_fc1;           /* [F, H], [F] */
+    const float *w_fc2, *b_fc2;           /* [H, F], [H] */
+} oracle_bias_layer;
+
+/* LayerNorm: out = (x - mean) / sqrt(var + eps) * g + b, biased variance, row by row. */
+void oracle_layernorm(const double *x, const float *g, const float *b, int M, int H, double eps, double *out)
+{
+    for (int m = 0; m < M; ++m) {
+        double mean = 0.0, var = 0.0;
+        for (int j = 0; j < H; ++j) mean += x[(size_t)m * H + j];
+        mean /= (double)H;
+        for (int j = 0; j < H; ++j) { double c = x[(size_t)m * H + j] - mean; var += c * c; }
+        var /= (double)H;
+        double r = 1.0 / sqrt(var + eps);
+        for (int j = 0; j < H; ++j) out[(size_t)m * H + j] = (x[(size_t)m * H + j] - mean) * r * (double)g[j] + (double)b[j];
+    }
+}
+
+static void add_bias_cols(double *y, int M, int n_len, int ldy, const float *bias, int n0)
+{
+    for (int m = 0; m < M; ++m)
+        for (int n = 0; n < n_len; ++n) y[(size_t)m * ldy + n] += (double)bias[n0 + n];
+}
+
+/* mode 1: synchronous TP block.  mode 0: SPD block with bias (Sec. 4.1.2): the MLP input of device i
+ * is X + P_i + b; P_i is added before the kept all-reduce, b and X after it:
+ * X + sum_i P_i + b + sum_i Z_i.  mode 2: the rejected design of Table 1(b), b added before the
+ * all-reduce (and so T times).  p_out: optional [T, B*S, H] partial products P_i (without b). */
+static int block_sharded_bias(const oracle_dims *D, const oracle_bias_layer *W, int mode, const double *x, int B, int S,
+                              const int32_t *pos0, double *kcache, double *vcache, int max_len, double *out, double *p_out)
+{
+    const int H = D->hidden, nq = D->n_q_heads, nkv = D->n_kv_heads, d = D->head_dim;
+    const int F = D->ffn, T = D->T, M = B * S;
+    const int qh = nq / T, kvh = nkv / T, Fs = F / T, group = nq / nkv;
+    const size_t kvw = (size_t)nkv * d;
+    int sync_points = 0;
+
+    double *h = malloc(sizeof(double) * (size_t)M * H);
+    double *P = malloc(sizeof(double) * (size_t)T * M * H);
+    double *Z = malloc(sizeof(double) * (size_t)T * M * H);
+    oracle_layernorm(x, W->attn_norm, W->attn_norm_b, M, H, D->rms_eps, h);
+
+    double **Qs = malloc(sizeof(double *) * (size_t)T);
+    for (int i = 0; i < T; ++i) {
+        double *Q = malloc(sizeof(double) * (size_t)M * qh * d);
+        double *K = malloc(sizeof(double) * (size_t)M * kvh * d);
+        double *V = malloc(sizeof(double) * (size_t)M * kvh * d);
+        linear_slice(h, M, H, H, W->wq, H, i * qh * d, qh * d, 0, Q, qh * d);
+        linear_slice(h, M, H, H, W->wk, H, i * kvh * d, kvh * d, 0, K, kvh * d);
+        linear_slice(h, M, H, H, W->wv, H, i * kvh * d, kvh * d, 0, V, kvh * d);
+        add_bias_cols(Q, M, qh * d, qh * d, W->bq, i * qh * d);
+        add_bias_cols(K, M, kvh * d, kvh * d, W->bk, i * kvh * d);
+        add_bias_cols(V, M, kvh * d, kvh * d, W->bv, i * kvh * d);
+        for (int b = 0; b < B; ++b)
+            for (int s = 0; s < S; ++s) {
+                int m = b * S + s, pos = pos0[b] + s;
+                memcpy(kcache + ((size_t)b * max_len + pos) * kvw + (size_t)i * kvh * d, K + (size_t)m * kvh * d, sizeof(double) * (size_t)kvh * d);
+                memcpy(vcache + ((size_t)b * max_len + pos) * kvw + (size_t)i * kvh * d, V + (size_t)m * kvh * d, sizeof(double) * (size_t)kvh * d);
+            }
+        Qs[i] = Q;
+        free(K);
+        free(V);
+    }
+    for (int i = 0; i < T; ++i) {
+        double *A = malloc(sizeof(double) * (size_t)M * qh * d);
+#pragma omp parallel for collapse(2) schedule(dynamic)
+        for (int m = 0; m < M; ++m)
+            for (int j = 0; j < qh; ++j) {
+                int b = m / S, s = m % S, pos = pos0[b] + s;
+                int gkv = (i * qh + j) / group;
+                attend_one(Qs[i] + ((size_t)m * qh + j) * d, d, pos, kcache + (size_t)b * max_len * kvw + (size_t)gkv * d,
+                           vcache + (size_t)b * max_len * kvw + (size_t)gkv * d, kvw, A + ((size_t)m * qh + j) * d);
+            }
+        /* P_i: the partial product of device i's slice of the row-split out_proj, without its bias */
+        linear_slice(A, M, qh * d, qh * d, W->wo, nq * d, 0, H, i * qh * d, P + (size_t)i * M * H, H);
+        free(A);
+        free(Qs[i]);
+    }
+    free(Qs);
+    if (p_out) memcpy(p_out, P, sizeof(double) * (size_t)T * M * H);
+
+    double *R = malloc(sizeof(double) * (size_t)M * H);
+    double *u = malloc(sizeof(double) * (size_t)M * H);
+    double *a = malloc(sizeof(double) * (size_t)M * Fs);
+    if (mode == 1) {
+        /* sync-point #1: all-reduce of P_i, then the bias once, then the residual */
+        for (size_t e = 0; e < (size_t)M * H; ++e) {
+            double acc = 0.0;
+            for (int i = 0; i < T; ++i) acc += P[(size_t)i * M * H + e];
+            R[e] = x[e] + acc + (double)W->bo[e % H];
+        }
+        sync_points++;
+        oracle_layernorm(R, W->mlp_norm, W->mlp_norm_b, M, H, D->rms_eps, u);
+    }
+    for (int i = 0; i < T; ++i) {
+        if (mode != 1) {
+            /* SPD: the MLP input of device i is X + P_i + b */
+            for (size_t e = 0; e < (size_t)M * H; ++e) R[e] = x[e] + P[(size_t)i * M * H + e] + (double)W->bo[e % H];
+            oracle_layernorm(R, W->mlp_norm, W->mlp_norm_b, M, H, D->rms_eps, u);
+        }
+        linear_slice(u, M, H, H, W->w_fc1, H, i * Fs, Fs, 0, a, Fs);
+        add_bias_cols(a, M, Fs, Fs, W->b_fc1, i * Fs);
+        for (size_t e = 0; e < (size_t)M * Fs; ++e) a[e] = a[e] > 0.0 ? a[e] : 0.0;
+        linear_slice(a, M, Fs, Fs, W->w_fc2, F, 0, H, i * Fs, Z + (size_t)i * M * H, H);
+    }
+    for (size_t e = 0; e < (size_t)M * H; ++e) {
+        double accz = 0.0, accp = 0.0;
+        for (int i = 0; i < T; ++i) { accz += Z[(size_t)i * M * H + e]; accp += P[(size_t)i * M * H + e]; }
+        const double bo = (double)W->bo[e % H], b2 = (double)W->b_fc2[e % H];
+        if (mode == 1) out[e] = R[e] + accz + b2;                       /* sync-point #2 */
+        else if (mode == 0) out[e] = x[e] + (accp + accz) + bo + b2;    /* P_i before the all-reduce, b and X after */
+        else out[e] = x[e] + (accp + (double)T * bo + accz) + b2;       /* Table 1(b), rejected: b before the all-reduce */
+    }
+    sync_points++;
+    free(h); free(P); free(Z); free(R); free(u); free(a);
+    return sync_points;
+}
+
+/* the same block on one device, no device loop */
+static void block_unsharded_bias(const oracle_dims *D, const oracle_bias_layer *W, const double *x, int B, int S,
+                                 const int32_t *pos0, double *kcache, double *vcache, int max_len, double *out)
+{
+    const int H = D->hidden, nq = D->n_q_heads, nkv = D->n_kv_heads, d = D->head_dim;
+    const int F = D->ffn, M = B * S, group = nq / nkv;
+    const size_t kvw = (size_t)nkv * d;
+    double *h = malloc(sizeof(double) * (size_t)M * H);
+    double *Q = malloc(sizeof(double) * (size_t)M * nq * d);
+    double *K = malloc(sizeof(double) * (size_t)M * nkv * d);
+    double *V = malloc(sizeof(double) * (size_t)M * nkv * d);
+    double *A = malloc(sizeof(double) * (size_t)M * nq * d);
+    double *R = malloc(sizeof(double) * (size_t)M * H);
+    double *u = malloc(sizeof(double) * (size_t)M * H);
+    double *a = malloc(sizeof(double) * (size_t)M * F);
+    oracle_layernorm(x, W->attn_norm, W->attn_norm_b, M, H, D->rms_eps, h);
+    linear_slice(h, M, H, H, W->wq, H, 0, nq * d, 0, Q, nq * d);
+    linear_slice(h, M, H, H, W->wk, H, 0, nkv * d, 0, K, nkv * d);
+    linear_slice(h, M, H, H, W->wv, H, 0, nkv * d, 0, V, nkv * d);
+    add_bias_cols(Q, M, nq * d, nq * d, W->bq, 0);
+    add_bias_cols(K, M, nkv * d, nkv * d, W->bk, 0);
+    add_bias_cols(V, M, nkv * d, nkv * d, W->bv, 0);
+    for (int m = 0; m < M; ++m) {
+        int b = m / S, pos = pos0[b] + m % S;
+        memcpy(kcache + ((size_t)b * max_len + pos) * kvw, K + (size_t)m * kvw, sizeof(double) * kvw);
+        memcpy(vcache + ((size_t)b * max_len + pos) * kvw, V + (size_t)m * kvw, sizeof(double) * kvw);
+    }
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int m = 0; m < M; ++m)
+        for (int j = 0; j < nq; ++j) {
+            int b = m / S, pos = pos0[b] + m % S, gkv = j / group;
+            attend_one(Q + ((size_t)m * nq + j) * d, d, pos, kcache + (size_t)b * max_len * kvw + (size_t)gkv * d,
+                       vcache + (size_t)b * max_len * kvw + (size_t)gkv * d, kvw, A + ((size_t)m * nq + j) * d);
+        }
+    linear_slice(A, M, nq * d, nq * d, W->wo, nq * d, 0, H, 0, R, H);
+    add_bias_cols(R, M, H, H, W->bo, 0);
+    for (size_t e = 0; e < (size_t)M * H; ++e) R[e] += x[e];
+    oracle_layernorm(R, W->mlp_norm, W->mlp_norm_b, M, H, D->rms_eps, u);
+    linear_slice(u, M, H, H, W->w_fc1, H, 0, F, 0, a, F);
+    add_bias_cols(a, M, F, F, W->b_fc1, 0);
+    for (size_t e = 0; e < (size_t)M * F; ++e) a[e] = a[e] > 0.0 ? a[e] : 0.0;
+    linear_slice(a, M, F, F, W->w_fc2, F, 0, H, 0, out, H);
+    add_bias_cols(out, M, H, H, W->b_fc2, 0);
+    for (size_t e = 0; e < (size_t)M * H; ++e) out[e] += R[e];
+    free(h); free(Q); free(K); free(V); free(A); free(R); free(u); free(a);
+}
+
+/* ------------------------------------------------------------------ */
 /* exported entry points                                               */
 /* ------------------------------------------------------------------ */
 
@@ -406,4 +594,56 @@ int oracle_block_forward(const oracle_dims *D, const oracle_layer *layer, int mo
 void oracle_linear(const double *x, const float *w, int M, int N, int K, double *y)
 {
     linear_slice(x, M, K, K, w, K, 0, N, 0, y, N);
+}
+
+/* ---- the block with bias: stack, single-device stack, one block ------------------------------- */
+
+int oracle_bias_stack_forward(const oracle_dims *D, const uint8_t *mask, const oracle_bias_layer *layers, const double *x, int B,
+                              int S, const int32_t *pos0, double *kcache, double *vcache, int max_len, double *out)
+{
+    if (!dims_ok(D)) return -1;
+    for (int b = 0; b < B; ++b)
+        if (pos0[b] < 0 || pos0[b] + S > max_len) return -1;
+    const size_t MH = (size_t)B * S * D->hidden;
+    const size_t cache_l = (size_t)B * max_len * D->n_kv_heads * D->head_dim;
+    double *cur = malloc(sizeof(double) * MH), *nxt = malloc(sizeof(double) * MH);
+    memcpy(cur, x, sizeof(double) * MH);
+    int sync_points = 0;
+    for (int l = 0; l < D->n_layers; ++l) {
+        sync_points += block_sharded_bias(D, &layers[l], mask[l] ? 1 : 0, cur, B, S, pos0, kcache + (size_t)l * cache_l,
+                                          vcache + (size_t)l * cache_l, max_len, nxt, NULL);
+        double *t = cur; cur = nxt; nxt = t;
+    }
+    memcpy(out, cur, sizeof(double) * MH);
+    free(cur); free(nxt);
+    return sync_points;
+}
+
+int oracle_bias_unsharded_stack_forward(const oracle_dims *D, const oracle_bias_layer *layers, const double *x, int B, int S,
+                                        const int32_t *pos0, double *kcache, double *vcache, int max_len, double *out)
+{
+    if (!dims_ok(D)) return -1;
+    for (int b = 0; b < B; ++b)
+        if (pos0[b] < 0 || pos0[b] + S > max_len) return -1;
+    const size_t MH = (size_t)B * S * D->hidden;
+    const size_t cache_l = (size_t)B * max_len * D->n_kv_heads * D->head_dim;
+    double *cur = malloc(sizeof(double) * MH), *nxt = malloc(sizeof(double) * MH);
+    memcpy(cur, x, sizeof(double) * MH);
+    for (int l = 0; l < D->n_layers; ++l) {
+        block_unsharded_bias(D, &layers[l], cur, B, S, pos0, kcache + (size_t)l * cache_l, vcache + (size_t)l * cache_l, max_len, nxt);
+        double *t = cur; cur = nxt; nxt = t;
+    }
+    memcpy(out, cur, sizeof(double) * MH);
+    free(cur); free(nxt);
+    return 0;
+}
+
+/* mode 0 SPD (Sec. 4.1.2), 1 sync, 2 the rejected design of Table 1(b); p_out optional [T, B*S, H]. */
+int oracle_bias_block_forward(const oracle_dims *D, const oracle_bias_layer *layer, int mode, const double *x, int B, int S,
+                              const int32_t *pos0, double *kcache, double *vcache, int max_len, double *out, double *p_out)
+{
+    if (!dims_ok(D) || mode < 0 || mode > 2) return -1;
+    for (int b = 0; b < B; ++b)
+        if (pos0[b] < 0 || pos0[b] + S > max_len) return -1;
+    return block_sharded_bias(D, layer, mode, x, B, S, pos0, kcache, vcache, max_len, out, p_out);
 }

@@ -42,6 +42,7 @@ class Workload:
     rms_eps: float = 1e-5
     rope_base: float = 10000.0
     kv_block: int = 16
+    block: str = "llama"    # "llama": RMSNorm / rotary / SwiGLU, no bias; "opt": LayerNorm / biases / ReLU (Sec. 4.1.2)
 
     @property
     def torch_dtype(self):
@@ -100,7 +101,31 @@ def make_layer(w: Workload, layer: int, device="cpu", seed: int = 0) -> Dict[str
     return out
 
 
+BIAS_WEIGHT_NAMES = ("attn_norm", "attn_norm_b", "wq", "bq", "wk", "bk", "wv", "bv", "wo", "bo", "mlp_norm", "mlp_norm_b",
+                     "w_fc1", "b_fc1", "w_fc2", "b_fc2")
+
+
+def make_bias_layer(w: Workload, layer: int, device="cpu", seed: int = 0) -> Dict[str, torch.Tensor]:
+    """One OPT-style layer (shapes of the OPT models of Sec. 5.1): matrices ~ N(0, 0.02^2), biases and
+    LayerNorm shifts ~ N(0, 0.1^2) (large enough that a misplaced bias shows), LayerNorm gains ~ U(0.5, 1.5).
+    Draw order: wq, wk, wv, wo, w_fc1, w_fc2, then bq, bk, bv, bo, b_fc1, b_fc2, attn_norm_b, mlp_norm_b, then the gains."""
+    g = _gen(device, seed * 1000003 + layer + 500009)
+    H, qd, kd, F = w.hidden, w.n_q_heads * w.head_dim, w.n_kv_heads * w.head_dim, w.ffn
+    shapes = {"wq": (qd, H), "wk": (kd, H), "wv": (kd, H), "wo": (H, qd), "w_fc1": (F, H), "w_fc2": (H, F),
+              "bq": (qd,), "bk": (kd,), "bv": (kd,), "bo": (H,), "b_fc1": (F,), "b_fc2": (H,), "attn_norm_b": (H,), "mlp_norm_b": (H,)}
+    out: Dict[str, torch.Tensor] = {}
+    for n in ("wq", "wk", "wv", "wo", "w_fc1", "w_fc2"):
+        out[n] = (torch.randn(shapes[n], generator=g, device=device, dtype=torch.float32) * 0.02).to(w.torch_dtype).contiguous()
+    for n in ("bq", "bk", "bv", "bo", "b_fc1", "b_fc2", "attn_norm_b", "mlp_norm_b"):
+        out[n] = (torch.randn(shapes[n], generator=g, device=device, dtype=torch.float32) * 0.1).to(w.torch_dtype).contiguous()
+    for n in ("attn_norm", "mlp_norm"):
+        out[n] = (torch.rand((H,), generator=g, device=device, dtype=torch.float32) + 0.5).to(w.torch_dtype).contiguous()
+    return out
+
+
 def make_stack(w: Workload, device="cpu", seed: int = 0) -> List[Dict[str, torch.Tensor]]:
+    if w.block == "opt":
+        return [make_bias_layer(w, l, device, seed) for l in range(w.n_layers)]
     return [make_layer(w, l, device, seed) for l in range(w.n_layers)]
 
 
