@@ -54,6 +54,9 @@ typedef struct {
     int32_t max_batch;          /* largest B of spd_decode_step / spd_prefill                   */
     int32_t max_seq_len;        /* largest context (cached + new tokens) of one sequence        */
     int32_t max_prefill_tokens; /* tokens processed per internal prefill chunk (bounds workspace)*/
+    int32_t block_kind;         /* 0: block without bias (Sec. 4.1.1; RMSNorm, rotary, SwiGLU);
+                                   1: block with bias (Sec. 4.1.2; LayerNorm, biased projections, ReLU,
+                                      no rotary embedding; rms_eps is the LayerNorm eps)               */
 } spd_dims;
 
 typedef struct {
@@ -68,6 +71,17 @@ typedef struct {
     const void *w_down;    /* [hidden, ffn]                                                      */
     void *k_pages;         /* [n_pages, n_kv_heads, kv_block_size, head_dim]  written by the lib */
     void *v_pages;         /* same shape                                                         */
+    /* block_kind 1 only (ignored, may be null, for kind 0).  There w_gate is fc1 [ffn, hidden], w_down is
+     * fc2 [hidden, ffn] and w_up is not read.  Biases of column-split layers are split with them; the biases
+     * of the row-split layers (bo, b_fc2) cannot be split: each is added once, after the shard sum - in an
+     * SPD block bo also enters every device's MLP input X + P_i + b (Sec. 4.1.2). */
+    const void *attn_norm_b; /* [hidden]  LayerNorm shift before attention                       */
+    const void *bq;          /* [n_q_heads*head_dim]                                             */
+    const void *bk, *bv;     /* [n_kv_heads*head_dim]                                            */
+    const void *bo;          /* [hidden]  the b of Y_i = P_i + b                                 */
+    const void *mlp_norm_b;  /* [hidden]  LayerNorm shift before the MLP                         */
+    const void *b_fc1;       /* [ffn]                                                            */
+    const void *b_fc2;       /* [hidden]                                                         */
 } spd_layer;               /* device pointers, BORROWED: the caller keeps the tensors alive      */
 
 /* Bytes of device workspace spd_create needs for these dims and mask (host call, no GPU

@@ -19,6 +19,11 @@ SPD_OK = 0
 STATUS_NAMES = {0: "SPD_OK", -1: "SPD_EINVAL", -2: "SPD_ENULL", -3: "SPD_EWORKSPACE", -4: "SPD_ECAPACITY",
                 -5: "SPD_ECUDA", -6: "SPD_EDEVICE"}
 WEIGHT_NAMES = ("attn_norm", "wq", "wk", "wv", "wo", "mlp_norm", "w_gate", "w_up", "w_down")
+BIAS_FIELDS = ("attn_norm_b", "bq", "bk", "bv", "bo", "mlp_norm_b", "b_fc1", "b_fc2")
+# tensors of a layer of the block with bias (Sec. 4.1.2) -> fields of spd_layer
+BIAS_LAYER_FIELDS = {"attn_norm": "attn_norm", "attn_norm_b": "attn_norm_b", "wq": "wq", "bq": "bq", "wk": "wk", "bk": "bk", "wv": "wv",
+                     "bv": "bv", "wo": "wo", "bo": "bo", "mlp_norm": "mlp_norm", "mlp_norm_b": "mlp_norm_b", "w_fc1": "w_gate",
+                     "b_fc1": "b_fc1", "w_fc2": "w_down", "b_fc2": "b_fc2"}
 EXPORTS = ("spd_workspace_bytes", "spd_create", "spd_prefill", "spd_decode_step", "spd_sync_points",
            "spd_launches_per_decode_step", "spd_device_error", "spd_destroy", "spd_status_string",
            "spd_last_cuda_error", "spd_profile_begin", "spd_profile_end", "spd_profile_kinds",
@@ -38,11 +43,12 @@ class spd_dims(ctypes.Structure):
                 ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("ffn", ctypes.c_int32),
                 ("T", ctypes.c_int32), ("dtype", ctypes.c_int32), ("rms_eps", ctypes.c_float),
                 ("rope_base", ctypes.c_float), ("kv_block_size", ctypes.c_int32), ("max_batch", ctypes.c_int32),
-                ("max_seq_len", ctypes.c_int32), ("max_prefill_tokens", ctypes.c_int32)]
+                ("max_seq_len", ctypes.c_int32), ("max_prefill_tokens", ctypes.c_int32), ("block_kind", ctypes.c_int32)]
 
 
 class spd_layer(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_void_p) for n in WEIGHT_NAMES] + [("k_pages", ctypes.c_void_p), ("v_pages", ctypes.c_void_p)]
+    _fields_ = [(n, ctypes.c_void_p) for n in WEIGHT_NAMES] + [("k_pages", ctypes.c_void_p), ("v_pages", ctypes.c_void_p)] + \
+               [(n, ctypes.c_void_p) for n in BIAS_FIELDS]
 
 
 _lib = None
@@ -251,23 +257,28 @@ class SpdStack:
     def __init__(self, *, hidden: int, n_q_heads: int, n_kv_heads: int, head_dim: int, ffn: int, T: int,
                  sync_mask: Sequence[int], layers: List[Dict[str, torch.Tensor]], n_pages: int,
                  max_batch: int, max_seq_len: int, max_prefill_tokens: int, rms_eps: float = 1e-5,
-                 rope_base: float = 10000.0, kv_block_size: int = 16, device: Optional[torch.device] = None):
+                 rope_base: float = 10000.0, kv_block_size: int = 16, device: Optional[torch.device] = None, block: str = "llama"):
         self.lib = load_library()
         self.device = torch.device(device if device is not None else "cuda:0")
         dt = layers[0]["wq"].dtype
         if dt not in (torch.float32, torch.bfloat16):
             raise ValueError("weights must be float32 or bfloat16")
         self.dtype = dt
+        if block not in ("llama", "opt"):
+            raise ValueError("block: 'llama' (no bias) or 'opt' (with bias)")
+        self.block = block
+        # tensor name -> spd_layer field
+        self.fields = {n: n for n in WEIGHT_NAMES} if block == "llama" else dict(BIAS_LAYER_FIELDS)
         self.dims = spd_dims(len(layers), hidden, n_q_heads, n_kv_heads, head_dim, ffn, T,
                              0 if dt == torch.float32 else 1, rms_eps, rope_base, kv_block_size, max_batch,
-                             max_seq_len, max_prefill_tokens)
+                             max_seq_len, max_prefill_tokens, 0 if block == "llama" else 1)
         self.mask = (ctypes.c_uint8 * len(layers))(*[1 if m else 0 for m in sync_mask])
         if len(sync_mask) != len(layers):
             raise ValueError("one mask entry per layer")
         self.layers = layers
         self.n_pages = n_pages
         for lw in layers:
-            for n in WEIGHT_NAMES:
+            for n in self.fields:
                 t = lw[n]
                 if not (t.is_cuda and t.is_contiguous() and t.dtype == dt):
                     raise ValueError(f"{n}: need a contiguous CUDA tensor of dtype {dt}")
@@ -282,8 +293,8 @@ class SpdStack:
             base = (self.workspace.data_ptr() + 255) // 256 * 256
             arr = (spd_layer * len(layers))()
             for i, lw in enumerate(layers):
-                for n in WEIGHT_NAMES:
-                    setattr(arr[i], n, lw[n].data_ptr())
+                for n, field in self.fields.items():
+                    setattr(arr[i], field, lw[n].data_ptr())
                 arr[i].k_pages = self.k_pages[i].data_ptr()
                 arr[i].v_pages = self.v_pages[i].data_ptr()
             self._ctx = ctypes.c_void_p()
@@ -422,4 +433,4 @@ def stack_from_workload(w, layers, *, sync_mask=None, max_batch=None, max_seq_le
                     ffn=w.ffn, T=w.T, sync_mask=list(w.mask if sync_mask is None else sync_mask), layers=layers,
                     n_pages=n_pages, max_batch=max_batch, max_seq_len=max_seq_len,
                     max_prefill_tokens=max_prefill_tokens or min(w.batch * w.prompt, 8192), rms_eps=w.rms_eps,
-                    rope_base=w.rope_base, kv_block_size=w.kv_block, device=device)
+                    rope_base=w.rope_base, kv_block_size=w.kv_block, device=device, block=getattr(w, "block", "llama"))

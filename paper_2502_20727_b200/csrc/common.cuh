@@ -120,6 +120,10 @@ struct NormArgs {
     void *final_out;      // storage [M,H] copy of res_out, or null
     int M, H;
     float eps;
+    // block with bias (Sec. 4.1.2): `bias` (storage [H], the unsplittable bias of the row-split layer whose
+    // partials these are) is added to every group's residual and once to res_out; `shift` non-null turns the
+    // RMSNorm into a LayerNorm with that shift
+    const void *bias, *shift;
 };
 template <typename T> cudaError_t launch_residual_norm(const NormArgs &a, cudaStream_t st);
 
@@ -137,6 +141,7 @@ struct RopeKvArgs {
     int M, n_q_heads, head_dim;
     int use_rope;
     int *err;
+    const void *bq, *bk, *bv; // storage [nq*d], [nkv*d], [nkv*d] or null: biases of the column-split projections
 };
 template <typename T> cudaError_t launch_rope_kv(const RopeKvArgs &a, cudaStream_t st);
 
@@ -146,6 +151,8 @@ struct SiluMulArgs {
     int splits;
     void *act;              // storage [M,F]
     int M, F;
+    const void *bias;       // storage [F] or null
+    int relu;               // 1: act = relu(gate + bias) (fc1 of the block with bias; `up` is not read)
 };
 template <typename T> cudaError_t launch_silu_mul(const SiluMulArgs &a, cudaStream_t st);
 

@@ -66,12 +66,18 @@ __global__ void __launch_bounds__(512) residual_norm_kernel(NormArgs a)
     pdl_wait();
     __shared__ float red[32];
     const int m = blockIdx.x, H = a.H, G = a.n_groups, H4 = H >> 2;
-    float ss[MAX_T];
+    const bool ln = a.shift != nullptr;
+    float ss[MAX_T], sm[MAX_T];
 #pragma unroll
-    for (int g = 0; g < MAX_T; ++g) ss[g] = 0.f;
+    for (int g = 0; g < MAX_T; ++g) { ss[g] = 0.f; sm[g] = 0.f; }
+    auto base_of = [&](int c, long idx) {
+        float4 base = a.x_in ? load4<T>((const T *)a.x_in + idx) : *(const float4 *)(a.res_in + idx);
+        if (a.bias) base = f4add(base, load4<T>((const T *)a.bias + 4 * c)); // the row-split layer's bias, once
+        return base;
+    };
     for (int c = threadIdx.x; c < H4; c += blockDim.x) {
         const long idx = (long)m * H + 4 * c;
-        const float4 base = a.x_in ? load4<T>((const T *)a.x_in + idx) : *(const float4 *)(a.res_in + idx);
+        const float4 base = base_of(c, idx);
         float4 tot = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int g = 0; g < MAX_T; ++g) {
@@ -80,26 +86,40 @@ __global__ void __launch_bounds__(512) residual_norm_kernel(NormArgs a)
             tot = f4add(tot, y);
             const float4 r = f4add(base, y);
             ss[g] += r.x * r.x + r.y * r.y + r.z * r.z + r.w * r.w;
+            sm[g] += r.x + r.y + r.z + r.w;
         }
         const float4 r = f4add(base, tot);
         if (a.res_out) *(float4 *)(a.res_out + idx) = r;
         if (a.final_out) store4<T>((T *)a.final_out + idx, r);
     }
     if (!a.h_out) return;
-    float rs[MAX_T];
+    float rs[MAX_T], mu[MAX_T];
 #pragma unroll
-    for (int g = 0; g < MAX_T; ++g) rs[g] = (g < G) ? rsqrtf(block_sum(ss[g], red) / (float)H + a.eps) : 0.f;
+    for (int g = 0; g < MAX_T; ++g) {
+        rs[g] = 0.f;
+        mu[g] = 0.f;
+        if (g >= G) continue;
+        const float q = block_sum(ss[g], red) / (float)H;
+        if (ln) {
+            mu[g] = block_sum(sm[g], red) / (float)H;
+            rs[g] = rsqrtf(fmaxf(q - mu[g] * mu[g], 0.f) + a.eps);
+        } else {
+            rs[g] = rsqrtf(q + a.eps);
+        }
+    }
     const T *gain = (const T *)a.gain;
     for (int c = threadIdx.x; c < H4; c += blockDim.x) {
         const long idx = (long)m * H + 4 * c;
-        const float4 base = a.x_in ? load4<T>((const T *)a.x_in + idx) : *(const float4 *)(a.res_in + idx);
+        const float4 base = base_of(c, idx);
         const float4 gj = load4<T>(gain + 4 * c);
+        const float4 sh = ln ? load4<T>((const T *)a.shift + 4 * c) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int g = 0; g < MAX_T; ++g) {
             if (g >= G) continue;
             const float4 r = f4add(base, group_sum4(a, g, idx));
             store4<T>((T *)a.h_out + (long)g * a.h_stride + idx,
-                      make_float4(r.x * rs[g] * gj.x, r.y * rs[g] * gj.y, r.z * rs[g] * gj.z, r.w * rs[g] * gj.w));
+                      make_float4((r.x - mu[g]) * rs[g] * gj.x + sh.x, (r.y - mu[g]) * rs[g] * gj.y + sh.y,
+                                  (r.z - mu[g]) * rs[g] * gj.z + sh.z, (r.w - mu[g]) * rs[g] * gj.w + sh.w));
         }
     }
 }
@@ -197,7 +217,7 @@ template <typename T> cudaError_t launch_residual_norm(const NormArgs &a, cudaSt
     if (a.H % 4 || a.n_groups > MAX_T) return cudaErrorInvalidValue;
     const int h4 = a.H / 4;
     constexpr int CS = 8;
-    if (h4 % CS == 0 && h4 / CS <= 512 && (long)a.M * CS < 2147483647L) {
+    if (!a.bias && !a.shift && h4 % CS == 0 && h4 / CS <= 512 && (long)a.M * CS < 2147483647L) {
         const int cpc = h4 / CS;
         const int threads = cpc >= 256 ? 256 : (cpc + 31) / 32 * 32;
         const dim3 grid((unsigned)(a.M * CS));
@@ -263,6 +283,9 @@ template <typename T> __global__ void rope_kv_kernel(RopeKvArgs a)
             x1 += row[col_q + j + half];
             if (!is_q) { v0 += row[col_v + j]; v1 += row[col_v + j + half]; }
         }
+        if (is_q && a.bq) { x0 += to_f<T>(((const T *)a.bq)[col_q + j]); x1 += to_f<T>(((const T *)a.bq)[col_q + j + half]); }
+        if (!is_q && a.bk) { x0 += to_f<T>(((const T *)a.bk)[(long)kvh * d + j]); x1 += to_f<T>(((const T *)a.bk)[(long)kvh * d + j + half]); }
+        if (!is_q && a.bv) { v0 += to_f<T>(((const T *)a.bv)[(long)kvh * d + j]); v1 += to_f<T>(((const T *)a.bv)[(long)kvh * d + j + half]); }
         float c = 1.f, sn = 0.f;
         if (a.use_rope) { float2 cs = a.table[(long)m * half + j]; c = cs.x; sn = cs.y; }
         float r0 = x0 * c - x1 * sn, r1 = x1 * c + x0 * sn;
@@ -302,9 +325,10 @@ template <typename T> __global__ void silu_mul_kernel(SiluMulArgs a)
     float g = 0.f, u = 0.f;
     for (int s = 0; s < a.splits; ++s) {
         g += a.gate[(long)s * a.split_stride + m * a.ld + f];
-        u += a.up[(long)s * a.split_stride + m * a.ld + f];
+        if (!a.relu) u += a.up[(long)s * a.split_stride + m * a.ld + f];
     }
-    float act = g / (1.f + __expf(-g)) * u;
+    if (a.bias) g += to_f<T>(((const T *)a.bias)[f]);
+    float act = a.relu ? fmaxf(g, 0.f) : g / (1.f + __expf(-g)) * u;
     ((T *)a.act)[i] = from_f<T>(act);
 }
 

@@ -253,6 +253,7 @@ int check_dims(const spd_dims *d, const uint8_t *mask)
     if (d->dtype == 1 && (d->hidden % 8 || (d->ffn / d->T) % 8)) return SPD_EINVAL; // 16-byte rows for bf16 tiles
     if (d->kv_block_size < 1 || d->max_batch < 1 || d->max_seq_len < 1 || d->max_prefill_tokens < 1) return SPD_EINVAL;
     if (!(d->rms_eps > 0.f)) return SPD_EINVAL;
+    if (d->block_kind != 0 && d->block_kind != 1) return SPD_EINVAL;
     return SPD_OK;
 }
 
@@ -297,14 +298,17 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
     const bool swap = decode;
     const int tbox = TC ? tc_token_box(swap, M) : 0;
     int launches = 0;
+    const bool opt = d.block_kind == 1;              // block with bias (Sec. 4.1.2): LayerNorm, biases, ReLU, no rotary
+    const bool rope_on = d.rope_base > 0.f && !opt;
 
-    if (d.rope_base > 0.f) LAUNCH(K_ROPE_TABLE, launch_rope_table(c->rope, tm, M, d.head_dim, d.rope_base, st));
+    if (rope_on) LAUNCH(K_ROPE_TABLE, launch_rope_table(c->rope, tm, M, d.head_dim, d.rope_base, st));
 
     // block input -> fp32 residual stream and its attention RMSNorm
     {
         NormArgs a{};
         a.x_in = x; a.res_out = c->res[0]; a.h_out = c->h; a.h_stride = Mc * H;
         a.gain = c->layers[0].attn_norm; a.n_groups = 1; a.per_group = 0; a.M = M; a.H = H; a.eps = d.rms_eps;
+        if (opt) a.shift = c->layers[0].attn_norm_b;
         LAUNCH(K_NORM, launch_residual_norm<T>(a, st));
     }
     for (int l = 0; l < d.n_layers; ++l) {
@@ -340,7 +344,8 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
             RopeKvArgs a{};
             a.qkv = c->qkv32; a.ldq = nqkv; a.split_stride = (long)M * nqkv; a.splits = p.qkv_splits;
             a.table = c->rope; a.q_out = c->q; a.k_pages = w.k_pages; a.v_pages = w.v_pages; a.pt = pt; a.tm = tm;
-            a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.use_rope = d.rope_base > 0.f; a.err = c->err;
+            a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.use_rope = rope_on; a.err = c->err;
+            if (opt) { a.bq = w.bq; a.bk = w.bk; a.bv = w.bv; }
             LAUNCH(K_ROPE_KV, launch_rope_kv<T>(a, st));
         }
         // a4: attention, each shard over its own heads
@@ -378,6 +383,8 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
             a.n_groups = sync ? 1 : Tn; a.per_group = sync ? o_planes : p.o_per_group;
             a.res_out = c->res[1]; a.h_out = c->h; a.h_stride = Mc * H; a.gain = w.mlp_norm;
             a.M = M; a.H = H; a.eps = d.rms_eps;
+            // Y_i = P_i + b: b enters every device's MLP input and, once, the carried residual
+            if (opt) { a.bias = w.bo; a.shift = w.mlp_norm_b; }
             LAUNCH(K_NORM, launch_residual_norm<T>(a, st));
         }
         // a8: column-split gate / up; in an SPD block shard i reads its own MLP input plane
@@ -392,9 +399,9 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
                 g.c_off[0] = 0; g.c_off[1] = (long)p.gu_splits * M * F;
                 g.t_rows = M; g.w_rows[0] = g.w_rows[1] = F / Tn; g.batches = Tn; g.w_batched = 1; g.t_batched = sync ? 0 : 1;
                 g.num_kb = cdiv(H, 64); g.splits = p.gu_splits; g.err = c->err;
-                LAUNCH(K_GATE_UP, launch_gemm_tc(wmaps, 2, *am, g, swap, st));
+                LAUNCH(K_GATE_UP, launch_gemm_tc(wmaps, opt ? 1 : 2, *am, g, swap, st));
             }
-            for (int i = 0; i < 2 && !TC; ++i) {
+            for (int i = 0; i < (opt ? 1 : 2) && !TC; ++i) {
                 float *Cg = c->gu32 + (long)i * p.gu_splits * M * F;
                 {
                     GemmProblem g{};
@@ -409,6 +416,7 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
             SiluMulArgs a{};
             a.gate = c->gu32; a.up = c->gu32 + (long)p.gu_splits * M * F; a.ld = F; a.split_stride = (long)M * F;
             a.splits = p.gu_splits; a.act = c->act; a.M = M; a.F = F;
+            if (opt) { a.relu = 1; a.bias = w.b_fc1; }
             LAUNCH(K_SILU_MUL, launch_silu_mul<T>(a, st));
         }
         // a9: row-split down projection; summing over all of K = F IS the kept sync-point
@@ -432,8 +440,11 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
             NormArgs a{};
             a.res_in = c->res[1]; a.part = c->proj32; a.part_stride = (long)M * H; a.n_groups = 1; a.per_group = p.down_splits;
             a.res_out = c->res[0]; a.M = M; a.H = H; a.eps = d.rms_eps;
-            if (l + 1 < d.n_layers) { a.h_out = c->h; a.h_stride = Mc * H; a.gain = c->layers[l + 1].attn_norm; }
-            else a.final_out = out;
+            if (opt) a.bias = w.b_fc2;
+            if (l + 1 < d.n_layers) {
+                a.h_out = c->h; a.h_stride = Mc * H; a.gain = c->layers[l + 1].attn_norm;
+                if (opt) a.shift = c->layers[l + 1].attn_norm_b;
+            } else a.final_out = out;
             LAUNCH(K_NORM, launch_residual_norm<T>(a, st));
         }
     }
@@ -715,7 +726,7 @@ int build_weight_maps(Ctx &c)
         rc |= make_operand_map(&m.wo_full, w.wo, qd, H, 1, qd, 0, 128);
         rc |= make_operand_map(&m.wo_shard, w.wo, qd / T, H, T, qd, qd / T, 128);
         rc |= make_operand_map(&m.w_gate, w.w_gate, H, F / T, T, H, (F / T) * H, 128);
-        rc |= make_operand_map(&m.w_up, w.w_up, H, F / T, T, H, (F / T) * H, 128);
+        if (d.block_kind == 0) rc |= make_operand_map(&m.w_up, w.w_up, H, F / T, T, H, (F / T) * H, 128);
         rc |= make_operand_map(&m.w_down, w.w_down, F, H, 1, F, 0, 128);
         rc |= make_operand_map(&m.wq256, w.wq, H, qd, 1, H, 0, 256);
         rc |= make_operand_map(&m.wk256, w.wk, H, kd, 1, H, 0, 256);
@@ -730,7 +741,7 @@ int build_weight_maps(Ctx &c)
             rc |= make_operand_map(&m.vpages, w.v_pages, 128, rows, 1, 128, 0, 16);
         }
         rc |= make_operand_map(&m.w_gate64, w.w_gate, H, F / T, T, H, (F / T) * H, 64);
-        rc |= make_operand_map(&m.w_up64, w.w_up, H, F / T, T, H, (F / T) * H, 64);
+        if (d.block_kind == 0) rc |= make_operand_map(&m.w_up64, w.w_up, H, F / T, T, H, (F / T) * H, 64);
         if (rc) return SPD_EINVAL;
     }
     return SPD_OK;
@@ -762,8 +773,10 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     if (n_pages < 1) return SPD_EINVAL;
     for (int l = 0; l < dims->n_layers; ++l) {
         const spd_layer &w = layers[l];
-        if (!w.attn_norm || !w.wq || !w.wk || !w.wv || !w.wo || !w.mlp_norm || !w.w_gate || !w.w_up || !w.w_down ||
-            !w.k_pages || !w.v_pages)
+        if (!w.attn_norm || !w.wq || !w.wk || !w.wv || !w.wo || !w.mlp_norm || !w.w_gate || !w.w_down || !w.k_pages || !w.v_pages)
+            return SPD_ENULL;
+        if (dims->block_kind == 0 && !w.w_up) return SPD_ENULL;
+        if (dims->block_kind == 1 && (!w.attn_norm_b || !w.bq || !w.bk || !w.bv || !w.bo || !w.mlp_norm_b || !w.b_fc1 || !w.b_fc2))
             return SPD_ENULL;
     }
     int dev = 0;
@@ -831,7 +844,7 @@ int spd_prefill(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int32_t
     auto run = [&](int b0, int nb, int s0, int ns) -> int {
         TokMap tm{0, b0, ns, s0, nullptr};
         size_t off = ((size_t)b0 * S + s0) * d.hidden * es;
-        const bool fused = d.dtype == 1 && d.hidden % 16 == 0;
+        const bool fused = d.dtype == 1 && d.hidden % 16 == 0 && d.block_kind == 0;
         int rc = d.dtype == 0 ? run_tokens<float>(&c, (const char *)x + off, (char *)out + off, nb * ns, tm, block_table, max_pages, false, S, st)
                  : fused      ? run_prefill_fused(&c, (const char *)x + off, (char *)out + off, nb * ns, tm, block_table, max_pages, S, st)
                               : run_tokens<bf16>(&c, (const char *)x + off, (char *)out + off, nb * ns, tm, block_table, max_pages, false, S, st);
@@ -872,8 +885,9 @@ int spd_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_l
     if (ctx_bucket > d.max_seq_len) ctx_bucket = d.max_seq_len;
     if ((long)ctx_bucket > (long)max_pages * d.kv_block_size) ctx_bucket = max_pages * d.kv_block_size;
     auto run = [&]() {
-        return d.dtype == 0 ? run_tokens<float>(&c, x, out, B, tm, block_table, max_pages, true, ctx_bucket, st)
-                            : run_decode_fused(&c, x, out, B, tm, block_table, max_pages, ctx_bucket, st);
+        return d.dtype == 0        ? run_tokens<float>(&c, x, out, B, tm, block_table, max_pages, true, ctx_bucket, st)
+               : d.block_kind == 0 ? run_decode_fused(&c, x, out, B, tm, block_table, max_pages, ctx_bucket, st)
+                                   : run_tokens<bf16>(&c, x, out, B, tm, block_table, max_pages, true, ctx_bucket, st);
     };
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     CU_TRY(cudaStreamIsCapturing(st, &cap));
@@ -974,7 +988,7 @@ int spd_head_grouping_stats(spd_ctx *ctx, int32_t layer, const void *x, int32_t 
     if (!ctx || !x || !block_table || !sigma_scratch || !dist_dev || !dist || !norms) return SPD_ENULL;
     Ctx &c = ctx->c;
     const spd_dims &d = c.d;
-    if (d.dtype != 1 || d.hidden % 16 || layer < 0 || layer >= d.n_layers || B < 1 || S < 1 || B > d.max_batch) return SPD_EINVAL;
+    if (d.dtype != 1 || d.block_kind != 0 || d.hidden % 16 || layer < 0 || layer >= d.n_layers || B < 1 || S < 1 || B > d.max_batch) return SPD_EINVAL;
     if ((long)B * S > d.max_prefill_tokens) return SPD_EINVAL; // one chunk
     if (S > d.max_seq_len || (long)max_pages * d.kv_block_size < S) return SPD_ECAPACITY;
     if (!c.any_spd) return SPD_EWORKSPACE;

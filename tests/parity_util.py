@@ -58,9 +58,16 @@ class Pair:
                                              max_prefill_tokens=max_prefill_tokens or 4096, device=device)
         self.pos = np.zeros(self.B, dtype=np.int32)
 
+    def _oracle(self, x):
+        """The oracle's forward pass of the workload's block kind: (out, sync_points)."""
+        if getattr(self.w, "block", "llama") == "opt":
+            return oracle.bias_stack_forward(self.dims, self.mask, self.layers_np, x, self.pos, self.cache)
+        out, syncs, _ = oracle.stack_forward(self.dims, self.mask, self.layers_np, x, self.pos, self.cache)
+        return out, syncs
+
     def prefill(self, S, seed=0):
         x = si.make_hidden(self.w, (self.B, S, self.w.hidden), "cpu", seed, 0)
-        ref, syncs, _ = oracle.stack_forward(self.dims, self.mask, self.layers_np, to_np(x), self.pos, self.cache)
+        ref, syncs = self._oracle(to_np(x))
         got = self.stack.prefill(x.to(self.device), self.block_table)
         torch.cuda.synchronize()
         self.pos = self.pos + S
@@ -68,7 +75,7 @@ class Pair:
 
     def decode(self, t, seed=0):
         x = si.make_hidden(self.w, (self.B, self.w.hidden), "cpu", seed, 1 + t)
-        ref, _, _ = oracle.stack_forward(self.dims, self.mask, self.layers_np, to_np(x)[:, None, :], self.pos, self.cache)
+        ref, _ = self._oracle(to_np(x)[:, None, :])
         # fixed device buffers, as a serving loop has them: after the first step the library
         # replays its captured graph, so both the capture and the replay path are compared
         if not hasattr(self, "x_dev"):
