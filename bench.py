@@ -125,12 +125,12 @@ def decode_bytes(w: si.Workload, B: int, ctx: float):
 def gemm_weight_bytes(w: si.Workload):
     es = 2 if w.dtype == "bf16" else 4
     H, qd, kd, F = w.hidden, w.n_q_heads * w.head_dim, w.n_kv_heads * w.head_dim, w.ffn
-    return {"gemm_qkv": (qd + 2 * kd) * H * es, "gemm_o_proj": H * qd * es, "gemm_gate_up": 2 * F * H * es,
-            "gemm_down": H * F * es}
+    fc1 = (1 if w.block == "opt" else 2) * F * H * es  # fc1 alone, or gate and up
+    return {"gemm_qkv": (qd + 2 * kd) * H * es, "gemm_o_proj": H * qd * es, "gemm_gate_up": fc1, "gemm_down": H * F * es}
 
 
 def prefill_flops(w: si.Workload, B: int, S: int):
-    gemm = 2.0 * (w.params_per_layer() - 2 * w.hidden) * B * S
+    gemm = 2.0 * sum(gemm_weight_bytes(w).values()) / (2 if w.dtype == "bf16" else 4) * B * S
     attn = 2.0 * S * S * w.n_q_heads * w.head_dim * B  # causal: half of 4 S^2 nq d
     return w.n_layers * (gemm + attn)
 
@@ -258,7 +258,7 @@ def run_native(args, rank, world):
         "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": f"{w.name}: {w.n_layers} layers, hidden {w.hidden}, {w.n_q_heads}/{w.n_kv_heads} heads x "
                                f"{w.head_dim}, FFN {w.ffn}, T={w.T}, batch {B}, prompt {S}, decode",
-                   "mask": list(mask), "mask_name": args.mask, "l2": "weights per step exceed L2 (inputs larger than L2)",
+                   "block": w.block, "mask": list(mask), "mask_name": args.mask, "l2": "weights per step exceed L2 (inputs larger than L2)",
                    "context_mid": mid_ctx, "multi_gpu": "replicas only" if world > 1 else "single"},
         "e2e": {"value": B * world * K / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": B * w.hidden * es,
                 "d2h_bytes_per_step": B * w.hidden * es},
@@ -288,6 +288,10 @@ def run_native(args, rank, world):
 def oracle_decode_setup(w, mask, B, ctx0, seed=0):
     import oracle
     layers = si.to_oracle_layers(si.make_stack(w, "cpu", seed))
+    if w.block == "opt":  # same call shape for both block kinds
+        fwd = oracle.bias_stack_forward
+        oracle = type("O", (), {"stack_forward": staticmethod(lambda d, m, l, x, p, c: fwd(d, m, l, x, p, c) + (None,)),
+                                "Dims": oracle.Dims, "Cache": oracle.Cache})
     dims = oracle.Dims(w.n_layers, w.hidden, w.n_q_heads, w.n_kv_heads, w.head_dim, w.ffn, w.T, w.rms_eps, w.rope_base)
     cache = oracle.Cache(dims, B, ctx0 + 4096)
     rng = np.random.default_rng(seed)

@@ -136,18 +136,20 @@ __global__ void __launch_bounds__(256) residual_norm_cluster_kernel(NormArgs a)
     const int CS = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
     const int m = blockIdx.x / CS, H = a.H, G = a.n_groups, P = a.per_group;
     const int cpc = (H >> 2) / CS; // float4 chunks per CTA
-    __shared__ float warp_ss[8][MAX_T];
-    __shared__ float cta_ss[MAX_T];
+    __shared__ float warp_ss[8][2 * MAX_T];
+    __shared__ float cta_ss[2 * MAX_T]; // sums of squares, then (LayerNorm) sums
+    const bool ln = a.shift != nullptr;
     float4 base[NCH], y[NCH][MAX_T];
-    float ss[MAX_T];
+    float ss[MAX_T], sm[MAX_T];
 #pragma unroll
-    for (int g = 0; g < MAX_T; ++g) ss[g] = 0.f;
+    for (int g = 0; g < MAX_T; ++g) { ss[g] = 0.f; sm[g] = 0.f; }
 #pragma unroll
     for (int i = 0; i < NCH; ++i) {
         const int lc = threadIdx.x + i * blockDim.x;
         if (lc >= cpc) continue;
         const long idx = (long)m * H + 4 * (rank * cpc + lc);
         base[i] = a.x_in ? load4<T>((const T *)a.x_in + idx) : *(const float4 *)(a.res_in + idx);
+        if (a.bias) base[i] = f4add(base[i], load4<T>((const T *)a.bias + 4 * (rank * cpc + lc))); // the row-split layer's bias, once
         float4 tot = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int g = 0; g < MAX_T; ++g) {
@@ -162,6 +164,7 @@ __global__ void __launch_bounds__(256) residual_norm_cluster_kernel(NormArgs a)
             tot = f4add(tot, acc);
             const float4 r = f4add(base[i], acc);
             ss[g] += r.x * r.x + r.y * r.y + r.z * r.z + r.w * r.w;
+            sm[g] += r.x + r.y + r.z + r.w;
         }
         const float4 r = f4add(base[i], tot);
         if (a.res_out) *(float4 *)(a.res_out + idx) = r;
@@ -172,25 +175,31 @@ __global__ void __launch_bounds__(256) residual_norm_cluster_kernel(NormArgs a)
 #pragma unroll
     for (int g = 0; g < MAX_T; ++g) {
         if (g >= G) continue;
-        const float v = warp_sum(ss[g]);
-        if (lane == 0) warp_ss[warp][g] = v;
+        const float v = warp_sum(ss[g]), u = warp_sum(sm[g]);
+        if (lane == 0) { warp_ss[warp][g] = v; warp_ss[warp][MAX_T + g] = u; }
     }
     __syncthreads();
-    if (threadIdx.x < MAX_T) {
+    if (threadIdx.x < 2 * MAX_T) {
         float v = 0.f;
-        if ((int)threadIdx.x < G)
+        if ((int)(threadIdx.x % MAX_T) < G)
             for (int w = 0; w < nw; ++w) v += warp_ss[w][threadIdx.x];
         cta_ss[threadIdx.x] = v;
     }
     cluster.sync();
-    float rs[MAX_T];
+    float rs[MAX_T], mu[MAX_T];
 #pragma unroll
     for (int g = 0; g < MAX_T; ++g) {
         rs[g] = 0.f;
+        mu[g] = 0.f;
         if (g >= G) continue;
-        float tot = 0.f;
-        for (int r = 0; r < CS; ++r) tot += cluster.map_shared_rank(cta_ss, r)[g];
-        rs[g] = rsqrtf(tot / (float)H + a.eps);
+        float tot = 0.f, tsum = 0.f;
+        for (int r = 0; r < CS; ++r) { tot += cluster.map_shared_rank(cta_ss, r)[g]; tsum += cluster.map_shared_rank(cta_ss, r)[MAX_T + g]; }
+        if (ln) {
+            mu[g] = tsum / (float)H;
+            rs[g] = rsqrtf(fmaxf(tot / (float)H - mu[g] * mu[g], 0.f) + a.eps);
+        } else {
+            rs[g] = rsqrtf(tot / (float)H + a.eps);
+        }
     }
     cluster.sync(); // no CTA may exit while its shared memory is still being read
     const T *gain = (const T *)a.gain;
@@ -201,12 +210,14 @@ __global__ void __launch_bounds__(256) residual_norm_cluster_kernel(NormArgs a)
         const int col = 4 * (rank * cpc + lc);
         const long idx = (long)m * H + col;
         const float4 gj = load4<T>(gain + col);
+        const float4 sh = ln ? load4<T>((const T *)a.shift + col) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int g = 0; g < MAX_T; ++g) {
             if (g >= G) continue;
             const float4 r = f4add(base[i], y[i][g]);
             store4<T>((T *)a.h_out + (long)g * a.h_stride + idx,
-                      make_float4(r.x * rs[g] * gj.x, r.y * rs[g] * gj.y, r.z * rs[g] * gj.z, r.w * rs[g] * gj.w));
+                      make_float4((r.x - mu[g]) * rs[g] * gj.x + sh.x, (r.y - mu[g]) * rs[g] * gj.y + sh.y,
+                                  (r.z - mu[g]) * rs[g] * gj.z + sh.z, (r.w - mu[g]) * rs[g] * gj.w + sh.w));
         }
     }
 }
@@ -217,7 +228,7 @@ template <typename T> cudaError_t launch_residual_norm(const NormArgs &a, cudaSt
     if (a.H % 4 || a.n_groups > MAX_T) return cudaErrorInvalidValue;
     const int h4 = a.H / 4;
     constexpr int CS = 8;
-    if (!a.bias && !a.shift && h4 % CS == 0 && h4 / CS <= 512 && (long)a.M * CS < 2147483647L) {
+    if (h4 % CS == 0 && h4 / CS <= 512 && (long)a.M * CS < 2147483647L) {
         const int cpc = h4 / CS;
         const int threads = cpc >= 256 ? 256 : (cpc + 31) / 32 * 32;
         const dim3 grid((unsigned)(a.M * CS));

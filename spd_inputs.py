@@ -60,6 +60,9 @@ class Workload:
                 "wo": (H, qd), "w_gate": (F, H), "w_up": (F, H), "w_down": (H, F)}[name]
 
     def params_per_layer(self) -> int:
+        if self.block == "opt":
+            H, qd, kd, F = self.hidden, self.n_q_heads * self.head_dim, self.n_kv_heads * self.head_dim, self.ffn
+            return qd * H + 2 * kd * H + H * qd + 2 * F * H + (qd + 2 * kd + H + F + H) + 4 * H
         return sum(int(np.prod(self.shape_of(n))) for n in WEIGHT_NAMES)
 
 
@@ -79,6 +82,8 @@ WORKLOADS: Dict[str, Workload] = {
     "c4_b1": Workload("c4_b1", "bf16", 8, 8192, 64, 8, 128, 28672, 8, (0,) * 8, 1, 2048, 256),
     "c4_b32": Workload("c4_b32", "bf16", 8, 8192, 64, 8, 128, 28672, 8, (0,) * 8, 32, 2048, 256),
     "c5": Workload("c5", "bf16", 40, 8192, 64, 8, 128, 28672, 8, c5_mask(), 64, 512, 512),
+    # the block with bias (Sec. 4.1.2) at OPT-6.7B's shape (Sec. 5.1): 4 layers, hidden 4096, 32 heads x 128, ffn 16384
+    "opt67": Workload("opt67", "bf16", 4, 4096, 32, 32, 128, 16384, 8, (0,) * 4, 8, 512, 128, block="opt"),
 }
 
 
