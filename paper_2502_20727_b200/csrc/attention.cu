@@ -409,6 +409,80 @@ __device__ __forceinline__ void merge_splits(const AttnArgs &a, int b, int hq0, 
     }
 }
 
+// Tail of the paged decode kernels: merge the four compute warps of the block, then the context
+// splits.  With up to 8 splits the blocks of one (sequence, head tile) form a thread-block cluster:
+// each parks its merged, un-normalised partial in shared memory and, after one cluster barrier,
+// block r finishes every splits-th output element from its peers' shared memory - no partial goes
+// through global memory.  More splits: partials in global memory, last block to arrive merges.
+template <typename T, int D, int GT>
+__device__ __forceinline__ void finish_decode_attention(const AttnArgs &a, int b, int hq0, int sp, float (*sm_o)[GT][D],
+                                                        float (*sm_ml)[GT][2], float *sm_pml, int *sm_last)
+{
+    const bool clustered = a.cluster_merge && a.splits > 1;
+    const long pbase = ((long)b * a.n_q_heads + hq0) * a.splits + sp;
+    for (int idx = threadIdx.x; idx < GT * D; idx += blockDim.x) {
+        const int g = idx / D, dd = idx % D;
+        float gm = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) gm = fmaxf(gm, sm_ml[w][g][0]);
+        float acc = 0.f, gden = 0.f;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const float c = (sm_ml[w][g][0] == -INFINITY) ? 0.f : exp2f(sm_ml[w][g][0] - gm);
+            acc += sm_o[w][g][dd] * c;
+            gden += sm_ml[w][g][1] * c;
+        }
+        if (a.splits == 1) {
+            ((T *)a.out)[((long)b * a.n_q_heads + hq0 + g) * D + dd] = from_f<T>(gden > 0.f ? acc / gden : 0.f);
+        } else if (clustered) {
+            sm_o[0][g][dd] = acc; // only this thread reads (g, dd) of the warps' partials
+            if (dd == 0) { sm_pml[2 * g] = gm; sm_pml[2 * g + 1] = gden; }
+        } else {
+            const long pi = pbase + (long)g * a.splits;
+            a.part_o[pi * D + dd] = acc; // un-normalised
+            if (dd == 0) { a.part_ml[pi * 2] = gm; a.part_ml[pi * 2 + 1] = gden; }
+        }
+    }
+    if (a.splits == 1) return;
+    if (clustered) {
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+        const uint32_t o_base = tc::smem_u32(&sm_o[0][0][0]), ml_base = tc::smem_u32(sm_pml);
+        auto peer_f = [](uint32_t addr, int rank) {
+            uint32_t ra;
+            float v;
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(addr), "r"(rank));
+            asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(ra) : "memory");
+            return v;
+        };
+        for (int idx = sp + a.splits * (int)threadIdx.x; idx < GT * D; idx += a.splits * (int)blockDim.x) {
+            const int g = idx / D;
+            float gm = -INFINITY;
+            for (int s2 = 0; s2 < a.splits; ++s2) gm = fmaxf(gm, peer_f(ml_base + 8 * g, s2));
+            float acc = 0.f, gden = 0.f;
+            for (int s2 = 0; s2 < a.splits; ++s2) {
+                const float m2 = peer_f(ml_base + 8 * g, s2);
+                const float c = (m2 == -INFINITY) ? 0.f : exp2f(m2 - gm);
+                acc += peer_f(o_base + 4 * idx, s2) * c;
+                gden += peer_f(ml_base + 8 * g + 4, s2) * c;
+            }
+            ((T *)a.out)[((long)b * a.n_q_heads + hq0) * D + idx] = from_f<T>(gden > 0.f ? acc / gden : 0.f);
+        }
+        // no block may exit while a peer still reads its shared memory
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+        return;
+    }
+    // the last block of this (sequence, head tile) to arrive merges the splits
+    __threadfence();
+    __syncthreads();
+    int *cnt = a.counters + (long)b * gridDim.x + blockIdx.x;
+    if (threadIdx.x == 0) *sm_last = (atomicAdd(cnt, 1) == a.splits - 1);
+    __syncthreads();
+    if (!*sm_last) return;
+    __threadfence();
+    merge_splits<T, D, GT>(a, b, hq0, &sm_o[0][0][0]);
+    if (threadIdx.x == 0) *cnt = 0; // ready for the next launch
+}
+
 // Ring of the bulk-copy decode kernel: K and V page per slot, 32 KB in all (measured better than
 // 64 KB: four thread blocks per SM keep every block of a step resident at once).
 template <typename T, int D> struct DecodeRing {
@@ -610,6 +684,7 @@ __global__ void __launch_bounds__(160) decode_attention_ring_kernel(AttnArgs a)
     int *sm_bt = (int *)(tail + 2 * R * 8);           // pages of this block's range
     volatile int *abort_flag = (volatile int *)(sm_bt + DECODE_MAX_PAGES_PER_BLOCK);
     int *sm_last = (int *)(sm_bt + DECODE_MAX_PAGES_PER_BLOCK + 1);
+    float *sm_pml = (float *)(sm_bt + DECODE_MAX_PAGES_PER_BLOCK + 2); // [GT][2] merged max, denominator of this block
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (R + s); };
 
@@ -764,46 +839,14 @@ __global__ void __launch_bounds__(160) decode_attention_ring_kernel(AttnArgs a)
     }
     __syncthreads();
     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_MAIN_DONE);
-    // merge the 4 warps; thread -> (head of the tile, dim)
-    const long pbase = ((long)b * a.n_q_heads + hq0) * a.splits + sp;
-    for (int idx = threadIdx.x; idx < GT * D; idx += blockDim.x) {
-        const int g = idx / D, dd = idx % D;
-        float gm = -INFINITY;
-#pragma unroll
-        for (int w = 0; w < 4; ++w) gm = fmaxf(gm, sm_ml[w][g][0]);
-        float acc = 0.f, gden = 0.f;
-#pragma unroll
-        for (int w = 0; w < 4; ++w) {
-            const float c = (sm_ml[w][g][0] == -INFINITY) ? 0.f : exp2f(sm_ml[w][g][0] - gm);
-            acc += sm_o[w][g][dd] * c;
-            gden += sm_ml[w][g][1] * c;
-        }
-        if (a.splits == 1) {
-            ((T *)a.out)[((long)b * a.n_q_heads + hq0 + g) * D + dd] = from_f<T>(gden > 0.f ? acc / gden : 0.f);
-        } else {
-            const long pi = pbase + (long)g * a.splits;
-            a.part_o[pi * D + dd] = acc; // un-normalised
-            if (dd == 0) { a.part_ml[pi * 2] = gm; a.part_ml[pi * 2 + 1] = gden; }
-        }
-    }
-    if (a.splits == 1) return;
-    // the last block of this (sequence, head tile) to arrive merges the splits
-    __threadfence();
-    __syncthreads();
-    int *cnt = a.counters + (long)b * gridDim.x + blockIdx.x;
-    if (threadIdx.x == 0) *sm_last = (atomicAdd(cnt, 1) == a.splits - 1);
-    __syncthreads();
-    if (!*sm_last) return;
-    __threadfence();
-    merge_splits<T, D, GT>(a, b, hq0, &sm_o[0][0][0]);
-    if (threadIdx.x == 0) *cnt = 0; // ready for the next launch
+    finish_decode_attention<T, D, GT>(a, b, hq0, sp, sm_o, sm_ml, sm_pml, sm_last);
     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_END);
 }
 
 template <typename T, int D, int GT> cudaError_t launch_ring(const AttnArgs &a, cudaStream_t st)
 {
     constexpr int PAGE_BYTES = 16 * D * (int)sizeof(T), R = DecodeRing<T, D>::SLOTS;
-    constexpr int SMEM = R * 2 * PAGE_BYTES + 4 * GT * D * 4 + 4 * GT * 2 * 4 + 2 * R * 8 + (DECODE_MAX_PAGES_PER_BLOCK + 2) * 4;
+    constexpr int SMEM = R * 2 * PAGE_BYTES + 4 * GT * D * 4 + 4 * GT * 2 * 4 + 2 * R * 8 + (DECODE_MAX_PAGES_PER_BLOCK + 2 + 2 * GT) * 4;
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(decode_attention_ring_kernel<T, D, GT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
@@ -815,7 +858,9 @@ template <typename T, int D, int GT> cudaError_t launch_ring(const AttnArgs &a, 
         attr_done = true;
     }
     dim3 grid(a.n_q_heads / GT, a.B, a.splits);
-    return launch_kernel(decode_attention_ring_kernel<T, D, GT>, grid, dim3(160), SMEM, st, 0, a);
+    AttnArgs b = a;
+    b.cluster_merge = a.splits > 1 && a.splits <= 8;
+    return launch_kernel_z(decode_attention_ring_kernel<T, D, GT>, grid, dim3(160), SMEM, st, b.cluster_merge ? a.splits : 1, b);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -846,6 +891,7 @@ __global__ void __launch_bounds__(160) decode_attention_mma_kernel(const __grid_
     int *sm_bt = (int *)(tail + 2 * R * 8);
     volatile int *abort_flag = (volatile int *)(sm_bt + DECODE_MAX_PAGES_PER_BLOCK);
     int *sm_last = (int *)(sm_bt + DECODE_MAX_PAGES_PER_BLOCK + 1);
+    float *sm_pml = (float *)(sm_bt + DECODE_MAX_PAGES_PER_BLOCK + 2); // [GT][2] merged max, denominator of this block
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (R + s); };
 
@@ -987,45 +1033,13 @@ __global__ void __launch_bounds__(160) decode_attention_mma_kernel(const __grid_
     }
     __syncthreads();
     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_MAIN_DONE);
-    // merge the 4 warps; thread -> (head of the tile, dim)
-    const long pbase = ((long)b * a.n_q_heads + hq0) * a.splits + sp;
-    for (int idx = threadIdx.x; idx < GT * D; idx += blockDim.x) {
-        const int gg = idx / D, dd = idx % D;
-        float gm = -INFINITY;
-#pragma unroll
-        for (int w = 0; w < 4; ++w) gm = fmaxf(gm, sm_ml[w][gg][0]);
-        float acc = 0.f, gden = 0.f;
-#pragma unroll
-        for (int w = 0; w < 4; ++w) {
-            const float c = (sm_ml[w][gg][0] == -INFINITY) ? 0.f : exp2f(sm_ml[w][gg][0] - gm);
-            acc += sm_o[w][gg][dd] * c;
-            gden += sm_ml[w][gg][1] * c;
-        }
-        if (a.splits == 1) {
-            ((bf16 *)a.out)[((long)b * a.n_q_heads + hq0 + gg) * D + dd] = __float2bfloat16_rn(gden > 0.f ? acc / gden : 0.f);
-        } else {
-            const long pi = pbase + (long)gg * a.splits;
-            a.part_o[pi * D + dd] = acc; // un-normalised
-            if (dd == 0) { a.part_ml[pi * 2] = gm; a.part_ml[pi * 2 + 1] = gden; }
-        }
-    }
-    if (a.splits == 1) return;
-    // the last block of this (sequence, head tile) to arrive merges the splits
-    __threadfence();
-    __syncthreads();
-    int *cnt = a.counters + (long)b * gridDim.x + blockIdx.x;
-    if (threadIdx.x == 0) *sm_last = (atomicAdd(cnt, 1) == a.splits - 1);
-    __syncthreads();
-    if (!*sm_last) return;
-    __threadfence();
-    merge_splits<bf16, D, GT>(a, b, hq0, &sm_o[0][0][0]);
-    if (threadIdx.x == 0) *cnt = 0; // ready for the next launch
+    finish_decode_attention<bf16, D, GT>(a, b, hq0, sp, sm_o, sm_ml, sm_pml, sm_last);
     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_END);
 }
 
 template <int GT> cudaError_t launch_decode_mma(const AttnArgs &a, cudaStream_t st)
 {
-    constexpr int SMEM = 1024 + 4 * 8192 + 4 * GT * 128 * 4 + 4 * GT * 2 * 4 + 2 * 4 * 8 + (DECODE_MAX_PAGES_PER_BLOCK + 2) * 4;
+    constexpr int SMEM = 1024 + 4 * 8192 + 4 * GT * 128 * 4 + 4 * GT * 2 * 4 + 2 * 4 * 8 + (DECODE_MAX_PAGES_PER_BLOCK + 2 + 2 * GT) * 4;
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(decode_attention_mma_kernel<GT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
@@ -1033,8 +1047,10 @@ template <int GT> cudaError_t launch_decode_mma(const AttnArgs &a, cudaStream_t 
         attr_done = true;
     }
     dim3 grid(a.n_q_heads / GT, a.B, a.splits);
-    return launch_kernel(decode_attention_mma_kernel<GT>, grid, dim3(160), SMEM, st, 0, *(const CUtensorMap *)a.k_map,
-                         *(const CUtensorMap *)a.v_map, a);
+    AttnArgs b = a;
+    b.cluster_merge = a.splits > 1 && a.splits <= 8;
+    return launch_kernel_z(decode_attention_mma_kernel<GT>, grid, dim3(160), SMEM, st, b.cluster_merge ? a.splits : 1,
+                           *(const CUtensorMap *)a.k_map, *(const CUtensorMap *)a.v_map, b);
 }
 
 template <typename T, int D> cudaError_t launch_decode_d(const AttnArgs &a, cudaStream_t st)

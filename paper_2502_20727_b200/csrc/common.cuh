@@ -56,6 +56,28 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// The same with a thread-block cluster along grid z.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel_z(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                   int cluster_z, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    at[1].id = cudaLaunchAttributeClusterDimension;
+    at[1].val.clusterDim.x = 1;
+    at[1].val.clusterDim.y = 1;
+    at[1].val.clusterDim.z = (unsigned)(cluster_z > 1 ? cluster_z : 1);
+    cfg.attrs = at;
+    cfg.numAttrs = cluster_z > 1 ? 2 : 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 __device__ __forceinline__ float warp_sum(float v)
 {
 #pragma unroll
@@ -172,6 +194,7 @@ struct AttnArgs {
     // optional (decode, bf16, head_dim 128, 16-token pages): tensor maps over the K and V pages seen as
     // [n_pages * n_kv_heads * 16 rows][head_dim], box 64 x 16, 128-byte swizzle (host pointers to CUtensorMap)
     const void *k_map, *v_map;
+    int cluster_merge;      // set by the launcher: the splits of a (sequence, head tile) are one thread-block cluster
 };
 // Paged decode attention with 16-token pages: query heads per thread block for a GQA group
 // size, and the most pages one block may be given (the host picks splits accordingly).

@@ -21,6 +21,8 @@
 // they fetch what the epilogue needs (rstd, page addresses).  Warp 4 issues the TMA loads,
 // warp 5 the MMAs.
 #include "gemm_decode.cuh"
+
+#include <math.h>
 #include "tc_ptx.cuh"
 #include "trace.cuh"
 
@@ -486,10 +488,22 @@ cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
 }
 
 // One thread block per 128 columns, all tokens: the same outputs EPI_DOWN leaves for the next block.
-__global__ void __launch_bounds__(128) decode_prologue_kernel(PrologueArgs a)
+__global__ void __launch_bounds__(128) decode_prologue_kernel(PrologueArgs a, int h_tiles, double log_base)
 {
     pdl_launch_dependents();
     pdl_wait();
+    if ((int)blockIdx.x >= h_tiles) {
+        // rotary table of this step, evaluated in double and shared by all blocks of the stack
+        const int half = a.head_dim / 2, i = ((int)blockIdx.x - h_tiles) * 128 + threadIdx.x;
+        if (i >= a.M * half) return;
+        int m = i / half, j = i % half, b, pos;
+        a.tm.locate(m, b, pos);
+        const double theta = exp(-2.0 * (double)j / (double)a.head_dim * log_base);
+        double sn, cs;
+        sincos((double)pos * theta, &sn, &cs);
+        a.rope_table[i] = make_float2((float)cs, (float)sn);
+        return;
+    }
     __shared__ float sm[4];
     const int r = threadIdx.x, warp = r >> 5, lane = r & 31, n = blockIdx.x * 128 + r;
     const bool valid = n < a.H;
@@ -563,7 +577,10 @@ cudaError_t launch_gemm_decode(DecEpilogue epi, const TcMap *const *weights, con
 cudaError_t launch_decode_prologue(const PrologueArgs &a, cudaStream_t st)
 {
     if (a.M <= 0) return cudaSuccess;
-    return launch_kernel(decode_prologue_kernel, dim3((a.H + 127) / 128), dim3(128), 0, st, 0, a);
+    const int h_tiles = (a.H + 127) / 128;
+    const int table_blocks = a.rope_table ? (a.M * (a.head_dim / 2) + 127) / 128 : 0;
+    return launch_kernel(decode_prologue_kernel, dim3(h_tiles + table_blocks), dim3(128), 0, st, 0, a, h_tiles,
+                         a.rope_table ? log((double)a.rope_base) : 0.0);
 }
 
 } // namespace spd

@@ -81,6 +81,11 @@ struct PrologueArgs {
     float *ss_out;     // [tiles][1][Mcap]
     long Mcap;
     int M, H;
+    // decode: the same launch also fills the rotary table of the step (cos, sin of pos * base^(-2j/d))
+    float2 *rope_table; // [M][head_dim/2] or null
+    TokMap tm;
+    int head_dim;
+    float rope_base;
 };
 cudaError_t launch_decode_prologue(const PrologueArgs &a, cudaStream_t st);
 

@@ -472,11 +472,11 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
         const SiteGeom sg = site_geom(d, site);
         return decode_splits(sg.tiles * tok_tiles, sg.num_kb, c->split_override[site], 8 / sg.shard_ranges);
     };
-    if (rope) LAUNCH(K_ROPE_TABLE, launch_rope_table(c->rope, tm, M, d.head_dim, d.rope_base, st));
     {
         PrologueArgs a{};
         a.x = x; a.res_out = c->res[0]; a.gain = c->layers[0].attn_norm; a.hg = c->h; a.ss_out = c->ss_attn;
         a.Mcap = Mc; a.M = M; a.H = H;
+        if (rope) { a.rope_table = c->rope; a.tm = tm; a.head_dim = d.head_dim; a.rope_base = d.rope_base; }
         LAUNCH(K_NORM, launch_decode_prologue(a, st));
     }
     auto base_args = [&]() {
