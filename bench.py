@@ -187,11 +187,20 @@ def run_native(args, rank, world):
     x_in = torch.empty_like(xs[0])
     seq_in = torch.empty_like(seq_all[0])
 
+    if args.rank_mode:
+        # every rank of a T-GPU group executed on this GPU: shard sums as exchanges through global memory
+        stack.tp_attach_local()
+        out_ranks = torch.empty((w.T, B, w.hidden), dtype=xs.dtype, device=dev)
+        out = out_ranks[0]
+
     def step(t, x_ready=False):
         if not x_ready:
             x_in.copy_(xs[t])
         seq_in.copy_(seq_all[t])
-        stack.decode_step(x_in, seq_in, bt, S + t + 1, out)
+        if args.rank_mode:
+            stack.tp_decode_step(x_in, seq_in, bt, S + t + 1, out_ranks)
+        else:
+            stack.decode_step(x_in, seq_in, bt, S + t + 1, out)
 
     def barrier():
         torch.cuda.synchronize()
@@ -258,7 +267,7 @@ def run_native(args, rank, world):
         "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": f"{w.name}: {w.n_layers} layers, hidden {w.hidden}, {w.n_q_heads}/{w.n_kv_heads} heads x "
                                f"{w.head_dim}, FFN {w.ffn}, T={w.T}, batch {B}, prompt {S}, decode",
-                   "block": w.block, "mask": list(mask), "mask_name": args.mask, "l2": "weights per step exceed L2 (inputs larger than L2)",
+                   "block": w.block, "rank_mode": bool(args.rank_mode), "mask": list(mask), "mask_name": args.mask, "l2": "weights per step exceed L2 (inputs larger than L2)",
                    "context_mid": mid_ctx, "multi_gpu": "replicas only" if world > 1 else "single"},
         "e2e": {"value": B * world * K / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": B * w.hidden * es,
                 "d2h_bytes_per_step": B * w.hidden * es},
@@ -270,7 +279,7 @@ def run_native(args, rank, world):
         "roofline": {"bound": "hbm", "kernel": "weight-streaming projection GEMM (qkv, o_proj, gate/up, down)",
                      "achieved": gemm_gbs, "peak": hbm_peak, "unit": "GB/s",
                      "frac": (gemm_gbs / hbm_peak) if gemm_gbs else None,
-                     "traffic": NCU_TRAFFIC_PER_LAUNCH.get(w.name) if not args.tune else None,
+                     "traffic": NCU_TRAFFIC_PER_LAUNCH.get(w.name) if not (args.tune or args.rank_mode) else None,
                      "algorithmic_bytes_per_launch": gemm_bytes_step / max(gemm_launches / K, 1), "peak_kind": peak_kind,
                      "launches_per_step": gemm_launches / K, "avg_launch_us": gemm_ms * 1e3 / max(gemm_launches, 1),
                      "bytes_per_step": gemm_bytes_step},
@@ -352,6 +361,8 @@ def main():
     ap.add_argument("--prefill-reps", type=int, default=3)
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--rank-mode", action="store_true",
+                    help="decode through spd_tp_decode_step: all T ranks of a tensor-parallel group executed on this GPU")
     ap.add_argument("--tune", default="", help="decode tuning knobs, e.g. qkv_splits=4,l2_prefetch_blocks=8 (see spd_set_tuning)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", 0))

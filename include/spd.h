@@ -246,6 +246,51 @@ int spd_head_scatter(const float *dist, int32_t n_heads, int32_t heads_per_unit,
  * Pure host function.  Errors: SPD_ENULL, SPD_EINVAL (T > 8). */
 int spd_mlp_match(const double *norms, int32_t T, int32_t *mlp_of_device, double *objective);
 
+/* ---- Tensor parallelism across GPUs (Sec. 3: one shard per device; Sec. 4.1.1: what an SPD block
+ * still exchanges) --------------------------------------------------------------------------------
+ *
+ * A context created from the dims of ONE shard (T = 1; n_q_heads, n_kv_heads, ffn and the weight
+ * matrices those of the shard: rows [r*n/T, (r+1)*n/T) of wq / wk / wv / w_gate / w_up, columns
+ * [r*k/T, (r+1)*k/T) of wo / w_down stored as a contiguous matrix) becomes rank r of a group of T
+ * ranks once it is attached to the group's regions.  A region is spd_tp_region_bytes() of device
+ * memory owned by one rank and WRITABLE BY EVERY RANK (peer-mapped: CUDA IPC, the driver's
+ * virtual-memory mappings or a symmetric-memory allocator; plain stores and loads only, no
+ * multicast).  It holds the rank's receive planes and arrival flags and the rank's private copy
+ * of the residual stream.  `regions` is a host array of T device pointers as mapped in the
+ * calling process; entry j is rank j's region; 1024-byte aligned.
+ *
+ * A context created with T > 1 shards (the emulation all other entry points use) can be attached
+ * with rank_base = 0 and group size T = dims.T: then ONE GPU executes all T ranks, every launch
+ * covering all ranks' data, through exactly the same kernels and exchange protocol; its T regions
+ * must lie at equal distances (regions[j] = regions[0] + j * stride).  All thread blocks of such
+ * a launch have to be resident at once (they wait on one another): a launch that does not fit is
+ * refused with SPD_ECUDA (cudaErrorCooperativeLaunchTooLarge) before anything runs.
+ *
+ * Attaching zeroes the local regions on `stream`.  It is collective: every rank attaches, then
+ * the group synchronises on the host (stream synchronize + barrier) before anyone's first step.
+ * bf16 LLaMA-style stacks only (dtype 1, block_kind 0, hidden % 16 == 0).
+ * Errors: SPD_ENULL, SPD_EINVAL, SPD_EWORKSPACE (region too small / misaligned), SPD_ECUDA. */
+int spd_tp_region_bytes(const spd_ctx *ctx, int32_t T, size_t *out_bytes);
+int spd_tp_attach(spd_ctx *ctx, int32_t T, int32_t rank_base, void *const *regions, size_t region_bytes,
+                  void *stream);
+int spd_tp_detach(spd_ctx *ctx);
+
+/* One decode step of an attached context (same arguments as spd_decode_step; every rank of the
+ * group calls it with the same x, seq_lens and block-table contents, and the same number of
+ * times).  Per block and rank: QKV on the rank's heads, attention, o_proj, gate/up, down - and
+ * the shard sums the block keeps as one-shot exchanges inside the tail of the projection that
+ * produces the partial: each rank stores its fp32 partial rows into every rank's receive planes,
+ * publishes the step number in the peers' flags and adds the T planes in rank order, so all
+ * ranks hold bit-identical residual streams.  A TP block exchanges twice (Y_i after o_proj,
+ * Z_i after down: Sec. 3), an SPD block once (Y_i + Z_i after down: Sec. 4.1.1).
+ *   out : [ranks held by the context][B][hidden] bf16 - every rank's copy of the output
+ * A wait for a peer gives up after about one second: the kernels then return normally, the
+ * step's output is undefined and spd_device_error reports bit 8; the context stays usable.
+ * Errors: SPD_ENULL, SPD_EINVAL (not attached, B > max_batch), SPD_ECAPACITY, SPD_ECUDA. */
+int spd_tp_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_lens,
+                       const int32_t *block_table, int32_t max_pages, int32_t max_context, void *out,
+                       void *stream);
+
 /* Number of shard sums ("sync-points", Sec. 3) one forward pass of this stack executes:
  * 2 per TP block, 1 per SPD block. */
 int spd_sync_points(const spd_ctx *ctx);
@@ -254,7 +299,8 @@ int spd_sync_points(const spd_ctx *ctx);
 int spd_launches_per_decode_step(const spd_ctx *ctx);
 
 /* Read and clear the device error flag (synchronises `stream`).  0 = clean; otherwise a bit
- * set: 1 block-table entry out of range, 2 position beyond capacity, 4 bounded wait gave up.
+ * set: 1 block-table entry out of range, 2 position beyond capacity, 4 bounded wait gave up,
+ * 8 a wait for another rank's partial sums gave up.
  * Kernels that meet such a condition skip the access, set the flag and return normally. */
 int spd_device_error(spd_ctx *ctx, void *stream, int32_t *out_flag);
 

@@ -89,6 +89,10 @@ def load_library() -> ctypes.CDLL:
     lib.spd_alg1_plan.argtypes = [ctypes.POINTER(ctypes.c_double), i32, i32, ctypes.c_double, ctypes.c_double, vp, vp]
     lib.spd_set_tuning.argtypes = [vp, ctypes.c_char_p, i32]
     lib.spd_gemm_bf16_sum_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, vp]
+    lib.spd_tp_region_bytes.argtypes = [vp, i32, ctypes.POINTER(sz)]
+    lib.spd_tp_attach.argtypes = [vp, i32, i32, ctypes.POINTER(vp), sz, vp]
+    lib.spd_tp_detach.argtypes = [vp]
+    lib.spd_tp_decode_step.argtypes = [vp, vp, i32, vp, vp, i32, i32, vp, vp]
     lib.spd_profile_begin.argtypes = [vp]
     lib.spd_profile_end.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     lib.spd_profile_kinds.argtypes = []
@@ -246,6 +250,22 @@ def permute_layer(lw: Dict[str, torch.Tensor], *, n_q_heads: int, n_kv_heads: in
     return out
 
 
+def shard_layer(lw: Dict[str, torch.Tensor], r: int, T: int) -> Dict[str, torch.Tensor]:
+    """The tensors rank r of a T-GPU group holds of one LLaMA-style layer (Sec. 3): rows r of the
+    column-parallel matrices, columns r of the row-parallel ones (as contiguous matrices), the norm gains whole."""
+    def rows(t):
+        n = t.shape[0] // T
+        return t[r * n:(r + 1) * n].contiguous()
+
+    def cols(t):
+        n = t.shape[1] // T
+        return t[:, r * n:(r + 1) * n].contiguous()
+
+    return {"attn_norm": lw["attn_norm"], "mlp_norm": lw["mlp_norm"], "wq": rows(lw["wq"]), "wk": rows(lw["wk"]),
+            "wv": rows(lw["wv"]), "wo": cols(lw["wo"]), "w_gate": rows(lw["w_gate"]), "w_up": rows(lw["w_up"]),
+            "w_down": cols(lw["w_down"])}
+
+
 class SpdStack:
     """A stack of TP / SPD decoder blocks over caller-held weights and paged KV tensors.
 
@@ -395,6 +415,65 @@ class SpdStack:
         see spd_set_tuning."""
         for k, v in kw.items():
             _check("spd_set_tuning", self.lib.spd_set_tuning(self._ctx, k.encode(), int(v)))
+
+    # -- tensor parallelism across GPUs (spd_tp_*) ------------------------------------------
+    def tp_region_bytes(self, T: int) -> int:
+        n = ctypes.c_size_t(0)
+        _check("spd_tp_region_bytes", self.lib.spd_tp_region_bytes(self._ctx, int(T), ctypes.byref(n)))
+        return n.value
+
+    def tp_attach(self, T: int, rank_base: int, region_ptrs: Sequence[int], region_bytes: int):
+        """Make this context rank ``rank_base`` (and the following ones, if it holds several shards) of a
+        group of T ranks; region_ptrs[j] = device address of rank j's region as mapped in this process."""
+        if len(region_ptrs) != T:
+            raise ValueError("one region per rank")
+        arr = (ctypes.c_void_p * T)(*[ctypes.c_void_p(int(p)) for p in region_ptrs])
+        with torch.cuda.device(self.device):
+            _check("spd_tp_attach", self.lib.spd_tp_attach(self._ctx, int(T), int(rank_base), arr, int(region_bytes),
+                                                            _stream_ptr()))
+
+    def tp_attach_local(self):
+        """All T ranks of the group on this GPU (every launch covers all ranks' data): regions in one tensor."""
+        T = self.dims.T
+        stride = (self.tp_region_bytes(T) + 1023) // 1024 * 1024
+        with torch.cuda.device(self.device):
+            self._tp_regions = torch.empty(T * stride + 1024, dtype=torch.uint8, device=self.device)
+        base = (self._tp_regions.data_ptr() + 1023) // 1024 * 1024
+        self.tp_attach(T, 0, [base + j * stride for j in range(T)], stride)
+
+    def tp_attach_symmetric(self, rank: int, world: int, group=None):
+        """Rank ``rank`` of a real group of ``world`` GPUs (one process per GPU, torch.distributed initialised
+        with NCCL): the region is a symmetric-memory allocation whose peer mappings the rendezvous returns."""
+        import torch.distributed as dist
+        import torch.distributed._symmetric_memory as symm
+        group = group if group is not None else dist.group.WORLD
+        nbytes = (self.tp_region_bytes(world) + 1023) // 1024 * 1024
+        with torch.cuda.device(self.device):
+            self._tp_regions = symm.empty(nbytes, dtype=torch.uint8, device=self.device)
+            handle = symm.rendezvous(self._tp_regions, group.group_name if hasattr(group, "group_name") else group)
+            ptrs = [int(p) for p in handle.buffer_ptrs]
+            self.tp_attach(world, rank, ptrs, nbytes)
+            torch.cuda.current_stream().synchronize()
+        dist.barrier(group=group)
+        self._tp_handle = handle
+
+    def tp_detach(self):
+        _check("spd_tp_detach", self.lib.spd_tp_detach(self._ctx))
+
+    def tp_decode_step(self, x: torch.Tensor, seq_lens: torch.Tensor, block_table: torch.Tensor, max_context: int,
+                       out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """One decode step in rank mode; returns [ranks held by this context, B, hidden]."""
+        B, H = x.shape
+        self._check_io(x, block_table)
+        if not (seq_lens.is_cuda and seq_lens.dtype == torch.int32 and seq_lens.numel() == B):
+            raise ValueError("seq_lens: int32 CUDA tensor [B]")
+        if out is None:
+            out = torch.empty((self.dims.T, B, H), dtype=x.dtype, device=x.device)
+        with torch.cuda.device(self.device):
+            _check("spd_tp_decode_step", self.lib.spd_tp_decode_step(self._ctx, x.data_ptr(), B, seq_lens.data_ptr(),
+                                                                      block_table.data_ptr(), block_table.shape[1],
+                                                                      int(max_context), out.data_ptr(), _stream_ptr()))
+        return out
 
     def sync_points(self) -> int:
         return self.lib.spd_sync_points(self._ctx)

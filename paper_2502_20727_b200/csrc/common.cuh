@@ -13,6 +13,7 @@ enum : int {
     ERR_PAGE_RANGE = 1,   // block-table entry outside [0, n_pages)
     ERR_CAPACITY = 2,     // position beyond the block-table row / max_context
     ERR_WAIT_TIMEOUT = 4, // a bounded mbarrier wait gave up
+    ERR_PEER_TIMEOUT = 8, // a bounded wait for another rank's partial sums gave up
 };
 
 template <typename T> __device__ __forceinline__ float to_f(T v);

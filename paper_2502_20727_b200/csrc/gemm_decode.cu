@@ -16,6 +16,10 @@
 //   EPI_GATEUP : MLP-RMSNorm rstd (per device in an SPD block), SwiGLU                 (a8)
 //   EPI_DOWN   : the kept sync-point (sum over devices = K accumulation over all of F), output
 //                residual, next block's gain-scaled input / final output               (a9, a10)
+//   EPI_RESID_TP : o_proj / down of a rank that holds ONE shard (tensor parallelism across GPUs,
+//                Sec. 3): the cluster adds up the K ranges of the rank's own partial, and the
+//                sum over ranks - where the block keeps that sync-point - is an exchange through
+//                peer-writable memory in the same tail (see TpArgs)
 //
 // Warps 0-3 own the accumulator rows (TMEM lanes) and run the epilogue; while the main loop runs
 // they fetch what the epilogue needs (rstd, page addresses).  Warp 4 issues the TMA loads,
@@ -147,7 +151,8 @@ __device__ __forceinline__ void epilogue_qkv(const DecGemmArgs &g, const DecTile
                                              const float *sm_rstd, const long *sm_kvoff)
 {
     const int r = threadIdx.x, d = g.head_dim, half = d >> 1;
-    const int row = t.w_row0 + r, head = row / d, jd = row % d, nq = g.n_q_heads;
+    // weights batched by shard (rank mode): batch z holds heads z * heads_per_shard ...
+    const int row = t.w_row0 + r, head = row / d + t.z * (g.w_rows[t.wi] / d), jd = row % d, nq = g.n_q_heads;
     const bool row_valid = row < g.w_rows[t.wi];
     const bool rot = t.wi < 2 && g.rope != nullptr;
     // the rotary factors do not depend on the gather: request them first
@@ -276,6 +281,117 @@ __device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const De
     }
 }
 
+__device__ __forceinline__ unsigned ld_acquire_sys(const unsigned *p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_sys(unsigned *p, unsigned v)
+{
+    asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+constexpr unsigned long long PEER_WAIT_NS = 1000000000ull; // one second
+
+// Rank z's partial rows (its K ranges added up through the cluster), optionally exchanged with the
+// other ranks and summed in rank order, then the residual, the gain-scaled input of the next GEMM
+// and its partial sums of squares - all in rank z's own planes.
+template <int BN>
+__device__ __forceinline__ void epilogue_resid_tp(const DecGemmArgs &g, const DecTile &t, const float *S, volatile int *abort_flag)
+{
+    const TpArgs &tp = g.tp;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n = t.w_row0 + 4 * lane, H = g.H;
+    const bool valid = n < H;
+    const long zoff = (long)t.z * tp.z_stride;
+    const int me = tp.rank_base + t.z;
+    const unsigned step = *(const unsigned *)((const char *)tp.step + zoff);
+    const long buf_off = (long)(tp.buf & 1) * tp.buf_bytes;
+    const float4 one = make_float4(1.f, 1.f, 1.f, 1.f);
+    float4 gn = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (valid && g.gain) {
+        const uint2 u = *(const uint2 *)((const bf16 *)g.gain + n);
+        const float2 a = __bfloat1622float2(*(const __nv_bfloat162 *)&u.x), b = __bfloat1622float2(*(const __nv_bfloat162 *)&u.y);
+        gn = make_float4(a.x, a.y, b.x, b.y);
+    }
+    // token m, columns n..n+3: the summed update `tot` joins the rank's residual stream
+    auto finish = [&](int m, float4 tot) {
+        const long idx = (long)m * H + n;
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (valid) {
+            x = *(const float4 *)((const char *)g.res_in + zoff + idx * 4);
+            add4(x, tot);
+            if (g.res_out) *(float4 *)((char *)g.res_out + zoff + idx * 4) = x;
+            if (g.final_out) store_bf16x4((bf16 *)((char *)g.final_out + (long)t.z * tp.out_stride) + idx, x, one);
+            if (g.hg) store_bf16x4((bf16 *)((char *)g.hg + zoff) + idx, x, gn);
+        }
+        if (g.ss_out) {
+            const float sq = warp_sum(valid ? sq4(x) : 0.f);
+            if (lane == 0) ((float *)((char *)g.ss_out + zoff))[(long)t.wt * g.Mcap + m] = sq;
+        }
+    };
+    for (int q = warp;; q += 4) {
+        const int j = t.rank + t.P * q, m = t.t_row0 + j;
+        if (j >= BN || m >= g.t_rows) break;
+        const long idx = (long)m * H + n;
+        float4 y[MAX_P];
+        load_partials(y, S, j, lane, t.P);
+        float4 p = y[0];
+#pragma unroll
+        for (int s = 1; s < MAX_P; ++s)
+            if (s < t.P) add4(p, y[s]);
+        if (valid) {
+            if (tp.addend) add4(p, *(const float4 *)((const char *)tp.addend + zoff + idx * 4));
+            if (tp.ysave) *(float4 *)((char *)tp.ysave + zoff + idx * 4) = p;
+            if (tp.exchange)
+                for (int i = 0; i < tp.T; ++i) { // own rank first, then the peers round the ring: no two ranks aim at one peer at once
+                    const int r = me + i < tp.T ? me + i : me + i - tp.T;
+                    *(float4 *)(tp.rx[r] + buf_off + (long)me * tp.src_bytes + idx * 4) = p;
+                }
+        }
+        if (!tp.exchange) finish(m, p);
+    }
+    if (!tp.exchange) return;
+    // every row of this block is on its way: publish the step on every rank, then wait for all sources
+    epi_sync();
+    const long tile_flags = ((long)t.wt * gridDim.y + blockIdx.y) * tp.T * TP_FLAG_RANGES;
+    if ((int)threadIdx.x < tp.T) { // the release orders the block's rows (made visible to this thread by the barrier) before the flag
+        st_release_sys(tp.flags[threadIdx.x] + tile_flags + me * TP_FLAG_RANGES + t.rank, step);
+    }
+    if (warp == 0) {
+        const unsigned *mine = tp.flags[me] + tile_flags;
+        const unsigned long long t0 = global_ns();
+        for (;;) {
+            bool done = true;
+            for (int e = lane; e < tp.T * TP_FLAG_RANGES; e += 32)
+                if (e % TP_FLAG_RANGES < t.P && (int)(ld_acquire_sys(mine + e) - step) < 0) done = false;
+            if (__all_sync(0xffffffffu, done)) break;
+            // a rank that never arrives (or an earlier give-up in this step) ends the wait: no trap, the host reads the flag
+            if (*abort_flag || (*(volatile int *)g.err & ERR_PEER_TIMEOUT) || global_ns() - t0 > PEER_WAIT_NS) {
+                if (lane == 0) { *abort_flag = 1; atomicOr(g.err, ERR_PEER_TIMEOUT); }
+                break;
+            }
+        }
+    }
+    epi_sync();
+    if (*abort_flag) return;
+    for (int q = warp;; q += 4) {
+        const int j = t.rank + t.P * q, m = t.t_row0 + j;
+        if (j >= BN || m >= g.t_rows) break;
+        float4 tot = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (valid)
+            for (int r = 0; r < tp.T; ++r)
+                add4(tot, __ldcg((const float4 *)(tp.rx[me] + buf_off + (long)r * tp.src_bytes + ((long)m * H + n) * 4)));
+        finish(m, tot);
+    }
+}
+
 template <int BN, int EPI>
 __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_w0,
                                                               const __grid_constant__ CUtensorMap tm_w1,
@@ -397,8 +513,11 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
     } else {
         // epilogue warps: fetch what the tail needs while the weights stream
         pdl_wait();
-        if (EPI == EPI_QKV || EPI == EPI_GATEUP)
-            compute_rstd<BN>(g.ss_in, (EPI == EPI_GATEUP && g.rstd_per_shard) ? t.z : 0, t.t_row0, g.t_rows, sm_red, sm_rstd);
+        if (EPI == EPI_QKV || EPI == EPI_GATEUP) {
+            SumSq ss = g.ss_in;
+            if (g.tp.on) ss.part = (const float *)((const char *)ss.part + (long)t.z * g.tp.z_stride); // rank z's own sums
+            compute_rstd<BN>(ss, (EPI == EPI_GATEUP && g.rstd_per_shard && !g.tp.on) ? t.z : 0, t.t_row0, g.t_rows, sm_red, sm_rstd);
+        }
         if (EPI == EPI_QKV && t.wi > 0 && threadIdx.x < BN) {
             // where this token's K / V row of kv head 0 goes; < 0: skip (the error flag says why)
             const int m = t.t_row0 + threadIdx.x;
@@ -450,6 +569,7 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
         float *Gb = (float *)gen_base + BN * 128; // this block's gathered tokens
         if (EPI == EPI_QKV) epilogue_qkv<BN>(g, t, S, Gb, sm_rstd, sm_kvoff);
         else if (EPI == EPI_GATEUP) epilogue_gateup<BN>(g, t, S, Gb, sm_rstd);
+        else if (EPI == EPI_RESID_TP) epilogue_resid_tp<BN>(g, t, S, abort_flag);
         else epilogue_residual<BN>(g, t, S, EPI == EPI_OPROJ && g.n_groups > 1);
         if (threadIdx.x == 0) SPD_TRACE_EVENT(EPI, TR_END);
     }
@@ -484,6 +604,30 @@ cudaError_t launch_cfg(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
     at[1].val.clusterDim.z = (unsigned)L.P;
     cfg.attrs = at;
     cfg.numAttrs = L.P > 1 ? 2 : 1;
+    if (EPI == EPI_RESID_TP && L.g.tp.exchange && L.g.batches > 1) {
+        // Several ranks in one launch: their blocks wait on one another, so all of them must be resident at once.
+        // Blocks per SM from the kernel's own footprint (the launch takes the largest shared-memory carveout, which
+        // the occupancy query does not assume), clusters per GPU scaled from the query's answer.
+        cudaLaunchConfig_t occ = cfg;
+        occ.numAttrs = 2;
+        int clusters = 0, api_per_sm = 0, dev = 0, smem_sm = 0, smem_rsv = 0, regs_sm = 0;
+        cudaFuncAttributes fa;
+        cudaError_t e = cudaOccupancyMaxActiveClusters(&clusters, gemm_decode_kernel<BN, EPI>, &occ);
+        if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&api_per_sm, gemm_decode_kernel<BN, EPI>, THREADS, C::SMEM_BYTES);
+        if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, gemm_decode_kernel<BN, EPI>);
+        if (e == cudaSuccess) e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&smem_rsv, cudaDevAttrReservedSharedMemoryPerBlock, dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&regs_sm, cudaDevAttrMaxRegistersPerMultiprocessor, dev);
+        if (e != cudaSuccess) return e;
+        const long by_smem = smem_sm / (long)(C::SMEM_BYTES + fa.sharedSizeBytes + smem_rsv);
+        const long by_regs = regs_sm / (long)(((fa.numRegs + 7) / 8 * 8) * THREADS);
+        long per_sm = by_smem < by_regs ? by_smem : by_regs;
+        if (per_sm > 2048 / THREADS) per_sm = 2048 / THREADS;
+        if (api_per_sm < 1 || per_sm < api_per_sm) per_sm = api_per_sm < 1 ? 0 : api_per_sm;
+        const long capacity = api_per_sm < 1 ? 0 : (long)clusters * per_sm / api_per_sm;
+        if ((long)grid.x * grid.y > capacity) return cudaErrorCooperativeLaunchTooLarge;
+    }
     return cudaLaunchKernelEx(&cfg, gemm_decode_kernel<BN, EPI>, *tw[0], *tw[1], *tw[2], tt, L);
 }
 
@@ -500,6 +644,7 @@ cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
 }
 
 // One thread block per 128 columns, all tokens: the same outputs EPI_DOWN leaves for the next block.
+// Rank mode: blockIdx.y = local rank, whose planes lie z_stride bytes apart and whose step number advances here.
 __global__ void __launch_bounds__(128) decode_prologue_kernel(PrologueArgs a, int h_tiles, double log_base)
 {
     pdl_launch_dependents();
@@ -507,7 +652,7 @@ __global__ void __launch_bounds__(128) decode_prologue_kernel(PrologueArgs a, in
     if ((int)blockIdx.x >= h_tiles) {
         // rotary table of this step, evaluated in double and shared by all blocks of the stack
         const int half = a.head_dim / 2, i = ((int)blockIdx.x - h_tiles) * 128 + threadIdx.x;
-        if (i >= a.M * half) return;
+        if (blockIdx.y != 0 || i >= a.M * half) return;
         int m = i / half, j = i % half, b, pos;
         a.tm.locate(m, b, pos);
         const double theta = exp(-2.0 * (double)j / (double)a.head_dim * log_base);
@@ -517,6 +662,10 @@ __global__ void __launch_bounds__(128) decode_prologue_kernel(PrologueArgs a, in
         return;
     }
     __shared__ float sm[4];
+    const long zoff = (long)blockIdx.y * a.z_stride;
+    float *res_out = (float *)((char *)a.res_out + zoff), *ss_out = (float *)((char *)a.ss_out + zoff);
+    bf16 *hg = (bf16 *)((char *)a.hg + zoff);
+    if (a.step && blockIdx.x == 0 && threadIdx.x == 0) *(unsigned *)((char *)a.step + zoff) += 1u;
     const int r = threadIdx.x, warp = r >> 5, lane = r & 31, n = blockIdx.x * 128 + r;
     const bool valid = n < a.H;
     const float gn = valid ? __bfloat162float(((const bf16 *)a.gain)[n]) : 0.f;
@@ -524,14 +673,14 @@ __global__ void __launch_bounds__(128) decode_prologue_kernel(PrologueArgs a, in
         const long idx = (long)m * a.H + n;
         const float x = valid ? __bfloat162float(((const bf16 *)a.x)[idx]) : 0.f;
         if (valid) {
-            a.res_out[idx] = x;
-            ((bf16 *)a.hg)[idx] = __float2bfloat16_rn(x * gn);
+            res_out[idx] = x;
+            hg[idx] = __float2bfloat16_rn(x * gn);
         }
         const float q = warp_sum(x * x);
         __syncthreads();
         if (lane == 0) sm[warp] = q;
         __syncthreads();
-        if (r == 0) a.ss_out[(long)blockIdx.x * a.Mcap + m] = sm[0] + sm[1] + sm[2] + sm[3];
+        if (r == 0) ss_out[(long)blockIdx.x * a.Mcap + m] = sm[0] + sm[1] + sm[2] + sm[3];
     }
 }
 
@@ -556,6 +705,9 @@ cudaError_t launch_gemm_decode(DecEpilogue epi, const TcMap *const *weights, con
     if (P > MAX_P) return cudaErrorInvalidValue;
     if (epi == EPI_OPROJ && g.n_groups > 1 && (g.n_groups != g.batches || !g.z_is_plane)) return cudaErrorInvalidValue;
     if (epi == EPI_QKV && (BM % g.head_dim) != 0) return cudaErrorInvalidValue;
+    if (epi == EPI_RESID_TP && (!g.tp.on || g.z_is_plane || g.tp.T < 1 || g.tp.T > TP_MAX_RANKS || P > TP_FLAG_RANGES ||
+                                g.tp.rank_base < 0 || g.tp.rank_base + g.batches > g.tp.T || !g.tp.step || !g.res_in))
+        return cudaErrorInvalidValue;
     const CUtensorMap *tw[3];
     for (int i = 0; i < 3; ++i) tw[i] = (const CUtensorMap *)weights[i < nw ? i : 0];
     const CUtensorMap &tt = *(const CUtensorMap *)&tokens;
@@ -582,6 +734,7 @@ cudaError_t launch_gemm_decode(DecEpilogue epi, const TcMap *const *weights, con
     case EPI_QKV: return launch_epi<EPI_QKV>(tw, tt, L, tiles, st);
     case EPI_OPROJ: return launch_epi<EPI_OPROJ>(tw, tt, L, tiles, st);
     case EPI_GATEUP: return launch_epi<EPI_GATEUP>(tw, tt, L, tiles, st);
+    case EPI_RESID_TP: return launch_epi<EPI_RESID_TP>(tw, tt, L, tiles, st);
     default: return launch_epi<EPI_DOWN>(tw, tt, L, tiles, st);
     }
 }
@@ -591,7 +744,7 @@ cudaError_t launch_decode_prologue(const PrologueArgs &a, cudaStream_t st)
     if (a.M <= 0) return cudaSuccess;
     const int h_tiles = (a.H + 127) / 128;
     const int table_blocks = a.rope_table ? (a.M * (a.head_dim / 2) + 127) / 128 : 0;
-    return launch_kernel(decode_prologue_kernel, dim3(h_tiles + table_blocks), dim3(128), 0, st, 0, a, h_tiles,
+    return launch_kernel(decode_prologue_kernel, dim3(h_tiles + table_blocks, a.n_z > 1 ? a.n_z : 1), dim3(128), 0, st, 0, a, h_tiles,
                          a.rope_table ? log((double)a.rope_base) : 0.0);
 }
 

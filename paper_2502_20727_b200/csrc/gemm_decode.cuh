@@ -13,6 +13,36 @@ enum DecEpilogue {
     EPI_OPROJ = 1, // a5-a7: Y_i, residual add(s), gain-scaled MLP inputs and their row sums of squares
     EPI_GATEUP = 2,// a8: rstd of the MLP RMSNorm, SwiGLU
     EPI_DOWN = 3,  // a9 + a10: shard sum (the K accumulation), output residual, next block's norm input
+    EPI_RESID_TP = 4, // o_proj / down of a rank that holds one shard: the shard sum is an exchange with the other ranks
+};
+
+constexpr int TP_MAX_RANKS = 8;
+constexpr int TP_FLAG_RANGES = 8; // flag words per (tile, source rank): one per K range of the source's cluster
+
+// Tensor-parallel execution proper (Sec. 3): every rank of the group holds one shard and owns a
+// region of device memory that its peers can write.  Batch z of a launch is local rank z (one per
+// launch on a real group; all T when one GPU executes every rank), and every rank-private pointer
+// of the launch is that of local rank 0, rank z's lying z_stride bytes further on.
+//
+// A shard sum (sync-point) is a one-shot exchange folded into the tail of the projection whose
+// output it adds up: each rank writes its fp32 partial rows into every rank's receive planes
+// (plane = source rank), publishes the step number in one flag word per (tile, source, K range)
+// on every rank, waits - with a time limit - until its own flags show this step for all sources,
+// and adds the T planes in rank order, so that all ranks hold bit-identical sums.  Two receive
+// buffers alternate between consecutive exchanges; kernel boundaries order their reuse.
+struct TpArgs {
+    int on;                // 0: not a rank-mode launch
+    int T, rank_base;      // group size; group rank of local rank 0
+    long z_stride;         // bytes between the regions of consecutive local ranks
+    long out_stride;       // bytes between the final outputs of consecutive local ranks
+    int exchange;          // 1: the partial rows are summed over the group; 0: they stay local (SPD o_proj)
+    int buf;               // receive buffer (0 / 1) of this exchange; consecutive exchanges alternate
+    long buf_bytes, src_bytes; // one receive buffer ([T][Mcap][H] fp32); one source plane of it
+    char *rx[TP_MAX_RANKS];        // rank j's receive buffers (buffer 0 first)
+    unsigned *flags[TP_MAX_RANKS]; // rank j's flag words of this exchange: [tile][token tile][source][TP_FLAG_RANGES]
+    const unsigned *step;  // step number (> 0, same on all ranks)
+    const float *addend;   // fp32 [Mcap][H] added to the partial before the exchange (Y_i of an SPD block), or null
+    float *ysave;          // fp32 [Mcap][H]: the partial is kept here (Y_i), or null
 };
 
 // RMSNorm is split in two: the producer of a residual stream stores x * gain (bf16, the
@@ -62,6 +92,7 @@ struct DecGemmArgs {
     // GATEUP
     void *act;             // bf16 [tokens][F]
     int F, Fs;
+    TpArgs tp;
 };
 
 // Tensor maps: weights with 128-row boxes (64-row boxes for EPI_GATEUP: gate and up rows of the
@@ -86,6 +117,10 @@ struct PrologueArgs {
     TokMap tm;
     int head_dim;
     float rope_base;
+    // rank mode: n_z local ranks, whose res_out / hg / ss_out / step lie z_stride bytes apart; step (or null) is advanced by one
+    int n_z;
+    long z_stride;
+    unsigned *step;
 };
 cudaError_t launch_decode_prologue(const PrologueArgs &a, cudaStream_t st);
 

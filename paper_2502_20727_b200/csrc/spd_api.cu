@@ -64,13 +64,34 @@ struct GraphKey {
     const int32_t *seq_lens, *block_table;
     void *out;
     int B, max_pages, ctx_bucket;
+    int mode; // 0: spd_decode_step; rank mode: 1 + receive buffer of the step's first exchange
     bool operator==(const GraphKey &o) const
     {
         return x == o.x && seq_lens == o.seq_lens && block_table == o.block_table && out == o.out && B == o.B &&
-               max_pages == o.max_pages && ctx_bucket == o.ctx_bucket;
+               max_pages == o.max_pages && ctx_bucket == o.ctx_bucket && mode == o.mode;
     }
 };
 struct GraphEntry { GraphKey key; cudaGraphExec_t exec; unsigned long long last_use; int launches; };
+
+// One rank's region of a tensor-parallel group (offsets in bytes; every rank uses the same layout).
+struct TpLayout {
+    size_t flags, rx, res0, res1, ysave, hg, ss_attn, ss_mlp, step, total;
+    size_t site_flags; // flag words of one (layer, exchange site)
+    size_t buf_bytes, src_bytes;
+    long Mb;           // token capacity (max_batch)
+    int tok_tiles;
+};
+
+struct TpState {
+    bool on;
+    int T, rank_base;
+    long z_stride;
+    unsigned long long exchanges; // exchanges launched since the attach (the same number on every rank)
+    TpLayout L;
+    char *regions[TP_MAX_RANKS];
+    std::vector<TcMap> qkv_maps; // per layer: wq, wk, wv with one batch per local shard
+    TcMap h_maps[3];             // the local ranks' gain-scaled inputs, token boxes 16 / 32 / 64
+};
 
 struct Ctx {
     spd_dims d;
@@ -94,6 +115,7 @@ struct Ctx {
     int split_override[SITE_COUNT];
     int l2_prefetch_kb;          // K blocks per thread block prefetched into L2 by the decode GEMMs
     int launches_last;
+    TpState tp;
     // activation tensor maps, by buffer and token box (16, 32, 64, 128), built on first use
     TcMap act_maps[AB_COUNT][4];
     bool act_map_ready[AB_COUNT][4];
@@ -236,6 +258,30 @@ Layout make_layout(const spd_dims &d, bool any_spd)
     const size_t h_tiles = (H + 127) / 128;
     L.ss_attn = take(h_tiles * Mmax * 4);
     L.ss_mlp = take(h_tiles * T * Mmax * 4);
+    L.total = off;
+    return L;
+}
+
+TpLayout tp_layout(const spd_dims &d, int T)
+{
+    TpLayout L{};
+    const size_t H = d.hidden, h_tiles = (H + 127) / 128;
+    L.Mb = d.max_batch;
+    L.tok_tiles = (d.max_batch + 15) / 16; // an upper bound for every token box
+    L.site_flags = h_tiles * L.tok_tiles * T * TP_FLAG_RANGES;
+    L.src_bytes = (size_t)L.Mb * H * 4;
+    L.buf_bytes = L.src_bytes * T;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
+    L.step = take(256);
+    L.flags = take((size_t)d.n_layers * 2 * L.site_flags * 4);
+    L.rx = take(2 * L.buf_bytes);
+    L.res0 = take(L.src_bytes);
+    L.res1 = take(L.src_bytes);
+    L.ysave = take(L.src_bytes);
+    L.hg = take((size_t)L.Mb * H * 2);
+    L.ss_attn = take(h_tiles * L.Mb * 4);
+    L.ss_mlp = take(h_tiles * L.Mb * 4);
     L.total = off;
     return L;
 }
@@ -549,6 +595,122 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
     return SPD_OK;
 }
 
+// One decode step in rank mode (tensor parallelism across GPUs, Sec. 3): every local rank runs
+// the block on its own shard and its own copy of the residual stream; the shard sums that the
+// block keeps (o_proj of a TP block, down of every block; Sec. 4.1.1) are exchanges with the
+// other ranks of the group inside the projection's tail.  out: [local ranks][M][H].
+int run_decode_tp(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t *bt, int max_pages,
+                  int max_context, cudaStream_t st)
+{
+    const spd_dims &d = c->d;
+    TpState &tp = c->tp;
+    const TpLayout &TL = tp.L;
+    const int H = d.hidden, qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, F = d.ffn, nl = d.T;
+    const int Fs = F / nl;
+    const long Mb = TL.Mb;
+    const Plan p = make_plan(d, M, true, max_context, c->split_override[SITE_ATTN]);
+    PageTable pt{bt, max_pages, c->n_pages, d.kv_block_size, d.n_kv_heads};
+    const int tbox = tc_token_box(true, M);
+    const int tok_tiles = cdiv(M, tbox), h_tiles = cdiv(H, 128);
+    if (tok_tiles > TL.tok_tiles) return SPD_EINVAL;
+    const TcMap *hmap = &tp.h_maps[box_index(tbox)];
+    int launches = 0;
+    const bool rope = d.rope_base > 0.f;
+    char *r0 = tp.regions[tp.rank_base];
+    {   // a1 of the first block for every local rank; the ranks' step numbers advance
+        PrologueArgs a{};
+        a.x = x; a.res_out = (float *)(r0 + TL.res0); a.gain = c->layers[0].attn_norm; a.hg = r0 + TL.hg;
+        a.ss_out = (float *)(r0 + TL.ss_attn); a.Mcap = Mb; a.M = M; a.H = H;
+        a.n_z = nl; a.z_stride = tp.z_stride; a.step = (unsigned *)(r0 + TL.step);
+        if (rope) { a.rope_table = c->rope; a.tm = tm; a.head_dim = d.head_dim; a.rope_base = d.rope_base; }
+        LAUNCH(K_NORM, launch_decode_prologue(a, st));
+    }
+    auto base_args = [&]() {
+        DecGemmArgs g{};
+        g.t_rows = M; g.err = c->err; g.H = H; g.Mcap = Mb; g.batches = nl; g.w_batched = 1; g.t_batched = 1;
+        g.n_weights = 1; g.n_groups = 1;
+        g.tp.on = 1; g.tp.T = tp.T; g.tp.rank_base = tp.rank_base; g.tp.z_stride = tp.z_stride;
+        g.tp.step = (const unsigned *)(r0 + TL.step);
+        return g;
+    };
+    int exchange = 0;
+    // the exchange of block l at site s (0: o_proj, 1: down)
+    auto with_exchange = [&](DecGemmArgs &g, int l, int s) {
+        g.tp.exchange = 1;
+        g.tp.buf = (int)((tp.exchanges + exchange++) & 1);
+        g.tp.buf_bytes = (long)TL.buf_bytes; g.tp.src_bytes = (long)TL.src_bytes;
+        for (int j = 0; j < tp.T; ++j) {
+            g.tp.rx[j] = tp.regions[j] + TL.rx;
+            g.tp.flags[j] = (unsigned *)(tp.regions[j] + TL.flags) + ((size_t)l * 2 + s) * TL.site_flags;
+        }
+    };
+    for (int l = 0; l < d.n_layers; ++l) {
+        const spd_layer &w = c->layers[l];
+        const bool sync = c->mask[l] != 0;
+        {   // a2 + a3: rank z projects its own heads from its own copy of the normalised input
+            DecGemmArgs g = base_args();
+            const TcMap *wmaps[3] = {&tp.qkv_maps[3 * l], &tp.qkv_maps[3 * l + 1], &tp.qkv_maps[3 * l + 2]};
+            g.n_weights = 3; g.w_rows[0] = qd / nl; g.w_rows[1] = g.w_rows[2] = kd / nl;
+            g.num_kb = cdiv(H, 64);
+            g.splits = decode_splits((long)decode_tiles_per_batch(EPI_QKV, g.w_rows, 3) * nl * tok_tiles, g.num_kb,
+                                     c->split_override[SITE_QKV], 8);
+            g.ss_in = SumSq{(const float *)(r0 + TL.ss_attn), h_tiles, 1, Mb, H, d.rms_eps};
+            g.rope = rope ? c->rope : nullptr; g.q_out = c->q; g.k_pages = w.k_pages; g.v_pages = w.v_pages; g.pt = pt; g.tm = tm;
+            g.n_q_heads = d.n_q_heads; g.head_dim = d.head_dim;
+            LAUNCH(K_QKV, launch_gemm_decode(EPI_QKV, wmaps, *hmap, g, st));
+        }
+        {   // a4: heads are rank-local by construction
+            AttnArgs a{};
+            a.q = c->q; a.k_pages = w.k_pages; a.v_pages = w.v_pages; a.pt = pt; a.tm = tm; a.out = c->attn;
+            a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.B = M; a.splits = p.attn_splits;
+            a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.counters = c->attn_cnt; a.err = c->err;
+            if (d.head_dim == 128 && d.kv_block_size == 16) { a.k_map = &c->maps[l].kpages; a.v_map = &c->maps[l].vpages; }
+            LAUNCH(K_ATTN, launch_decode_attention<bf16>(a, st));
+        }
+        {   // a5 - a7: Y_z from the rank's own heads.  TP block: R = X + sum over ranks (sync-point 1);
+            // SPD block: the sync-point is dropped, R_z = X + Y_z feeds the rank's MLP and Y_z is kept for a10
+            DecGemmArgs g = base_args();
+            const TcMap *wmaps[1] = {&c->maps[l].wo_shard};
+            MAP_OR_FAIL(am, act_map(c, AB_ATTN_SHARD, tbox));
+            g.w_rows[0] = H;
+            g.num_kb = cdiv(qd / nl, 64);
+            g.splits = decode_splits((long)h_tiles * nl * tok_tiles, g.num_kb, c->split_override[SITE_O], 8);
+            g.res_in = (const float *)(r0 + TL.res0); g.gain = w.mlp_norm; g.hg = r0 + TL.hg; g.ss_out = (float *)(r0 + TL.ss_mlp);
+            if (sync) { with_exchange(g, l, 0); g.res_out = (float *)(r0 + TL.res1); }
+            else g.tp.ysave = (float *)(r0 + TL.ysave);
+            LAUNCH(K_OPROJ, launch_gemm_decode(EPI_RESID_TP, wmaps, *am, g, st));
+        }
+        {   // a8
+            DecGemmArgs g = base_args();
+            const TcMap *wmaps[2] = {&c->maps[l].w_gate64, &c->maps[l].w_up64};
+            g.n_weights = 2; g.w_rows[0] = g.w_rows[1] = Fs;
+            g.num_kb = cdiv(H, 64);
+            g.splits = decode_splits((long)decode_tiles_per_batch(EPI_GATEUP, g.w_rows, 2) * nl * tok_tiles, g.num_kb,
+                                     c->split_override[SITE_GU], 8);
+            g.ss_in = SumSq{(const float *)(r0 + TL.ss_mlp), h_tiles, 1, Mb, H, d.rms_eps};
+            g.act = c->act; g.F = F; g.Fs = Fs;
+            LAUNCH(K_GATE_UP, launch_gemm_decode(EPI_GATEUP, wmaps, *hmap, g, st));
+        }
+        {   // a9 + a10, the kept sync-point.  TP block: out = R + sum_z Z_z;  SPD block: out = X + sum_z (Y_z + Z_z)
+            DecGemmArgs g = base_args();
+            const TcMap *wmaps[1] = {&c->maps[l].wd_shard};
+            MAP_OR_FAIL(am, act_map(c, AB_ACT_SHARD, tbox));
+            g.w_rows[0] = H;
+            g.num_kb = cdiv(Fs, 64);
+            g.splits = decode_splits((long)h_tiles * nl * tok_tiles, g.num_kb, c->split_override[SITE_DOWN], 8);
+            with_exchange(g, l, 1);
+            g.res_in = (const float *)(r0 + (sync ? TL.res1 : TL.res0));
+            if (!sync) g.tp.addend = (const float *)(r0 + TL.ysave);
+            g.res_out = (float *)(r0 + TL.res0);
+            if (l + 1 < d.n_layers) { g.gain = c->layers[l + 1].attn_norm; g.hg = r0 + TL.hg; g.ss_out = (float *)(r0 + TL.ss_attn); }
+            else { g.final_out = out; g.tp.out_stride = (long)M * H * 2; }
+            LAUNCH(K_DOWN, launch_gemm_decode(EPI_RESID_TP, wmaps, *am, g, st));
+        }
+    }
+    c->launches_last = launches;
+    return SPD_OK;
+}
+
 // Head-grouping measurements (Sec. 4.2.4) taken at one block while a prompt batch runs through the
 // TP blocks before it: attention scores of every head and their pairwise distances (Eq. 2), and the
 // sums of squares of MLP_m(norm(X + Y_i)) for every (device i, MLP partition m) (Eq. 3).
@@ -747,6 +909,45 @@ int build_weight_maps(Ctx &c)
     return SPD_OK;
 }
 
+// Runs a decode step from its captured graph, capturing it first when no graph matches `key`;
+// directly when graphs are off, a profile is being taken or the stream cannot be captured.
+template <typename Run>
+int replay_or_run(Ctx &c, const GraphKey &key, Run run, cudaStream_t st)
+{
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    CU_TRY(cudaStreamIsCapturing(st, &cap));
+    // (the legacy default stream cannot be captured)
+    if (!c.use_graphs || c.profiling || cap != cudaStreamCaptureStatusNone || st == 0 || st == cudaStreamLegacy) return run();
+    GraphEntry *hit = nullptr;
+    for (GraphEntry &e : c.graphs)
+        if (e.key == key) hit = &e;
+    if (!hit) {
+        CU_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+        const int rc = run();
+        cudaGraph_t graph = nullptr;
+        cudaError_t e = cudaStreamEndCapture(st, &graph);
+        if (rc != SPD_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
+        if (e != cudaSuccess) { g_last_cuda_error = (int)e; return SPD_ECUDA; }
+        cudaGraphExec_t exec = nullptr;
+        e = cudaGraphInstantiate(&exec, graph, 0);
+        cudaGraphDestroy(graph);
+        if (e != cudaSuccess) { g_last_cuda_error = (int)e; return SPD_ECUDA; }
+        if (c.graphs.size() >= 8) { // evict the least recently used
+            size_t lru = 0;
+            for (size_t i = 1; i < c.graphs.size(); ++i)
+                if (c.graphs[i].last_use < c.graphs[lru].last_use) lru = i;
+            cudaGraphExecDestroy(c.graphs[lru].exec);
+            c.graphs.erase(c.graphs.begin() + lru);
+        }
+        c.graphs.push_back(GraphEntry{key, exec, 0, c.launches_last});
+        hit = &c.graphs.back();
+    }
+    hit->last_use = ++c.graph_clock;
+    c.launches_last = hit->launches;
+    CU_TRY(cudaGraphLaunch(hit->exec, st));
+    return SPD_OK;
+}
+
 } // namespace
 
 struct spd_ctx { Ctx c; };
@@ -812,6 +1013,7 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     for (int i = 0; i < SITE_COUNT; ++i) c.split_override[i] = 0;
     c.l2_prefetch_kb = 0;
     c.launches_last = 0;
+    c.tp.on = false;
     c.use_graphs = true;
     c.graph_clock = 0;
     c.profiling = false;
@@ -889,40 +1091,8 @@ int spd_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_l
                : d.block_kind == 0 ? run_decode_fused(&c, x, out, B, tm, block_table, max_pages, ctx_bucket, st)
                                    : run_tokens<bf16>(&c, x, out, B, tm, block_table, max_pages, true, ctx_bucket, st);
     };
-    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-    CU_TRY(cudaStreamIsCapturing(st, &cap));
-    // (the legacy default stream cannot be captured)
-    if (!c.use_graphs || c.profiling || cap != cudaStreamCaptureStatusNone || st == 0 || st == cudaStreamLegacy) return run();
-
-    const GraphKey key{x, seq_lens, block_table, out, B, max_pages, ctx_bucket};
-    GraphEntry *hit = nullptr;
-    for (GraphEntry &e : c.graphs)
-        if (e.key == key) hit = &e;
-    if (!hit) {
-        CU_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
-        const int rc = run();
-        cudaGraph_t graph = nullptr;
-        cudaError_t e = cudaStreamEndCapture(st, &graph);
-        if (rc != SPD_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
-        if (e != cudaSuccess) { g_last_cuda_error = (int)e; return SPD_ECUDA; }
-        cudaGraphExec_t exec = nullptr;
-        e = cudaGraphInstantiate(&exec, graph, 0);
-        cudaGraphDestroy(graph);
-        if (e != cudaSuccess) { g_last_cuda_error = (int)e; return SPD_ECUDA; }
-        if (c.graphs.size() >= 8) { // evict the least recently used
-            size_t lru = 0;
-            for (size_t i = 1; i < c.graphs.size(); ++i)
-                if (c.graphs[i].last_use < c.graphs[lru].last_use) lru = i;
-            cudaGraphExecDestroy(c.graphs[lru].exec);
-            c.graphs.erase(c.graphs.begin() + lru);
-        }
-        c.graphs.push_back(GraphEntry{key, exec, 0, c.launches_last});
-        hit = &c.graphs.back();
-    }
-    hit->last_use = ++c.graph_clock;
-    c.launches_last = hit->launches;
-    CU_TRY(cudaGraphLaunch(hit->exec, st));
-    return SPD_OK;
+    const GraphKey key{x, seq_lens, block_table, out, B, max_pages, ctx_bucket, 0};
+    return replay_or_run(c, key, run, st);
 }
 
 static void drop_graphs(Ctx &c)
@@ -1023,6 +1193,89 @@ int spd_set_tuning(spd_ctx *ctx, const char *key, int32_t value)
     if (!found) return SPD_EINVAL;
     for (GraphEntry &g : c.graphs) cudaGraphExecDestroy(g.exec); // captured steps used the old setting
     c.graphs.clear();
+    return SPD_OK;
+}
+
+int spd_tp_region_bytes(const spd_ctx *ctx, int32_t T, size_t *out_bytes)
+{
+    if (!ctx || !out_bytes) return SPD_ENULL;
+    if (T < 1 || T > TP_MAX_RANKS) return SPD_EINVAL;
+    *out_bytes = tp_layout(ctx->c.d, T).total;
+    return SPD_OK;
+}
+
+int spd_tp_attach(spd_ctx *ctx, int32_t T, int32_t rank_base, void *const *regions, size_t region_bytes, void *stream)
+{
+    if (!ctx || !regions) return SPD_ENULL;
+    Ctx &c = ctx->c;
+    const spd_dims &d = c.d;
+    const int nl = d.T;
+    if (T < 1 || T > TP_MAX_RANKS || rank_base < 0 || rank_base + nl > T) return SPD_EINVAL;
+    if (!(nl == 1 || (nl == T && rank_base == 0))) return SPD_EINVAL;
+    if (d.dtype != 1 || d.block_kind != 0 || d.hidden % 16 != 0 || 128 % d.head_dim != 0) return SPD_EINVAL;
+    if ((d.n_q_heads / nl) * d.head_dim % 8 != 0) return SPD_EINVAL;
+    const TpLayout TL = tp_layout(d, T);
+    if (region_bytes < TL.total) return SPD_EWORKSPACE;
+    for (int j = 0; j < T; ++j) {
+        if (!regions[j]) return SPD_ENULL;
+        if ((uintptr_t)regions[j] & 1023) return SPD_EWORKSPACE;
+    }
+    const long z_stride = nl > 1 ? (long)((char *)regions[rank_base + 1] - (char *)regions[rank_base]) : 0;
+    for (int z = 1; z < nl; ++z)
+        if ((char *)regions[rank_base + z] - (char *)regions[rank_base] != z * z_stride) return SPD_EINVAL;
+    if (nl > 1 && (z_stride < (long)TL.total || (z_stride & 1023))) return SPD_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    TpState &tp = c.tp;
+    tp.on = false;
+    tp.T = T; tp.rank_base = rank_base; tp.z_stride = z_stride; tp.L = TL; tp.exchanges = 0;
+    for (int j = 0; j < T; ++j) tp.regions[j] = (char *)regions[j];
+    const long H = d.hidden, qd = (long)d.n_q_heads * d.head_dim, kd = (long)d.n_kv_heads * d.head_dim;
+    tp.qkv_maps.resize((size_t)3 * d.n_layers);
+    int rc = 0;
+    for (int l = 0; l < d.n_layers; ++l) {
+        const spd_layer &w = c.layers[l];
+        rc |= make_operand_map(&tp.qkv_maps[3 * l], w.wq, H, qd / nl, nl, H, (qd / nl) * H, 128);
+        rc |= make_operand_map(&tp.qkv_maps[3 * l + 1], w.wk, H, kd / nl, nl, H, (kd / nl) * H, 128);
+        rc |= make_operand_map(&tp.qkv_maps[3 * l + 2], w.wv, H, kd / nl, nl, H, (kd / nl) * H, 128);
+    }
+    const int boxes[3] = {16, 32, 64};
+    for (int i = 0; i < 3; ++i)
+        rc |= make_operand_map(&tp.h_maps[i], tp.regions[rank_base] + TL.hg, H, TL.Mb, nl, H, nl > 1 ? z_stride / 2 : TL.Mb * H, boxes[i]);
+    if (rc) return SPD_EINVAL;
+    // the local ranks' regions start from zero: step 0, no flag set, token rows beyond a batch read as zero
+    for (int z = 0; z < nl; ++z) CU_TRY(cudaMemsetAsync(tp.regions[rank_base + z], 0, TL.total, st));
+    drop_graphs(c);
+    tp.on = true;
+    return SPD_OK;
+}
+
+int spd_tp_detach(spd_ctx *ctx)
+{
+    if (!ctx) return SPD_ENULL;
+    ctx->c.tp.on = false;
+    return SPD_OK;
+}
+
+int spd_tp_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_lens, const int32_t *block_table,
+                       int32_t max_pages, int32_t max_context, void *out, void *stream)
+{
+    if (!ctx || !x || !seq_lens || !block_table || !out) return SPD_ENULL;
+    Ctx &c = ctx->c;
+    const spd_dims &d = c.d;
+    if (!c.tp.on) return SPD_EINVAL;
+    if (B < 1 || B > d.max_batch || x == out || max_context < 1) return SPD_EINVAL;
+    if (max_context > d.max_seq_len || (long)max_pages * d.kv_block_size < max_context) return SPD_ECAPACITY;
+    TokMap tm{1, 0, 1, 0, seq_lens};
+    int ctx_bucket = (max_context + 255) / 256 * 256;
+    if (ctx_bucket > d.max_seq_len) ctx_bucket = d.max_seq_len;
+    if ((long)ctx_bucket > (long)max_pages * d.kv_block_size) ctx_bucket = max_pages * d.kv_block_size;
+    cudaStream_t st = (cudaStream_t)stream;
+    // A captured step is valid for one receive-buffer phase: consecutive exchanges alternate between the
+    // two buffers, so a stack with an odd number of exchanges per step needs one graph per phase.
+    const GraphKey key{x, seq_lens, block_table, out, B, max_pages, ctx_bucket, 1 + (int)(c.tp.exchanges & 1)};
+    const int rc = replay_or_run(c, key, [&]() { return run_decode_tp(&c, x, out, B, tm, block_table, max_pages, ctx_bucket, st); }, st);
+    if (rc != SPD_OK) return rc;
+    for (int l = 0; l < d.n_layers; ++l) c.tp.exchanges += c.mask[l] ? 2 : 1; // the same on every rank of the group
     return SPD_OK;
 }
 

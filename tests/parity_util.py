@@ -89,6 +89,23 @@ class Pair:
         self.pos = self.pos + 1
         return to_np(got), ref[:, 0, :]
 
+    def tp_decode(self, t, seed=0):
+        """One decode step in rank mode (the stack attached as all T ranks of a group on this GPU):
+        every rank's output [T, B, H] and the oracle's."""
+        x = si.make_hidden(self.w, (self.B, self.w.hidden), "cpu", seed, 1 + t)
+        ref, _ = self._oracle(to_np(x)[:, None, :])
+        # fixed device buffers: later steps replay the captured graphs (one per receive-buffer phase)
+        if not hasattr(self, "tp_x"):
+            self.tp_x = torch.empty((self.B, self.w.hidden), dtype=self.w.torch_dtype, device=self.device)
+            self.tp_seq = torch.empty(self.B, dtype=torch.int32, device=self.device)
+            self.tp_out = torch.empty((self.w.T, self.B, self.w.hidden), dtype=self.w.torch_dtype, device=self.device)
+        self.tp_x.copy_(x)
+        self.tp_seq.copy_(torch.from_numpy(self.pos.copy()))
+        got = self.stack.tp_decode_step(self.tp_x, self.tp_seq, self.block_table, int(self.pos.max()) + 1, self.tp_out)
+        torch.cuda.synchronize()
+        self.pos = self.pos + 1
+        return to_np(got), ref[:, 0, :]
+
     def fill_cache(self, lens, seed=0):
         """Put the same synthetic K/V (N(0,1), storage dtype) into the GPU pages and the oracle's
         cache for positions [0, lens[b]) of every sequence and layer."""

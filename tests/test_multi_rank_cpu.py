@@ -1,5 +1,7 @@
 """N > 1 on CPU: two gloo ranks run the rank plumbing of bench.py (replicas only: no collective on the
-data path, timing = max over ranks, rank 0 prints the one line)."""
+data path, timing = max over ranks, rank 0 prints the one line), and the shard / exchange logic of
+tensor parallelism across ranks (one shard per rank, partial sums exchanged where the block keeps
+its sync-points)."""
 import json
 import os
 import socket
@@ -43,3 +45,17 @@ def test_reference_arm_prints_one_line_under_torchrun():
     res = json.loads(lines[0])
     assert res["impl"] == "reference" and res["n_gpus"] == 2 and res["value"] > 0
     assert res["cpu_baseline"]["kind"] == "oracle" and res["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_two_ranks_hold_one_shard_each_and_exchange_partial_sums():
+    """Sec. 3 / Sec. 4.1.1 across real ranks: shard r from shard_layer, the block's kept sync-points as
+    all-reduces - the result equals the oracle's sharded block, with 2 exchanges (TP) or 1 (SPD)."""
+    out = torchrun([os.path.join(ROOT, "tests", "tp_rank_worker.py")])
+    lines = [l for l in out.splitlines() if l.startswith("WORKER ")]
+    assert len(lines) == 1
+    res = json.loads(lines[0][7:])
+    assert res["world"] == 2
+    for r in res["ranks"]:
+        assert r["spd"]["err"] < 1e-12 and r["sync"]["err"] < 1e-12
+        assert r["spd"]["exchanges"] == 1 == r["spd"]["syncs"]
+        assert r["sync"]["exchanges"] == 2 == r["sync"]["syncs"]

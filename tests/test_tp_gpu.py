@@ -1,0 +1,119 @@
+"""GPU parity of the rank-mode decode step (tensor parallelism across GPUs, Sec. 3 / Sec. 4.1.1):
+all T ranks of a group executed on one GPU - every launch covers all ranks' data, and the shard
+sums are exchanges through per-rank receive planes and arrival flags in global memory, the same
+kernels and protocol a group of T GPUs runs over peer-mapped memory - against the CPU oracle's
+sharded block, element by element.  Bound: max|gpu-ref|/max|ref| <= 2e-2 (bfloat16)."""
+import numpy as np
+import pytest
+import torch
+
+import spd_inputs as si
+from parity_util import TOL, Pair, rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+def run_tp_case(w, mask, B, lens, steps):
+    p = Pair(w, mask=mask, B=B, max_len=int(max(lens)) + steps + 1)
+    p.fill_cache(np.asarray(lens, dtype=np.int32))
+    p.stack.tp_attach_local()
+    torch.cuda.synchronize()
+    for t in range(steps):
+        got, ref = p.tp_decode(t)
+        assert got.shape == (w.T,) + ref.shape
+        for r in range(w.T):
+            e = rel_err(got[r], ref)
+            assert e <= TOL["bf16"], f"step {t} rank {r}: rel err {e}"
+        # every rank adds the same planes in the same order: the copies are bit-identical
+        for r in range(1, w.T):
+            assert np.array_equal(got[r], got[0]), f"step {t}: rank {r} differs from rank 0"
+    assert p.stack.device_error() == 0
+    return p
+
+
+@pytest.mark.parametrize("mask", [(0, 0), (1, 1), (0, 1, 0)])
+@pytest.mark.parametrize("T", [2, 4])
+def test_rank_mode_small(T, mask):
+    """Ragged contexts over page boundaries, FFN/T not a tile multiple, GQA 8/4, mixed masks."""
+    w = si.Workload("tp_small", "bf16", len(mask), 512, 8, 4, 64, 1376, T, mask, 3, 37, 3)
+    p = run_tp_case(w, mask, 3, [37, 5, 16], 5)   # (0, 1, 0): 4 exchanges a step; (0, 0): 2; (1, 1): 4
+    p.stack.close()
+
+
+def test_rank_mode_odd_number_of_exchanges_alternates_two_graphs():
+    """One SPD block = one exchange a step: consecutive steps use the two receive buffers in turn, each
+    phase replaying its own captured graph."""
+    mask = (0,)
+    w = si.Workload("tp_odd", "bf16", 1, 512, 8, 4, 64, 1376, 4, mask, 3, 37, 3)
+    p = run_tp_case(w, mask, 3, [20, 5, 16], 6)
+    p.stack.close()
+
+
+def test_rank_mode_eight_ranks_head_dim_128():
+    """T = 8 at head_dim 128 (tensor-core decode attention for the GQA group of 4), batch 5."""
+    mask = (1, 0)
+    w = si.Workload("tp8", "bf16", 2, 1024, 32, 8, 128, 2048, 8, mask, 5, 70, 2)
+    p = run_tp_case(w, mask, 5, [70, 1, 33, 64, 17], 2)
+    p.stack.close()
+
+
+def test_rank_mode_matches_the_single_launch_emulation():
+    """The same stack through spd_decode_step (shards as one cluster per tile) and through the rank-mode
+    step: two implementations of one function, equal to rounding."""
+    mask = (0, 1)
+    w = si.Workload("tp_vs", "bf16", 2, 1024, 16, 16, 64, 2752, 4, mask, 4, 50, 2)
+    p = Pair(w, mask=mask, B=4, max_len=64)
+    lens = np.array([50, 3, 31, 48], dtype=np.int32)
+    p.fill_cache(lens)
+    x = si.make_hidden(w, (4, w.hidden), "cpu", 0, 1).to("cuda:0")
+    seq = torch.from_numpy(lens.copy()).to("cuda:0")
+    a = p.stack.decode_step(x, seq, p.block_table, 51).float().cpu().numpy()
+    # the step appended K/V at position lens[b]; the rank-mode step rewrites the same slots
+    p.stack.tp_attach_local()
+    b = p.stack.tp_decode_step(x, seq, p.block_table, 51).float().cpu().numpy()
+    torch.cuda.synchronize()
+    assert rel_err(b[0], a) <= 1e-2
+    assert p.stack.device_error() == 0
+    p.stack.close()
+
+
+def test_configs1_shape_one_layer_all_ranks():
+    """configs[1] dims (hidden 4096, 32 heads x 128, FFN 11008, T = 8), one TP and one SPD layer, batch 8 on a
+    synthetic cache: 256 thread blocks per exchange launch, all resident at once."""
+    mask = (1, 0)
+    w = si.WORKLOADS["c2"].with_(n_layers=2, mask=mask)
+    p = run_tp_case(w, mask, 8, [200, 17, 1, 130, 64, 199, 100, 5], 1)
+    p.stack.close()
+
+
+def test_a_rank_that_never_arrives_is_reported_not_waited_for():
+    """Rank 0 of a group of two whose peer never runs: the wait for the peer's partial sums ends after
+    its time limit, the step returns, the error flag says so, and the context stays usable."""
+    import paper_2502_20727_b200 as spd
+    mask = (0,)
+    full = si.Workload("tp_alone", "bf16", 1, 256, 4, 4, 64, 512, 2, mask, 2, 8, 1)
+    layers = si.make_stack(full, "cpu", 0)
+    shard = [{n: t.to("cuda:0") for n, t in spd.shard_layer(lw, 0, 2).items()} for lw in layers]
+    one = full.with_(n_q_heads=2, n_kv_heads=2, ffn=256, T=1)
+    stream = torch.cuda.Stream(device="cuda:0")
+    torch.cuda.set_stream(stream)
+    stack = spd.stack_from_workload(one, shard, sync_mask=mask, max_batch=2, max_seq_len=16, n_pages=4,
+                                    max_prefill_tokens=64, device="cuda:0")
+    nbytes = (stack.tp_region_bytes(2) + 1023) // 1024 * 1024
+    regions = torch.zeros(2 * nbytes + 1024, dtype=torch.uint8, device="cuda:0")
+    base = (regions.data_ptr() + 1023) // 1024 * 1024
+    stack.tp_attach(2, 0, [base, base + nbytes], nbytes)   # rank 1's region exists, but nobody plays rank 1
+    x = si.make_hidden(one, (2, one.hidden), "cpu", 0, 1).to("cuda:0")
+    seq = torch.zeros(2, dtype=torch.int32, device="cuda:0")
+    bt = torch.tensor([[0], [1]], dtype=torch.int32, device="cuda:0")
+    out = stack.tp_decode_step(x, seq, bt, 1)
+    torch.cuda.synchronize()
+    assert out.shape == (1, 2, 256)
+    assert stack.device_error() & 8
+    # usable afterwards: the ordinary single-GPU step of the shard's stack runs clean
+    stack.tp_detach()
+    y = stack.decode_step(x, seq, bt, 1)
+    torch.cuda.synchronize()
+    assert torch.isfinite(y.float()).all()
+    assert stack.device_error() == 0
+    stack.close()
