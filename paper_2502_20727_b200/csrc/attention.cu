@@ -316,6 +316,7 @@ template <> cudaError_t launch_prefill_attention_tc<bf16>(const AttnArgs &a, cud
     done = false;
     if (a.tm.decode || a.tm.ns <= 0 || a.M % a.tm.ns) return cudaSuccess;
     done = true;
+    if (a.head_dim == 128 && a.pt.block == 16 && a.q_map && a.k_map && a.v_map) return launch_prefill_attention_umma(a, st);
     switch (a.head_dim) {
     case 128: return fa::launch<128>(a, a.M / a.tm.ns, st);
     case 64: return fa::launch<64>(a, a.M / a.tm.ns, st);

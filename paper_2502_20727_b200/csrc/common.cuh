@@ -195,6 +195,8 @@ struct AttnArgs {
     // optional (decode, bf16, head_dim 128, 16-token pages): tensor maps over the K and V pages seen as
     // [n_pages * n_kv_heads * 16 rows][head_dim], box 64 x 16, 128-byte swizzle (host pointers to CUtensorMap)
     const void *k_map, *v_map;
+    // optional (prefill, same conditions): tensor map over q as [tokens][n_q_heads * head_dim], box 64 x 128
+    const void *q_map;
     int cluster_merge;      // set by the launcher: the splits of a (sequence, head tile) are one thread-block cluster
 };
 // Paged decode attention with 16-token pages: query heads per thread block for a GQA group
@@ -205,6 +207,7 @@ inline int decode_heads_per_block(int group) { return group % 4 == 0 ? 4 : (grou
 inline bool decode_uses_mma(int group, int head_dim, int dtype_bf16, int kv_block) { return dtype_bf16 && head_dim == 128 && kv_block == 16 && group % 4 == 0; }
 inline int decode_heads_per_block_mma(int group) { return group % 8 == 0 ? 8 : 4; }
 template <typename T> cudaError_t launch_prefill_attention(const AttnArgs &a, cudaStream_t st);
+cudaError_t launch_prefill_attention_umma(const AttnArgs &a, cudaStream_t st); // attention_prefill_tc.cu
 template <typename T> cudaError_t launch_decode_attention(const AttnArgs &a, cudaStream_t st);
 
 // head grouping measurements (head_grouping.cu)

@@ -50,7 +50,7 @@ int want_splits(long tiles, int cap)
     return (int)(s < 1 ? 1 : s);
 }
 
-enum ActBuf { AB_H = 0, AB_ATTN, AB_ATTN_SHARD, AB_ACT, AB_ACT_SHARD, AB_COUNT };
+enum ActBuf { AB_H = 0, AB_ATTN, AB_ATTN_SHARD, AB_ACT, AB_ACT_SHARD, AB_Q, AB_COUNT };
 enum Kind { K_NORM = 0, K_QKV, K_ROPE_KV, K_ATTN, K_OPROJ, K_GATE_UP, K_SILU_MUL, K_DOWN, K_ROPE_TABLE, K_COUNT };
 enum Site { SITE_QKV = 0, SITE_O, SITE_GU, SITE_DOWN, SITE_ATTN, SITE_COUNT };
 const char *const kind_names[K_COUNT] = {"residual_rmsnorm", "gemm_qkv", "rope_kv_append", "attention", "gemm_o_proj",
@@ -319,6 +319,7 @@ const TcMap *act_map(Ctx *c, ActBuf buf, int box)
     case AB_ATTN_SHARD: rc = make_operand_map(&c->act_maps[buf][bi], c->attn, qd / T, Mc, T, qd, qd / T, box); break;
     case AB_ACT: rc = make_operand_map(&c->act_maps[buf][bi], c->act, F, Mc, 1, F, 0, box); break;
     case AB_ACT_SHARD: rc = make_operand_map(&c->act_maps[buf][bi], c->act, F / T, Mc, T, F, F / T, box); break;
+    case AB_Q: rc = make_operand_map(&c->act_maps[buf][bi], c->q, qd, Mc, 1, qd, 0, box); break;
     default: break;
     }
     if (rc) return nullptr;
@@ -400,6 +401,10 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
             a.q = c->q; a.k_pages = w.k_pages; a.v_pages = w.v_pages; a.pt = pt; a.tm = tm; a.out = c->attn;
             a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.B = M; a.splits = p.attn_splits;
             a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.counters = c->attn_cnt; a.err = c->err;
+            if (!decode && d.dtype == 1 && d.head_dim == 128 && d.kv_block_size == 16) {
+                MAP_OR_FAIL(qm, act_map(c, AB_Q, 128));
+                a.q_map = qm; a.k_map = &c->maps[l].kpages; a.v_map = &c->maps[l].vpages;
+            }
             if (decode) LAUNCH(K_ATTN, launch_decode_attention<T>(a, st));
             else LAUNCH(K_ATTN, launch_prefill_attention<T>(a, st));
         }
@@ -772,6 +777,10 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
             a.q = c->q; a.k_pages = w.k_pages; a.v_pages = w.v_pages; a.pt = pt; a.tm = tm; a.out = c->attn;
             a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.B = M; a.splits = 1;
             a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.counters = c->attn_cnt; a.err = c->err;
+            if (d.head_dim == 128 && d.kv_block_size == 16) {
+                MAP_OR_FAIL(qm, act_map(c, AB_Q, 128));
+                a.q_map = qm; a.k_map = &c->maps[l].kpages; a.v_map = &c->maps[l].vpages;
+            }
             LAUNCH(K_ATTN, launch_prefill_attention<bf16>(a, st));
         }
         int mlp_tiles, mlp_groups;
