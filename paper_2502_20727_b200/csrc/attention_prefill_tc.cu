@@ -7,13 +7,12 @@
 //   P = softmax    warps 0-7: thread = (query row = TMEM lane, half of the tile's 128 columns); the
 //                  two threads of a row exchange their maxima through shared memory; running
 //                  maximum and sums in base 2, P rounded to bf16 into a K-major swizzled tile
-//   O_j = P V      tcgen05.mma with V as the MN-major operand: V pages are [token][dim], i.e.
+//   O += P V       tcgen05.mma with V as the MN-major operand: V pages are [token][dim], i.e.
 //                  rows of the K dimension with the N dimension contiguous, exactly as TMA
-//                  delivers them; a fresh accumulator per tile
-//   O = O * c + O_j  in registers (c = 2^(m_old - m_new)), one tile behind the softmax so that
-//                  the tensor cores work on S of the next tile and on P V of this one meanwhile
-// S and O_j are double-buffered in tensor memory (4 x 128 columns), K and V tiles in two-stage
-// rings (one for K, one for V), P in two buffers.  Warps 8 and 9 issue the TMA loads, warp 10 the MMAs.
+//                  delivers them; O accumulates in tensor memory over all tiles and is rescaled
+//                  there (load, multiply, store) only when the running maximum has grown by
+//                  more than 2^8 since the last rescale; S of the next tile is computed meanwhile
+// S is double-buffered in tensor memory, K and V tiles in two-stage rings (one for K, one for V).  Warps 8 and 9 issue the TMA loads, warp 10 the MMAs.
 // Every wait is bounded.
 #include "common.cuh"
 #include "gemm_tc.cuh"
@@ -31,7 +30,7 @@ constexpr int HALF_TILE = 128 * 64 * 2;           // [128 rows][64 bf16]: one sw
 constexpr int TILE = 2 * HALF_TILE;               // 128 x 128 bf16
 constexpr int OFF_Q = 0, OFF_KV = TILE, OFF_P = OFF_KV + 2 * 2 * TILE, OFF_RED = OFF_P + TILE, OFF_BAR = OFF_RED + 4096;
 constexpr int F_SMEM = OFF_BAR + 256 + 1024;      // + alignment slack
-constexpr uint32_t TMEM_COLS = 512;               // S0, S1, O0, O1
+constexpr uint32_t TMEM_COLS = 512;               // S0, S1 at columns 0 and 128, O at 256
 
 // MN-major 128B-swizzled operand: 64 elements of the N dimension are contiguous (one 128-byte row
 // per K index), 8 K rows form a 1024-byte swizzle atom; `lbo` = bytes between 64-wide N blocks,
@@ -62,6 +61,22 @@ __device__ __forceinline__ void tmem_ld32(uint32_t ta, float *v)
                  : "memory");
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// ... and back (the caller waits for the stores with tcgen05.wait::st)
+__device__ __forceinline__ void tmem_st32(uint32_t ta, const float *v)
+{
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+        asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+                     ::"r"(ta + 16u * h), "r"(__float_as_uint(v[16 * h + 0])), "r"(__float_as_uint(v[16 * h + 1])),
+                       "r"(__float_as_uint(v[16 * h + 2])), "r"(__float_as_uint(v[16 * h + 3])), "r"(__float_as_uint(v[16 * h + 4])),
+                       "r"(__float_as_uint(v[16 * h + 5])), "r"(__float_as_uint(v[16 * h + 6])), "r"(__float_as_uint(v[16 * h + 7])),
+                       "r"(__float_as_uint(v[16 * h + 8])), "r"(__float_as_uint(v[16 * h + 9])), "r"(__float_as_uint(v[16 * h + 10])),
+                       "r"(__float_as_uint(v[16 * h + 11])), "r"(__float_as_uint(v[16 * h + 12])), "r"(__float_as_uint(v[16 * h + 13])),
+                       "r"(__float_as_uint(v[16 * h + 14])), "r"(__float_as_uint(v[16 * h + 15]))
+                     : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi)
@@ -104,28 +119,41 @@ __global__ void __launch_bounds__(F_THREADS, 1) prefill_attention_umma_kernel(co
     const int n_tiles = (kv_len + FKV - 1) / FKV;
 
     pdl_launch_dependents();
-    if (threadIdx.x == 0) {
-        mbar_init(q_full, 1);
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(k_full(s), 1);
-            mbar_init(v_full(s), 1);
-            mbar_init(k_empty(s), 1);
-            mbar_init(v_empty(s), 1);
-            mbar_init(s_full(s), 1);
-            mbar_init(p_ready(s), 16);
-            mbar_init(o_full(s), 1);
+    // The two load warps set up the barriers themselves and only ARRIVE at the set-up barrier, so that the first
+    // tiles are on their way while the others still wait for the tensor-memory allocation.
+    uint32_t tmem = 0;
+    if (warp == 16 || warp == 17) {
+        if (lane == 0) {
+            *abort_flag = 0;
+            if (warp == 16) {
+                mbar_init(q_full, 1);
+                for (int s = 0; s < 2; ++s) {
+                    mbar_init(k_full(s), 1);
+                    mbar_init(k_empty(s), 1);
+                    mbar_init(s_full(s), 1);
+                    mbar_init(p_ready(s), 16);
+                    mbar_init(o_full(s), 1);
+                }
+            } else {
+                for (int s = 0; s < 2; ++s) {
+                    mbar_init(v_full(s), 1);
+                    mbar_init(v_empty(s), 1);
+                }
+            }
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        __syncwarp();
+        asm volatile("bar.arrive 2, 608;" ::: "memory");
+    } else {
+        if (warp == 18) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        asm volatile("bar.sync 2, 608;" ::: "memory");
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        tmem = *tmem_slot;
     }
-    if (warp == 18) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t tmem = *tmem_slot;
     pdl_wait();
 
     if (warp == 16 || warp == 17) {
@@ -196,14 +224,14 @@ __global__ void __launch_bounds__(F_THREADS, 1) prefill_attention_umma_kernel(co
                 if (!mbar_wait(p_ready(s), (j >> 1) & 1, a.err, abort_flag)) break;
                 if (!mbar_wait(v_full(s), (j >> 1) & 1, a.err, abort_flag)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t acc = tmem + 256u + (uint32_t)s * 128u;
+                const uint32_t acc = tmem + 256u; // O accumulates over the tiles
 #pragma unroll
                 for (int kk = 0; kk < FKV / UMMA_K; ++kk) {
                     const uint64_t da = make_desc(sP + (kk >> 2) * HALF_TILE) + (uint64_t)((kk & 3) * UMMA_K * 2 / 16);
                     const uint64_t db = make_desc_mn(sV(s) + kk * UMMA_K * 128, HALF_TILE, 1024);
-                    umma(acc, da, db, idesc_o, kk > 0 ? 1u : 0u);
+                    umma(acc, da, db, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
                 }
-                umma_commit(o_full(s));
+                umma_commit(o_full(0));
                 umma_commit(v_empty(s));
             }
         }
@@ -215,15 +243,17 @@ __global__ void __launch_bounds__(F_THREADS, 1) prefill_attention_umma_kernel(co
         const int pos_q = row < q_rows ? s0 + q0 + row : -1;
         const float sc = rsqrtf((float)FD) * 1.4426950408889634f;
         float *red = (float *)(gen + OFF_RED); // [2 tile parities][4 quarters][128 rows]
-        float o_acc[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) o_acc[i] = 0.f;
-        float m_run = -INFINITY, l_run = 0.f;
+        // m_used: the maximum the accumulated O (in tensor memory) and the row sum are relative to.  It follows the
+        // true running maximum lazily: O and the sum are only rescaled when the maximum has grown by more than 2^8
+        // since (P stays below 2^8, exact enough in bf16 and far from fp32 overflow), which is rare after the first tiles.
+        float m_used = -INFINITY, l_run = 0.f;
         bool ok = true;
         auto ex2 = [](float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; };
+        const uint32_t t_o = tmem + lane_off + 256u + (uint32_t)qt * 32u;
         for (int j = 0; j < n_tiles; ++j) {
             const int s = j & 1;
             if (ok && !mbar_wait(s_full(s), (j >> 1) & 1, a.err, abort_flag)) ok = false;
+            ok = __all_sync(0xffffffffu, ok); // warp-uniform: the tensor-memory accesses below are warp-wide
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int key0 = j * FKV + qt * 32;
             // keys of this tile beyond the row's own position are masked (only tiles that reach the diagonal)
@@ -245,55 +275,53 @@ __global__ void __launch_bounds__(F_THREADS, 1) prefill_attention_umma_kernel(co
             // the four threads of a row exchange the maxima of their quarters (sc > 0: maxima of the scaled scores)
             red[(s * 4 + qt) * 128 + row] = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sc;
             asm volatile("bar.sync 1, 512;" ::: "memory");
-            float mx = m_run;
+            float mx = m_used;
 #pragma unroll
             for (int t = 0; t < 4; ++t) mx = fmaxf(mx, red[(s * 4 + t) * 128 + row]);
-            const float mbase = mx == -INFINITY ? 0.f : mx;
-            const float corr = m_run == -INFINITY ? 0.f : ex2(m_run - mbase);
-            // O_{j-1} joins the running output (its P V product also was the last reader of the P tile)
-            if (ok && j > 0) {
-                if (!mbar_wait(o_full(s ^ 1), ((j - 1) >> 1) & 1, a.err, abort_flag)) ok = false;
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                if (ok) {
-                    float v[32];
-                    tmem_ld32(tmem + lane_off + 256u + (uint32_t)(s ^ 1) * 128u + (uint32_t)qt * 32u, v);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) o_acc[i] = (o_acc[i] + v[i]) * corr;
-                }
-            }
+            float factor = 1.f;
+            if (m_used == -INFINITY) m_used = mx;                 // nothing accumulated yet
+            else if (mx > m_used + 8.f) { factor = ex2(m_used - mx); m_used = mx; }
+            const float mbase = m_used == -INFINITY ? 0.f : m_used;
             float rs0 = 0.f, rs1 = 0.f;
-            uint8_t *prow = gen + OFF_P + (qt >> 1) * HALF_TILE + row * 128;
-            if (ok) {
+            uint32_t pk[16];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) { // 16-byte chunk (qt & 1) * 4 + q of the row's 64-key block, swizzled by row
-                    uint32_t pk[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float p0 = ex2(sv[q * 8 + 2 * e] * sc - mbase), p1 = ex2(sv[q * 8 + 2 * e + 1] * sc - mbase);
-                        rs0 += p0;
-                        rs1 += p1;
-                        pk[e] = pack2(p0, p1);
-                    }
-                    *(uint4 *)(prow + ((((qt & 1) * 4 + q) ^ (row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                }
+            for (int i = 0; i < 32; i += 2) {
+                const float p0 = ex2(sv[i] * sc - mbase), p1 = ex2(sv[i + 1] * sc - mbase);
+                rs0 += p0;
+                rs1 += p1;
+                pk[i >> 1] = pack2(p0, p1);
             }
-            l_run = l_run * corr + (rs0 + rs1);
-            m_run = mx;
+            l_run = l_run * factor + (rs0 + rs1);
+            // the previous P V product has read the P tile and settled O
+            if (ok && j > 0 && !mbar_wait(o_full(0), (j - 1) & 1, a.err, abort_flag)) ok = false;
+            ok = __all_sync(0xffffffffu, ok);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (__any_sync(0xffffffffu, factor != 1.f) && ok) {
+                float v[32];
+                tmem_ld32(t_o, v);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] *= factor;
+                tmem_st32(t_o, v);
+            }
+            if (ok) {
+                uint8_t *prow = gen + OFF_P + (qt >> 1) * HALF_TILE + row * 128;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) // 16-byte chunk (qt & 1) * 4 + q of the row's 64-key block, swizzled by row
+                    *(uint4 *)(prow + ((((qt & 1) * 4 + q) ^ (row & 7)) << 4)) = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+            }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             fence_proxy_async();
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(p_ready(s)) : "memory");
         }
-        if (ok && n_tiles > 0) {
-            const int s = (n_tiles - 1) & 1;
-            if (!mbar_wait(o_full(s), ((n_tiles - 1) >> 1) & 1, a.err, abort_flag)) ok = false;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            if (ok) {
-                float v[32];
-                tmem_ld32(tmem + lane_off + 256u + (uint32_t)s * 128u + (uint32_t)qt * 32u, v);
+        float o_acc[32];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) o_acc[i] += v[i];
-            }
+        for (int i = 0; i < 32; ++i) o_acc[i] = 0.f;
+        if (ok && n_tiles > 0) {
+            if (!mbar_wait(o_full(0), (n_tiles - 1) & 1, a.err, abort_flag)) ok = false;
+            ok = __all_sync(0xffffffffu, ok);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (ok) tmem_ld32(t_o, o_acc);
         }
         // the row's sum is the sum over its four threads (all ran on the same maxima)
         if (!ok) l_run = 0.f;
