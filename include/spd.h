@@ -148,6 +148,12 @@ int spd_set_graphs(spd_ctx *ctx, int32_t enabled);
  *   "l2_prefetch_blocks"
  *       64-wide K blocks of weights each thread block of a projection pulls into L2 before it
  *       waits for the preceding kernel (default 0 = off, at most 64; measured neutral to harmful).
+ *   "prefill_rescale_log2"
+ *       prefill attention on the tensor cores keeps its output accumulator relative to a row
+ *       maximum that follows the true running maximum lazily: the accumulator is rescaled only
+ *       when the maximum has grown by more than 2^value since the last rescale (default 8, at
+ *       most 16; 0 = follow the maximum exactly, every growth rescales).  The result is the same
+ *       softmax either way; only the rounding of the bf16 probabilities differs.
  * Errors: SPD_ENULL, SPD_EINVAL (unknown key, negative value). */
 int spd_set_tuning(spd_ctx *ctx, const char *key, int32_t value);
 

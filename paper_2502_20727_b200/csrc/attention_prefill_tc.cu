@@ -244,8 +244,9 @@ __global__ void __launch_bounds__(F_THREADS, 1) prefill_attention_umma_kernel(co
         const float sc = rsqrtf((float)FD) * 1.4426950408889634f;
         float *red = (float *)(gen + OFF_RED); // [2 tile parities][4 quarters][128 rows]
         // m_used: the maximum the accumulated O (in tensor memory) and the row sum are relative to.  It follows the
-        // true running maximum lazily: O and the sum are only rescaled when the maximum has grown by more than 2^8
-        // since (P stays below 2^8, exact enough in bf16 and far from fp32 overflow), which is rare after the first tiles.
+        // true running maximum lazily: O and the sum are only rescaled when the maximum has grown by more than
+        // 2^rescale_log2 since (default 8: P stays below 2^8, exact enough in bf16 and far from fp32 overflow), which
+        // is rare after the first tiles; 0 follows the maximum exactly.
         float m_used = -INFINITY, l_run = 0.f;
         bool ok = true;
         auto ex2 = [](float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; };
@@ -280,7 +281,7 @@ __global__ void __launch_bounds__(F_THREADS, 1) prefill_attention_umma_kernel(co
             for (int t = 0; t < 4; ++t) mx = fmaxf(mx, red[(s * 4 + t) * 128 + row]);
             float factor = 1.f;
             if (m_used == -INFINITY) m_used = mx;                 // nothing accumulated yet
-            else if (mx > m_used + 8.f) { factor = ex2(m_used - mx); m_used = mx; }
+            else if (mx > m_used + a.rescale_log2) { factor = ex2(m_used - mx); m_used = mx; }
             const float mbase = m_used == -INFINITY ? 0.f : m_used;
             float rs0 = 0.f, rs1 = 0.f;
             uint32_t pk[16];

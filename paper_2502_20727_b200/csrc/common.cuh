@@ -197,6 +197,8 @@ struct AttnArgs {
     const void *k_map, *v_map;
     // optional (prefill, same conditions): tensor map over q as [tokens][n_q_heads * head_dim], box 64 x 128
     const void *q_map;
+    // ... and how far (in powers of two) the running row maximum may grow before the accumulated output is rescaled
+    float rescale_log2;
     int cluster_merge;      // set by the launcher: the splits of a (sequence, head tile) are one thread-block cluster
 };
 // Paged decode attention with 16-token pages: query heads per thread block for a GQA group

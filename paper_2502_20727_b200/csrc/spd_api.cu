@@ -114,6 +114,7 @@ struct Ctx {
     float *ss_attn, *ss_mlp;     // partial row sums of squares (fused decode path)
     int split_override[SITE_COUNT];
     int l2_prefetch_kb;          // K blocks per thread block prefetched into L2 by the decode GEMMs
+    int prefill_rescale_log2;    // tcgen05 prefill attention: growth of the row maximum (log2) that triggers a rescale
     int launches_last;
     TpState tp;
     // activation tensor maps, by buffer and token box (16, 32, 64, 128), built on first use
@@ -403,7 +404,7 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
             a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.counters = c->attn_cnt; a.err = c->err;
             if (!decode && d.dtype == 1 && d.head_dim == 128 && d.kv_block_size == 16) {
                 MAP_OR_FAIL(qm, act_map(c, AB_Q, 128));
-                a.q_map = qm; a.k_map = &c->maps[l].kpages; a.v_map = &c->maps[l].vpages;
+                a.q_map = qm; a.k_map = &c->maps[l].kpages; a.v_map = &c->maps[l].vpages; a.rescale_log2 = (float)c->prefill_rescale_log2;
             }
             if (decode) LAUNCH(K_ATTN, launch_decode_attention<T>(a, st));
             else LAUNCH(K_ATTN, launch_prefill_attention<T>(a, st));
@@ -779,7 +780,7 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
             a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.counters = c->attn_cnt; a.err = c->err;
             if (d.head_dim == 128 && d.kv_block_size == 16) {
                 MAP_OR_FAIL(qm, act_map(c, AB_Q, 128));
-                a.q_map = qm; a.k_map = &c->maps[l].kpages; a.v_map = &c->maps[l].vpages;
+                a.q_map = qm; a.k_map = &c->maps[l].kpages; a.v_map = &c->maps[l].vpages; a.rescale_log2 = (float)c->prefill_rescale_log2;
             }
             LAUNCH(K_ATTN, launch_prefill_attention<bf16>(a, st));
         }
@@ -1021,6 +1022,7 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     c.ss_attn = (float *)(c.ws + L.ss_attn); c.ss_mlp = (float *)(c.ws + L.ss_mlp);
     for (int i = 0; i < SITE_COUNT; ++i) c.split_override[i] = 0;
     c.l2_prefetch_kb = 0;
+    c.prefill_rescale_log2 = 8;
     c.launches_last = 0;
     c.tp.on = false;
     c.use_graphs = true;
@@ -1198,6 +1200,7 @@ int spd_set_tuning(spd_ctx *ctx, const char *key, int32_t value)
     bool found = false;
     for (int i = 0; i < SITE_COUNT; ++i)
         if (!strcmp(key, site_keys[i])) { c.split_override[i] = value; found = true; }
+    if (!strcmp(key, "prefill_rescale_log2")) { c.prefill_rescale_log2 = value > 16 ? 16 : value; found = true; }
     if (!strcmp(key, "l2_prefetch_blocks")) { c.l2_prefetch_kb = value > 64 ? 64 : value; found = true; }
     if (!found) return SPD_EINVAL;
     for (GraphEntry &g : c.graphs) cudaGraphExecDestroy(g.exec); // captured steps used the old setting

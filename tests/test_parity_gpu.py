@@ -201,3 +201,21 @@ def test_run_twice_bitwise_identical():
         b, _ = p.decode(0)
         outs.append((a, b))
     assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+
+
+@pytest.mark.parametrize("rescale_log2", [0, 2])
+def test_prefill_attention_rescale_path(rescale_log2):
+    """The tensor-core prefill attention rescales its accumulated output in tensor memory whenever the running
+    row maximum outgrows the one in use by more than 2^rescale_log2: with 0 every growth goes through that path
+    (with the default of 8 and N(0,1) inputs it hardly ever runs).  700 tokens = 6 key tiles with a ragged last
+    one, GQA group of 4, head_dim 128, second sequence chunked inside the prompt."""
+    w = si.Workload("fa_rescale", "bf16", 2, 512, 8, 2, 128, 1024, 2, (0, 1), 2, 700, 1)
+    p = Pair(w, mask=(0, 1), B=2, max_len=704, max_prefill_tokens=512)
+    p.stack.set_tuning(prefill_rescale_log2=rescale_log2)
+    got, ref, _ = p.prefill(700)
+    e = rel_err(got, ref)
+    assert e <= TOL["bf16"], f"prefill rel err {e}"
+    got, ref = p.decode(0)
+    assert rel_err(got, ref) <= TOL["bf16"]
+    assert p.stack.device_error() == 0
+    p.stack.close()
