@@ -57,6 +57,16 @@ def test_rank_mode_eight_ranks_head_dim_128():
     p.stack.close()
 
 
+@pytest.mark.parametrize("B", [20, 40])
+def test_rank_mode_larger_batches(B):
+    """Token tiles of 32 and 64 (other instantiations of the exchange tail), ragged contexts, mixed mask."""
+    mask = (1, 0)
+    w = si.Workload("tp_batch", "bf16", 2, 512, 8, 4, 64, 1376, 4, mask, B, 40, 2)
+    lens = [1 + (7 * i) % 40 for i in range(B)]
+    p = run_tp_case(w, mask, B, lens, 2)
+    p.stack.close()
+
+
 def test_rank_mode_matches_the_single_launch_emulation():
     """The same stack through spd_decode_step (shards as one cluster per tile) and through the rank-mode
     step: two implementations of one function, equal to rounding."""
