@@ -297,6 +297,17 @@ int spd_tp_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *se
                        const int32_t *block_table, int32_t max_pages, int32_t max_context, void *out,
                        void *stream);
 
+/* Prompt processing of an attached context (same arguments as spd_prefill, same collective
+ * rules as spd_tp_decode_step): the prompts go through the rank-mode step in chunks of at most
+ * 512 tokens (fewer when several ranks share one launch: all thread blocks of an exchange launch
+ * must be resident), every chunk attending to the cached positions before it.  The projections
+ * are the weight-streaming kernels of the decode step with 64-token tiles - functionally the
+ * block of Sec. 3 / Sec. 4.1.1 for any number of tokens, not a throughput path.
+ *   out : [ranks held by the context][B][S][hidden] bf16
+ * Errors: SPD_ENULL, SPD_EINVAL (not attached, B > max_batch), SPD_ECAPACITY, SPD_ECUDA. */
+int spd_tp_prefill(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int32_t *block_table,
+                   int32_t max_pages, void *out, void *stream);
+
 /* Number of shard sums ("sync-points", Sec. 3) one forward pass of this stack executes:
  * 2 per TP block, 1 per SPD block. */
 int spd_sync_points(const spd_ctx *ctx);

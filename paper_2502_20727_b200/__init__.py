@@ -93,6 +93,7 @@ def load_library() -> ctypes.CDLL:
     lib.spd_tp_attach.argtypes = [vp, i32, i32, ctypes.POINTER(vp), sz, vp]
     lib.spd_tp_detach.argtypes = [vp]
     lib.spd_tp_decode_step.argtypes = [vp, vp, i32, vp, vp, i32, i32, vp, vp]
+    lib.spd_tp_prefill.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp]
     lib.spd_profile_begin.argtypes = [vp]
     lib.spd_profile_end.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     lib.spd_profile_kinds.argtypes = []
@@ -459,6 +460,17 @@ class SpdStack:
 
     def tp_detach(self):
         _check("spd_tp_detach", self.lib.spd_tp_detach(self._ctx))
+
+    def tp_prefill(self, x: torch.Tensor, block_table: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Prompts in rank mode; returns [ranks held by this context, B, S, hidden]."""
+        B, S, H = x.shape
+        self._check_io(x, block_table)
+        if out is None:
+            out = torch.empty((self.dims.T, B, S, H), dtype=x.dtype, device=x.device)
+        with torch.cuda.device(self.device):
+            _check("spd_tp_prefill", self.lib.spd_tp_prefill(self._ctx, x.data_ptr(), B, S, block_table.data_ptr(),
+                                                              block_table.shape[1], out.data_ptr(), _stream_ptr()))
+        return out
 
     def tp_decode_step(self, x: torch.Tensor, seq_lens: torch.Tensor, block_table: torch.Tensor, max_context: int,
                        out: Optional[torch.Tensor] = None) -> torch.Tensor:

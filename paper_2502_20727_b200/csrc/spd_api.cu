@@ -267,8 +267,10 @@ TpLayout tp_layout(const spd_dims &d, int T)
 {
     TpLayout L{};
     const size_t H = d.hidden, h_tiles = (H + 127) / 128;
-    L.Mb = d.max_batch;
-    L.tok_tiles = (d.max_batch + 15) / 16; // an upper bound for every token box
+    // token capacity: a decode batch, or a prompt chunk of up to 512 tokens
+    const long chunk = d.max_prefill_tokens < 512 ? d.max_prefill_tokens : 512;
+    L.Mb = d.max_batch > chunk ? d.max_batch : chunk;
+    L.tok_tiles = (int)((L.Mb + 15) / 16); // an upper bound for every token box
     L.site_flags = h_tiles * L.tok_tiles * T * TP_FLAG_RANGES;
     L.src_bytes = (size_t)L.Mb * H * 4;
     L.buf_bytes = L.src_bytes * T;
@@ -601,12 +603,13 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
     return SPD_OK;
 }
 
-// One decode step in rank mode (tensor parallelism across GPUs, Sec. 3): every local rank runs
-// the block on its own shard and its own copy of the residual stream; the shard sums that the
-// block keeps (o_proj of a TP block, down of every block; Sec. 4.1.1) are exchanges with the
-// other ranks of the group inside the projection's tail.  out: [local ranks][M][H].
-int run_decode_tp(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t *bt, int max_pages,
-                  int max_context, cudaStream_t st)
+// M tokens (one decode step, or a prompt chunk) in rank mode (tensor parallelism across GPUs, Sec. 3):
+// every local rank runs the block on its own shard and its own copy of the residual stream; the shard
+// sums that the block keeps (o_proj of a TP block, down of every block; Sec. 4.1.1) are exchanges with
+// the other ranks of the group inside the projection's tail.  out: rank z's [M][H] rows lie out_stride
+// bytes after rank z-1's.  Prompt chunks go through the same weight-streaming kernels, 64 tokens per tile.
+int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, const int32_t *bt, int max_pages,
+           bool decode, int max_context, cudaStream_t st)
 {
     const spd_dims &d = c->d;
     TpState &tp = c->tp;
@@ -614,11 +617,11 @@ int run_decode_tp(Ctx *c, const void *x, void *out, int M, TokMap tm, const int3
     const int H = d.hidden, qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, F = d.ffn, nl = d.T;
     const int Fs = F / nl;
     const long Mb = TL.Mb;
-    const Plan p = make_plan(d, M, true, max_context, c->split_override[SITE_ATTN]);
+    const Plan p = make_plan(d, M, decode, max_context, c->split_override[SITE_ATTN]);
     PageTable pt{bt, max_pages, c->n_pages, d.kv_block_size, d.n_kv_heads};
     const int tbox = tc_token_box(true, M);
     const int tok_tiles = cdiv(M, tbox), h_tiles = cdiv(H, 128);
-    if (tok_tiles > TL.tok_tiles) return SPD_EINVAL;
+    if (tok_tiles > TL.tok_tiles || M > TL.Mb) return SPD_EINVAL;
     const TcMap *hmap = &tp.h_maps[box_index(tbox)];
     int launches = 0;
     const bool rope = d.rope_base > 0.f;
@@ -671,7 +674,15 @@ int run_decode_tp(Ctx *c, const void *x, void *out, int M, TokMap tm, const int3
             a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.B = M; a.splits = p.attn_splits;
             a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.counters = c->attn_cnt; a.err = c->err;
             if (d.head_dim == 128 && d.kv_block_size == 16) { a.k_map = &c->maps[l].kpages; a.v_map = &c->maps[l].vpages; }
-            LAUNCH(K_ATTN, launch_decode_attention<bf16>(a, st));
+            if (decode) LAUNCH(K_ATTN, launch_decode_attention<bf16>(a, st));
+            else {
+                a.splits = 1;
+                if (a.k_map) {
+                    MAP_OR_FAIL(qm, act_map(c, AB_Q, 128));
+                    a.q_map = qm; a.rescale_log2 = (float)c->prefill_rescale_log2;
+                }
+                LAUNCH(K_ATTN, launch_prefill_attention<bf16>(a, st));
+            }
         }
         {   // a5 - a7: Y_z from the rank's own heads.  TP block: R = X + sum over ranks (sync-point 1);
             // SPD block: the sync-point is dropped, R_z = X + Y_z feeds the rank's MLP and Y_z is kept for a10
@@ -709,7 +720,7 @@ int run_decode_tp(Ctx *c, const void *x, void *out, int M, TokMap tm, const int3
             if (!sync) g.tp.addend = (const float *)(r0 + TL.ysave);
             g.res_out = (float *)(r0 + TL.res0);
             if (l + 1 < d.n_layers) { g.gain = c->layers[l + 1].attn_norm; g.hg = r0 + TL.hg; g.ss_out = (float *)(r0 + TL.ss_attn); }
-            else { g.final_out = out; g.tp.out_stride = (long)M * H * 2; }
+            else { g.final_out = out; g.tp.out_stride = out_stride; }
             LAUNCH(K_DOWN, launch_gemm_decode(EPI_RESID_TP, wmaps, *am, g, st));
         }
     }
@@ -1268,6 +1279,53 @@ int spd_tp_detach(spd_ctx *ctx)
     return SPD_OK;
 }
 
+int spd_tp_prefill(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int32_t *block_table, int32_t max_pages,
+                   void *out, void *stream)
+{
+    if (!ctx || !x || !block_table || !out) return SPD_ENULL;
+    Ctx &c = ctx->c;
+    const spd_dims &d = c.d;
+    if (!c.tp.on) return SPD_EINVAL;
+    if (B < 1 || S < 1 || B > d.max_batch || x == out) return SPD_EINVAL;
+    if (S > d.max_seq_len || (long)max_pages * d.kv_block_size < S) return SPD_ECAPACITY;
+    cudaStream_t st = (cudaStream_t)stream;
+    // Tokens per launch: the region's capacity; with several ranks in one launch also what keeps every thread
+    // block of an exchange launch resident (three blocks per SM, one block per 128 columns, rank and 64 tokens).
+    long chunk = c.tp.L.Mb;
+    if (d.T > 1) {
+        const long tiles = (long)cdiv(d.hidden, 128) * d.T, fit = (3L * N_SM) / tiles;
+        if (fit < 1) { g_last_cuda_error = (int)cudaErrorCooperativeLaunchTooLarge; return SPD_ECUDA; }
+        if (fit * 64 < chunk) chunk = fit * 64;
+    }
+    const long rank_stride = (long)B * S * d.hidden * 2;
+    int total_launches = 0;
+    auto run = [&](int b0, int nb, int s0, int ns) -> int {
+        TokMap tm{0, b0, ns, s0, nullptr};
+        const size_t off = ((size_t)b0 * S + s0) * d.hidden * 2;
+        const int rc = run_tp(&c, (const char *)x + off, (char *)out + off, rank_stride, nb * ns, tm, block_table, max_pages, false, S, st);
+        if (rc == SPD_OK) {
+            for (int l = 0; l < d.n_layers; ++l) c.tp.exchanges += c.mask[l] ? 2 : 1;
+            total_launches += c.launches_last;
+        }
+        return rc;
+    };
+    if (S <= chunk) {
+        const int nb = (int)(chunk / S);
+        for (int b0 = 0; b0 < B; b0 += nb) {
+            const int rc = run(b0, B - b0 < nb ? B - b0 : nb, 0, S);
+            if (rc) return rc;
+        }
+    } else {
+        for (int b = 0; b < B; ++b)
+            for (int s0 = 0; s0 < S; s0 += (int)chunk) {
+                const int rc = run(b, 1, s0, S - s0 < chunk ? S - s0 : (int)chunk);
+                if (rc) return rc;
+            }
+    }
+    c.launches_last = total_launches;
+    return SPD_OK;
+}
+
 int spd_tp_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_lens, const int32_t *block_table,
                        int32_t max_pages, int32_t max_context, void *out, void *stream)
 {
@@ -1285,7 +1343,7 @@ int spd_tp_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *se
     // A captured step is valid for one receive-buffer phase: consecutive exchanges alternate between the
     // two buffers, so a stack with an odd number of exchanges per step needs one graph per phase.
     const GraphKey key{x, seq_lens, block_table, out, B, max_pages, ctx_bucket, 1 + (int)(c.tp.exchanges & 1)};
-    const int rc = replay_or_run(c, key, [&]() { return run_decode_tp(&c, x, out, B, tm, block_table, max_pages, ctx_bucket, st); }, st);
+    const int rc = replay_or_run(c, key, [&]() { return run_tp(&c, x, out, (long)B * d.hidden * 2, B, tm, block_table, max_pages, true, ctx_bucket, st); }, st);
     if (rc != SPD_OK) return rc;
     for (int l = 0; l < d.n_layers; ++l) c.tp.exchanges += c.mask[l] ? 2 : 1; // the same on every rank of the group
     return SPD_OK;

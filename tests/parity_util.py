@@ -89,6 +89,15 @@ class Pair:
         self.pos = self.pos + 1
         return to_np(got), ref[:, 0, :]
 
+    def tp_prefill(self, S, seed=0):
+        """Prompts in rank mode: every rank's output [T, B, S, H] and the oracle's."""
+        x = si.make_hidden(self.w, (self.B, S, self.w.hidden), "cpu", seed, 0)
+        ref, syncs = self._oracle(to_np(x))
+        got = self.stack.tp_prefill(x.to(self.device), self.block_table)
+        torch.cuda.synchronize()
+        self.pos = self.pos + S
+        return to_np(got), ref, syncs
+
     def tp_decode(self, t, seed=0):
         """One decode step in rank mode (the stack attached as all T ranks of a group on this GPU):
         every rank's output [T, B, H] and the oracle's."""

@@ -57,6 +57,45 @@ def test_rank_mode_eight_ranks_head_dim_128():
     p.stack.close()
 
 
+@pytest.mark.parametrize("mask,T,S", [((0, 1, 0), 4, 37), ((1, 0), 2, 150)])
+def test_rank_mode_prompts_then_decode(mask, T, S):
+    """Prompts through the rank-mode step (several 64-token tiles, chunks that attend to the chunks before them),
+    then decode steps on the caches it filled."""
+    w = si.Workload("tp_prompt", "bf16", len(mask), 512, 8, 4, 64, 1376, T, mask, 3, S, 2)
+    p = Pair(w, mask=mask, B=3, max_len=S + 2)
+    p.stack.tp_attach_local()
+    torch.cuda.synchronize()
+    got, ref, _ = p.tp_prefill(S)
+    for r in range(T):
+        e = rel_err(got[r], ref)
+        assert e <= TOL["bf16"], f"prompt, rank {r}: rel err {e}"
+        assert np.array_equal(got[r], got[0])
+    for t in range(2):
+        got, ref = p.tp_decode(t)
+        for r in range(T):
+            assert rel_err(got[r], ref) <= TOL["bf16"]
+    assert p.stack.device_error() == 0
+    p.stack.close()
+
+
+def test_rank_mode_prompt_head_dim_128_chunked():
+    """head_dim 128 (tensor-core prompt attention), 8 ranks: 128 tiles per 64 tokens, so the prompt goes in
+    chunks of 192 tokens; 300-token prompts are cut inside the sequence."""
+    mask = (0, 1)
+    w = si.Workload("tp_prompt128", "bf16", 2, 1024, 16, 8, 128, 2048, 8, mask, 2, 300, 1)
+    p = Pair(w, mask=mask, B=2, max_len=304)
+    p.stack.tp_attach_local()
+    torch.cuda.synchronize()
+    got, ref, _ = p.tp_prefill(300)
+    for r in (0, 3, 7):
+        e = rel_err(got[r], ref)
+        assert e <= TOL["bf16"], f"prompt, rank {r}: rel err {e}"
+    got, ref = p.tp_decode(0)
+    assert rel_err(got[0], ref) <= TOL["bf16"]
+    assert p.stack.device_error() == 0
+    p.stack.close()
+
+
 @pytest.mark.parametrize("B", [20, 40])
 def test_rank_mode_larger_batches(B):
     """Token tiles of 32 and 64 (other instantiations of the exchange tail), ragged contexts, mixed mask."""
