@@ -222,6 +222,40 @@ __device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const De
         gn = make_float4(a.x, a.y, b.x, b.y);
     }
     if (spd_groups) {
+        const int rows = (g.t_rows - t.t_row0 < BN ? g.t_rows - t.t_row0 : BN) - t.rank; // this block's tokens: every P-th of them
+        if (rows > 3 * t.P) {
+            // Four tokens or more: one token per warp at a time, the devices of a token in turn (one gather of the
+            // partials per token instead of one per warp and token).
+            for (int q = warp;; q += 4) {
+                const int j = t.rank + t.P * q, m = t.t_row0 + j;
+                if (j >= BN || m >= g.t_rows) break;
+                const long idx = (long)m * H + n;
+                float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (valid) x = *(const float4 *)(g.res_in + idx);
+                float4 y[MAX_P];
+                load_partials(y, S, j, lane, t.P);
+                float4 tot = make_float4(0.f, 0.f, 0.f, 0.f), yi = make_float4(0.f, 0.f, 0.f, 0.f);
+                int cnt = 0, i = 0;
+#pragma unroll
+                for (int s = 0; s < MAX_P; ++s) {
+                    if (s >= t.P) continue;
+                    add4(yi, y[s]);
+                    if (++cnt < per) continue;
+                    add4(tot, yi);
+                    float4 ri = x;
+                    add4(ri, yi);
+                    if (valid && g.hg) store_bf16x4((bf16 *)g.hg + (long)i * g.hg_stride + idx, ri, gn);
+                    const float sq = warp_sum(valid ? sq4(ri) : 0.f);
+                    if (lane == 0 && g.ss_out) g.ss_out[((long)t.wt * G + i) * g.Mcap + m] = sq;
+                    yi = make_float4(0.f, 0.f, 0.f, 0.f);
+                    cnt = 0;
+                    ++i;
+                }
+                add4(x, tot);
+                if (valid && g.res_out) *(float4 *)(g.res_out + idx) = x;
+            }
+            return;
+        }
         // All four warps work on the same token; warp w finishes devices w, w+4 (ranges i*per .. i*per+per-1 are
         // device i), so that the per-device stores and reductions of a block with few tokens run side by side.
         for (int q = 0;; ++q) {
