@@ -38,6 +38,10 @@ template <int EPI> struct PCfg {
     static constexpr int STAGES = (192 * 1024 - X_BYTES - H_BYTES) / STAGE_BYTES;
     static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
     static constexpr int SMEM_BYTES = RING_BYTES + X_BYTES + H_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    // Epilogue warps: 0-3 (one per accumulator lane quarter); PRE_OPROJ_SPD, whose tail is T times the work per MMA
+    // of the others, adds warps 6-9: two threads per row, 64 of the tile's 128 columns each.
+    static constexpr int EPI_WARPS = (EPI == PRE_OPROJ_SPD) ? 8 : 4;
+    static constexpr int THREADS_ = 64 + 32 * EPI_WARPS;
 };
 
 struct PreLaunch {
@@ -311,15 +315,15 @@ __device__ __forceinline__ void epi_resid(const PreGemmArgs &g, const PreTile &t
     if (valid && g.ss_out) g.ss_out[(long)t.nt * g.Mcap + m] = ssq;
 }
 
-__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+template <int N_THREADS> __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(N_THREADS) : "memory"); }
 
 // SPD o_proj: the X tile of an output tile is parked in tensor memory twice - once as is (every
 // device's R_i = X + Y_i needs it) and once as the start of X + sum_i Y_i - by the thread that owns
 // the row, while the MMA warp works on the first K slice.
-__device__ __forceinline__ void spd_park_x(const PreGemmArgs &g, const PreTile &t, uint32_t tx, uint32_t ttot, int m, bool valid)
+__device__ __forceinline__ void spd_park_x(const PreGemmArgs &g, const PreTile &t, uint32_t tx, uint32_t ttot, int m, bool valid, int half)
 {
 #pragma unroll 1
-    for (int c = 0; c < 8; ++c) {
+    for (int c = half * 4; c < half * 4 + 4; ++c) {
         const int n = t.row0 + c * 16;
         if (n >= g.H) break;
         float x[16];
@@ -335,11 +339,11 @@ __device__ __forceinline__ void spd_park_x(const PreGemmArgs &g, const PreTile &
 }
 
 // Sum of squares of this row's 128 accumulator columns (MLP matching: norm of a partition's output).
-__device__ __forceinline__ float epi_row_sumsq(const PreGemmArgs &g, const PreTile &t, uint32_t tacc)
+__device__ __forceinline__ float epi_row_sumsq(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, int half)
 {
     float ssq = 0.f;
 #pragma unroll 1
-    for (int c = 0; c < 8; c += 2) {
+    for (int c = half * 4; c < half * 4 + 4; c += 2) {
         const int n = t.row0 + c * 16;
         if (n >= g.H) break;
         float ya[16], yb[16];
@@ -357,12 +361,12 @@ __device__ __forceinline__ float epi_row_sumsq(const PreGemmArgs &g, const PreTi
 // 128 rows, 128-byte swizzle: thread = row, eight consecutive rows hit eight different 16-byte
 // columns) and leaves through a TMA store; X + sum_i Y_i is written by the last pass.
 __device__ __forceinline__ float epi_oproj_spd(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, uint32_t tx, uint32_t ttot, int z,
-                                               int m, bool valid, uint8_t *hs)
+                                               int m, bool valid, uint8_t *hs, int r, int half)
 {
-    const int T = g.batches, r = threadIdx.x, sw = r & 7;
+    const int T = g.batches, sw = r & 7; // r: row of the tile
     float ssq = 0.f;
 #pragma unroll 1
-    for (int c = 0; c < 4; ++c) { // 32 columns per round: few tensor-memory round trips on the critical path
+    for (int c = half * 2; c < half * 2 + 2; ++c) { // 32 columns per round: few tensor-memory round trips on the critical path
         const int n = t.row0 + c * 32;
         if (n >= g.H) break;
         float y[32], x[32], tot[32];
@@ -398,7 +402,7 @@ __device__ __forceinline__ float epi_oproj_spd(const PreGemmArgs &g, const PreTi
 }
 
 template <int EPI>
-__global__ void __launch_bounds__(THREADS, 1) gemm_prefill_kernel(const __grid_constant__ CUtensorMap tm_w0,
+__global__ void __launch_bounds__(PCfg<EPI>::THREADS_, 1) gemm_prefill_kernel(const __grid_constant__ CUtensorMap tm_w0,
                                                                   const __grid_constant__ CUtensorMap tm_w1,
                                                                   const __grid_constant__ CUtensorMap tm_w2,
                                                                   const __grid_constant__ CUtensorMap tm_t,
@@ -429,7 +433,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_prefill_kernel(const __grid_c
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), C::EPI_WARPS); }
         mbar_init(xfull_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -504,12 +508,16 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_prefill_kernel(const __grid_c
     } else {
         uint32_t pc = 0, tile_cnt = 0;
         bool ok = true;
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        // accumulator lane quarter of this warp (a warp reaches lanes 32 * (warp % 4) ..), and which half of the
+        // columns it finishes when two warps share a quarter
+        const int quarter = warp & 3, half = warp >= 6 ? 1 : 0;
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_cnt) {
             const PreTile t = decode_tile(L, EPI, tile);
-            const int m = t.m0 + warp * 32 + lane;
+            const int m = t.m0 + quarter * 32 + lane;
             const bool valid = m < g.t_rows;
-            if (EPI == PRE_OPROJ_SPD && !g.norm_only) spd_park_x(g, t, tmem_base + lane_base + X_COL, tmem_base + lane_base + TOT_COL, m, valid);
+            if (EPI == PRE_OPROJ_SPD && !g.norm_only)
+                spd_park_x(g, t, tmem_base + lane_base + X_COL, tmem_base + lane_base + TOT_COL, m, valid, half);
             for (int pass = 0; pass < L.passes; ++pass, ++pc) {
                 const int buf = pc & 1;
                 if (!mbar_wait(tfull_bar(buf), (pc >> 1) & 1, g.err, abort_flag)) { ok = false; break; }
@@ -520,19 +528,20 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_prefill_kernel(const __grid_c
                 else if (EPI == PRE_GATEUP) epi_gateup(g, t, tacc, m, valid);
                 else if (EPI == PRE_RESID) epi_resid(g, t, tacc, m, valid);
                 else if (g.norm_only) {
-                    const float ssq = epi_row_sumsq(g, t, tacc);
-                    if (valid) g.ss_out[((long)t.nt * g.batches + pass) * g.Mcap + m] = ssq;
+                    const float ssq = epi_row_sumsq(g, t, tacc, half);
+                    if (valid) g.ss_out[((long)(t.nt * 2 + half) * g.batches + pass) * g.Mcap + m] = ssq;
                 } else {
                     // two staging tiles in turn: the store issued two passes ago has read its source
                     uint8_t *hst = hs + (pc & 1) * 32768;
                     if (threadIdx.x == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                    epi_sync();
+                    epi_sync<32 * C::EPI_WARPS>();
                     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_PREFILL + EPI, TR_DEP_DONE);
-                    const float ssq = epi_oproj_spd(g, t, tacc, tmem_base + lane_base + X_COL, tmem_base + lane_base + TOT_COL, pass, m, valid, hst);
-                    if (valid && g.ss_out) g.ss_out[((long)t.nt * g.batches + pass) * g.Mcap + m] = ssq;
+                    const float ssq = epi_oproj_spd(g, t, tacc, tmem_base + lane_base + X_COL, tmem_base + lane_base + TOT_COL, pass, m, valid, hst,
+                                                    quarter * 32 + lane, half);
+                    if (valid && g.ss_out) g.ss_out[((long)(t.nt * 2 + half) * g.batches + pass) * g.Mcap + m] = ssq;
                     fence_proxy_async();
                     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_PREFILL + EPI, TR_MAIN_DONE);
-                    epi_sync();
+                    epi_sync<32 * C::EPI_WARPS>();
                     if (threadIdx.x == 0) {
                         tma_store_3d(&tm_h, smem_u32(hst), t.row0, t.m0, pass);
                         tma_store_3d(&tm_h, smem_u32(hst) + 16384, t.row0 + 64, t.m0, pass);
@@ -573,7 +582,7 @@ cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
     }
     const int total = L.m_tiles * L.n_tiles;
     const dim3 grid(total < n_sm ? total : n_sm);
-    return launch_kernel(gemm_prefill_kernel<EPI>, grid, dim3(THREADS), C::SMEM_BYTES, st, 0, *tw[0], *tw[1], *tw[2], tt, tx, tr, th, L);
+    return launch_kernel(gemm_prefill_kernel<EPI>, grid, dim3(C::THREADS_), C::SMEM_BYTES, st, 0, *tw[0], *tw[1], *tw[2], tt, tx, tr, th, L);
 }
 
 // One thread block per token: whole-row sum of squares in one partial.
@@ -607,7 +616,8 @@ __global__ void __launch_bounds__(256) prefill_prologue_kernel(PrologueArgs a)
 
 } // namespace
 
-int pre_ss_tiles(PreEpilogue epi, int H) { return epi == PRE_OPROJ_SPD ? (H + 127) / 128 : (H + 255) / 256; }
+// (PRE_OPROJ_SPD: two partials per 128-column tile, one per thread of a row)
+int pre_ss_tiles(PreEpilogue epi, int H) { return epi == PRE_OPROJ_SPD ? 2 * ((H + 127) / 128) : (H + 255) / 256; }
 
 cudaError_t launch_gemm_prefill(PreEpilogue epi, const TcMap *const *weights, const TcMap &tokens, const PreGemmArgs &g,
                                 cudaStream_t st)

@@ -262,7 +262,7 @@ Layout make_layout(const spd_dims &d, bool any_spd)
     // fused decode path: partial sums of squares per 128-column tile
     const size_t h_tiles = (H + 127) / 128;
     L.ss_attn = take(h_tiles * Mmax * 4);
-    L.ss_mlp = take(h_tiles * T * Mmax * 4);
+    L.ss_mlp = take(2 * h_tiles * T * Mmax * 4); // the SPD o_proj of the prefill path leaves two partials per tile
     L.total = off;
     return L;
 }
