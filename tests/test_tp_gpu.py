@@ -166,3 +166,58 @@ def test_a_rank_that_never_arrives_is_reported_not_waited_for():
     assert torch.isfinite(y.float()).all()
     assert stack.device_error() == 0
     stack.close()
+
+
+def test_attach_argument_checks_and_mask_change_while_attached():
+    """Bad groups / regions are refused with a status code; the per-block mask may change between steps of an
+    attached context (every rank does so at the same step): the exchanges keep alternating their buffers."""
+    import paper_2502_20727_b200 as spd
+    mask = (0, 0)
+    w = si.Workload("tp_args", "bf16", 2, 512, 8, 4, 64, 1376, 4, mask, 3, 20, 4)
+    p = Pair(w, mask=mask, B=3, max_len=32)
+    st = p.stack
+    with pytest.raises(spd.SpdError):                      # not attached yet
+        st.tp_decode_step(torch.zeros((3, 512), dtype=torch.bfloat16, device="cuda:0"),
+                          torch.zeros(3, dtype=torch.int32, device="cuda:0"), p.block_table, 1)
+    nbytes = (st.tp_region_bytes(4) + 1023) // 1024 * 1024
+    buf = torch.zeros(4 * nbytes + 2048, dtype=torch.uint8, device="cuda:0")
+    base = (buf.data_ptr() + 1023) // 1024 * 1024
+    good = [base + j * nbytes for j in range(4)]
+    with pytest.raises(spd.SpdError):                      # a context of 4 shards is ranks 0..3 of a group of 4, nothing else
+        st.tp_attach(8, 0, good + good, nbytes)
+    with pytest.raises(spd.SpdError):                      # misaligned region
+        st.tp_attach(4, 0, [g + 16 for g in good], nbytes)
+    with pytest.raises(spd.SpdError):                      # region too small
+        st.tp_attach(4, 0, good, nbytes // 2)
+    with pytest.raises(spd.SpdError):                      # regions of the local ranks not at equal distances
+        st.tp_attach(4, 0, [good[0], good[1], good[3], good[2]], nbytes)
+    st.tp_attach(4, 0, good, nbytes)
+    torch.cuda.synchronize()
+    p.fill_cache(np.array([20, 3, 11], dtype=np.int32))
+    for t, m in enumerate([(0, 0), (1, 0), (1, 1), (0, 1)]):   # 2, 3, 4, 3 exchanges per step
+        st.set_mask(m)
+        p.mask = list(m)
+        got, ref = p.tp_decode(t)
+        for r in range(4):
+            assert rel_err(got[r], ref) <= TOL["bf16"], f"mask {m}, rank {r}"
+    assert st.device_error() == 0
+    st.close()
+
+
+def test_a_launch_whose_ranks_cannot_all_be_resident_is_refused():
+    """8 ranks at hidden 16384: 1024 thread blocks per exchange launch wait on one another, more than the GPU holds at
+    once - refused before anything runs, not left to time out."""
+    import paper_2502_20727_b200 as spd
+    mask = (0,)
+    w = si.Workload("tp_big", "bf16", 1, 16384, 8, 8, 128, 2048, 8, mask, 1, 4, 1)
+    p = Pair(w, mask=mask, B=1, max_len=16)
+    p.fill_cache(np.array([4], dtype=np.int32))
+    p.stack.tp_attach_local()
+    x = torch.zeros((1, 16384), dtype=torch.bfloat16, device="cuda:0")
+    with pytest.raises(spd.SpdError) as e:
+        p.stack.tp_decode_step(x, torch.full((1,), 4, dtype=torch.int32, device="cuda:0"), p.block_table, 5)
+    assert e.value.status == -5   # SPD_ECUDA (cooperative launch too large)
+    torch.cuda.synchronize()
+    p.stack.tp_detach()
+    assert p.stack.device_error() == 0
+    p.stack.close()
