@@ -219,3 +219,17 @@ def test_prefill_attention_rescale_path(rescale_log2):
     assert rel_err(got, ref) <= TOL["bf16"]
     assert p.stack.device_error() == 0
     p.stack.close()
+
+
+def test_prefill_attention_long_prompt_many_key_tiles():
+    """1500-token prompts: up to 12 key tiles per query tile (each K / V ring slot reused six times, a ragged last
+    tile), GQA group of 4, head_dim 128, prompt cut into chunks of 1024 tokens that attend to the cache."""
+    w = si.Workload("fa_long", "bf16", 1, 512, 8, 2, 128, 1024, 2, (0,), 2, 1500, 1)
+    p = Pair(w, mask=(0,), B=2, max_len=1504, max_prefill_tokens=1024)
+    got, ref, _ = p.prefill(1500)
+    e = rel_err(got, ref)
+    assert e <= TOL["bf16"], f"prefill rel err {e}"
+    got, ref = p.decode(0)
+    assert rel_err(got, ref) <= TOL["bf16"]
+    assert p.stack.device_error() == 0
+    p.stack.close()
