@@ -439,9 +439,8 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
     const DecGemmArgs &g = L.g;
     extern __shared__ uint8_t smem_raw[];
     __shared__ float sm_red[128];
-    // (sized by the token tile: at 16 tokens the static part stays under the 768 bytes that let a fourth block fit an SM)
-    __shared__ float sm_rstd[BN];
-    __shared__ long sm_kvoff[BN];
+    __shared__ float sm_rstd[64];
+    __shared__ long sm_kvoff[64];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t bars = base + C::STAGES * C::STAGE_BYTES; // full[S], empty[S], tmem_full
