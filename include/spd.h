@@ -148,6 +148,10 @@ int spd_set_graphs(spd_ctx *ctx, int32_t enabled);
  *   "l2_prefetch_blocks"
  *       64-wide K blocks of weights each thread block of a projection pulls into L2 before it
  *       waits for the preceding kernel (default 0 = off, at most 64; measured neutral to harmful).
+ *   "decode_ring_stages"
+ *       stages of the shared-memory ring the weight tiles of a decode projection stream through:
+ *       3, 4 or (16-token tiles) 5; 0 = chosen per launch (four stages; three where a launch of
+ *       16-token tiles only then stays resident at once).
  *   "prefill_rescale_log2"
  *       prefill attention on the tensor cores keeps its output accumulator relative to a row
  *       maximum that follows the true running maximum lazily: the accumulator is rescaled only

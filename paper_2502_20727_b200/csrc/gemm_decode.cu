@@ -39,14 +39,16 @@ using namespace tc;
 constexpr int MAX_GROUPS = 8; // emulated devices
 constexpr int MAX_P = 8;      // portable cluster size
 constexpr int THREADS = 192;
+constexpr int N_SM_DECODE = 148; // SMs the ring-depth rule is tuned for
 
-template <int BN> struct DCfg {
+// ST = stages of the operand ring.  What a launch needs in flight to keep HBM busy is about 16 MB over all of its
+// blocks (bandwidth x loaded latency): launches of 250-450 blocks want four stages (72-98 KB per block, three or two
+// blocks per SM), not three; a third stage less only pays where it lets a launch of more than 444 blocks of 16-token
+// tiles stay resident at once (four blocks per SM).  Chosen per launch, see launch_epi.
+template <int BN, int ST> struct DCfg {
     static constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    // Three thread blocks per SM with a short ring each (measured faster than two blocks with a
-    // deep ring: more blocks pull weights at once, and clusters of up to 8 blocks always find room).
-    static constexpr int RING_BYTES = 56 * 1024;
-    static constexpr int STAGES = RING_BYTES / STAGE_BYTES < 3 ? 3 : RING_BYTES / STAGE_BYTES;
+    static constexpr int STAGES = ST;
     static constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
     static_assert(STAGES * STAGE_BYTES >= 2 * BN * 128 * 4, "ring too small for the staging tiles");
@@ -426,14 +428,14 @@ __device__ __forceinline__ void epilogue_resid_tp(const DecGemmArgs &g, const De
     }
 }
 
-template <int BN, int EPI>
+template <int BN, int EPI, int ST>
 __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_w0,
                                                               const __grid_constant__ CUtensorMap tm_w1,
                                                               const __grid_constant__ CUtensorMap tm_w2,
                                                               const __grid_constant__ CUtensorMap tm_t,
                                                               const __grid_constant__ DecLaunch L)
 {
-    using C = DCfg<BN>;
+    using C = DCfg<BN, ST>;
     constexpr int SUB = (EPI == EPI_GATEUP) ? 2 : 1; // weight boxes per tile
     constexpr int ROWS = BM / SUB;                   // weight rows per box
     const DecGemmArgs &g = L.g;
@@ -611,15 +613,15 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
     if (t.P > 1) cluster_sync_all();
 }
 
-template <int BN, int EPI>
+template <int BN, int EPI, int ST>
 cudaError_t launch_cfg(const CUtensorMap *const *tw, const CUtensorMap &tt, const DecLaunch &L, dim3 grid, cudaStream_t st)
 {
-    using C = DCfg<BN>;
+    using C = DCfg<BN, ST>;
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_decode_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(gemm_decode_kernel<BN, EPI, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(gemm_decode_kernel<BN, EPI>, cudaFuncAttributePreferredSharedMemoryCarveout,
+        e = cudaFuncSetAttribute(gemm_decode_kernel<BN, EPI, ST>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                  (int)cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         attr_done = true;
@@ -646,9 +648,9 @@ cudaError_t launch_cfg(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
         occ.numAttrs = 2;
         int clusters = 0, api_per_sm = 0, dev = 0, smem_sm = 0, smem_rsv = 0, regs_sm = 0;
         cudaFuncAttributes fa;
-        cudaError_t e = cudaOccupancyMaxActiveClusters(&clusters, gemm_decode_kernel<BN, EPI>, &occ);
-        if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&api_per_sm, gemm_decode_kernel<BN, EPI>, THREADS, C::SMEM_BYTES);
-        if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, gemm_decode_kernel<BN, EPI>);
+        cudaError_t e = cudaOccupancyMaxActiveClusters(&clusters, gemm_decode_kernel<BN, EPI, ST>, &occ);
+        if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&api_per_sm, gemm_decode_kernel<BN, EPI, ST>, THREADS, C::SMEM_BYTES);
+        if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, gemm_decode_kernel<BN, EPI, ST>);
         if (e == cudaSuccess) e = cudaGetDevice(&dev);
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev);
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&smem_rsv, cudaDevAttrReservedSharedMemoryPerBlock, dev);
@@ -662,7 +664,7 @@ cudaError_t launch_cfg(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
         const long capacity = api_per_sm < 1 ? 0 : (long)clusters * per_sm / api_per_sm;
         if ((long)grid.x * grid.y > capacity) return cudaErrorCooperativeLaunchTooLarge;
     }
-    return cudaLaunchKernelEx(&cfg, gemm_decode_kernel<BN, EPI>, *tw[0], *tw[1], *tw[2], tt, L);
+    return cudaLaunchKernelEx(&cfg, gemm_decode_kernel<BN, EPI, ST>, *tw[0], *tw[1], *tw[2], tt, L);
 }
 
 template <int EPI>
@@ -670,10 +672,24 @@ cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
 {
     const int bn = tc_token_box(true, L.g.t_rows);
     dim3 grid(tiles * (L.g.z_is_plane ? 1 : L.g.batches), (L.g.t_rows + bn - 1) / bn, L.P);
+    // ring depth: four stages; three where that keeps a launch of 16-token tiles resident at once (four blocks per SM
+    // instead of three); five (16-token tiles only) on request
+    const long blocks = (long)grid.x * grid.y * grid.z;
+    int stages = L.g.ring_stages;
+    if (stages == 0) stages = (bn == 16 && blocks > 3L * N_SM_DECODE) ? 3 : 4;
+    // several ranks in one launch wait on one another: as many resident blocks as possible
+    if (L.g.ring_stages == 0 && EPI == EPI_RESID_TP && L.g.tp.exchange && L.g.batches > 1) stages = 3;
     switch (bn) {
-    case 16: return launch_cfg<16, EPI>(tw, tt, L, grid, st);
-    case 32: return launch_cfg<32, EPI>(tw, tt, L, grid, st);
-    default: return launch_cfg<64, EPI>(tw, tt, L, grid, st);
+    case 16:
+        if (stages <= 3) return launch_cfg<16, EPI, 3>(tw, tt, L, grid, st);
+        if (stages == 4) return launch_cfg<16, EPI, 4>(tw, tt, L, grid, st);
+        return launch_cfg<16, EPI, 5>(tw, tt, L, grid, st);
+    case 32:
+        if (stages <= 3) return launch_cfg<32, EPI, 3>(tw, tt, L, grid, st);
+        return launch_cfg<32, EPI, 4>(tw, tt, L, grid, st);
+    default:
+        if (stages <= 3) return launch_cfg<64, EPI, 3>(tw, tt, L, grid, st);
+        return launch_cfg<64, EPI, 4>(tw, tt, L, grid, st);
     }
 }
 

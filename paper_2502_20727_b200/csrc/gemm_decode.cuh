@@ -67,6 +67,7 @@ struct DecGemmArgs {
     int n_weights;
     int z_is_plane;        // o_proj: batch z is a K range of the same output tile (the K slice of shard z)
     int l2_prefetch_kb;    // K blocks of weights per thread block pulled into L2 before the dependency wait
+    int ring_stages;       // stages of the operand ring (3, 4; 5 at 16-token tiles); 0 = chosen per launch
     int *err;
     // ---- epilogue operands -----------------------------------------------------------
     SumSq ss_in;           // QKV, GATEUP: sums of squares of the GEMM input's rows

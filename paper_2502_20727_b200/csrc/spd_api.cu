@@ -114,6 +114,7 @@ struct Ctx {
     float *ss_attn, *ss_mlp;     // partial row sums of squares (fused decode path)
     int split_override[SITE_COUNT];
     int l2_prefetch_kb;          // K blocks per thread block prefetched into L2 by the decode GEMMs
+    int ring_stages;             // decode GEMMs: stages of the operand ring (0 = per launch)
     int prefill_rescale_log2;    // tcgen05 prefill attention: growth of the row maximum (log2) that triggers a rescale
     int launches_last;
     TpState tp;
@@ -541,6 +542,7 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
         DecGemmArgs g{};
         g.t_rows = M; g.err = c->err; g.H = H; g.Mcap = Mc; g.batches = 1; g.n_weights = 1; g.n_groups = 1;
         g.l2_prefetch_kb = c->l2_prefetch_kb;
+        g.ring_stages = c->ring_stages;
         return g;
     };
     for (int l = 0; l < d.n_layers; ++l) {
@@ -642,6 +644,7 @@ int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, 
         DecGemmArgs g{};
         g.t_rows = M; g.err = c->err; g.H = H; g.Mcap = Mb; g.batches = nl; g.w_batched = 1; g.t_batched = 1;
         g.n_weights = 1; g.n_groups = 1;
+        g.ring_stages = c->ring_stages;
         g.tp.on = 1; g.tp.T = tp.T; g.tp.rank_base = tp.rank_base; g.tp.z_stride = tp.z_stride;
         g.tp.step = (const unsigned *)(r0 + TL.step);
         return g;
@@ -1038,6 +1041,7 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     for (int i = 0; i < SITE_COUNT; ++i) c.split_override[i] = 0;
     c.l2_prefetch_kb = 0;
     c.prefill_rescale_log2 = 8;
+    c.ring_stages = 0;
     c.launches_last = 0;
     c.tp.on = false;
     c.use_graphs = true;
@@ -1215,6 +1219,7 @@ int spd_set_tuning(spd_ctx *ctx, const char *key, int32_t value)
     bool found = false;
     for (int i = 0; i < SITE_COUNT; ++i)
         if (!strcmp(key, site_keys[i])) { c.split_override[i] = value; found = true; }
+    if (!strcmp(key, "decode_ring_stages")) { c.ring_stages = (value == 0 || (value >= 3 && value <= 5)) ? value : 0; found = true; }
     if (!strcmp(key, "prefill_rescale_log2")) { c.prefill_rescale_log2 = value > 16 ? 16 : value; found = true; }
     if (!strcmp(key, "l2_prefetch_blocks")) { c.l2_prefetch_kb = value > 64 ? 64 : value; found = true; }
     if (!found) return SPD_EINVAL;
