@@ -200,12 +200,13 @@ Plan make_plan(const spd_dims &d, int M, bool decode, int max_context, int attn_
     return p;
 }
 
-// K ranges of a fused decode GEMM: as many as keep the launch within three resident thread blocks
-// per SM, each at least four K blocks long, at most `max_ranges` (the ranges of one output tile
-// form a thread-block cluster of at most 8 blocks).
-int decode_splits(long tiles, int num_kb, int override_, int max_ranges)
+// K ranges of a fused decode GEMM: as many as keep the launch within the thread blocks that are resident
+// at once (three per SM at 16-token tiles, two at 32 and 64 tokens: the operand ring is 72-98 KB), each at
+// least four K blocks long, at most `max_ranges` (the ranges of one output tile form a thread-block
+// cluster of at most 8 blocks).
+int decode_splits(long tiles, int num_kb, int override_, int max_ranges, int blocks_per_sm = 3)
 {
-    long s = override_ > 0 ? override_ : (3L * N_SM) / (tiles < 1 ? 1 : tiles);
+    long s = override_ > 0 ? override_ : ((long)blocks_per_sm * N_SM) / (tiles < 1 ? 1 : tiles);
     const long cap = num_kb / 4 < 1 ? 1 : num_kb / 4;
     if (s > cap) s = cap;
     if (s > max_ranges) s = max_ranges;
@@ -529,7 +530,7 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
     // K ranges of a site: automatic or overridden; a tile's ranges (times the shards for o_proj) fit a cluster of 8
     auto splits_of = [&](int site) {
         const SiteGeom sg = site_geom(d, site);
-        return decode_splits(sg.tiles * tok_tiles, sg.num_kb, c->split_override[site], 8 / sg.shard_ranges);
+        return decode_splits(sg.tiles * tok_tiles, sg.num_kb, c->split_override[site], 8 / sg.shard_ranges, tbox == 16 ? 3 : 2);
     };
     {
         PrologueArgs a{};
