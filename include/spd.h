@@ -150,8 +150,9 @@ int spd_set_graphs(spd_ctx *ctx, int32_t enabled);
  *       waits for the preceding kernel (default 0 = off, at most 64; measured neutral to harmful).
  *   "decode_ring_stages"
  *       stages of the shared-memory ring the weight tiles of a decode projection stream through:
- *       3, 4 or (16-token tiles) 5; 0 = chosen per launch (four stages; three where a launch of
- *       16-token tiles only then stays resident at once).
+ *       3, 4 or (16-token tiles) 5; 0 = chosen per launch (four stages; at 16-token tiles five for
+ *       launches of at most two thread blocks per SM and three where a launch only then stays
+ *       resident at once).
  *   "prefill_rescale_log2"
  *       prefill attention on the tensor cores keeps its output accumulator relative to a row
  *       maximum that follows the true running maximum lazily: the accumulator is rescaled only

@@ -672,11 +672,12 @@ cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
 {
     const int bn = tc_token_box(true, L.g.t_rows);
     dim3 grid(tiles * (L.g.z_is_plane ? 1 : L.g.batches), (L.g.t_rows + bn - 1) / bn, L.P);
-    // ring depth: four stages; three where that keeps a launch of 16-token tiles resident at once (four blocks per SM
-    // instead of three); five (16-token tiles only) on request
+    // ring depth at 16-token tiles: five stages for launches of at most two blocks per SM (they all stay resident and
+    // each block has more in flight), four up to three blocks per SM, three beyond (four blocks per SM keep the
+    // launch resident at once); four stages at 32- and 64-token tiles
     const long blocks = (long)grid.x * grid.y * grid.z;
     int stages = L.g.ring_stages;
-    if (stages == 0) stages = (bn == 16 && blocks > 3L * N_SM_DECODE) ? 3 : 4;
+    if (stages == 0) stages = (bn == 16 && blocks > 3L * N_SM_DECODE) ? 3 : ((bn == 16 && blocks <= 2L * N_SM_DECODE) ? 5 : 4);
     // several ranks in one launch wait on one another: as many resident blocks as possible
     if (L.g.ring_stages == 0 && EPI == EPI_RESID_TP && L.g.tp.exchange && L.g.batches > 1) stages = 3;
     switch (bn) {
