@@ -32,7 +32,7 @@ GEMM_KINDS = ("gemm_qkv", "gemm_o_proj", "gemm_gate_up", "gemm_down")
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the projection GEMM (average of the four
 # launches of a block), from the ncu capture summarised in profiles/dram_decode_kernels_c2.md.  Valid for
 # that workload with automatic tuning only; set to None when the kernel changes until it is captured again.
-NCU_TRAFFIC_PER_LAUNCH = {"c2": 101.98e6}
+NCU_TRAFFIC_PER_LAUNCH = {"c2": 101.86e6}
 
 
 def measured_peaks():
