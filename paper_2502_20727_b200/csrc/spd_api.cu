@@ -670,7 +670,7 @@ int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, 
             g.n_weights = 3; g.w_rows[0] = qd / nl; g.w_rows[1] = g.w_rows[2] = kd / nl;
             g.num_kb = cdiv(H, 64);
             g.splits = decode_splits((long)decode_tiles_per_batch(EPI_QKV, g.w_rows, 3) * nl * tok_tiles, g.num_kb,
-                                     c->split_override[SITE_QKV], 8);
+                                     c->split_override[SITE_QKV], 8, tbox == 16 ? 3 : 2);
             g.ss_in = SumSq{(const float *)(r0 + TL.ss_attn), h_tiles, 1, Mb, H, d.rms_eps};
             g.rope = rope ? c->rope : nullptr; g.q_out = c->q; g.k_pages = w.k_pages; g.v_pages = w.v_pages; g.pt = pt; g.tm = tm;
             g.n_q_heads = d.n_q_heads; g.head_dim = d.head_dim;
@@ -699,7 +699,7 @@ int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, 
             MAP_OR_FAIL(am, act_map(c, AB_ATTN_SHARD, tbox));
             g.w_rows[0] = H;
             g.num_kb = cdiv(qd / nl, 64);
-            g.splits = decode_splits((long)h_tiles * nl * tok_tiles, g.num_kb, c->split_override[SITE_O], 8);
+            g.splits = decode_splits((long)h_tiles * nl * tok_tiles, g.num_kb, c->split_override[SITE_O], 8, tbox == 16 ? 3 : 2);
             g.res_in = (const float *)(r0 + TL.res0); g.gain = w.mlp_norm; g.hg = r0 + TL.hg; g.ss_out = (float *)(r0 + TL.ss_mlp);
             if (sync) { with_exchange(g, l, 0); g.res_out = (float *)(r0 + TL.res1); }
             else g.tp.ysave = (float *)(r0 + TL.ysave);
@@ -711,7 +711,7 @@ int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, 
             g.n_weights = 2; g.w_rows[0] = g.w_rows[1] = Fs;
             g.num_kb = cdiv(H, 64);
             g.splits = decode_splits((long)decode_tiles_per_batch(EPI_GATEUP, g.w_rows, 2) * nl * tok_tiles, g.num_kb,
-                                     c->split_override[SITE_GU], 8);
+                                     c->split_override[SITE_GU], 8, tbox == 16 ? 3 : 2);
             g.ss_in = SumSq{(const float *)(r0 + TL.ss_mlp), h_tiles, 1, Mb, H, d.rms_eps};
             g.act = c->act; g.F = F; g.Fs = Fs;
             LAUNCH(K_GATE_UP, launch_gemm_decode(EPI_GATEUP, wmaps, *hmap, g, st));
@@ -722,7 +722,7 @@ int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, 
             MAP_OR_FAIL(am, act_map(c, AB_ACT_SHARD, tbox));
             g.w_rows[0] = H;
             g.num_kb = cdiv(Fs, 64);
-            g.splits = decode_splits((long)h_tiles * nl * tok_tiles, g.num_kb, c->split_override[SITE_DOWN], 8);
+            g.splits = decode_splits((long)h_tiles * nl * tok_tiles, g.num_kb, c->split_override[SITE_DOWN], 8, tbox == 16 ? 3 : 2);
             with_exchange(g, l, 1);
             g.res_in = (const float *)(r0 + (sync ? TL.res1 : TL.res0));
             if (!sync) g.tp.addend = (const float *)(r0 + TL.ysave);
