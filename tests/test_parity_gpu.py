@@ -233,3 +233,23 @@ def test_prefill_attention_long_prompt_many_key_tiles():
     assert rel_err(got, ref) <= TOL["bf16"]
     assert p.stack.device_error() == 0
     p.stack.close()
+
+
+@pytest.mark.parametrize("stages", [3, 4, 5])
+def test_decode_ring_depth_is_only_a_schedule(stages):
+    """The weight tiles of a decode projection stream through a ring of 3, 4 or 5 stages (chosen per launch by
+    default): any depth gives the same numbers, bit for bit."""
+    w = si.Workload("ring", "bf16", 2, 1024, 8, 4, 128, 2752, 4, (0, 1), 5, 40, 2)
+    outs = []
+    for st in (0, stages):
+        p = Pair(w, mask=(0, 1), B=5, max_len=48)
+        p.fill_cache(np.array([40, 7, 16, 33, 1], dtype=np.int32))
+        p.stack.set_tuning(decode_ring_stages=st)
+        got, ref = p.decode(0)
+        assert rel_err(got, ref) <= TOL["bf16"]
+        got2, ref2 = p.decode(1)
+        assert rel_err(got2, ref2) <= TOL["bf16"]
+        assert p.stack.device_error() == 0
+        outs.append((got, got2))
+        p.stack.close()
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
