@@ -712,26 +712,31 @@ __global__ void __launch_bounds__(128) decode_prologue_kernel(PrologueArgs a, in
         a.rope_table[i] = make_float2((float)cs, (float)sn);
         return;
     }
-    __shared__ float sm[4];
     const long zoff = (long)blockIdx.y * a.z_stride;
     float *res_out = (float *)((char *)a.res_out + zoff), *ss_out = (float *)((char *)a.ss_out + zoff);
     bf16 *hg = (bf16 *)((char *)a.hg + zoff);
     if (a.step && blockIdx.x == 0 && threadIdx.x == 0) *(unsigned *)((char *)a.step + zoff) += 1u;
-    const int r = threadIdx.x, warp = r >> 5, lane = r & 31, n = blockIdx.x * 128 + r;
-    const bool valid = n < a.H;
-    const float gn = valid ? __bfloat162float(((const bf16 *)a.gain)[n]) : 0.f;
-    for (int m = 0; m < a.M; ++m) {
+    // warp w takes tokens w, w+4, ...; lane l the columns 4l .. 4l+3 of the block's 128: no block-wide barrier
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n = blockIdx.x * 128 + 4 * lane;
+    const bool valid = n < a.H; // H is a multiple of 4
+    float4 gn = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (valid) {
+        const uint2 u = *(const uint2 *)((const bf16 *)a.gain + n);
+        const float2 g0 = __bfloat1622float2(*(const __nv_bfloat162 *)&u.x), g1 = __bfloat1622float2(*(const __nv_bfloat162 *)&u.y);
+        gn = make_float4(g0.x, g0.y, g1.x, g1.y);
+    }
+    for (int m = warp; m < a.M; m += 4) {
         const long idx = (long)m * a.H + n;
-        const float x = valid ? __bfloat162float(((const bf16 *)a.x)[idx]) : 0.f;
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
         if (valid) {
-            res_out[idx] = x;
-            hg[idx] = __float2bfloat16_rn(x * gn);
+            const uint2 u = *(const uint2 *)((const bf16 *)a.x + idx);
+            const float2 x0 = __bfloat1622float2(*(const __nv_bfloat162 *)&u.x), x1 = __bfloat1622float2(*(const __nv_bfloat162 *)&u.y);
+            x = make_float4(x0.x, x0.y, x1.x, x1.y);
+            *(float4 *)(res_out + idx) = x;
+            store_bf16x4(hg + idx, x, gn);
         }
-        const float q = warp_sum(x * x);
-        __syncthreads();
-        if (lane == 0) sm[warp] = q;
-        __syncthreads();
-        if (r == 0) ss_out[(long)blockIdx.x * a.Mcap + m] = sm[0] + sm[1] + sm[2] + sm[3];
+        const float q = warp_sum(sq4(x));
+        if (lane == 0) ss_out[(long)blockIdx.x * a.Mcap + m] = q;
     }
 }
 
