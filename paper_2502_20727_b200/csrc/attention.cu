@@ -669,8 +669,11 @@ __global__ void __launch_bounds__(128) decode_attention_kernel(AttnArgs a)
 // independent of the arithmetic, and pages that hold only earlier steps' tokens are requested
 // before the dependency wait (only the page receiving this step's token is written by the
 // preceding kernel).  grid (n_q_heads / GT, B, splits); GT query heads share the KV head.
-template <typename T, int D, int GT>
-__global__ void __launch_bounds__(160) decode_attention_ring_kernel(AttnArgs a)
+// DENSE: compiled for five resident blocks per SM instead of four (72 registers); each block is a little slower,
+// but a launch of 593-740 blocks (16 sequences x 40 heads, say) is resident at once instead of leaving a short
+// second wave - chosen by the launcher.
+template <typename T, int D, int GT, bool DENSE>
+__global__ void __launch_bounds__(160, DENSE ? 5 : 4) decode_attention_ring_kernel(AttnArgs a)
 {
     using namespace tc;
     constexpr int E = Row16<T>::E, LPT = D / E, TPW = 32 / LPT, BLK = 16, NG = BLK / TPW;
@@ -844,16 +847,16 @@ __global__ void __launch_bounds__(160) decode_attention_ring_kernel(AttnArgs a)
     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_END);
 }
 
-template <typename T, int D, int GT> cudaError_t launch_ring(const AttnArgs &a, cudaStream_t st)
+template <typename T, int D, int GT, bool DENSE> cudaError_t launch_ring_as(const AttnArgs &a, cudaStream_t st)
 {
     constexpr int PAGE_BYTES = 16 * D * (int)sizeof(T), R = DecodeRing<T, D>::SLOTS;
     constexpr int SMEM = R * 2 * PAGE_BYTES + 4 * GT * D * 4 + 4 * GT * 2 * 4 + 2 * R * 8 + (DECODE_MAX_PAGES_PER_BLOCK + 2 + 2 * GT) * 4;
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(decode_attention_ring_kernel<T, D, GT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+        cudaError_t e = cudaFuncSetAttribute(decode_attention_ring_kernel<T, D, GT, DENSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
         if (e != cudaSuccess) return e;
-        // ask for the largest shared-memory carve-out so that four blocks fit an SM
-        e = cudaFuncSetAttribute(decode_attention_ring_kernel<T, D, GT>, cudaFuncAttributePreferredSharedMemoryCarveout,
+        // ask for the largest shared-memory carve-out so that four (five) blocks fit an SM
+        e = cudaFuncSetAttribute(decode_attention_ring_kernel<T, D, GT, DENSE>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                  (int)cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         attr_done = true;
@@ -861,7 +864,17 @@ template <typename T, int D, int GT> cudaError_t launch_ring(const AttnArgs &a, 
     dim3 grid(a.n_q_heads / GT, a.B, a.splits);
     AttnArgs b = a;
     b.cluster_merge = a.splits > 1 && a.splits <= 8;
-    return launch_kernel_z(decode_attention_ring_kernel<T, D, GT>, grid, dim3(160), SMEM, st, b.cluster_merge ? a.splits : 1, b);
+    return launch_kernel_z(decode_attention_ring_kernel<T, D, GT, DENSE>, grid, dim3(160), SMEM, st, b.cluster_merge ? a.splits : 1, b);
+}
+
+template <typename T, int D, int GT> cudaError_t launch_ring(const AttnArgs &a, cudaStream_t st)
+{
+    // five blocks per SM where that saves a wave (one query head per block only: the wider blocks would spill)
+    constexpr int SMS = 148;
+    const long blocks = (long)(a.n_q_heads / GT) * a.B * a.splits;
+    const bool dense = GT == 1 && (blocks + 5 * SMS - 1) / (5 * SMS) < (blocks + 4 * SMS - 1) / (4 * SMS);
+    if (GT == 1 && dense) return launch_ring_as<T, D, 1, true>(a, st);
+    return launch_ring_as<T, D, GT, false>(a, st);
 }
 
 // ---------------------------------------------------------------------------------------
