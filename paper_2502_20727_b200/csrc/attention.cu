@@ -885,8 +885,10 @@ template <typename T, int D, int GT> cudaError_t launch_ring(const AttnArgs &a, 
 // Pages arrive through TMA tensor copies (4 boxes of 64 dims x 16 tokens per page: K and V,
 // low and high half of the head dimension) in the 128-byte swizzle that ldmatrix reads without
 // bank conflicts.  Warp roles, page ring, split merge: as in the bulk-copy kernel.
-template <int GT>
-__global__ void __launch_bounds__(160) decode_attention_mma_kernel(const __grid_constant__ CUtensorMap tm_k,
+// DENSE: compiled for four resident blocks per SM instead of three (96 registers), taken by the launcher where it
+// saves a wave.
+template <int GT, bool DENSE>
+__global__ void __launch_bounds__(160, DENSE ? 4 : 3) decode_attention_mma_kernel(const __grid_constant__ CUtensorMap tm_k,
                                                                    const __grid_constant__ CUtensorMap tm_v, AttnArgs a)
 {
     using namespace tc;
@@ -1051,20 +1053,28 @@ __global__ void __launch_bounds__(160) decode_attention_mma_kernel(const __grid_
     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_END);
 }
 
-template <int GT> cudaError_t launch_decode_mma(const AttnArgs &a, cudaStream_t st)
+template <int GT, bool DENSE> cudaError_t launch_decode_mma_as(const AttnArgs &a, cudaStream_t st)
 {
     constexpr int SMEM = 1024 + 4 * 8192 + 4 * GT * 128 * 4 + 4 * GT * 2 * 4 + 2 * 4 * 8 + (DECODE_MAX_PAGES_PER_BLOCK + 2 + 2 * GT) * 4;
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(decode_attention_mma_kernel<GT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+        cudaError_t e = cudaFuncSetAttribute(decode_attention_mma_kernel<GT, DENSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
     dim3 grid(a.n_q_heads / GT, a.B, a.splits);
     AttnArgs b = a;
     b.cluster_merge = a.splits > 1 && a.splits <= 8;
-    return launch_kernel_z(decode_attention_mma_kernel<GT>, grid, dim3(160), SMEM, st, b.cluster_merge ? a.splits : 1,
+    return launch_kernel_z(decode_attention_mma_kernel<GT, DENSE>, grid, dim3(160), SMEM, st, b.cluster_merge ? a.splits : 1,
                            *(const CUtensorMap *)a.k_map, *(const CUtensorMap *)a.v_map, b);
+}
+
+template <int GT> cudaError_t launch_decode_mma(const AttnArgs &a, cudaStream_t st)
+{
+    constexpr int SMS = 148;
+    const long blocks = (long)(a.n_q_heads / GT) * a.B * a.splits;
+    if ((blocks + 4 * SMS - 1) / (4 * SMS) < (blocks + 3 * SMS - 1) / (3 * SMS)) return launch_decode_mma_as<GT, true>(a, st);
+    return launch_decode_mma_as<GT, false>(a, st);
 }
 
 template <typename T, int D> cudaError_t launch_decode_d(const AttnArgs &a, cudaStream_t st)
