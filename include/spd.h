@@ -96,7 +96,10 @@ int spd_workspace_bytes(const spd_dims *dims, const uint8_t *sync_mask, size_t *
  *   n_pages   : pages in every k_pages / v_pages tensor (block-table entries are checked
  *               against it on the device)
  *   workspace : device memory, 256-byte aligned, >= spd_workspace_bytes(); borrowed until
- *               spd_destroy; must not be shared by contexts running concurrently
+ *               spd_destroy; must not be shared by contexts running concurrently.  spd_create
+ *               zeroes it (error flag, arrival counters, pad rows) between two device-wide
+ *               synchronisations and returns only when that has completed, so the first call
+ *               may use any stream.  A set-up call: not to be made during a stream capture.
  * Requires a CUDA device of compute capability 10.x as the current device.
  * Errors: SPD_ENULL, SPD_EINVAL, SPD_EWORKSPACE, SPD_ECUDA. */
 int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *layers,
@@ -159,6 +162,11 @@ int spd_set_graphs(spd_ctx *ctx, int32_t enabled);
  *       when the maximum has grown by more than 2^value since the last rescale (default 8, at
  *       most 16; 0 = follow the maximum exactly, every growth rescales).  The result is the same
  *       softmax either way; only the rounding of the bf16 probabilities differs.
+ *   "peer_wait_ms"
+ *       rank mode (spd_tp_*): milliseconds a rank waits for the other ranks' partial sums before
+ *       it gives up with error bit 8 (default and value 0: 1000; at most 60000).  Always bounded.
+ *       Raise it where the ranks' hosts can be skewed by more than a second (a rank that is still
+ *       instantiating its graph), lower it to fail fast.
  * Errors: SPD_ENULL, SPD_EINVAL (unknown key, negative value). */
 int spd_set_tuning(spd_ctx *ctx, const char *key, int32_t value);
 
@@ -295,7 +303,7 @@ int spd_tp_detach(spd_ctx *ctx);
  * ranks hold bit-identical residual streams.  A TP block exchanges twice (Y_i after o_proj,
  * Z_i after down: Sec. 3), an SPD block once (Y_i + Z_i after down: Sec. 4.1.1).
  *   out : [ranks held by the context][B][hidden] bf16 - every rank's copy of the output
- * A wait for a peer gives up after about one second: the kernels then return normally, the
+ * A wait for a peer gives up after about one second ("peer_wait_ms" of spd_set_tuning): the kernels then return normally, the
  * step's output is undefined and spd_device_error reports bit 8; the context stays usable.
  * Errors: SPD_ENULL, SPD_EINVAL (not attached, B > max_batch), SPD_ECAPACITY, SPD_ECUDA. */
 int spd_tp_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_lens,

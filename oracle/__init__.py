@@ -158,6 +158,25 @@ def block_forward(dims: Dims, layer, mode: int, x, pos0, cache: Cache, layer_ind
     return out, y, rc
 
 
+def stack_forward_streamed(dims: Dims, mask, layer_source, x, pos0, cache: Cache, want_layers: bool = False):
+    """The masked stack of ``stack_forward`` with the weights supplied one layer at a time:
+    ``layer_source(l)`` returns the dict of layer l, which is dropped again before layer l+1 is
+    asked for, so a deep stack of wide layers never sits in host memory as a whole.  Block l's
+    output is block l+1's input, nothing else (Algorithm 1's block list, run in order).
+
+    Returns (out [B,S,H], sync_points, layer_out [L, B*S, H] or None)."""
+    cur = np.ascontiguousarray(x, dtype=np.float64)
+    B, S, H = cur.shape
+    lo = np.empty((dims.n_layers, B * S, H), dtype=np.float64) if want_layers else None
+    syncs = 0
+    for l in range(dims.n_layers):
+        cur, _, n = block_forward(dims, layer_source(l), 1 if mask[l] else 0, cur, pos0, cache, layer_index=l)
+        syncs += n
+        if lo is not None:
+            lo[l] = cur.reshape(B * S, H)
+    return cur, syncs, lo
+
+
 def rmsnorm(x, g, eps):
     x = np.ascontiguousarray(x, dtype=np.float64)
     g = _f32(g)

@@ -870,7 +870,7 @@ template <typename T, int D, int GT, bool DENSE> cudaError_t launch_ring_as(cons
 template <typename T, int D, int GT> cudaError_t launch_ring(const AttnArgs &a, cudaStream_t st)
 {
     // five blocks per SM where that saves a wave (one query head per block only: the wider blocks would spill)
-    constexpr int SMS = 148;
+    const long SMS = sm_count();
     const long blocks = (long)(a.n_q_heads / GT) * a.B * a.splits;
     const bool dense = GT == 1 && (blocks + 5 * SMS - 1) / (5 * SMS) < (blocks + 4 * SMS - 1) / (4 * SMS);
     if (GT == 1 && dense) return launch_ring_as<T, D, 1, true>(a, st);
@@ -1071,7 +1071,7 @@ template <int GT, bool DENSE> cudaError_t launch_decode_mma_as(const AttnArgs &a
 
 template <int GT> cudaError_t launch_decode_mma(const AttnArgs &a, cudaStream_t st)
 {
-    constexpr int SMS = 148;
+    const long SMS = sm_count();
     const long blocks = (long)(a.n_q_heads / GT) * a.B * a.splits;
     if ((blocks + 4 * SMS - 1) / (4 * SMS) < (blocks + 3 * SMS - 1) / (3 * SMS)) return launch_decode_mma_as<GT, true>(a, st);
     return launch_decode_mma_as<GT, false>(a, st);

@@ -16,6 +16,12 @@ enum : int {
     ERR_PEER_TIMEOUT = 8, // a bounded wait for another rank's partial sums gave up
 };
 
+// Remember a failing CUDA call for spd_last_cuda_error() (per thread); used by every file that returns SPD_ECUDA.
+void note_cuda_error(cudaError_t e);
+// Streaming multiprocessors of the current device (queried once per device; 148, the B200's count, when there is
+// no device to ask, as in host-only calls).  Launch shapes and split counts are sized from it.
+int sm_count();
+
 template <typename T> __device__ __forceinline__ float to_f(T v);
 template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ float to_f<bf16>(bf16 v) { return __bfloat162float(v); }

@@ -39,7 +39,6 @@ using namespace tc;
 constexpr int MAX_GROUPS = 8; // emulated devices
 constexpr int MAX_P = 8;      // portable cluster size
 constexpr int THREADS = 192;
-constexpr int N_SM_DECODE = 148; // SMs the ring-depth rule is tuned for
 
 // ST = stages of the operand ring.  What a launch needs in flight to keep HBM busy is about 16 MB over all of its
 // blocks (bandwidth x loaded latency): launches of 250-450 blocks want four stages (72-98 KB per block, three or two
@@ -333,7 +332,6 @@ __device__ __forceinline__ unsigned long long global_ns()
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-constexpr unsigned long long PEER_WAIT_NS = 1000000000ull; // one second
 
 // Rank z's partial rows (its K ranges added up through the cluster), optionally exchanged with the
 // other ranks and summed in rank order, then the residual, the gain-scaled input of the next GEMM
@@ -409,7 +407,7 @@ __device__ __forceinline__ void epilogue_resid_tp(const DecGemmArgs &g, const De
                 if (e % TP_FLAG_RANGES < t.P && (int)(ld_acquire_sys(mine + e) - step) < 0) done = false;
             if (__all_sync(0xffffffffu, done)) break;
             // a rank that never arrives (or an earlier give-up in this step) ends the wait: no trap, the host reads the flag
-            if (*abort_flag || (*(volatile int *)g.err & ERR_PEER_TIMEOUT) || global_ns() - t0 > PEER_WAIT_NS) {
+            if (*abort_flag || (*(volatile int *)g.err & ERR_PEER_TIMEOUT) || global_ns() - t0 > g.tp.wait_ns) {
                 if (lane == 0) { *abort_flag = 1; atomicOr(g.err, ERR_PEER_TIMEOUT); }
                 break;
             }
@@ -677,7 +675,8 @@ cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
     // launch resident at once); four stages at 32- and 64-token tiles
     const long blocks = (long)grid.x * grid.y * grid.z;
     int stages = L.g.ring_stages;
-    if (stages == 0) stages = (bn == 16 && blocks > 3L * N_SM_DECODE) ? 3 : ((bn == 16 && blocks <= 2L * N_SM_DECODE) ? 5 : 4);
+    const long n_sm = sm_count();
+    if (stages == 0) stages = (bn == 16 && blocks > 3L * n_sm) ? 3 : ((bn == 16 && blocks <= 2L * n_sm) ? 5 : 4);
     // several ranks in one launch wait on one another: as many resident blocks as possible
     if (L.g.ring_stages == 0 && EPI == EPI_RESID_TP && L.g.tp.exchange && L.g.batches > 1) stages = 3;
     switch (bn) {

@@ -41,6 +41,7 @@ struct TpArgs {
     char *rx[TP_MAX_RANKS];        // rank j's receive buffers (buffer 0 first)
     unsigned *flags[TP_MAX_RANKS]; // rank j's flag words of this exchange: [tile][token tile][source][TP_FLAG_RANGES]
     const unsigned *step;  // step number (> 0, same on all ranks)
+    unsigned long long wait_ns; // how long a rank waits for its peers' rows before it gives up (error bit 8)
     const float *addend;   // fp32 [Mcap][H] added to the partial before the exchange (Y_i of an SPD block), or null
     float *ysave;          // fp32 [Mcap][H]: the partial is kept here (Y_i), or null
 };

@@ -5,6 +5,7 @@
 #include "common.cuh"
 #include "gemm_tc.cuh"
 
+#include <initializer_list>
 #include <mutex>
 
 using namespace spd;
@@ -41,12 +42,18 @@ extern "C" int spd_gemm_bf16_sum_static(const void *a, const void *w, float *c, 
 {
     if (!a || !w || !c || !err_flag) return SPD_ENULL;
     if (M < 1 || N < 1 || K < 8 || K % 8 || batches < 1 || splits < 1 || splits > (K + 63) / 64) return SPD_EINVAL;
+    // factor by factor, so that no product of the four 32-bit sizes can wrap before it is compared
+    size_t room = SCRATCH_FLOATS;
+    for (const int32_t f : {M, batches, N, splits}) {
+        if ((size_t)f > room) return SPD_EWORKSPACE;
+        room /= (size_t)f;
+    }
     const size_t plane_elems = (size_t)M * (size_t)batches * (size_t)N;
-    if (plane_elems > SCRATCH_FLOATS || plane_elems * (size_t)splits > SCRATCH_FLOATS) return SPD_EWORKSPACE;
 
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return SPD_ECUDA;
+    if (e != cudaSuccess) { note_cuda_error(e); return SPD_ECUDA; }
+    if (dev < 0 || dev >= MAX_DEVICES) { note_cuda_error(cudaErrorInvalidDevice); return SPD_ECUDA; }
     float *planes = nullptr;
     {
         // once per device, with that device current: resolve the array's device address
@@ -54,7 +61,7 @@ extern "C" int spd_gemm_bf16_sum_static(const void *a, const void *w, float *c, 
         if (!g_planes_of_device[dev]) {
             float *p = nullptr;
             e = cudaGetSymbolAddress((void **)&p, g_static_planes);
-            if (e != cudaSuccess || !p) return SPD_ECUDA;
+            if (e != cudaSuccess || !p) { note_cuda_error(e != cudaSuccess ? e : cudaErrorInvalidSymbol); return SPD_ECUDA; }
             g_planes_of_device[dev] = p;
         }
         planes = g_planes_of_device[dev];
@@ -70,11 +77,10 @@ extern "C" int spd_gemm_bf16_sum_static(const void *a, const void *w, float *c, 
     g.num_kb = (K + 63) / 64; g.splits = splits; g.err = err_flag;
     const TcMap *wmaps[1] = {&wm};
     cudaStream_t st = (cudaStream_t)stream;
-    if (launch_gemm_tc(wmaps, 1, am, g, swap != 0, st) != cudaSuccess) return SPD_ECUDA;
+    if ((e = launch_gemm_tc(wmaps, 1, am, g, swap != 0, st)) != cudaSuccess) { note_cuda_error(e); return SPD_ECUDA; }
     // Every element the sum reads was written by the launch above, so nothing has to be cleared.
     const unsigned blocks = (unsigned)((plane_elems + 255) / 256);
-    if (launch_kernel(sum_planes_kernel, dim3(blocks), dim3(256), 0, st, 0, (const float *)planes, c, (long)plane_elems,
-                      (int)splits) != cudaSuccess)
-        return SPD_ECUDA;
+    e = launch_kernel(sum_planes_kernel, dim3(blocks), dim3(256), 0, st, 0, (const float *)planes, c, (long)plane_elems, (int)splits);
+    if (e != cudaSuccess) { note_cuda_error(e); return SPD_ECUDA; }
     return SPD_OK;
 }

@@ -15,6 +15,18 @@ using namespace spd;
 
 static thread_local int g_last_cuda_error = 0;
 
+void spd::note_cuda_error(cudaError_t e) { g_last_cuda_error = (int)e; }
+
+int spd::sm_count()
+{
+    static int cached[64] = {};
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return 148; }
+    if (cached[dev]) return cached[dev];
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) { cudaGetLastError(); return 148; }
+    return cached[dev] = n;
+}
+
 #define CU_TRY(expr)                                                   \
     do {                                                               \
         cudaError_t e__ = (expr);                                      \
@@ -22,8 +34,6 @@ static thread_local int g_last_cuda_error = 0;
     } while (0)
 
 namespace {
-
-constexpr int N_SM = 148;
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline int cdiv(int a, int b) { return (a + b - 1) / b; }
@@ -45,7 +55,7 @@ int fit_splits(int K, int want, int align)
 
 int want_splits(long tiles, int cap)
 {
-    long s = (2 * N_SM + tiles - 1) / tiles;
+    long s = (2 * sm_count() + tiles - 1) / tiles;
     if (s > cap) s = cap;
     return (int)(s < 1 ? 1 : s);
 }
@@ -116,6 +126,7 @@ struct Ctx {
     int l2_prefetch_kb;          // K blocks per thread block prefetched into L2 by the decode GEMMs
     int ring_stages;             // decode GEMMs: stages of the operand ring (0 = per launch)
     int prefill_rescale_log2;    // tcgen05 prefill attention: growth of the row maximum (log2) that triggers a rescale
+    int peer_wait_ms;            // rank mode: how long a rank waits for its peers' partial sums
     int launches_last;
     TpState tp;
     // activation tensor maps, by buffer and token box (16, 32, 64, 128), built on first use
@@ -186,7 +197,7 @@ Plan make_plan(const spd_dims &d, int M, bool decode, int max_context, int attn_
                                                                                            : decode_heads_per_block(group);
         const long ctas = (long)M * (d.n_q_heads / gt);
         const int pages = cdiv(max_context, 16);
-        int s = attn_override > 0 ? attn_override : (int)((4L * N_SM) / ctas);
+        int s = attn_override > 0 ? attn_override : (int)((4L * sm_count()) / ctas);
         if (s < 1) s = 1;
         if (s > pages / 4) s = pages / 4;
         if (s > 32) s = 32;
@@ -206,7 +217,7 @@ Plan make_plan(const spd_dims &d, int M, bool decode, int max_context, int attn_
 // cluster of at most 8 blocks).
 int decode_splits(long tiles, int num_kb, int override_, int max_ranges, int blocks_per_sm = 3)
 {
-    long s = override_ > 0 ? override_ : ((long)blocks_per_sm * N_SM) / (tiles < 1 ? 1 : tiles);
+    long s = override_ > 0 ? override_ : ((long)blocks_per_sm * sm_count()) / (tiles < 1 ? 1 : tiles);
     const long cap = num_kb / 4 < 1 ? 1 : num_kb / 4;
     if (s > cap) s = cap;
     if (s > max_ranges) s = max_ranges;
@@ -648,6 +659,7 @@ int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, 
         g.ring_stages = c->ring_stages;
         g.tp.on = 1; g.tp.T = tp.T; g.tp.rank_base = tp.rank_base; g.tp.z_stride = tp.z_stride;
         g.tp.step = (const unsigned *)(r0 + TL.step);
+        g.tp.wait_ns = (unsigned long long)c->peer_wait_ms * 1000000ull;
         return g;
     };
     int exchange = 0;
@@ -1042,6 +1054,7 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     for (int i = 0; i < SITE_COUNT; ++i) c.split_override[i] = 0;
     c.l2_prefetch_kb = 0;
     c.prefill_rescale_log2 = 8;
+    c.peer_wait_ms = 1000;
     c.ring_stages = 0;
     c.launches_last = 0;
     c.tp.on = false;
@@ -1055,8 +1068,14 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
         rc = build_weight_maps(c);
         if (rc) { delete h; return rc; }
     }
-    // zero the workspace once: token rows beyond a launch's M are read (never used) by tiled loads
-    cudaError_t e = cudaMemset(workspace, 0, L.total);
+    // Zero the workspace once: the error flag, the arrival counters of the attention merge, and token rows
+    // beyond a launch's M that tiled loads read (never use).  A memset of device memory returns before it
+    // has run and is ordered only with the legacy default stream, while the caller's allocator and every
+    // later call work on other (possibly non-blocking) streams: wait for the device on both sides, so that
+    // neither an earlier user of this memory nor a first kernel can overlap the zeroing.
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemset(workspace, 0, L.total);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { g_last_cuda_error = (int)e; delete h; return SPD_ECUDA; }
     *out = h;
     return SPD_OK;
@@ -1223,6 +1242,7 @@ int spd_set_tuning(spd_ctx *ctx, const char *key, int32_t value)
     if (!strcmp(key, "decode_ring_stages")) { c.ring_stages = (value == 0 || (value >= 3 && value <= 5)) ? value : 0; found = true; }
     if (!strcmp(key, "prefill_rescale_log2")) { c.prefill_rescale_log2 = value > 16 ? 16 : value; found = true; }
     if (!strcmp(key, "l2_prefetch_blocks")) { c.l2_prefetch_kb = value > 64 ? 64 : value; found = true; }
+    if (!strcmp(key, "peer_wait_ms")) { c.peer_wait_ms = value < 1 ? 1000 : (value > 60000 ? 60000 : value); found = true; }
     if (!found) return SPD_EINVAL;
     for (GraphEntry &g : c.graphs) cudaGraphExecDestroy(g.exec); // captured steps used the old setting
     c.graphs.clear();
@@ -1303,7 +1323,7 @@ int spd_tp_prefill(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int3
     // block of an exchange launch resident (three blocks per SM, one block per 128 columns, rank and 64 tokens).
     long chunk = c.tp.L.Mb;
     if (d.T > 1) {
-        const long tiles = (long)cdiv(d.hidden, 128) * d.T, fit = (3L * N_SM) / tiles;
+        const long tiles = (long)cdiv(d.hidden, 128) * d.T, fit = (3L * sm_count()) / tiles;
         if (fit < 1) { g_last_cuda_error = (int)cudaErrorCooperativeLaunchTooLarge; return SPD_ECUDA; }
         if (fit * 64 < chunk) chunk = fit * 64;
     }

@@ -32,7 +32,11 @@ class Pair:
     """One workload instantiated on both sides."""
 
     def __init__(self, w: si.Workload, *, mask=None, B=None, max_len=None, max_prefill_tokens=None, seed=0,
-                 device="cuda:0", n_pages=None, layers=None):
+                 device="cuda:0", n_pages=None, layers=None, weights_on="cpu", stream_oracle=False):
+        """weights_on: where the seeded generator of ``spd_inputs`` draws the weights ("cpu", or the CUDA
+        device for wide layers: torch's device generator, seconds instead of minutes per 70B-shaped layer).
+        stream_oracle: the oracle gets the layers one at a time (up-cast copies of one layer in host memory
+        instead of the whole stack)."""
         import paper_2502_20727_b200 as spd
         # a non-default stream: the legacy default stream cannot be captured into the graphs
         # that replay decode steps
@@ -45,9 +49,10 @@ class Pair:
         self.max_len = max_len or (w.prompt + w.decode_steps)
         self.mask = list(w.mask if mask is None else mask)
         self.device = device
-        self.layers = layers if layers is not None else si.make_stack(w, "cpu", seed)
+        self.layers = layers if layers is not None else si.make_stack(w, weights_on, seed)
         self.layers_gpu = [{n: t.to(device) for n, t in lw.items()} for lw in self.layers]
-        self.layers_np = si.to_oracle_layers(self.layers)
+        self.layers_np = None if stream_oracle else si.to_oracle_layers(self.layers)
+        self.layer_out = None  # the oracle's per-layer outputs of the last call made with want_layers
         self.dims = oracle_dims(w)
         self.cache = oracle.Cache(self.dims, self.B, self.max_len)
         pages_per_seq = (self.max_len + w.kv_block - 1) // w.kv_block
@@ -58,16 +63,21 @@ class Pair:
                                              max_prefill_tokens=max_prefill_tokens or 4096, device=device)
         self.pos = np.zeros(self.B, dtype=np.int32)
 
-    def _oracle(self, x):
+    def _oracle(self, x, want_layers=False):
         """The oracle's forward pass of the workload's block kind: (out, sync_points)."""
         if getattr(self.w, "block", "llama") == "opt":
             return oracle.bias_stack_forward(self.dims, self.mask, self.layers_np, x, self.pos, self.cache)
-        out, syncs, _ = oracle.stack_forward(self.dims, self.mask, self.layers_np, x, self.pos, self.cache)
+        if self.layers_np is None:
+            out, syncs, self.layer_out = oracle.stack_forward_streamed(
+                self.dims, self.mask, lambda l: si.to_oracle_layers([self.layers[l]])[0], x, self.pos, self.cache, want_layers)
+        else:
+            out, syncs, self.layer_out = oracle.stack_forward(self.dims, self.mask, self.layers_np, x, self.pos, self.cache,
+                                                              want_layers)
         return out, syncs
 
-    def prefill(self, S, seed=0):
+    def prefill(self, S, seed=0, want_layers=False):
         x = si.make_hidden(self.w, (self.B, S, self.w.hidden), "cpu", seed, 0)
-        ref, syncs = self._oracle(to_np(x))
+        ref, syncs = self._oracle(to_np(x), want_layers)
         got = self.stack.prefill(x.to(self.device), self.block_table)
         torch.cuda.synchronize()
         self.pos = self.pos + S
@@ -88,6 +98,22 @@ class Pair:
         torch.cuda.synchronize()
         self.pos = self.pos + 1
         return to_np(got), ref[:, 0, :]
+
+    def prefix_prefill(self, depth, S, seed=0):
+        """The GPU's output after the first `depth` blocks for the prompts of prefill(S, seed): a second context
+        over the same weight tensors and block table with pages of its own (compare with layer_out[depth - 1])."""
+        import paper_2502_20727_b200 as spd
+        w = self.w.with_(n_layers=depth, mask=tuple(self.mask[:depth]))
+        st = spd.stack_from_workload(w, self.layers_gpu[:depth], sync_mask=self.mask[:depth], max_batch=self.B,
+                                     max_seq_len=self.max_len, n_pages=self.n_pages, max_prefill_tokens=self.B * S,
+                                     device=self.device)
+        x = si.make_hidden(self.w, (self.B, S, self.w.hidden), "cpu", seed, 0)
+        got = st.prefill(x.to(self.device), self.block_table)
+        torch.cuda.synchronize()
+        err = st.device_error()
+        st.close()
+        assert err == 0
+        return to_np(got).reshape(self.B * S, self.w.hidden)
 
     def tp_prefill(self, S, seed=0):
         """Prompts in rank mode: every rank's output [T, B, S, H] and the oracle's."""

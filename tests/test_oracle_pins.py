@@ -354,6 +354,32 @@ def test_mask_is_honoured_per_layer():
         assert rel_err(a, b) > 1e-4
 
 
+def test_layer_streamed_stack_is_the_stack():
+    """Feeding the blocks one layer at a time (deep, wide stacks whose weights do not fit in host
+    memory at once) is the same chain of blocks: outputs, per-layer outputs, caches and the
+    sync-point count are bit-identical to the whole-stack routine, prompt and decode step alike."""
+    dims = Dims(5, T=4, **DIMS_GQA)
+    layers = [small_layer(dims, 60 + l) for l in range(5)]
+    mask = [1, 0, 0, 1, 0]
+    B, S = 2, 5
+    x, x1 = x_of(B, S, 32), x_of(B, 1, 32, seed=3)
+    ca, cb = Cache(dims, B, S + 1), Cache(dims, B, S + 1)
+    asked = []
+
+    def source(l):
+        asked.append(l)
+        return layers[l]
+
+    z = np.zeros(B, np.int32)
+    a = oracle.stack_forward(dims, mask, layers, x, z, ca, True)
+    b = oracle.stack_forward_streamed(dims, mask, source, x, z, cb, True)
+    assert asked == [0, 1, 2, 3, 4]
+    assert np.array_equal(a[0], b[0]) and a[1] == b[1] == 7 and np.array_equal(a[2], b[2])
+    a1 = oracle.stack_forward(dims, mask, layers, x1, np.full(B, S, np.int32), ca)
+    b1 = oracle.stack_forward_streamed(dims, mask, source, x1, np.full(B, S, np.int32), cb)
+    assert np.array_equal(a1[0], b1[0]) and np.array_equal(ca.k, cb.k) and np.array_equal(ca.v, cb.v)
+
+
 # ---------------------------------------------------------------- cache consistency
 
 @pytest.mark.parametrize("mask", [[1, 1], [0, 0], [0, 1]])

@@ -3,6 +3,8 @@ all T ranks of a group executed on one GPU - every launch covers all ranks' data
 sums are exchanges through per-rank receive planes and arrival flags in global memory, the same
 kernels and protocol a group of T GPUs runs over peer-mapped memory - against the CPU oracle's
 sharded block, element by element.  Bound: max|gpu-ref|/max|ref| <= 2e-2 (bfloat16)."""
+import time
+
 import numpy as np
 import pytest
 import torch
@@ -144,28 +146,31 @@ def test_a_rank_that_never_arrives_is_reported_not_waited_for():
     layers = si.make_stack(full, "cpu", 0)
     shard = [{n: t.to("cuda:0") for n, t in spd.shard_layer(lw, 0, 2).items()} for lw in layers]
     one = full.with_(n_q_heads=2, n_kv_heads=2, ffn=256, T=1)
-    stream = torch.cuda.Stream(device="cuda:0")
-    torch.cuda.set_stream(stream)
-    stack = spd.stack_from_workload(one, shard, sync_mask=mask, max_batch=2, max_seq_len=16, n_pages=4,
-                                    max_prefill_tokens=64, device="cuda:0")
-    nbytes = (stack.tp_region_bytes(2) + 1023) // 1024 * 1024
-    regions = torch.zeros(2 * nbytes + 1024, dtype=torch.uint8, device="cuda:0")
-    base = (regions.data_ptr() + 1023) // 1024 * 1024
-    stack.tp_attach(2, 0, [base, base + nbytes], nbytes)   # rank 1's region exists, but nobody plays rank 1
-    x = si.make_hidden(one, (2, one.hidden), "cpu", 0, 1).to("cuda:0")
-    seq = torch.zeros(2, dtype=torch.int32, device="cuda:0")
-    bt = torch.tensor([[0], [1]], dtype=torch.int32, device="cuda:0")
-    out = stack.tp_decode_step(x, seq, bt, 1)
-    torch.cuda.synchronize()
-    assert out.shape == (1, 2, 256)
-    assert stack.device_error() & 8
-    # usable afterwards: the ordinary single-GPU step of the shard's stack runs clean
-    stack.tp_detach()
-    y = stack.decode_step(x, seq, bt, 1)
-    torch.cuda.synchronize()
-    assert torch.isfinite(y.float()).all()
-    assert stack.device_error() == 0
-    stack.close()
+    with torch.cuda.stream(torch.cuda.Stream(device="cuda:0")):   # the previous current stream comes back afterwards
+        stack = spd.stack_from_workload(one, shard, sync_mask=mask, max_batch=2, max_seq_len=16, n_pages=4,
+                                        max_prefill_tokens=64, device="cuda:0")
+        nbytes = (stack.tp_region_bytes(2) + 1023) // 1024 * 1024
+        regions = torch.zeros(2 * nbytes + 1024, dtype=torch.uint8, device="cuda:0")
+        base = (regions.data_ptr() + 1023) // 1024 * 1024
+        stack.tp_attach(2, 0, [base, base + nbytes], nbytes)   # rank 1's region exists, but nobody plays rank 1
+        stack.set_tuning(peer_wait_ms=20)                      # the limit is a tuning key: fail fast here
+        x = si.make_hidden(one, (2, one.hidden), "cpu", 0, 1).to("cuda:0")
+        seq = torch.zeros(2, dtype=torch.int32, device="cuda:0")
+        bt = torch.tensor([[0], [1]], dtype=torch.int32, device="cuda:0")
+        t0 = time.perf_counter()
+        out = stack.tp_decode_step(x, seq, bt, 1)
+        torch.cuda.synchronize()
+        waited = time.perf_counter() - t0
+        assert out.shape == (1, 2, 256)
+        assert stack.device_error() & 8
+        assert waited < 0.5, f"gave up after {waited:.3f} s with a 20 ms limit"
+        # usable afterwards: the ordinary single-GPU step of the shard's stack runs clean
+        stack.tp_detach()
+        y = stack.decode_step(x, seq, bt, 1)
+        torch.cuda.synchronize()
+        assert torch.isfinite(y.float()).all()
+        assert stack.device_error() == 0
+        stack.close()
 
 
 def test_attach_argument_checks_and_mask_change_while_attached():

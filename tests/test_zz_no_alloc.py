@@ -3,10 +3,14 @@ while they call the library (an engine whose allocator owns the GPU, a plugin un
 no-cudaMalloc rule).  Its split planes live in a fixed array inside the library, shared by all
 calls, so the check runs it twice in a row with different shapes (the second call finds the
 first one's leftovers in the array) and compares each result with the sum of the planes that the
-ordinary entry point, spd_gemm_bf16, writes to caller memory.  Collected last on purpose."""
+ordinary entry point, spd_gemm_bf16, writes to caller memory - and with the CPU oracle's linear layer.
+A further check watches the device allocator around a call: nothing may be allocated.  Collected last
+on purpose."""
+import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2502_20727_b200 as spd
 from parity_util import rel_err
 
@@ -16,6 +20,13 @@ pytestmark = pytest.mark.gpu
 def rand_bf16(shape, seed):
     g = torch.Generator().manual_seed(seed)
     return torch.randn(shape, generator=g).to(torch.bfloat16)
+
+
+def oracle_linear(a, w):
+    """The oracle's linear layer per shard block: [M, batches*N] (a, w on the host)."""
+    wb = w if w.dim() == 3 else w[None]
+    cols = [oracle.linear((a[z] if a.dim() == 3 else a).double().numpy(), wb[z].float().numpy()) for z in range(wb.shape[0])]
+    return np.concatenate(cols, axis=1)
 
 
 def both(a, w, splits, swap):
@@ -31,15 +42,34 @@ def both(a, w, splits, swap):
 
 
 @pytest.mark.parametrize("swap", [True, False])
-def test_two_calls_in_a_row_match_the_allocating_entry_point(swap):
+def test_two_calls_in_a_row_match_the_allocating_entry_point_and_the_oracle(swap):
     # first call: 4 shard blocks of 344 rows with one input per shard, 3 splits (ragged tiles)
-    a1, w1 = rand_bf16((4, 24, 512), 11).cuda(), rand_bf16((4, 344, 512), 12).cuda()
-    got, ref = both(a1, w1, 3, swap)
+    a1, w1 = rand_bf16((4, 24, 512), 11), rand_bf16((4, 344, 512), 12)
+    got, ref = both(a1.cuda(), w1.cuda(), 3, swap)
     assert rel_err(got, ref) < 2e-5
+    assert rel_err(got, oracle_linear(a1, w1)) < 2e-5  # fp32 accumulation of exact bf16 products
     # second call: smaller and differently shaped, so stale planes of the first call lie around it
-    a2, w2 = rand_bf16((8, 1376), 13).cuda(), rand_bf16((200, 1376), 14).cuda()
-    got, ref = both(a2, w2, 5, swap)
+    a2, w2 = rand_bf16((8, 1376), 13), rand_bf16((200, 1376), 14)
+    got, ref = both(a2.cuda(), w2.cuda(), 5, swap)
     assert rel_err(got, ref) < 2e-5
+    assert rel_err(got, oracle_linear(a2, w2)) < 2e-5
+
+
+def test_a_call_allocates_no_device_memory():
+    """What the entry point is for: once the first call on the device has looked up the array's address, a call
+    leaves the torch allocator's and the driver's view of device memory exactly as it found them."""
+    a, w = rand_bf16((8, 1376), 21).cuda(), rand_bf16((200, 1376), 22).cuda()
+    out = torch.empty((8, 200), dtype=torch.float32, device="cuda")
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    spd.gemm_bf16_sum_static(a, w, out, err, splits=4, swap=True)  # warm-up: symbol look-up, kernel images
+    torch.cuda.synchronize()
+    before = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0])
+    spd.gemm_bf16_sum_static(a, w, out, err, splits=4, swap=True)
+    torch.cuda.synchronize()
+    after = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0])
+    assert before == after
+    assert int(err.item()) == 0
+    assert rel_err(out.double().cpu().numpy(), oracle_linear(a.cpu(), w.cpu())) < 2e-5
 
 
 def test_a_problem_larger_than_the_array_is_refused():
