@@ -131,7 +131,9 @@ int spd_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_l
  * (x, seq_lens, block_table, out, B, max_pages, max_context rounded up to 256) captures the
  * step's kernels on `stream` and later calls with the same values launch the captured graph;
  * tensor CONTENTS (inputs, seq_lens, block table) may change freely between calls.  Up to 8
- * graphs are kept per context.  A caller that passes fresh pointers every step should turn
+ * graphs are kept per context.  A growing context changes bucket every 256 steps; the graph of the
+ * next bucket is captured (not run) once max_context is within 32 of the edge, so the step that
+ * crosses over finds its graph ready and the capture overlaps the steps still queued on the device.  A caller that passes fresh pointers every step should turn
  * this off (each new pointer set costs a capture).  Calls on the legacy default stream (which
  * cannot be captured), calls made while `stream` is itself being captured, and calls made
  * while profiling launch the kernels directly. */
@@ -344,6 +346,27 @@ int spd_profile_begin(spd_ctx *ctx);
 int spd_profile_end(spd_ctx *ctx, void *stream, float *ms_by_kind, int32_t *launches_by_kind);
 int spd_profile_kinds(void);
 const char *spd_profile_kind_name(int kind);
+
+/* Launch timeline for benchmarks: when and how long every kernel of a call ran INSIDE the call as it is
+ * normally issued - decode steps replayed from their graph, launches overlapping through programmatic
+ * dependent launch - with nothing inserted between the launches (spd_profile_* brackets every launch with
+ * events, which serialises them).  After spd_timeline_begin every kernel of the bf16 prompt and decode paths
+ * (block_kind 0; the kernels of the other paths carry no stamps and are left out) gets a slot in the
+ * workspace; one thread of each of its blocks records the GPU's global nanosecond timer at block start and
+ * end, and the slot keeps the earliest start and the latest end.  Each spd_prefill / spd_decode_step /
+ * spd_tp_decode_step call starts the slots afresh, so read after every call:
+ *   spd_timeline_read : synchronises `stream`; for the first min(launches, max_launches) launches of the
+ *                       last call, in launch order: kinds[i] (index of spd_profile_kind_name), start_ns[i],
+ *                       end_ns[i] (both 0 for a launch that did not run); *n_launches = entries written.
+ *                       A call with more than 6 * n_layers + 16 launches (chunked prompts) reports the first ones.
+ * Consecutive launches overlap (the next kernel's blocks start, and request their first weights, under the
+ * tail of the one before): end[i] - max(start[i], end[i-1]) is launch i's own share of the call's duration.
+ * spd_timeline_begin / _end drop the captured decode graphs (a step is captured again with / without slots).
+ * Errors: SPD_ENULL, SPD_EINVAL (read without begin), SPD_ECUDA. */
+int spd_timeline_begin(spd_ctx *ctx);
+int spd_timeline_read(spd_ctx *ctx, void *stream, int32_t max_launches, int32_t *kinds, uint64_t *start_ns,
+                      uint64_t *end_ns, int32_t *n_launches);
+int spd_timeline_end(spd_ctx *ctx);
 
 /* Free the context (host state, descriptors, graphs).  Never touches caller tensors. */
 void spd_destroy(spd_ctx *ctx);

@@ -29,7 +29,9 @@ EXPORTS = ("spd_workspace_bytes", "spd_create", "spd_prefill", "spd_decode_step"
            "spd_last_cuda_error", "spd_profile_begin", "spd_profile_end", "spd_profile_kinds",
            "spd_profile_kind_name", "spd_gemm_bf16", "spd_set_graphs", "spd_gemm_bf16_sum_static",
            "spd_set_tuning", "spd_set_mask", "spd_sensitivity_scan", "spd_alg1_plan",
-           "spd_head_grouping_stats", "spd_head_scatter", "spd_mlp_match")
+           "spd_head_grouping_stats", "spd_head_scatter", "spd_mlp_match", "spd_timeline_begin", "spd_timeline_read",
+           "spd_timeline_end", "spd_tp_region_bytes", "spd_tp_attach", "spd_tp_detach", "spd_tp_decode_step",
+           "spd_tp_prefill")
 
 
 class SpdError(RuntimeError):
@@ -96,6 +98,10 @@ def load_library() -> ctypes.CDLL:
     lib.spd_tp_prefill.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp]
     lib.spd_profile_begin.argtypes = [vp]
     lib.spd_profile_end.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
+    lib.spd_timeline_begin.argtypes = [vp]
+    lib.spd_timeline_end.argtypes = [vp]
+    lib.spd_timeline_read.argtypes = [vp, vp, i32, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_uint64),
+                                      ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(i32)]
     lib.spd_profile_kinds.argtypes = []
     lib.spd_profile_kind_name.argtypes = [ctypes.c_int]
     lib.spd_profile_kind_name.restype = ctypes.c_char_p
@@ -364,6 +370,25 @@ class SpdStack:
             _check("spd_profile_end", self.lib.spd_profile_end(self._ctx, _stream_ptr(), ms, cnt))
         return {self.lib.spd_profile_kind_name(i).decode(): {"ms": float(ms[i]), "launches": int(cnt[i])}
                 for i in range(n)}
+
+    def timeline_begin(self):
+        """Stamp every kernel of the following calls (start / end on the GPU's nanosecond timer); see spd_timeline_begin."""
+        _check("spd_timeline_begin", self.lib.spd_timeline_begin(self._ctx))
+
+    def timeline_end(self):
+        _check("spd_timeline_end", self.lib.spd_timeline_end(self._ctx))
+
+    def timeline_read(self):
+        """[(kind name, start_ns, end_ns)] of the last call's launches, in launch order; see spd_timeline_read."""
+        cap = 6 * self.dims.n_layers + 16
+        kinds = (ctypes.c_int32 * cap)()
+        t0 = (ctypes.c_uint64 * cap)()
+        t1 = (ctypes.c_uint64 * cap)()
+        n = ctypes.c_int32(0)
+        with torch.cuda.device(self.device):
+            _check("spd_timeline_read", self.lib.spd_timeline_read(self._ctx, _stream_ptr(), cap, kinds, t0, t1, ctypes.byref(n)))
+        names = [self.lib.spd_profile_kind_name(i).decode() for i in range(self.lib.spd_profile_kinds())]
+        return [(names[kinds[i]], int(t0[i]), int(t1[i])) for i in range(n.value)]
 
     def set_mask(self, sync_mask: Sequence[int]):
         """Replace the per-block mask (1 = TP block, 0 = SPD block); see spd_set_mask."""

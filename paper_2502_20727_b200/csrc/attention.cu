@@ -143,6 +143,7 @@ __global__ void __launch_bounds__(FA_THREADS, 2) prefill_attention_mma_kernel(At
     extern __shared__ __align__(128) uint8_t fa_smem[];
     const uint32_t sQ = tc::smem_u32(fa_smem), sK = sQ + BQ * D * 2, sV = sK + 2 * BKV * D * 2;
     pdl_launch_dependents();
+    if (threadIdx.x == 0) stamp_entry(a.stamp);
     pdl_wait();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
     const int q0 = ((int)gridDim.x - 1 - (int)blockIdx.x) * BQ, hq = blockIdx.y, bi = blockIdx.z; // longest rows first
@@ -293,6 +294,7 @@ __global__ void __launch_bounds__(FA_THREADS, 2) prefill_attention_mma_kernel(At
         for (int dt = 0; dt < DT; ++dt)
             *(uint32_t *)(dst + dt * 8 + 2 * t4) = pack_bf16(o[dt][2 * h] * inv, o[dt][2 * h + 1] * inv);
     }
+    if (threadIdx.x == 0) stamp_exit(a.stamp);
 }
 
 template <int D> cudaError_t launch(const AttnArgs &a, int n_seq, cudaStream_t st)
@@ -495,7 +497,7 @@ template <typename T, int D, int GT>
 __global__ void __launch_bounds__(128) decode_attention_kernel(AttnArgs a)
 {
     pdl_launch_dependents();
-    if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_START);
+    if (threadIdx.x == 0) { SPD_TRACE_EVENT(TRK_ATTN, TR_START); stamp_entry(a.stamp); }
     pdl_wait();
     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_DEP_DONE);
     constexpr int E = Row16<T>::E, LPT = D / E, TPW = 32 / LPT, NG = 8, CHUNK = NG * TPW;
@@ -632,7 +634,7 @@ __global__ void __launch_bounds__(128) decode_attention_kernel(AttnArgs a)
             if (dd == 0) { a.part_ml[pi * 2] = gm; a.part_ml[pi * 2 + 1] = gden; }
         }
     }
-    if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_MAIN_DONE);
+    if (threadIdx.x == 0) { SPD_TRACE_EVENT(TRK_ATTN, TR_MAIN_DONE); stamp_exit(a.stamp); }
     if (a.splits == 1) return;
     // the last CTA of this (sequence, head tile) to arrive merges the splits
     __threadfence();
@@ -657,7 +659,7 @@ __global__ void __launch_bounds__(128) decode_attention_kernel(AttnArgs a)
         ((T *)a.out)[((long)b * a.n_q_heads + hq0 + g) * D + dd] = from_f<T>(gden > 0.f ? acc / gden : 0.f);
     }
     if (threadIdx.x == 0) *cnt = 0; // ready for the next launch
-    if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_END);
+    if (threadIdx.x == 0) { SPD_TRACE_EVENT(TRK_ATTN, TR_END); stamp_exit(a.stamp); }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -699,6 +701,7 @@ __global__ void __launch_bounds__(160, DENSE ? 5 : 4) decode_attention_ring_kern
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
         SPD_TRACE_EVENT(TRK_ATTN, TR_START);
+        stamp_entry(a.stamp);
         for (int s = 0; s < R; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -844,7 +847,7 @@ __global__ void __launch_bounds__(160, DENSE ? 5 : 4) decode_attention_ring_kern
     __syncthreads();
     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_MAIN_DONE);
     finish_decode_attention<T, D, GT>(a, b, hq0, sp, sm_o, sm_ml, sm_pml, sm_last);
-    if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_END);
+    if (threadIdx.x == 0) { SPD_TRACE_EVENT(TRK_ATTN, TR_END); stamp_exit(a.stamp); }
 }
 
 template <typename T, int D, int GT, bool DENSE> cudaError_t launch_ring_as(const AttnArgs &a, cudaStream_t st)
@@ -918,6 +921,7 @@ __global__ void __launch_bounds__(160, DENSE ? 4 : 3) decode_attention_mma_kerne
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
         SPD_TRACE_EVENT(TRK_ATTN, TR_START);
+        stamp_entry(a.stamp);
         for (int s = 0; s < R; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1050,7 +1054,7 @@ __global__ void __launch_bounds__(160, DENSE ? 4 : 3) decode_attention_mma_kerne
     __syncthreads();
     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_MAIN_DONE);
     finish_decode_attention<bf16, D, GT>(a, b, hq0, sp, sm_o, sm_ml, sm_pml, sm_last);
-    if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_END);
+    if (threadIdx.x == 0) { SPD_TRACE_EVENT(TRK_ATTN, TR_END); stamp_exit(a.stamp); }
 }
 
 template <int GT, bool DENSE> cudaError_t launch_decode_mma_as(const AttnArgs &a, cudaStream_t st)

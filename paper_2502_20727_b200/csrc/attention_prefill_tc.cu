@@ -119,6 +119,7 @@ __global__ void __launch_bounds__(F_THREADS, 1) prefill_attention_umma_kernel(co
     const int n_tiles = (kv_len + FKV - 1) / FKV;
 
     pdl_launch_dependents();
+    if (threadIdx.x == 0) stamp_entry(a.stamp);
     // The two load warps set up the barriers themselves and only ARRIVE at the set-up barrier, so that the first
     // tiles are on their way while the others still wait for the tensor-memory allocation.
     uint32_t tmem = 0;
@@ -341,6 +342,7 @@ __global__ void __launch_bounds__(F_THREADS, 1) prefill_attention_umma_kernel(co
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if (threadIdx.x == 0) stamp_exit(a.stamp);
     if (warp == 18) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");

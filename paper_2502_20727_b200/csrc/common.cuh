@@ -36,6 +36,25 @@ template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __flo
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// Launch stamps (optional; spd_timeline_*).  A launch may be handed a slot of two 64-bit words preset to all
+// ones.  One thread of every block lowers word 0 to the global nanosecond timer when the block starts and word 1
+// to the timer's complement when it ends, so that afterwards word 0 is the launch's earliest block start and
+// ~word 1 its latest block end - taken inside a replayed graph, with nothing inserted between the launches.
+__device__ __forceinline__ void stamp_entry(unsigned long long *slot)
+{
+    if (!slot) return;
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    atomicMin(slot, t);
+}
+__device__ __forceinline__ void stamp_exit(unsigned long long *slot)
+{
+    if (!slot) return;
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    atomicMin(slot + 1, ~t);
+}
+
 // Launch with the programmatic-stream-serialization attribute (and an optional cluster size).
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
@@ -156,7 +175,8 @@ struct NormArgs {
 };
 template <typename T> cudaError_t launch_residual_norm(const NormArgs &a, cudaStream_t st);
 
-cudaError_t launch_rope_table(float2 *table, TokMap tm, int M, int head_dim, float base, cudaStream_t st);
+cudaError_t launch_rope_table(float2 *table, TokMap tm, int M, int head_dim, float base, cudaStream_t st,
+                              unsigned long long *stamp = nullptr);
 
 struct RopeKvArgs {
     const float *qkv;     // fp32 [splits][M][ldq]: columns [q | k | v]
@@ -206,6 +226,7 @@ struct AttnArgs {
     // ... and how far (in powers of two) the running row maximum may grow before the accumulated output is rescaled
     float rescale_log2;
     int cluster_merge;      // set by the launcher: the splits of a (sequence, head tile) are one thread-block cluster
+    unsigned long long *stamp; // launch stamp slot or null
 };
 // Paged decode attention with 16-token pages: query heads per thread block for a GQA group
 // size, and the most pages one block may be given (the host picks splits accordingly).

@@ -242,26 +242,29 @@ template cudaError_t launch_residual_norm<float>(const NormArgs &, cudaStream_t)
 template cudaError_t launch_residual_norm<bf16>(const NormArgs &, cudaStream_t);
 
 // cos/sin of pos * base^(-2j/d), evaluated in double once per call and shared by all layers.
-__global__ void rope_table_kernel(float2 *table, TokMap tm, int M, int half, double log_base, int d)
+__global__ void rope_table_kernel(float2 *table, TokMap tm, int M, int half, double log_base, int d, unsigned long long *stamp)
 {
     pdl_launch_dependents();
+    if (threadIdx.x == 0) stamp_entry(stamp);
     pdl_wait();
     int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= M * half) return;
-    int m = i / half, j = i % half, b, pos;
-    tm.locate(m, b, pos);
-    double theta = exp(-2.0 * (double)j / (double)d * log_base);
-    double s, c;
-    sincos((double)pos * theta, &s, &c);
-    table[i] = make_float2((float)c, (float)s);
+    if (i < M * half) {
+        int m = i / half, j = i % half, b, pos;
+        tm.locate(m, b, pos);
+        double theta = exp(-2.0 * (double)j / (double)d * log_base);
+        double s, c;
+        sincos((double)pos * theta, &s, &c);
+        table[i] = make_float2((float)c, (float)s);
+    }
+    if (threadIdx.x == 0) stamp_exit(stamp);
 }
 
-cudaError_t launch_rope_table(float2 *table, TokMap tm, int M, int head_dim, float base, cudaStream_t st)
+cudaError_t launch_rope_table(float2 *table, TokMap tm, int M, int head_dim, float base, cudaStream_t st, unsigned long long *stamp)
 {
     int n = M * (head_dim / 2);
     if (n <= 0) return cudaSuccess;
     return launch_kernel(rope_table_kernel, dim3((n + 255) / 256), dim3(256), 0, st, 0, table, tm, M, head_dim / 2,
-                         log((double)base), head_dim);
+                         log((double)base), head_dim, stamp);
 }
 
 // grid (M, n_q_heads + n_kv_heads): sums the split-K planes of one head's projection, rotates

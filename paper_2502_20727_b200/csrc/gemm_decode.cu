@@ -482,6 +482,7 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
         // accumulator allocation nor the other warps, so this GEMM's weight stream starts the
         // moment the block is resident - under the tail of whatever ran before.
         SPD_TRACE_EVENT(EPI, TR_START);
+        stamp_entry(g.stamp);
         for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         mbar_init(tmem_full_bar, 1);
         *abort_flag = 0;
@@ -605,7 +606,7 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
         else if (EPI == EPI_GATEUP) epilogue_gateup<BN>(g, t, S, Gb, sm_rstd);
         else if (EPI == EPI_RESID_TP) epilogue_resid_tp<BN>(g, t, S, abort_flag);
         else epilogue_residual<BN>(g, t, S, EPI == EPI_OPROJ && g.n_groups > 1);
-        if (threadIdx.x == 0) SPD_TRACE_EVENT(EPI, TR_END);
+        if (threadIdx.x == 0) { SPD_TRACE_EVENT(EPI, TR_END); stamp_exit(g.stamp); }
     }
     // no block may exit while a peer still reads its shared memory
     if (t.P > 1) cluster_sync_all();
@@ -698,6 +699,7 @@ cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
 __global__ void __launch_bounds__(128) decode_prologue_kernel(PrologueArgs a, int h_tiles, double log_base)
 {
     pdl_launch_dependents();
+    if (threadIdx.x == 0) stamp_entry(a.stamp);
     pdl_wait();
     if ((int)blockIdx.x >= h_tiles) {
         // rotary table of this step, evaluated in double and shared by all blocks of the stack
@@ -737,6 +739,7 @@ __global__ void __launch_bounds__(128) decode_prologue_kernel(PrologueArgs a, in
         const float q = warp_sum(sq4(x));
         if (lane == 0) ss_out[(long)blockIdx.x * a.Mcap + m] = q;
     }
+    if (threadIdx.x == 0) stamp_exit(a.stamp);
 }
 
 } // namespace

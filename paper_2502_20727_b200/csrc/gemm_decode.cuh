@@ -70,6 +70,7 @@ struct DecGemmArgs {
     int l2_prefetch_kb;    // K blocks of weights per thread block pulled into L2 before the dependency wait
     int ring_stages;       // stages of the operand ring (3, 4; 5 at 16-token tiles); 0 = chosen per launch
     int *err;
+    unsigned long long *stamp; // launch stamp slot or null
     // ---- epilogue operands -----------------------------------------------------------
     SumSq ss_in;           // QKV, GATEUP: sums of squares of the GEMM input's rows
     int rstd_per_shard;    // GATEUP in an SPD block: shard z reads group z
@@ -123,6 +124,7 @@ struct PrologueArgs {
     int n_z;
     long z_stride;
     unsigned *step;
+    unsigned long long *stamp; // launch stamp slot or null
 };
 cudaError_t launch_decode_prologue(const PrologueArgs &a, cudaStream_t st);
 

@@ -432,6 +432,7 @@ __global__ void __launch_bounds__(PCfg<EPI>::THREADS_, 1) gemm_prefill_kernel(co
 
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
+        stamp_entry(g.stamp);
         for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), C::EPI_WARPS); }
         mbar_init(xfull_bar, 1);
@@ -558,6 +559,7 @@ __global__ void __launch_bounds__(PCfg<EPI>::THREADS_, 1) gemm_prefill_kernel(co
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if (threadIdx.x == 0) stamp_exit(g.stamp);
     if (warp == 5) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_ALL) : "memory");
@@ -589,6 +591,7 @@ cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
 __global__ void __launch_bounds__(256) prefill_prologue_kernel(PrologueArgs a)
 {
     pdl_launch_dependents();
+    if (threadIdx.x == 0) stamp_entry(a.stamp);
     pdl_wait();
     __shared__ float red[8];
     const int m = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -611,6 +614,7 @@ __global__ void __launch_bounds__(256) prefill_prologue_kernel(PrologueArgs a)
         float tot = 0.f;
         for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];
         a.ss_out[m] = tot;
+        stamp_exit(a.stamp);
     }
 }
 

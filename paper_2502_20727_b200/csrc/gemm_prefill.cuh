@@ -23,6 +23,7 @@ struct PreGemmArgs {
     int w_rows[3];       // valid rows (per device for GATEUP) of weight i
     int n_weights;
     int *err;
+    unsigned long long *stamp; // launch stamp slot or null
     SumSq ss_in;         // QKV, GATEUP
     int rstd_per_shard;
     // QKV

@@ -81,7 +81,7 @@ struct GraphKey {
                max_pages == o.max_pages && ctx_bucket == o.ctx_bucket && mode == o.mode;
     }
 };
-struct GraphEntry { GraphKey key; cudaGraphExec_t exec; unsigned long long last_use; int launches; };
+struct GraphEntry { GraphKey key; cudaGraphExec_t exec; unsigned long long last_use; int launches; std::vector<int> tl_kind; };
 
 // One rank's region of a tensor-parallel group (offsets in bytes; every rank uses the same layout).
 struct TpLayout {
@@ -133,6 +133,12 @@ struct Ctx {
     TcMap act_maps[AB_COUNT][4];
     bool act_map_ready[AB_COUNT][4];
 
+    // optional launch stamps (spd_timeline_*): slot i = earliest block start / latest block end of the call's i-th launch
+    bool timeline;
+    unsigned long long *stamps;
+    int stamps_cap, tl_next;
+    std::vector<int> tl_kind;
+
     // optional per-kernel-kind timing (spd_profile_begin / spd_profile_end)
     bool profiling;
     std::vector<cudaEvent_t> ev_pool;
@@ -153,6 +159,23 @@ cudaError_t prof_mark(Ctx *c, int kind, cudaStream_t st)
     return cudaEventRecord(c->ev_pool[c->ev_used++], st);
 }
 
+// The stamp slot of the call's next launch (null when no timeline is being taken or the slots are used up).
+unsigned long long *next_stamp(Ctx *c, int kind)
+{
+    if (!c->timeline || c->tl_next >= c->stamps_cap) return nullptr;
+    c->tl_kind.push_back(kind);
+    return c->stamps + 2 * (size_t)c->tl_next++;
+}
+
+// A call starts its timeline afresh: slots preset to all ones, in stream order before the first launch.
+cudaError_t timeline_restart(Ctx *c, cudaStream_t st)
+{
+    if (!c->timeline) return cudaSuccess;
+    c->tl_next = 0;
+    c->tl_kind.clear();
+    return cudaMemsetAsync(c->stamps, 0xFF, (size_t)c->stamps_cap * 16, st);
+}
+
 #define LAUNCH(kind, expr)                   \
     do {                                     \
         CU_TRY(prof_mark(c, (kind), st));    \
@@ -161,7 +184,16 @@ cudaError_t prof_mark(Ctx *c, int kind, cudaStream_t st)
         ++launches;                          \
     } while (0)
 
+// ... for a launch whose argument struct carries a stamp slot
+#define LAUNCH_S(kind, args, expr)                \
+    do {                                          \
+        (args).stamp = next_stamp(c, (kind));     \
+        LAUNCH(kind, expr);                       \
+    } while (0)
+
 size_t esize(const spd_dims &d) { return d.dtype == 0 ? 4 : 2; }
+
+int stamp_slots(const spd_dims &d) { return 6 * d.n_layers + 16; }
 
 // M = tokens of the launch.  decode: few tokens, the weight-streaming GEMMs are cut along K so
 // that about two CTAs per SM are in flight; prefill: no K splits.
@@ -239,7 +271,7 @@ SiteGeom site_geom(const spd_dims &d, int site)
 }
 
 struct Layout {
-    size_t res[2], h, q, attn, act, qkv32, proj32, gu32, part_o, part_ml, attn_cnt, rope, err, ss_attn, ss_mlp, total;
+    size_t res[2], h, q, attn, act, qkv32, proj32, gu32, part_o, part_ml, attn_cnt, rope, err, ss_attn, ss_mlp, stamps, total;
     size_t Mcap;
 };
 
@@ -276,6 +308,7 @@ Layout make_layout(const spd_dims &d, bool any_spd)
     const size_t h_tiles = (H + 127) / 128;
     L.ss_attn = take(h_tiles * Mmax * 4);
     L.ss_mlp = take(2 * h_tiles * T * Mmax * 4); // the SPD o_proj of the prefill path leaves two partials per tile
+    L.stamps = take((size_t)stamp_slots(d) * 16);
     L.total = off;
     return L;
 }
@@ -548,7 +581,7 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
         a.x = x; a.res_out = c->res[0]; a.gain = c->layers[0].attn_norm; a.hg = c->h; a.ss_out = c->ss_attn;
         a.Mcap = Mc; a.M = M; a.H = H;
         if (rope) { a.rope_table = c->rope; a.tm = tm; a.head_dim = d.head_dim; a.rope_base = d.rope_base; }
-        LAUNCH(K_NORM, launch_decode_prologue(a, st));
+        LAUNCH_S(K_NORM, a, launch_decode_prologue(a, st));
     }
     auto base_args = [&]() {
         DecGemmArgs g{};
@@ -570,7 +603,7 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
             g.ss_in = SumSq{c->ss_attn, h_tiles, 1, Mc, H, d.rms_eps};
             g.rope = rope ? c->rope : nullptr; g.q_out = c->q; g.k_pages = w.k_pages; g.v_pages = w.v_pages; g.pt = pt; g.tm = tm;
             g.n_q_heads = d.n_q_heads; g.head_dim = d.head_dim;
-            LAUNCH(K_QKV, launch_gemm_decode(EPI_QKV, wmaps, *am, g, st));
+            LAUNCH_S(K_QKV, g, launch_gemm_decode(EPI_QKV, wmaps, *am, g, st));
         }
         {   // a4
             AttnArgs a{};
@@ -578,7 +611,7 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
             a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.B = M; a.splits = p.attn_splits;
             a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.counters = c->attn_cnt; a.err = c->err;
             if (d.head_dim == 128 && d.kv_block_size == 16) { a.k_map = &c->maps[l].kpages; a.v_map = &c->maps[l].vpages; }
-            LAUNCH(K_ATTN, launch_decode_attention<bf16>(a, st));
+            LAUNCH_S(K_ATTN, a, launch_decode_attention<bf16>(a, st));
         }
         {   // a5 - a7: shard i's K slice gives the plane group Y_i
             DecGemmArgs g = base_args();
@@ -590,7 +623,7 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
             g.res_in = c->res[0]; g.res_out = c->res[1]; g.gain = w.mlp_norm; g.hg = c->h; g.hg_stride = Mc * H;
             g.ss_out = c->ss_mlp;
             g.n_groups = sync ? 1 : Tn;
-            LAUNCH(K_OPROJ, launch_gemm_decode(EPI_OPROJ, wmaps, *am, g, st));
+            LAUNCH_S(K_OPROJ, g, launch_gemm_decode(EPI_OPROJ, wmaps, *am, g, st));
         }
         {   // a8: 64 gate rows and the 64 up rows of the same FFN columns per tile
             DecGemmArgs g = base_args();
@@ -602,7 +635,7 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
             g.ss_in = SumSq{c->ss_mlp, h_tiles, sync ? 1 : Tn, Mc, H, d.rms_eps};
             g.rstd_per_shard = sync ? 0 : 1;
             g.act = c->act; g.F = F; g.Fs = Fs;
-            LAUNCH(K_GATE_UP, launch_gemm_decode(EPI_GATEUP, wmaps, *am, g, st));
+            LAUNCH_S(K_GATE_UP, g, launch_gemm_decode(EPI_GATEUP, wmaps, *am, g, st));
         }
         {   // a9 + a10: res[1] holds X + sum_i Y_i in both modes, so out = res[1] + sum_i Z_i
             DecGemmArgs g = base_args();
@@ -614,7 +647,7 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
             g.res_in = c->res[1]; g.res_out = c->res[0];
             if (l + 1 < d.n_layers) { g.gain = c->layers[l + 1].attn_norm; g.hg = c->h; g.hg_stride = Mc * H; g.ss_out = c->ss_attn; }
             else g.final_out = out;
-            LAUNCH(K_DOWN, launch_gemm_decode(EPI_DOWN, wmaps, *am, g, st));
+            LAUNCH_S(K_DOWN, g, launch_gemm_decode(EPI_DOWN, wmaps, *am, g, st));
         }
     }
     c->launches_last = launches;
@@ -650,7 +683,7 @@ int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, 
         a.ss_out = (float *)(r0 + TL.ss_attn); a.Mcap = Mb; a.M = M; a.H = H;
         a.n_z = nl; a.z_stride = tp.z_stride; a.step = (unsigned *)(r0 + TL.step);
         if (rope) { a.rope_table = c->rope; a.tm = tm; a.head_dim = d.head_dim; a.rope_base = d.rope_base; }
-        LAUNCH(K_NORM, launch_decode_prologue(a, st));
+        LAUNCH_S(K_NORM, a, launch_decode_prologue(a, st));
     }
     auto base_args = [&]() {
         DecGemmArgs g{};
@@ -686,7 +719,7 @@ int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, 
             g.ss_in = SumSq{(const float *)(r0 + TL.ss_attn), h_tiles, 1, Mb, H, d.rms_eps};
             g.rope = rope ? c->rope : nullptr; g.q_out = c->q; g.k_pages = w.k_pages; g.v_pages = w.v_pages; g.pt = pt; g.tm = tm;
             g.n_q_heads = d.n_q_heads; g.head_dim = d.head_dim;
-            LAUNCH(K_QKV, launch_gemm_decode(EPI_QKV, wmaps, *hmap, g, st));
+            LAUNCH_S(K_QKV, g, launch_gemm_decode(EPI_QKV, wmaps, *hmap, g, st));
         }
         {   // a4: heads are rank-local by construction
             AttnArgs a{};
@@ -694,14 +727,14 @@ int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, 
             a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.B = M; a.splits = p.attn_splits;
             a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.counters = c->attn_cnt; a.err = c->err;
             if (d.head_dim == 128 && d.kv_block_size == 16) { a.k_map = &c->maps[l].kpages; a.v_map = &c->maps[l].vpages; }
-            if (decode) LAUNCH(K_ATTN, launch_decode_attention<bf16>(a, st));
+            if (decode) LAUNCH_S(K_ATTN, a, launch_decode_attention<bf16>(a, st));
             else {
                 a.splits = 1;
                 if (a.k_map) {
                     MAP_OR_FAIL(qm, act_map(c, AB_Q, 128));
                     a.q_map = qm; a.rescale_log2 = (float)c->prefill_rescale_log2;
                 }
-                LAUNCH(K_ATTN, launch_prefill_attention<bf16>(a, st));
+                LAUNCH_S(K_ATTN, a, launch_prefill_attention<bf16>(a, st));
             }
         }
         {   // a5 - a7: Y_z from the rank's own heads.  TP block: R = X + sum over ranks (sync-point 1);
@@ -715,7 +748,7 @@ int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, 
             g.res_in = (const float *)(r0 + TL.res0); g.gain = w.mlp_norm; g.hg = r0 + TL.hg; g.ss_out = (float *)(r0 + TL.ss_mlp);
             if (sync) { with_exchange(g, l, 0); g.res_out = (float *)(r0 + TL.res1); }
             else g.tp.ysave = (float *)(r0 + TL.ysave);
-            LAUNCH(K_OPROJ, launch_gemm_decode(EPI_RESID_TP, wmaps, *am, g, st));
+            LAUNCH_S(K_OPROJ, g, launch_gemm_decode(EPI_RESID_TP, wmaps, *am, g, st));
         }
         {   // a8
             DecGemmArgs g = base_args();
@@ -726,7 +759,7 @@ int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, 
                                      c->split_override[SITE_GU], 8, tbox == 16 ? 3 : 2);
             g.ss_in = SumSq{(const float *)(r0 + TL.ss_mlp), h_tiles, 1, Mb, H, d.rms_eps};
             g.act = c->act; g.F = F; g.Fs = Fs;
-            LAUNCH(K_GATE_UP, launch_gemm_decode(EPI_GATEUP, wmaps, *hmap, g, st));
+            LAUNCH_S(K_GATE_UP, g, launch_gemm_decode(EPI_GATEUP, wmaps, *hmap, g, st));
         }
         {   // a9 + a10, the kept sync-point.  TP block: out = R + sum_z Z_z;  SPD block: out = X + sum_z (Y_z + Z_z)
             DecGemmArgs g = base_args();
@@ -741,7 +774,7 @@ int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, 
             g.res_out = (float *)(r0 + TL.res0);
             if (l + 1 < d.n_layers) { g.gain = c->layers[l + 1].attn_norm; g.hg = r0 + TL.hg; g.ss_out = (float *)(r0 + TL.ss_attn); }
             else { g.final_out = out; g.tp.out_stride = out_stride; }
-            LAUNCH(K_DOWN, launch_gemm_decode(EPI_RESID_TP, wmaps, *am, g, st));
+            LAUNCH_S(K_DOWN, g, launch_gemm_decode(EPI_RESID_TP, wmaps, *am, g, st));
         }
     }
     c->launches_last = launches;
@@ -770,12 +803,12 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
     PageTable pt{bt, max_pages, c->n_pages, d.kv_block_size, d.n_kv_heads};
     int launches = 0;
     const bool rope = d.rope_base > 0.f;
-    if (rope) LAUNCH(K_ROPE_TABLE, launch_rope_table(c->rope, tm, M, d.head_dim, d.rope_base, st));
+    if (rope) LAUNCH(K_ROPE_TABLE, launch_rope_table(c->rope, tm, M, d.head_dim, d.rope_base, st, next_stamp(c, K_ROPE_TABLE)));
     {
         PrologueArgs a{};
         a.x = x; a.res_out = c->res[0]; a.gain = c->layers[0].attn_norm; a.hg = c->h; a.ss_out = c->ss_attn;
         a.Mcap = Mc; a.M = M; a.H = H;
-        LAUNCH(K_NORM, launch_prefill_prologue(a, st));
+        LAUNCH_S(K_NORM, a, launch_prefill_prologue(a, st));
     }
     int attn_tiles = 1; // partial sums of squares per token in ss_attn
     auto base_args = [&]() {
@@ -797,7 +830,7 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
             g.ss_in = SumSq{c->ss_attn, attn_tiles, 1, Mc, H, d.rms_eps};
             g.rope = rope ? c->rope : nullptr; g.q_out = c->q; g.k_pages = w.k_pages; g.v_pages = w.v_pages; g.pt = pt; g.tm = tm;
             g.n_q_heads = d.n_q_heads; g.head_dim = d.head_dim;
-            LAUNCH(K_QKV, launch_gemm_prefill(PRE_QKV, wmaps, *am, g, st));
+            LAUNCH_S(K_QKV, g, launch_gemm_prefill(PRE_QKV, wmaps, *am, g, st));
         }
         if (probing) {   // Eq. 2: attention score of every head as one long vector, pairwise Euclidean distances
             CU_TRY(launch_head_scores<bf16>(c->q, w.k_pages, pt, tm.b0, probe->S, probe->n_seq, d.n_q_heads, d.head_dim, probe->sigma,
@@ -813,7 +846,7 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
                 MAP_OR_FAIL(qm, act_map(c, AB_Q, 128));
                 a.q_map = qm; a.k_map = &c->maps[l].kpages; a.v_map = &c->maps[l].vpages; a.rescale_log2 = (float)c->prefill_rescale_log2;
             }
-            LAUNCH(K_ATTN, launch_prefill_attention<bf16>(a, st));
+            LAUNCH_S(K_ATTN, a, launch_prefill_attention<bf16>(a, st));
         }
         int mlp_tiles, mlp_groups;
         if (sync) {   // a5 - a7, sync block: sum_i Y_i is the K accumulation over all heads
@@ -822,7 +855,7 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
             MAP_OR_FAIL(am, act_map(c, AB_ATTN, 128));
             g.w_rows[0] = H; g.num_kb = cdiv(qd, 64);
             g.res_in = c->res[0]; g.res_out = c->res[1]; g.gain = w.mlp_norm; g.hg = c->h; g.hg_stride = Mc * H; g.ss_out = c->ss_mlp;
-            LAUNCH(K_OPROJ, launch_gemm_prefill(PRE_RESID, wmaps, *am, g, st));
+            LAUNCH_S(K_OPROJ, g, launch_gemm_prefill(PRE_RESID, wmaps, *am, g, st));
             mlp_tiles = pre_ss_tiles(PRE_RESID, H); mlp_groups = 1;
         } else {      // a5 - a7, SPD block: device i's K slice gives Y_i, kept apart
             PreGemmArgs g = base_args();
@@ -832,7 +865,7 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
             g.res_in = c->res[0]; g.res_out = c->res[1]; g.gain = w.mlp_norm; g.hg = c->h; g.hg_stride = Mc * H; g.ss_out = c->ss_mlp;
             MAP_OR_FAIL(hm, act_map(c, AB_H, 128));
             g.h_map = hm;
-            LAUNCH(K_OPROJ, launch_gemm_prefill(PRE_OPROJ_SPD, wmaps, *am, g, st));
+            LAUNCH_S(K_OPROJ, g, launch_gemm_prefill(PRE_OPROJ_SPD, wmaps, *am, g, st));
             mlp_tiles = pre_ss_tiles(PRE_OPROJ_SPD, H); mlp_groups = Tn;
         }
         if (probing) {
@@ -884,7 +917,7 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
             g.ss_in = SumSq{c->ss_mlp, mlp_tiles, mlp_groups, Mc, H, d.rms_eps};
             g.rstd_per_shard = sync ? 0 : 1;
             g.act = c->act; g.F = F; g.Fs = Fs;
-            LAUNCH(K_GATE_UP, launch_gemm_prefill(PRE_GATEUP, wmaps, *am, g, st));
+            LAUNCH_S(K_GATE_UP, g, launch_gemm_prefill(PRE_GATEUP, wmaps, *am, g, st));
         }
         {   // a9 + a10: res[1] holds X + sum_i Y_i in both modes, so out = res[1] + sum_i Z_i
             PreGemmArgs g = base_args();
@@ -894,7 +927,7 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
             g.res_in = c->res[1]; g.res_out = c->res[0];
             if (l + 1 < d.n_layers) { g.gain = c->layers[l + 1].attn_norm; g.hg = c->h; g.hg_stride = Mc * H; g.ss_out = c->ss_attn; }
             else g.final_out = out;
-            LAUNCH(K_DOWN, launch_gemm_prefill(PRE_RESID, wmaps, *am, g, st));
+            LAUNCH_S(K_DOWN, g, launch_gemm_prefill(PRE_RESID, wmaps, *am, g, st));
             attn_tiles = pre_ss_tiles(PRE_RESID, H);
         }
     }
@@ -950,43 +983,87 @@ int build_weight_maps(Ctx &c)
     return SPD_OK;
 }
 
-// Runs a decode step from its captured graph, capturing it first when no graph matches `key`;
-// directly when graphs are off, a profile is being taken or the stream cannot be captured.
-template <typename Run>
-int replay_or_run(Ctx &c, const GraphKey &key, Run run, cudaStream_t st)
+// Captured decode steps.  A graph is valid for exactly one GraphKey; up to 8 are kept per context.
+GraphEntry *find_graph(Ctx &c, const GraphKey &key)
+{
+    for (GraphEntry &e : c.graphs)
+        if (e.key == key) return &e;
+    return nullptr;
+}
+
+// Whether a call on `st` may use graphs at all: not while profiling, not inside somebody else's capture, not on
+// the legacy default stream (which cannot be captured).
+int graphs_usable(Ctx &c, cudaStream_t st, bool *ok)
 {
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     CU_TRY(cudaStreamIsCapturing(st, &cap));
-    // (the legacy default stream cannot be captured)
-    if (!c.use_graphs || c.profiling || cap != cudaStreamCaptureStatusNone || st == 0 || st == cudaStreamLegacy) return run();
-    GraphEntry *hit = nullptr;
-    for (GraphEntry &e : c.graphs)
-        if (e.key == key) hit = &e;
-    if (!hit) {
-        CU_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
-        const int rc = run();
-        cudaGraph_t graph = nullptr;
-        cudaError_t e = cudaStreamEndCapture(st, &graph);
-        if (rc != SPD_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
-        if (e != cudaSuccess) { g_last_cuda_error = (int)e; return SPD_ECUDA; }
-        cudaGraphExec_t exec = nullptr;
-        e = cudaGraphInstantiate(&exec, graph, 0);
-        cudaGraphDestroy(graph);
-        if (e != cudaSuccess) { g_last_cuda_error = (int)e; return SPD_ECUDA; }
-        if (c.graphs.size() >= 8) { // evict the least recently used
-            size_t lru = 0;
-            for (size_t i = 1; i < c.graphs.size(); ++i)
-                if (c.graphs[i].last_use < c.graphs[lru].last_use) lru = i;
-            cudaGraphExecDestroy(c.graphs[lru].exec);
-            c.graphs.erase(c.graphs.begin() + lru);
-        }
-        c.graphs.push_back(GraphEntry{key, exec, 0, c.launches_last});
-        hit = &c.graphs.back();
+    *ok = c.use_graphs && !c.profiling && cap == cudaStreamCaptureStatusNone && st != 0 && st != cudaStreamLegacy;
+    return SPD_OK;
+}
+
+// Captures run() on `st` (nothing executes) and keeps the instantiated graph under `key`.
+template <typename Run>
+int capture_graph(Ctx &c, const GraphKey &key, Run run, cudaStream_t st, GraphEntry **out)
+{
+    CU_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+    const int rc = run();
+    cudaGraph_t graph = nullptr;
+    cudaError_t e = cudaStreamEndCapture(st, &graph);
+    if (rc != SPD_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
+    if (e != cudaSuccess) { g_last_cuda_error = (int)e; return SPD_ECUDA; }
+    cudaGraphExec_t exec = nullptr;
+    e = cudaGraphInstantiate(&exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e != cudaSuccess) { g_last_cuda_error = (int)e; return SPD_ECUDA; }
+    if (c.graphs.size() >= 8) { // evict the least recently used
+        size_t lru = 0;
+        for (size_t i = 1; i < c.graphs.size(); ++i)
+            if (c.graphs[i].last_use < c.graphs[lru].last_use) lru = i;
+        cudaGraphExecDestroy(c.graphs[lru].exec);
+        c.graphs.erase(c.graphs.begin() + lru);
     }
+    c.graphs.push_back(GraphEntry{key, exec, ++c.graph_clock, c.launches_last, c.tl_kind});
+    *out = &c.graphs.back();
+    return SPD_OK;
+}
+
+// Runs a decode step from its captured graph, capturing it first when no graph matches `key`;
+// directly when graphs cannot be used.
+template <typename Run>
+int replay_or_run(Ctx &c, const GraphKey &key, Run run, cudaStream_t st)
+{
+    bool usable = false;
+    int rc = graphs_usable(c, st, &usable);
+    if (rc != SPD_OK) return rc;
+    if (!usable) return run();
+    GraphEntry *hit = find_graph(c, key);
+    if (!hit && (rc = capture_graph(c, key, run, st, &hit)) != SPD_OK) return rc;
     hit->last_use = ++c.graph_clock;
     c.launches_last = hit->launches;
+    if (c.timeline) { c.tl_kind = hit->tl_kind; c.tl_next = (int)hit->tl_kind.size(); } // the replay stamps the slots of its capture
     CU_TRY(cudaGraphLaunch(hit->exec, st));
     return SPD_OK;
+}
+
+// The step's launch shape changes with the context bucket.  So that a growing context does not meet a capture at
+// the very step that crosses into the next bucket, that bucket's graph is captured (not run) once the context is
+// within GRAPH_AHEAD_STEPS of the edge - while the device is still busy with the steps already queued.
+constexpr int GRAPH_AHEAD_STEPS = 32;
+template <typename Run>
+int capture_ahead(Ctx &c, const GraphKey &key, Run run, cudaStream_t st)
+{
+    bool usable = false;
+    int rc = graphs_usable(c, st, &usable);
+    if (rc != SPD_OK || !usable || find_graph(c, key)) return rc;
+    const int launches = c.launches_last;
+    const std::vector<int> kinds = c.tl_kind;
+    const int next = c.tl_next;
+    GraphEntry *e = nullptr;
+    rc = capture_graph(c, key, run, st, &e);
+    c.launches_last = launches; // bookkeeping stays that of the step that ran
+    c.tl_kind = kinds;
+    c.tl_next = next;
+    return rc;
 }
 
 } // namespace
@@ -1051,6 +1128,10 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     c.part_o = (float *)(c.ws + L.part_o); c.part_ml = (float *)(c.ws + L.part_ml);
     c.attn_cnt = (int *)(c.ws + L.attn_cnt);
     c.ss_attn = (float *)(c.ws + L.ss_attn); c.ss_mlp = (float *)(c.ws + L.ss_mlp);
+    c.stamps = (unsigned long long *)(c.ws + L.stamps);
+    c.stamps_cap = stamp_slots(*dims);
+    c.timeline = false;
+    c.tl_next = 0;
     for (int i = 0; i < SITE_COUNT; ++i) c.split_override[i] = 0;
     c.l2_prefetch_kb = 0;
     c.prefill_rescale_log2 = 8;
@@ -1093,6 +1174,7 @@ int spd_prefill(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int32_t
     const size_t es = esize(d);
     const int Mp = d.max_prefill_tokens;
     int total_launches = 0;
+    CU_TRY(timeline_restart(&c, st));
     auto run = [&](int b0, int nb, int s0, int ns) -> int {
         TokMap tm{0, b0, ns, s0, nullptr};
         size_t off = ((size_t)b0 * S + s0) * d.hidden * es;
@@ -1133,16 +1215,30 @@ int spd_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_l
     // The launch sequence only depends on a coarse bucket of the context bound (it sizes the
     // KV split), so a step can be replayed from a captured graph until a pointer or the
     // bucket changes.
-    int ctx_bucket = (max_context + 255) / 256 * 256;
-    if (ctx_bucket > d.max_seq_len) ctx_bucket = d.max_seq_len;
-    if ((long)ctx_bucket > (long)max_pages * d.kv_block_size) ctx_bucket = max_pages * d.kv_block_size;
-    auto run = [&]() {
-        return d.dtype == 0        ? run_tokens<float>(&c, x, out, B, tm, block_table, max_pages, true, ctx_bucket, st)
-               : d.block_kind == 0 ? run_decode_fused(&c, x, out, B, tm, block_table, max_pages, ctx_bucket, st)
-                                   : run_tokens<bf16>(&c, x, out, B, tm, block_table, max_pages, true, ctx_bucket, st);
+    auto bucket_of = [&](int mc) {
+        int b = (mc + 255) / 256 * 256;
+        if (b > d.max_seq_len) b = d.max_seq_len;
+        if ((long)b > (long)max_pages * d.kv_block_size) b = max_pages * d.kv_block_size;
+        return b;
+    };
+    const int ctx_bucket = bucket_of(max_context);
+    auto run_at = [&](int bucket) {
+        return [&, bucket]() -> int {
+            CU_TRY(timeline_restart(&c, st)); // inside the captured step: every replay presets the slots first
+            return d.dtype == 0        ? run_tokens<float>(&c, x, out, B, tm, block_table, max_pages, true, bucket, st)
+                   : d.block_kind == 0 ? run_decode_fused(&c, x, out, B, tm, block_table, max_pages, bucket, st)
+                                       : run_tokens<bf16>(&c, x, out, B, tm, block_table, max_pages, true, bucket, st);
+        };
     };
     const GraphKey key{x, seq_lens, block_table, out, B, max_pages, ctx_bucket, 0};
-    return replay_or_run(c, key, run, st);
+    int rc = replay_or_run(c, key, run_at(ctx_bucket), st);
+    if (rc != SPD_OK) return rc;
+    const int next_bucket = bucket_of(ctx_bucket + 1);
+    if (next_bucket > ctx_bucket && max_context + GRAPH_AHEAD_STEPS > ctx_bucket) {
+        const GraphKey ahead{x, seq_lens, block_table, out, B, max_pages, next_bucket, 0};
+        rc = capture_ahead(c, ahead, run_at(next_bucket), st);
+    }
+    return rc;
 }
 
 static void drop_graphs(Ctx &c)
@@ -1373,7 +1469,10 @@ int spd_tp_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *se
     // A captured step is valid for one receive-buffer phase: consecutive exchanges alternate between the
     // two buffers, so a stack with an odd number of exchanges per step needs one graph per phase.
     const GraphKey key{x, seq_lens, block_table, out, B, max_pages, ctx_bucket, 1 + (int)(c.tp.exchanges & 1)};
-    const int rc = replay_or_run(c, key, [&]() { return run_tp(&c, x, out, (long)B * d.hidden * 2, B, tm, block_table, max_pages, true, ctx_bucket, st); }, st);
+    const int rc = replay_or_run(c, key, [&]() {
+        CU_TRY(timeline_restart(&c, st));
+        return run_tp(&c, x, out, (long)B * d.hidden * 2, B, tm, block_table, max_pages, true, ctx_bucket, st);
+    }, st);
     if (rc != SPD_OK) return rc;
     for (int l = 0; l < d.n_layers; ++l) c.tp.exchanges += c.mask[l] ? 2 : 1; // the same on every rank of the group
     return SPD_OK;
@@ -1440,6 +1539,50 @@ int spd_profile_end(spd_ctx *ctx, void *stream, float *ms_by_kind, int32_t *laun
     }
     c.ev_used = 0;
     c.ev_kind.clear();
+    return SPD_OK;
+}
+
+int spd_timeline_begin(spd_ctx *ctx)
+{
+    if (!ctx) return SPD_ENULL;
+    Ctx &c = ctx->c;
+    drop_graphs(c); // captured steps carry no stamp slots
+    c.timeline = true;
+    c.tl_next = 0;
+    c.tl_kind.clear();
+    return SPD_OK;
+}
+
+int spd_timeline_end(spd_ctx *ctx)
+{
+    if (!ctx) return SPD_ENULL;
+    Ctx &c = ctx->c;
+    drop_graphs(c);
+    c.timeline = false;
+    c.tl_next = 0;
+    c.tl_kind.clear();
+    return SPD_OK;
+}
+
+int spd_timeline_read(spd_ctx *ctx, void *stream, int32_t max_launches, int32_t *kinds, uint64_t *start_ns, uint64_t *end_ns,
+                      int32_t *n_launches)
+{
+    if (!ctx || !kinds || !start_ns || !end_ns || !n_launches) return SPD_ENULL;
+    Ctx &c = ctx->c;
+    if (!c.timeline || max_launches < 0) return SPD_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int n = c.tl_next < max_launches ? c.tl_next : max_launches;
+    std::vector<unsigned long long> host((size_t)2 * (n > 0 ? n : 1));
+    if (n > 0) CU_TRY(cudaMemcpyAsync(host.data(), c.stamps, (size_t)n * 16, cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaStreamSynchronize(st));
+    for (int i = 0; i < n; ++i) {
+        const unsigned long long s0 = host[2 * i], e1 = ~host[2 * i + 1];
+        const bool stamped = host[2 * i] != ~0ull && host[2 * i + 1] != ~0ull;
+        kinds[i] = c.tl_kind[i];
+        start_ns[i] = stamped ? s0 : 0;
+        end_ns[i] = stamped ? e1 : 0;
+    }
+    *n_launches = n;
     return SPD_OK;
 }
 

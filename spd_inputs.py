@@ -43,6 +43,8 @@ class Workload:
     rope_base: float = 10000.0
     kv_block: int = 16
     block: str = "llama"    # "llama": RMSNorm / rotary / SwiGLU, no bias; "opt": LayerNorm / biases / ReLU (Sec. 4.1.2)
+    prefill_batch: int = 0  # prompts of the prefill measurement when they differ from the decode batch (0: batch x prompt)
+    prefill_len: int = 0
 
     @property
     def torch_dtype(self):
@@ -81,7 +83,8 @@ WORKLOADS: Dict[str, Workload] = {
     "c3_t8": Workload("c3_t8", "bf16", 8, 5120, 40, 40, 128, 13824, 8, (1, 0, 0, 0, 0, 0, 0, 1), 16, 1024, 256),
     "c4_b1": Workload("c4_b1", "bf16", 8, 8192, 64, 8, 128, 28672, 8, (0,) * 8, 1, 2048, 256),
     "c4_b32": Workload("c4_b32", "bf16", 8, 8192, 64, 8, 128, 28672, 8, (0,) * 8, 32, 2048, 256),
-    "c5": Workload("c5", "bf16", 40, 8192, 64, 8, 128, 28672, 8, c5_mask(), 64, 512, 512),
+    # prefill of 4 x 4096 tokens; decode of batch 64 for 512 steps on caches pre-filled to 512 tokens
+    "c5": Workload("c5", "bf16", 40, 8192, 64, 8, 128, 28672, 8, c5_mask(), 64, 512, 512, prefill_batch=4, prefill_len=4096),
     # the block with bias (Sec. 4.1.2) at OPT-6.7B's shape (Sec. 5.1): 4 layers, hidden 4096, 32 heads x 128, ffn 16384
     "opt67": Workload("opt67", "bf16", 4, 4096, 32, 32, 128, 16384, 8, (0,) * 4, 8, 512, 128, block="opt"),
 }

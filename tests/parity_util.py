@@ -9,6 +9,15 @@ import oracle
 import spd_inputs as si
 
 TOL = {"fp32": 1e-4, "bf16": 2e-2}
+
+
+def stack_tol(dtype: str, depth: int) -> float:
+    """Bound on the output of `depth` blocks run one after the other on their own outputs.  The stated
+    tolerances are those of a block's output.  Behind one another the blocks' rounding errors (each at most
+    TOL, independent of each other) travel down the residual stream and add in quadrature: TOL * sqrt(depth).
+    (Measured at the 70B shape: 0.4-0.8e-2 per block fed with the oracle's input at every depth, 2.8e-2 after
+    eight blocks on their own outputs - about 1e-2 * sqrt(depth).)"""
+    return TOL[dtype] * float(np.sqrt(depth))
 _STREAM = None
 
 
@@ -109,6 +118,22 @@ class Pair:
                                      device=self.device)
         x = si.make_hidden(self.w, (self.B, S, self.w.hidden), "cpu", seed, 0)
         got = st.prefill(x.to(self.device), self.block_table)
+        torch.cuda.synchronize()
+        err = st.device_error()
+        st.close()
+        assert err == 0
+        return to_np(got).reshape(self.B * S, self.w.hidden)
+
+    def block_prefill(self, l, x_in, S):
+        """Block l alone on the GPU, fed with x_in [B*S, H] (the oracle's input of that block, rounded to the storage
+        dtype): its output [B*S, H] - the comparison that the per-block tolerance is stated for, at any depth."""
+        import paper_2502_20727_b200 as spd
+        w = self.w.with_(n_layers=1, mask=(self.mask[l],))
+        st = spd.stack_from_workload(w, self.layers_gpu[l:l + 1], sync_mask=[self.mask[l]], max_batch=self.B,
+                                     max_seq_len=self.max_len, n_pages=self.n_pages, max_prefill_tokens=self.B * S,
+                                     device=self.device)
+        x = torch.from_numpy(np.ascontiguousarray(x_in).reshape(self.B, S, self.w.hidden)).to(self.w.torch_dtype).to(self.device)
+        got = st.prefill(x, self.block_table)
         torch.cuda.synchronize()
         err = st.device_error()
         st.close()

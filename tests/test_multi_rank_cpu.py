@@ -59,3 +59,29 @@ def test_two_ranks_hold_one_shard_each_and_exchange_partial_sums():
         assert r["spd"]["err"] < 1e-12 and r["sync"]["err"] < 1e-12
         assert r["spd"]["exchanges"] == 1 == r["spd"]["syncs"]
         assert r["sync"]["exchanges"] == 2 == r["sync"]["syncs"]
+
+
+def test_bench_starts_its_own_ranks_when_no_launcher_did():
+    """`bench.py --gpus 2` without torchrun around it: the process becomes the launcher (one child per rank with RANK /
+    WORLD_SIZE / MASTER_* set), and still exactly one line comes out, from rank 0, saying n_gpus 2."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    env["OMP_NUM_THREADS"] = "2"
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "c1", "--gpus", "2",
+                        "--steps", "2", "--warmup", "1"], cwd=ROOT, env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    res = json.loads(lines[0])
+    assert res["impl"] == "reference" and res["n_gpus"] == 2 and res["value"] > 0
+
+
+def test_spawned_ranks_form_a_group_and_a_failing_rank_fails_the_job():
+    """spawn_ranks gives every child its rank and a common rendezvous: two gloo ranks find each other through it
+    (the worker checks world size, seeds and the max-over-ranks timing), and a non-zero exit of any rank is returned."""
+    sys.path.insert(0, ROOT)
+    import bench
+    env = dict(os.environ, OMP_NUM_THREADS="2")
+    for k in ("RANK", "LOCAL_RANK", "WORLD_SIZE"):
+        env.pop(k, None)
+    assert bench.spawn_ranks(2, [sys.executable, os.path.join(ROOT, "tests", "rank_worker.py")], env=env, timeout=600) == 0
+    assert bench.spawn_ranks(2, [sys.executable, "-c", "import os, sys; sys.exit(3 if os.environ['RANK'] == '1' else 0)"], env=env) == 3

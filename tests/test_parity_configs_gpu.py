@@ -1,5 +1,8 @@
 """GPU parity at the depth, widths and masks of the listed configurations: the CUDA library through its C ABI
-against the CPU oracle, element by element (max|gpu-ref|/max|ref| <= 2e-2, bfloat16).
+against the CPU oracle, element by element.  Two comparisons per stack: every block on its own, fed with the
+oracle's input of that block (max|gpu-ref|/max|ref| <= 2e-2, the bound stated for block outputs in bfloat16, at
+every depth), and the stack running on its own outputs (<= 2e-2 * sqrt(depth): the blocks' rounding errors add in
+quadrature along the residual stream).
 
 What the small-shape tests cannot show is covered here: whole 8-layer stacks at the 13B and 70B shapes with the
 configurations' own masks, the 40-layer stack with its seeded 25 %-sync mask (how the bfloat16 error grows with
@@ -12,43 +15,49 @@ import pytest
 import torch
 
 import spd_inputs as si
-from parity_util import TOL, Pair, rel_err
+from parity_util import TOL, Pair, rel_err, stack_tol, to_np
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
 def run_stack(w, mask, B, S, steps, *, depths=(), capsys=None, label=""):
-    """Prompt of S tokens per sequence, then `steps` decode steps; returns the prefill error per depth."""
+    """Prompt of S tokens per sequence, then `steps` decode steps.  depths: where the stack's output is also compared
+    inside the stack (contexts over the first d blocks); every block is compared on its own in any case.  Returns
+    (error of the stack after depth d, error of block d on the oracle's input)."""
     p = Pair(w, mask=mask, B=B, max_len=S + steps, max_prefill_tokens=B * S, weights_on=DEV, stream_oracle=True)
-    tol = TOL[w.dtype]
-    got, ref, syncs = p.prefill(S, want_layers=bool(depths))
+    L = w.n_layers
+    got, ref, syncs = p.prefill(S, want_layers=True)
     layer_out = p.layer_out
-    e = rel_err(got, ref)
-    assert e <= tol, f"{label} prefill rel err {e}"
-    assert p.stack.sync_points() == syncs == sum(2 if m else 1 for m in mask)
-    profile = {}
-    for depth in depths:
-        g = got.reshape(B * S, w.hidden) if depth == w.n_layers else p.prefix_prefill(depth, S)
-        profile[depth] = rel_err(g, layer_out[depth - 1])
-    if depths and capsys is not None:
+    x0 = to_np(si.make_hidden(w, (B, S, w.hidden), "cpu", 0, 0)).reshape(B * S, w.hidden)
+    per_block = [rel_err(p.block_prefill(l, x0 if l == 0 else layer_out[l - 1], S), layer_out[l]) for l in range(L)]
+    stack = {}
+    for depth in sorted(set(depths) | {L}):
+        g = got.reshape(B * S, w.hidden) if depth == L else p.prefix_prefill(depth, S)
+        stack[depth] = rel_err(g, layer_out[depth - 1])
+    if capsys is not None:
         with capsys.disabled():
-            print(f"\n[{label}] max-abs-rel error of the block output after depth d (mask {''.join(map(str, mask))}): "
-                  + ", ".join(f"d={d}: {v:.2e}" for d, v in profile.items()))
-    for depth, v in profile.items():
-        assert v <= tol, f"{label} depth {depth} rel err {v}"
+            print(f"\n[{label}] mask {''.join(map(str, mask))}; max-abs-rel error\n  block l on the oracle's input, l = 1..{L}: "
+                  + " ".join(f"{v:.1e}" for v in per_block) + "\n  stack on its own outputs after depth d: "
+                  + ", ".join(f"d={d}: {v:.1e}" for d, v in stack.items()))
+    for l, v in enumerate(per_block):
+        assert v <= TOL[w.dtype], f"{label} block {l} rel err {v}"
+    for depth, v in stack.items():
+        assert v <= stack_tol(w.dtype, depth), f"{label} depth {depth} rel err {v}"
+    assert p.stack.sync_points() == syncs == sum(2 if m else 1 for m in mask)
+    tol = stack_tol(w.dtype, L)
     for t in range(steps):
         got, ref = p.decode(t)
         e = rel_err(got, ref)
         assert e <= tol, f"{label} decode step {t} rel err {e}"
     n = S + steps
-    for l in (0, w.n_layers - 1):
+    for l in (0, L - 1):
         for which in ("k", "v"):
             e = rel_err(p.gpu_cache(l, which, B - 1, n), getattr(p.cache, which)[l, B - 1, :n])
-            assert e <= tol, f"{label} {which} cache layer {l} rel err {e}"
+            assert e <= stack_tol(w.dtype, l + 1), f"{label} {which} cache layer {l} rel err {e}"
     assert p.stack.device_error() == 0
     p.stack.close()
-    return profile
+    return stack, per_block
 
 
 def decode_on_synthetic_cache(w, mask, lens, steps, label=""):
@@ -60,7 +69,7 @@ def decode_on_synthetic_cache(w, mask, lens, steps, label=""):
     for t in range(steps):
         got, ref = p.decode(t)
         e = rel_err(got, ref)
-        assert e <= TOL[w.dtype], f"{label} decode step {t} rel err {e}"
+        assert e <= stack_tol(w.dtype, w.n_layers), f"{label} decode step {t} rel err {e}"
     assert p.stack.device_error() == 0
     p.stack.close()
 
@@ -86,7 +95,7 @@ def test_prompt_over_several_tiles_at_70b_widths(mask):
     of the 8192 / 28672 wide projections - for the SPD block the T-pass o_proj tile -, three query tiles of the
     tensor-core attention with 8 query heads per KV head; then one decode step on the cache it filled."""
     w = si.WORKLOADS["c4_b1"].with_(n_layers=1, mask=mask)
-    run_stack(w, mask, 1, 300, 1, label=f"70B widths mask {mask}")
+    run_stack(w, mask, 1, 300, 1, capsys=None, label=f"70B widths mask {mask}")
 
 
 def test_c5_decode_tiles_of_64_at_70b_widths():
@@ -105,8 +114,8 @@ def test_c5_mask_40_layers_reduced_width(capsys):
     that it always runs: prompts with the error after depth 1 ... 40, decode steps, and decode batches of 64."""
     w = si.WORKLOADS["c5"].with_(**C5_SMALL)
     assert sum(w.mask) == 10 and len(w.mask) == 40
-    prof = run_stack(w, w.mask, 2, 40, 2, depths=(1, 2, 5, 10, 20, 30, 40), capsys=capsys, label="c5 mask, width/8")
-    assert prof[40] <= TOL["bf16"]
+    stack, _ = run_stack(w, w.mask, 2, 40, 2, depths=(1, 2, 5, 10, 20, 30, 40), capsys=capsys, label="c5 mask, width/8")
+    assert stack[40] <= TOL["bf16"]  # at this width the early blocks dominate the stream: no growth with depth
     decode_on_synthetic_cache(w, w.mask, 1 + (np.arange(64) * 29) % 70, 2, label="c5 mask, width/8, B=64")
 
 
