@@ -204,21 +204,6 @@ def captured_traffic(w: si.Workload):
     return None
 
 
-def exclusive_times(tl):
-    """[(kind, start, end)] of one call, in launch order -> ({kind: ns that only this launch accounts for}, span ns).
-    Launches overlap (the next one starts under the tail of the one before): launch i's own share of the call is
-    end_i - max(start_i, end_{i-1}), so the shares add up to at most the call's span."""
-    own, prev_end, first = {}, None, None
-    for kind, t0, t1 in tl:
-        if t1 == 0:
-            continue
-        first = t0 if first is None else min(first, t0)
-        begin = t0 if prev_end is None else max(t0, prev_end)
-        own[kind] = own.get(kind, 0) + max(0, t1 - begin)
-        prev_end = t1 if prev_end is None else max(prev_end, t1)
-    return own, (0 if first is None else prev_end - first)
-
-
 # ----------------------------------------------------------------------------------------
 class Run:
     """One configuration resident on the device: weights, stack, block tables."""
@@ -301,8 +286,18 @@ class Run:
         torch.cuda.synchronize()
         self.filled = True
 
+    def settle(self, seconds):
+        """Untimed decode steps at the starting context until the GPU has been under THIS load for `seconds`: the prompt
+        phase before it runs the chip into its power cap, and the clocks need a moment to find the decode level."""
+        t0 = time.perf_counter()
+        while time.perf_counter() - t0 < seconds:
+            for _ in range(self.W):
+                self.step(0)
+            torch.cuda.synchronize()
+
     def decode_ms(self, barrier):
-        """W warm-up steps, then K timed steps between two events: (ms, host window)."""
+        """Settling, W warm-up steps, then K timed steps between two events: (ms, host window)."""
+        self.settle(self.args.settle_s)
         for t in range(self.W):
             self.step(t)
         barrier()
@@ -318,26 +313,30 @@ class Run:
             raise RuntimeError("device error flag set during the timed region")
         return e0.elapsed_time(e1), (h0, h1)
 
-    def timeline(self, n_steps):
-        """Per-kind share of a decode step from the kernels' own start / end stamps inside the replayed graph."""
-        self.stack.timeline_begin()
+    def timeline(self, barrier):
+        """Every launch's own share of a decode step, from the kernels' start / end stamps folded on the device, over K
+        steps replayed back to back exactly as in the timed region (and timed the same way, for comparison)."""
         base = 2 * (self.W + self.K)
-        for t in range(3):
+        self.stack.timeline_begin()
+        for t in range(self.W):
             self.step(base + t)
-        self.stack.timeline_read()
-        own_ns, spans, launches = {}, [], {}
-        for i in range(n_steps):
-            self.step(base + 3 + i)
-            tl = self.stack.timeline_read()
-            own, span = exclusive_times(tl)
-            spans.append(span)
-            for k, v in own.items():
-                own_ns[k] = own_ns.get(k, 0) + v
-            if i == 0:
-                for k, _, t1 in tl:
-                    launches[k] = launches.get(k, 0) + (1 if t1 else 0)
+        barrier()
+        self.stack.timeline_begin()  # clear the totals of the warm-up steps
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for t in range(self.W, self.W + self.K):
+            self.step(base + t)
+        e1.record()
+        barrier()
+        per_launch, span_ns, calls = self.stack.timeline_read()
         self.stack.timeline_end()
-        return {k: v / n_steps * 1e-6 for k, v in own_ns.items()}, float(np.mean(spans)) * 1e-6, launches
+        if calls != self.K:
+            raise RuntimeError(f"timeline folded {calls} calls, expected {self.K}")
+        own_ms, launches = {}, {}
+        for kind, ns in per_launch:
+            own_ms[kind] = own_ms.get(kind, 0.0) + ns / calls * 1e-6
+            launches[kind] = launches.get(kind, 0) + 1
+        return own_ms, span_ns / calls * 1e-6, launches, e0.elapsed_time(e1) / self.K
 
 
 def roofline_entry(w, B, mid_ctx, ms_per_step, hbm_peak, peak_kind):
@@ -438,9 +437,10 @@ def run_native(args, rank, world):
         # ---- where the step's time goes ------------------------------------------------------
         gw = gemm_weight_bytes(w)
         if fused:
-            kind_ms, span_ms, kind_launches = run.timeline(min(K, 16))
-            how = ("kernel start/end stamps inside the replayed graph; a launch's share = its end minus the later of its "
-                   "start and the previous launch's end, so the shares add up to at most the step")
+            kind_ms, span_ms, kind_launches, tl_step_ms = run.timeline(barrier)
+            how = ("kernel start/end stamps folded on the device over K graph-replayed steps issued back to back as in the timed "
+                   "region; a launch's share = its end minus the later of its start and the latest end before it, so the shares "
+                   "add up to at most the step; timeline_ms_per_step is that pass timed with events like ms_per_step")
         else:
             for t in range(3):
                 run.step(2 * (W + K) + t)
@@ -452,7 +452,7 @@ def run_native(args, rank, world):
             prof = run.stack.profile_end()
             kind_ms = {k: v["ms"] / n_prof for k, v in prof.items()}
             kind_launches = {k: v["launches"] // n_prof for k, v in prof.items()}
-            span_ms = None
+            span_ms = tl_step_ms = None
             how = "events around every launch: serialised (no overlap between launches), a lower bound of what the kernels reach in the step"
 
         dev_ms, e2e_s = max_over_ranks([dev_ms, e2e_s], dev)
@@ -490,7 +490,8 @@ def run_native(args, rank, world):
                              "algorithmic_bytes_per_launch": gemm_bytes_step / max(gemm_launches, 1), "peak_kind": peak_kind,
                              "launches_per_step": gemm_launches, "avg_launch_us": gemm_ms * 1e3 / max(gemm_launches, 1),
                              "bytes_per_step": gemm_bytes_step, "how": how, "by_kind": by_kind},
-                "kernel_ms_per_step": kind_ms, "sum_kernel_ms": sum(kind_ms.values()), "timeline_step_ms": span_ms,
+                "kernel_ms_per_step": kind_ms, "sum_kernel_ms": sum(kind_ms.values()), "timeline_span_ms": span_ms,
+                "timeline_ms_per_step": tl_step_ms,
                 "prefill": prefill_entry(w, run.Bp, run.Sp, pre_ms, tf_peak),
             }
 
@@ -623,6 +624,7 @@ def main():
     ap.add_argument("--prefill-chunk", type=int, default=8192)
     ap.add_argument("--prefill-reps", type=int, default=3)
     ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--settle-s", type=float, default=0.5, help="seconds of untimed decode steps before every timed decode region")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--rank-mode", action="store_true",
                     help="decode through spd_tp_decode_step: all T ranks of a tensor-parallel group executed on this GPU")

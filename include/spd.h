@@ -347,25 +347,30 @@ int spd_profile_end(spd_ctx *ctx, void *stream, float *ms_by_kind, int32_t *laun
 int spd_profile_kinds(void);
 const char *spd_profile_kind_name(int kind);
 
-/* Launch timeline for benchmarks: when and how long every kernel of a call ran INSIDE the call as it is
- * normally issued - decode steps replayed from their graph, launches overlapping through programmatic
- * dependent launch - with nothing inserted between the launches (spd_profile_* brackets every launch with
- * events, which serialises them).  After spd_timeline_begin every kernel of the bf16 prompt and decode paths
- * (block_kind 0; the kernels of the other paths carry no stamps and are left out) gets a slot in the
- * workspace; one thread of each of its blocks records the GPU's global nanosecond timer at block start and
- * end, and the slot keeps the earliest start and the latest end.  Each spd_prefill / spd_decode_step /
- * spd_tp_decode_step call starts the slots afresh, so read after every call:
- *   spd_timeline_read : synchronises `stream`; for the first min(launches, max_launches) launches of the
- *                       last call, in launch order: kinds[i] (index of spd_profile_kind_name), start_ns[i],
- *                       end_ns[i] (both 0 for a launch that did not run); *n_launches = entries written.
- *                       A call with more than 6 * n_layers + 16 launches (chunked prompts) reports the first ones.
- * Consecutive launches overlap (the next kernel's blocks start, and request their first weights, under the
- * tail of the one before): end[i] - max(start[i], end[i-1]) is launch i's own share of the call's duration.
- * spd_timeline_begin / _end drop the captured decode graphs (a step is captured again with / without slots).
+/* Launch timeline for benchmarks: how much of a call's duration every kernel accounts for INSIDE the call as it
+ * is normally issued - decode steps replayed from their graph, back to back, launches overlapping through
+ * programmatic dependent launch - with nothing inserted between the launches and no host round trip between
+ * the calls (spd_profile_* brackets every launch with events, which serialises them).  After spd_timeline_begin
+ * every kernel of the bf16 prompt and decode paths (block_kind 0; the kernels of the other paths carry no stamps
+ * and are left out) gets a slot in the workspace: one thread of each of its blocks records the GPU's global
+ * nanosecond timer at block start and end, the slot keeps the earliest start and the latest end.  A small
+ * kernel at the end of each spd_prefill / spd_decode_step / spd_tp_decode_step call (part of the captured
+ * step) folds the stamps into running totals: launch i's own share of the call = end[i] minus the later of
+ * start[i] and the latest end before it (consecutive launches overlap: the next kernel's blocks start, and
+ * request their first weights, under the tail of the one before), and the call's span = latest end - earliest
+ * start; the shares add up to at most the span.
+ *   spd_timeline_begin : presets slots and totals on `stream`; the first begin drops the captured decode graphs (a
+ *                        step is captured again, with slots), a further begin only clears the totals
+ *   spd_timeline_read  : synchronises `stream`; totals since spd_timeline_begin over *n_calls calls, for the first
+ *                        min(launches of the last call, max_launches) launches in launch order: kinds[i] (index
+ *                        of spd_profile_kind_name) and own_ns[i]; *span_ns = sum of the calls' spans.  Meaningful
+ *                        when all calls since begin had the same launch sequence (same call, B, mask).  A call
+ *                        with more than 6 * n_layers + 16 launches (chunked prompts) accounts for the first ones.
+ *   spd_timeline_end   : stops stamping, drops the captured graphs
  * Errors: SPD_ENULL, SPD_EINVAL (read without begin), SPD_ECUDA. */
-int spd_timeline_begin(spd_ctx *ctx);
-int spd_timeline_read(spd_ctx *ctx, void *stream, int32_t max_launches, int32_t *kinds, uint64_t *start_ns,
-                      uint64_t *end_ns, int32_t *n_launches);
+int spd_timeline_begin(spd_ctx *ctx, void *stream);
+int spd_timeline_read(spd_ctx *ctx, void *stream, int32_t max_launches, int32_t *kinds, uint64_t *own_ns,
+                      int32_t *n_launches, uint64_t *span_ns, uint64_t *n_calls);
 int spd_timeline_end(spd_ctx *ctx);
 
 /* Free the context (host state, descriptors, graphs).  Never touches caller tensors. */

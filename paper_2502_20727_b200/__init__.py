@@ -98,10 +98,10 @@ def load_library() -> ctypes.CDLL:
     lib.spd_tp_prefill.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp]
     lib.spd_profile_begin.argtypes = [vp]
     lib.spd_profile_end.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
-    lib.spd_timeline_begin.argtypes = [vp]
+    lib.spd_timeline_begin.argtypes = [vp, vp]
     lib.spd_timeline_end.argtypes = [vp]
-    lib.spd_timeline_read.argtypes = [vp, vp, i32, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_uint64),
-                                      ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(i32)]
+    lib.spd_timeline_read.argtypes = [vp, vp, i32, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(i32),
+                                      ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)]
     lib.spd_profile_kinds.argtypes = []
     lib.spd_profile_kind_name.argtypes = [ctypes.c_int]
     lib.spd_profile_kind_name.restype = ctypes.c_char_p
@@ -372,23 +372,26 @@ class SpdStack:
                 for i in range(n)}
 
     def timeline_begin(self):
-        """Stamp every kernel of the following calls (start / end on the GPU's nanosecond timer); see spd_timeline_begin."""
-        _check("spd_timeline_begin", self.lib.spd_timeline_begin(self._ctx))
+        """Stamp every kernel of the following calls and fold the stamps into per-launch totals; see spd_timeline_begin."""
+        with torch.cuda.device(self.device):
+            _check("spd_timeline_begin", self.lib.spd_timeline_begin(self._ctx, _stream_ptr()))
 
     def timeline_end(self):
         _check("spd_timeline_end", self.lib.spd_timeline_end(self._ctx))
 
     def timeline_read(self):
-        """[(kind name, start_ns, end_ns)] of the last call's launches, in launch order; see spd_timeline_read."""
+        """([(kind name, own_ns summed over the calls)] in launch order, span_ns summed, number of calls) since
+        timeline_begin; see spd_timeline_read."""
         cap = 6 * self.dims.n_layers + 16
         kinds = (ctypes.c_int32 * cap)()
-        t0 = (ctypes.c_uint64 * cap)()
-        t1 = (ctypes.c_uint64 * cap)()
+        own = (ctypes.c_uint64 * cap)()
         n = ctypes.c_int32(0)
+        span, calls = ctypes.c_uint64(0), ctypes.c_uint64(0)
         with torch.cuda.device(self.device):
-            _check("spd_timeline_read", self.lib.spd_timeline_read(self._ctx, _stream_ptr(), cap, kinds, t0, t1, ctypes.byref(n)))
+            _check("spd_timeline_read", self.lib.spd_timeline_read(self._ctx, _stream_ptr(), cap, kinds, own, ctypes.byref(n),
+                                                                    ctypes.byref(span), ctypes.byref(calls)))
         names = [self.lib.spd_profile_kind_name(i).decode() for i in range(self.lib.spd_profile_kinds())]
-        return [(names[kinds[i]], int(t0[i]), int(t1[i])) for i in range(n.value)]
+        return [(names[kinds[i]], int(own[i])) for i in range(n.value)], int(span.value), int(calls.value)
 
     def set_mask(self, sync_mask: Sequence[int]):
         """Replace the per-block mask (1 = TP block, 0 = SPD block); see spd_set_mask."""

@@ -4,16 +4,16 @@
 // One thread block per (128 queries, query head, sequence).  Per tile of 128 cached keys:
 //   S = Q K^T      tcgen05.mma, Q and K as K-major 128B-swizzled tiles (K pages land there as
 //                  TMA boxes of 16 tokens x 64 dims), accumulator in tensor memory
-//   P = softmax    warps 0-7: thread = (query row = TMEM lane, half of the tile's 128 columns); the
-//                  two threads of a row exchange their maxima through shared memory; running
+//   P = softmax    warps 0-15: thread = (query row = TMEM lane, a quarter of the tile's 128 columns); the
+//                  four threads of a row exchange their maxima through shared memory; running
 //                  maximum and sums in base 2, P rounded to bf16 into a K-major swizzled tile
 //   O += P V       tcgen05.mma with V as the MN-major operand: V pages are [token][dim], i.e.
 //                  rows of the K dimension with the N dimension contiguous, exactly as TMA
 //                  delivers them; O accumulates in tensor memory over all tiles and is rescaled
 //                  there (load, multiply, store) only when the running maximum has grown by
 //                  more than 2^8 since the last rescale; S of the next tile is computed meanwhile
-// S is double-buffered in tensor memory, K and V tiles in two-stage rings (one for K, one for V).  Warps 8 and 9 issue the TMA loads, warp 10 the MMAs.
-// Every wait is bounded.
+// S is double-buffered in tensor memory, K and V tiles in two-stage rings (one for K, one for V).  19 warps:
+// 0-15 softmax, 16 loads Q and the K tiles, 17 the V tiles (TMA), 18 issues the MMAs.  Every wait is bounded.
 #include "common.cuh"
 #include "gemm_tc.cuh"
 #include "tc_ptx.cuh"

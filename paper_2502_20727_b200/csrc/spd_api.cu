@@ -167,13 +167,71 @@ unsigned long long *next_stamp(Ctx *c, int kind)
     return c->stamps + 2 * (size_t)c->tl_next++;
 }
 
-// A call starts its timeline afresh: slots preset to all ones, in stream order before the first launch.
-cudaError_t timeline_restart(Ctx *c, cudaStream_t st)
+// A call starts its timeline afresh (the slots were preset by spd_timeline_begin or by the fold of the call before).
+cudaError_t timeline_restart(Ctx *c, cudaStream_t)
 {
     if (!c->timeline) return cudaSuccess;
     c->tl_next = 0;
     c->tl_kind.clear();
-    return cudaMemsetAsync(c->stamps, 0xFF, (size_t)c->stamps_cap * 16, st);
+    return cudaSuccess;
+}
+
+// Last launch of a stamped call.  Turns the stamps into every launch's own share of the call - its end minus the
+// later of its start and the latest end of the launches before it, so overlapping launches are not counted twice
+// and the shares add up to at most the call's span -, adds shares and span to running totals and presets the
+// slots for the next call: stamped steps can then run back to back, replayed from their graph, with no host
+// round trip in between.  acc: [cap] shares, then span, then number of calls (all in ns / counts, 64-bit).
+__global__ void __launch_bounds__(256) timeline_fold_kernel(unsigned long long *slots, int n, unsigned long long *acc, int cap)
+{
+    pdl_launch_dependents();
+    pdl_wait(); // every launch of the call has completed: each waited for the one before it
+    __shared__ unsigned long long sm_end[256];
+    __shared__ unsigned long long sm_carry, sm_first;
+    const int t = threadIdx.x;
+    if (t == 0) { sm_carry = 0; sm_first = ~0ull; }
+    __syncthreads();
+    for (int base = 0; base < n; base += 256) {
+        const int i = base + t;
+        unsigned long long s = 0, e = 0;
+        bool ok = false;
+        if (i < n) {
+            const unsigned long long a = slots[2 * i], b = slots[2 * i + 1];
+            ok = a != ~0ull && b != ~0ull;
+            s = a; e = ok ? ~b : 0;
+            slots[2 * i] = ~0ull; slots[2 * i + 1] = ~0ull;
+        }
+        // inclusive running maximum of the ends (launches that did not run count as 0)
+        sm_end[t] = e;
+        __syncthreads();
+        for (int d = 1; d < 256; d <<= 1) {
+            const unsigned long long o = t >= d ? sm_end[t - d] : 0;
+            __syncthreads();
+            if (o > sm_end[t]) sm_end[t] = o;
+            __syncthreads();
+        }
+        const unsigned long long carry = sm_carry;
+        unsigned long long before = t > 0 ? sm_end[t - 1] : 0;
+        if (carry > before) before = carry;
+        if (ok) {
+            const unsigned long long begin = s > before ? s : before;
+            if (e > begin) acc[i] += e - begin;
+            atomicMin(&sm_first, s);
+        }
+        __syncthreads();
+        if (t == 255) sm_carry = sm_end[255] > carry ? sm_end[255] : carry;
+        __syncthreads();
+    }
+    if (t == 0) {
+        if (sm_first != ~0ull && sm_carry > sm_first) acc[cap] += sm_carry - sm_first;
+        acc[cap + 1] += 1;
+    }
+}
+
+cudaError_t timeline_fold(Ctx *c, cudaStream_t st)
+{
+    if (!c->timeline || c->tl_next == 0) return cudaSuccess;
+    return launch_kernel(timeline_fold_kernel, dim3(1), dim3(256), 0, st, 0, c->stamps, c->tl_next,
+                         c->stamps + 2 * (size_t)c->stamps_cap, c->stamps_cap);
 }
 
 #define LAUNCH(kind, expr)                   \
@@ -308,7 +366,7 @@ Layout make_layout(const spd_dims &d, bool any_spd)
     const size_t h_tiles = (H + 127) / 128;
     L.ss_attn = take(h_tiles * Mmax * 4);
     L.ss_mlp = take(2 * h_tiles * T * Mmax * 4); // the SPD o_proj of the prefill path leaves two partials per tile
-    L.stamps = take((size_t)stamp_slots(d) * 16);
+    L.stamps = take((size_t)stamp_slots(d) * 16 + ((size_t)stamp_slots(d) + 2) * 8); // slots, then the running totals
     L.total = off;
     return L;
 }
@@ -1199,6 +1257,7 @@ int spd_prefill(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int32_t
             }
     }
     c.launches_last = total_launches;
+    CU_TRY(timeline_fold(&c, st));
     return SPD_OK;
 }
 
@@ -1224,10 +1283,13 @@ int spd_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_l
     const int ctx_bucket = bucket_of(max_context);
     auto run_at = [&](int bucket) {
         return [&, bucket]() -> int {
-            CU_TRY(timeline_restart(&c, st)); // inside the captured step: every replay presets the slots first
-            return d.dtype == 0        ? run_tokens<float>(&c, x, out, B, tm, block_table, max_pages, true, bucket, st)
-                   : d.block_kind == 0 ? run_decode_fused(&c, x, out, B, tm, block_table, max_pages, bucket, st)
-                                       : run_tokens<bf16>(&c, x, out, B, tm, block_table, max_pages, true, bucket, st);
+            CU_TRY(timeline_restart(&c, st));
+            const int rc = d.dtype == 0        ? run_tokens<float>(&c, x, out, B, tm, block_table, max_pages, true, bucket, st)
+                           : d.block_kind == 0 ? run_decode_fused(&c, x, out, B, tm, block_table, max_pages, bucket, st)
+                                               : run_tokens<bf16>(&c, x, out, B, tm, block_table, max_pages, true, bucket, st);
+            if (rc != SPD_OK) return rc;
+            CU_TRY(timeline_fold(&c, st)); // part of the captured step: every replay folds its own stamps
+            return SPD_OK;
         };
     };
     const GraphKey key{x, seq_lens, block_table, out, B, max_pages, ctx_bucket, 0};
@@ -1471,7 +1533,10 @@ int spd_tp_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *se
     const GraphKey key{x, seq_lens, block_table, out, B, max_pages, ctx_bucket, 1 + (int)(c.tp.exchanges & 1)};
     const int rc = replay_or_run(c, key, [&]() {
         CU_TRY(timeline_restart(&c, st));
-        return run_tp(&c, x, out, (long)B * d.hidden * 2, B, tm, block_table, max_pages, true, ctx_bucket, st);
+        const int rc2 = run_tp(&c, x, out, (long)B * d.hidden * 2, B, tm, block_table, max_pages, true, ctx_bucket, st);
+        if (rc2 != SPD_OK) return rc2;
+        CU_TRY(timeline_fold(&c, st));
+        return SPD_OK;
     }, st);
     if (rc != SPD_OK) return rc;
     for (int l = 0; l < d.n_layers; ++l) c.tp.exchanges += c.mask[l] ? 2 : 1; // the same on every rank of the group
@@ -1542,11 +1607,14 @@ int spd_profile_end(spd_ctx *ctx, void *stream, float *ms_by_kind, int32_t *laun
     return SPD_OK;
 }
 
-int spd_timeline_begin(spd_ctx *ctx)
+int spd_timeline_begin(spd_ctx *ctx, void *stream)
 {
     if (!ctx) return SPD_ENULL;
     Ctx &c = ctx->c;
-    drop_graphs(c); // captured steps carry no stamp slots
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!c.timeline) drop_graphs(c); // steps captured so far carry no stamp slots; a second begin only clears the totals
+    CU_TRY(cudaMemsetAsync(c.stamps, 0xFF, (size_t)c.stamps_cap * 16, st));
+    CU_TRY(cudaMemsetAsync(c.stamps + 2 * (size_t)c.stamps_cap, 0, ((size_t)c.stamps_cap + 2) * 8, st));
     c.timeline = true;
     c.tl_next = 0;
     c.tl_kind.clear();
@@ -1564,25 +1632,21 @@ int spd_timeline_end(spd_ctx *ctx)
     return SPD_OK;
 }
 
-int spd_timeline_read(spd_ctx *ctx, void *stream, int32_t max_launches, int32_t *kinds, uint64_t *start_ns, uint64_t *end_ns,
-                      int32_t *n_launches)
+int spd_timeline_read(spd_ctx *ctx, void *stream, int32_t max_launches, int32_t *kinds, uint64_t *own_ns, int32_t *n_launches,
+                      uint64_t *span_ns, uint64_t *n_calls)
 {
-    if (!ctx || !kinds || !start_ns || !end_ns || !n_launches) return SPD_ENULL;
+    if (!ctx || !kinds || !own_ns || !n_launches || !span_ns || !n_calls) return SPD_ENULL;
     Ctx &c = ctx->c;
     if (!c.timeline || max_launches < 0) return SPD_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
     const int n = c.tl_next < max_launches ? c.tl_next : max_launches;
-    std::vector<unsigned long long> host((size_t)2 * (n > 0 ? n : 1));
-    if (n > 0) CU_TRY(cudaMemcpyAsync(host.data(), c.stamps, (size_t)n * 16, cudaMemcpyDeviceToHost, st));
+    std::vector<unsigned long long> host((size_t)c.stamps_cap + 2);
+    CU_TRY(cudaMemcpyAsync(host.data(), c.stamps + 2 * (size_t)c.stamps_cap, host.size() * 8, cudaMemcpyDeviceToHost, st));
     CU_TRY(cudaStreamSynchronize(st));
-    for (int i = 0; i < n; ++i) {
-        const unsigned long long s0 = host[2 * i], e1 = ~host[2 * i + 1];
-        const bool stamped = host[2 * i] != ~0ull && host[2 * i + 1] != ~0ull;
-        kinds[i] = c.tl_kind[i];
-        start_ns[i] = stamped ? s0 : 0;
-        end_ns[i] = stamped ? e1 : 0;
-    }
+    for (int i = 0; i < n; ++i) { kinds[i] = c.tl_kind[i]; own_ns[i] = host[i]; }
     *n_launches = n;
+    *span_ns = host[c.stamps_cap];
+    *n_calls = host[(size_t)c.stamps_cap + 1];
     return SPD_OK;
 }
 

@@ -1,5 +1,4 @@
-"""Host-side logic of bench.py that needs no GPU: the per-launch accounting of a step's timeline, the masks a
-configuration is run with, the bounded oracle sample, and the byte / flop counts of the roofline."""
+"""Host-side logic of bench.py that needs no GPU: the masks a configuration is run with, the bounded oracle sample, and the byte / flop counts of the roofline."""
 import os
 import sys
 
@@ -8,15 +7,6 @@ sys.path.insert(0, ROOT)
 
 import bench  # noqa: E402
 import spd_inputs as si  # noqa: E402
-
-
-def test_overlapping_launches_share_the_step_without_double_counting():
-    # launch b starts under a's tail, c after a gap, d never ran
-    tl = [("a", 100, 200), ("b", 150, 260), ("c", 300, 330), ("d", 0, 0), ("b", 320, 400)]
-    own, span = bench.exclusive_times(tl)
-    assert own == {"a": 100, "b": 60 + 70, "c": 30}
-    assert span == 300 and sum(own.values()) <= span
-    assert bench.exclusive_times([]) == ({}, 0)
 
 
 def test_masks_per_configuration():
