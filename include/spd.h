@@ -164,6 +164,10 @@ int spd_set_graphs(spd_ctx *ctx, int32_t enabled);
  *       when the maximum has grown by more than 2^value since the last rescale (default 8, at
  *       most 16; 0 = follow the maximum exactly, every growth rescales).  The result is the same
  *       softmax either way; only the rounding of the bf16 probabilities differs.
+ *   "prefill_pairs"
+ *       prompt projections on pairs of thread blocks (one 256-token tile and one tensor-core instruction over
+ *       two SMs, each block loading half of the tile's weight rows): 1 (default) wherever a launch has more
+ *       than 128 tokens, 0 = always one block per 128-token tile.  Same results bit for bit.
  *   "peer_wait_ms"
  *       rank mode (spd_tp_*): milliseconds a rank waits for the other ranks' partial sums before
  *       it gives up with error bit 8 (default and value 0: 1000; at most 60000).  Always bounded.

@@ -29,9 +29,12 @@ constexpr int TMEM_ALL = 512;
 constexpr int TOT_COL = 256; // PRE_OPROJ_SPD: X + running sum of the Y_i
 constexpr int X_COL = 384;   // PRE_OPROJ_SPD: the X tile
 
-template <int EPI> struct PCfg {
+// PAIR: two CTAs of a cluster work on one tile of 256 tokens as one M = 256 MMA (cta_group::2): each loads its own
+// 128 token rows and HALF of the tile's weight rows, so per MMA flop only two thirds (three quarters for the SPD
+// o_proj) of the operand bytes cross from L2 into shared memory, and the ring holds more K blocks.
+template <int EPI, int PAIR> struct PCfg {
     static constexpr int BN = (EPI == PRE_OPROJ_SPD) ? 128 : 256;
-    static constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
+    static constexpr int A_BYTES = BM * BK * 2, B_BYTES = (BN / (PAIR ? 2 : 1)) * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     // PRE_OPROJ_SPD stages outgoing R_i * g tiles (bf16, 32 KB each) in shared memory
     static constexpr int X_BYTES = 0, H_BYTES = (EPI == PRE_OPROJ_SPD) ? 2 * 128 * 128 * 2 : 0; // two staging tiles
@@ -46,7 +49,7 @@ template <int EPI> struct PCfg {
 
 struct PreLaunch {
     PreGemmArgs g;
-    int m_tiles, n_tiles, passes;
+    int m_tiles, n_tiles, passes; // m_tiles: token tiles of 128 rows, or of 256 for a CTA pair
     int tile_start[3]; // QKV: first n-tile of weight i
     int f_tiles;       // GATEUP: n-tiles per device
 };
@@ -59,11 +62,11 @@ struct PreTile {
     int nt;     // n-tile index (for the sums of squares)
 };
 
-__device__ __forceinline__ PreTile decode_tile(const PreLaunch &L, int EPI, int tile)
+__device__ __forceinline__ PreTile decode_tile(const PreLaunch &L, int EPI, int tile, int pair, int crank)
 {
     PreTile t;
     const int mt = tile % L.m_tiles, nt = tile / L.m_tiles;
-    t.m0 = mt * BM;
+    t.m0 = pair ? mt * 2 * BM + crank * BM : mt * BM; // this CTA's 128 token rows
     t.nt = nt;
     t.wi = 0;
     t.z = 0;
@@ -401,8 +404,8 @@ __device__ __forceinline__ float epi_oproj_spd(const PreGemmArgs &g, const PreTi
     return ssq;
 }
 
-template <int EPI>
-__global__ void __launch_bounds__(PCfg<EPI>::THREADS_, 1) gemm_prefill_kernel(const __grid_constant__ CUtensorMap tm_w0,
+template <int EPI, int PAIR>
+__global__ void __launch_bounds__(PCfg<EPI, PAIR>::THREADS_, 1) gemm_prefill_kernel(const __grid_constant__ CUtensorMap tm_w0,
                                                                   const __grid_constant__ CUtensorMap tm_w1,
                                                                   const __grid_constant__ CUtensorMap tm_w2,
                                                                   const __grid_constant__ CUtensorMap tm_t,
@@ -411,9 +414,13 @@ __global__ void __launch_bounds__(PCfg<EPI>::THREADS_, 1) gemm_prefill_kernel(co
                                                                   const __grid_constant__ CUtensorMap tm_h,
                                                                   const __grid_constant__ PreLaunch L)
 {
-    using C = PCfg<EPI>;
+    using C = PCfg<EPI, PAIR>;
     constexpr int BN = C::BN, S = C::STAGES;
     const PreGemmArgs &g = L.g;
+    // a pair's leader (even cluster rank) issues the MMAs for both CTAs and owns the barriers they are counted on
+    const int crank = PAIR ? (int)cluster_ctarank() : 0;
+    const bool leader = crank == 0;
+    const int tile0 = PAIR ? (int)blockIdx.x / 2 : (int)blockIdx.x, tile_step = PAIR ? (int)gridDim.x / 2 : (int)gridDim.x;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
@@ -434,17 +441,24 @@ __global__ void __launch_bounds__(PCfg<EPI>::THREADS_, 1) gemm_prefill_kernel(co
     if (threadIdx.x == 0) {
         stamp_entry(g.stamp);
         for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), C::EPI_WARPS); }
+        // an accumulator is free again when the epilogue warps of both CTAs of a pair have drained their rows
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), C::EPI_WARPS * (PAIR ? 2 : 1)); }
         mbar_init(xfull_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 5) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_ALL) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (PAIR) { // one allocation over the tensor memory of both CTAs, made by the same warp of each
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_ALL) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_ALL) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
+    if (PAIR) cluster_sync(); // the partner's barriers are initialised before anything of ours can reach them
+    else __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
     pdl_wait();
@@ -453,10 +467,11 @@ __global__ void __launch_bounds__(PCfg<EPI>::THREADS_, 1) gemm_prefill_kernel(co
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_w0) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_t) : "memory");
+            const uint64_t keep = policy_evict_normal();
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const PreTile t = decode_tile(L, EPI, tile);
+            for (int tile = tile0; tile < total_tiles && ok; tile += tile_step) {
+                const PreTile t = decode_tile(L, EPI, tile, PAIR, crank);
                 const CUtensorMap *tm_w = t.wi == 0 ? &tm_w0 : (t.wi == 1 ? &tm_w1 : &tm_w2);
                 for (int pass = 0; pass < L.passes && ok; ++pass) {
                     const int tz = EPI == PRE_OPROJ_SPD ? pass : (EPI == PRE_GATEUP && g.t_batched ? t.z : 0);
@@ -464,26 +479,41 @@ __global__ void __launch_bounds__(PCfg<EPI>::THREADS_, 1) gemm_prefill_kernel(co
                     for (int kb = 0; kb < g.num_kb; ++kb, ++it) {
                         const int s = it % S;
                         if (!mbar_wait(empty_bar(s), ((it / S) & 1) ^ 1, g.err, abort_flag)) { ok = false; break; }
-                        mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
                         const uint32_t sa = base + s * C::STAGE_BYTES, sb = sa + C::A_BYTES;
-                        tma_load_3d(sa, &tm_t, kb * BK, t.m0, tz, full_bar(s));
-                        if (EPI == PRE_GATEUP) {
-                            tma_load_3d(sb, &tm_w0, kb * BK, t.row0, wz, full_bar(s));
-                            tma_load_3d(sb + 128 * BK * 2, &tm_w1, kb * BK, t.row0, wz, full_bar(s));
+                        if (PAIR) {
+                            // both CTAs' bytes of this stage are counted on the leader's barrier, which the MMA thread waits on
+                            if (leader) mbar_expect_tx(full_bar(s), 2 * C::STAGE_BYTES);
+                            const uint32_t fb = mapa_shared(full_bar(s), 0);
+                            tma_load_3d_pair(sa, &tm_t, kb * BK, t.m0, tz, fb, keep);
+                            // this CTA's half of the tile's weight rows (GATEUP: the leader holds the gate rows, its partner the up rows)
+                            if (EPI == PRE_GATEUP) tma_load_3d_pair(sb, leader ? &tm_w0 : &tm_w1, kb * BK, t.row0, wz, fb, keep);
+                            else tma_load_3d_pair(sb, tm_w, kb * BK, t.row0 + crank * (BN / 2), wz, fb, keep);
                         } else {
-                            tma_load_3d(sb, tm_w, kb * BK, t.row0, wz, full_bar(s));
+                            mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
+                            tma_load_3d(sa, &tm_t, kb * BK, t.m0, tz, full_bar(s));
+                            if (EPI == PRE_GATEUP) {
+                                tma_load_3d(sb, &tm_w0, kb * BK, t.row0, wz, full_bar(s));
+                                tma_load_3d(sb + 128 * BK * 2, &tm_w1, kb * BK, t.row0, wz, full_bar(s));
+                            } else {
+                                tma_load_3d(sb, tm_w, kb * BK, t.row0, wz, full_bar(s));
+                            }
                         }
                     }
                 }
             }
+            // A pair member must not leave while the leader's last commits are still on their way to its barriers:
+            // wait (bounded) until every stage it filled has been released.
+            if (PAIR)
+                for (uint32_t j = it; j < it + S && ok; ++j)
+                    if (j >= (uint32_t)S && !mbar_wait(empty_bar(j % S), ((j / S) & 1) ^ 1, g.err, abort_flag)) ok = false;
         }
         __syncwarp();
     } else if (warp == 5) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(BN);
+        if (lane == 0 && leader) {
+            constexpr uint32_t idesc = make_idesc(BN, PAIR ? 2 * BM : BM);
             uint32_t it = 0, pc = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            for (int tile = tile0; tile < total_tiles && ok; tile += tile_step) {
                 for (int pass = 0; pass < L.passes && ok; ++pass, ++pc) {
                     const int buf = pc & 1;
                     if (!mbar_wait(tempty_bar(buf), ((pc >> 1) & 1) ^ 1, g.err, abort_flag)) { ok = false; break; }
@@ -496,12 +526,20 @@ __global__ void __launch_bounds__(PCfg<EPI>::THREADS_, 1) gemm_prefill_kernel(co
                         const uint32_t sa = base + s * C::STAGE_BYTES, sb = sa + C::A_BYTES;
                         const uint64_t da = make_desc(sa), db = make_desc(sb);
 #pragma unroll
-                        for (int k = 0; k < BK / UMMA_K; ++k)
-                            umma(tacc, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
-                                 (kb > 0 || k > 0) ? 1u : 0u);
-                        umma_commit(empty_bar(s));
+                        for (int k = 0; k < BK / UMMA_K; ++k) {
+                            if (PAIR) umma_pair(tacc, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
+                                                (kb > 0 || k > 0) ? 1u : 0u);
+                            else umma(tacc, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
+                                      (kb > 0 || k > 0) ? 1u : 0u);
+                        }
+                        // the stage is free in both CTAs once these MMAs have read it
+                        if (PAIR) umma_commit_pair(empty_bar(s));
+                        else umma_commit(empty_bar(s));
                     }
-                    if (ok) umma_commit(tfull_bar(buf));
+                    if (ok) {
+                        if (PAIR) umma_commit_pair(tfull_bar(buf));
+                        else umma_commit(tfull_bar(buf));
+                    }
                 }
             }
         }
@@ -513,8 +551,9 @@ __global__ void __launch_bounds__(PCfg<EPI>::THREADS_, 1) gemm_prefill_kernel(co
         // columns it finishes when two warps share a quarter
         const int quarter = warp & 3, half = warp >= 6 ? 1 : 0;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_cnt) {
-            const PreTile t = decode_tile(L, EPI, tile);
+        const uint32_t tempty_leader0 = PAIR ? mapa_shared(tempty_bar(0), 0) : 0, tempty_leader1 = PAIR ? mapa_shared(tempty_bar(1), 0) : 0;
+        for (int tile = tile0; tile < total_tiles && ok; tile += tile_step, ++tile_cnt) {
+            const PreTile t = decode_tile(L, EPI, tile, PAIR, crank);
             const int m = t.m0 + quarter * 32 + lane;
             const bool valid = m < g.t_rows;
             if (EPI == PRE_OPROJ_SPD && !g.norm_only)
@@ -551,40 +590,48 @@ __global__ void __launch_bounds__(PCfg<EPI>::THREADS_, 1) gemm_prefill_kernel(co
                 }
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 __syncwarp();
-                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(tempty_bar(buf)) : "memory");
+                if (lane == 0) {
+                    if (PAIR) mbar_arrive_cluster(buf ? tempty_leader1 : tempty_leader0); // the leader's MMA thread waits for both CTAs' warps
+                    else asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(tempty_bar(buf)) : "memory");
+                }
                 if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_PREFILL + EPI, TR_END);
             }
         }
         if (EPI == PRE_OPROJ_SPD && threadIdx.x == 0) tma_store_wait_all(); // results in memory before the block ends
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
+    // a pair ends together: neither CTA's shared or tensor memory may go while the partner's MMAs or arrivals can reach it
+    if (PAIR) cluster_sync();
+    else __syncthreads();
     if (threadIdx.x == 0) stamp_exit(g.stamp);
     if (warp == 5) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_ALL) : "memory");
+        if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_ALL) : "memory");
+        else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_ALL) : "memory");
     }
 }
 
-template <int EPI>
+template <int EPI, int PAIR>
 cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, const PreLaunch &L, cudaStream_t st)
 {
     const bool spd = EPI == PRE_OPROJ_SPD;
     const CUtensorMap &tx = tt, &tr = tt; // spare tensor-map slots
     const CUtensorMap &th = *(const CUtensorMap *)((spd && !L.g.norm_only) ? L.g.h_map : (const void *)&tt);
-    using C = PCfg<EPI>;
-    static int n_sm = 0;
-    if (!n_sm) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_prefill_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+    using C = PCfg<EPI, PAIR>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_prefill_kernel<EPI, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
         if (e != cudaSuccess) return e;
-        int dev = 0, n = 0;
-        if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-        if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-        n_sm = n;
+        attr_done = true;
     }
+    const int n_sm = sm_count();
     const int total = L.m_tiles * L.n_tiles;
+    if (PAIR) { // one pair per two SMs, persistent over the 256-token tiles
+        const int pairs = total < n_sm / 2 ? total : n_sm / 2;
+        return launch_kernel(gemm_prefill_kernel<EPI, PAIR>, dim3(2 * pairs), dim3(C::THREADS_), C::SMEM_BYTES, st, 2, *tw[0], *tw[1], *tw[2], tt, tx, tr, th, L);
+    }
     const dim3 grid(total < n_sm ? total : n_sm);
-    return launch_kernel(gemm_prefill_kernel<EPI>, grid, dim3(C::THREADS_), C::SMEM_BYTES, st, 0, *tw[0], *tw[1], *tw[2], tt, tx, tr, th, L);
+    return launch_kernel(gemm_prefill_kernel<EPI, PAIR>, grid, dim3(C::THREADS_), C::SMEM_BYTES, st, 0, *tw[0], *tw[1], *tw[2], tt, tx, tr, th, L);
 }
 
 // One thread block per token: whole-row sum of squares in one partial.
@@ -640,7 +687,9 @@ cudaError_t launch_gemm_prefill(PreEpilogue epi, const TcMap *const *weights, co
     for (int i = 0; i < 3; ++i) tw[i] = (const CUtensorMap *)weights[i < nw ? i : 0];
     PreLaunch L;
     L.g = g;
-    L.m_tiles = (g.t_rows + BM - 1) / BM;
+    const bool pair = g.pair != 0;
+    if (pair && g.norm_only) return cudaErrorInvalidValue;
+    L.m_tiles = pair ? (g.t_rows + 2 * BM - 1) / (2 * BM) : (g.t_rows + BM - 1) / BM;
     L.passes = 1;
     L.f_tiles = 1;
     for (int i = 0; i < 3; ++i) L.tile_start[i] = 1 << 30;
@@ -653,19 +702,19 @@ cudaError_t launch_gemm_prefill(PreEpilogue epi, const TcMap *const *weights, co
             tiles += (g.w_rows[i] + 255) / 256;
         }
         L.n_tiles = tiles;
-        return launch_epi<PRE_QKV>(tw, *(const CUtensorMap *)&tokens, L, st);
+        return pair ? launch_epi<PRE_QKV, 1>(tw, *(const CUtensorMap *)&tokens, L, st) : launch_epi<PRE_QKV, 0>(tw, *(const CUtensorMap *)&tokens, L, st);
     }
     case PRE_GATEUP:
         L.f_tiles = (g.Fs + 127) / 128;
         L.n_tiles = L.f_tiles * g.batches;
-        return launch_epi<PRE_GATEUP>(tw, *(const CUtensorMap *)&tokens, L, st);
+        return pair ? launch_epi<PRE_GATEUP, 1>(tw, *(const CUtensorMap *)&tokens, L, st) : launch_epi<PRE_GATEUP, 0>(tw, *(const CUtensorMap *)&tokens, L, st);
     case PRE_OPROJ_SPD:
         L.n_tiles = (g.H + 127) / 128;
         L.passes = g.batches;
-        return launch_epi<PRE_OPROJ_SPD>(tw, *(const CUtensorMap *)&tokens, L, st);
+        return pair ? launch_epi<PRE_OPROJ_SPD, 1>(tw, *(const CUtensorMap *)&tokens, L, st) : launch_epi<PRE_OPROJ_SPD, 0>(tw, *(const CUtensorMap *)&tokens, L, st);
     default:
         L.n_tiles = (g.H + 255) / 256;
-        return launch_epi<PRE_RESID>(tw, *(const CUtensorMap *)&tokens, L, st);
+        return pair ? launch_epi<PRE_RESID, 1>(tw, *(const CUtensorMap *)&tokens, L, st) : launch_epi<PRE_RESID, 0>(tw, *(const CUtensorMap *)&tokens, L, st);
     }
 }
 

@@ -54,10 +54,14 @@ struct PreGemmArgs {
     // K slice and token, the sum of squares of the slice's output to ss_out (no residual, no operand planes).
     int w_rot;
     int norm_only;
+    // CTA pairs: two CTAs of a cluster share one tile of 256 tokens (one M = 256 MMA over both), each loading half
+    // of the tile's weight rows.  The weight maps must then have boxes of HALF the tile's rows: 128 (QKV, RESID,
+    // GATEUP: gate rows in one CTA, up rows in the other), 64 (OPROJ_SPD).  Not with norm_only.
+    int pair;
 };
 
 // Weight maps: 256-row boxes (QKV, RESID), 128-row boxes (GATEUP: gate and up; OPROJ_SPD: the
-// shard-sliced W_O).  Token map: 128-row box.
+// shard-sliced W_O); with g.pair, boxes of half as many rows (see PreGemmArgs::pair).  Token map: 128-row box.
 cudaError_t launch_gemm_prefill(PreEpilogue epi, const TcMap *const *weights, const TcMap &tokens, const PreGemmArgs &g,
                                 cudaStream_t st);
 

@@ -66,7 +66,7 @@ enum Site { SITE_QKV = 0, SITE_O, SITE_GU, SITE_DOWN, SITE_ATTN, SITE_COUNT };
 const char *const kind_names[K_COUNT] = {"residual_rmsnorm", "gemm_qkv", "rope_kv_append", "attention", "gemm_o_proj",
                                          "gemm_gate_up", "silu_mul", "gemm_down", "rope_table"};
 
-struct LayerMaps { TcMap wq, wk, wv, wo_full, wo_shard, w_gate, w_up, w_down, w_gate64, w_up64, wq256, wk256, wv256, wo256, wd256, wd_shard, kpages, vpages; };
+struct LayerMaps { TcMap wq, wk, wv, wo_full, wo_shard, wo_shard64, w_gate, w_up, w_down, w_gate64, w_up64, wq256, wk256, wv256, wo256, wd256, wd_shard, kpages, vpages; };
 
 // A captured decode step is valid for exactly these arguments.
 struct GraphKey {
@@ -127,6 +127,7 @@ struct Ctx {
     int ring_stages;             // decode GEMMs: stages of the operand ring (0 = per launch)
     int prefill_rescale_log2;    // tcgen05 prefill attention: growth of the row maximum (log2) that triggers a rescale
     int peer_wait_ms;            // rank mode: how long a rank waits for its peers' partial sums
+    int prefill_pairs;           // prompt projections: CTA pairs (256-token tiles) where a launch has more than 128 tokens
     int launches_last;
     TpState tp;
     // activation tensor maps, by buffer and token box (16, 32, 64, 128), built on first use
@@ -869,9 +870,11 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
         LAUNCH_S(K_NORM, a, launch_prefill_prologue(a, st));
     }
     int attn_tiles = 1; // partial sums of squares per token in ss_attn
+    // more than one 128-token tile: CTA pairs, 256 tokens per tile, weight maps with boxes of half a tile's rows
+    const int pair = (M > 128 && c->prefill_pairs) ? 1 : 0;
     auto base_args = [&]() {
         PreGemmArgs g{};
-        g.t_rows = M; g.err = c->err; g.H = H; g.Mcap = Mc; g.batches = 1; g.n_weights = 1;
+        g.t_rows = M; g.err = c->err; g.H = H; g.Mcap = Mc; g.batches = 1; g.n_weights = 1; g.pair = pair;
         return g;
     };
     for (int l = 0; l < d.n_layers; ++l) {
@@ -881,7 +884,8 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
         const bool sync = probe ? !probing : c->mask[l] != 0;
         {   // a2 + a3
             PreGemmArgs g = base_args();
-            const TcMap *wmaps[3] = {&c->maps[l].wq256, &c->maps[l].wk256, &c->maps[l].wv256};
+            const LayerMaps &lm = c->maps[l];
+            const TcMap *wmaps[3] = {pair ? &lm.wq : &lm.wq256, pair ? &lm.wk : &lm.wk256, pair ? &lm.wv : &lm.wv256};
             MAP_OR_FAIL(am, act_map(c, AB_H, 128));
             g.n_weights = 3; g.w_rows[0] = qd; g.w_rows[1] = g.w_rows[2] = kd;
             g.num_kb = cdiv(H, 64);
@@ -909,7 +913,7 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
         int mlp_tiles, mlp_groups;
         if (sync) {   // a5 - a7, sync block: sum_i Y_i is the K accumulation over all heads
             PreGemmArgs g = base_args();
-            const TcMap *wmaps[1] = {&c->maps[l].wo256};
+            const TcMap *wmaps[1] = {pair ? &c->maps[l].wo_full : &c->maps[l].wo256};
             MAP_OR_FAIL(am, act_map(c, AB_ATTN, 128));
             g.w_rows[0] = H; g.num_kb = cdiv(qd, 64);
             g.res_in = c->res[0]; g.res_out = c->res[1]; g.gain = w.mlp_norm; g.hg = c->h; g.hg_stride = Mc * H; g.ss_out = c->ss_mlp;
@@ -917,7 +921,7 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
             mlp_tiles = pre_ss_tiles(PRE_RESID, H); mlp_groups = 1;
         } else {      // a5 - a7, SPD block: device i's K slice gives Y_i, kept apart
             PreGemmArgs g = base_args();
-            const TcMap *wmaps[1] = {&c->maps[l].wo_shard};
+            const TcMap *wmaps[1] = {pair ? &c->maps[l].wo_shard64 : &c->maps[l].wo_shard};
             MAP_OR_FAIL(am, act_map(c, AB_ATTN_SHARD, 128));
             g.w_rows[0] = H; g.num_kb = cdiv(qd / Tn, 64); g.batches = Tn;
             g.res_in = c->res[0]; g.res_out = c->res[1]; g.gain = w.mlp_norm; g.hg = c->h; g.hg_stride = Mc * H; g.ss_out = c->ss_mlp;
@@ -938,7 +942,7 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
                     PreGemmArgs g = base_args();
                     const TcMap *wmaps[2] = {&c->maps[l].w_gate, &c->maps[l].w_up};
                     MAP_OR_FAIL(am, act_map(c, AB_H, 128));
-                    g.n_weights = 2; g.w_rows[0] = g.w_rows[1] = Fs; g.batches = Tn; g.t_batched = 1; g.w_rot = r;
+                    g.n_weights = 2; g.w_rows[0] = g.w_rows[1] = Fs; g.batches = Tn; g.t_batched = 1; g.w_rot = r; g.pair = 0;
                     g.num_kb = cdiv(H, 64);
                     g.ss_in = SumSq{c->ss_mlp, mlp_tiles, mlp_groups, Mc, H, d.rms_eps};
                     g.rstd_per_shard = 1;
@@ -949,7 +953,7 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
                     PreGemmArgs g = base_args();
                     const TcMap *wmaps[1] = {&c->maps[l].wd_shard};
                     MAP_OR_FAIL(am, act_map(c, AB_ACT_SHARD, 128));
-                    g.w_rows[0] = H; g.num_kb = cdiv(Fs, 64); g.batches = Tn; g.norm_only = 1; g.ss_out = ssq;
+                    g.w_rows[0] = H; g.num_kb = cdiv(Fs, 64); g.batches = Tn; g.norm_only = 1; g.ss_out = ssq; g.pair = 0;
                     LAUNCH(K_DOWN, launch_gemm_prefill(PRE_OPROJ_SPD, wmaps, *am, g, st));
                 }
                 CU_TRY(cudaMemcpy2DAsync(host.data(), (size_t)M * 4, ssq, (size_t)Mc * 4, (size_t)M * 4, (size_t)nt * Tn,
@@ -979,7 +983,7 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
         }
         {   // a9 + a10: res[1] holds X + sum_i Y_i in both modes, so out = res[1] + sum_i Z_i
             PreGemmArgs g = base_args();
-            const TcMap *wmaps[1] = {&c->maps[l].wd256};
+            const TcMap *wmaps[1] = {pair ? &c->maps[l].w_down : &c->maps[l].wd256};
             MAP_OR_FAIL(am, act_map(c, AB_ACT, 128));
             g.w_rows[0] = H; g.num_kb = cdiv(F, 64);
             g.res_in = c->res[1]; g.res_out = c->res[0];
@@ -1019,6 +1023,7 @@ int build_weight_maps(Ctx &c)
         rc |= make_operand_map(&m.wv, w.wv, H, kd, 1, H, 0, 128);
         rc |= make_operand_map(&m.wo_full, w.wo, qd, H, 1, qd, 0, 128);
         rc |= make_operand_map(&m.wo_shard, w.wo, qd / T, H, T, qd, qd / T, 128);
+        rc |= make_operand_map(&m.wo_shard64, w.wo, qd / T, H, T, qd, qd / T, 64);
         rc |= make_operand_map(&m.w_gate, w.w_gate, H, F / T, T, H, (F / T) * H, 128);
         if (d.block_kind == 0) rc |= make_operand_map(&m.w_up, w.w_up, H, F / T, T, H, (F / T) * H, 128);
         rc |= make_operand_map(&m.w_down, w.w_down, F, H, 1, F, 0, 128);
@@ -1194,6 +1199,7 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     c.l2_prefetch_kb = 0;
     c.prefill_rescale_log2 = 8;
     c.peer_wait_ms = 1000;
+    c.prefill_pairs = 1;
     c.ring_stages = 0;
     c.launches_last = 0;
     c.tp.on = false;
@@ -1400,6 +1406,7 @@ int spd_set_tuning(spd_ctx *ctx, const char *key, int32_t value)
     if (!strcmp(key, "decode_ring_stages")) { c.ring_stages = (value == 0 || (value >= 3 && value <= 5)) ? value : 0; found = true; }
     if (!strcmp(key, "prefill_rescale_log2")) { c.prefill_rescale_log2 = value > 16 ? 16 : value; found = true; }
     if (!strcmp(key, "l2_prefetch_blocks")) { c.l2_prefetch_kb = value > 64 ? 64 : value; found = true; }
+    if (!strcmp(key, "prefill_pairs")) { c.prefill_pairs = value != 0; found = true; }
     if (!strcmp(key, "peer_wait_ms")) { c.peer_wait_ms = value < 1 ? 1000 : (value > 60000 ? 60000 : value); found = true; }
     if (!found) return SPD_EINVAL;
     for (GraphEntry &g : c.graphs) cudaGraphExecDestroy(g.exec); // captured steps used the old setting

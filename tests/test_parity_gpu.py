@@ -253,3 +253,24 @@ def test_decode_ring_depth_is_only_a_schedule(stages):
         outs.append((got, got2))
         p.stack.close()
     assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+
+
+@pytest.mark.parametrize("mask", [(1, 1), (0, 0), (0, 1)])
+def test_prefill_on_cta_pairs_equals_prefill_on_single_blocks(mask):
+    """Launches with more than 128 tokens run their projections on pairs of thread blocks (256-token tiles, one
+    tensor-core instruction over two SMs, each block loading half of the tile's weight rows).  Same K order, same
+    accumulators: the output is bit-identical to the one-block-per-tile schedule, and both match the oracle.
+    520 tokens = two full 256-token tiles and a third whose second block has only 8 valid rows; FFN / T = 344."""
+    w = si.Workload("pairs", "bf16", 2, 512, 8, 4, 64, 1376, 4, mask, 2, 260, 1)
+    outs = []
+    for pairs in (1, 0):
+        p = Pair(w, mask=mask, B=2, max_len=264, max_prefill_tokens=1024)
+        p.stack.set_tuning(prefill_pairs=pairs)
+        got, ref, _ = p.prefill(260)
+        assert rel_err(got, ref) <= TOL["bf16"]
+        got_d, ref_d = p.decode(0)
+        assert rel_err(got_d, ref_d) <= TOL["bf16"]
+        assert p.stack.device_error() == 0
+        outs.append((got, got_d))
+        p.stack.close()
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
