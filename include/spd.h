@@ -168,6 +168,11 @@ int spd_set_graphs(spd_ctx *ctx, int32_t enabled);
  *       prompt projections on pairs of thread blocks (one 256-token tile and one tensor-core instruction over
  *       two SMs, each block loading half of the tile's weight rows): 1 (default) wherever a launch has more
  *       than 128 tokens, 0 = always one block per 128-token tile.  Same results bit for bit.
+ *   "prefill_group_m"
+ *       tile order of the prompt projections: token tiles are taken in groups of this many, and inside a group
+ *       the token tile runs fastest, then the weight tile, so that a group's token panels stay in L2 while the
+ *       weight tiles sweep past (0 = default: 2048 tokens per group; a value >= the number of token tiles gives
+ *       the plain order with all token tiles fastest).  A schedule only: same results.
  *   "peer_wait_ms"
  *       rank mode (spd_tp_*): milliseconds a rank waits for the other ranks' partial sums before
  *       it gives up with error bit 8 (default and value 0: 1000; at most 60000).  Always bounded.

@@ -14,6 +14,10 @@
 //                   device i's pass gives Y_i, from which R_i = X + Y_i (its own MLP input) is
 //                   stored, while a third tensor-memory buffer adds up sum_i Y_i for the
 //                   residual that is carried to the block output.
+// Launches with more than 128 tokens run on pairs of thread blocks (cta_group::2): one 256-token tile
+// and one M = 256 instruction over two SMs, each block loading its own token rows and half of the
+// tile's weight rows.  The operand ring takes all of a block's shared memory: tile loads have a
+// loaded latency of about 1.6 us, so bytes in flight are what bounds the feed of the tensor cores.
 #include "gemm_prefill.cuh"
 #include "tc_ptx.cuh"
 #include "trace.cuh"
@@ -24,10 +28,8 @@ namespace {
 
 using namespace tc;
 
-constexpr int THREADS = 192;
 constexpr int TMEM_ALL = 512;
-constexpr int TOT_COL = 256; // PRE_OPROJ_SPD: X + running sum of the Y_i
-constexpr int X_COL = 384;   // PRE_OPROJ_SPD: the X tile
+constexpr int X_COL = 256;   // PRE_OPROJ_SPD: the X tile (columns 0-255 hold the two accumulators)
 
 // PAIR: two CTAs of a cluster work on one tile of 256 tokens as one M = 256 MMA (cta_group::2): each loads its own
 // 128 token rows and HALF of the tile's weight rows, so per MMA flop only two thirds (three quarters for the SPD
@@ -36,9 +38,10 @@ template <int EPI, int PAIR> struct PCfg {
     static constexpr int BN = (EPI == PRE_OPROJ_SPD) ? 128 : 256;
     static constexpr int A_BYTES = BM * BK * 2, B_BYTES = (BN / (PAIR ? 2 : 1)) * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    // PRE_OPROJ_SPD stages outgoing R_i * g tiles (bf16, 32 KB each) in shared memory
-    static constexpr int X_BYTES = 0, H_BYTES = (EPI == PRE_OPROJ_SPD) ? 2 * 128 * 128 * 2 : 0; // two staging tiles
-    static constexpr int STAGES = (192 * 1024 - X_BYTES - H_BYTES) / STAGE_BYTES;
+    static constexpr int X_BYTES = 0, H_BYTES = 0;
+    // the ring takes all the shared memory a block may have: the loaded latency of a tile load is about 1.6 us, so
+    // what the tensor cores can be fed per SM is (bytes in flight) / 1.6 us
+    static constexpr int STAGES = (216 * 1024 - X_BYTES - H_BYTES) / STAGE_BYTES;
     static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
     static constexpr int SMEM_BYTES = RING_BYTES + X_BYTES + H_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
     // Epilogue warps: 0-3 (one per accumulator lane quarter); PRE_OPROJ_SPD, whose tail is T times the work per MMA
@@ -50,6 +53,7 @@ template <int EPI, int PAIR> struct PCfg {
 struct PreLaunch {
     PreGemmArgs g;
     int m_tiles, n_tiles, passes; // m_tiles: token tiles of 128 rows, or of 256 for a CTA pair
+    int group_m;                  // token tiles per group of the tile order (see decode_tile)
     int tile_start[3]; // QKV: first n-tile of weight i
     int f_tiles;       // GATEUP: n-tiles per device
 };
@@ -65,7 +69,14 @@ struct PreTile {
 __device__ __forceinline__ PreTile decode_tile(const PreLaunch &L, int EPI, int tile, int pair, int crank)
 {
     PreTile t;
-    const int mt = tile % L.m_tiles, nt = tile / L.m_tiles;
+    // Tile order: groups of group_m token tiles; inside a group the token tile runs fastest, then the weight tile.
+    // The blocks at work at any time then cover about group_m token tiles x (blocks / group_m) weight tiles - a
+    // near-square patch, whose operand panels are fetched from HBM once and shared through L2 - and a group's
+    // token panels stay in L2 for the whole sweep over the weight tiles, instead of being streamed again for
+    // every few weight tiles as they are when ALL token tiles run fastest (they do not fit L2 at thousands of tokens).
+    const int per_group = L.group_m * L.n_tiles, grp = tile / per_group, r = tile % per_group;
+    const int gm = min(L.group_m, L.m_tiles - grp * L.group_m);
+    const int mt = grp * L.group_m + r % gm, nt = r / gm;
     t.m0 = pair ? mt * 2 * BM + crank * BM : mt * BM; // this CTA's 128 token rows
     t.nt = nt;
     t.wi = 0;
@@ -111,47 +122,19 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float *v)
                  : "memory");
 }
 
-// three 16-column chunks of this thread's row, one wait
-__device__ __forceinline__ void tmem_ld16x3(uint32_t ta, uint32_t tb, uint32_t tc3, float *va, float *vb, float *vc)
+// two 32-column chunks of this thread's row, one wait
+__device__ __forceinline__ void tmem_ld32x2(uint32_t ta, uint32_t tb, float *va, float *vb)
 {
-    uint32_t r[48];
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%48];\n\t"
-                 "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%49];\n\t"
-                 "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47}, [%50];\n\t"
+    uint32_t r[64];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%64];\n\t"
+                 "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%65];\n\t"
                  "tcgen05.wait::ld.sync.aligned;"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]),
-                   "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]),
-                   "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47])
-                 : "r"(ta), "r"(tb), "r"(tc3)
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+                 : "r"(ta), "r"(tb)
                  : "memory");
 #pragma unroll
-    for (int i = 0; i < 16; ++i) { va[i] = __uint_as_float(r[i]); vb[i] = __uint_as_float(r[16 + i]); vc[i] = __uint_as_float(r[32 + i]); }
+    for (int i = 0; i < 32; ++i) { va[i] = __uint_as_float(r[i]); vb[i] = __uint_as_float(r[32 + i]); }
 }
-
-// three 32-column chunks of this thread's row, one wait
-__device__ __forceinline__ void tmem_ld32x3(uint32_t ta, uint32_t tb, uint32_t tc3, float *va, float *vb, float *vc)
-{
-    uint32_t r[96];
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%96];\n\t"
-                 "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%97];\n\t"
-                 "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%64,%65,%66,%67,%68,%69,%70,%71,%72,%73,%74,%75,%76,%77,%78,%79,%80,%81,%82,%83,%84,%85,%86,%87,%88,%89,%90,%91,%92,%93,%94,%95}, [%98];\n\t"
-                 "tcgen05.wait::ld.sync.aligned;"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63]), "=r"(r[64]), "=r"(r[65]), "=r"(r[66]), "=r"(r[67]), "=r"(r[68]), "=r"(r[69]), "=r"(r[70]), "=r"(r[71]), "=r"(r[72]), "=r"(r[73]), "=r"(r[74]), "=r"(r[75]), "=r"(r[76]), "=r"(r[77]), "=r"(r[78]), "=r"(r[79]), "=r"(r[80]), "=r"(r[81]), "=r"(r[82]), "=r"(r[83]), "=r"(r[84]), "=r"(r[85]), "=r"(r[86]), "=r"(r[87]), "=r"(r[88]), "=r"(r[89]), "=r"(r[90]), "=r"(r[91]), "=r"(r[92]), "=r"(r[93]), "=r"(r[94]), "=r"(r[95])
-                 : "r"(ta), "r"(tb), "r"(tc3)
-                 : "memory");
-#pragma unroll
-    for (int i = 0; i < 32; ++i) { va[i] = __uint_as_float(r[i]); vb[i] = __uint_as_float(r[32 + i]); vc[i] = __uint_as_float(r[64 + i]); }
-}
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float *v)
-{
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
-                 :: "r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])), "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])), "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
-                 : "memory");
-}
-
 // 8 consecutive bf16 (16 bytes) from 8 floats
 __device__ __forceinline__ uint4 pack8(const float *v)
 {
@@ -320,23 +303,25 @@ __device__ __forceinline__ void epi_resid(const PreGemmArgs &g, const PreTile &t
 
 template <int N_THREADS> __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(N_THREADS) : "memory"); }
 
-// SPD o_proj: the X tile of an output tile is parked in tensor memory twice - once as is (every
-// device's R_i = X + Y_i needs it) and once as the start of X + sum_i Y_i - by the thread that owns
-// the row, while the MMA warp works on the first K slice.
-__device__ __forceinline__ void spd_park_x(const PreGemmArgs &g, const PreTile &t, uint32_t tx, uint32_t ttot, int m, bool valid, int half)
+// SPD o_proj: the X tile of an output tile is parked in tensor memory (every device's R_i = X + Y_i needs it) by
+// the thread that owns the row, while the MMA warp works on the first K slice; the same thread starts its running
+// X + sum_i Y_i - 64 columns, kept in registers across the passes - from it.  (Tensor memory serves the MMAs'
+// accumulator traffic and the epilogue's loads and stores alike: with a K slice of only a few hundred per pass the
+// epilogue's share decides the MMA rate, so the running sum stays out of it.)
+__device__ __forceinline__ void spd_park_x(const PreGemmArgs &g, const PreTile &t, uint32_t tx, int m, bool valid, int half, float (&tot)[64])
 {
-#pragma unroll 1
-    for (int c = half * 4; c < half * 4 + 4; ++c) {
-        const int n = t.row0 + c * 16;
-        if (n >= g.H) break;
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc) {
+        const int c = half * 4 + cc, n = t.row0 + c * 16;
         float x[16];
-        if (valid) load_x16(g.res_in + (long)m * g.H + n, x);
+        if (valid && n < g.H) load_x16(g.res_in + (long)m * g.H + n, x);
         else {
 #pragma unroll
             for (int i = 0; i < 16; ++i) x[i] = 0.f;
         }
         tmem_st16(tx + c * 16, x);
-        tmem_st16(ttot + c * 16, x);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) tot[cc * 16 + i] = x[i];
     }
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
@@ -360,47 +345,45 @@ __device__ __forceinline__ float epi_row_sumsq(const PreGemmArgs &g, const PreTi
     return ssq;
 }
 
-// One pass (device z) of an SPD o_proj tile.  R_z * g is staged in hs (two 64-column bf16 boxes of
-// 128 rows, 128-byte swizzle: thread = row, eight consecutive rows hit eight different 16-byte
-// columns) and leaves through a TMA store; X + sum_i Y_i is written by the last pass.
-__device__ __forceinline__ float epi_oproj_spd(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, uint32_t tx, uint32_t ttot, int z,
-                                               int m, bool valid, uint8_t *hs, int r, int half)
+// One pass (device z) of an SPD o_proj tile: R_z * g goes straight from the thread's registers to device z's
+// plane (32-byte stores, whole sectors; shared memory is left to the operand ring); X + sum_i Y_i, carried in
+// tot, is written by the last pass.
+__device__ __forceinline__ float epi_oproj_spd(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, uint32_t tx, int z,
+                                               int m, bool valid, int half, float (&tot)[64])
 {
-    const int T = g.batches, sw = r & 7; // r: row of the tile
+    const int T = g.batches;
     float ssq = 0.f;
-#pragma unroll 1
-    for (int c = half * 2; c < half * 2 + 2; ++c) { // 32 columns per round: few tensor-memory round trips on the critical path
-        const int n = t.row0 + c * 32;
-        if (n >= g.H) break;
-        float y[32], x[32], tot[32];
-        tmem_ld32x3(tacc + c * 32, tx + c * 32, ttot + c * 32, y, x, tot);
+    bf16 *plane = (bf16 *)g.hg + (long)z * g.hg_stride + (long)m * g.H;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) tot[i] += y[i];
-        if (z + 1 < T) tmem_st32(ttot + c * 32, tot);
+    for (int cc = 0; cc < 2; ++cc) { // 32 columns per round: few tensor-memory round trips on the critical path
+        const int c = half * 2 + cc, n = t.row0 + c * 32;
+        float y[32], x[32];
+        tmem_ld32x2(tacc + c * 32, tx + c * 32, y, x);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) tot[cc * 32 + i] += y[i];
         // device z only ever sees its own partial attention output: R_z = X + Y_z
-        uint8_t *hrow = hs + (c >> 1) * 16384 + r * 128;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            float gn[8];
-            const bool in_h = n + 8 * q < g.H; // a tile may reach past the last column
-            unpack8(in_h ? *(const uint4 *)((const bf16 *)g.gain + n + 8 * q) : make_uint4(0, 0, 0, 0), gn);
+        for (int q = 0; q < 2; ++q) {
+            if (!valid || n + 16 * q >= g.H) continue; // a tile may reach past the last column (H is a multiple of 16)
+            float gn[16];
+            unpack8(*(const uint4 *)((const bf16 *)g.gain + n + 16 * q), gn);
+            unpack8(*(const uint4 *)((const bf16 *)g.gain + n + 16 * q + 8), gn + 8);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const float ri = in_h ? x[8 * q + i] + y[8 * q + i] : 0.f;
+            for (int i = 0; i < 16; ++i) {
+                const float ri = x[16 * q + i] + y[16 * q + i];
                 ssq = fmaf(ri, ri, ssq);
                 gn[i] *= ri;
             }
-            *(uint4 *)(hrow + ((((c & 1) * 4 + q) ^ sw) << 4)) = pack8(gn);
+            stg16_bf16(plane + n + 16 * q, gn);
         }
         if (z + 1 == T && valid) {
             // the residual carried to the block output has collected every Y_i
             float *dst = g.res_out + (long)m * g.H + n;
 #pragma unroll
             for (int k = 0; k < 4; ++k)
-                if (n + 8 * k < g.H) stg8(dst + 8 * k, tot + 8 * k);
+                if (n + 8 * k < g.H) stg8(dst + 8 * k, &tot[cc * 32 + 8 * k]);
         }
     }
-    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     return ssq;
 }
 
@@ -424,7 +407,6 @@ __global__ void __launch_bounds__(PCfg<EPI, PAIR>::THREADS_, 1) gemm_prefill_ker
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
-    uint8_t *hs = gen_base + C::RING_BYTES; // PRE_OPROJ_SPD staging (1024-byte aligned)
     const uint32_t bars = base + C::RING_BYTES + C::X_BYTES + C::H_BYTES; // full[S], empty[S], tmem_full[2], tmem_empty[2], x_full
     uint32_t *tmem_slot = (uint32_t *)(gen_base + C::RING_BYTES + C::X_BYTES + C::H_BYTES + 8 * (2 * S + 5));
     const uint32_t xfull_bar = bars + 8u * (2 * S + 4);
@@ -516,12 +498,16 @@ __global__ void __launch_bounds__(PCfg<EPI, PAIR>::THREADS_, 1) gemm_prefill_ker
             for (int tile = tile0; tile < total_tiles && ok; tile += tile_step) {
                 for (int pass = 0; pass < L.passes && ok; ++pass, ++pc) {
                     const int buf = pc & 1;
+                    SPD_TRACE_EVENT(TRK_PREFILL + 8 + EPI, TR_START);
                     if (!mbar_wait(tempty_bar(buf), ((pc >> 1) & 1) ^ 1, g.err, abort_flag)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    SPD_TRACE_EVENT(TRK_PREFILL + 8 + EPI, TR_DEP_DONE);
                     const uint32_t tacc = tmem_base + (uint32_t)(buf * BN);
                     for (int kb = 0; kb < g.num_kb; ++kb, ++it) {
                         const int s = it % S;
+                        if (kb == 0 || kb == g.num_kb - 1) SPD_TRACE_EVENT(TRK_PREFILL + 8 + EPI, TR_ARRIVED);
                         if (!mbar_wait(full_bar(s), (it / S) & 1, g.err, abort_flag)) { ok = false; break; }
+                        if (kb == 0 || kb == g.num_kb - 1) SPD_TRACE_EVENT(TRK_PREFILL + 8 + EPI, TR_MAIN_DONE);
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                         const uint32_t sa = base + s * C::STAGE_BYTES, sb = sa + C::A_BYTES;
                         const uint64_t da = make_desc(sa), db = make_desc(sb);
@@ -540,6 +526,7 @@ __global__ void __launch_bounds__(PCfg<EPI, PAIR>::THREADS_, 1) gemm_prefill_ker
                         if (PAIR) umma_commit_pair(tfull_bar(buf));
                         else umma_commit(tfull_bar(buf));
                     }
+                    SPD_TRACE_EVENT(TRK_PREFILL + 8 + EPI, TR_END);
                 }
             }
         }
@@ -547,6 +534,7 @@ __global__ void __launch_bounds__(PCfg<EPI, PAIR>::THREADS_, 1) gemm_prefill_ker
     } else {
         uint32_t pc = 0, tile_cnt = 0;
         bool ok = true;
+        float tot[64]; // PRE_OPROJ_SPD only: this thread's 64 columns of X + sum_i Y_i (optimised away elsewhere)
         // accumulator lane quarter of this warp (a warp reaches lanes 32 * (warp % 4) ..), and which half of the
         // columns it finishes when two warps share a quarter
         const int quarter = warp & 3, half = warp >= 6 ? 1 : 0;
@@ -556,8 +544,7 @@ __global__ void __launch_bounds__(PCfg<EPI, PAIR>::THREADS_, 1) gemm_prefill_ker
             const PreTile t = decode_tile(L, EPI, tile, PAIR, crank);
             const int m = t.m0 + quarter * 32 + lane;
             const bool valid = m < g.t_rows;
-            if (EPI == PRE_OPROJ_SPD && !g.norm_only)
-                spd_park_x(g, t, tmem_base + lane_base + X_COL, tmem_base + lane_base + TOT_COL, m, valid, half);
+            if (EPI == PRE_OPROJ_SPD && !g.norm_only) spd_park_x(g, t, tmem_base + lane_base + X_COL, m, valid, half, tot);
             for (int pass = 0; pass < L.passes; ++pass, ++pc) {
                 const int buf = pc & 1;
                 if (!mbar_wait(tfull_bar(buf), (pc >> 1) & 1, g.err, abort_flag)) { ok = false; break; }
@@ -571,22 +558,10 @@ __global__ void __launch_bounds__(PCfg<EPI, PAIR>::THREADS_, 1) gemm_prefill_ker
                     const float ssq = epi_row_sumsq(g, t, tacc, half);
                     if (valid) g.ss_out[((long)(t.nt * 2 + half) * g.batches + pass) * g.Mcap + m] = ssq;
                 } else {
-                    // two staging tiles in turn: the store issued two passes ago has read its source
-                    uint8_t *hst = hs + (pc & 1) * 32768;
-                    if (threadIdx.x == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                    epi_sync<32 * C::EPI_WARPS>();
                     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_PREFILL + EPI, TR_DEP_DONE);
-                    const float ssq = epi_oproj_spd(g, t, tacc, tmem_base + lane_base + X_COL, tmem_base + lane_base + TOT_COL, pass, m, valid, hst,
-                                                    quarter * 32 + lane, half);
+                    const float ssq = epi_oproj_spd(g, t, tacc, tmem_base + lane_base + X_COL, pass, m, valid, half, tot);
                     if (valid && g.ss_out) g.ss_out[((long)(t.nt * 2 + half) * g.batches + pass) * g.Mcap + m] = ssq;
-                    fence_proxy_async();
                     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_PREFILL + EPI, TR_MAIN_DONE);
-                    epi_sync<32 * C::EPI_WARPS>();
-                    if (threadIdx.x == 0) {
-                        tma_store_3d(&tm_h, smem_u32(hst), t.row0, t.m0, pass);
-                        tma_store_3d(&tm_h, smem_u32(hst) + 16384, t.row0 + 64, t.m0, pass);
-                        tma_store_commit();
-                    }
                 }
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 __syncwarp();
@@ -597,7 +572,6 @@ __global__ void __launch_bounds__(PCfg<EPI, PAIR>::THREADS_, 1) gemm_prefill_ker
                 if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_PREFILL + EPI, TR_END);
             }
         }
-        if (EPI == PRE_OPROJ_SPD && threadIdx.x == 0) tma_store_wait_all(); // results in memory before the block ends
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     // a pair ends together: neither CTA's shared or tensor memory may go while the partner's MMAs or arrivals can reach it
@@ -614,9 +588,8 @@ __global__ void __launch_bounds__(PCfg<EPI, PAIR>::THREADS_, 1) gemm_prefill_ker
 template <int EPI, int PAIR>
 cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, const PreLaunch &L, cudaStream_t st)
 {
-    const bool spd = EPI == PRE_OPROJ_SPD;
     const CUtensorMap &tx = tt, &tr = tt; // spare tensor-map slots
-    const CUtensorMap &th = *(const CUtensorMap *)((spd && !L.g.norm_only) ? L.g.h_map : (const void *)&tt);
+    const CUtensorMap &th = tt;
     using C = PCfg<EPI, PAIR>;
     static bool attr_done = false;
     if (!attr_done) {
@@ -679,7 +652,7 @@ cudaError_t launch_gemm_prefill(PreEpilogue epi, const TcMap *const *weights, co
     if (g.num_kb < 1 || g.batches < 1 || g.batches > 8) return cudaErrorInvalidValue;
     if (epi == PRE_QKV && (256 % g.head_dim || g.head_dim < 32)) return cudaErrorInvalidValue;
     if ((epi == PRE_RESID || epi == PRE_OPROJ_SPD) && g.H % 16) return cudaErrorInvalidValue;
-    if (epi == PRE_OPROJ_SPD && !g.norm_only && (!g.h_map || !g.gain || !g.hg || !g.res_out)) return cudaErrorInvalidValue;
+    if (epi == PRE_OPROJ_SPD && !g.norm_only && (!g.gain || !g.hg || !g.res_out)) return cudaErrorInvalidValue;
     if (epi == PRE_OPROJ_SPD && g.norm_only && !g.ss_out) return cudaErrorInvalidValue;
     if (g.w_rot < 0 || g.w_rot >= g.batches) return cudaErrorInvalidValue;
     if (epi == PRE_GATEUP && g.Fs % 8) return cudaErrorInvalidValue;
@@ -690,6 +663,7 @@ cudaError_t launch_gemm_prefill(PreEpilogue epi, const TcMap *const *weights, co
     const bool pair = g.pair != 0;
     if (pair && g.norm_only) return cudaErrorInvalidValue;
     L.m_tiles = pair ? (g.t_rows + 2 * BM - 1) / (2 * BM) : (g.t_rows + BM - 1) / BM;
+    L.group_m = g.group_m > 0 ? g.group_m : (pair ? 8 : 16);
     L.passes = 1;
     L.f_tiles = 1;
     for (int i = 0; i < 3; ++i) L.tile_start[i] = 1 << 30;

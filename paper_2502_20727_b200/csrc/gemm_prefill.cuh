@@ -58,6 +58,7 @@ struct PreGemmArgs {
     // of the tile's weight rows.  The weight maps must then have boxes of HALF the tile's rows: 128 (QKV, RESID,
     // GATEUP: gate rows in one CTA, up rows in the other), 64 (OPROJ_SPD).  Not with norm_only.
     int pair;
+    int group_m;         // token tiles per group of the tile order; 0 = default (8 pair tiles / 16 single tiles = 2048 tokens)
 };
 
 // Weight maps: 256-row boxes (QKV, RESID), 128-row boxes (GATEUP: gate and up; OPROJ_SPD: the

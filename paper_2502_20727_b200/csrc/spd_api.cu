@@ -127,6 +127,7 @@ struct Ctx {
     int ring_stages;             // decode GEMMs: stages of the operand ring (0 = per launch)
     int prefill_rescale_log2;    // tcgen05 prefill attention: growth of the row maximum (log2) that triggers a rescale
     int peer_wait_ms;            // rank mode: how long a rank waits for its peers' partial sums
+    int prefill_group_m;         // prompt projections: token tiles per group of the tile order (0 = default)
     int prefill_pairs;           // prompt projections: CTA pairs (256-token tiles) where a launch has more than 128 tokens
     int launches_last;
     TpState tp;
@@ -875,6 +876,7 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
     auto base_args = [&]() {
         PreGemmArgs g{};
         g.t_rows = M; g.err = c->err; g.H = H; g.Mcap = Mc; g.batches = 1; g.n_weights = 1; g.pair = pair;
+        g.group_m = c->prefill_group_m;
         return g;
     };
     for (int l = 0; l < d.n_layers; ++l) {
@@ -1200,6 +1202,7 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     c.prefill_rescale_log2 = 8;
     c.peer_wait_ms = 1000;
     c.prefill_pairs = 1;
+    c.prefill_group_m = 0;
     c.ring_stages = 0;
     c.launches_last = 0;
     c.tp.on = false;
@@ -1406,6 +1409,7 @@ int spd_set_tuning(spd_ctx *ctx, const char *key, int32_t value)
     if (!strcmp(key, "decode_ring_stages")) { c.ring_stages = (value == 0 || (value >= 3 && value <= 5)) ? value : 0; found = true; }
     if (!strcmp(key, "prefill_rescale_log2")) { c.prefill_rescale_log2 = value > 16 ? 16 : value; found = true; }
     if (!strcmp(key, "l2_prefetch_blocks")) { c.l2_prefetch_kb = value > 64 ? 64 : value; found = true; }
+    if (!strcmp(key, "prefill_group_m")) { c.prefill_group_m = value > 4096 ? 4096 : value; found = true; }
     if (!strcmp(key, "prefill_pairs")) { c.prefill_pairs = value != 0; found = true; }
     if (!strcmp(key, "peer_wait_ms")) { c.peer_wait_ms = value < 1 ? 1000 : (value > 60000 ? 60000 : value); found = true; }
     if (!found) return SPD_EINVAL;
