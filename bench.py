@@ -295,17 +295,23 @@ class Run:
                 self.step(0)
             torch.cuda.synchronize()
 
-    def decode_ms(self, barrier):
-        """Settling, W warm-up steps, then K timed steps between two events: (ms, host window)."""
+    def decode_ms(self, barrier, base=0, stamped=False):
+        """Settling, W warm-up steps, then K timed steps between two events: (ms, host window).  stamped: the kernels
+        record their start / end and a fold kernel ends every step (see SpdStack.timeline_begin), so that the region
+        that gives the step time also gives every kernel's share of it."""
+        if stamped:
+            self.stack.timeline_begin()
         self.settle(self.args.settle_s)
         for t in range(self.W):
-            self.step(t)
+            self.step(base + t)
         barrier()
+        if stamped:
+            self.stack.timeline_begin()  # clear the totals of the settling and warm-up steps
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         h0 = time.perf_counter()
         e0.record()
         for t in range(self.W, self.W + self.K):
-            self.step(t)
+            self.step(base + t)
         e1.record()
         barrier()
         h1 = time.perf_counter()
@@ -313,21 +319,9 @@ class Run:
             raise RuntimeError("device error flag set during the timed region")
         return e0.elapsed_time(e1), (h0, h1)
 
-    def timeline(self, barrier):
-        """Every launch's own share of a decode step, from the kernels' start / end stamps folded on the device, over K
-        steps replayed back to back exactly as in the timed region (and timed the same way, for comparison)."""
-        base = 2 * (self.W + self.K)
-        self.stack.timeline_begin()
-        for t in range(self.W):
-            self.step(base + t)
-        barrier()
-        self.stack.timeline_begin()  # clear the totals of the warm-up steps
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for t in range(self.W, self.W + self.K):
-            self.step(base + t)
-        e1.record()
-        barrier()
+    def timeline_totals(self):
+        """Every launch's own share of a step (ms), the steps' mean span and the launches per kind, from the stamps of
+        the K steps of the last decode_ms(stamped=True); ends the stamping."""
         per_launch, span_ns, calls = self.stack.timeline_read()
         self.stack.timeline_end()
         if calls != self.K:
@@ -336,8 +330,7 @@ class Run:
         for kind, ns in per_launch:
             own_ms[kind] = own_ms.get(kind, 0.0) + ns / calls * 1e-6
             launches[kind] = launches.get(kind, 0) + 1
-        return own_ms, span_ns / calls * 1e-6, launches, e0.elapsed_time(e1) / self.K
-
+        return own_ms, span_ns / calls * 1e-6, launches
 
 def roofline_entry(w, B, mid_ctx, ms_per_step, hbm_peak, peak_kind):
     wbytes, kvbytes = decode_bytes(w, B, mid_ctx)
@@ -415,9 +408,19 @@ def run_native(args, rank, world):
         run.fill_cache()
 
         # ---- headline: K decode steps, device-timed --------------------------------------
-        dev_ms, (h0, h1) = run.decode_ms(barrier)
+        # (fused path: with the kernels' own start / end stamps on, so that the same region gives the step time and
+        # every kernel's share of it; the unstamped region after it shows what the stamps cost)
+        dev_ms, (h0, h1) = run.decode_ms(barrier, stamped=fused)
         launches = run.stack.launches_last_call() * K
         clocks = clk.window(h0, h1)
+        if fused:
+            kind_ms, span_ms, kind_launches = run.timeline_totals()
+            plain_ms, _ = run.decode_ms(barrier, base=2 * (W + K))
+            plain_ms /= K
+            how = ("kernel start/end stamps (two atomics per thread block) folded on the device by a small kernel at the end of "
+                   "every graph-replayed step, taken over the K steps of the timed region itself; a launch's share = its end "
+                   "minus the later of its start and the latest end before it, so the shares add up to at most the step; "
+                   "ms_per_step_unstamped is the same K steps timed again without stamps")
 
         # ---- end to end: host buffers, copies inside the timed region, result read every step
         x_host = run.xs[W:].cpu().pin_memory()
@@ -434,14 +437,8 @@ def run_native(args, rank, world):
         e2e_s = time.perf_counter() - t0
         barrier()
 
-        # ---- where the step's time goes ------------------------------------------------------
-        gw = gemm_weight_bytes(w)
-        if fused:
-            kind_ms, span_ms, kind_launches, tl_step_ms = run.timeline(barrier)
-            how = ("kernel start/end stamps folded on the device over K graph-replayed steps issued back to back as in the timed "
-                   "region; a launch's share = its end minus the later of its start and the latest end before it, so the shares "
-                   "add up to at most the step; timeline_ms_per_step is that pass timed with events like ms_per_step")
-        else:
+        # ---- where the step's time goes, for the paths whose kernels carry no stamps -------------
+        if not fused:
             for t in range(3):
                 run.step(2 * (W + K) + t)
             torch.cuda.synchronize()
@@ -452,7 +449,7 @@ def run_native(args, rank, world):
             prof = run.stack.profile_end()
             kind_ms = {k: v["ms"] / n_prof for k, v in prof.items()}
             kind_launches = {k: v["launches"] // n_prof for k, v in prof.items()}
-            span_ms = tl_step_ms = None
+            span_ms = plain_ms = None
             how = "events around every launch: serialised (no overlap between launches), a lower bound of what the kernels reach in the step"
 
         dev_ms, e2e_s = max_over_ranks([dev_ms, e2e_s], dev)
@@ -491,7 +488,7 @@ def run_native(args, rank, world):
                              "launches_per_step": gemm_launches, "avg_launch_us": gemm_ms * 1e3 / max(gemm_launches, 1),
                              "bytes_per_step": gemm_bytes_step, "how": how, "by_kind": by_kind},
                 "kernel_ms_per_step": kind_ms, "sum_kernel_ms": sum(kind_ms.values()), "timeline_span_ms": span_ms,
-                "timeline_ms_per_step": tl_step_ms,
+                "ms_per_step_unstamped": plain_ms,
                 "prefill": prefill_entry(w, run.Bp, run.Sp, pre_ms, tf_peak),
             }
 
