@@ -332,6 +332,106 @@ class Run:
             launches[kind] = launches.get(kind, 0) + 1
         return own_ms, span_ns / calls * 1e-6, launches
 
+def run_tp(args, rank, world):
+    """ONE model over the ranks of the job (Sec. 3: shard r on GPU r), decode steps only: --tp fused runs the rank mode
+    (shard sums exchanged inside the projection tails over peer-mapped memory), --tp baseline the same shards with
+    an NCCL all-reduce between kernels at every sync-point the mask keeps.  The workload's T becomes the world size.
+    Strong scaling: the batch is the workload's, whatever the number of ranks."""
+    import paper_2502_20727_b200 as spd
+    from paper_2502_20727_b200 import build as spd_build
+    import torch.distributed as dist
+    dev = torch.device(f"cuda:{int(os.environ.get('LOCAL_RANK', 0))}")
+    torch.cuda.set_device(dev)
+    torch.cuda.set_stream(torch.cuda.Stream(device=dev))
+    if rank == 0:
+        spd_build.build()
+    dist.barrier()
+    T, K, W = world, args.steps, args.warmup
+    w0 = si.WORKLOADS[args.workload]
+    if args.layers:
+        w0 = w0.with_(n_layers=args.layers, mask=tuple(w0.mask[:args.layers]))
+    w = w0.with_(T=T)
+    mask = pick_mask(w, args.mask)
+    B, ctx0 = w.batch, w.prompt + max(0, (w.decode_steps - (W + K)) // 2)
+    one = w.with_(n_q_heads=w.n_q_heads // T, n_kv_heads=w.n_kv_heads // T, ffn=w.ffn // T, T=1)
+    shard = []
+    for l in range(w.n_layers):  # every rank draws the same layer (same seed) and keeps its own rows / columns
+        shard.append(spd.shard_layer(si.make_layer(w, l, dev, 0), rank, T))
+    max_len = ctx0 + W + K + 2
+    pages = (max_len + w.kv_block - 1) // w.kv_block
+    stack = spd.stack_from_workload(one, shard, sync_mask=mask, max_batch=B, max_seq_len=max_len, n_pages=B * pages,
+                                    max_prefill_tokens=min(B * ctx0, args.prefill_chunk), device=dev)
+    bt = si.make_block_table(B, pages, B * pages, 0).to(dev)
+    xs = si.make_hidden(w, (W + K, B, w.hidden), dev, 0, 1)
+    x_in, seq_in = torch.empty_like(xs[0]), torch.empty(B, dtype=torch.int32, device=dev)
+    collective = spd.CollectiveAllReduce()
+    if args.tp == "fused":
+        if T > 1:
+            stack.tp_attach_symmetric(rank, T)
+        else:
+            stack.tp_attach(1, 0, [_one_region(stack, dev)], stack.tp_region_bytes(1))
+        out = torch.empty((1, B, w.hidden), dtype=xs.dtype, device=dev)
+    else:
+        out = torch.empty((B, w.hidden), dtype=xs.dtype, device=dev)
+
+    def step(t):
+        x_in.copy_(xs[t])
+        seq_in.fill_(ctx0 + t)
+        if args.tp == "fused":
+            stack.tp_decode_step(x_in, seq_in, bt, ctx0 + t + 1, out)
+        else:
+            stack.tp_baseline_decode_step(x_in, seq_in, bt, ctx0 + t + 1, collective, out)
+
+    def barrier():
+        torch.cuda.synchronize()
+        dist.barrier()
+        torch.cuda.synchronize()
+
+    with ClockSampler(dev.index or 0) as clk:
+        for t in range(W):
+            step(t)
+        barrier()
+        calls0 = collective.calls
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0 = time.perf_counter()
+        e0.record()
+        for t in range(W, W + K):
+            step(t)
+        e1.record()
+        barrier()
+        h1 = time.perf_counter()
+        if stack.device_error() != 0:
+            raise RuntimeError("device error flag set during the timed region")
+        dev_ms, = max_over_ranks([e0.elapsed_time(e1)], dev)
+        clocks = clk.window(h0, h1)
+    if rank != 0:
+        return None
+    hbm_peak, _, peak_kind = measured_peaks()
+    mid_ctx = ctx0 + W + (K + 1) / 2.0
+    wbytes, kvbytes = decode_bytes(w, B, mid_ctx)
+    per_rank = (wbytes + kvbytes) / T  # every rank streams its own shard of the weights and of the K/V
+    sync_points = sum(2 if m else 1 for m in mask)
+    return {"metric": METRIC, "value": B * K / (dev_ms * 1e-3), "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": dev_ms / K, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": w.dtype,
+            "data": "synthetic",
+            "config": {"workload": f"{w.name}: {w.n_layers} layers over {T} ranks (one shard per GPU), batch {B}, context {ctx0}+",
+                       "rank_mode": "fused exchange in the projection tails" if args.tp == "fused" else "NCCL all-reduce between kernels",
+                       "mask": list(mask), "mask_name": args.mask, "sync_points_per_step": sync_points,
+                       "all_reduce_calls_per_step": (collective.calls - calls0) / K if args.tp == "baseline" else None,
+                       "exchange_bytes_per_rank_per_step": sync_points * B * w.hidden * 4 * (T - 1),
+                       "l2": "weights per step exceed L2 (inputs larger than L2)" if wbytes / T > 126e6 else "rank's shard fits L2",
+                       "multi_gpu": "tensor parallel"},
+            "gpu_launches": stack.launches_last_call() * K, "clocks": clocks,
+            "step_roofline": {"bytes_per_step_per_rank": per_rank, "achieved_gbs_per_rank": per_rank / (dev_ms / K * 1e-3) / 1e9,
+                              "frac": per_rank / (dev_ms / K * 1e-3) / 1e9 / hbm_peak, "peak": hbm_peak, "peak_kind": peak_kind}}
+
+
+def _one_region(stack, dev):
+    n = (stack.tp_region_bytes(1) + 1023) // 1024 * 1024
+    stack._tp_regions = torch.empty(n + 1024, dtype=torch.uint8, device=dev)
+    return (stack._tp_regions.data_ptr() + 1023) // 1024 * 1024
+
+
 def roofline_entry(w, B, mid_ctx, ms_per_step, hbm_peak, peak_kind):
     wbytes, kvbytes = decode_bytes(w, B, mid_ctx)
     gbs = (wbytes + kvbytes) / (ms_per_step * 1e-3) / 1e9
@@ -457,6 +557,7 @@ def run_native(args, rank, world):
         if rank == 0:
             mid_ctx = run.ctx0 + W + (K + 1) / 2.0
             ms_per_step = dev_ms / K
+            gw = gemm_weight_bytes(w)
             gemm_ms = sum(kind_ms.get(k, 0.0) for k in GEMM_KINDS)
             gemm_launches = sum(kind_launches.get(k, 0) for k in GEMM_KINDS)
             gemm_bytes_step = w.n_layers * sum(gw.values())
@@ -625,6 +726,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--rank-mode", action="store_true",
                     help="decode through spd_tp_decode_step: all T ranks of a tensor-parallel group executed on this GPU")
+    ap.add_argument("--tp", default="", choices=["", "fused", "baseline"],
+                    help="ONE model over the job's ranks, shard r on rank r (launch under torchrun with as many ranks as shards): "
+                         "fused = exchanges inside the projection tails (rank mode), baseline = NCCL all-reduce between kernels")
     ap.add_argument("--tune", default="", help="decode tuning knobs, e.g. qkv_splits=4,l2_prefetch_blocks=8 (see spd_set_tuning)")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
@@ -640,13 +744,16 @@ def main():
         return
     args.steps = args.steps if args.steps is not None else 32
     args.warmup = max(args.warmup if args.warmup is not None else 5, 3)
-    if world > 1:
+    if world > 1 or args.tp:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", str(free_port()))
+        os.environ.setdefault("RANK", "0")
+        os.environ.setdefault("WORLD_SIZE", "1")
         torch.distributed.init_process_group("nccl", device_id=torch.device(f"cuda:{int(os.environ.get('LOCAL_RANK', 0))}"))
-    res = run_native(args, rank, world)
+    res = run_tp(args, rank, world) if args.tp else run_native(args, rank, world)
     if rank == 0:
         print(json.dumps(res), flush=True)
-    if world > 1:
+    if world > 1 or args.tp:
         torch.distributed.destroy_process_group()
 
 

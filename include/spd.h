@@ -41,6 +41,7 @@ extern "C" {
 #define SPD_ECAPACITY (-4)  /* sequence would outgrow max_seq_len or the block table                  */
 #define SPD_ECUDA (-5)      /* a CUDA call failed; see spd_last_cuda_error()                          */
 #define SPD_EDEVICE (-6)    /* a kernel recorded a bounds / bounded-wait failure in its error flag   */
+#define SPD_ECALLBACK (-7)  /* the all-reduce callback of spd_tp_baseline_* returned non-zero          */
 
 typedef struct spd_ctx spd_ctx; /* opaque; owned by the library, freed by spd_destroy */
 
@@ -331,6 +332,32 @@ int spd_tp_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *se
  * Errors: SPD_ENULL, SPD_EINVAL (not attached, B > max_batch), SPD_ECAPACITY, SPD_ECUDA. */
 int spd_tp_prefill(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int32_t *block_table,
                    int32_t max_pages, void *out, void *stream);
+
+/* Baseline of the rank mode: the same shard-per-rank execution with the shard sums done by a library collective
+ * BETWEEN kernels - how tensor parallelism is normally run (Sec. 3: two all-reduces per TP block, NCCL in the
+ * paper's measurements) - instead of the exchange fused into the projection's tail.  The context is ONE shard's
+ * stack (created with T = 1 from the shard's dims and weights, exactly as for spd_tp_attach; not attached).  The
+ * step runs the projections as K-split GEMMs with separate residual / norm kernels and calls `all_reduce` on
+ * `stream`'s behalf at every sync-point the block keeps: a TP block twice (Y_r after o_proj, Z_r after down),
+ * an SPD block once (Y_r + Z_r after down; R_r = X + Y_r feeds the rank's own MLP, X joins after the sum:
+ * Sec. 4.1.1).
+ *   all_reduce(user, buf, count, stream) : must leave in buf (device, fp32, `count` = tokens of the launch x hidden
+ *       elements) the element-wise SUM of all ranks' buf, ordered on `stream` after the work enqueued so far and
+ *       before what is enqueued next (e.g. ncclAllReduce on that stream); returns 0, anything else aborts the
+ *       call with SPD_ECALLBACK.  Every rank makes the same calls in the same order.
+ *   scratch : device, fp32, at least 2 x (tokens per launch) x hidden floats; tokens per launch = B for a decode
+ *       step, min(B * S, max_prefill_tokens) for prompts
+ * Launched directly (no graph replay: the collective is the caller's).  bf16 LLaMA-style stacks only.
+ * Errors: SPD_ENULL, SPD_EINVAL (context holds more than one shard, ...), SPD_ECAPACITY, SPD_EWORKSPACE (scratch too
+ * small), SPD_ECALLBACK, SPD_ECUDA. */
+typedef int (*spd_allreduce_fn)(void *user, float *buf, size_t count, void *stream);
+int spd_tp_baseline_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_lens,
+                                const int32_t *block_table, int32_t max_pages, int32_t max_context, void *out,
+                                float *scratch, size_t scratch_floats, spd_allreduce_fn all_reduce, void *user,
+                                void *stream);
+int spd_tp_baseline_prefill(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int32_t *block_table,
+                            int32_t max_pages, void *out, float *scratch, size_t scratch_floats,
+                            spd_allreduce_fn all_reduce, void *user, void *stream);
 
 /* Number of shard sums ("sync-points", Sec. 3) one forward pass of this stack executes:
  * 2 per TP block, 1 per SPD block. */

@@ -17,7 +17,8 @@ LIB_PATH = os.path.join(_HERE, "libspd_b200.so")
 
 SPD_OK = 0
 STATUS_NAMES = {0: "SPD_OK", -1: "SPD_EINVAL", -2: "SPD_ENULL", -3: "SPD_EWORKSPACE", -4: "SPD_ECAPACITY",
-                -5: "SPD_ECUDA", -6: "SPD_EDEVICE"}
+                -5: "SPD_ECUDA", -6: "SPD_EDEVICE", -7: "SPD_ECALLBACK"}
+ALLREDUCE_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p)
 WEIGHT_NAMES = ("attn_norm", "wq", "wk", "wv", "wo", "mlp_norm", "w_gate", "w_up", "w_down")
 BIAS_FIELDS = ("attn_norm_b", "bq", "bk", "bv", "bo", "mlp_norm_b", "b_fc1", "b_fc2")
 # tensors of a layer of the block with bias (Sec. 4.1.2) -> fields of spd_layer
@@ -31,7 +32,7 @@ EXPORTS = ("spd_workspace_bytes", "spd_create", "spd_prefill", "spd_decode_step"
            "spd_set_tuning", "spd_set_mask", "spd_sensitivity_scan", "spd_alg1_plan",
            "spd_head_grouping_stats", "spd_head_scatter", "spd_mlp_match", "spd_timeline_begin", "spd_timeline_read",
            "spd_timeline_end", "spd_tp_region_bytes", "spd_tp_attach", "spd_tp_detach", "spd_tp_decode_step",
-           "spd_tp_prefill")
+           "spd_tp_prefill", "spd_tp_baseline_decode_step", "spd_tp_baseline_prefill")
 
 
 class SpdError(RuntimeError):
@@ -96,6 +97,8 @@ def load_library() -> ctypes.CDLL:
     lib.spd_tp_detach.argtypes = [vp]
     lib.spd_tp_decode_step.argtypes = [vp, vp, i32, vp, vp, i32, i32, vp, vp]
     lib.spd_tp_prefill.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp]
+    lib.spd_tp_baseline_decode_step.argtypes = [vp, vp, i32, vp, vp, i32, i32, vp, vp, sz, ALLREDUCE_FN, vp, vp]
+    lib.spd_tp_baseline_prefill.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, sz, ALLREDUCE_FN, vp, vp]
     lib.spd_profile_begin.argtypes = [vp]
     lib.spd_profile_end.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     lib.spd_timeline_begin.argtypes = [vp, vp]
@@ -271,6 +274,21 @@ def shard_layer(lw: Dict[str, torch.Tensor], r: int, T: int) -> Dict[str, torch.
     return {"attn_norm": lw["attn_norm"], "mlp_norm": lw["mlp_norm"], "wq": rows(lw["wq"]), "wk": rows(lw["wk"]),
             "wv": rows(lw["wv"]), "wo": cols(lw["wo"]), "w_gate": rows(lw["w_gate"]), "w_up": rows(lw["w_up"]),
             "w_down": cols(lw["w_down"])}
+
+
+class CollectiveAllReduce:
+    """The all-reduce of the rank-mode baseline as a torch.distributed collective (NCCL on GPUs, gloo on CPU tensors):
+    sums the view over the group in place on the current stream and counts the calls - one per sync-point the
+    blocks keep (Sec. 3: two per TP block; Sec. 4.1.1: one per SPD block)."""
+
+    def __init__(self, group=None):
+        self.group, self.calls, self.elements = group, 0, 0
+
+    def __call__(self, view: torch.Tensor):
+        import torch.distributed as dist
+        dist.all_reduce(view, op=dist.ReduceOp.SUM, group=self.group)
+        self.calls += 1
+        self.elements += view.numel()
 
 
 class SpdStack:
@@ -513,6 +531,56 @@ class SpdStack:
             _check("spd_tp_decode_step", self.lib.spd_tp_decode_step(self._ctx, x.data_ptr(), B, seq_lens.data_ptr(),
                                                                       block_table.data_ptr(), block_table.shape[1],
                                                                       int(max_context), out.data_ptr(), _stream_ptr()))
+        return out
+
+    # -- baseline of the rank mode: the shard sums as a collective between kernels (spd_tp_baseline_*) ---------
+    def _baseline_hook(self, all_reduce, tokens):
+        """(ctypes callback, scratch tensor) for one call: the library hands the callback a pointer into `scratch`;
+        the caller's all_reduce gets the matching fp32 view and sums it over the ranks in place."""
+        need = 2 * tokens * self.dims.hidden
+        if getattr(self, "_baseline_scratch", None) is None or self._baseline_scratch.numel() < need:
+            self._baseline_scratch = torch.empty(need, dtype=torch.float32, device=self.device)
+        scratch, self._baseline_error = self._baseline_scratch, None
+
+        def hook(user, buf, count, stream):
+            try:
+                first = (int(buf) - scratch.data_ptr()) // 4
+                all_reduce(scratch[first:first + int(count)])
+                return 0
+            except Exception as e:  # surfaces as SPD_ECALLBACK; the exception itself is re-raised by the caller
+                self._baseline_error = e
+                return 1
+        return ALLREDUCE_FN(hook), scratch
+
+    def tp_baseline_decode_step(self, x, seq_lens, block_table, max_context, all_reduce, out=None):
+        """One decode step of ONE shard's stack (this context: T = 1, the shard's weights) with the block's kept shard
+        sums done by ``all_reduce(view)`` - an in-place sum of a float32 CUDA view over all ranks, enqueued on the
+        current stream (e.g. ``torch.distributed.all_reduce``); see spd_tp_baseline_decode_step."""
+        B, H = x.shape
+        self._check_io(x, block_table)
+        out = torch.empty_like(x) if out is None else out
+        fn, scratch = self._baseline_hook(all_reduce, B)
+        with torch.cuda.device(self.device):
+            rc = self.lib.spd_tp_baseline_decode_step(self._ctx, x.data_ptr(), B, seq_lens.data_ptr(), block_table.data_ptr(),
+                                                      block_table.shape[1], int(max_context), out.data_ptr(), scratch.data_ptr(),
+                                                      scratch.numel(), fn, None, _stream_ptr())
+        if self._baseline_error is not None:
+            raise self._baseline_error
+        _check("spd_tp_baseline_decode_step", rc)
+        return out
+
+    def tp_baseline_prefill(self, x, block_table, all_reduce, out=None):
+        """Prompts through ONE shard's stack with the kept shard sums done by ``all_reduce``; see spd_tp_baseline_prefill."""
+        B, S, H = x.shape
+        self._check_io(x, block_table)
+        out = torch.empty_like(x) if out is None else out
+        fn, scratch = self._baseline_hook(all_reduce, min(B * S, self.dims.max_prefill_tokens))
+        with torch.cuda.device(self.device):
+            rc = self.lib.spd_tp_baseline_prefill(self._ctx, x.data_ptr(), B, S, block_table.data_ptr(), block_table.shape[1],
+                                                  out.data_ptr(), scratch.data_ptr(), scratch.numel(), fn, None, _stream_ptr())
+        if self._baseline_error is not None:
+            raise self._baseline_error
+        _check("spd_tp_baseline_prefill", rc)
         return out
 
     def sync_points(self) -> int:

@@ -616,6 +616,134 @@ int run_tokens(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t
     return SPD_OK;
 }
 
+// Baseline of the rank mode (Sec. 3): ONE shard's stack (a context created with T = 1 from the shard's dims and
+// weights, as for spd_tp_attach) run through the unfused kernels, with every shard sum the block keeps handed to
+// a caller-supplied all-reduce - a library collective (NCCL) between kernels instead of the exchange inside the
+// projection's tail.  A TP block calls it twice (Y_r after o_proj, Z_r after down), an SPD block once
+// (Y_r + Z_r after down; R_r = X + Y_r stays on the rank, X joins after the sum: Sec. 4.1.1).
+// scratch: 2 * M * H floats.  cur / other: the two residual-stream buffers.
+int run_tp_baseline(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t *bt, int max_pages, bool decode,
+                    int max_context, float *scratch, spd_allreduce_fn fn, void *user, cudaStream_t st)
+{
+    const spd_dims &d = c->d;
+    const int H = d.hidden, qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, F = d.ffn;
+    const int nqkv = qd + 2 * kd;
+    const long Mc = c->Mcap;
+    const Plan p = make_plan(d, M, decode, max_context);
+    PageTable pt{bt, max_pages, c->n_pages, d.kv_block_size, d.n_kv_heads};
+    const bool swap = decode;
+    const int tbox = tc_token_box(swap, M);
+    const bool rope_on = d.rope_base > 0.f;
+    const long MH = (long)M * H;
+    float *ybuf = scratch, *zbuf = scratch + MH;
+    float *cur = c->res[0], *other = c->res[1];
+    int launches = 0;
+    // dst = base + sum of n planes (fp32 [M][H] each); base may be null (then plane 0 serves as base)
+    auto add_planes = [&](float *dst, const float *base, const float *planes, int n) -> cudaError_t {
+        NormArgs a{};
+        a.res_in = base ? base : planes;
+        a.part = base ? planes : (n > 1 ? planes + MH : nullptr);
+        a.part_stride = MH; a.n_groups = 1; a.per_group = base ? n : n - 1;
+        a.res_out = dst; a.M = M; a.H = H; a.eps = d.rms_eps;
+        return launch_residual_norm<bf16>(a, st);
+    };
+    auto all_reduce = [&](float *buf) -> int {
+        if (fn(user, buf, (size_t)MH, (void *)st) != 0) return SPD_ECALLBACK;
+        return SPD_OK;
+    };
+    auto gemm = [&](Kind kind, const TcMap *const *wmaps, int nw, ActBuf ab, float *C, long ldc, const int *w_rows, const long *c_off,
+                    int K, int splits) -> int {
+        MAP_OR_FAIL(am, act_map(c, ab, tbox));
+        TcGemmArgs g{};
+        g.C = C; g.ldc = ldc; g.c_batch_stride = 0; g.c_split_stride = (long)M * ldc;
+        for (int i = 0; i < nw; ++i) { g.w_rows[i] = w_rows[i]; g.c_off[i] = c_off[i]; }
+        g.t_rows = M; g.batches = 1; g.w_batched = 0; g.t_batched = 0;
+        g.num_kb = cdiv(K, 64); g.splits = splits; g.err = c->err;
+        LAUNCH(kind, launch_gemm_tc(wmaps, nw, *am, g, swap, st));
+        return SPD_OK;
+    };
+
+    if (rope_on) LAUNCH(K_ROPE_TABLE, launch_rope_table(c->rope, tm, M, d.head_dim, d.rope_base, st));
+    {
+        NormArgs a{};
+        a.x_in = x; a.res_out = cur; a.h_out = c->h; a.h_stride = Mc * H;
+        a.gain = c->layers[0].attn_norm; a.n_groups = 1; a.per_group = 0; a.M = M; a.H = H; a.eps = d.rms_eps;
+        LAUNCH(K_NORM, launch_residual_norm<bf16>(a, st));
+    }
+    for (int l = 0; l < d.n_layers; ++l) {
+        const spd_layer &w = c->layers[l];
+        const LayerMaps &lm = c->maps[l];
+        const bool sync = c->mask[l] != 0;
+        int rc;
+        {   // a2 - a4 on the rank's own heads
+            const TcMap *wmaps[3] = {&lm.wq, &lm.wk, &lm.wv};
+            const int wn[3] = {qd, kd, kd};
+            const long wcol[3] = {0, qd, (long)qd + kd};
+            if ((rc = gemm(K_QKV, wmaps, 3, AB_H, c->qkv32, nqkv, wn, wcol, H, p.qkv_splits)) != SPD_OK) return rc;
+            RopeKvArgs a{};
+            a.qkv = c->qkv32; a.ldq = nqkv; a.split_stride = (long)M * nqkv; a.splits = p.qkv_splits;
+            a.table = c->rope; a.q_out = c->q; a.k_pages = w.k_pages; a.v_pages = w.v_pages; a.pt = pt; a.tm = tm;
+            a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.use_rope = rope_on; a.err = c->err;
+            LAUNCH(K_ROPE_KV, launch_rope_kv<bf16>(a, st));
+            AttnArgs t{};
+            t.q = c->q; t.k_pages = w.k_pages; t.v_pages = w.v_pages; t.pt = pt; t.tm = tm; t.out = c->attn;
+            t.M = M; t.n_q_heads = d.n_q_heads; t.head_dim = d.head_dim; t.B = M; t.splits = p.attn_splits;
+            t.max_context = max_context; t.part_o = c->part_o; t.part_ml = c->part_ml; t.counters = c->attn_cnt; t.err = c->err;
+            if (!decode && d.head_dim == 128 && d.kv_block_size == 16) {
+                MAP_OR_FAIL(qm, act_map(c, AB_Q, 128));
+                t.q_map = qm; t.k_map = &lm.kpages; t.v_map = &lm.vpages; t.rescale_log2 = (float)c->prefill_rescale_log2;
+            }
+            if (decode) LAUNCH(K_ATTN, launch_decode_attention<bf16>(t, st));
+            else LAUNCH(K_ATTN, launch_prefill_attention<bf16>(t, st));
+        }
+        {   // a5: the rank's partial attention output Y_r, in K-range planes, then as one [M][H] buffer
+            const TcMap *wmaps[1] = {&lm.wo_full};
+            const int wn[1] = {H};
+            const long wcol[1] = {0};
+            if ((rc = gemm(K_OPROJ, wmaps, 1, AB_ATTN, c->proj32, H, wn, wcol, qd, p.o_per_group)) != SPD_OK) return rc;
+            LAUNCH(K_NORM, add_planes(ybuf, nullptr, c->proj32, p.o_per_group));
+        }
+        // a6: sync-point 1 is an all-reduce of Y_r in a TP block and is dropped in an SPD block (R_r = X + Y_r)
+        if (sync && (rc = all_reduce(ybuf)) != SPD_OK) return rc;
+        {   // a7
+            NormArgs a{};
+            a.res_in = cur; a.part = ybuf; a.part_stride = MH; a.n_groups = 1; a.per_group = 1;
+            a.res_out = other; a.h_out = c->h; a.h_stride = Mc * H; a.gain = w.mlp_norm; a.M = M; a.H = H; a.eps = d.rms_eps;
+            LAUNCH(K_NORM, launch_residual_norm<bf16>(a, st));
+        }
+        {   // a8, a9 on the rank's MLP slice
+            const TcMap *wmaps[2] = {&lm.w_gate, &lm.w_up};
+            const int wn[2] = {F, F};
+            const long wcol[2] = {0, (long)p.gu_splits * M * F};
+            if ((rc = gemm(K_GATE_UP, wmaps, 2, AB_H, c->gu32, F, wn, wcol, H, p.gu_splits)) != SPD_OK) return rc;
+            SiluMulArgs a{};
+            a.gate = c->gu32; a.up = c->gu32 + (long)p.gu_splits * M * F; a.ld = F; a.split_stride = (long)M * F;
+            a.splits = p.gu_splits; a.act = c->act; a.M = M; a.F = F;
+            LAUNCH(K_SILU_MUL, launch_silu_mul<bf16>(a, st));
+            const TcMap *dmaps[1] = {&lm.w_down};
+            const int dn[1] = {H};
+            const long dcol[1] = {0};
+            if ((rc = gemm(K_DOWN, dmaps, 1, AB_ACT, c->proj32, H, dn, dcol, F, p.down_splits)) != SPD_OK) return rc;
+        }
+        // the kept sync-point: Z_r in a TP block, Y_r + Z_r in an SPD block
+        LAUNCH(K_NORM, add_planes(zbuf, sync ? nullptr : ybuf, c->proj32, p.down_splits));
+        if ((rc = all_reduce(zbuf)) != SPD_OK) return rc;
+        {   // a10: TP block out = R + sum Z; SPD block out = X + sum (Y + Z)
+            // TP block: R (in other) + sum Z goes back into the block's input buffer.  SPD block: X (still in cur) + the
+            // sum goes over R_r, which is no longer needed, and the two buffers change roles.
+            NormArgs a{};
+            a.res_in = sync ? other : cur; a.part = zbuf; a.part_stride = MH; a.n_groups = 1; a.per_group = 1;
+            a.res_out = sync ? cur : other; a.M = M; a.H = H; a.eps = d.rms_eps;
+            if (l + 1 < d.n_layers) { a.h_out = c->h; a.h_stride = Mc * H; a.gain = c->layers[l + 1].attn_norm; }
+            else a.final_out = out;
+            LAUNCH(K_NORM, launch_residual_norm<bf16>(a, st));
+            if (!sync) { float *t2 = cur; cur = other; other = t2; }
+        }
+    }
+    c->launches_last = launches;
+    return SPD_OK;
+}
+
 // One decode step of the bf16 stack with the fused projections: per block QKV(+rotary, KV append),
 // paged attention, o_proj(+residuals, MLP norm input), gate/up(+SwiGLU), down(+shard sum, residual).
 int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const int32_t *bt, int max_pages,
@@ -1554,6 +1682,60 @@ int spd_tp_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *se
     return SPD_OK;
 }
 
+int spd_tp_baseline_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_lens, const int32_t *block_table,
+                                int32_t max_pages, int32_t max_context, void *out, float *scratch, size_t scratch_floats,
+                                spd_allreduce_fn fn, void *user, void *stream)
+{
+    if (!ctx || !x || !seq_lens || !block_table || !out || !scratch || !fn) return SPD_ENULL;
+    Ctx &c = ctx->c;
+    const spd_dims &d = c.d;
+    if (d.T != 1 || d.dtype != 1 || d.block_kind != 0 || d.hidden % 16) return SPD_EINVAL; // one shard's stack, bf16, no bias
+    if (B < 1 || B > d.max_batch || x == out || max_context < 1) return SPD_EINVAL;
+    if (max_context > d.max_seq_len || (long)max_pages * d.kv_block_size < max_context) return SPD_ECAPACITY;
+    if (scratch_floats < (size_t)2 * B * d.hidden) return SPD_EWORKSPACE;
+    TokMap tm{1, 0, 1, 0, seq_lens};
+    return run_tp_baseline(&c, x, out, B, tm, block_table, max_pages, true, max_context, scratch, fn, user, (cudaStream_t)stream);
+}
+
+int spd_tp_baseline_prefill(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int32_t *block_table, int32_t max_pages,
+                            void *out, float *scratch, size_t scratch_floats, spd_allreduce_fn fn, void *user, void *stream)
+{
+    if (!ctx || !x || !block_table || !out || !scratch || !fn) return SPD_ENULL;
+    Ctx &c = ctx->c;
+    const spd_dims &d = c.d;
+    if (d.T != 1 || d.dtype != 1 || d.block_kind != 0 || d.hidden % 16) return SPD_EINVAL;
+    if (B < 1 || S < 1 || B > d.max_batch || x == out) return SPD_EINVAL;
+    if (S > d.max_seq_len || (long)max_pages * d.kv_block_size < S) return SPD_ECAPACITY;
+    const int Mp = d.max_prefill_tokens;
+    const long chunk = (long)B * S < Mp ? (long)B * S : Mp;
+    if (scratch_floats < (size_t)2 * chunk * d.hidden) return SPD_EWORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    int total_launches = 0;
+    auto run = [&](int b0, int nb, int s0, int ns) -> int {
+        TokMap tm{0, b0, ns, s0, nullptr};
+        const size_t off = ((size_t)b0 * S + s0) * d.hidden * 2;
+        const int rc = run_tp_baseline(&c, (const char *)x + off, (char *)out + off, nb * ns, tm, block_table, max_pages, false, S, scratch,
+                                       fn, user, st);
+        total_launches += c.launches_last;
+        return rc;
+    };
+    if (S <= Mp) {
+        const int nb = Mp / S;
+        for (int b0 = 0; b0 < B; b0 += nb) {
+            const int rc = run(b0, B - b0 < nb ? B - b0 : nb, 0, S);
+            if (rc) return rc;
+        }
+    } else {
+        for (int b = 0; b < B; ++b)
+            for (int s0 = 0; s0 < S; s0 += Mp) {
+                const int rc = run(b, 1, s0, S - s0 < Mp ? S - s0 : Mp);
+                if (rc) return rc;
+            }
+    }
+    c.launches_last = total_launches;
+    return SPD_OK;
+}
+
 int spd_gemm_bf16(const void *a, const void *w, float *c, int32_t M, int32_t N, int32_t K, int32_t batches,
                   int32_t a_batched, int32_t splits, int32_t swap, int32_t *err_flag, void *stream)
 {
@@ -1683,6 +1865,7 @@ const char *spd_status_string(int s)
     case SPD_ECAPACITY: return "sequence exceeds the KV capacity";
     case SPD_ECUDA: return "CUDA error";
     case SPD_EDEVICE: return "device-side error flag set";
+    case SPD_ECALLBACK: return "the caller's all-reduce callback reported a failure";
     default: return "unknown status";
     }
 }

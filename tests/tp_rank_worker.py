@@ -19,10 +19,10 @@ import paper_2502_20727_b200 as spd  # noqa: E402
 import spd_inputs as si  # noqa: E402
 
 
-def all_reduce(a, counter):
+def all_reduce(a, collective):
+    """Through the same helper the GPU baseline arm hands to spd_tp_baseline_* (there over NCCL, here over gloo)."""
     t = torch.from_numpy(np.ascontiguousarray(a))
-    dist.all_reduce(t)
-    counter[0] += 1
+    collective(t)
     return t.numpy()
 
 
@@ -42,7 +42,7 @@ def main():
     res = {}
     for mode, name in ((0, "spd"), (1, "sync")):
         ref, _, ref_syncs = oracle.block_forward(dims, to_np(full), mode, x, pos0, oracle.Cache(dims, B, S))
-        n = [0]
+        n = spd.CollectiveAllReduce()
         if mode == 0:
             # R_r = X + Y_r stays on the rank; one exchange of Y_r + Z_r; X joins after the sum
             out_r, _, _ = oracle.block_forward(one, to_np(mine), 0, x, pos0, oracle.Cache(one, B, S))
@@ -54,7 +54,7 @@ def main():
             no_attn = dict(mine, wo=torch.zeros_like(mine["wo"]))
             z_r, _, _ = oracle.block_forward(one, to_np(no_attn), 1, r, pos0, oracle.Cache(one, B, S))
             out = r + all_reduce(z_r - r, n)
-        res[name] = {"err": float(np.max(np.abs(out - ref)) / np.max(np.abs(ref))), "exchanges": n[0], "syncs": int(ref_syncs)}
+        res[name] = {"err": float(np.max(np.abs(out - ref)) / np.max(np.abs(ref))), "exchanges": n.calls, "syncs": int(ref_syncs)}
     gathered = [None] * T
     dist.all_gather_object(gathered, res)
     if rank == 0:
