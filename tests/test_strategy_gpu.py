@@ -13,8 +13,23 @@ from parity_util import Pair
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("dtype,tol", [("fp32", 2e-3), ("bf16", 0.1)])
-def test_scan_matches_the_oracle_and_gives_the_same_plan(dtype, tol):
+def metric_tolerance(dtype, ref_out, scale):
+    """Absolute tolerance of a metric = mean((out_a - out_b)^2) of two stack outputs.
+    bf16: each output element v is rounded once more to bf16 on its way out, an error uniform within +-u|v|, u = 2^-8,
+    independent between the two passes wherever they differ; it does not cancel in the difference but adds its variance,
+    2 u^2 mean(v^2) / 3, to the mean square (the cross term with the true difference averages out over the elements).
+    The bf16 roundings inside the blocks that differ between the passes are of the same size: the floor is doubled.
+    That is what the outputs can resolve, not a margin of the kernels - here about a tenth of the largest metric, because
+    the SPD / TP difference (rms 0.02) is small against the outputs themselves (up to 7).
+    fp32: the same floor with u = 2^-24 is nil; 2e-3 of the largest metric covers the fp32 reassociation of the sums."""
+    if dtype == "fp32":
+        return 2e-3 * scale
+    u = 2.0 ** -8
+    return 2 * (2 * u * u * float(np.mean(np.square(ref_out))) / 3)
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_scan_matches_the_oracle_and_gives_the_same_plan(dtype):
     L, T = 4, 4
     w = si.Workload("scan", dtype, L, 256, 8, 8, 32, 512, T, (0,) * L, 2, 40, 0)
     layers = si.make_stack(w, "cpu", 7)
@@ -27,9 +42,13 @@ def test_scan_matches_the_oracle_and_gives_the_same_plan(dtype, tol):
     ref_s, ref_m = ostrat.sensitivity_scan(p.dims, p.layers_np, x.double().numpy())
     scale = max(ref_m)
     assert scale > 0
-    assert np.max(np.abs(np.array(metric) - np.array(ref_m))) <= tol * scale
-    assert np.max(np.abs(np.array(sens) - np.array(ref_s))) <= tol * scale
-    assert abs(sens[2]) <= tol * scale
+    ref_out, _, _ = oracle.stack_forward(p.dims, [1] * L, p.layers_np, x.double().numpy(), np.zeros(2, np.int32),
+                                         oracle.Cache(p.dims, 2, 40))
+    tol = metric_tolerance(dtype, ref_out, scale)
+    assert tol <= 0.15 * scale                                 # the floor stays a fraction of what is being measured
+    assert np.max(np.abs(np.array(metric) - np.array(ref_m))) <= tol
+    assert np.max(np.abs(np.array(sens) - np.array(ref_s))) <= 2 * tol   # a difference of two metrics
+    assert abs(sens[2]) <= 2 * tol
     # thresholds in the gaps of the oracle's values: both sides must take the same decisions
     order = np.sort(ref_s)
     tau1, tau2 = (order[0] + order[1]) / 2, (order[2] + order[3]) / 2
