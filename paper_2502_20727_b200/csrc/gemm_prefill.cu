@@ -36,6 +36,7 @@ constexpr int X_COL = 256;   // PRE_OPROJ_SPD: the X tile (columns 0-255 hold th
 // o_proj) of the operand bytes cross from L2 into shared memory, and the ring holds more K blocks.
 template <int EPI, int PAIR> struct PCfg {
     static constexpr int BN = (EPI == PRE_OPROJ_SPD) ? 128 : 256;
+    static_assert(EPI != PRE_SCATTER || PAIR, "the scatter epilogue is only built for CTA pairs");
     static constexpr int A_BYTES = BM * BK * 2, B_BYTES = (BN / (PAIR ? 2 : 1)) * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int X_BYTES = 0, H_BYTES = 0;
@@ -198,7 +199,7 @@ __device__ __forceinline__ void epi_qkv(const PreGemmArgs &g, const PreTile &t, 
     for (int hh = 0; hh < heads; ++hh) {
         const int row_h = t.row0 + hh * d;
         if (row_h >= g.w_rows[t.wi]) break;
-        const int head = row_h / d;
+        const int head = row_h / d + (t.wi == 0 ? g.q_head0 : g.kv_head0);
         bf16 *dst = nullptr;
         if (valid) {
             if (t.wi == 0) dst = (bf16 *)g.q_out + ((long)m * nq + head) * d;
@@ -233,7 +234,7 @@ __device__ __forceinline__ void epi_qkv(const PreGemmArgs &g, const PreTile &t, 
 __device__ __forceinline__ void epi_gateup(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, int m, bool valid)
 {
     const float rs = valid ? row_rstd(g.ss_in, g.rstd_per_shard ? t.z : 0, m) : 0.f;
-    bf16 *dst = (bf16 *)g.act + (long)m * g.F + (long)((t.z + g.w_rot) % g.batches) * g.Fs + t.row0;
+    bf16 *dst = (bf16 *)g.act + (long)m * g.F + g.act_col0 + (long)((t.z + g.w_rot) % g.batches) * g.Fs + t.row0;
 #pragma unroll 1
     for (int c = 0; c < 8; ++c) {
         const int f = t.row0 + c * 16;
@@ -292,13 +293,50 @@ __device__ __forceinline__ void epi_resid(const PreGemmArgs &g, const PreTile &t
         const long idx = (long)m * g.H + n;
         float x[16];
         load_x16(g.res_in + idx, x);
+        if (g.ysave) { stg8(g.ysave + idx, ya); stg8(g.ysave + idx + 8, ya + 8); }
         ssq += resid_chunk(g, idx, n, x, ya, g.hg ? (bf16 *)g.hg : nullptr, true);
         if (n + 16 < g.H) {
             load_x16(g.res_in + idx + 16, x);
+            if (g.ysave) { stg8(g.ysave + idx + 16, yb); stg8(g.ysave + idx + 24, yb + 8); }
             ssq += resid_chunk(g, idx + 16, n + 16, x, yb, g.hg ? (bf16 *)g.hg : nullptr, true);
         }
     }
     if (valid && g.ss_out) g.ss_out[(long)t.nt * g.Mcap + m] = ssq;
+}
+
+// Rank mode, shot one of a two-shot exchange (see TpScatter): this block's 128 partial rows go to the rank that owns
+// the tile, then the step number is published in the owner's flag word for (slot, column tile, this rank).
+__device__ __forceinline__ void epi_scatter(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, int m, bool valid, int r)
+{
+    const TpScatter &sc = g.sc;
+    const int tile128 = t.m0 / BM, owner = tile128 % sc.T, slot = tile128 / sc.T;
+    float *dst = (float *)(sc.rx[owner] + (long)sc.me * sc.src_stride) + ((long)slot * BM + r) * g.H;
+#pragma unroll 1
+    for (int c = 0; c < 16; c += 2) {
+        const int n = t.row0 + c * 16;
+        if (n >= g.H) break;
+        float ya[16], yb[16];
+        tmem_ld16x2(tacc + c * 16, tacc + c * 16 + 16, ya, yb);
+        if (!valid) continue;
+        if (sc.addend) {
+            float a[16];
+            load_x16(sc.addend + (long)m * g.H + n, a);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) ya[i] += a[i];
+        }
+        stg8(dst + n, ya);
+        stg8(dst + n + 8, ya + 8);
+        if (n + 16 < g.H) {
+            if (sc.addend) {
+                float a[16];
+                load_x16(sc.addend + (long)m * g.H + n + 16, a);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) yb[i] += a[i];
+            }
+            stg8(dst + n + 16, yb);
+            stg8(dst + n + 24, yb + 8);
+        }
+    }
 }
 
 template <int N_THREADS> __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(N_THREADS) : "memory"); }
@@ -456,8 +494,8 @@ __global__ void __launch_bounds__(PCfg<EPI, PAIR>::THREADS_, 1) gemm_prefill_ker
                 const PreTile t = decode_tile(L, EPI, tile, PAIR, crank);
                 const CUtensorMap *tm_w = t.wi == 0 ? &tm_w0 : (t.wi == 1 ? &tm_w1 : &tm_w2);
                 for (int pass = 0; pass < L.passes && ok; ++pass) {
-                    const int tz = EPI == PRE_OPROJ_SPD ? pass : (EPI == PRE_GATEUP && g.t_batched ? t.z : 0);
-                    const int wz = EPI == PRE_OPROJ_SPD ? pass : (EPI == PRE_GATEUP ? (t.z + g.w_rot) % g.batches : t.z);
+                    const int tz = g.t_z + (EPI == PRE_OPROJ_SPD ? pass : (EPI == PRE_GATEUP && g.t_batched ? t.z : 0));
+                    const int wz = g.w_z + (EPI == PRE_OPROJ_SPD ? pass : (EPI == PRE_GATEUP ? (t.z + g.w_rot) % g.batches : t.z));
                     for (int kb = 0; kb < g.num_kb; ++kb, ++it) {
                         const int s = it % S;
                         if (!mbar_wait(empty_bar(s), ((it / S) & 1) ^ 1, g.err, abort_flag)) { ok = false; break; }
@@ -554,6 +592,17 @@ __global__ void __launch_bounds__(PCfg<EPI, PAIR>::THREADS_, 1) gemm_prefill_ker
                 if (EPI == PRE_QKV) epi_qkv(g, t, tacc, m, valid);
                 else if (EPI == PRE_GATEUP) epi_gateup(g, t, tacc, m, valid);
                 else if (EPI == PRE_RESID) epi_resid(g, t, tacc, m, valid);
+                else if (EPI == PRE_SCATTER) {
+                    epi_scatter(g, t, tacc, m, valid, quarter * 32 + lane);
+                    // every row of the tile is on its way: the release below orders them (made visible to the
+                    // publishing thread by the barrier) before the flag
+                    epi_sync<32 * C::EPI_WARPS>();
+                    if (threadIdx.x == 0 && t.m0 < g.t_rows) { // (a pair's second block may lie wholly past the last token: nobody owns that tile)
+                        const int tile128 = t.m0 / BM, owner = tile128 % g.sc.T, slot = tile128 / g.sc.T;
+                        unsigned *flag = g.sc.flags[owner] + ((long)slot * g.sc.n_tiles + t.nt) * g.sc.T + g.sc.me;
+                        asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(flag), "r"(*g.sc.step) : "memory");
+                    }
+                }
                 else if (g.norm_only) {
                     const float ssq = epi_row_sumsq(g, t, tacc, half);
                     if (valid) g.ss_out[((long)(t.nt * 2 + half) * g.batches + pass) * g.Mcap + m] = ssq;
@@ -613,6 +662,7 @@ __global__ void __launch_bounds__(256) prefill_prologue_kernel(PrologueArgs a)
     pdl_launch_dependents();
     if (threadIdx.x == 0) stamp_entry(a.stamp);
     pdl_wait();
+    if (a.step && blockIdx.x == 0 && threadIdx.x == 0) *a.step += 1u; // rank mode: the rank's step number advances with every launch sequence
     __shared__ float red[8];
     const int m = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     float sq = 0.f;
@@ -651,7 +701,8 @@ cudaError_t launch_gemm_prefill(PreEpilogue epi, const TcMap *const *weights, co
     if (g.t_rows <= 0) return cudaSuccess;
     if (g.num_kb < 1 || g.batches < 1 || g.batches > 8) return cudaErrorInvalidValue;
     if (epi == PRE_QKV && (256 % g.head_dim || g.head_dim < 32)) return cudaErrorInvalidValue;
-    if ((epi == PRE_RESID || epi == PRE_OPROJ_SPD) && g.H % 16) return cudaErrorInvalidValue;
+    if ((epi == PRE_RESID || epi == PRE_OPROJ_SPD || epi == PRE_SCATTER) && g.H % 16) return cudaErrorInvalidValue;
+    if (epi == PRE_SCATTER && (!g.pair || g.sc.T < 1 || g.sc.T > TP_MAX_RANKS || !g.sc.step)) return cudaErrorInvalidValue;
     if (epi == PRE_OPROJ_SPD && !g.norm_only && (!g.gain || !g.hg || !g.res_out)) return cudaErrorInvalidValue;
     if (epi == PRE_OPROJ_SPD && g.norm_only && !g.ss_out) return cudaErrorInvalidValue;
     if (g.w_rot < 0 || g.w_rot >= g.batches) return cudaErrorInvalidValue;
@@ -686,6 +737,9 @@ cudaError_t launch_gemm_prefill(PreEpilogue epi, const TcMap *const *weights, co
         L.n_tiles = (g.H + 127) / 128;
         L.passes = g.batches;
         return pair ? launch_epi<PRE_OPROJ_SPD, 1>(tw, *(const CUtensorMap *)&tokens, L, st) : launch_epi<PRE_OPROJ_SPD, 0>(tw, *(const CUtensorMap *)&tokens, L, st);
+    case PRE_SCATTER:
+        L.n_tiles = (g.H + 255) / 256;
+        return launch_epi<PRE_SCATTER, 1>(tw, *(const CUtensorMap *)&tokens, L, st);
     default:
         L.n_tiles = (g.H + 255) / 256;
         return pair ? launch_epi<PRE_RESID, 1>(tw, *(const CUtensorMap *)&tokens, L, st) : launch_epi<PRE_RESID, 0>(tw, *(const CUtensorMap *)&tokens, L, st);

@@ -13,6 +13,22 @@ enum PreEpilogue {
     PRE_RESID = 1,     // sync o_proj (a5-a7) and down (a9, a10): residual add, next norm's input and sums of squares
     PRE_GATEUP = 2,    // a8: rstd (per emulated device in an SPD block), SwiGLU
     PRE_OPROJ_SPD = 3, // a5-a7 of an SPD block: the T K-slices of one output tile in turn, R_i = X + Y_i kept apart
+    PRE_SCATTER = 4,   // rank mode: the rank's partial rows of a row-split projection go to the ranks that own them
+};
+
+// Rank mode (one shard per rank, Sec. 3), prompts: the shard sums a block keeps are two-shot exchanges.  Shot one
+// (PRE_SCATTER, the tail of the projection that produces the partial): the 128-token tiles of a launch are dealt
+// round-robin to the ranks (tile i belongs to rank i % T); a block stores its fp32 partial rows of tile i into the
+// owner's receive plane [source = own rank][slot = i / T][128 rows][H] with plain peer stores and then publishes the
+// step number in the owner's flag word [slot][column tile][source].  Shot two is the finishing kernel of tp_prefill.cu.
+struct TpScatter {
+    int T, me;                     // group size; this rank
+    int n_tiles;                   // column tiles of the launch (flag words per slot and source)
+    long src_stride;               // bytes between the source planes of a receive buffer
+    char *rx[TP_MAX_RANKS];        // rank j's receive buffer of this exchange
+    unsigned *flags[TP_MAX_RANKS]; // rank j's scatter flags of this exchange: [slot][column tile][source]
+    const float *addend;           // fp32 [tokens][H] added to the partial before it leaves (Y_r of an SPD block), or null
+    const unsigned *step;          // this rank's step number (> 0, the same on all ranks)
 };
 
 struct PreGemmArgs {
@@ -58,6 +74,12 @@ struct PreGemmArgs {
     // of the tile's weight rows.  The weight maps must then have boxes of HALF the tile's rows: 128 (QKV, RESID,
     // GATEUP: gate rows in one CTA, up rows in the other), 64 (OPROJ_SPD).  Not with norm_only.
     int pair;
+    // rank mode: fixed batch coordinate of the weight and of the token map (the rank's shard / the rank's plane)
+    int w_z, t_z;
+    int q_head0, kv_head0; // QKV: first query / KV head of the rank in q_out and in the pages
+    int act_col0;          // GATEUP: first column of the rank's slice in act
+    float *ysave;          // RESID: fp32 [tokens][H] copy of the projection's output (Y_r of an SPD block), or null
+    TpScatter sc;          // SCATTER
     int group_m;         // token tiles per group of the tile order; 0 = default (8 pair tiles / 16 single tiles = 2048 tokens)
 };
 

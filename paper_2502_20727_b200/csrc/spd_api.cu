@@ -5,6 +5,7 @@
 #include "gemm_tc.cuh"
 #include "gemm_decode.cuh"
 #include "gemm_prefill.cuh"
+#include "tp_prefill.cuh"
 
 #include <math.h>
 #include <new>
@@ -86,10 +87,16 @@ struct GraphEntry { GraphKey key; cudaGraphExec_t exec; unsigned long long last_
 // One rank's region of a tensor-parallel group (offsets in bytes; every rank uses the same layout).
 struct TpLayout {
     size_t flags, rx, res0, res1, ysave, hg, ss_attn, ss_mlp, step, total;
-    size_t site_flags; // flag words of one (layer, exchange site)
+    size_t site_flags; // flag words of one (layer, exchange site) of the decode step's one-shot exchange
     size_t buf_bytes, src_bytes;
-    long Mb;           // token capacity (max_batch)
+    long Mb;           // token capacity of the residual / operand / sums planes: a decode batch or a prompt chunk
+    long Md;           // token capacity of the decode step's receive planes (max_batch)
     int tok_tiles;
+    // prompts: two-shot exchange over 128-token tiles dealt round-robin to the ranks
+    size_t rs_rx, sflags, gflags;       // receive buffers (two), scatter flags, gather flags
+    size_t rs_src_stride, rs_buf_bytes; // one source plane ([slot][128][H] fp32); one receive buffer (T source planes)
+    size_t sflag_words, gflag_words;    // flag words of one (layer, exchange site)
+    int slots_cap, n_tiles;             // 128-token tiles a rank can own per launch; 256-column tiles of H
 };
 
 struct TpState {
@@ -100,7 +107,7 @@ struct TpState {
     TpLayout L;
     char *regions[TP_MAX_RANKS];
     std::vector<TcMap> qkv_maps; // per layer: wq, wk, wv with one batch per local shard
-    TcMap h_maps[3];             // the local ranks' gain-scaled inputs, token boxes 16 / 32 / 64
+    TcMap h_maps[4];             // the local ranks' gain-scaled inputs, token boxes 16 / 32 / 64 / 128
 };
 
 struct Ctx {
@@ -377,21 +384,33 @@ TpLayout tp_layout(const spd_dims &d, int T)
 {
     TpLayout L{};
     const size_t H = d.hidden, h_tiles = (H + 127) / 128;
-    // token capacity: a decode batch, or a prompt chunk of up to 512 tokens
-    const long chunk = d.max_prefill_tokens < 512 ? d.max_prefill_tokens : 512;
+    // rows: a decode batch, or a prompt chunk of up to 2048 tokens
+    const long chunk = d.max_prefill_tokens < 2048 ? d.max_prefill_tokens : 2048;
     L.Mb = d.max_batch > chunk ? d.max_batch : chunk;
-    L.tok_tiles = (int)((L.Mb + 15) / 16); // an upper bound for every token box
+    L.Md = d.max_batch;
+    L.tok_tiles = (int)((L.Md + 15) / 16); // an upper bound for every token box
     L.site_flags = h_tiles * L.tok_tiles * T * TP_FLAG_RANGES;
-    L.src_bytes = (size_t)L.Mb * H * 4;
+    L.src_bytes = (size_t)L.Md * H * 4;
     L.buf_bytes = L.src_bytes * T;
+    const size_t plane = (size_t)L.Mb * H * 4;
+    const int m128_cap = (int)((L.Mb + 127) / 128);
+    L.slots_cap = (m128_cap + T - 1) / T;
+    L.n_tiles = (int)((H + 255) / 256);
+    L.rs_src_stride = (size_t)L.slots_cap * 128 * H * 4;
+    L.rs_buf_bytes = L.rs_src_stride * T;
+    L.sflag_words = (size_t)L.slots_cap * L.n_tiles * T;
+    L.gflag_words = (size_t)m128_cap * tp_finish_blocks_per_tile();
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
     L.step = take(256);
     L.flags = take((size_t)d.n_layers * 2 * L.site_flags * 4);
+    L.sflags = take((size_t)d.n_layers * 2 * L.sflag_words * 4);
+    L.gflags = take((size_t)d.n_layers * 2 * L.gflag_words * 4);
     L.rx = take(2 * L.buf_bytes);
-    L.res0 = take(L.src_bytes);
-    L.res1 = take(L.src_bytes);
-    L.ysave = take(L.src_bytes);
+    L.rs_rx = take(2 * L.rs_buf_bytes);
+    L.res0 = take(plane);
+    L.res1 = take(plane);
+    L.ysave = take(plane);
     L.hg = take((size_t)L.Mb * H * 2);
     L.ss_attn = take(h_tiles * L.Mb * 4);
     L.ss_mlp = take(h_tiles * L.Mb * 4);
@@ -860,7 +879,7 @@ int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, 
     PageTable pt{bt, max_pages, c->n_pages, d.kv_block_size, d.n_kv_heads};
     const int tbox = tc_token_box(true, M);
     const int tok_tiles = cdiv(M, tbox), h_tiles = cdiv(H, 128);
-    if (tok_tiles > TL.tok_tiles || M > TL.Mb) return SPD_EINVAL;
+    if (tok_tiles > TL.tok_tiles || M > TL.Md) return SPD_EINVAL;
     const TcMap *hmap = &tp.h_maps[box_index(tbox)];
     int launches = 0;
     const bool rope = d.rope_base > 0.f;
@@ -965,6 +984,154 @@ int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, 
             LAUNCH_S(K_DOWN, g, launch_gemm_decode(EPI_RESID_TP, wmaps, *am, g, st));
         }
     }
+    c->launches_last = launches;
+    return SPD_OK;
+}
+
+// A prompt chunk of M tokens in rank mode at tensor-core speed: every local rank runs the prompt projections
+// (gemm_prefill.cu, CTA pairs) on its own shard and its own copy of the residual stream; the shard sums the
+// block keeps are two-shot exchanges - the projection's tail scatters the rank's partial rows to the ranks that
+// own them (128-token tiles dealt round-robin), the owner adds the T planes in rank order, applies the residual
+// and writes the finished rows into every rank's planes, and a small kernel waits for all owners before the next
+// projection starts (tp_prefill.cu).  A TP block exchanges Y_r after o_proj and Z_r after down (Sec. 3), an SPD
+// block keeps R_r = X + Y_r on the rank and exchanges Y_r + Z_r after down (Sec. 4.1.1).  With several local
+// ranks (all ranks on one GPU) every kernel is launched once per rank, all scatters before any finish: no
+// kernel then waits for one launched after it.
+int run_tp_prefill(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, const int32_t *bt, int max_pages,
+                   int max_context, cudaStream_t st)
+{
+    const spd_dims &d = c->d;
+    TpState &tp = c->tp;
+    const TpLayout &TL = tp.L;
+    const int H = d.hidden, qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, F = d.ffn, nl = d.T;
+    const int qd_r = qd / nl, kd_r = kd / nl, Fs = F / nl;
+    const long Mb = TL.Mb;
+    if (M > Mb) return SPD_EINVAL;
+    PageTable pt{bt, max_pages, c->n_pages, d.kv_block_size, d.n_kv_heads};
+    int launches = 0;
+    const bool rope = d.rope_base > 0.f;
+    const TcMap *hmap = &tp.h_maps[3]; // 128-token boxes
+    auto reg = [&](int z) { return tp.regions[tp.rank_base + z]; };
+    const unsigned long long wait_ns = (unsigned long long)c->peer_wait_ms * 1000000ull;
+    if (rope) LAUNCH(K_ROPE_TABLE, launch_rope_table(c->rope, tm, M, d.head_dim, d.rope_base, st, next_stamp(c, K_ROPE_TABLE)));
+    for (int z = 0; z < nl; ++z) {   // a1 of the first block; the rank's step number advances
+        PrologueArgs a{};
+        a.x = x; a.res_out = (float *)(reg(z) + TL.res0); a.gain = c->layers[0].attn_norm; a.hg = reg(z) + TL.hg;
+        a.ss_out = (float *)(reg(z) + TL.ss_attn); a.Mcap = Mb; a.M = M; a.H = H; a.step = (unsigned *)(reg(z) + TL.step);
+        LAUNCH_S(K_NORM, a, launch_prefill_prologue(a, st));
+    }
+    auto base_args = [&](int z) {
+        PreGemmArgs g{};
+        g.t_rows = M; g.err = c->err; g.H = H; g.Mcap = Mb; g.batches = 1; g.n_weights = 1; g.pair = 1;
+        g.group_m = c->prefill_group_m; g.w_z = z; g.t_z = z;
+        return g;
+    };
+    int exchange = 0;
+    // the exchange of block l at site s (0: o_proj, 1: down): scatter by every local rank, then finish, then wait
+    auto scatter_args = [&](PreGemmArgs &g, int z, int l, int s, int buf, const float *addend) {
+        g.sc.T = tp.T; g.sc.me = tp.rank_base + z; g.sc.n_tiles = TL.n_tiles; g.sc.src_stride = (long)TL.rs_src_stride;
+        for (int j = 0; j < tp.T; ++j) {
+            g.sc.rx[j] = tp.regions[j] + TL.rs_rx + (size_t)buf * TL.rs_buf_bytes;
+            g.sc.flags[j] = (unsigned *)(tp.regions[j] + TL.sflags) + ((size_t)l * 2 + s) * TL.sflag_words;
+        }
+        g.sc.addend = addend;
+        g.sc.step = (const unsigned *)(reg(z) + TL.step);
+    };
+    auto finish_and_wait = [&](int l, int s, int buf, size_t res_in_off, size_t res_out_off, const void *gain, size_t ss_off) -> int {
+        const size_t goff = TL.gflags + (((size_t)l * 2 + s) * TL.gflag_words) * 4;
+        for (int z = 0; z < nl; ++z) {
+            TpFinishArgs a{};
+            a.T = tp.T; a.me = tp.rank_base + z; a.M = M; a.H = H; a.n_tiles = TL.n_tiles;
+            a.rx = reg(z) + TL.rs_rx + (size_t)buf * TL.rs_buf_bytes; a.src_stride = (long)TL.rs_src_stride;
+            a.sflags = (const unsigned *)(reg(z) + TL.sflags) + ((size_t)l * 2 + s) * TL.sflag_words;
+            a.step = (const unsigned *)(reg(z) + TL.step);
+            a.res_in = (const float *)(reg(z) + res_in_off); a.gain = gain;
+            for (int j = 0; j < tp.T; ++j) a.region[j] = tp.regions[j];
+            a.off_res_out = (long)res_out_off; a.off_hg = (long)TL.hg; a.off_ss = (long)ss_off; a.off_gflags = (long)goff;
+            a.wait_ns = wait_ns; a.err = c->err;
+            LAUNCH_S(K_NORM, a, launch_tp_finish(a, st));
+        }
+        for (int z = 0; z < nl; ++z)
+            LAUNCH(K_NORM, launch_tp_gather_wait((const unsigned *)(reg(z) + goff), M, (const unsigned *)(reg(z) + TL.step), wait_ns, c->err, st));
+        return SPD_OK;
+    };
+    for (int l = 0; l < d.n_layers; ++l) {
+        const spd_layer &w = c->layers[l];
+        const LayerMaps &lm = c->maps[l];
+        const bool sync = c->mask[l] != 0;
+        int rc;
+        for (int z = 0; z < nl; ++z) {   // a2 + a3: rank z projects its own heads from its own copy of the normalised input
+            PreGemmArgs g = base_args(z);
+            const TcMap *wmaps[3] = {&tp.qkv_maps[3 * l], &tp.qkv_maps[3 * l + 1], &tp.qkv_maps[3 * l + 2]};
+            g.n_weights = 3; g.w_rows[0] = qd_r; g.w_rows[1] = g.w_rows[2] = kd_r;
+            g.num_kb = cdiv(H, 64);
+            g.ss_in = SumSq{(const float *)(reg(z) + TL.ss_attn), 1, 1, Mb, H, d.rms_eps};
+            g.rope = rope ? c->rope : nullptr; g.q_out = c->q; g.k_pages = w.k_pages; g.v_pages = w.v_pages; g.pt = pt; g.tm = tm;
+            g.n_q_heads = d.n_q_heads; g.head_dim = d.head_dim;
+            g.q_head0 = z * (d.n_q_heads / nl); g.kv_head0 = z * (d.n_kv_heads / nl);
+            LAUNCH_S(K_QKV, g, launch_gemm_prefill(PRE_QKV, wmaps, *hmap, g, st));
+        }
+        {   // a4: heads are rank-local by construction
+            AttnArgs a{};
+            a.q = c->q; a.k_pages = w.k_pages; a.v_pages = w.v_pages; a.pt = pt; a.tm = tm; a.out = c->attn;
+            a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.B = M; a.splits = 1;
+            a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.counters = c->attn_cnt; a.err = c->err;
+            if (d.head_dim == 128 && d.kv_block_size == 16) {
+                MAP_OR_FAIL(qm, act_map(c, AB_Q, 128));
+                a.q_map = qm; a.k_map = &lm.kpages; a.v_map = &lm.vpages; a.rescale_log2 = (float)c->prefill_rescale_log2;
+            }
+            LAUNCH_S(K_ATTN, a, launch_prefill_attention<bf16>(a, st));
+        }
+        int mlp_tiles = 1;
+        MAP_OR_FAIL(attn_map, act_map(c, AB_ATTN_SHARD, 128));
+        if (sync) {   // a5 - a7, TP block: sync-point 1 = exchange of Y_r; R = X + sum over ranks
+            const int buf = (int)((tp.exchanges + exchange++) & 1);
+            for (int z = 0; z < nl; ++z) {
+                PreGemmArgs g = base_args(z);
+                const TcMap *wmaps[1] = {&lm.wo_shard};
+                g.w_rows[0] = H; g.num_kb = cdiv(qd_r, 64);
+                scatter_args(g, z, l, 0, buf, nullptr);
+                LAUNCH_S(K_OPROJ, g, launch_gemm_prefill(PRE_SCATTER, wmaps, *attn_map, g, st));
+            }
+            if ((rc = finish_and_wait(l, 0, buf, TL.res0, TL.res1, w.mlp_norm, TL.ss_mlp)) != SPD_OK) return rc;
+        } else {      // SPD block: the sync-point is dropped, R_r = X + Y_r feeds the rank's MLP and Y_r is kept for a10
+            for (int z = 0; z < nl; ++z) {
+                PreGemmArgs g = base_args(z);
+                const TcMap *wmaps[1] = {&lm.wo_shard};
+                g.w_rows[0] = H; g.num_kb = cdiv(qd_r, 64);
+                g.res_in = (const float *)(reg(z) + TL.res0); g.res_out = (float *)(reg(z) + TL.res1); g.gain = w.mlp_norm;
+                g.hg = reg(z) + TL.hg; g.hg_stride = Mb * H; g.ss_out = (float *)(reg(z) + TL.ss_mlp);
+                g.ysave = (float *)(reg(z) + TL.ysave);
+                LAUNCH_S(K_OPROJ, g, launch_gemm_prefill(PRE_RESID, wmaps, *attn_map, g, st));
+            }
+            mlp_tiles = pre_ss_tiles(PRE_RESID, H);
+        }
+        for (int z = 0; z < nl; ++z) {   // a8 on the rank's MLP slice
+            PreGemmArgs g = base_args(z);
+            const TcMap *wmaps[2] = {&lm.w_gate, &lm.w_up};
+            g.n_weights = 2; g.w_rows[0] = g.w_rows[1] = Fs;
+            g.num_kb = cdiv(H, 64);
+            g.ss_in = SumSq{(const float *)(reg(z) + TL.ss_mlp), mlp_tiles, 1, Mb, H, d.rms_eps};
+            g.act = c->act; g.F = F; g.Fs = Fs; g.act_col0 = z * Fs;
+            LAUNCH_S(K_GATE_UP, g, launch_gemm_prefill(PRE_GATEUP, wmaps, *hmap, g, st));
+        }
+        {   // a9 + a10, the kept sync-point.  TP block: out = R + sum_r Z_r;  SPD block: out = X + sum_r (Y_r + Z_r)
+            MAP_OR_FAIL(act_shard, act_map(c, AB_ACT_SHARD, 128));
+            const int buf = (int)((tp.exchanges + exchange++) & 1);
+            for (int z = 0; z < nl; ++z) {
+                PreGemmArgs g = base_args(z);
+                const TcMap *wmaps[1] = {&lm.wd_shard};
+                g.w_rows[0] = H; g.num_kb = cdiv(Fs, 64);
+                scatter_args(g, z, l, 1, buf, sync ? nullptr : (const float *)(reg(z) + TL.ysave));
+                LAUNCH_S(K_DOWN, g, launch_gemm_prefill(PRE_SCATTER, wmaps, *act_shard, g, st));
+            }
+            const void *gain = l + 1 < d.n_layers ? c->layers[l + 1].attn_norm : nullptr; // last block: the bf16 copy is the output
+            if ((rc = finish_and_wait(l, 1, buf, sync ? TL.res1 : TL.res0, TL.res0, gain, TL.ss_attn)) != SPD_OK) return rc;
+        }
+    }
+    // the last block's bf16 rows lie in every rank's operand plane: hand each local rank's copy to the caller
+    for (int z = 0; z < nl; ++z)
+        CU_TRY(cudaMemcpyAsync((char *)out + (long)z * out_stride, reg(z) + TL.hg, (size_t)M * H * 2, cudaMemcpyDeviceToDevice, st));
     c->launches_last = launches;
     return SPD_OK;
 }
@@ -1588,8 +1755,8 @@ int spd_tp_attach(spd_ctx *ctx, int32_t T, int32_t rank_base, void *const *regio
         rc |= make_operand_map(&tp.qkv_maps[3 * l + 1], w.wk, H, kd / nl, nl, H, (kd / nl) * H, 128);
         rc |= make_operand_map(&tp.qkv_maps[3 * l + 2], w.wv, H, kd / nl, nl, H, (kd / nl) * H, 128);
     }
-    const int boxes[3] = {16, 32, 64};
-    for (int i = 0; i < 3; ++i)
+    const int boxes[4] = {16, 32, 64, 128};
+    for (int i = 0; i < 4; ++i)
         rc |= make_operand_map(&tp.h_maps[i], tp.regions[rank_base] + TL.hg, H, TL.Mb, nl, H, nl > 1 ? z_stride / 2 : TL.Mb * H, boxes[i]);
     if (rc) return SPD_EINVAL;
     // the local ranks' regions start from zero: step 0, no flag set, token rows beyond a batch read as zero
@@ -1616,20 +1783,16 @@ int spd_tp_prefill(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int3
     if (B < 1 || S < 1 || B > d.max_batch || x == out) return SPD_EINVAL;
     if (S > d.max_seq_len || (long)max_pages * d.kv_block_size < S) return SPD_ECAPACITY;
     cudaStream_t st = (cudaStream_t)stream;
-    // Tokens per launch: the region's capacity; with several ranks in one launch also what keeps every thread
-    // block of an exchange launch resident (three blocks per SM, one block per 128 columns, rank and 64 tokens).
-    long chunk = c.tp.L.Mb;
-    if (d.T > 1) {
-        const long tiles = (long)cdiv(d.hidden, 128) * d.T, fit = (3L * sm_count()) / tiles;
-        if (fit < 1) { g_last_cuda_error = (int)cudaErrorCooperativeLaunchTooLarge; return SPD_ECUDA; }
-        if (fit * 64 < chunk) chunk = fit * 64;
-    }
+    // tokens per launch: the capacity of the ranks' planes and of the shared activation buffers
+    long chunk = c.tp.L.Mb < c.Mcap ? c.tp.L.Mb : c.Mcap;
+    if (chunk > d.max_prefill_tokens) chunk = d.max_prefill_tokens;
+    CU_TRY(timeline_restart(&c, st));
     const long rank_stride = (long)B * S * d.hidden * 2;
     int total_launches = 0;
     auto run = [&](int b0, int nb, int s0, int ns) -> int {
         TokMap tm{0, b0, ns, s0, nullptr};
         const size_t off = ((size_t)b0 * S + s0) * d.hidden * 2;
-        const int rc = run_tp(&c, (const char *)x + off, (char *)out + off, rank_stride, nb * ns, tm, block_table, max_pages, false, S, st);
+        const int rc = run_tp_prefill(&c, (const char *)x + off, (char *)out + off, rank_stride, nb * ns, tm, block_table, max_pages, S, st);
         if (rc == SPD_OK) {
             for (int l = 0; l < d.n_layers; ++l) c.tp.exchanges += c.mask[l] ? 2 : 1;
             total_launches += c.launches_last;
@@ -1650,6 +1813,7 @@ int spd_tp_prefill(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int3
             }
     }
     c.launches_last = total_launches;
+    CU_TRY(timeline_fold(&c, st));
     return SPD_OK;
 }
 

@@ -226,3 +226,26 @@ def test_a_launch_whose_ranks_cannot_all_be_resident_is_refused():
     p.stack.tp_detach()
     assert p.stack.device_error() == 0
     p.stack.close()
+
+
+@pytest.mark.parametrize("T,mask,B,S,chunk", [(4, (1, 0, 1), 2, 300, 4096), (2, (0, 0), 3, 200, 256), (8, (1,), 1, 130, 4096)])
+def test_rank_mode_prompts_over_many_tiles(T, mask, B, S, chunk):
+    """Prompts at tensor-core speed in rank mode: the prompt projections on CTA pairs per rank, the kept shard sums as
+    two-shot exchanges over 128-token tiles dealt round-robin to the ranks.  600 tokens = five tiles for four ranks (one
+    rank owns two); chunks of 256 tokens cut prompts inside the sequence; 130 tokens for 8 ranks leave six ranks without
+    a tile.  Every rank against the oracle, ranks bit-identical, then decode steps on the caches."""
+    w = si.Workload("tp_fast", "bf16", len(mask), 512, 8, 8, 64, 1024, T, mask, B, S, 2)
+    p = Pair(w, mask=mask, B=B, max_len=S + 2, max_prefill_tokens=chunk)
+    p.stack.tp_attach_local()
+    torch.cuda.synchronize()
+    got, ref, _ = p.tp_prefill(S)
+    for r in range(T):
+        e = rel_err(got[r], ref)
+        assert e <= TOL["bf16"], f"prompt, rank {r}: rel err {e}"
+        assert np.array_equal(got[r], got[0])
+    for t in range(2):
+        got, ref = p.tp_decode(t)
+        for r in range(T):
+            assert rel_err(got[r], ref) <= TOL["bf16"]
+    assert p.stack.device_error() == 0
+    p.stack.close()
