@@ -259,14 +259,19 @@ class Run:
         """The configuration's prompt phase (Bp prompts of Sp tokens), median of `reps` after one warm-up."""
         w = self.w
         xp = si.make_hidden(w, (self.Bp, self.Sp, w.hidden), self.dev, 0, 0)
-        outp = torch.empty_like(xp)
-        self.stack.prefill(xp, self.bt_p, outp)
+        if self.rank_mode:  # every rank's copy of the output; prompts through the two-shot exchanges
+            outp = torch.empty((w.T,) + tuple(xp.shape), dtype=xp.dtype, device=self.dev)
+            prefill = self.stack.tp_prefill
+        else:
+            outp = torch.empty_like(xp)
+            prefill = self.stack.prefill
+        prefill(xp, self.bt_p, outp)
         torch.cuda.synchronize()
         ms = []
         for _ in range(reps):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            self.stack.prefill(xp, self.bt_p, outp)
+            prefill(xp, self.bt_p, outp)
             e1.record()
             torch.cuda.synchronize()
             ms.append(e0.elapsed_time(e1))

@@ -322,13 +322,18 @@ int spd_tp_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *se
                        const int32_t *block_table, int32_t max_pages, int32_t max_context, void *out,
                        void *stream);
 
-/* Prompt processing of an attached context (same arguments as spd_prefill, same collective
- * rules as spd_tp_decode_step): the prompts go through the rank-mode step in chunks of at most
- * 512 tokens (fewer when several ranks share one launch: all thread blocks of an exchange launch
- * must be resident), every chunk attending to the cached positions before it.  The projections
- * are the weight-streaming kernels of the decode step with 64-token tiles - functionally the
- * block of Sec. 3 / Sec. 4.1.1 for any number of tokens, not a throughput path.
+/* Prompt processing of an attached context (same arguments as spd_prefill, same collective rules as
+ * spd_tp_decode_step), at tensor-core speed: every rank runs the prompt projections on its own shard, and every
+ * shard sum the block keeps is a two-shot exchange.  Shot one is the tail of the projection that produces the
+ * partial: the 128-token tiles of a launch are dealt round-robin to the ranks, and each rank stores its fp32
+ * partial rows of a tile into the owner's receive plane (plain peer stores) and publishes the step number in the
+ * owner's flags.  Shot two: the owner adds the T planes in rank order (all ranks end up with the same bits), adds
+ * the residual and writes the finished rows - residual stream, operand of the next projection, sums of squares -
+ * into every rank's planes; a small kernel on each rank waits for all owners before the next projection starts.
+ * A TP block exchanges Y_r and Z_r (Sec. 3), an SPD block only Y_r + Z_r (Sec. 4.1.1).  Prompts go in chunks of
+ * at most min(max_prefill_tokens, 2048) tokens, every chunk attending to the cached positions before it.
  *   out : [ranks held by the context][B][S][hidden] bf16
+ * Waits for peers are bounded as in spd_tp_decode_step (error bit 8, "peer_wait_ms").
  * Errors: SPD_ENULL, SPD_EINVAL (not attached, B > max_batch), SPD_ECAPACITY, SPD_ECUDA. */
 int spd_tp_prefill(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int32_t *block_table,
                    int32_t max_pages, void *out, void *stream);

@@ -260,6 +260,12 @@ def permute_layer(lw: Dict[str, torch.Tensor], *, n_q_heads: int, n_kv_heads: in
     return out
 
 
+def tp_tile_owner(tile: int, T: int):
+    """Rank-mode prompts: (owner rank, slot in the owner's receive planes) of the 128-token tile `tile` of a launch -
+    tiles are dealt round-robin, so tile i is summed and redistributed by rank i % T (spd_tp_prefill)."""
+    return tile % T, tile // T
+
+
 def shard_layer(lw: Dict[str, torch.Tensor], r: int, T: int) -> Dict[str, torch.Tensor]:
     """The tensors rank r of a T-GPU group holds of one LLaMA-style layer (Sec. 3): rows r of the
     column-parallel matrices, columns r of the row-parallel ones (as contiguous matrices), the norm gains whole."""

@@ -861,14 +861,14 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
     return SPD_OK;
 }
 
-// M tokens (one decode step, or a prompt chunk) in rank mode (tensor parallelism across GPUs, Sec. 3):
-// every local rank runs the block on its own shard and its own copy of the residual stream; the shard
-// sums that the block keeps (o_proj of a TP block, down of every block; Sec. 4.1.1) are exchanges with
-// the other ranks of the group inside the projection's tail.  out: rank z's [M][H] rows lie out_stride
-// bytes after rank z-1's.  Prompt chunks go through the same weight-streaming kernels, 64 tokens per tile.
+// One decode step of M tokens in rank mode (tensor parallelism across GPUs, Sec. 3): every local rank runs
+// the block on its own shard and its own copy of the residual stream; the shard sums that the block keeps
+// (o_proj of a TP block, down of every block; Sec. 4.1.1) are one-shot exchanges with the other ranks of the
+// group inside the projection's tail.  out: rank z's [M][H] rows lie out_stride bytes after rank z-1's.
 int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, const int32_t *bt, int max_pages,
-           bool decode, int max_context, cudaStream_t st)
+           int max_context, cudaStream_t st)
 {
+    constexpr bool decode = true;
     const spd_dims &d = c->d;
     TpState &tp = c->tp;
     const TpLayout &TL = tp.L;
@@ -934,15 +934,7 @@ int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, 
             a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.B = M; a.splits = p.attn_splits;
             a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.counters = c->attn_cnt; a.err = c->err;
             if (d.head_dim == 128 && d.kv_block_size == 16) { a.k_map = &c->maps[l].kpages; a.v_map = &c->maps[l].vpages; }
-            if (decode) LAUNCH_S(K_ATTN, a, launch_decode_attention<bf16>(a, st));
-            else {
-                a.splits = 1;
-                if (a.k_map) {
-                    MAP_OR_FAIL(qm, act_map(c, AB_Q, 128));
-                    a.q_map = qm; a.rescale_log2 = (float)c->prefill_rescale_log2;
-                }
-                LAUNCH_S(K_ATTN, a, launch_prefill_attention<bf16>(a, st));
-            }
+            LAUNCH_S(K_ATTN, a, launch_decode_attention<bf16>(a, st));
         }
         {   // a5 - a7: Y_z from the rank's own heads.  TP block: R = X + sum over ranks (sync-point 1);
             // SPD block: the sync-point is dropped, R_z = X + Y_z feeds the rank's MLP and Y_z is kept for a10
@@ -1836,7 +1828,7 @@ int spd_tp_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *se
     const GraphKey key{x, seq_lens, block_table, out, B, max_pages, ctx_bucket, 1 + (int)(c.tp.exchanges & 1)};
     const int rc = replay_or_run(c, key, [&]() {
         CU_TRY(timeline_restart(&c, st));
-        const int rc2 = run_tp(&c, x, out, (long)B * d.hidden * 2, B, tm, block_table, max_pages, true, ctx_bucket, st);
+        const int rc2 = run_tp(&c, x, out, (long)B * d.hidden * 2, B, tm, block_table, max_pages, ctx_bucket, st);
         if (rc2 != SPD_OK) return rc2;
         CU_TRY(timeline_fold(&c, st));
         return SPD_OK;

@@ -85,3 +85,18 @@ def test_spawned_ranks_form_a_group_and_a_failing_rank_fails_the_job():
         env.pop(k, None)
     assert bench.spawn_ranks(2, [sys.executable, os.path.join(ROOT, "tests", "rank_worker.py")], env=env, timeout=600) == 0
     assert bench.spawn_ranks(2, [sys.executable, "-c", "import os, sys; sys.exit(3 if os.environ['RANK'] == '1' else 0)"], env=env) == 3
+
+
+def test_two_shot_exchange_index_logic_over_gloo_ranks():
+    """The prompt exchange of the rank mode on CPU ranks: 128-token tiles dealt round-robin (tile i -> rank i % T, slot
+    i // T), partial rows sent to the owner, summed there in rank order, finished rows sent to everyone.  The result is
+    the all-reduce, every (owner, slot) is hit exactly once, and the owner's receive planes hold (tiles it owns) x T
+    source planes - the counts the device-side flags are sized by."""
+    out = torchrun([os.path.join(ROOT, "tests", "tp_two_shot_worker.py")], n=3)
+    lines = [l for l in out.splitlines() if l.startswith("WORKER ")]
+    assert len(lines) == 1
+    res = json.loads(lines[0][7:])
+    assert res["world"] == 3 and res["tiles"] == 5
+    assert res["max_err"] == 0.0                      # same sums in the same (rank) order on every rank
+    assert res["owned"] == [2, 2, 1]                  # tiles 0,3 | 1,4 | 2
+    assert res["planes_received"] == [6, 6, 3]        # owned tiles x T sources

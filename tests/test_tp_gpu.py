@@ -249,3 +249,36 @@ def test_rank_mode_prompts_over_many_tiles(T, mask, B, S, chunk):
             assert rel_err(got[r], ref) <= TOL["bf16"]
     assert p.stack.device_error() == 0
     p.stack.close()
+
+
+def test_a_prompt_whose_peer_never_runs_is_reported_not_waited_for():
+    """Rank 0 of a group of two, its peer absent: the owner's wait for the peer's partial rows and the wait for the
+    peer's finished tile both run out (20 ms each), the call returns, error bit 8 is set, the context stays usable."""
+    import paper_2502_20727_b200 as spd
+    mask = (1,)
+    full = si.Workload("tp_alone_p", "bf16", 1, 256, 4, 4, 64, 512, 2, mask, 1, 200, 0)
+    layers = si.make_stack(full, "cpu", 0)
+    shard = [{n: t.to("cuda:0") for n, t in spd.shard_layer(lw, 0, 2).items()} for lw in layers]
+    one = full.with_(n_q_heads=2, n_kv_heads=2, ffn=256, T=1)
+    with torch.cuda.stream(torch.cuda.Stream(device="cuda:0")):
+        stack = spd.stack_from_workload(one, shard, sync_mask=mask, max_batch=1, max_seq_len=208, n_pages=14,
+                                        max_prefill_tokens=256, device="cuda:0")
+        nbytes = (stack.tp_region_bytes(2) + 1023) // 1024 * 1024
+        regions = torch.zeros(2 * nbytes + 1024, dtype=torch.uint8, device="cuda:0")
+        base = (regions.data_ptr() + 1023) // 1024 * 1024
+        stack.tp_attach(2, 0, [base, base + nbytes], nbytes)
+        stack.set_tuning(peer_wait_ms=20)
+        x = si.make_hidden(one, (1, 200, one.hidden), "cpu", 0, 0).to("cuda:0")
+        bt = torch.arange(13, dtype=torch.int32, device="cuda:0")[None]
+        t0 = time.perf_counter()
+        out = stack.tp_prefill(x, bt)
+        torch.cuda.synchronize()
+        waited = time.perf_counter() - t0
+        assert out.shape == (1, 1, 200, 256)
+        assert stack.device_error() & 8
+        assert waited < 1.0, f"gave up after {waited:.3f} s with a 20 ms limit"
+        stack.tp_detach()
+        y = stack.prefill(x, bt)
+        torch.cuda.synchronize()
+        assert torch.isfinite(y.float()).all() and stack.device_error() == 0
+        stack.close()
