@@ -174,6 +174,13 @@ int spd_set_graphs(spd_ctx *ctx, int32_t enabled);
  *       the token tile runs fastest, then the weight tile, so that a group's token panels stay in L2 while the
  *       weight tiles sweep past (0 = default: 2048 tokens per group; a value >= the number of token tiles gives
  *       the plain order with all token tiles fastest).  A schedule only: same results.
+ *   "bias_fused"
+ *       block with bias (Sec. 4.1.2) in bf16: 1 (default) = the same five fused projections per block as the
+ *       block without bias - LayerNorm enters the QKV and fc1 tails through two vectors per layer folded from
+ *       the weights at spd_create (sum_k g_k W_nk and sum_k beta_k W_nk + b_n) and the row mean and variance
+ *       the preceding tail left; out_proj / fc2 biases and ReLU in the tails; 0 = K-split GEMMs with separate
+ *       LayerNorm, bias and activation kernels.  The two differ in rounding only.  The fold subtracts
+ *       mean * sum_k g_k W_nk from the accumulator: rows whose mean dwarfs their spread lose that much precision.
  *   "peer_wait_ms"
  *       rank mode (spd_tp_*): milliseconds a rank waits for the other ranks' partial sums before
  *       it gives up with error bit 8 (default and value 0: 1000; at most 60000).  Always bounded.

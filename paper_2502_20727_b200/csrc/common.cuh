@@ -175,6 +175,9 @@ struct NormArgs {
 };
 template <typename T> cudaError_t launch_residual_norm(const NormArgs &a, cudaStream_t st);
 
+// wg[n] = sum_k g[k] W[n][k], wb[n] = sum_k beta[k] W[n][k] + b[n] (b may be null); W bf16 [N][K] (block with bias, Sec. 4.1.2)
+cudaError_t launch_ln_fold(const void *W, int N, int K, const void *g, const void *beta, const void *b, float *wg, float *wb, cudaStream_t st);
+
 cudaError_t launch_rope_table(float2 *table, TokMap tm, int M, int head_dim, float base, cudaStream_t st,
                               unsigned long long *stamp = nullptr);
 

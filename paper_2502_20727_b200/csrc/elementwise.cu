@@ -241,6 +241,32 @@ template <typename T> cudaError_t launch_residual_norm(const NormArgs &a, cudaSt
 template cudaError_t launch_residual_norm<float>(const NormArgs &, cudaStream_t);
 template cudaError_t launch_residual_norm<bf16>(const NormArgs &, cudaStream_t);
 
+// Block with bias: the two vectors that let a LayerNorm commute with the projection that follows it,
+// wg[n] = sum_k g[k] W[n][k] and wb[n] = sum_k beta[k] W[n][k] + b[n] (one warp per weight row, fp32 sums of the
+// exact bf16 products).  Run once per projection when the context is created.
+__global__ void __launch_bounds__(256) ln_fold_kernel(const bf16 *W, int N, int K, const bf16 *g, const bf16 *beta, const bf16 *b, float *wg,
+                                                      float *wb)
+{
+    const int n = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (n >= N) return;
+    float sg = 0.f, sb = 0.f;
+    for (int k = lane; k < K; k += 32) {
+        const float w = __bfloat162float(W[(long)n * K + k]);
+        sg = fmaf(__bfloat162float(g[k]), w, sg);
+        sb = fmaf(__bfloat162float(beta[k]), w, sb);
+    }
+    sg = warp_sum(sg);
+    sb = warp_sum(sb);
+    if (lane == 0) { wg[n] = sg; wb[n] = sb + (b ? __bfloat162float(b[n]) : 0.f); }
+}
+
+cudaError_t launch_ln_fold(const void *W, int N, int K, const void *g, const void *beta, const void *b, float *wg, float *wb, cudaStream_t st)
+{
+    if (N <= 0) return cudaSuccess;
+    ln_fold_kernel<<<(N + 7) / 8, 256, 0, st>>>((const bf16 *)W, N, K, (const bf16 *)g, (const bf16 *)beta, (const bf16 *)b, wg, wb);
+    return cudaGetLastError();
+}
+
 // cos/sin of pos * base^(-2j/d), evaluated in double once per call and shared by all layers.
 __global__ void rope_table_kernel(float2 *table, TokMap tm, int M, int half, double log_base, int d, unsigned long long *stamp)
 {

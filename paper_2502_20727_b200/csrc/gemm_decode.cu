@@ -110,20 +110,33 @@ __device__ __forceinline__ void load_partials(float4 (&y)[MAX_P], const float *S
 // rstd of the tile's tokens from the partial sums of squares, by the 128 epilogue threads:
 // thread t adds every (128/BN)-th partial of token t % BN, then the parts are added in order.
 template <int BN>
-__device__ __forceinline__ void compute_rstd(const SumSq &ss, int group, int t_row0, int t_rows, float *red, float *sm_rstd)
+__device__ __forceinline__ void compute_rstd(const SumSq &ss, int group, int t_row0, int t_rows, float *red, float *sm_rstd, float *sm_mu)
 {
     constexpr int PARTS = 128 / BN;
     const int t = threadIdx.x, j = t % BN, part = t / BN, m = t_row0 + j;
-    float acc = 0.f;
+    float acc = 0.f, sum = 0.f;
     if (m < t_rows)
-        for (int tile = part; tile < ss.tiles; tile += PARTS) acc += __ldcg(ss.part + ((long)tile * ss.groups + group) * ss.Mcap + m);
+        for (int tile = part; tile < ss.tiles; tile += PARTS) {
+            const long i = ((long)tile * ss.groups + group) * ss.Mcap + m;
+            acc += __ldcg(ss.part + i);
+            if (ss.sum) sum += __ldcg(ss.sum + i);
+        }
     red[t] = acc;
+    if (ss.sum) red[128 + t] = sum;
     epi_sync();
     if (t < BN) {
-        float tot = 0.f;
+        float tot = 0.f, mu = 0.f;
 #pragma unroll
         for (int q = 0; q < PARTS; ++q) tot += red[q * BN + t];
-        sm_rstd[t] = rsqrtf(tot / (float)ss.H + ss.eps);
+        if (ss.sum) {   // LayerNorm: variance about the mean
+#pragma unroll
+            for (int q = 0; q < PARTS; ++q) mu += red[128 + q * BN + t];
+            mu /= (float)ss.H;
+            sm_rstd[t] = rsqrtf(fmaxf(tot / (float)ss.H - mu * mu, 0.f) + ss.eps);
+        } else {
+            sm_rstd[t] = rsqrtf(tot / (float)ss.H + ss.eps);
+        }
+        sm_mu[t] = mu;
     }
 }
 
@@ -149,7 +162,7 @@ __device__ __forceinline__ void gather_my_tokens(const DecGemmArgs &g, const Dec
 
 template <int BN>
 __device__ __forceinline__ void epilogue_qkv(const DecGemmArgs &g, const DecTile &t, const float *S, float *Gb,
-                                             const float *sm_rstd, const long *sm_kvoff)
+                                             const float *sm_rstd, const float *sm_mu, const long *sm_kvoff)
 {
     const int r = threadIdx.x, d = g.head_dim, half = d >> 1;
     // weights batched by shard (rank mode): batch z holds heads z * heads_per_shard ...
@@ -168,10 +181,17 @@ __device__ __forceinline__ void epilogue_qkv(const DecGemmArgs &g, const DecTile
     epi_sync();
     if (!row_valid) return;
     const int partner = jd < half ? r + half : r - half;
+    // LayerNorm folded into the tail: this weight row's sum of g * W and its beta * W + bias
+    float wg = 0.f, wb = 0.f;
+    if (g.ln_wg) {
+        const int vrow = (t.wi == 0 ? 0 : (t.wi == 1 ? g.w_rows[0] : g.w_rows[0] + g.w_rows[1])) + row;
+        wg = g.ln_wg[vrow];
+        wb = g.ln_wb[vrow];
+    }
     for (int q = 0;; ++q) {
         const int j = t.rank + t.P * q, m = t.t_row0 + j;
         if (j >= BN || m >= g.t_rows) break;
-        float v = Gb[q * 128 + r] * sm_rstd[j];
+        float v = (Gb[q * 128 + r] - sm_mu[j] * wg) * sm_rstd[j] + wb;
         if (rot) {
             const float2 c = q < 4 ? cs[q < 4 ? q : 0] : g.rope[(long)m * half + (jd < half ? jd : jd - half)];
             const float o = Gb[q * 128 + partner] * sm_rstd[j];
@@ -187,10 +207,25 @@ __device__ __forceinline__ void epilogue_qkv(const DecGemmArgs &g, const DecTile
 }
 
 template <int BN>
-__device__ __forceinline__ void epilogue_gateup(const DecGemmArgs &g, const DecTile &t, const float *S, float *Gb, const float *sm_rstd)
+__device__ __forceinline__ void epilogue_gateup(const DecGemmArgs &g, const DecTile &t, const float *S, float *Gb, const float *sm_rstd,
+                                                const float *sm_mu)
 {
     gather_my_tokens<BN>(g, t, S, Gb);
     epi_sync();
+    if (g.fc1_only) {
+        // block with bias: the tile holds 128 consecutive rows of fc1; LayerNorm folded in, bias, ReLU
+        for (int idx = threadIdx.x;; idx += 128) {
+            const int q = idx >> 6, rr = 2 * (idx & 63), j = t.rank + t.P * q, m = t.t_row0 + j, f = t.w_row0 + rr;
+            if (j >= BN || m >= g.t_rows) break;
+            if (f >= g.Fs) continue;
+            const float rs = sm_rstd[j], mu = sm_mu[j];
+            const float2 a = *(const float2 *)(Gb + q * 128 + rr);
+            const float2 wg = *(const float2 *)(g.ln_wg + (long)t.z * g.Fs + f), wb = *(const float2 *)(g.ln_wb + (long)t.z * g.Fs + f);
+            *(__nv_bfloat162 *)((bf16 *)g.act + (long)m * g.F + (long)t.z * g.Fs + f) =
+                __floats2bfloat162_rn(fmaxf((a.x - mu * wg.x) * rs + wb.x, 0.f), fmaxf((a.y - mu * wg.y) * rs + wb.y, 0.f));
+        }
+        return;
+    }
     // two FFN columns per thread: 32 threads cover the tile's 64 columns of one token
     for (int idx = threadIdx.x;; idx += 128) {
         const int q = idx >> 5, rr = 2 * (idx & 31), j = t.rank + t.P * q, m = t.t_row0 + j, f = t.w_row0 + rr;
@@ -222,6 +257,14 @@ __device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const De
         const float2 a = __bfloat1622float2(*(const __nv_bfloat162 *)&u.x), b = __bfloat1622float2(*(const __nv_bfloat162 *)&u.y);
         gn = make_float4(a.x, a.y, b.x, b.y);
     }
+    // block with bias: the bias of the row-split layer joins the residual stream once - and with it every device's X + P_i
+    float4 bias = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (valid && g.bias) {
+        const uint2 u = *(const uint2 *)((const bf16 *)g.bias + n);
+        const float2 a = __bfloat1622float2(*(const __nv_bfloat162 *)&u.x), b = __bfloat1622float2(*(const __nv_bfloat162 *)&u.y);
+        bias = make_float4(a.x, a.y, b.x, b.y);
+    }
+    auto sum4 = [](float4 v) { return v.x + v.y + v.z + v.w; };
     if (spd_groups) {
         const int rows = (g.t_rows - t.t_row0 < BN ? g.t_rows - t.t_row0 : BN) - t.rank; // this block's tokens: every P-th of them
         if (rows > 3 * t.P) {
@@ -232,7 +275,7 @@ __device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const De
                 if (j >= BN || m >= g.t_rows) break;
                 const long idx = (long)m * H + n;
                 float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (valid) x = *(const float4 *)(g.res_in + idx);
+                if (valid) { x = *(const float4 *)(g.res_in + idx); add4(x, bias); }
                 float4 y[MAX_P];
                 load_partials(y, S, j, lane, t.P);
                 float4 tot = make_float4(0.f, 0.f, 0.f, 0.f), yi = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -248,6 +291,10 @@ __device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const De
                     if (valid && g.hg) store_bf16x4((bf16 *)g.hg + (long)i * g.hg_stride + idx, ri, gn);
                     const float sq = warp_sum(valid ? sq4(ri) : 0.f);
                     if (lane == 0 && g.ss_out) g.ss_out[((long)t.wt * G + i) * g.Mcap + m] = sq;
+                    if (g.sum_out) {
+                        const float sm = warp_sum(valid ? sum4(ri) : 0.f);
+                        if (lane == 0) g.sum_out[((long)t.wt * G + i) * g.Mcap + m] = sm;
+                    }
                     yi = make_float4(0.f, 0.f, 0.f, 0.f);
                     cnt = 0;
                     ++i;
@@ -264,7 +311,7 @@ __device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const De
             if (j >= BN || m >= g.t_rows) break;
             const long idx = (long)m * H + n;
             float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (valid) x = *(const float4 *)(g.res_in + idx);
+            if (valid) { x = *(const float4 *)(g.res_in + idx); add4(x, bias); }
             float4 y[MAX_P];
             load_partials(y, S, j, lane, t.P);
             float4 tot = make_float4(0.f, 0.f, 0.f, 0.f), yi = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -281,6 +328,10 @@ __device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const De
                     if (valid && g.hg) store_bf16x4((bf16 *)g.hg + (long)i * g.hg_stride + idx, ri, gn);
                     const float sq = warp_sum(valid ? sq4(ri) : 0.f);
                     if (lane == 0 && g.ss_out) g.ss_out[((long)t.wt * G + i) * g.Mcap + m] = sq;
+                    if (g.sum_out) {
+                        const float sm = warp_sum(valid ? sum4(ri) : 0.f);
+                        if (lane == 0) g.sum_out[((long)t.wt * G + i) * g.Mcap + m] = sm;
+                    }
                 }
                 yi = make_float4(0.f, 0.f, 0.f, 0.f);
                 cnt = 0;
@@ -296,7 +347,7 @@ __device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const De
         if (j >= BN || m >= g.t_rows) break;
         const long idx = (long)m * H + n;
         float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (valid) x = *(const float4 *)(g.res_in + idx);
+        if (valid) { x = *(const float4 *)(g.res_in + idx); add4(x, bias); }
         float4 y[MAX_P];
         load_partials(y, S, j, lane, t.P);
         float4 tot = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -312,6 +363,10 @@ __device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const De
         if (g.ss_out) {
             const float sq = warp_sum(valid ? sq4(x) : 0.f);
             if (lane == 0) g.ss_out[(long)t.wt * g.Mcap + m] = sq;
+        }
+        if (g.sum_out) {
+            const float sm = warp_sum(valid ? sum4(x) : 0.f);
+            if (lane == 0) g.sum_out[(long)t.wt * g.Mcap + m] = sm;
         }
     }
 }
@@ -438,8 +493,8 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
     constexpr int ROWS = BM / SUB;                   // weight rows per box
     const DecGemmArgs &g = L.g;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ float sm_red[128];
-    __shared__ float sm_rstd[64];
+    __shared__ float sm_red[256];
+    __shared__ float sm_rstd[64], sm_mu[64];
     __shared__ long sm_kvoff[64];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
@@ -457,7 +512,7 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
     if (g.z_is_plane) { t.z = t.rank / g.splits; t.split = t.rank % g.splits; t.wt = blockIdx.x; }
     else { t.z = blockIdx.x / L.w_tiles_per_batch; t.split = t.rank; t.wt = blockIdx.x % L.w_tiles_per_batch; }
     t.wi = (SUB == 2) ? 0 : ((t.wt >= L.tile_start[2]) ? 2 : ((t.wt >= L.tile_start[1]) ? 1 : 0));
-    t.w_row0 = (t.wt - L.tile_start[t.wi]) * ROWS;
+    t.w_row0 = (t.wt - L.tile_start[t.wi]) * ((EPI == EPI_GATEUP && g.fc1_only) ? BM : ROWS);
     t.t_row0 = blockIdx.y * BN;
     const CUtensorMap *tm_w = t.wi == 0 ? &tm_w0 : (t.wi == 1 ? &tm_w1 : &tm_w2);
     const int kb_begin = (int)((long)g.num_kb * t.split / g.splits);
@@ -472,7 +527,8 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
         if (SUB == 1) tma_load_3d_hint(sa, tm_w, kx, t.w_row0, a_z, full_bar(s), stream_once);
         else {
             tma_load_3d_hint(sa, &tm_w0, kx, t.w_row0, a_z, full_bar(s), stream_once);
-            tma_load_3d_hint(sa + ROWS * BK * 2, &tm_w1, kx, t.w_row0, a_z, full_bar(s), stream_once);
+            if (g.fc1_only) tma_load_3d_hint(sa + ROWS * BK * 2, &tm_w0, kx, t.w_row0 + ROWS, a_z, full_bar(s), stream_once);
+            else tma_load_3d_hint(sa + ROWS * BK * 2, &tm_w1, kx, t.w_row0, a_z, full_bar(s), stream_once);
         }
     };
     const int pre = n_kb < C::STAGES ? n_kb : C::STAGES;
@@ -499,7 +555,7 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
         for (int i = pre; i < pf_end; ++i) {
             const int kx = (kb_begin + i) * BK;
             if (SUB == 1) tma_prefetch_l2_3d(tm_w, kx, t.w_row0, a_z);
-            else { tma_prefetch_l2_3d(&tm_w0, kx, t.w_row0, a_z); tma_prefetch_l2_3d(&tm_w1, kx, t.w_row0, a_z); }
+            else { tma_prefetch_l2_3d(&tm_w0, kx, t.w_row0, a_z); tma_prefetch_l2_3d(g.fc1_only ? &tm_w0 : &tm_w1, kx, t.w_row0 + (g.fc1_only ? ROWS : 0), a_z); }
         }
     }
     if (warp == 5) {
@@ -551,7 +607,7 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
         if (EPI == EPI_QKV || EPI == EPI_GATEUP) {
             SumSq ss = g.ss_in;
             if (g.tp.on) ss.part = (const float *)((const char *)ss.part + (long)t.z * g.tp.z_stride); // rank z's own sums
-            compute_rstd<BN>(ss, (EPI == EPI_GATEUP && g.rstd_per_shard && !g.tp.on) ? t.z : 0, t.t_row0, g.t_rows, sm_red, sm_rstd);
+            compute_rstd<BN>(ss, (EPI == EPI_GATEUP && g.rstd_per_shard && !g.tp.on) ? t.z : 0, t.t_row0, g.t_rows, sm_red, sm_rstd, sm_mu);
         }
         if (EPI == EPI_QKV && t.wi > 0 && threadIdx.x < BN) {
             // where this token's K / V row of kv head 0 goes; < 0: skip (the error flag says why)
@@ -602,8 +658,8 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
         if (threadIdx.x == 0) SPD_TRACE_EVENT(EPI, TR_ARRIVED);
         const float *S = (const float *)gen_base;
         float *Gb = (float *)gen_base + BN * 128; // this block's gathered tokens
-        if (EPI == EPI_QKV) epilogue_qkv<BN>(g, t, S, Gb, sm_rstd, sm_kvoff);
-        else if (EPI == EPI_GATEUP) epilogue_gateup<BN>(g, t, S, Gb, sm_rstd);
+        if (EPI == EPI_QKV) epilogue_qkv<BN>(g, t, S, Gb, sm_rstd, sm_mu, sm_kvoff);
+        else if (EPI == EPI_GATEUP) epilogue_gateup<BN>(g, t, S, Gb, sm_rstd, sm_mu);
         else if (EPI == EPI_RESID_TP) epilogue_resid_tp<BN>(g, t, S, abort_flag);
         else epilogue_residual<BN>(g, t, S, EPI == EPI_OPROJ && g.n_groups > 1);
         if (threadIdx.x == 0) { SPD_TRACE_EVENT(EPI, TR_END); stamp_exit(g.stamp); }
@@ -715,6 +771,7 @@ __global__ void __launch_bounds__(128) decode_prologue_kernel(PrologueArgs a, in
     }
     const long zoff = (long)blockIdx.y * a.z_stride;
     float *res_out = (float *)((char *)a.res_out + zoff), *ss_out = (float *)((char *)a.ss_out + zoff);
+    float *sum_out = a.sum_out ? (float *)((char *)a.sum_out + zoff) : nullptr;
     bf16 *hg = (bf16 *)((char *)a.hg + zoff);
     if (a.step && blockIdx.x == 0 && threadIdx.x == 0) *(unsigned *)((char *)a.step + zoff) += 1u;
     // warp w takes tokens w, w+4, ...; lane l the columns 4l .. 4l+3 of the block's 128: no block-wide barrier
@@ -738,6 +795,10 @@ __global__ void __launch_bounds__(128) decode_prologue_kernel(PrologueArgs a, in
         }
         const float q = warp_sum(sq4(x));
         if (lane == 0) ss_out[(long)blockIdx.x * a.Mcap + m] = q;
+        if (sum_out) {
+            const float sm = warp_sum(x.x + x.y + x.z + x.w);
+            if (lane == 0) sum_out[(long)blockIdx.x * a.Mcap + m] = sm;
+        }
     }
     if (threadIdx.x == 0) stamp_exit(a.stamp);
 }
@@ -756,7 +817,8 @@ cudaError_t launch_gemm_decode(DecEpilogue epi, const TcMap *const *weights, con
                                cudaStream_t st)
 {
     const int nw = g.n_weights;
-    if (nw < 1 || nw > 3 || (epi == EPI_GATEUP && nw != 2)) return cudaErrorInvalidValue;
+    if (nw < 1 || nw > 3 || (epi == EPI_GATEUP && nw != (g.fc1_only ? 1 : 2))) return cudaErrorInvalidValue;
+    if (epi == EPI_GATEUP && g.fc1_only && (!g.ln_wg || !g.ln_wb || g.Fs % 2)) return cudaErrorInvalidValue;
     if (g.t_rows <= 0) return cudaSuccess;
     if (g.splits < 1 || g.splits > g.num_kb || g.n_groups > MAX_GROUPS) return cudaErrorInvalidValue;
     const int P = g.z_is_plane ? g.batches * g.splits : g.splits;
@@ -782,7 +844,7 @@ cudaError_t launch_gemm_decode(DecEpilogue epi, const TcMap *const *weights, con
         }
     }
     if (epi == EPI_GATEUP) {
-        tiles = (g.w_rows[0] + 63) / 64;
+        tiles = g.fc1_only ? (g.w_rows[0] + BM - 1) / BM : (g.w_rows[0] + 63) / 64;
         L.tile_start[0] = 0;
         L.tile_start[1] = L.tile_start[2] = 1 << 30;
     }

@@ -50,12 +50,17 @@ struct TpArgs {
 // next GEMM's input) and per-128-column partial sums of x^2; the consumer GEMM multiplies its
 // fp32 result by rstd = rsqrt(sum / H + eps), a per-token (and per-shard) scalar that commutes
 // with the projection.
+// For the block with bias (Sec. 4.1.2) the norm is a LayerNorm, u = (x - mean) * rstd * g + beta, and commutes the same
+// way once two vectors per projection are known: u W^T + b = rstd * ((x * g) W^T - mean * wg) + wb with
+// wg[n] = sum_k g[k] W[n][k] and wb[n] = sum_k beta[k] W[n][k] + b[n] (computed once, when the context is created).
+// The producer then also stores partial row sums of x (`sum`, same layout as `part`).
 struct SumSq {
     const float *part; // [tiles][groups][Mcap]
     int tiles, groups;
     long Mcap;
     int H;
     float eps;
+    const float *sum;  // partial row sums, same layout, or null (RMSNorm)
 };
 
 struct DecGemmArgs {
@@ -74,6 +79,12 @@ struct DecGemmArgs {
     // ---- epilogue operands -----------------------------------------------------------
     SumSq ss_in;           // QKV, GATEUP: sums of squares of the GEMM input's rows
     int rstd_per_shard;    // GATEUP in an SPD block: shard z reads group z
+    // block with bias: LayerNorm folded into the tail (see SumSq): fp32 vectors over the launch's weight rows (QKV: q, k, v
+    // rows one after the other; GATEUP: the rows of fc1), or null
+    const float *ln_wg, *ln_wb;
+    int fc1_only;          // GATEUP: one weight (fc1), 128 consecutive rows per tile, ReLU instead of SwiGLU
+    const void *bias;      // OPROJ, DOWN: bf16 [H] bias of the row-split layer, added once to the residual stream (and so to every device's X + P_i)
+    float *sum_out;        // OPROJ, DOWN: partial row sums of the new residual, same layout as ss_out, or null
     // QKV
     const float2 *rope;    // [tokens][d/2] cos,sin or null
     void *q_out;           // bf16 [tokens][nq*d]
@@ -125,6 +136,7 @@ struct PrologueArgs {
     long z_stride;
     unsigned *step;
     unsigned long long *stamp; // launch stamp slot or null
+    float *sum_out;    // block with bias: partial row sums of x, same layout as ss_out, or null
 };
 cudaError_t launch_decode_prologue(const PrologueArgs &a, cudaStream_t st);
 

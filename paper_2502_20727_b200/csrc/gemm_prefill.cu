@@ -87,7 +87,7 @@ __device__ __forceinline__ PreTile decode_tile(const PreLaunch &L, int EPI, int 
         t.row0 = (nt - L.tile_start[t.wi]) * 256;
     } else if (EPI == PRE_GATEUP) {
         t.z = nt / L.f_tiles;
-        t.row0 = (nt % L.f_tiles) * 128;
+        t.row0 = (nt % L.f_tiles) * (L.g.fc1_only ? 256 : 128);
     } else if (EPI == PRE_OPROJ_SPD) {
         t.row0 = nt * 128;
     } else {
@@ -169,11 +169,17 @@ __device__ __forceinline__ void stg16_bf16(bf16 *p, const float *v)
                  ::"l"(p), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w) : "memory");
 }
 
-__device__ __forceinline__ float row_rstd(const SumSq &s, int group, int m)
+// rstd of a token row from the partial sums of squares (RMSNorm); with partial sums as well (LayerNorm) also the mean
+__device__ __forceinline__ float row_rstd(const SumSq &s, int group, int m, float &mu)
 {
-    float acc = 0.f;
-    for (int t = 0; t < s.tiles; ++t) acc += s.part[((long)t * s.groups + group) * s.Mcap + m];
-    return rsqrtf(acc / (float)s.H + s.eps);
+    float acc = 0.f, sum = 0.f;
+    for (int t = 0; t < s.tiles; ++t) {
+        const long i = ((long)t * s.groups + group) * s.Mcap + m;
+        acc += s.part[i];
+        if (s.sum) sum += s.sum[i];
+    }
+    mu = sum / (float)s.H;
+    return s.sum ? rsqrtf(fmaxf(acc / (float)s.H - mu * mu, 0.f) + s.eps) : rsqrtf(acc / (float)s.H + s.eps);
 }
 
 // ---- epilogues: thread = token row m, columns read from tensor memory 16 at a time ----------------
@@ -181,8 +187,11 @@ __device__ __forceinline__ float row_rstd(const SumSq &s, int group, int m)
 __device__ __forceinline__ void epi_qkv(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, int m, bool valid)
 {
     const int d = g.head_dim, half = d >> 1, nq = g.n_q_heads;
-    const float rs = valid ? row_rstd(g.ss_in, 0, m) : 0.f;
+    float mu = 0.f;
+    const float rs = valid ? row_rstd(g.ss_in, 0, m, mu) : 0.f;
     const bool rot = t.wi < 2 && g.rope != nullptr;
+    // block with bias: first entry of this weight in the folded-LayerNorm vectors (rows of q, k, v one after the other)
+    const int vbase = t.wi == 0 ? 0 : (t.wi == 1 ? g.w_rows[0] : g.w_rows[0] + g.w_rows[1]);
     long kv_off = -1;
     if (t.wi > 0 && valid) {
         int b, pos;
@@ -221,6 +230,13 @@ __device__ __forceinline__ void epi_qkv(const PreGemmArgs &g, const PreTile &t, 
                     olo[2 * i + 1] = a1 * c2.z - b1 * c2.w;
                     ohi[2 * i + 1] = b1 * c2.z + a1 * c2.w;
                 }
+            } else if (g.ln_wg) {
+                const float *wgl = g.ln_wg + vbase + row_h + j0, *wbl = g.ln_wb + vbase + row_h + j0;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    olo[i] = (lo[i] - mu * wgl[i]) * rs + wbl[i];
+                    ohi[i] = (hi[i] - mu * wgl[half + i]) * rs + wbl[half + i];
+                }
             } else {
 #pragma unroll
                 for (int i = 0; i < 16; ++i) { olo[i] = lo[i] * rs; ohi[i] = hi[i] * rs; }
@@ -233,8 +249,32 @@ __device__ __forceinline__ void epi_qkv(const PreGemmArgs &g, const PreTile &t, 
 
 __device__ __forceinline__ void epi_gateup(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, int m, bool valid)
 {
-    const float rs = valid ? row_rstd(g.ss_in, g.rstd_per_shard ? t.z : 0, m) : 0.f;
+    float mu = 0.f;
+    const float rs = valid ? row_rstd(g.ss_in, g.rstd_per_shard ? t.z : 0, m, mu) : 0.f;
     bf16 *dst = (bf16 *)g.act + (long)m * g.F + g.act_col0 + (long)((t.z + g.w_rot) % g.batches) * g.Fs + t.row0;
+    if (g.fc1_only) {
+        // block with bias: the tile's 256 columns are 256 consecutive rows of fc1; LayerNorm folded in, bias, ReLU
+        const float *wgl = g.ln_wg + (long)t.z * g.Fs + t.row0, *wbl = g.ln_wb + (long)t.z * g.Fs + t.row0;
+#pragma unroll 1
+        for (int c = 0; c < 16; c += 2) {
+            const int f = t.row0 + c * 16;
+            if (f >= g.Fs) break;
+            float a[16], b[16], o[16];
+            tmem_ld16x2(tacc + c * 16, tacc + c * 16 + 16, a, b);
+            if (!valid) continue;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) o[i] = fmaxf((a[i] - mu * wgl[c * 16 + i]) * rs + wbl[c * 16 + i], 0.f);
+            *(uint4 *)(dst + c * 16) = pack8(o);
+            if (f + 8 < g.Fs) *(uint4 *)(dst + c * 16 + 8) = pack8(o + 8);
+            if (f + 16 < g.Fs) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) o[i] = fmaxf((b[i] - mu * wgl[c * 16 + 16 + i]) * rs + wbl[c * 16 + 16 + i], 0.f);
+                *(uint4 *)(dst + c * 16 + 16) = pack8(o);
+                if (f + 24 < g.Fs) *(uint4 *)(dst + c * 16 + 24) = pack8(o + 8);
+            }
+        }
+        return;
+    }
 #pragma unroll 1
     for (int c = 0; c < 8; ++c) {
         const int f = t.row0 + c * 16;
@@ -254,11 +294,11 @@ __device__ __forceinline__ void epi_gateup(const PreGemmArgs &g, const PreTile &
 
 // y: 16 accumulator columns at output column n.  r = x + y; stores what the arguments ask for.
 __device__ __forceinline__ float resid_chunk(const PreGemmArgs &g, long idx, int n, const float *x, const float *y, bf16 *hg,
-                                             bool store_res)
+                                             bool store_res, float &sum)
 {
     float r[16], sq = 0.f;
 #pragma unroll
-    for (int i = 0; i < 16; ++i) { r[i] = x[i] + y[i]; sq = fmaf(r[i], r[i], sq); }
+    for (int i = 0; i < 16; ++i) { r[i] = x[i] + y[i]; sq = fmaf(r[i], r[i], sq); sum += r[i]; }
     if (store_res) {
         if (g.res_out) { stg8(g.res_out + idx, r); stg8(g.res_out + idx + 8, r + 8); }
         if (g.final_out) stg16_bf16((bf16 *)g.final_out + idx, r);
@@ -279,10 +319,20 @@ __device__ __forceinline__ void load_x16(const float *p, float *x)
     ldg8(p, x);
     ldg8(p + 8, x + 8);
 }
+// x += bias[n .. n+16) (bf16), the bias of a row-split layer of the block with bias
+__device__ __forceinline__ void add_bias16(const void *bias, int n, float *x)
+{
+    if (!bias) return;
+    float b[16];
+    unpack8(*(const uint4 *)((const bf16 *)bias + n), b);
+    unpack8(*(const uint4 *)((const bf16 *)bias + n + 8), b + 8);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) x[i] += b[i];
+}
 
 __device__ __forceinline__ void epi_resid(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, int m, bool valid)
 {
-    float ssq = 0.f;
+    float ssq = 0.f, sum = 0.f;
 #pragma unroll 1
     for (int c = 0; c < 16; c += 2) {
         const int n = t.row0 + c * 16;
@@ -293,15 +343,18 @@ __device__ __forceinline__ void epi_resid(const PreGemmArgs &g, const PreTile &t
         const long idx = (long)m * g.H + n;
         float x[16];
         load_x16(g.res_in + idx, x);
+        add_bias16(g.bias, n, x);
         if (g.ysave) { stg8(g.ysave + idx, ya); stg8(g.ysave + idx + 8, ya + 8); }
-        ssq += resid_chunk(g, idx, n, x, ya, g.hg ? (bf16 *)g.hg : nullptr, true);
+        ssq += resid_chunk(g, idx, n, x, ya, g.hg ? (bf16 *)g.hg : nullptr, true, sum);
         if (n + 16 < g.H) {
             load_x16(g.res_in + idx + 16, x);
+            add_bias16(g.bias, n + 16, x);
             if (g.ysave) { stg8(g.ysave + idx + 16, yb); stg8(g.ysave + idx + 24, yb + 8); }
-            ssq += resid_chunk(g, idx + 16, n + 16, x, yb, g.hg ? (bf16 *)g.hg : nullptr, true);
+            ssq += resid_chunk(g, idx + 16, n + 16, x, yb, g.hg ? (bf16 *)g.hg : nullptr, true, sum);
         }
     }
     if (valid && g.ss_out) g.ss_out[(long)t.nt * g.Mcap + m] = ssq;
+    if (valid && g.sum_out) g.sum_out[(long)t.nt * g.Mcap + m] = sum;
 }
 
 // Rank mode, shot one of a two-shot exchange (see TpScatter): this block's 128 partial rows go to the rank that owns
@@ -352,8 +405,10 @@ __device__ __forceinline__ void spd_park_x(const PreGemmArgs &g, const PreTile &
     for (int cc = 0; cc < 4; ++cc) {
         const int c = half * 4 + cc, n = t.row0 + c * 16;
         float x[16];
-        if (valid && n < g.H) load_x16(g.res_in + (long)m * g.H + n, x);
-        else {
+        if (valid && n < g.H) {
+            load_x16(g.res_in + (long)m * g.H + n, x);
+            add_bias16(g.bias, n, x); // block with bias: b joins X once - and so every device's X + P_i + b and the carried sum
+        } else {
 #pragma unroll
             for (int i = 0; i < 16; ++i) x[i] = 0.f;
         }
@@ -387,7 +442,7 @@ __device__ __forceinline__ float epi_row_sumsq(const PreGemmArgs &g, const PreTi
 // plane (32-byte stores, whole sectors; shared memory is left to the operand ring); X + sum_i Y_i, carried in
 // tot, is written by the last pass.
 __device__ __forceinline__ float epi_oproj_spd(const PreGemmArgs &g, const PreTile &t, uint32_t tacc, uint32_t tx, int z,
-                                               int m, bool valid, int half, float (&tot)[64])
+                                               int m, bool valid, int half, float (&tot)[64], float &sum)
 {
     const int T = g.batches;
     float ssq = 0.f;
@@ -410,6 +465,7 @@ __device__ __forceinline__ float epi_oproj_spd(const PreGemmArgs &g, const PreTi
             for (int i = 0; i < 16; ++i) {
                 const float ri = x[16 * q + i] + y[16 * q + i];
                 ssq = fmaf(ri, ri, ssq);
+                sum += ri;
                 gn[i] *= ri;
             }
             stg16_bf16(plane + n + 16 * q, gn);
@@ -506,14 +562,16 @@ __global__ void __launch_bounds__(PCfg<EPI, PAIR>::THREADS_, 1) gemm_prefill_ker
                             const uint32_t fb = mapa_shared(full_bar(s), 0);
                             tma_load_3d_pair(sa, &tm_t, kb * BK, t.m0, tz, fb, keep);
                             // this CTA's half of the tile's weight rows (GATEUP: the leader holds the gate rows, its partner the up rows)
-                            if (EPI == PRE_GATEUP) tma_load_3d_pair(sb, leader ? &tm_w0 : &tm_w1, kb * BK, t.row0, wz, fb, keep);
+                            if (EPI == PRE_GATEUP && g.fc1_only) tma_load_3d_pair(sb, &tm_w0, kb * BK, t.row0 + crank * 128, wz, fb, keep);
+                            else if (EPI == PRE_GATEUP) tma_load_3d_pair(sb, leader ? &tm_w0 : &tm_w1, kb * BK, t.row0, wz, fb, keep);
                             else tma_load_3d_pair(sb, tm_w, kb * BK, t.row0 + crank * (BN / 2), wz, fb, keep);
                         } else {
                             mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
                             tma_load_3d(sa, &tm_t, kb * BK, t.m0, tz, full_bar(s));
                             if (EPI == PRE_GATEUP) {
                                 tma_load_3d(sb, &tm_w0, kb * BK, t.row0, wz, full_bar(s));
-                                tma_load_3d(sb + 128 * BK * 2, &tm_w1, kb * BK, t.row0, wz, full_bar(s));
+                                if (g.fc1_only) tma_load_3d(sb + 128 * BK * 2, &tm_w0, kb * BK, t.row0 + 128, wz, full_bar(s));
+                                else tma_load_3d(sb + 128 * BK * 2, &tm_w1, kb * BK, t.row0, wz, full_bar(s));
                             } else {
                                 tma_load_3d(sb, tm_w, kb * BK, t.row0, wz, full_bar(s));
                             }
@@ -608,8 +666,10 @@ __global__ void __launch_bounds__(PCfg<EPI, PAIR>::THREADS_, 1) gemm_prefill_ker
                     if (valid) g.ss_out[((long)(t.nt * 2 + half) * g.batches + pass) * g.Mcap + m] = ssq;
                 } else {
                     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_PREFILL + EPI, TR_DEP_DONE);
-                    const float ssq = epi_oproj_spd(g, t, tacc, tmem_base + lane_base + X_COL, pass, m, valid, half, tot);
+                    float sum = 0.f;
+                    const float ssq = epi_oproj_spd(g, t, tacc, tmem_base + lane_base + X_COL, pass, m, valid, half, tot, sum);
                     if (valid && g.ss_out) g.ss_out[((long)(t.nt * 2 + half) * g.batches + pass) * g.Mcap + m] = ssq;
+                    if (valid && g.sum_out) g.sum_out[((long)(t.nt * 2 + half) * g.batches + pass) * g.Mcap + m] = sum;
                     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_PREFILL + EPI, TR_MAIN_DONE);
                 }
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -665,25 +725,28 @@ __global__ void __launch_bounds__(256) prefill_prologue_kernel(PrologueArgs a)
     if (a.step && blockIdx.x == 0 && threadIdx.x == 0) *a.step += 1u; // rank mode: the rank's step number advances with every launch sequence
     __shared__ float red[8];
     const int m = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    float sq = 0.f;
+    float sq = 0.f, sum = 0.f;
     for (int n = threadIdx.x * 8; n < a.H; n += blockDim.x * 8) {
         const long idx = (long)m * a.H + n;
         float x[8], gn[8];
         unpack8(*(const uint4 *)((const bf16 *)a.x + idx), x);
         unpack8(*(const uint4 *)((const bf16 *)a.gain + n), gn);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { sq = fmaf(x[i], x[i], sq); gn[i] *= x[i]; }
+        for (int i = 0; i < 8; ++i) { sq = fmaf(x[i], x[i], sq); sum += x[i]; gn[i] *= x[i]; }
         *(float4 *)(a.res_out + idx) = make_float4(x[0], x[1], x[2], x[3]);
         *(float4 *)(a.res_out + idx + 4) = make_float4(x[4], x[5], x[6], x[7]);
         *(uint4 *)((bf16 *)a.hg + idx) = pack8(gn);
     }
     sq = warp_sum(sq);
-    if (lane == 0) red[warp] = sq;
+    sum = warp_sum(sum);
+    __shared__ float red_sum[8];
+    if (lane == 0) { red[warp] = sq; red_sum[warp] = sum; }
     __syncthreads();
     if (threadIdx.x == 0) {
-        float tot = 0.f;
-        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];
+        float tot = 0.f, tsum = 0.f;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { tot += red[w]; tsum += red_sum[w]; }
         a.ss_out[m] = tot;
+        if (a.sum_out) a.sum_out[m] = tsum;
         stamp_exit(a.stamp);
     }
 }
@@ -697,7 +760,8 @@ cudaError_t launch_gemm_prefill(PreEpilogue epi, const TcMap *const *weights, co
                                 cudaStream_t st)
 {
     const int nw = g.n_weights;
-    if (nw < 1 || nw > 3 || (epi == PRE_GATEUP && nw != 2)) return cudaErrorInvalidValue;
+    if (nw < 1 || nw > 3 || (epi == PRE_GATEUP && nw != (g.fc1_only ? 1 : 2))) return cudaErrorInvalidValue;
+    if (epi == PRE_GATEUP && g.fc1_only && (!g.ln_wg || !g.ln_wb)) return cudaErrorInvalidValue;
     if (g.t_rows <= 0) return cudaSuccess;
     if (g.num_kb < 1 || g.batches < 1 || g.batches > 8) return cudaErrorInvalidValue;
     if (epi == PRE_QKV && (256 % g.head_dim || g.head_dim < 32)) return cudaErrorInvalidValue;
@@ -730,7 +794,7 @@ cudaError_t launch_gemm_prefill(PreEpilogue epi, const TcMap *const *weights, co
         return pair ? launch_epi<PRE_QKV, 1>(tw, *(const CUtensorMap *)&tokens, L, st) : launch_epi<PRE_QKV, 0>(tw, *(const CUtensorMap *)&tokens, L, st);
     }
     case PRE_GATEUP:
-        L.f_tiles = (g.Fs + 127) / 128;
+        L.f_tiles = g.fc1_only ? (g.Fs + 255) / 256 : (g.Fs + 127) / 128;
         L.n_tiles = L.f_tiles * g.batches;
         return pair ? launch_epi<PRE_GATEUP, 1>(tw, *(const CUtensorMap *)&tokens, L, st) : launch_epi<PRE_GATEUP, 0>(tw, *(const CUtensorMap *)&tokens, L, st);
     case PRE_OPROJ_SPD:

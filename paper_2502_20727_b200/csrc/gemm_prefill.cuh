@@ -42,6 +42,12 @@ struct PreGemmArgs {
     unsigned long long *stamp; // launch stamp slot or null
     SumSq ss_in;         // QKV, GATEUP
     int rstd_per_shard;
+    // block with bias (Sec. 4.1.2): LayerNorm folded into the tail (see SumSq): fp32 vectors over the launch's weight rows
+    // (QKV: q, k, v rows one after the other; GATEUP: the rows of fc1), or null
+    const float *ln_wg, *ln_wb;
+    int fc1_only;        // GATEUP: one weight (fc1), 256 consecutive rows per tile, ReLU instead of SwiGLU
+    const void *bias;    // RESID, OPROJ_SPD: bf16 [H] bias of the row-split layer, added once to the residual stream
+    float *sum_out;      // RESID, OPROJ_SPD: partial row sums of the new residual, same layout as ss_out, or null
     // QKV
     const float2 *rope;  // [tokens][d/2] cos,sin or null
     void *q_out;         // bf16 [tokens][nq*d]

@@ -129,6 +129,9 @@ struct Ctx {
     float2 *rope;
     int *err, *attn_cnt;
     float *ss_attn, *ss_mlp;     // partial row sums of squares (fused decode path)
+    float *sm_attn, *sm_mlp;     // block with bias: partial row sums (LayerNorm means)
+    float *lnvec;                // block with bias: per layer wg_qkv[nqkv], wb_qkv[nqkv], wg_fc1[F], wb_fc1[F]
+    int bias_fused;              // block with bias on the fused projections (1) or on the K-split GEMMs with separate row kernels (0)
     int split_override[SITE_COUNT];
     int l2_prefetch_kb;          // K blocks per thread block prefetched into L2 by the decode GEMMs
     int ring_stages;             // decode GEMMs: stages of the operand ring (0 = per launch)
@@ -339,6 +342,7 @@ SiteGeom site_geom(const spd_dims &d, int site)
 
 struct Layout {
     size_t res[2], h, q, attn, act, qkv32, proj32, gu32, part_o, part_ml, attn_cnt, rope, err, ss_attn, ss_mlp, stamps, total;
+    size_t sm_attn, sm_mlp, lnvec; // block with bias: partial row sums beside the sums of squares; folded-LayerNorm vectors
     size_t Mcap;
 };
 
@@ -376,6 +380,10 @@ Layout make_layout(const spd_dims &d, bool any_spd)
     L.ss_attn = take(h_tiles * Mmax * 4);
     L.ss_mlp = take(2 * h_tiles * T * Mmax * 4); // the SPD o_proj of the prefill path leaves two partials per tile
     L.stamps = take((size_t)stamp_slots(d) * 16 + ((size_t)stamp_slots(d) + 2) * 8); // slots, then the running totals
+    const bool bias_block = d.block_kind == 1 && d.dtype == 1;
+    L.sm_attn = take(bias_block ? h_tiles * Mmax * 4 : 0);
+    L.sm_mlp = take(bias_block ? 2 * h_tiles * T * Mmax * 4 : 0);
+    L.lnvec = take(bias_block ? (size_t)d.n_layers * 2 * (nqkv + F) * 4 : 0); // per layer: wg_qkv, wb_qkv, wg_fc1, wb_fc1
     L.total = off;
     return L;
 }
@@ -777,7 +785,11 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
     const int tbox = tc_token_box(true, M);
     const int tok_tiles = cdiv(M, tbox), h_tiles = cdiv(H, 128);
     int launches = 0;
-    const bool rope = d.rope_base > 0.f;
+    // block with bias (Sec. 4.1.2): LayerNorm folded into the QKV / fc1 tails, biases in the tails, ReLU, no rotary embedding
+    const bool opt = d.block_kind == 1;
+    const bool rope = d.rope_base > 0.f && !opt;
+    const int nqkv = qd + 2 * kd;
+    auto lnvec = [&](int l) { return c->lnvec + (size_t)l * 2 * (nqkv + F); }; // wg_qkv, wb_qkv, wg_fc1, wb_fc1
     // K ranges of a site: automatic or overridden; a tile's ranges (times the shards for o_proj) fit a cluster of 8
     auto splits_of = [&](int site) {
         const SiteGeom sg = site_geom(d, site);
@@ -788,6 +800,7 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
         a.x = x; a.res_out = c->res[0]; a.gain = c->layers[0].attn_norm; a.hg = c->h; a.ss_out = c->ss_attn;
         a.Mcap = Mc; a.M = M; a.H = H;
         if (rope) { a.rope_table = c->rope; a.tm = tm; a.head_dim = d.head_dim; a.rope_base = d.rope_base; }
+        if (opt) a.sum_out = c->sm_attn;
         LAUNCH_S(K_NORM, a, launch_decode_prologue(a, st));
     }
     auto base_args = [&]() {
@@ -807,7 +820,8 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
             g.n_weights = 3; g.w_rows[0] = qd; g.w_rows[1] = g.w_rows[2] = kd;
             g.num_kb = cdiv(H, 64);
             g.splits = splits_of(SITE_QKV);
-            g.ss_in = SumSq{c->ss_attn, h_tiles, 1, Mc, H, d.rms_eps};
+            g.ss_in = SumSq{c->ss_attn, h_tiles, 1, Mc, H, d.rms_eps, opt ? c->sm_attn : nullptr};
+            if (opt) { g.ln_wg = lnvec(l); g.ln_wb = lnvec(l) + nqkv; }
             g.rope = rope ? c->rope : nullptr; g.q_out = c->q; g.k_pages = w.k_pages; g.v_pages = w.v_pages; g.pt = pt; g.tm = tm;
             g.n_q_heads = d.n_q_heads; g.head_dim = d.head_dim;
             LAUNCH_S(K_QKV, g, launch_gemm_decode(EPI_QKV, wmaps, *am, g, st));
@@ -830,6 +844,7 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
             g.res_in = c->res[0]; g.res_out = c->res[1]; g.gain = w.mlp_norm; g.hg = c->h; g.hg_stride = Mc * H;
             g.ss_out = c->ss_mlp;
             g.n_groups = sync ? 1 : Tn;
+            if (opt) { g.bias = w.bo; g.sum_out = c->sm_mlp; } // Y_i = P_i + b: b once in the stream, and in every device's MLP input
             LAUNCH_S(K_OPROJ, g, launch_gemm_decode(EPI_OPROJ, wmaps, *am, g, st));
         }
         {   // a8: 64 gate rows and the 64 up rows of the same FFN columns per tile
@@ -839,7 +854,11 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
             g.n_weights = 2; g.w_rows[0] = g.w_rows[1] = Fs; g.batches = Tn; g.w_batched = 1; g.t_batched = sync ? 0 : 1;
             g.num_kb = cdiv(H, 64);
             g.splits = splits_of(SITE_GU);
-            g.ss_in = SumSq{c->ss_mlp, h_tiles, sync ? 1 : Tn, Mc, H, d.rms_eps};
+            g.ss_in = SumSq{c->ss_mlp, h_tiles, sync ? 1 : Tn, Mc, H, d.rms_eps, opt ? c->sm_mlp : nullptr};
+            if (opt) {   // fc1 alone: 128 of its rows per tile, bias and ReLU in the tail
+                g.n_weights = 1; g.fc1_only = 1; g.ln_wg = lnvec(l) + 2 * nqkv; g.ln_wb = lnvec(l) + 2 * nqkv + F;
+                g.splits = decode_splits((long)cdiv(Fs, 128) * Tn * tok_tiles, g.num_kb, c->split_override[SITE_GU], 8, tbox == 16 ? 3 : 2);
+            }
             g.rstd_per_shard = sync ? 0 : 1;
             g.act = c->act; g.F = F; g.Fs = Fs;
             LAUNCH_S(K_GATE_UP, g, launch_gemm_decode(EPI_GATEUP, wmaps, *am, g, st));
@@ -854,6 +873,7 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
             g.res_in = c->res[1]; g.res_out = c->res[0];
             if (l + 1 < d.n_layers) { g.gain = c->layers[l + 1].attn_norm; g.hg = c->h; g.hg_stride = Mc * H; g.ss_out = c->ss_attn; }
             else g.final_out = out;
+            if (opt) { g.bias = w.b_fc2; if (l + 1 < d.n_layers) g.sum_out = c->sm_attn; }
             LAUNCH_S(K_DOWN, g, launch_gemm_decode(EPI_DOWN, wmaps, *am, g, st));
         }
     }
@@ -1149,12 +1169,17 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
     const long Mc = c->Mcap;
     PageTable pt{bt, max_pages, c->n_pages, d.kv_block_size, d.n_kv_heads};
     int launches = 0;
-    const bool rope = d.rope_base > 0.f;
+    // block with bias (Sec. 4.1.2): LayerNorm folded into the QKV / fc1 tails, biases in the tails, ReLU, no rotary embedding
+    const bool opt = d.block_kind == 1;
+    const bool rope = d.rope_base > 0.f && !opt;
+    const int nqkv = qd + 2 * kd;
+    auto lnvec = [&](int l) { return c->lnvec + (size_t)l * 2 * (nqkv + F); }; // wg_qkv, wb_qkv, wg_fc1, wb_fc1
     if (rope) LAUNCH(K_ROPE_TABLE, launch_rope_table(c->rope, tm, M, d.head_dim, d.rope_base, st, next_stamp(c, K_ROPE_TABLE)));
     {
         PrologueArgs a{};
         a.x = x; a.res_out = c->res[0]; a.gain = c->layers[0].attn_norm; a.hg = c->h; a.ss_out = c->ss_attn;
         a.Mcap = Mc; a.M = M; a.H = H;
+        if (opt) a.sum_out = c->sm_attn;
         LAUNCH_S(K_NORM, a, launch_prefill_prologue(a, st));
     }
     int attn_tiles = 1; // partial sums of squares per token in ss_attn
@@ -1178,7 +1203,8 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
             MAP_OR_FAIL(am, act_map(c, AB_H, 128));
             g.n_weights = 3; g.w_rows[0] = qd; g.w_rows[1] = g.w_rows[2] = kd;
             g.num_kb = cdiv(H, 64);
-            g.ss_in = SumSq{c->ss_attn, attn_tiles, 1, Mc, H, d.rms_eps};
+            g.ss_in = SumSq{c->ss_attn, attn_tiles, 1, Mc, H, d.rms_eps, opt ? c->sm_attn : nullptr};
+            if (opt) { g.ln_wg = lnvec(l); g.ln_wb = lnvec(l) + nqkv; }
             g.rope = rope ? c->rope : nullptr; g.q_out = c->q; g.k_pages = w.k_pages; g.v_pages = w.v_pages; g.pt = pt; g.tm = tm;
             g.n_q_heads = d.n_q_heads; g.head_dim = d.head_dim;
             LAUNCH_S(K_QKV, g, launch_gemm_prefill(PRE_QKV, wmaps, *am, g, st));
@@ -1206,6 +1232,7 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
             MAP_OR_FAIL(am, act_map(c, AB_ATTN, 128));
             g.w_rows[0] = H; g.num_kb = cdiv(qd, 64);
             g.res_in = c->res[0]; g.res_out = c->res[1]; g.gain = w.mlp_norm; g.hg = c->h; g.hg_stride = Mc * H; g.ss_out = c->ss_mlp;
+            if (opt) { g.bias = w.bo; g.sum_out = c->sm_mlp; }
             LAUNCH_S(K_OPROJ, g, launch_gemm_prefill(PRE_RESID, wmaps, *am, g, st));
             mlp_tiles = pre_ss_tiles(PRE_RESID, H); mlp_groups = 1;
         } else {      // a5 - a7, SPD block: device i's K slice gives Y_i, kept apart
@@ -1216,6 +1243,7 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
             g.res_in = c->res[0]; g.res_out = c->res[1]; g.gain = w.mlp_norm; g.hg = c->h; g.hg_stride = Mc * H; g.ss_out = c->ss_mlp;
             MAP_OR_FAIL(hm, act_map(c, AB_H, 128));
             g.h_map = hm;
+            if (opt) { g.bias = w.bo; g.sum_out = c->sm_mlp; } // Y_i = P_i + b: b once in the carried sum, and in every device's MLP input
             LAUNCH_S(K_OPROJ, g, launch_gemm_prefill(PRE_OPROJ_SPD, wmaps, *am, g, st));
             mlp_tiles = pre_ss_tiles(PRE_OPROJ_SPD, H); mlp_groups = Tn;
         }
@@ -1265,9 +1293,10 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
             MAP_OR_FAIL(am, act_map(c, AB_H, 128));
             g.n_weights = 2; g.w_rows[0] = g.w_rows[1] = Fs; g.batches = Tn; g.t_batched = sync ? 0 : 1;
             g.num_kb = cdiv(H, 64);
-            g.ss_in = SumSq{c->ss_mlp, mlp_tiles, mlp_groups, Mc, H, d.rms_eps};
+            g.ss_in = SumSq{c->ss_mlp, mlp_tiles, mlp_groups, Mc, H, d.rms_eps, opt ? c->sm_mlp : nullptr};
             g.rstd_per_shard = sync ? 0 : 1;
             g.act = c->act; g.F = F; g.Fs = Fs;
+            if (opt) { g.n_weights = 1; g.fc1_only = 1; g.ln_wg = lnvec(l) + 2 * nqkv; g.ln_wb = lnvec(l) + 2 * nqkv + F; } // fc1 alone: bias, ReLU
             LAUNCH_S(K_GATE_UP, g, launch_gemm_prefill(PRE_GATEUP, wmaps, *am, g, st));
         }
         {   // a9 + a10: res[1] holds X + sum_i Y_i in both modes, so out = res[1] + sum_i Z_i
@@ -1278,6 +1307,7 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
             g.res_in = c->res[1]; g.res_out = c->res[0];
             if (l + 1 < d.n_layers) { g.gain = c->layers[l + 1].attn_norm; g.hg = c->h; g.hg_stride = Mc * H; g.ss_out = c->ss_attn; }
             else g.final_out = out;
+            if (opt) { g.bias = w.b_fc2; if (l + 1 < d.n_layers) g.sum_out = c->sm_attn; }
             LAUNCH_S(K_DOWN, g, launch_gemm_prefill(PRE_RESID, wmaps, *am, g, st));
             attn_tiles = pre_ss_tiles(PRE_RESID, H);
         }
@@ -1480,6 +1510,8 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     c.part_o = (float *)(c.ws + L.part_o); c.part_ml = (float *)(c.ws + L.part_ml);
     c.attn_cnt = (int *)(c.ws + L.attn_cnt);
     c.ss_attn = (float *)(c.ws + L.ss_attn); c.ss_mlp = (float *)(c.ws + L.ss_mlp);
+    c.sm_attn = (float *)(c.ws + L.sm_attn); c.sm_mlp = (float *)(c.ws + L.sm_mlp); c.lnvec = (float *)(c.ws + L.lnvec);
+    c.bias_fused = 1;
     c.stamps = (unsigned long long *)(c.ws + L.stamps);
     c.stamps_cap = stamp_slots(*dims);
     c.timeline = false;
@@ -1510,6 +1542,19 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     // neither an earlier user of this memory nor a first kernel can overlap the zeroing.
     cudaError_t e = cudaDeviceSynchronize();
     if (e == cudaSuccess) e = cudaMemset(workspace, 0, L.total);
+    if (dims->block_kind == 1 && dims->dtype == 1) {
+        // block with bias: fold each LayerNorm into the projection that follows it (see SumSq)
+        const int H = dims->hidden, qd = dims->n_q_heads * dims->head_dim, kd = dims->n_kv_heads * dims->head_dim, F = dims->ffn;
+        const size_t per_layer = 2 * (size_t)(qd + 2 * kd + F);
+        for (int l = 0; l < dims->n_layers && e == cudaSuccess; ++l) {
+            const spd_layer &w = c.layers[l];
+            float *wg = c.lnvec + l * per_layer, *wb = wg + (qd + 2 * kd), *fg = wb + (qd + 2 * kd), *fb = fg + F;
+            e = launch_ln_fold(w.wq, qd, H, w.attn_norm, w.attn_norm_b, w.bq, wg, wb, 0);
+            if (e == cudaSuccess) e = launch_ln_fold(w.wk, kd, H, w.attn_norm, w.attn_norm_b, w.bk, wg + qd, wb + qd, 0);
+            if (e == cudaSuccess) e = launch_ln_fold(w.wv, kd, H, w.attn_norm, w.attn_norm_b, w.bv, wg + qd + kd, wb + qd + kd, 0);
+            if (e == cudaSuccess) e = launch_ln_fold(w.w_gate, F, H, w.mlp_norm, w.mlp_norm_b, w.b_fc1, fg, fb, 0);
+        }
+    }
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { g_last_cuda_error = (int)e; delete h; return SPD_ECUDA; }
     *out = h;
@@ -1532,7 +1577,7 @@ int spd_prefill(spd_ctx *ctx, const void *x, int32_t B, int32_t S, const int32_t
     auto run = [&](int b0, int nb, int s0, int ns) -> int {
         TokMap tm{0, b0, ns, s0, nullptr};
         size_t off = ((size_t)b0 * S + s0) * d.hidden * es;
-        const bool fused = d.dtype == 1 && d.hidden % 16 == 0 && d.block_kind == 0;
+        const bool fused = d.dtype == 1 && d.hidden % 16 == 0 && (d.block_kind == 0 || c.bias_fused);
         int rc = d.dtype == 0 ? run_tokens<float>(&c, (const char *)x + off, (char *)out + off, nb * ns, tm, block_table, max_pages, false, S, st)
                  : fused      ? run_prefill_fused(&c, (const char *)x + off, (char *)out + off, nb * ns, tm, block_table, max_pages, S, st)
                               : run_tokens<bf16>(&c, (const char *)x + off, (char *)out + off, nb * ns, tm, block_table, max_pages, false, S, st);
@@ -1581,7 +1626,7 @@ int spd_decode_step(spd_ctx *ctx, const void *x, int32_t B, const int32_t *seq_l
         return [&, bucket]() -> int {
             CU_TRY(timeline_restart(&c, st));
             const int rc = d.dtype == 0        ? run_tokens<float>(&c, x, out, B, tm, block_table, max_pages, true, bucket, st)
-                           : d.block_kind == 0 ? run_decode_fused(&c, x, out, B, tm, block_table, max_pages, bucket, st)
+                           : (d.block_kind == 0 || c.bias_fused) ? run_decode_fused(&c, x, out, B, tm, block_table, max_pages, bucket, st)
                                                : run_tokens<bf16>(&c, x, out, B, tm, block_table, max_pages, true, bucket, st);
             if (rc != SPD_OK) return rc;
             CU_TRY(timeline_fold(&c, st)); // part of the captured step: every replay folds its own stamps
@@ -1697,6 +1742,7 @@ int spd_set_tuning(spd_ctx *ctx, const char *key, int32_t value)
     if (!strcmp(key, "prefill_rescale_log2")) { c.prefill_rescale_log2 = value > 16 ? 16 : value; found = true; }
     if (!strcmp(key, "l2_prefetch_blocks")) { c.l2_prefetch_kb = value > 64 ? 64 : value; found = true; }
     if (!strcmp(key, "prefill_group_m")) { c.prefill_group_m = value > 4096 ? 4096 : value; found = true; }
+    if (!strcmp(key, "bias_fused")) { c.bias_fused = value != 0; found = true; }
     if (!strcmp(key, "prefill_pairs")) { c.prefill_pairs = value != 0; found = true; }
     if (!strcmp(key, "peer_wait_ms")) { c.peer_wait_ms = value < 1 ? 1000 : (value > 60000 ? 60000 : value); found = true; }
     if (!found) return SPD_EINVAL;

@@ -28,6 +28,41 @@ def test_bf16_small_ragged(mask):
     run_case(w, mask, 3, 37, 3)
 
 
+@pytest.mark.parametrize("mask", [(0, 1, 0), (1, 1, 1)])
+def test_bf16_on_the_unfused_sequence(mask):
+    """The K-split GEMMs with separate LayerNorm / bias kernels stay selectable (tuning key bias_fused = 0)."""
+    w = opt("optbf", "bf16", 3, 512, 8, 8, 64, 1376, 4, mask, 3, 37, 3)
+    run_case(w, mask, 3, 37, 3, tuning={"bias_fused": 0})
+
+
+@pytest.mark.parametrize("mask", [(0, 0), (1, 1), (0, 1)])
+def test_bf16_prompt_over_several_token_tiles_and_a_ragged_fc1_tile(mask):
+    """300 prompt tokens (CTA pairs, a ragged last tile), 688 fc1 rows per shard (not a multiple of the fc1 tile),
+    then decode steps at a batch of 2; LayerNorm is folded into the QKV and fc1 tails on this path."""
+    w = opt("optbf2", "bf16", 2, 1024, 8, 8, 128, 2752, 4, mask, 2, 150, 3)
+    run_case(w, mask, 2, 150, 3)
+
+
+def test_bf16_decode_batch_of_several_token_boxes():
+    """Decode at a batch of 40 (token box 64) after a short prompt, both block kinds in one stack."""
+    w = opt("optbf3", "bf16", 2, 1024, 8, 8, 128, 2048, 8, (0, 1), 40, 9, 2)
+    run_case(w, (0, 1), 40, 9, 2)
+
+
+def test_fused_and_unfused_sequences_agree():
+    """Same stack, same inputs: folding LayerNorm into the tails changes rounding, nothing else."""
+    w = opt("optbf4", "bf16", 2, 1024, 8, 8, 128, 2752, 4, (0, 1), 2, 150, 0)
+    outs = []
+    for fused in (1, 0):
+        p = Pair(w, mask=(0, 1), B=2, max_len=150)
+        p.stack.set_tuning(bias_fused=fused)
+        got, ref, _ = p.prefill(150)
+        assert rel_err(got, ref) <= TOL["bf16"]
+        outs.append(got)
+        p.stack.close()
+    assert rel_err(outs[0], outs[1]) <= TOL["bf16"]
+
+
 def test_opt_6_7b_dims_reduced_tokens():
     """hidden 4096, 32 heads x 128, ffn 16384 (OPT-6.7B, Sec. 5.1), T = 8, one SPD block, few tokens."""
     w = opt("opt67", "bf16", 1, 4096, 32, 32, 128, 16384, 8, (0,), 2, 20, 2)

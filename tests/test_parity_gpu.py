@@ -10,8 +10,10 @@ from parity_util import TOL, Pair, rel_err
 pytestmark = pytest.mark.gpu
 
 
-def run_case(w, mask, B, S, steps, max_prefill_tokens=None, check_cache=True):
+def run_case(w, mask, B, S, steps, max_prefill_tokens=None, check_cache=True, tuning=None):
     p = Pair(w, mask=mask, B=B, max_len=S + steps, max_prefill_tokens=max_prefill_tokens)
+    if tuning:
+        p.stack.set_tuning(**tuning)
     tol = TOL[w.dtype]
     got, ref, syncs = p.prefill(S)
     assert got.shape == ref.shape
