@@ -887,9 +887,14 @@ template <typename T, int D, int GT> cudaError_t launch_ring(const AttnArgs &a, 
 // rows of an m16n8k16 MMA: S[heads x 16 tokens] = Q K^T and O[heads x 128] += P V per page.
 // Pages arrive through TMA tensor copies (4 boxes of 64 dims x 16 tokens per page: K and V,
 // low and high half of the head dimension) in the 128-byte swizzle that ldmatrix reads without
-// bank conflicts.  Warp roles, page ring, split merge: as in the bulk-copy kernel.
-// DENSE: compiled for four resident blocks per SM instead of three (96 registers), taken by the launcher where it
-// saves a wave.
+// bank conflicts.  Warp roles and split merge: as in the bulk-copy kernel.  The page ring has more slots than
+// compute warps (six or eight for four warps): page i goes to slot i % R and to warp i % 4, so a warp's next page is
+// on its way while it works on the current one - with one slot per warp every page would cost a full memory latency.
+// The warps' partial outputs are merged through the ring's own bytes once every page has been read.
+// DENSE: compiled for four resident blocks per SM instead of three (96 registers, six slots instead of eight), taken
+// by the launcher where it saves a wave.
+template <bool DENSE> struct DecodeMmaRing { static constexpr int SLOTS = DENSE ? 6 : 8; };
+
 template <int GT, bool DENSE>
 __global__ void __launch_bounds__(160, DENSE ? 4 : 3) decode_attention_mma_kernel(const __grid_constant__ CUtensorMap tm_k,
                                                                    const __grid_constant__ CUtensorMap tm_v, AttnArgs a)
@@ -899,13 +904,14 @@ __global__ void __launch_bounds__(160, DENSE ? 4 : 3) decode_attention_mma_kerne
     using fa::ldsm_x4_t;
     using fa::mma_bf16;
     using fa::pack_bf16;
-    constexpr int D = 128, BLK = 16, R = 4, SUB = 2048 /* 16 tokens x 64 dims */, SLOT = 4 * SUB;
+    constexpr int D = 128, BLK = 16, R = DecodeMmaRing<DENSE>::SLOTS, SUB = 2048 /* 16 tokens x 64 dims */, SLOT = 4 * SUB;
+    static_assert(R * SLOT >= 4 * GT * D * 4 + 4 * GT * 2 * 4, "the merge area lives in the ring");
     extern __shared__ uint8_t smem_dyn[];
     const uint32_t ring = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     uint8_t *gen = smem_dyn + (ring - smem_u32(smem_dyn));
-    float(*sm_o)[GT][D] = (float(*)[GT][D])(gen + R * SLOT);
-    float(*sm_ml)[GT][2] = (float(*)[GT][2])(gen + R * SLOT + 4 * GT * D * 4);
-    uint8_t *tail = gen + R * SLOT + 4 * GT * D * 4 + 4 * GT * 2 * 4;
+    float(*sm_o)[GT][D] = (float(*)[GT][D])gen; // over the ring, after its last read
+    float(*sm_ml)[GT][2] = (float(*)[GT][2])(gen + 4 * GT * D * 4);
+    uint8_t *tail = gen + R * SLOT;
     const uint32_t bars = smem_u32(tail);             // full[R], empty[R]
     int *sm_bt = (int *)(tail + 2 * R * 8);
     volatile int *abort_flag = (volatile int *)(sm_bt + DECODE_MAX_PAGES_PER_BLOCK);
@@ -968,87 +974,95 @@ __global__ void __launch_bounds__(160, DENSE ? 4 : 3) decode_attention_mma_kerne
     if (threadIdx.x == 0) SPD_TRACE_EVENT(TRK_ATTN, TR_DEP_DONE);
 
     if (warp < 4) {
-        // A fragments of Q: MMA row g = query head hq0 + g (rows >= GT are padding)
-        uint32_t qf[8][4];
+        // Tokens are the MMA rows and the group's query heads its 8 columns, so that no row of a 16 x 8 tile is
+        // padding: S^T[16 tokens x 8 heads] = K Q^T and O^T[128 dims x 8 heads] += V^T P^T, 8 + 8 MMAs per page.
+        // B fragments of Q^T: column g = query head hq0 + g (columns >= GT are padding), rows = 16 dims per step.
+        uint32_t qb[8][2];
         {
             const bf16 *qp = (const bf16 *)a.q + ((long)b * a.n_q_heads + hq0 + g) * D;
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk) {
-                qf[kk][0] = g < GT ? *(const uint32_t *)(qp + kk * 16 + 2 * t4) : 0u;
-                qf[kk][2] = g < GT ? *(const uint32_t *)(qp + kk * 16 + 8 + 2 * t4) : 0u;
-                qf[kk][1] = 0u;
-                qf[kk][3] = 0u;
+                qb[kk][0] = g < GT ? *(const uint32_t *)(qp + kk * 16 + 2 * t4) : 0u;
+                qb[kk][1] = g < GT ? *(const uint32_t *)(qp + kk * 16 + 8 + 2 * t4) : 0u;
             }
         }
-        float o[16][4];
+        // this lane's share of O^T: dims dp*16 + g (o[dp][0..1]) and dp*16 + g + 8 (o[dp][2..3]), heads 2*t4 + {0,1}
+        float o[8][4];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
-        float m_run = -INFINITY, l_run = 0.f;
+        for (int i = 0; i < 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+        float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f}; // heads 2*t4 + {0,1}; l_run: this lane's tokens only
         const float sc = rsqrtf((float)D) * 1.4426950408889634f;
         for (int pi = warp; pi < n_pages; pi += 4) {
             const int s = pi % R;
+            // Where the slots are not a multiple of the warps, the page that had this slot before (pi - R) belonged to
+            // another warp, which may be behind: a parity wait can only tell a phase from the one next to it, so wait
+            // until that page has been released (the slot's "empty" phase) before waiting for this one to be full.
+            if (R % 4 != 0 && pi >= R && !mbar_wait(empty_bar(s), ((pi / R) & 1) ^ 1, a.err, abort_flag)) break;
             if (!mbar_wait(full_bar(s), (pi / R) & 1, a.err, abort_flag)) break;
             const uint32_t kb = ring + s * SLOT, vb = kb + 2 * SUB;
-            float sv[2][4];
-#pragma unroll
-            for (int i = 0; i < 2; ++i) { sv[i][0] = sv[i][1] = sv[i][2] = sv[i][3] = 0.f; }
+            float sv[4] = {0.f, 0.f, 0.f, 0.f}; // tokens g (sv[0..1]) and g + 8 (sv[2..3]) x heads 2*t4 + {0,1}
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk) {
-                uint32_t kf[4];
-                const int r = (lane & 7) + ((lane >> 4) << 3), c = (kk & 3) * 2 + ((lane >> 3) & 1);
+                uint32_t kf[4]; // A fragment: tokens x 16 dims
+                const int r = (lane & 7) + (((lane >> 3) & 1) << 3), c = (kk & 3) * 2 + (lane >> 4);
                 ldsm_x4(kf, kb + (kk >> 2) * SUB + r * 128 + ((c ^ (r & 7)) << 4));
-                mma_bf16(sv[0], qf[kk], kf[0], kf[1]);
-                mma_bf16(sv[1], qf[kk], kf[2], kf[3]);
+                mma_bf16(sv, kf, qb[kk][0], qb[kk][1]);
             }
-            // this thread's row g: tokens nt*8 + 2*t4 + {0,1}
             const int tbase = (p0 + pi) * BLK;
-            float pv[2][2], mx = m_run;
+            const bool ok0 = tbase + g < ctx, ok1 = tbase + g + 8 < ctx;
+            float pv[2][2], corr[2]; // [head][token g / g + 8]
 #pragma unroll
-            for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const bool ok = tbase + nt * 8 + 2 * t4 + e < ctx;
-                    pv[nt][e] = ok ? sv[nt][e] * sc : -INFINITY;
-                    mx = fmaxf(mx, pv[nt][e]);
-                }
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-            const float base = mx == -INFINITY ? 0.f : mx;
-            const float corr = m_run == -INFINITY ? 0.f : exp2f(m_run - base);
-            m_run = mx;
-            float rs = 0.f;
-#pragma unroll
-            for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-                for (int e = 0; e < 2; ++e) { pv[nt][e] = exp2f(pv[nt][e] - base); rs += pv[nt][e]; }
-            l_run = l_run * corr + rs;
-            uint32_t pf[4];
-            pf[0] = pack_bf16(pv[0][0], pv[0][1]);
-            pf[1] = 0u;
-            pf[2] = pack_bf16(pv[1][0], pv[1][1]);
-            pf[3] = 0u;
-#pragma unroll
-            for (int dt = 0; dt < 16; ++dt) { o[dt][0] *= corr; o[dt][1] *= corr; }
+            for (int e = 0; e < 2; ++e) {
+                pv[e][0] = ok0 ? sv[e] * sc : -INFINITY;
+                pv[e][1] = ok1 ? sv[2 + e] * sc : -INFINITY;
+                float mx = fmaxf(m_run[e], fmaxf(pv[e][0], pv[e][1]));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+                const float base = mx == -INFINITY ? 0.f : mx;
+                corr[e] = m_run[e] == -INFINITY ? 0.f : exp2f(m_run[e] - base);
+                m_run[e] = mx;
+                pv[e][0] = exp2f(pv[e][0] - base);
+                pv[e][1] = exp2f(pv[e][1] - base);
+                l_run[e] = l_run[e] * corr[e] + pv[e][0] + pv[e][1];
+            }
+            // P^T as the B operand (16 tokens x 8 heads): the accumulator layout holds (token g; heads 2*t4, 2*t4+1),
+            // the operand wants (head g; tokens 2*t4, 2*t4+1) - an 8 x 8 transpose across the warp per token half
+            uint32_t pb0, pb1;
+            {
+                const uint32_t lo = pack_bf16(pv[0][0], pv[1][0]), hi = pack_bf16(pv[0][1], pv[1][1]);
+                asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(pb0) : "r"(lo));
+                asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(pb1) : "r"(hi));
+            }
 #pragma unroll
             for (int dp = 0; dp < 8; ++dp) {
-                uint32_t vf[4];
-                const int r = (lane & 7) + (((lane >> 3) & 1) << 3), c = (dp & 3) * 2 + (lane >> 4);
+                o[dp][0] *= corr[0]; o[dp][1] *= corr[1]; o[dp][2] *= corr[0]; o[dp][3] *= corr[1];
+                uint32_t vf[4]; // A fragment of V^T: 16 dims x 16 tokens, read transposed from the [token][dim] page
+                const int r = (lane & 7) + ((lane >> 4) << 3), c = (dp & 3) * 2 + ((lane >> 3) & 1);
                 ldsm_x4_t(vf, vb + (dp >> 2) * SUB + r * 128 + ((c ^ (r & 7)) << 4));
-                mma_bf16(o[2 * dp], pf, vf[0], vf[1]);
-                mma_bf16(o[2 * dp + 1], pf, vf[2], vf[3]);
+                mma_bf16(o[dp], vf, pb0, pb1);
             }
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(s)) : "memory");
         }
-        l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-        l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-        if (g < GT) {
 #pragma unroll
-            for (int dt = 0; dt < 16; ++dt) {
-                sm_o[warp][g][dt * 8 + 2 * t4] = o[dt][0];
-                sm_o[warp][g][dt * 8 + 2 * t4 + 1] = o[dt][1];
+        for (int e = 0; e < 2; ++e) {
+            l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 4);
+            l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 8);
+            l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 16);
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory"); // every compute warp is done with the ring: the merge area may overwrite it
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int h = 2 * t4 + e;
+            if (h < GT) {
+#pragma unroll
+                for (int dp = 0; dp < 8; ++dp) {
+                    sm_o[warp][h][dp * 16 + g] = o[dp][e];
+                    sm_o[warp][h][dp * 16 + g + 8] = o[dp][2 + e];
+                }
+                if (g == 0) { sm_ml[warp][h][0] = m_run[e]; sm_ml[warp][h][1] = l_run[e]; }
             }
-            if (t4 == 0) { sm_ml[warp][g][0] = m_run; sm_ml[warp][g][1] = l_run; }
         }
     }
     __syncthreads();
@@ -1059,10 +1073,14 @@ __global__ void __launch_bounds__(160, DENSE ? 4 : 3) decode_attention_mma_kerne
 
 template <int GT, bool DENSE> cudaError_t launch_decode_mma_as(const AttnArgs &a, cudaStream_t st)
 {
-    constexpr int SMEM = 1024 + 4 * 8192 + 4 * GT * 128 * 4 + 4 * GT * 2 * 4 + 2 * 4 * 8 + (DECODE_MAX_PAGES_PER_BLOCK + 2 + 2 * GT) * 4;
+    constexpr int R = DecodeMmaRing<DENSE>::SLOTS;
+    constexpr int SMEM = 1024 + R * 8192 + 2 * R * 8 + (DECODE_MAX_PAGES_PER_BLOCK + 2 + 2 * GT) * 4;
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(decode_attention_mma_kernel<GT, DENSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(decode_attention_mma_kernel<GT, DENSE>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 (int)cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }

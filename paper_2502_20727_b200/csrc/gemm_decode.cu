@@ -55,6 +55,7 @@ template <int BN, int ST> struct DCfg {
 
 struct DecTile {
     int z, wt, wi, w_row0, t_row0, split, rank, P;
+    int CL, zs; // blocks per cluster; partial planes per block (P = CL * zs planes add up to one output tile)
 };
 
 // Launcher-filled tiling constants travel behind the public arguments.
@@ -62,7 +63,8 @@ struct DecLaunch {
     DecGemmArgs g;
     int w_tiles_per_batch;
     int tile_start[3];
-    int P; // K ranges per output tile = cluster size = gridDim.z
+    int P;  // partial planes per output tile (K ranges, shard slices)
+    int zs; // planes one block computes one after the other (row-split projection: shard slices); cluster size = gridDim.z = P / zs
 };
 
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
@@ -97,14 +99,28 @@ __device__ __forceinline__ void store_bf16x4(bf16 *p, float4 v, float4 gn)
 }
 
 // The partials of token j, columns 4*lane..4*lane+3, from every block of the cluster (y[s] = range s).
-__device__ __forceinline__ void load_partials(float4 (&y)[MAX_P], const float *S, int j, int lane, int P)
+// Plane s lies in block s / zs of the cluster, `plane_bytes` after that block's plane s - 1 (zs > 1).
+__device__ __forceinline__ void load_partials(float4 (&y)[MAX_P], const float *S, int j, int lane, const DecTile &t, int plane_bytes)
 {
     const float *src = S + j * 128 + 4 * lane;
-    if (P == 1) { y[0] = *(const float4 *)src; return; }
+    if (t.P == 1) { y[0] = *(const float4 *)src; return; }
     const uint32_t a = smem_u32(src);
+    if (t.zs == 1) {
 #pragma unroll
-    for (int s = 0; s < MAX_P; ++s)
-        if (s < P) y[s] = ld_peer4(a, (uint32_t)s);
+        for (int s = 0; s < MAX_P; ++s)
+            if (s < t.P) y[s] = ld_peer4(a, (uint32_t)s);
+    } else {
+#pragma unroll
+        for (int s = 0; s < MAX_P; ++s)
+            if (s < t.P) y[s] = ld_peer4(a + (uint32_t)((s % t.zs) * plane_bytes), (uint32_t)(s / t.zs));
+    }
+}
+
+// How many tokens of its tile this block finishes: tokens rank, rank + CL, ... below the tile's (ragged) end.
+template <int BN> __device__ __forceinline__ int my_token_count(const DecGemmArgs &g, const DecTile &t)
+{
+    const int lim = g.t_rows - t.t_row0 < BN ? g.t_rows - t.t_row0 : BN;
+    return lim > t.rank ? (lim - t.rank + t.CL - 1) / t.CL : 0;
 }
 
 // rstd of the tile's tokens from the partial sums of squares, by the 128 epilogue threads:
@@ -147,11 +163,12 @@ template <int BN>
 __device__ __forceinline__ void gather_my_tokens(const DecGemmArgs &g, const DecTile &t, const float *S, float *Gb)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int q = warp;; q += 4) {
-        const int j = t.rank + t.P * q;
-        if (j >= BN || t.t_row0 + j >= g.t_rows) break;
+    const int mine = my_token_count<BN>(g, t);
+#pragma unroll 2
+    for (int q = warp; q < mine; q += 4) {
+        const int j = t.rank + t.CL * q;
         float4 y[MAX_P];
-        load_partials(y, S, j, lane, t.P);
+        load_partials(y, S, j, lane, t, BN * 128 * 4);
         float4 v = y[0];
 #pragma unroll
         for (int s = 1; s < MAX_P; ++s)
@@ -169,14 +186,20 @@ __device__ __forceinline__ void epilogue_qkv(const DecGemmArgs &g, const DecTile
     const int row = t.w_row0 + r, head = row / d + t.z * (g.w_rows[t.wi] / d), jd = row % d, nq = g.n_q_heads;
     const bool row_valid = row < g.w_rows[t.wi];
     const bool rot = t.wi < 2 && g.rope != nullptr;
-    // the rotary factors do not depend on the gather: request them first
-    float2 cs[4];
+    // The rotary factors do not depend on the gather: the first chunk is requested before it, and every later chunk
+    // while the chunk before it is written, so that the loop never waits for a load it has only just issued.
+    const int mine = my_token_count<BN>(g, t);
+    constexpr int CH = 8;
+    const int jj = jd < half ? jd : jd - half;
+    float2 nxt[CH];
+    auto fetch = [&](int q0) {
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        const int m = t.t_row0 + t.rank + t.P * q;
-        cs[q] = make_float2(1.f, 0.f);
-        if (rot && row_valid && t.rank + t.P * q < BN && m < g.t_rows) cs[q] = g.rope[(long)m * half + (jd < half ? jd : jd - half)];
-    }
+        for (int u = 0; u < CH; ++u) {
+            nxt[u] = make_float2(1.f, 0.f);
+            if (rot && row_valid && q0 + u < mine) nxt[u] = g.rope[(long)(t.t_row0 + t.rank + t.CL * (q0 + u)) * half + jj];
+        }
+    };
+    fetch(0);
     gather_my_tokens<BN>(g, t, S, Gb);
     epi_sync();
     if (!row_valid) return;
@@ -188,20 +211,28 @@ __device__ __forceinline__ void epilogue_qkv(const DecGemmArgs &g, const DecTile
         wg = g.ln_wg[vrow];
         wb = g.ln_wb[vrow];
     }
-    for (int q = 0;; ++q) {
-        const int j = t.rank + t.P * q, m = t.t_row0 + j;
-        if (j >= BN || m >= g.t_rows) break;
-        float v = (Gb[q * 128 + r] - sm_mu[j] * wg) * sm_rstd[j] + wb;
-        if (rot) {
-            const float2 c = q < 4 ? cs[q < 4 ? q : 0] : g.rope[(long)m * half + (jd < half ? jd : jd - half)];
-            const float o = Gb[q * 128 + partner] * sm_rstd[j];
-            v = jd < half ? v * c.x - o * c.y : v * c.x + o * c.y;
-        }
-        if (t.wi == 0) {
-            ((bf16 *)g.q_out)[((long)m * nq + head) * d + jd] = __float2bfloat16_rn(v);
-        } else {
-            const long off = sm_kvoff[j];
-            if (off >= 0) ((bf16 *)(t.wi == 1 ? g.k_pages : g.v_pages))[off + (long)head * g.pt.block * d + jd] = __float2bfloat16_rn(v);
+    bf16 *const dst = t.wi == 0 ? (bf16 *)g.q_out : (bf16 *)(t.wi == 1 ? g.k_pages : g.v_pages);
+    for (int q0 = 0; q0 < mine; q0 += CH) {
+        float2 cur[CH];
+#pragma unroll
+        for (int u = 0; u < CH; ++u) cur[u] = nxt[u];
+        if (rot && q0 + CH < mine) fetch(q0 + CH);
+#pragma unroll
+        for (int u = 0; u < CH; ++u) {
+            const int q = q0 + u;
+            if (q >= mine) break;
+            const int j = t.rank + t.CL * q, m = t.t_row0 + j;
+            float v = (Gb[q * 128 + r] - sm_mu[j] * wg) * sm_rstd[j] + wb;
+            if (rot) {
+                const float o = Gb[q * 128 + partner] * sm_rstd[j];
+                v = jd < half ? v * cur[u].x - o * cur[u].y : v * cur[u].x + o * cur[u].y;
+            }
+            if (t.wi == 0) {
+                dst[((long)m * nq + head) * d + jd] = __float2bfloat16_rn(v);
+            } else {
+                const long off = sm_kvoff[j];
+                if (off >= 0) dst[off + (long)head * g.pt.block * d + jd] = __float2bfloat16_rn(v);
+            }
         }
     }
 }
@@ -215,7 +246,7 @@ __device__ __forceinline__ void epilogue_gateup(const DecGemmArgs &g, const DecT
     if (g.fc1_only) {
         // block with bias: the tile holds 128 consecutive rows of fc1; LayerNorm folded in, bias, ReLU
         for (int idx = threadIdx.x;; idx += 128) {
-            const int q = idx >> 6, rr = 2 * (idx & 63), j = t.rank + t.P * q, m = t.t_row0 + j, f = t.w_row0 + rr;
+            const int q = idx >> 6, rr = 2 * (idx & 63), j = t.rank + t.CL * q, m = t.t_row0 + j, f = t.w_row0 + rr;
             if (j >= BN || m >= g.t_rows) break;
             if (f >= g.Fs) continue;
             const float rs = sm_rstd[j], mu = sm_mu[j];
@@ -228,7 +259,7 @@ __device__ __forceinline__ void epilogue_gateup(const DecGemmArgs &g, const DecT
     }
     // two FFN columns per thread: 32 threads cover the tile's 64 columns of one token
     for (int idx = threadIdx.x;; idx += 128) {
-        const int q = idx >> 5, rr = 2 * (idx & 31), j = t.rank + t.P * q, m = t.t_row0 + j, f = t.w_row0 + rr;
+        const int q = idx >> 5, rr = 2 * (idx & 31), j = t.rank + t.CL * q, m = t.t_row0 + j, f = t.w_row0 + rr;
         if (j >= BN || m >= g.t_rows) break;
         if (f >= g.Fs) continue;
         const float rs = sm_rstd[j];
@@ -239,12 +270,40 @@ __device__ __forceinline__ void epilogue_gateup(const DecGemmArgs &g, const DecT
     }
 }
 
+// xpre[u] for a run-time u in 0..3 without indexing the register array.
+__device__ __forceinline__ float4 pick4(const float4 (&v)[4], int u)
+{
+    float4 r = v[0];
+    if (u == 1) r = v[1];
+    if (u == 2) r = v[2];
+    if (u == 3) r = v[3];
+    return r;
+}
+
+// Eight per-lane values, each to be summed over the warp: instead of eight butterflies (40 shuffles) the lanes swap
+// halves of the value list while they halve the lane distance (4 + 2 + 1 shuffles), then two plain steps.  Returns, in
+// every lane, the warp total of v[4 * bit4(lane) + 2 * bit3(lane) + bit2(lane)].
+__device__ __forceinline__ float warp_sum8(const float (&v)[8], int lane)
+{
+    const bool h16 = (lane & 16) != 0, h8 = (lane & 8) != 0, h4 = (lane & 4) != 0;
+    float a[4], b[2];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) a[i] = (h16 ? v[i + 4] : v[i]) + __shfl_xor_sync(0xffffffffu, h16 ? v[i] : v[i + 4], 16);
+#pragma unroll
+    for (int i = 0; i < 2; ++i) b[i] = (h8 ? a[i + 2] : a[i]) + __shfl_xor_sync(0xffffffffu, h8 ? a[i] : a[i + 2], 8);
+    float w = (h4 ? b[1] : b[0]) + __shfl_xor_sync(0xffffffffu, h4 ? b[0] : b[1], 4);
+    w += __shfl_xor_sync(0xffffffffu, w, 2);
+    w += __shfl_xor_sync(0xffffffffu, w, 1);
+    return w;
+}
+
 // Residual stream out, gain-scaled bf16 copy (the next GEMM's input) and the tile's partial sums
 // of squares.  spd_groups (o_proj of an SPD block): range i of the cluster is emulated device i,
 // which only ever sees its own partial attention output Y_i (R_i = X + Y_i), while the carried
 // residual collects every Y_i.
 template <int BN>
-__device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const DecTile &t, const float *S, bool spd_groups)
+__device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const DecTile &t, const float *S, bool spd_groups,
+                                                  const float4 (&xpre)[4])
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n = t.w_row0 + 4 * lane, H = g.H;
@@ -267,18 +326,22 @@ __device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const De
     auto sum4 = [](float4 v) { return v.x + v.y + v.z + v.w; };
     if (spd_groups) {
         const int rows = (g.t_rows - t.t_row0 < BN ? g.t_rows - t.t_row0 : BN) - t.rank; // this block's tokens: every P-th of them
-        if (rows > 3 * t.P) {
+        if (rows > 3 * t.CL) {
             // Four tokens or more: one token per warp at a time, the devices of a token in turn (one gather of the
-            // partials per token instead of one per warp and token).
-            for (int q = warp;; q += 4) {
-                const int j = t.rank + t.P * q, m = t.t_row0 + j;
-                if (j >= BN || m >= g.t_rows) break;
+            // partials per token instead of one per warp and token); the per-device row sums are reduced together.
+            const int mine = my_token_count<BN>(g, t);
+            const int dev_of_lane = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
+            for (int q = warp, u = 0; q < mine; q += 4, ++u) {
+                const int j = t.rank + t.CL * q, m = t.t_row0 + j;
                 const long idx = (long)m * H + n;
                 float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (valid) { x = *(const float4 *)(g.res_in + idx); add4(x, bias); }
+                if (valid) { x = u < 4 ? pick4(xpre, u) : *(const float4 *)(g.res_in + idx); add4(x, bias); }
                 float4 y[MAX_P];
-                load_partials(y, S, j, lane, t.P);
+                load_partials(y, S, j, lane, t, BN * 128 * 4);
                 float4 tot = make_float4(0.f, 0.f, 0.f, 0.f), yi = make_float4(0.f, 0.f, 0.f, 0.f);
+                float sq[8], sm[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) sq[i] = sm[i] = 0.f;
                 int cnt = 0, i = 0;
 #pragma unroll
                 for (int s = 0; s < MAX_P; ++s) {
@@ -289,15 +352,19 @@ __device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const De
                     float4 ri = x;
                     add4(ri, yi);
                     if (valid && g.hg) store_bf16x4((bf16 *)g.hg + (long)i * g.hg_stride + idx, ri, gn);
-                    const float sq = warp_sum(valid ? sq4(ri) : 0.f);
-                    if (lane == 0 && g.ss_out) g.ss_out[((long)t.wt * G + i) * g.Mcap + m] = sq;
-                    if (g.sum_out) {
-                        const float sm = warp_sum(valid ? sum4(ri) : 0.f);
-                        if (lane == 0) g.sum_out[((long)t.wt * G + i) * g.Mcap + m] = sm;
-                    }
+                    // device i's slot: i only grows with s, so after unrolling every index below is a constant
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        if (e == i) { sq[e] = valid ? sq4(ri) : 0.f; sm[e] = valid ? sum4(ri) : 0.f; }
                     yi = make_float4(0.f, 0.f, 0.f, 0.f);
                     cnt = 0;
                     ++i;
+                }
+                const float sqt = warp_sum8(sq, lane);
+                if ((lane & 3) == 0 && dev_of_lane < G && g.ss_out) g.ss_out[((long)t.wt * G + dev_of_lane) * g.Mcap + m] = sqt;
+                if (g.sum_out) {
+                    const float smt = warp_sum8(sm, lane);
+                    if ((lane & 3) == 0 && dev_of_lane < G) g.sum_out[((long)t.wt * G + dev_of_lane) * g.Mcap + m] = smt;
                 }
                 add4(x, tot);
                 if (valid && g.res_out) *(float4 *)(g.res_out + idx) = x;
@@ -307,13 +374,13 @@ __device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const De
         // All four warps work on the same token; warp w finishes devices w, w+4 (ranges i*per .. i*per+per-1 are
         // device i), so that the per-device stores and reductions of a block with few tokens run side by side.
         for (int q = 0;; ++q) {
-            const int j = t.rank + t.P * q, m = t.t_row0 + j;
+            const int j = t.rank + t.CL * q, m = t.t_row0 + j;
             if (j >= BN || m >= g.t_rows) break;
             const long idx = (long)m * H + n;
             float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
             if (valid) { x = *(const float4 *)(g.res_in + idx); add4(x, bias); }
             float4 y[MAX_P];
-            load_partials(y, S, j, lane, t.P);
+            load_partials(y, S, j, lane, t, BN * 128 * 4);
             float4 tot = make_float4(0.f, 0.f, 0.f, 0.f), yi = make_float4(0.f, 0.f, 0.f, 0.f);
             int cnt = 0, i = 0;
 #pragma unroll
@@ -342,14 +409,14 @@ __device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const De
         }
         return;
     }
-    for (int q = warp;; q += 4) {
-        const int j = t.rank + t.P * q, m = t.t_row0 + j;
-        if (j >= BN || m >= g.t_rows) break;
+    const int mine = my_token_count<BN>(g, t);
+    for (int q = warp, u = 0; q < mine; q += 4, ++u) {
+        const int j = t.rank + t.CL * q, m = t.t_row0 + j;
         const long idx = (long)m * H + n;
         float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (valid) { x = *(const float4 *)(g.res_in + idx); add4(x, bias); }
+        if (valid) { x = u < 4 ? pick4(xpre, u) : *(const float4 *)(g.res_in + idx); add4(x, bias); }
         float4 y[MAX_P];
-        load_partials(y, S, j, lane, t.P);
+        load_partials(y, S, j, lane, t, BN * 128 * 4);
         float4 tot = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int s = 0; s < MAX_P; ++s)
@@ -426,11 +493,11 @@ __device__ __forceinline__ void epilogue_resid_tp(const DecGemmArgs &g, const De
         }
     };
     for (int q = warp;; q += 4) {
-        const int j = t.rank + t.P * q, m = t.t_row0 + j;
+        const int j = t.rank + t.CL * q, m = t.t_row0 + j;
         if (j >= BN || m >= g.t_rows) break;
         const long idx = (long)m * H + n;
         float4 y[MAX_P];
-        load_partials(y, S, j, lane, t.P);
+        load_partials(y, S, j, lane, t, BN * 128 * 4);
         float4 p = y[0];
 #pragma unroll
         for (int s = 1; s < MAX_P; ++s)
@@ -471,7 +538,7 @@ __device__ __forceinline__ void epilogue_resid_tp(const DecGemmArgs &g, const De
     epi_sync();
     if (*abort_flag) return;
     for (int q = warp;; q += 4) {
-        const int j = t.rank + t.P * q, m = t.t_row0 + j;
+        const int j = t.rank + t.CL * q, m = t.t_row0 + j;
         if (j >= BN || m >= g.t_rows) break;
         float4 tot = make_float4(0.f, 0.f, 0.f, 0.f);
         if (valid)
@@ -506,10 +573,14 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
     const uint32_t tmem_full_bar = bars + 8u * (2 * C::STAGES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float4 xpre[4] = {}; // epilogue warps of the residual tails: residual rows fetched ahead
     DecTile t;
     t.P = L.P;
-    t.rank = t.P > 1 ? (int)cluster_rank() : 0;
-    if (g.z_is_plane) { t.z = t.rank / g.splits; t.split = t.rank % g.splits; t.wt = blockIdx.x; }
+    t.zs = L.zs;
+    t.CL = L.P / L.zs;
+    t.rank = t.CL > 1 ? (int)cluster_rank() : 0;
+    // zs > 1 (whole shard slices only, splits == 1): this block computes planes rank * zs ... rank * zs + zs - 1
+    if (g.z_is_plane) { t.z = t.zs > 1 ? t.rank * t.zs : t.rank / g.splits; t.split = t.zs > 1 ? 0 : t.rank % g.splits; t.wt = blockIdx.x; }
     else { t.z = blockIdx.x / L.w_tiles_per_batch; t.split = t.rank; t.wt = blockIdx.x % L.w_tiles_per_batch; }
     t.wi = (SUB == 2) ? 0 : ((t.wt >= L.tile_start[2]) ? 2 : ((t.wt >= L.tile_start[1]) ? 1 : 0));
     t.w_row0 = (t.wt - L.tile_start[t.wi]) * ((EPI == EPI_GATEUP && g.fc1_only) ? BM : ROWS);
@@ -518,11 +589,14 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
     const int kb_begin = (int)((long)g.num_kb * t.split / g.splits);
     const int kb_end = (int)((long)g.num_kb * (t.split + 1) / g.splits);
     const int n_kb = kb_end - kb_begin;
+    const int n_it = n_kb * t.zs; // ring iterations: the K blocks of plane 0, then those of plane 1, ...
+    const uint32_t tmem_cols = (uint32_t)(BN * t.zs < 32 ? 32 : BN * t.zs); // zs is 1 or 2: a power of two
 
     pdl_launch_dependents();
-    const int a_z = g.w_batched ? t.z : 0, b_z = g.t_batched ? t.z : 0;
+    const int az0 = g.w_batched ? t.z : 0, bz0 = g.t_batched ? t.z : 0;
     const uint64_t stream_once = policy_evict_first();
-    auto load_w = [&](int s, int kx) {
+    auto load_w = [&](int s, int it) {
+        const int kx = (kb_begin + it % n_kb) * BK, a_z = az0 + it / n_kb;
         const uint32_t sa = base + s * C::STAGE_BYTES;
         if (SUB == 1) tma_load_3d_hint(sa, tm_w, kx, t.w_row0, a_z, full_bar(s), stream_once);
         else {
@@ -531,7 +605,7 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
             else tma_load_3d_hint(sa + ROWS * BK * 2, &tm_w1, kx, t.w_row0, a_z, full_bar(s), stream_once);
         }
     };
-    const int pre = n_kb < C::STAGES ? n_kb : C::STAGES;
+    const int pre = n_it < C::STAGES ? n_it : C::STAGES;
     if (warp == 4 && lane == 0) {
         // The TMA thread sets up the barriers itself and requests the first ring of weight tiles
         // at once: weights do not depend on the preceding kernel, and they need neither the
@@ -548,18 +622,18 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_t) : "memory");
         for (int i = 0; i < pre; ++i) {
             mbar_expect_tx(full_bar(i), C::STAGE_BYTES);
-            load_w(i, (kb_begin + i) * BK);
+            load_w(i, i);
         }
         // optionally the K blocks after the ring are pulled into L2
         const int pf_end = n_kb < pre + g.l2_prefetch_kb ? n_kb : pre + g.l2_prefetch_kb;
         for (int i = pre; i < pf_end; ++i) {
-            const int kx = (kb_begin + i) * BK;
+            const int kx = (kb_begin + i) * BK, a_z = az0;
             if (SUB == 1) tma_prefetch_l2_3d(tm_w, kx, t.w_row0, a_z);
             else { tma_prefetch_l2_3d(&tm_w0, kx, t.w_row0, a_z); tma_prefetch_l2_3d(g.fc1_only ? &tm_w0 : &tm_w1, kx, t.w_row0 + (g.fc1_only ? ROWS : 0), a_z); }
         }
     }
     if (warp == 5) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::TMEM_COLS) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -571,31 +645,32 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
         if (lane == 0) {
             pdl_wait();
             SPD_TRACE_EVENT(EPI, TR_DEP_DONE);
-            for (int i = 0; i < n_kb; ++i) {
+            for (int i = 0; i < n_it; ++i) {
                 const int s = i % C::STAGES;
-                const int kx = (kb_begin + i) * BK;
                 if (i >= pre) {
                     if (!mbar_wait(empty_bar(s), ((i / C::STAGES) & 1) ^ 1, g.err, abort_flag)) break;
                     mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
-                    load_w(s, kx);
+                    load_w(s, i);
                 }
-                tma_load_3d(base + s * C::STAGE_BYTES + C::A_BYTES, &tm_t, kx, t.t_row0, b_z, full_bar(s));
+                tma_load_3d(base + s * C::STAGE_BYTES + C::A_BYTES, &tm_t, (kb_begin + i % n_kb) * BK, t.t_row0, bz0 + i / n_kb, full_bar(s));
             }
         }
         __syncwarp();
     } else if (warp == 5) {
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc(BN);
-            for (int i = 0; i < n_kb; ++i) {
+            for (int i = 0; i < n_it; ++i) {
                 const int s = i % C::STAGES;
                 if (!mbar_wait(full_bar(s), (i / C::STAGES) & 1, g.err, abort_flag)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t sa = base + s * C::STAGE_BYTES, sb = sa + C::A_BYTES;
                 const uint64_t da = make_desc(sa), db = make_desc(sb);
+                const int kk = i % n_kb;
+                const uint32_t acc = tmem_acc + (uint32_t)((i / n_kb) * BN); // plane i / n_kb: its own accumulator columns
 #pragma unroll
                 for (int k = 0; k < BK / UMMA_K; ++k)
-                    umma(tmem_acc, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
-                         (i > 0 || k > 0) ? 1u : 0u);
+                    umma(acc, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
+                         (kk > 0 || k > 0) ? 1u : 0u);
                 umma_commit(empty_bar(s));
             }
             umma_commit(tmem_full_bar);
@@ -626,33 +701,43 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
             }
             sm_kvoff[threadIdx.x] = off;
         }
+        if (EPI == EPI_OPROJ || EPI == EPI_DOWN) {
+            // the residual rows this warp will finish first (tokens rank + CL * (warp + 4u)): requested while the weights stream
+            const int n = t.w_row0 + 4 * lane, mine = my_token_count<BN>(g, t);
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (n < g.H && warp + 4 * u < mine)
+                    xpre[u] = *(const float4 *)(g.res_in + (long)(t.t_row0 + t.rank + t.CL * (warp + 4 * u)) * g.H + n);
+        }
         // accumulator -> registers: warp w owns TMEM lanes [32w, 32w+32); thread r = accumulator row r
         const bool acc_ok = mbar_wait(tmem_full_bar, 0, g.err, abort_flag);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         __syncwarp();
         if (threadIdx.x == 0) SPD_TRACE_EVENT(EPI, TR_MAIN_DONE);
-        float acc[BN];
+        // The ring is free once the accumulators are complete (every TMA write has landed and every
+        // MMA has read its operands): park the partial tiles there, token-major, plane after plane.
+        for (int lp = 0; lp < t.zs; ++lp) {
+            float acc[BN];
 #pragma unroll
-        for (int c0 = 0; c0 < BN; c0 += 16) {
-            if (acc_ok) tmem_ld16(tmem_acc + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, acc + c0);
-            else {
+            for (int c0 = 0; c0 < BN; c0 += 16) {
+                if (acc_ok) tmem_ld16(tmem_acc + ((uint32_t)(warp * 32) << 16) + (uint32_t)(lp * BN + c0), acc + c0);
+                else {
 #pragma unroll
-                for (int i = 0; i < 16; ++i) acc[c0 + i] = 0.f;
+                    for (int i = 0; i < 16; ++i) acc[c0 + i] = 0.f;
+                }
             }
+            float *S = (float *)gen_base + lp * BN * 128;
+#pragma unroll
+            for (int j = 0; j < BN; ++j) S[j * 128 + threadIdx.x] = acc[j];
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        // The ring is free once the accumulator is complete (every TMA write has landed and every
-        // MMA has read its operands): park the partial tile there, token-major.
-        float *S = (float *)gen_base;
-#pragma unroll
-        for (int j = 0; j < BN; ++j) S[j * 128 + threadIdx.x] = acc[j];
     }
     // partial tiles of all ranges visible cluster-wide
-    if (t.P > 1) cluster_sync_all();
+    if (t.CL > 1) cluster_sync_all();
     else __syncthreads();
     if (warp == 5) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(C::TMEM_COLS) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(tmem_cols) : "memory");
     }
     if (warp < 4) {
         if (threadIdx.x == 0) SPD_TRACE_EVENT(EPI, TR_ARRIVED);
@@ -661,11 +746,11 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
         if (EPI == EPI_QKV) epilogue_qkv<BN>(g, t, S, Gb, sm_rstd, sm_mu, sm_kvoff);
         else if (EPI == EPI_GATEUP) epilogue_gateup<BN>(g, t, S, Gb, sm_rstd, sm_mu);
         else if (EPI == EPI_RESID_TP) epilogue_resid_tp<BN>(g, t, S, abort_flag);
-        else epilogue_residual<BN>(g, t, S, EPI == EPI_OPROJ && g.n_groups > 1);
+        else epilogue_residual<BN>(g, t, S, EPI == EPI_OPROJ && g.n_groups > 1, xpre);
         if (threadIdx.x == 0) { SPD_TRACE_EVENT(EPI, TR_END); stamp_exit(g.stamp); }
     }
     // no block may exit while a peer still reads its shared memory
-    if (t.P > 1) cluster_sync_all();
+    if (t.CL > 1) cluster_sync_all();
 }
 
 template <int BN, int EPI, int ST>
@@ -692,9 +777,9 @@ cudaError_t launch_cfg(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
     at[1].id = cudaLaunchAttributeClusterDimension;
     at[1].val.clusterDim.x = 1;
     at[1].val.clusterDim.y = 1;
-    at[1].val.clusterDim.z = (unsigned)L.P;
+    at[1].val.clusterDim.z = grid.z;
     cfg.attrs = at;
-    cfg.numAttrs = L.P > 1 ? 2 : 1;
+    cfg.numAttrs = grid.z > 1 ? 2 : 1;
     if (EPI == EPI_RESID_TP && L.g.tp.exchange && L.g.batches > 1) {
         // Several ranks in one launch: their blocks wait on one another, so all of them must be resident at once.
         // Blocks per SM from the kernel's own footprint (the launch takes the largest shared-memory carveout, which
@@ -723,16 +808,25 @@ cudaError_t launch_cfg(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
 }
 
 template <int EPI>
-cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, const DecLaunch &L, int tiles, cudaStream_t st)
+cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, const DecLaunch &L0, int tiles, cudaStream_t st)
 {
+    DecLaunch L = L0;
     const int bn = tc_token_box(true, L.g.t_rows);
-    dim3 grid(tiles * (L.g.z_is_plane ? 1 : L.g.batches), (L.g.t_rows + bn - 1) / bn, L.P);
+    const long n_sm = sm_count();
+    // Shard slices as planes: one slice per block is the default.  Where that launch would not be resident at once
+    // (two blocks per SM with a four-stage ring at 32- and 64-token tiles, three at 16), a block takes two slices one
+    // after the other into two accumulators: half the blocks, twice the K blocks each, one wave instead of two.
+    L.zs = 1;
+    if (L.g.z_is_plane && L.g.splits == 1 && L.g.batches % 2 == 0 && L.g.batches >= 4) {
+        const long one_each = (long)tiles * ((L.g.t_rows + bn - 1) / bn) * L.P;
+        if (L.g.planes_per_block == 2 || (L.g.planes_per_block == 0 && one_each > (bn == 16 ? 3 : 2) * n_sm)) L.zs = 2;
+    }
+    dim3 grid(tiles * (L.g.z_is_plane ? 1 : L.g.batches), (L.g.t_rows + bn - 1) / bn, L.P / L.zs);
     // ring depth at 16-token tiles: five stages for launches of at most two blocks per SM (they all stay resident and
     // each block has more in flight), four up to three blocks per SM, three beyond (four blocks per SM keep the
     // launch resident at once); four stages at 32- and 64-token tiles
     const long blocks = (long)grid.x * grid.y * grid.z;
     int stages = L.g.ring_stages;
-    const long n_sm = sm_count();
     if (stages == 0) stages = (bn == 16 && blocks > 3L * n_sm) ? 3 : ((bn == 16 && blocks <= 2L * n_sm) ? 5 : 4);
     // several ranks in one launch wait on one another: as many resident blocks as possible
     if (L.g.ring_stages == 0 && EPI == EPI_RESID_TP && L.g.tp.exchange && L.g.batches > 1) stages = 3;
@@ -850,6 +944,7 @@ cudaError_t launch_gemm_decode(DecEpilogue epi, const TcMap *const *weights, con
     }
     L.w_tiles_per_batch = tiles;
     L.P = P;
+    L.zs = 1;
     switch (epi) {
     case EPI_QKV: return launch_epi<EPI_QKV>(tw, tt, L, tiles, st);
     case EPI_OPROJ: return launch_epi<EPI_OPROJ>(tw, tt, L, tiles, st);

@@ -74,6 +74,8 @@ struct DecGemmArgs {
     int z_is_plane;        // o_proj: batch z is a K range of the same output tile (the K slice of shard z)
     int l2_prefetch_kb;    // K blocks of weights per thread block pulled into L2 before the dependency wait
     int ring_stages;       // stages of the operand ring (3, 4; 5 at 16-token tiles); 0 = chosen per launch
+    int planes_per_block;  // z_is_plane with splits == 1: shard slices one block computes one after the other, each into
+                           // its own accumulator columns (1 or 2; 0 = two where one per block would not be resident at once)
     int *err;
     unsigned long long *stamp; // launch stamp slot or null
     // ---- epilogue operands -----------------------------------------------------------

@@ -135,6 +135,7 @@ struct Ctx {
     int split_override[SITE_COUNT];
     int l2_prefetch_kb;          // K blocks per thread block prefetched into L2 by the decode GEMMs
     int ring_stages;             // decode GEMMs: stages of the operand ring (0 = per launch)
+    int oproj_planes;            // decode o_proj: shard slices per thread block (0 = per launch, 1, 2)
     int prefill_rescale_log2;    // tcgen05 prefill attention: growth of the row maximum (log2) that triggers a rescale
     int peer_wait_ms;            // rank mode: how long a rank waits for its peers' partial sums
     int prefill_group_m;         // prompt projections: token tiles per group of the tile order (0 = default)
@@ -808,6 +809,7 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
         g.t_rows = M; g.err = c->err; g.H = H; g.Mcap = Mc; g.batches = 1; g.n_weights = 1; g.n_groups = 1;
         g.l2_prefetch_kb = c->l2_prefetch_kb;
         g.ring_stages = c->ring_stages;
+        g.planes_per_block = c->oproj_planes;
         return g;
     };
     for (int l = 0; l < d.n_layers; ++l) {
@@ -917,6 +919,7 @@ int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, 
         g.t_rows = M; g.err = c->err; g.H = H; g.Mcap = Mb; g.batches = nl; g.w_batched = 1; g.t_batched = 1;
         g.n_weights = 1; g.n_groups = 1;
         g.ring_stages = c->ring_stages;
+        g.planes_per_block = c->oproj_planes;
         g.tp.on = 1; g.tp.T = tp.T; g.tp.rank_base = tp.rank_base; g.tp.z_stride = tp.z_stride;
         g.tp.step = (const unsigned *)(r0 + TL.step);
         g.tp.wait_ns = (unsigned long long)c->peer_wait_ms * 1000000ull;
@@ -1523,6 +1526,7 @@ int spd_create(const spd_dims *dims, const uint8_t *sync_mask, const spd_layer *
     c.prefill_pairs = 1;
     c.prefill_group_m = 0;
     c.ring_stages = 0;
+    c.oproj_planes = 0;
     c.launches_last = 0;
     c.tp.on = false;
     c.use_graphs = true;
@@ -1738,6 +1742,7 @@ int spd_set_tuning(spd_ctx *ctx, const char *key, int32_t value)
     bool found = false;
     for (int i = 0; i < SITE_COUNT; ++i)
         if (!strcmp(key, site_keys[i])) { c.split_override[i] = value; found = true; }
+    if (!strcmp(key, "o_proj_planes")) { c.oproj_planes = value > 2 ? 0 : value; found = true; }
     if (!strcmp(key, "decode_ring_stages")) { c.ring_stages = (value == 0 || (value >= 3 && value <= 5)) ? value : 0; found = true; }
     if (!strcmp(key, "prefill_rescale_log2")) { c.prefill_rescale_log2 = value > 16 ? 16 : value; found = true; }
     if (!strcmp(key, "l2_prefetch_blocks")) { c.l2_prefetch_kb = value > 64 ? 64 : value; found = true; }
