@@ -159,6 +159,10 @@ int spd_set_graphs(spd_ctx *ctx, int32_t enabled);
  *       3, 4 or (16-token tiles) 5; 0 = chosen per launch (four stages; at 16-token tiles five for
  *       launches of at most two thread blocks per SM and three where a launch only then stays
  *       resident at once).
+ *   "o_proj_planes"
+ *       decode o_proj: shard slices one thread block computes one after the other, each into its own accumulator
+ *       columns (1 or 2; 0 = chosen per launch: two where one slice per block would not be resident at once - T * H/128
+ *       blocks against two resident blocks per SM at 32- and 64-token tiles, three at 16).  Same sums in the same order.
  *   "prefill_rescale_log2"
  *       prefill attention on the tensor cores keeps its output accumulator relative to a row
  *       maximum that follows the true running maximum lazily: the accumulator is rescaled only

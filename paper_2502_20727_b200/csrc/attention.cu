@@ -885,9 +885,8 @@ template <typename T, int D, int GT> cudaError_t launch_ring(const AttnArgs &a, 
 // GQA group of 8 query heads per KV head the CUDA-core kernel above is bound by arithmetic
 // (8 x 2 flops per cached element), not by the KV stream.  Here the group's query heads are the
 // rows of an m16n8k16 MMA: S[heads x 16 tokens] = Q K^T and O[heads x 128] += P V per page.
-// Pages arrive through TMA tensor copies (4 boxes of 64 dims x 16 tokens per page: K and V,
-// low and high half of the head dimension) in the 128-byte swizzle that ldmatrix reads without
-// bank conflicts.  Warp roles and split merge: as in the bulk-copy kernel.  The page ring has more slots than
+// Pages arrive through TMA tensor copies (one box per page and tensor: 64 dims x 16 tokens x the two
+// halves of the head dimension) in the 128-byte swizzle that ldmatrix reads without bank conflicts.  Warp roles and split merge: as in the bulk-copy kernel.  The page ring has more slots than
 // compute warps (six or eight for four warps): page i goes to slot i % R and to warp i % 4, so a warp's next page is
 // on its way while it works on the current one - with one slot per warp every page would cost a full memory latency.
 // The warps' partial outputs are merged through the ring's own bytes once every page has been read.
@@ -962,10 +961,8 @@ __global__ void __launch_bounds__(160, DENSE ? 4 : 3) decode_attention_mma_kerne
                 const int row = (sm_bt[i] * a.pt.n_kv_heads + kvh) * BLK; // first of the page's 16 token rows
                 const uint32_t dst = ring + s * SLOT;
                 mbar_expect_tx(full_bar(s), SLOT);
-                tma_load_3d(dst, &tm_k, 0, row, 0, full_bar(s));
-                tma_load_3d(dst + SUB, &tm_k, 64, row, 0, full_bar(s));
+                tma_load_3d(dst, &tm_k, 0, row, 0, full_bar(s));           // both halves of the head dimension: 2 x (16 x 64)
                 tma_load_3d(dst + 2 * SUB, &tm_v, 0, row, 0, full_bar(s));
-                tma_load_3d(dst + 3 * SUB, &tm_v, 64, row, 0, full_bar(s));
             }
         }
         __syncwarp();

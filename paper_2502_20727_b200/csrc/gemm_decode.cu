@@ -326,16 +326,52 @@ __device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const De
     auto sum4 = [](float4 v) { return v.x + v.y + v.z + v.w; };
     if (spd_groups) {
         const int rows = (g.t_rows - t.t_row0 < BN ? g.t_rows - t.t_row0 : BN) - t.rank; // this block's tokens: every P-th of them
-        if (rows > 3 * t.CL) {
+        if (BN < 64 && rows > 3 * t.CL) {
             // Four tokens or more: one token per warp at a time, the devices of a token in turn (one gather of the
-            // partials per token instead of one per warp and token); the per-device row sums are reduced together.
+            // partials per token instead of one per warp and token).
+            for (int q = warp;; q += 4) {
+                const int j = t.rank + t.CL * q, m = t.t_row0 + j;
+                if (j >= BN || m >= g.t_rows) break;
+                const long idx = (long)m * H + n;
+                float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (valid) { x = *(const float4 *)(g.res_in + idx); add4(x, bias); }
+                float4 y[MAX_P];
+                load_partials(y, S, j, lane, t, BN * 128 * 4);
+                float4 tot = make_float4(0.f, 0.f, 0.f, 0.f), yi = make_float4(0.f, 0.f, 0.f, 0.f);
+                int cnt = 0, i = 0;
+#pragma unroll
+                for (int s = 0; s < MAX_P; ++s) {
+                    if (s >= t.P) continue;
+                    add4(yi, y[s]);
+                    if (++cnt < per) continue;
+                    add4(tot, yi);
+                    float4 ri = x;
+                    add4(ri, yi);
+                    if (valid && g.hg) store_bf16x4((bf16 *)g.hg + (long)i * g.hg_stride + idx, ri, gn);
+                    const float sq = warp_sum(valid ? sq4(ri) : 0.f);
+                    if (lane == 0 && g.ss_out) g.ss_out[((long)t.wt * G + i) * g.Mcap + m] = sq;
+                    if (g.sum_out) {
+                        const float sm = warp_sum(valid ? sum4(ri) : 0.f);
+                        if (lane == 0) g.sum_out[((long)t.wt * G + i) * g.Mcap + m] = sm;
+                    }
+                    yi = make_float4(0.f, 0.f, 0.f, 0.f);
+                    cnt = 0;
+                    ++i;
+                }
+                add4(x, tot);
+                if (valid && g.res_out) *(float4 *)(g.res_out + idx) = x;
+            }
+            return;
+        }
+        if (BN >= 64 && rows > 3 * t.CL) {
+            // 64-token tiles: as above, with the per-device row sums reduced together and the residual rows fetched ahead.
             const int mine = my_token_count<BN>(g, t);
             const int dev_of_lane = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
             for (int q = warp, u = 0; q < mine; q += 4, ++u) {
                 const int j = t.rank + t.CL * q, m = t.t_row0 + j;
                 const long idx = (long)m * H + n;
                 float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (valid) { x = u < 4 ? pick4(xpre, u) : *(const float4 *)(g.res_in + idx); add4(x, bias); }
+                if (valid) { x = (BN >= 64 && u < 4) ? pick4(xpre, u) : *(const float4 *)(g.res_in + idx); add4(x, bias); }
                 float4 y[MAX_P];
                 load_partials(y, S, j, lane, t, BN * 128 * 4);
                 float4 tot = make_float4(0.f, 0.f, 0.f, 0.f), yi = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -414,7 +450,7 @@ __device__ __forceinline__ void epilogue_residual(const DecGemmArgs &g, const De
         const int j = t.rank + t.CL * q, m = t.t_row0 + j;
         const long idx = (long)m * H + n;
         float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (valid) { x = u < 4 ? pick4(xpre, u) : *(const float4 *)(g.res_in + idx); add4(x, bias); }
+        if (valid) { x = (BN >= 64 && u < 4) ? pick4(xpre, u) : *(const float4 *)(g.res_in + idx); add4(x, bias); }
         float4 y[MAX_P];
         load_partials(y, S, j, lane, t, BN * 128 * 4);
         float4 tot = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -548,8 +584,10 @@ __device__ __forceinline__ void epilogue_resid_tp(const DecGemmArgs &g, const De
     }
 }
 
+// Resident blocks per SM the register file must allow: four at 16-token tiles (the three-stage ring), three at 32,
+// two at 64 (the ring, not the registers, is the limit there).
 template <int BN, int EPI, int ST>
-__global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_w0,
+__global__ void __launch_bounds__(THREADS, BN == 16 ? 4 : (BN == 32 ? 3 : 2)) gemm_decode_kernel(const __grid_constant__ CUtensorMap tm_w0,
                                                               const __grid_constant__ CUtensorMap tm_w1,
                                                               const __grid_constant__ CUtensorMap tm_w2,
                                                               const __grid_constant__ CUtensorMap tm_t,
@@ -596,7 +634,7 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
     const int az0 = g.w_batched ? t.z : 0, bz0 = g.t_batched ? t.z : 0;
     const uint64_t stream_once = policy_evict_first();
     auto load_w = [&](int s, int it) {
-        const int kx = (kb_begin + it % n_kb) * BK, a_z = az0 + it / n_kb;
+        const int lp = it >= n_kb ? 1 : 0, kx = (kb_begin + it - lp * n_kb) * BK, a_z = az0 + lp; // at most two planes
         const uint32_t sa = base + s * C::STAGE_BYTES;
         if (SUB == 1) tma_load_3d_hint(sa, tm_w, kx, t.w_row0, a_z, full_bar(s), stream_once);
         else {
@@ -604,6 +642,12 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
             if (g.fc1_only) tma_load_3d_hint(sa + ROWS * BK * 2, &tm_w0, kx, t.w_row0 + ROWS, a_z, full_bar(s), stream_once);
             else tma_load_3d_hint(sa + ROWS * BK * 2, &tm_w1, kx, t.w_row0, a_z, full_bar(s), stream_once);
         }
+    };
+    // the same tile requested into L2 only
+    auto prefetch_w = [&](int it) {
+        const int lp = it >= n_kb ? 1 : 0, kx = (kb_begin + it - lp * n_kb) * BK, a_z = az0 + lp; // at most two planes
+        if (SUB == 1) tma_prefetch_l2_3d(tm_w, kx, t.w_row0, a_z);
+        else { tma_prefetch_l2_3d(&tm_w0, kx, t.w_row0, a_z); tma_prefetch_l2_3d(g.fc1_only ? &tm_w0 : &tm_w1, kx, t.w_row0 + (g.fc1_only ? ROWS : 0), a_z); }
     };
     const int pre = n_it < C::STAGES ? n_it : C::STAGES;
     if (warp == 4 && lane == 0) {
@@ -624,13 +668,10 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
             mbar_expect_tx(full_bar(i), C::STAGE_BYTES);
             load_w(i, i);
         }
-        // optionally the K blocks after the ring are pulled into L2
-        const int pf_end = n_kb < pre + g.l2_prefetch_kb ? n_kb : pre + g.l2_prefetch_kb;
-        for (int i = pre; i < pf_end; ++i) {
-            const int kx = (kb_begin + i) * BK, a_z = az0;
-            if (SUB == 1) tma_prefetch_l2_3d(tm_w, kx, t.w_row0, a_z);
-            else { tma_prefetch_l2_3d(&tm_w0, kx, t.w_row0, a_z); tma_prefetch_l2_3d(g.fc1_only ? &tm_w0 : &tm_w1, kx, t.w_row0 + (g.fc1_only ? ROWS : 0), a_z); }
-        }
+        // optionally the K blocks after the ring are pulled into L2 (once: keeping that distance through the loop
+        // was measured 25 % slower at 64-token tiles)
+        const int pf_end = n_it < pre + g.l2_prefetch_kb ? n_it : pre + g.l2_prefetch_kb;
+        for (int i = pre; i < pf_end; ++i) prefetch_w(i);
     }
     if (warp == 5) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(tmem_cols) : "memory");
@@ -652,7 +693,8 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
                     mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
                     load_w(s, i);
                 }
-                tma_load_3d(base + s * C::STAGE_BYTES + C::A_BYTES, &tm_t, (kb_begin + i % n_kb) * BK, t.t_row0, bz0 + i / n_kb, full_bar(s));
+                const int lp = i >= n_kb ? 1 : 0;
+                tma_load_3d(base + s * C::STAGE_BYTES + C::A_BYTES, &tm_t, (kb_begin + i - lp * n_kb) * BK, t.t_row0, bz0 + lp, full_bar(s));
             }
         }
         __syncwarp();
@@ -665,8 +707,8 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t sa = base + s * C::STAGE_BYTES, sb = sa + C::A_BYTES;
                 const uint64_t da = make_desc(sa), db = make_desc(sb);
-                const int kk = i % n_kb;
-                const uint32_t acc = tmem_acc + (uint32_t)((i / n_kb) * BN); // plane i / n_kb: its own accumulator columns
+                const int lp = i >= n_kb ? 1 : 0, kk = i - lp * n_kb;
+                const uint32_t acc = tmem_acc + (uint32_t)(lp * BN); // each plane has its own accumulator columns
 #pragma unroll
                 for (int k = 0; k < BK / UMMA_K; ++k)
                     umma(acc, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
@@ -701,7 +743,7 @@ __global__ void __launch_bounds__(THREADS) gemm_decode_kernel(const __grid_const
             }
             sm_kvoff[threadIdx.x] = off;
         }
-        if (EPI == EPI_OPROJ || EPI == EPI_DOWN) {
+        if (BN >= 64 && (EPI == EPI_OPROJ || EPI == EPI_DOWN)) {
             // the residual rows this warp will finish first (tokens rank + CL * (warp + 4u)): requested while the weights stream
             const int n = t.w_row0 + 4 * lane, mine = my_token_count<BN>(g, t);
 #pragma unroll

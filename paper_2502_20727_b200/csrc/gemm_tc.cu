@@ -228,6 +228,24 @@ int make_operand_map(TcMap *out, const void *ptr, long k_inner, long rows, long 
     return r == CUDA_SUCCESS ? 0 : -3;
 }
 
+// A paged K or V cache ([pages][kv heads][16 tokens][128 dims] bf16, `rows` token rows in all) as a 3-D map {64 dims,
+// rows, 2 halves of the head dimension} with a {64, 16, 2} box: one copy brings a (page, head)'s 4 KB in as two
+// 16 x 64 tiles in the 128-byte swizzle, low half of the head dimension first.
+int make_page_map(TcMap *out, const void *ptr, long rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return -1;
+    if ((uintptr_t)ptr & 15) return -2;
+    cuuint64_t dims[3] = {64, (cuuint64_t)rows, 2};
+    cuuint64_t strides[2] = {256, 128};
+    cuuint32_t box[3] = {64, 16, 2};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn((CUtensorMap *)out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? 0 : -3;
+}
+
 int tc_token_box(bool swap, int tokens)
 {
     if (!swap) return BM;

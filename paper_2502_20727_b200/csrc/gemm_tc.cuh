@@ -31,6 +31,8 @@ struct TcGemmArgs {
 // Returns 0, or <0 when the driver entry point is missing / alignment is violated / encode fails.
 int make_operand_map(TcMap *out, const void *ptr, long k_inner, long rows, long batches, long ld_elems,
                      long batch_stride_elems, int box_rows);
+// A paged K / V cache (16-token pages, head_dim 128) as a map whose {64, 16, 2} box is one (page, head): see gemm_tc.cu.
+int make_page_map(TcMap *out, const void *ptr, long rows);
 
 // Box rows of the token-side operand for a given token count (swap: 16/32/64, else 128).
 int tc_token_box(bool swap, int tokens);

@@ -67,7 +67,7 @@ enum Site { SITE_QKV = 0, SITE_O, SITE_GU, SITE_DOWN, SITE_ATTN, SITE_COUNT };
 const char *const kind_names[K_COUNT] = {"residual_rmsnorm", "gemm_qkv", "rope_kv_append", "attention", "gemm_o_proj",
                                          "gemm_gate_up", "silu_mul", "gemm_down", "rope_table"};
 
-struct LayerMaps { TcMap wq, wk, wv, wo_full, wo_shard, wo_shard64, w_gate, w_up, w_down, w_gate64, w_up64, wq256, wk256, wv256, wo256, wd256, wd_shard, kpages, vpages; };
+struct LayerMaps { TcMap wq, wk, wv, wo_full, wo_shard, wo_shard64, w_gate, w_up, w_down, w_gate64, w_up64, wq256, wk256, wv256, wo256, wd256, wd_shard, kpages, vpages, kpage_whole, vpage_whole; };
 
 // A captured decode step is valid for exactly these arguments.
 struct GraphKey {
@@ -833,7 +833,7 @@ int run_decode_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const i
             a.q = c->q; a.k_pages = w.k_pages; a.v_pages = w.v_pages; a.pt = pt; a.tm = tm; a.out = c->attn;
             a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.B = M; a.splits = p.attn_splits;
             a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.counters = c->attn_cnt; a.err = c->err;
-            if (d.head_dim == 128 && d.kv_block_size == 16) { a.k_map = &c->maps[l].kpages; a.v_map = &c->maps[l].vpages; }
+            if (d.head_dim == 128 && d.kv_block_size == 16) { a.k_map = &c->maps[l].kpage_whole; a.v_map = &c->maps[l].vpage_whole; }
             LAUNCH_S(K_ATTN, a, launch_decode_attention<bf16>(a, st));
         }
         {   // a5 - a7: shard i's K slice gives the plane group Y_i
@@ -956,7 +956,7 @@ int run_tp(Ctx *c, const void *x, void *out, long out_stride, int M, TokMap tm, 
             a.q = c->q; a.k_pages = w.k_pages; a.v_pages = w.v_pages; a.pt = pt; a.tm = tm; a.out = c->attn;
             a.M = M; a.n_q_heads = d.n_q_heads; a.head_dim = d.head_dim; a.B = M; a.splits = p.attn_splits;
             a.max_context = max_context; a.part_o = c->part_o; a.part_ml = c->part_ml; a.counters = c->attn_cnt; a.err = c->err;
-            if (d.head_dim == 128 && d.kv_block_size == 16) { a.k_map = &c->maps[l].kpages; a.v_map = &c->maps[l].vpages; }
+            if (d.head_dim == 128 && d.kv_block_size == 16) { a.k_map = &c->maps[l].kpage_whole; a.v_map = &c->maps[l].vpage_whole; }
             LAUNCH_S(K_ATTN, a, launch_decode_attention<bf16>(a, st));
         }
         {   // a5 - a7: Y_z from the rank's own heads.  TP block: R = X + sum over ranks (sync-point 1);
@@ -1360,6 +1360,8 @@ int build_weight_maps(Ctx &c)
             const long rows = (long)c.n_pages * d.n_kv_heads * 16;
             rc |= make_operand_map(&m.kpages, w.k_pages, 128, rows, 1, 128, 0, 16);
             rc |= make_operand_map(&m.vpages, w.v_pages, 128, rows, 1, 128, 0, 16);
+            rc |= make_page_map(&m.kpage_whole, w.k_pages, rows); // decode attention: one copy per (page, head)
+            rc |= make_page_map(&m.vpage_whole, w.v_pages, rows);
         }
         rc |= make_operand_map(&m.w_gate64, w.w_gate, H, F / T, T, H, (F / T) * H, 64);
         if (d.block_kind == 0) rc |= make_operand_map(&m.w_up64, w.w_up, H, F / T, T, H, (F / T) * H, 64);
