@@ -615,7 +615,7 @@ def run_native(args, rank, world):
                             run.close()
                             run = None
                         r2 = Run(si.WORKLOADS[name], dev, plan["seed"], K, W, args, spd)
-                    entry = measure_config(r2, list(masks_of(r2.w)), clk, barrier, peaks, max(1, min(args.prefill_reps, 2)))
+                    entry = measure_config(r2, list(masks_of(r2.w)), clk, barrier, peaks, max(1, args.prefill_reps))
                     entry["workload"] = describe(r2.w, r2)
                     per_config[name] = entry
                 except Exception as e:  # one configuration failing must not lose the line
