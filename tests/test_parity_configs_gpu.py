@@ -106,6 +106,26 @@ def test_c5_decode_tiles_of_64_at_70b_widths():
     decode_on_synthetic_cache(w, (1, 0), lens, 2, label="c5 B=64")
 
 
+@pytest.mark.parametrize("B", [24, 64])
+def test_two_shard_slices_per_block_is_only_a_schedule(B):
+    """Decode o_proj at the 70B widths: with 32- and 64-token tiles a thread block takes two shard slices one after the
+    other (one wave of blocks instead of two).  Same partial sums added in the same order: bit-identical to one slice
+    per block, on a TP and an SPD block, at a ragged batch of 24 (32-token tile) and a full 64-token tile."""
+    w = si.WORKLOADS["c5"].with_(n_layers=2, mask=(1, 0))
+    lens = (1 + (np.arange(B) * 37) % 90).astype(np.int32)
+    outs = []
+    for planes in (2, 1):
+        p = Pair(w, mask=(1, 0), B=B, max_len=int(lens.max()) + 2, max_prefill_tokens=B, weights_on=DEV, stream_oracle=True)
+        p.stack.set_tuning(o_proj_planes=planes)
+        p.fill_cache(lens)
+        got, ref = p.decode(0)
+        assert rel_err(got, ref) <= stack_tol(w.dtype, 2)
+        assert p.stack.device_error() == 0
+        outs.append(got)
+        p.stack.close()
+    assert np.array_equal(outs[0], outs[1])
+
+
 C5_SMALL = dict(hidden=1024, n_q_heads=32, n_kv_heads=8, ffn=3584)
 
 
