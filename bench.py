@@ -507,7 +507,8 @@ def run_native(args, rank, world):
     with ClockSampler(dev.index or 0) as clk:
         run = Run(w, dev, plan["seed"], K, W, args, spd)
         B = run.Bd
-        fused = w.block == "llama" and not args.rank_mode
+        # bf16 stacks of either block kind run the five fused kernels per block, whose launches carry stamps
+        fused = w.dtype == "bf16" and not args.rank_mode and "bias_fused=0" not in (args.tune or "")
         run.stack.set_mask(mask)
         pre_ms = run.prefill_ms(args.prefill_reps) if args.prefill_reps > 0 else None
         run.fill_cache()

@@ -137,21 +137,27 @@ __device__ __forceinline__ void compute_rstd(const SumSq &ss, int group, int t_r
             acc += __ldcg(ss.part + i);
             if (ss.sum) sum += __ldcg(ss.sum + i);
         }
+    // (the row sums of LayerNorm go through the same 128 words in a second round: static shared memory decides whether
+    // a third block of 16-token tiles fits an SM)
+    float mu = 0.f;
+    if (ss.sum) {
+        red[t] = sum;
+        epi_sync();
+        if (t < BN) {
+#pragma unroll
+            for (int q = 0; q < PARTS; ++q) mu += red[q * BN + t];
+            mu /= (float)ss.H;
+        }
+        epi_sync();
+    }
     red[t] = acc;
-    if (ss.sum) red[128 + t] = sum;
     epi_sync();
     if (t < BN) {
-        float tot = 0.f, mu = 0.f;
+        float tot = 0.f;
 #pragma unroll
         for (int q = 0; q < PARTS; ++q) tot += red[q * BN + t];
-        if (ss.sum) {   // LayerNorm: variance about the mean
-#pragma unroll
-            for (int q = 0; q < PARTS; ++q) mu += red[128 + q * BN + t];
-            mu /= (float)ss.H;
-            sm_rstd[t] = rsqrtf(fmaxf(tot / (float)ss.H - mu * mu, 0.f) + ss.eps);
-        } else {
-            sm_rstd[t] = rsqrtf(tot / (float)ss.H + ss.eps);
-        }
+        // LayerNorm: variance about the mean
+        sm_rstd[t] = ss.sum ? rsqrtf(fmaxf(tot / (float)ss.H - mu * mu, 0.f) + ss.eps) : rsqrtf(tot / (float)ss.H + ss.eps);
         sm_mu[t] = mu;
     }
 }
@@ -598,7 +604,7 @@ __global__ void __launch_bounds__(THREADS, BN == 16 ? 4 : (BN == 32 ? 3 : 2)) ge
     constexpr int ROWS = BM / SUB;                   // weight rows per box
     const DecGemmArgs &g = L.g;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ float sm_red[256];
+    __shared__ float sm_red[128];
     __shared__ float sm_rstd[64], sm_mu[64];
     __shared__ long sm_kvoff[64];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
