@@ -49,7 +49,8 @@ template <int BN, int ST> struct DCfg {
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int STAGES = ST;
     static constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 128 /*barriers, slot, flag*/;
+    static_assert(8 * (2 * STAGES + 1) + 8 <= 128, "barrier area");
     static_assert(STAGES * STAGE_BYTES >= 2 * BN * 128 * 4, "ring too small for the staging tiles");
 };
 
@@ -152,10 +153,13 @@ __device__ __forceinline__ void compute_rstd(const SumSq &ss, int group, int t_r
     }
     red[t] = acc;
     epi_sync();
+    float tot = 0.f;
     if (t < BN) {
-        float tot = 0.f;
 #pragma unroll
         for (int q = 0; q < PARTS; ++q) tot += red[q * BN + t];
+    }
+    epi_sync(); // sm_rstd and sm_mu are the two halves of `red`: every partial has been read before they are written
+    if (t < BN) {
         // LayerNorm: variance about the mean
         sm_rstd[t] = ss.sum ? rsqrtf(fmaxf(tot / (float)ss.H - mu * mu, 0.f) + ss.eps) : rsqrtf(tot / (float)ss.H + ss.eps);
         sm_mu[t] = mu;
@@ -604,8 +608,10 @@ __global__ void __launch_bounds__(THREADS, BN == 16 ? 4 : (BN == 32 ? 3 : 2)) ge
     constexpr int ROWS = BM / SUB;                   // weight rows per box
     const DecGemmArgs &g = L.g;
     extern __shared__ uint8_t smem_raw[];
+    // Static shared memory counts: at 16-token tiles with a three-stage ring a fourth block fits an SM only while ring +
+    // barriers + this stay under 57 KB.  The reduction scratch of the row statistics becomes their home afterwards.
     __shared__ float sm_red[128];
-    __shared__ float sm_rstd[64], sm_mu[64];
+    float *const sm_rstd = sm_red, *const sm_mu = sm_red + 64;
     __shared__ long sm_kvoff[64];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
