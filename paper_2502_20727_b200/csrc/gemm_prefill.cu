@@ -39,12 +39,11 @@ template <int EPI, int PAIR> struct PCfg {
     static_assert(EPI != PRE_SCATTER || PAIR, "the scatter epilogue is only built for CTA pairs");
     static constexpr int A_BYTES = BM * BK * 2, B_BYTES = (BN / (PAIR ? 2 : 1)) * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int X_BYTES = 0, H_BYTES = 0;
     // the ring takes all the shared memory a block may have: the loaded latency of a tile load is about 1.6 us, so
     // what the tensor cores can be fed per SM is (bytes in flight) / 1.6 us
-    static constexpr int STAGES = (216 * 1024 - X_BYTES - H_BYTES) / STAGE_BYTES;
+    static constexpr int STAGES = (216 * 1024) / STAGE_BYTES;
     static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
-    static constexpr int SMEM_BYTES = RING_BYTES + X_BYTES + H_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int SMEM_BYTES = RING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
     // Epilogue warps: 0-3 (one per accumulator lane quarter); PRE_OPROJ_SPD, whose tail is T times the work per MMA
     // of the others, adds warps 6-9: two threads per row, 64 of the tile's 128 columns each.
     static constexpr int EPI_WARPS = (EPI == PRE_OPROJ_SPD) ? 8 : 4;
@@ -486,9 +485,6 @@ __global__ void __launch_bounds__(PCfg<EPI, PAIR>::THREADS_, 1) gemm_prefill_ker
                                                                   const __grid_constant__ CUtensorMap tm_w1,
                                                                   const __grid_constant__ CUtensorMap tm_w2,
                                                                   const __grid_constant__ CUtensorMap tm_t,
-                                                                  const __grid_constant__ CUtensorMap tm_x,
-                                                                  const __grid_constant__ CUtensorMap tm_r,
-                                                                  const __grid_constant__ CUtensorMap tm_h,
                                                                   const __grid_constant__ PreLaunch L)
 {
     using C = PCfg<EPI, PAIR>;
@@ -501,9 +497,8 @@ __global__ void __launch_bounds__(PCfg<EPI, PAIR>::THREADS_, 1) gemm_prefill_ker
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t bars = base + C::RING_BYTES + C::X_BYTES + C::H_BYTES; // full[S], empty[S], tmem_full[2], tmem_empty[2], x_full
-    uint32_t *tmem_slot = (uint32_t *)(gen_base + C::RING_BYTES + C::X_BYTES + C::H_BYTES + 8 * (2 * S + 5));
-    const uint32_t xfull_bar = bars + 8u * (2 * S + 4);
+    const uint32_t bars = base + C::RING_BYTES; // full[S], empty[S], tmem_full[2], tmem_empty[2]
+    uint32_t *tmem_slot = (uint32_t *)(gen_base + C::RING_BYTES + 8 * (2 * S + 4));
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (S + s); };
@@ -519,7 +514,6 @@ __global__ void __launch_bounds__(PCfg<EPI, PAIR>::THREADS_, 1) gemm_prefill_ker
         for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         // an accumulator is free again when the epilogue warps of both CTAs of a pair have drained their rows
         for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), C::EPI_WARPS * (PAIR ? 2 : 1)); }
-        mbar_init(xfull_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -697,8 +691,6 @@ __global__ void __launch_bounds__(PCfg<EPI, PAIR>::THREADS_, 1) gemm_prefill_ker
 template <int EPI, int PAIR>
 cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, const PreLaunch &L, cudaStream_t st)
 {
-    const CUtensorMap &tx = tt, &tr = tt; // spare tensor-map slots
-    const CUtensorMap &th = tt;
     using C = PCfg<EPI, PAIR>;
     static bool attr_done = false;
     if (!attr_done) {
@@ -710,10 +702,10 @@ cudaError_t launch_epi(const CUtensorMap *const *tw, const CUtensorMap &tt, cons
     const int total = L.m_tiles * L.n_tiles;
     if (PAIR) { // one pair per two SMs, persistent over the 256-token tiles
         const int pairs = total < n_sm / 2 ? total : n_sm / 2;
-        return launch_kernel(gemm_prefill_kernel<EPI, PAIR>, dim3(2 * pairs), dim3(C::THREADS_), C::SMEM_BYTES, st, 2, *tw[0], *tw[1], *tw[2], tt, tx, tr, th, L);
+        return launch_kernel(gemm_prefill_kernel<EPI, PAIR>, dim3(2 * pairs), dim3(C::THREADS_), C::SMEM_BYTES, st, 2, *tw[0], *tw[1], *tw[2], tt, L);
     }
     const dim3 grid(total < n_sm ? total : n_sm);
-    return launch_kernel(gemm_prefill_kernel<EPI, PAIR>, grid, dim3(C::THREADS_), C::SMEM_BYTES, st, 0, *tw[0], *tw[1], *tw[2], tt, tx, tr, th, L);
+    return launch_kernel(gemm_prefill_kernel<EPI, PAIR>, grid, dim3(C::THREADS_), C::SMEM_BYTES, st, 0, *tw[0], *tw[1], *tw[2], tt, L);
 }
 
 // One thread block per token: whole-row sum of squares in one partial.

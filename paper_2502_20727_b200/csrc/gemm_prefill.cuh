@@ -68,9 +68,6 @@ struct PreGemmArgs {
     // GATEUP
     void *act;           // bf16 [tokens][F]
     int F, Fs;
-    // OPROJ_SPD: the R_i * g planes leave through shared memory and TMA stores: host pointer to the tensor map of
-    // hg as bf16 [groups][Mcap][H] with a 64 x 128 box
-    const void *h_map;
     // Head grouping (Sec. 4.2.4, MLP matching): GATEUP with w_rot = r applies MLP partition (z + r) % T to the
     // input of device z (output in the partition's column block); OPROJ_SPD with norm_only != 0 only writes, per
     // K slice and token, the sum of squares of the slice's output to ss_out (no residual, no operand planes).

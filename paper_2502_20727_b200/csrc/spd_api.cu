@@ -1244,8 +1244,6 @@ int run_prefill_fused(Ctx *c, const void *x, void *out, int M, TokMap tm, const 
             MAP_OR_FAIL(am, act_map(c, AB_ATTN_SHARD, 128));
             g.w_rows[0] = H; g.num_kb = cdiv(qd / Tn, 64); g.batches = Tn;
             g.res_in = c->res[0]; g.res_out = c->res[1]; g.gain = w.mlp_norm; g.hg = c->h; g.hg_stride = Mc * H; g.ss_out = c->ss_mlp;
-            MAP_OR_FAIL(hm, act_map(c, AB_H, 128));
-            g.h_map = hm;
             if (opt) { g.bias = w.bo; g.sum_out = c->sm_mlp; } // Y_i = P_i + b: b once in the carried sum, and in every device's MLP input
             LAUNCH_S(K_OPROJ, g, launch_gemm_prefill(PRE_OPROJ_SPD, wmaps, *am, g, st));
             mlp_tiles = pre_ss_tiles(PRE_OPROJ_SPD, H); mlp_groups = Tn;
